@@ -1,0 +1,579 @@
+/*
+ * WnW decode-step ORACLE -- TEST INFRASTRUCTURE, NOT A PRODUCT PATH.
+ *
+ * A plain, slow CPU restatement of the decode-time hot path of the
+ * Waxing-and-Waning KV cache (Method section: "Method Overview", "Prefill
+ * Compression", "Decode-Step Score Aggregation" (Eq. 2), "Dynamic Chunk
+ * Selection"), in the chunk-granular, hard-budget, per-layer form this
+ * repository builds.  Only tests, the smoke check and the benchmark's CPU
+ * baseline leg may call it.  It shares no code with the CUDA library.
+ *
+ * How it differs in structure from the CUDA path, on purpose:
+ *   - it keeps the FULL, never-moved K and V of every head (also what fixed
+ *     heads discard and what tidal heads offload); there is no slot pool, no
+ *     host mirror and no copy;
+ *   - residency is a table of chunk ids; attention is a masked softmax over the
+ *     full key set, accumulated in double precision;
+ *   - every table update of a step happens in wnwo_step_end, after all layers
+ *     (the paper's order: "after attention is computed for all L layers").
+ *
+ * Pins (tests/, CPU only): softmax rows sum to one; budget 1.0 equals a dense
+ * softmax attention written separately with numpy; chunk scores sum to the
+ * anchor heads' audio attention mass; closed forms for identical keys and for a
+ * one-hot key; top-k against brute force; the table update against an
+ * independent set model and a hand-worked trace.  The numeric trajectory on
+ * seeded inputs has no printed example in the paper: beyond those invariants
+ * it is "parity unpinned".
+ *
+ * Conventions (all chosen readings are listed in the design document):
+ *   - inputs are bf16 bit patterns (uint16); all arithmetic is double;
+ *   - softmax runs over the head's whole allowed key set, text and audio
+ *     (Eq. 2 takes the audio entries of that softmax);
+ *   - score_sum[c] = sum over the layer's anchor q-heads and over tau in chunk
+ *     c of the softmax weight; the ranking key is the chunk MEAN,
+ *     (float)score_sum[c] / (float)len_c, compared as float, ties to the lower
+ *     chunk index;
+ *   - a layer without anchor heads ranks by the scores of the nearest layer
+ *     that has one (ties to the lower layer);
+ *   - a selection made at step s is used by tidal attention at step s+1;
+ *   - slots S = max(1, floor((double)budget * C + 1e-6)), capped at C;
+ *   - stamps: a chunk selected with rank r at step s gets s*topk + (topk-1-r);
+ *     prefill gives rank r the stamp -1-r.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define WNWO_OK 0
+#define WNWO_ERR_ARG 1
+#define WNWO_ERR_STATE 2
+#define WNWO_ERR_OOM 3
+
+#define ROLE_ANCHOR 0
+#define ROLE_TIDAL 1
+#define ROLE_FIXED 2
+
+typedef struct {
+  int placed_layers;   /* how many layers have been placed */
+  int T_a, T_t, T_cap; /* audio tokens, current text tokens, text capacity */
+  int C, S;            /* chunks, slots */
+  long long steps;     /* decode steps this sequence took part in */
+  uint16_t **audK, **audV; /* [L] -> [Hkv][T_a][d]   full audio K,V of every head */
+  uint16_t **txtK, **txtV; /* [L] -> [Hkv][T_cap][d] */
+  int *slot_chunk;         /* [L][S]  -1 = free */
+  long long *stamp;        /* [L][S] */
+  int *fixed_set;          /* [L][Hkv][S] */
+  int *fixed_n;            /* [L][Hkv] */
+  double *score_sum;       /* [L][C]  this step's scores (anchor layers) */
+  double *pre;             /* [L][Hkv][C] prefill scores */
+  int *sel;                /* [L][topk] */
+  int *n_sel;              /* [L] */
+  long long hits, misses, evictions;
+} Seq;
+
+typedef struct {
+  int L, Hq, Hkv, d, g, chunk, topk, max_batch, max_audio, max_text;
+  double budget, scale;
+  uint8_t *roles; /* [L][Hkv] */
+  int *src;       /* [L] score source layer, -1 if the layer has no tidal heads or no source */
+  Seq *seq;
+  int *active;
+  int n_active;
+  int in_step, next_layer, appended;
+} Oracle;
+
+static double bf16_to_double(uint16_t b) {
+  uint32_t u = (uint32_t)b << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+static int layer_has(const Oracle *o, int l, int role) {
+  for (int h = 0; h < o->Hkv; ++h)
+    if (o->roles[l * o->Hkv + h] == role) return 1;
+  return 0;
+}
+
+static int chunk_len(const Oracle *o, const Seq *s, int c) {
+  int lo = c * o->chunk, hi = lo + o->chunk;
+  if (hi > s->T_a) hi = s->T_a;
+  return hi - lo;
+}
+
+/* ------------------------------------------------------------------ */
+/* Pure pieces, exported so tests can drive them on arbitrary arrays.   */
+/* ------------------------------------------------------------------ */
+
+/* Dynamic Chunk Selection: rank chunks by mean score, (key desc, index asc).
+ * score_sum as float; lens = tokens per chunk.  Writes the first k ranks. */
+int wnwo_topk(const float *score_sum, const int *lens, int C, int k, int *sel_out) {
+  if (k > C) k = C;
+  unsigned char *taken = (unsigned char *)calloc((size_t)(C > 0 ? C : 1), 1);
+  if (!taken) return -1;
+  for (int r = 0; r < k; ++r) {
+    int best = -1;
+    float best_key = 0.f;
+    for (int c = 0; c < C; ++c) {
+      if (taken[c]) continue;
+      float key = score_sum[c] / (float)lens[c];
+      if (best < 0 || key > best_key) { /* strict > keeps the lower index on ties */
+        best = c;
+        best_key = key;
+      }
+    }
+    taken[best] = 1;
+    sel_out[r] = best;
+  }
+  free(taken);
+  return k;
+}
+
+/* Chunk swap under a fixed slot pool.  sel in rank order.  Updates the table in
+ * place; plan_chunk/plan_slot receive the misses (chunks to recall and where),
+ * evicted[] the chunk that was displaced or -1.  Returns the number of misses. */
+int wnwo_table_update(int *slot_chunk, long long *stamp, int S, const int *sel, int k, long long step, int topk,
+                      int *plan_chunk, int *plan_slot, int *evicted, int *n_hits) {
+  int n_plan = 0, hits = 0;
+  for (int r = 0; r < k; ++r) {
+    int c = sel[r];
+    long long st = step * (long long)topk + (long long)(topk - 1 - r);
+    int j = -1;
+    for (int i = 0; i < S; ++i)
+      if (slot_chunk[i] == c) j = i;
+    if (j >= 0) { /* hit: refresh recency */
+      stamp[j] = st;
+      ++hits;
+      continue;
+    }
+    for (int i = 0; i < S && j < 0; ++i)
+      if (slot_chunk[i] < 0) j = i; /* lowest-index free slot */
+    int victim = -1;
+    if (j < 0) { /* least recently selected resident that is not selected now */
+      for (int i = 0; i < S; ++i) {
+        int in_sel = 0;
+        for (int q = 0; q < k; ++q)
+          if (sel[q] == slot_chunk[i]) in_sel = 1;
+        if (in_sel) continue;
+        if (j < 0 || stamp[i] < stamp[j]) j = i;
+      }
+      if (j < 0) return -1; /* cannot happen when S >= k */
+      victim = slot_chunk[j];
+    }
+    slot_chunk[j] = c;
+    stamp[j] = st;
+    plan_chunk[n_plan] = c;
+    plan_slot[n_plan] = j;
+    evicted[n_plan] = victim;
+    ++n_plan;
+  }
+  if (n_hits) *n_hits = hits;
+  return n_plan;
+}
+
+/* ------------------------------------------------------------------ */
+/* Life cycle                                                           */
+/* ------------------------------------------------------------------ */
+
+static void free_seq(Oracle *o, Seq *s) {
+  if (s->audK)
+    for (int l = 0; l < o->L; ++l) { free(s->audK[l]); free(s->audV[l]); free(s->txtK[l]); free(s->txtV[l]); }
+  free(s->audK); free(s->audV); free(s->txtK); free(s->txtV);
+  free(s->slot_chunk); free(s->stamp); free(s->fixed_set); free(s->fixed_n);
+  free(s->score_sum); free(s->pre); free(s->sel); free(s->n_sel);
+  memset(s, 0, sizeof(*s));
+}
+
+void wnwo_destroy(Oracle *o) {
+  if (!o) return;
+  if (o->seq)
+    for (int b = 0; b < o->max_batch; ++b) free_seq(o, &o->seq[b]);
+  free(o->seq); free(o->roles); free(o->src); free(o->active);
+  free(o);
+}
+
+int wnwo_create(int L, int Hq, int Hkv, int d, int max_batch, int max_audio, int max_text, int chunk, int topk,
+                double budget, double scale, const uint8_t *roles, Oracle **out) {
+  if (!out || !roles || L < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv || d < 1 || max_batch < 1 || chunk < 1 || topk < 1)
+    return WNWO_ERR_ARG;
+  if (!(budget > 0.0 && budget <= 1.0)) return WNWO_ERR_ARG;
+  Oracle *o = (Oracle *)calloc(1, sizeof(Oracle));
+  if (!o) return WNWO_ERR_OOM;
+  o->L = L; o->Hq = Hq; o->Hkv = Hkv; o->d = d; o->g = Hq / Hkv; o->chunk = chunk; o->topk = topk;
+  o->max_batch = max_batch; o->max_audio = max_audio; o->max_text = max_text;
+  o->budget = budget;
+  o->scale = scale > 0.0 ? scale : 1.0 / sqrt((double)d); /* Eq. 2: q K^T / sqrt(d) */
+  o->roles = (uint8_t *)malloc((size_t)L * Hkv);
+  o->src = (int *)malloc(sizeof(int) * L);
+  o->seq = (Seq *)calloc((size_t)max_batch, sizeof(Seq));
+  o->active = (int *)calloc((size_t)max_batch, sizeof(int));
+  if (!o->roles || !o->src || !o->seq || !o->active) { wnwo_destroy(o); return WNWO_ERR_OOM; }
+  memcpy(o->roles, roles, (size_t)L * Hkv);
+  int any_anchor = 0, any_tidal = 0;
+  for (int i = 0; i < L * Hkv; ++i) {
+    if (roles[i] > ROLE_FIXED) { wnwo_destroy(o); return WNWO_ERR_ARG; }
+    any_anchor |= roles[i] == ROLE_ANCHOR;
+    any_tidal |= roles[i] == ROLE_TIDAL;
+  }
+  if (any_tidal && !any_anchor) { wnwo_destroy(o); return WNWO_ERR_ARG; }
+  /* score routing: own layer if it has an anchor, else the nearest anchor layer, ties to the lower one */
+  for (int l = 0; l < L; ++l) {
+    o->src[l] = -1;
+    if (!layer_has(o, l, ROLE_TIDAL)) continue;
+    int best = -1;
+    for (int a = 0; a < L; ++a) {
+      if (!layer_has(o, a, ROLE_ANCHOR)) continue;
+      if (best < 0 || abs(a - l) < abs(best - l)) best = a; /* ascending a: the lower layer wins a tie */
+    }
+    o->src[l] = best;
+  }
+  *out = o;
+  return WNWO_OK;
+}
+
+int wnwo_score_source(const Oracle *o, int layer) { return (layer >= 0 && layer < o->L) ? o->src[layer] : -2; }
+
+static int alloc_seq(Oracle *o, Seq *s, int T_a, int T_t) {
+  int L = o->L, Hkv = o->Hkv, d = o->d;
+  s->T_a = T_a; s->T_t = T_t; s->T_cap = o->max_text;
+  s->C = (T_a + o->chunk - 1) / o->chunk;
+  int S = (int)floor(o->budget * (double)s->C + 1e-6);
+  if (S < 1) S = 1;
+  if (S > s->C) S = s->C;
+  s->S = S;
+  size_t nS = (size_t)(S > 0 ? S : 1), nC = (size_t)(s->C > 0 ? s->C : 1);
+  s->audK = (uint16_t **)calloc((size_t)L, sizeof(void *)); s->audV = (uint16_t **)calloc((size_t)L, sizeof(void *));
+  s->txtK = (uint16_t **)calloc((size_t)L, sizeof(void *)); s->txtV = (uint16_t **)calloc((size_t)L, sizeof(void *));
+  s->slot_chunk = (int *)malloc(sizeof(int) * L * nS);
+  s->stamp = (long long *)calloc((size_t)L * nS, sizeof(long long));
+  s->fixed_set = (int *)malloc(sizeof(int) * L * Hkv * nS);
+  s->fixed_n = (int *)calloc((size_t)L * Hkv, sizeof(int));
+  s->score_sum = (double *)calloc((size_t)L * nC, sizeof(double));
+  s->pre = (double *)calloc((size_t)L * Hkv * nC, sizeof(double));
+  s->sel = (int *)malloc(sizeof(int) * L * o->topk);
+  s->n_sel = (int *)calloc((size_t)L, sizeof(int));
+  if (!s->audK || !s->audV || !s->txtK || !s->txtV || !s->slot_chunk || !s->stamp || !s->fixed_set || !s->fixed_n ||
+      !s->score_sum || !s->pre || !s->sel || !s->n_sel)
+    return WNWO_ERR_OOM;
+  for (size_t i = 0; i < (size_t)L * nS; ++i) s->slot_chunk[i] = -1;
+  for (size_t i = 0; i < (size_t)L * Hkv * nS; ++i) s->fixed_set[i] = -1;
+  for (int i = 0; i < L * o->topk; ++i) s->sel[i] = -1;
+  for (int l = 0; l < L; ++l) {
+    size_t na = (size_t)Hkv * (size_t)(T_a > 0 ? T_a : 1) * d, nt = (size_t)Hkv * (size_t)(s->T_cap > 0 ? s->T_cap : 1) * d;
+    s->audK[l] = (uint16_t *)calloc(na, 2); s->audV[l] = (uint16_t *)calloc(na, 2);
+    s->txtK[l] = (uint16_t *)calloc(nt, 2); s->txtV[l] = (uint16_t *)calloc(nt, 2);
+    if (!s->audK[l] || !s->audV[l] || !s->txtK[l] || !s->txtV[l]) return WNWO_ERR_OOM;
+  }
+  return WNWO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Attention of one query head over an allowed key set                  */
+/* ------------------------------------------------------------------ */
+
+/* allowed[c] != 0: chunk c's audio positions are visible.  All T_t text positions
+ * always are.  Writes out[d]; if chunk_mass != NULL adds the softmax weight of
+ * every audio position into chunk_mass[chunk of tau]; if p_row != NULL writes
+ * the whole probability row [T_t + T_a] (text first), zeros where masked. */
+static void attend(const Oracle *o, const Seq *s, int layer, int kvh, const uint16_t *q, int T_t,
+                   const unsigned char *allowed, double *out, double *chunk_mass, double *p_row) {
+  const int d = o->d, T_a = s->T_a;
+  const uint16_t *tK = s->txtK[layer] + (size_t)kvh * s->T_cap * d, *tV = s->txtV[layer] + (size_t)kvh * s->T_cap * d;
+  const uint16_t *aK = s->audK[layer] + (size_t)kvh * T_a * d, *aV = s->audV[layer] + (size_t)kvh * T_a * d;
+  const int n = T_t + T_a;
+  double *logit = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+  double mx = -INFINITY;
+  for (int i = 0; i < n; ++i) {
+    const uint16_t *krow;
+    int vis;
+    if (i < T_t) { krow = tK + (size_t)i * d; vis = 1; }
+    else { int tau = i - T_t; krow = aK + (size_t)tau * d; vis = allowed[tau / o->chunk] != 0; }
+    if (!vis) { logit[i] = -INFINITY; continue; }
+    double acc = 0.0;
+    for (int x = 0; x < d; ++x) acc += bf16_to_double(q[x]) * bf16_to_double(krow[x]);
+    logit[i] = acc * o->scale;
+    if (logit[i] > mx) mx = logit[i];
+  }
+  for (int x = 0; x < d; ++x) out[x] = 0.0;
+  if (p_row) for (int i = 0; i < n; ++i) p_row[i] = 0.0;
+  if (mx == -INFINITY) { free(logit); return; } /* empty key set: zero output */
+  double Z = 0.0;
+  for (int i = 0; i < n; ++i)
+    if (logit[i] != -INFINITY) Z += exp(logit[i] - mx);
+  for (int i = 0; i < n; ++i) {
+    if (logit[i] == -INFINITY) continue;
+    double p = exp(logit[i] - mx) / Z;
+    const uint16_t *vrow = (i < T_t) ? tV + (size_t)i * d : aV + (size_t)(i - T_t) * d;
+    for (int x = 0; x < d; ++x) out[x] += p * bf16_to_double(vrow[x]);
+    if (chunk_mass && i >= T_t) chunk_mass[(i - T_t) / o->chunk] += p;
+    if (p_row) p_row[i] = p;
+  }
+  free(logit);
+}
+
+static void allowed_for(const Oracle *o, const Seq *s, int layer, int kvh, unsigned char *allowed) {
+  int role = o->roles[layer * o->Hkv + kvh];
+  memset(allowed, 0, (size_t)(s->C > 0 ? s->C : 1));
+  if (role == ROLE_ANCHOR) {
+    for (int c = 0; c < s->C; ++c) allowed[c] = 1;
+  } else if (role == ROLE_TIDAL) {
+    for (int j = 0; j < s->S; ++j) {
+      int c = s->slot_chunk[(size_t)layer * s->S + j];
+      if (c >= 0) allowed[c] = 1;
+    }
+  } else {
+    const int *F = s->fixed_set + ((size_t)layer * o->Hkv + kvh) * s->S;
+    for (int j = 0; j < s->fixed_n[layer * o->Hkv + kvh]; ++j) allowed[F[j]] = 1;
+  }
+}
+
+/* ------------------------------------------------------------------ */
+/* Prefill placement (Prefill Compression, restated at chunk level)     */
+/* ------------------------------------------------------------------ */
+
+/* k,v: [n_tokens][Hkv][d] bf16 bits; audio = [audio_begin, audio_end); q_last: [Hq][d]. */
+int wnwo_place_prefill(Oracle *o, int seq, int layer, const uint16_t *k, const uint16_t *v, int n_tokens,
+                       int audio_begin, int audio_end, const uint16_t *q_last) {
+  if (!o || seq < 0 || seq >= o->max_batch || layer < 0 || layer >= o->L || !k || !v || n_tokens < 0) return WNWO_ERR_ARG;
+  if (audio_begin < 0 || audio_end < audio_begin || audio_end > n_tokens) return WNWO_ERR_ARG;
+  const int T_a = audio_end - audio_begin, T_t = n_tokens - T_a, Hkv = o->Hkv, d = o->d;
+  if (T_a > o->max_audio || T_t > o->max_text) return WNWO_ERR_ARG;
+  Seq *s = &o->seq[seq];
+  if (layer == 0 && s->placed_layers != 0) { free_seq(o, s); }
+  if (s->placed_layers == 0) {
+    if (layer != 0) return WNWO_ERR_STATE;
+    int rc = alloc_seq(o, s, T_a, T_t);
+    if (rc) return rc;
+  } else if (layer != s->placed_layers || T_a != s->T_a || T_t != s->T_t) {
+    return WNWO_ERR_STATE;
+  }
+  /* copy: text positions keep their order, audio positions keep theirs */
+  int ti = 0;
+  for (int i = 0; i < n_tokens; ++i) {
+    int is_audio = i >= audio_begin && i < audio_end;
+    for (int h = 0; h < Hkv; ++h) {
+      const uint16_t *ks = k + ((size_t)i * Hkv + h) * d, *vs = v + ((size_t)i * Hkv + h) * d;
+      uint16_t *kd, *vd;
+      if (is_audio) {
+        size_t off = ((size_t)h * T_a + (size_t)(i - audio_begin)) * d;
+        kd = s->audK[layer] + off; vd = s->audV[layer] + off;
+      } else {
+        size_t off = ((size_t)h * s->T_cap + (size_t)ti) * d;
+        kd = s->txtK[layer] + off; vd = s->txtV[layer] + off;
+      }
+      memcpy(kd, ks, (size_t)d * 2); memcpy(vd, vs, (size_t)d * 2);
+    }
+    if (!is_audio) ++ti;
+  }
+  s->placed_layers = layer + 1;
+  const int C = s->C, S = s->S;
+  if (C == 0) return WNWO_OK;
+  if (!q_last) return WNWO_ERR_ARG;
+  /* per non-anchor KV-head: pre[c] = sum over its q-heads and tau in c of softmax(q_last K / sqrt d) over text+audio */
+  unsigned char *all = (unsigned char *)malloc((size_t)C);
+  double *out = (double *)malloc(sizeof(double) * d);
+  int *lens = (int *)malloc(sizeof(int) * C);
+  float *keyf = (float *)malloc(sizeof(float) * C);
+  double *tid = (double *)calloc((size_t)C, sizeof(double));
+  memset(all, 1, (size_t)C);
+  for (int c = 0; c < C; ++c) lens[c] = chunk_len(o, s, c);
+  int n_tid = 0;
+  for (int h = 0; h < Hkv; ++h) {
+    double *pre = s->pre + ((size_t)layer * Hkv + h) * C;
+    for (int c = 0; c < C; ++c) pre[c] = 0.0;
+    int role = o->roles[layer * Hkv + h];
+    if (role == ROLE_ANCHOR) continue;
+    for (int j = 0; j < o->g; ++j)
+      attend(o, s, layer, h, q_last + (size_t)(h * o->g + j) * d, T_t, all, out, pre, NULL);
+    if (role == ROLE_FIXED) { /* its own top-S chunks, frozen */
+      for (int c = 0; c < C; ++c) keyf[c] = (float)pre[c];
+      int *F = s->fixed_set + ((size_t)layer * Hkv + h) * S;
+      s->fixed_n[layer * Hkv + h] = wnwo_topk(keyf, lens, C, S, F);
+    } else {
+      for (int c = 0; c < C; ++c) tid[c] += pre[c]; /* summed in head order */
+      ++n_tid;
+    }
+  }
+  if (n_tid > 0) { /* one table for the layer's tidal heads: rank r -> slot r, stamp -1-r */
+    for (int c = 0; c < C; ++c) keyf[c] = (float)tid[c];
+    int *tmp = (int *)malloc(sizeof(int) * S);
+    int n = wnwo_topk(keyf, lens, C, S, tmp);
+    for (int r = 0; r < n; ++r) {
+      s->slot_chunk[(size_t)layer * S + r] = tmp[r];
+      s->stamp[(size_t)layer * S + r] = -1 - (long long)r;
+    }
+    free(tmp);
+  }
+  free(all); free(out); free(lens); free(keyf); free(tid);
+  return WNWO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Decode step                                                          */
+/* ------------------------------------------------------------------ */
+
+int wnwo_step_begin(Oracle *o, const int *active, int n_active) {
+  if (!o || !active || n_active < 1 || n_active > o->max_batch) return WNWO_ERR_ARG;
+  if (o->in_step) return WNWO_ERR_STATE;
+  for (int i = 0; i < n_active; ++i) {
+    int b = active[i];
+    if (b < 0 || b >= o->max_batch) return WNWO_ERR_ARG;
+    if (o->seq[b].placed_layers != o->L) return WNWO_ERR_STATE;
+    for (int j = 0; j < i; ++j) if (active[j] == b) return WNWO_ERR_ARG;
+  }
+  memcpy(o->active, active, sizeof(int) * n_active);
+  o->n_active = n_active; o->in_step = 1; o->next_layer = 0; o->appended = -1;
+  return WNWO_OK;
+}
+
+/* q: [n_active][Hq][d]; k_new,v_new: [n_active][Hkv][d] or NULL; out: [n_active][Hq][d] double. */
+int wnwo_decode_layer(Oracle *o, int layer, const uint16_t *q, const uint16_t *k_new, const uint16_t *v_new, double *out) {
+  if (!o || !q || !out || (k_new == NULL) != (v_new == NULL)) return WNWO_ERR_ARG;
+  if (!o->in_step || layer != o->next_layer) return WNWO_ERR_STATE;
+  const int has_new = k_new != NULL;
+  if (o->appended >= 0 && o->appended != has_new) return WNWO_ERR_STATE;
+  const int Hq = o->Hq, Hkv = o->Hkv, d = o->d, g = o->g;
+  for (int i = 0; i < o->n_active; ++i)
+    if (has_new && o->seq[o->active[i]].T_t + 1 > o->seq[o->active[i]].T_cap) return WNWO_ERR_ARG;
+  o->appended = has_new;
+  const int anchor_layer = layer_has(o, layer, ROLE_ANCHOR);
+  for (int i = 0; i < o->n_active; ++i) {
+    Seq *s = &o->seq[o->active[i]];
+    int T_t = s->T_t;
+    if (has_new) { /* generated tokens are kept in full: append to the text region */
+      for (int h = 0; h < Hkv; ++h) {
+        size_t off = ((size_t)h * s->T_cap + (size_t)T_t) * d;
+        memcpy(s->txtK[layer] + off, k_new + ((size_t)i * Hkv + h) * d, (size_t)d * 2);
+        memcpy(s->txtV[layer] + off, v_new + ((size_t)i * Hkv + h) * d, (size_t)d * 2);
+      }
+      T_t += 1;
+    }
+    const int C = s->C;
+    double *mass = (double *)calloc((size_t)Hq * (size_t)(C > 0 ? C : 1), sizeof(double));
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int hq = 0; hq < Hq; ++hq) {
+      int kvh = hq / g;
+      unsigned char *allowed = (unsigned char *)malloc((size_t)(C > 0 ? C : 1));
+      allowed_for(o, s, layer, kvh, allowed);
+      int is_anchor = o->roles[layer * Hkv + kvh] == ROLE_ANCHOR;
+      attend(o, s, layer, kvh, q + ((size_t)i * Hq + hq) * d, T_t, allowed, out + ((size_t)i * Hq + hq) * d,
+             is_anchor ? mass + (size_t)hq * C : NULL, NULL);
+      free(allowed);
+    }
+    if (anchor_layer) { /* Eq. 2 summed over tau in c, over this layer's anchor q-heads, in head order */
+      double *sc = s->score_sum + (size_t)layer * C;
+      for (int c = 0; c < C; ++c) sc[c] = 0.0;
+      for (int hq = 0; hq < Hq; ++hq)
+        if (o->roles[layer * Hkv + hq / g] == ROLE_ANCHOR)
+          for (int c = 0; c < C; ++c) sc[c] += mass[(size_t)hq * C + c];
+    }
+    free(mass);
+  }
+  o->next_layer = layer + 1;
+  return WNWO_OK;
+}
+
+/* Selection + table update of every tidal layer, from this step's scores. */
+int wnwo_step_end(Oracle *o) {
+  if (!o || !o->in_step || o->next_layer != o->L) return WNWO_ERR_STATE;
+  for (int i = 0; i < o->n_active; ++i) {
+    Seq *s = &o->seq[o->active[i]];
+    const int C = s->C, S = s->S;
+    if (C > 0) {
+      int *lens = (int *)malloc(sizeof(int) * C);
+      float *sf = (float *)malloc(sizeof(float) * C);
+      int *pc = (int *)malloc(sizeof(int) * o->topk), *ps = (int *)malloc(sizeof(int) * o->topk),
+          *ev = (int *)malloc(sizeof(int) * o->topk);
+      for (int c = 0; c < C; ++c) lens[c] = chunk_len(o, s, c);
+      for (int l = 0; l < o->L; ++l) {
+        s->n_sel[l] = 0;
+        if (o->src[l] < 0) continue;
+        const double *sc = s->score_sum + (size_t)o->src[l] * C;
+        for (int c = 0; c < C; ++c) sf[c] = (float)sc[c];
+        int k = o->topk < S ? o->topk : S;
+        k = wnwo_topk(sf, lens, C, k, s->sel + (size_t)l * o->topk);
+        s->n_sel[l] = k;
+        int hits = 0;
+        int n = wnwo_table_update(s->slot_chunk + (size_t)l * S, s->stamp + (size_t)l * S, S, s->sel + (size_t)l * o->topk, k,
+                                  s->steps, o->topk, pc, ps, ev, &hits);
+        s->hits += hits; s->misses += n;
+        for (int j = 0; j < n; ++j) s->evictions += ev[j] >= 0;
+      }
+      free(lens); free(sf); free(pc); free(ps); free(ev);
+    }
+    s->steps += 1;
+    if (o->appended == 1) s->T_t += 1;
+  }
+  o->in_step = 0;
+  return WNWO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* Inspection and lock-step helpers                                     */
+/* ------------------------------------------------------------------ */
+
+int wnwo_get_dims(const Oracle *o, int seq, int *T_a, int *T_t, int *C, int *S) {
+  if (!o || seq < 0 || seq >= o->max_batch || o->seq[seq].placed_layers == 0) return WNWO_ERR_STATE;
+  const Seq *s = &o->seq[seq];
+  *T_a = s->T_a; *T_t = s->T_t; *C = s->C; *S = s->S;
+  return WNWO_OK;
+}
+int wnwo_get_chunk_scores(const Oracle *o, int seq, int layer, double *scores) {
+  const Seq *s = &o->seq[seq];
+  memcpy(scores, s->score_sum + (size_t)layer * s->C, sizeof(double) * s->C);
+  return WNWO_OK;
+}
+int wnwo_get_prefill_scores(const Oracle *o, int seq, int layer, int kvh, double *scores) {
+  const Seq *s = &o->seq[seq];
+  memcpy(scores, s->pre + ((size_t)layer * o->Hkv + kvh) * s->C, sizeof(double) * s->C);
+  return WNWO_OK;
+}
+int wnwo_get_selected(const Oracle *o, int seq, int layer, int *sel) {
+  const Seq *s = &o->seq[seq];
+  memcpy(sel, s->sel + (size_t)layer * o->topk, sizeof(int) * o->topk);
+  return s->n_sel[layer];
+}
+int wnwo_get_residency(const Oracle *o, int seq, int layer, int *slot_chunk, long long *stamp) {
+  const Seq *s = &o->seq[seq];
+  memcpy(slot_chunk, s->slot_chunk + (size_t)layer * s->S, sizeof(int) * s->S);
+  if (stamp) memcpy(stamp, s->stamp + (size_t)layer * s->S, sizeof(long long) * s->S);
+  return WNWO_OK;
+}
+int wnwo_set_residency(Oracle *o, int seq, int layer, const int *slot_chunk, const long long *stamp) {
+  Seq *s = &o->seq[seq];
+  memcpy(s->slot_chunk + (size_t)layer * s->S, slot_chunk, sizeof(int) * s->S);
+  memcpy(s->stamp + (size_t)layer * s->S, stamp, sizeof(long long) * s->S);
+  return WNWO_OK;
+}
+int wnwo_get_fixed_set(const Oracle *o, int seq, int layer, int kvh, int *chunks) {
+  const Seq *s = &o->seq[seq];
+  int n = s->fixed_n[layer * o->Hkv + kvh];
+  memcpy(chunks, s->fixed_set + ((size_t)layer * o->Hkv + kvh) * s->S, sizeof(int) * n);
+  return n;
+}
+int wnwo_set_fixed_set(Oracle *o, int seq, int layer, int kvh, const int *chunks, int n) {
+  Seq *s = &o->seq[seq];
+  if (n > s->S) return WNWO_ERR_ARG;
+  memcpy(s->fixed_set + ((size_t)layer * o->Hkv + kvh) * s->S, chunks, sizeof(int) * n);
+  s->fixed_n[layer * o->Hkv + kvh] = n;
+  return WNWO_OK;
+}
+int wnwo_get_stats(const Oracle *o, int seq, long long *hits, long long *misses, long long *evictions) {
+  const Seq *s = &o->seq[seq];
+  *hits = s->hits; *misses = s->misses; *evictions = s->evictions;
+  return WNWO_OK;
+}
+
+/* The probability row of one query head over [text | audio] as the oracle sees
+ * it now (no state change, no append).  p_row: [T_t + T_a]; out: [d]. */
+int wnwo_attention_row(const Oracle *o, int seq, int layer, int q_head, const uint16_t *q, double *p_row, double *out) {
+  if (!o || seq < 0 || seq >= o->max_batch || layer < 0 || layer >= o->L || q_head < 0 || q_head >= o->Hq) return WNWO_ERR_ARG;
+  const Seq *s = &o->seq[seq];
+  if (s->placed_layers <= layer) return WNWO_ERR_STATE;
+  unsigned char *allowed = (unsigned char *)malloc((size_t)(s->C > 0 ? s->C : 1));
+  allowed_for(o, s, layer, q_head / o->g, allowed);
+  attend(o, s, layer, q_head / o->g, q, s->T_t, allowed, out, NULL, p_row);
+  free(allowed);
+  return WNWO_OK;
+}
