@@ -1,0 +1,195 @@
+/*
+ * wnw.h -- C ABI of the WnW decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * WnW (Waxing-and-Waning KV cache) serves long-form speech LLM decoding with a
+ * GQA KV cache whose audio KV-heads carry offline-assigned roles (Method
+ * section, "Method Overview" and "Three-Way Classification"):
+ *   anchor  heads keep all audio KV on the GPU; their decode-time softmax
+ *           weights are the importance signal (Eq. 2);
+ *   tidal   heads keep a budgeted set of audio chunks on the GPU and the rest
+ *           in pinned host memory, recalled on demand ("Dynamic Chunk
+ *           Selection");
+ *   fixed   heads keep a static subset chosen at prefill ("Prefill
+ *           Compression"); the rest is discarded.
+ * Text KV (prompt and generated tokens) is always kept in full.
+ *
+ * This library implements the per-token, per-layer decode step in the
+ * chunk-granular form: non-overlapping chunks of `chunk_tokens` audio tokens
+ * are the unit of scoring, selection, residency and transfer; each non-anchor
+ * head keeps S = min(C, max(1, floor((double)budget * C + 1e-6))) chunks of the
+ * C = ceil(T_a / chunk_tokens) chunks of a sequence.
+ *
+ * Conventions
+ *   - All tensor arguments named *_dev are DEVICE pointers to bf16 data
+ *     (2 bytes per element, row-major, innermost index last), 16-byte aligned.
+ *     Arguments named *_host are HOST pointers.  The library never takes
+ *     ownership of caller buffers; they must stay valid until the work queued
+ *     on the given stream has completed.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - Every call returns a wnw_status_t and never throws or aborts.  On error,
+ *     out-parameters are left untouched.  Errors detected on the device
+ *     (table invariant violations) are sticky and reported by wnw_sync.
+ *   - A cache object is not thread-safe.  Calls for one cache must come from
+ *     one thread at a time.
+ *   - Position encoding (RoPE) is the caller's job: q and K arrive rotated.
+ */
+#ifndef WNW_H_
+#define WNW_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct wnw_cache wnw_cache_t; /* opaque, library-owned */
+
+typedef enum {
+  WNW_OK = 0,
+  WNW_ERR_INVALID_ARG = 1,
+  WNW_ERR_STATE = 2,      /* call out of order (decode before prefill, layer order, ...) */
+  WNW_ERR_OOM_DEVICE = 3,
+  WNW_ERR_OOM_HOST = 4,   /* pinned host allocation failed */
+  WNW_ERR_CUDA = 5,       /* a CUDA runtime call failed */
+  WNW_ERR_CAPACITY = 6,   /* text or audio capacity exceeded */
+  WNW_ERR_TIMEOUT = 7,    /* reserved */
+  WNW_ERR_UNSUPPORTED = 8,/* shape outside what the kernels are built for */
+  WNW_ERR_DEVICE_CHECK = 9/* a device-side consistency check failed (sticky) */
+} wnw_status_t;
+
+enum { WNW_ROLE_ANCHOR = 0, WNW_ROLE_TIDAL = 1, WNW_ROLE_FIXED = 2 };
+
+/* Storage mode.  TIERED is WnW.  FULL stores every head in full on the GPU
+ * (the "Full Cache" baseline of the Baselines paragraph) and serves
+ * wnw_decode_layer_full; roles are ignored for storage in that mode. */
+enum { WNW_MODE_TIERED = 0, WNW_MODE_FULL = 1 };
+
+/* How recall copies are issued (for measurement; results are identical for 0 and 1):
+ *   0  side stream, overlapped with the following layers (default)
+ *   1  on the caller's stream right after the layer (the paper's naive schedule, Limitations section)
+ *   2  skipped: tables update, no bytes move (timing experiments only; outputs become wrong) */
+enum { WNW_RECALL_SIDE_STREAM = 0, WNW_RECALL_INLINE = 1, WNW_RECALL_SKIP = 2 };
+
+typedef struct {
+  int32_t n_layers, n_q_heads, n_kv_heads; /* n_q_heads % n_kv_heads == 0, group <= 16 */
+  int32_t head_dim;                        /* 64 or 128 */
+  int32_t max_batch;                       /* sequences the cache can hold */
+  int32_t max_audio_tokens;                /* per sequence */
+  int32_t max_text_tokens;                 /* per sequence, prompt text + every decode append */
+  int32_t chunk_tokens;                    /* n_c; multiple of 16 */
+  int32_t topk;                            /* k, chunks selected per step; 0 -> 3 (the paper's k) */
+  int32_t evict_lag;                       /* the paper's delta; accepted, reserved (fixed pool evicts least-recent) */
+  float budget;                            /* (0,1]; see S above */
+  float softmax_scale;                     /* 0 -> 1/sqrt(head_dim) (Eq. 2) */
+  const uint8_t *roles;                    /* HOST [n_layers * n_kv_heads], WNW_ROLE_*, copied */
+  int32_t device;                          /* CUDA ordinal */
+  int32_t mode;                            /* WNW_MODE_* */
+  int32_t recall_mode;                     /* WNW_RECALL_* */
+} wnw_config_t;
+
+typedef struct {
+  int64_t steps;            /* decode steps completed (sum over sequences) */
+  int64_t hits, misses;     /* selected chunks found resident / recalled */
+  int64_t evictions;        /* residents displaced */
+  int64_t recall_bytes;     /* bytes copied host -> slot pool */
+  int64_t resident_audio_tokens; /* audio tokens on the GPU now, all heads (r_GPU numerator, Audio KV retention paragraph) */
+  int64_t host_audio_tokens;     /* audio tokens of tidal heads held in host memory and not on the GPU */
+  int64_t full_audio_tokens;     /* L * H_kv * T_a summed over placed sequences (denominator) */
+} wnw_stats_t;
+
+/* Create a cache: head roles from the offline triage, GPU budget, capacities.
+ * Allocates all device stores up front; pinned host mirrors are allocated per
+ * sequence at prefill.  Rejects: tidal heads with no anchor anywhere, head_dim
+ * not in {64,128}, chunk_tokens not a multiple of 16, budget outside (0,1],
+ * group > 16.  ("Three-Way Classification"; Eq. 1 budget; "Chunk Structure".) */
+wnw_status_t wnw_create(const wnw_config_t *cfg_host, wnw_cache_t **out);
+
+/* Frees everything the cache owns.  Synchronises the device first. */
+wnw_status_t wnw_destroy(wnw_cache_t *cache);
+
+/* Place one layer's prefill KV of one sequence ("Prefill Compression", chunk-level).
+ *   k_dev, v_dev : [n_tokens][n_kv_heads][head_dim] bf16; tokens [audio_begin, audio_end) are audio,
+ *                  all others text, order preserved within each kind.
+ *   q_last_dev   : [n_q_heads][head_dim] bf16, the last prefix query; ranks chunks for non-anchor heads:
+ *                  pre[c] = sum over the head's query group and tau in c of softmax(q_last K / sqrt d)_tau.
+ *                  Fixed head keeps its own top-S chunks; the layer's tidal heads share one table holding the
+ *                  top-S chunks of their summed pre (rank r in slot r).  May be NULL if the sequence has no audio
+ *                  or in FULL mode.
+ * Layers of a sequence must be placed in order 0..n_layers-1 with the same token counts; placing layer 0 again
+ * re-initialises the sequence.  Work is queued on cuda_stream; the caller's buffers may be released once that
+ * work has completed.  Tidal heads' audio KV is mirrored to pinned host memory allocated here. */
+wnw_status_t wnw_place_prefill(wnw_cache_t *cache, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                               int32_t n_tokens, int32_t audio_begin, int32_t audio_end, const void *q_last_dev,
+                               void *cuda_stream);
+
+/* Open a decode step for the given sequences (HOST array of distinct sequence ids, all fully placed).
+ * The order of active_seqs_host is the batch order of q/k_new/v_new/out in wnw_decode_layer. */
+wnw_status_t wnw_step_begin(wnw_cache_t *cache, const int32_t *active_seqs_host, int32_t n_active);
+
+/* One layer of one decode step ("Decode-Step Score Aggregation", "Dynamic Chunk Selection").
+ *   q_dev             : [n_active][n_q_heads][head_dim] bf16
+ *   k_new_dev,v_new_dev: [n_active][n_kv_heads][head_dim] bf16 of the token being generated, appended to the text
+ *                       region before attention; both NULL to attend without appending.  Either every layer of
+ *                       a step appends or none does.
+ *   out_dev           : [n_active][n_q_heads][head_dim] bf16 attention outputs:
+ *                       anchor heads over text + all audio; tidal heads over text + the chunks resident at the end
+ *                       of the previous step; fixed heads over text + their prefill subset.
+ * Also computed on the device, with no host round trip: this layer's chunk scores
+ * score_sum[c] = sum over the layer's anchor q-heads and tau in c of the softmax weight (Eq. 2 summed per chunk);
+ * for every tidal layer whose score source is now complete (its own anchors, else the nearest anchor layer, ties
+ * to the lower layer) the top-k chunks by mean score (ties to the lower index), the residency table update
+ * (hit: refresh; miss: lowest free slot, else least recently selected resident not selected now) and the recall
+ * of missing chunks from pinned host memory into the slot pool.  The updated table is used from the next step.
+ * Layers must be called in order 0..n_layers-1.  TIERED mode only. */
+wnw_status_t wnw_decode_layer(wnw_cache_t *cache, int32_t layer, const void *q_dev, const void *k_new_dev,
+                              const void *v_new_dev, void *out_dev, void *cuda_stream);
+
+/* Full-cache comparison path ("Full Cache" baseline): same arguments, every head attends to text + all audio,
+ * no scores, no selection.  FULL mode only. */
+wnw_status_t wnw_decode_layer_full(wnw_cache_t *cache, int32_t layer, const void *q_dev, const void *k_new_dev,
+                                   const void *v_new_dev, void *out_dev, void *cuda_stream);
+
+/* Close the step: per-sequence step counters and text lengths advance.  All layers must have been called. */
+wnw_status_t wnw_step_end(wnw_cache_t *cache, void *cuda_stream);
+
+/* Inspection.  Each call drains the cache's streams first.  Out-buffers are HOST memory owned by the caller.
+ *   chunk_scores : score_sum of the last completed step, [C] floats (anchor layers only)
+ *   prefill_scores: pre[c] of one non-anchor KV-head, [C] floats
+ *   selected     : chunk ids in rank order, up to topk
+ *   residency    : slot_chunk[S] (-1 = free) and, if stamp_host != NULL, the recency stamps
+ *   fixed_set    : the head's chunk ids in prefill rank order
+ *   seq_dims     : T_a, current T_t, C, S of a placed sequence
+ *   slot_kv      : the K or V rows of one tidal head in one slot, [chunk_tokens][head_dim] bf16 (which: 0 = K, 1 = V) */
+wnw_status_t wnw_get_chunk_scores(wnw_cache_t *cache, int32_t seq, int32_t layer, float *scores_host, int32_t *n_chunks);
+wnw_status_t wnw_get_prefill_scores(wnw_cache_t *cache, int32_t seq, int32_t layer, int32_t kv_head, float *scores_host,
+                                    int32_t *n_chunks);
+wnw_status_t wnw_get_selected(wnw_cache_t *cache, int32_t seq, int32_t layer, int32_t *sel_host, int32_t *n_sel);
+wnw_status_t wnw_get_residency(wnw_cache_t *cache, int32_t seq, int32_t layer, int32_t *slot_chunk_host,
+                               int64_t *stamp_host, int32_t *n_slots);
+wnw_status_t wnw_get_fixed_set(wnw_cache_t *cache, int32_t seq, int32_t layer, int32_t kv_head, int32_t *chunks_host,
+                               int32_t *n);
+wnw_status_t wnw_get_seq_dims(wnw_cache_t *cache, int32_t seq, int32_t *audio_tokens, int32_t *text_tokens,
+                              int32_t *n_chunks, int32_t *n_slots);
+wnw_status_t wnw_get_slot_kv(wnw_cache_t *cache, int32_t seq, int32_t layer, int32_t kv_head, int32_t slot, int32_t which,
+                             void *rows_host);
+wnw_status_t wnw_get_stats(wnw_cache_t *cache, wnw_stats_t *stats_host);
+
+/* Optional per-kernel timing: when enabled the library brackets its attention-kernel launches with CUDA events
+ * on the launching stream; wnw_get_kernel_time returns the accumulated milliseconds and launch count since the
+ * last call (drains the stream).  Off by default. */
+wnw_status_t wnw_set_kernel_timing(wnw_cache_t *cache, int32_t enable);
+wnw_status_t wnw_get_kernel_time(wnw_cache_t *cache, float *attn_ms, int32_t *attn_launches);
+
+/* Drain the caller's stream and the recall stream; returns the sticky asynchronous status. */
+wnw_status_t wnw_sync(wnw_cache_t *cache);
+
+/* Host-link probe used by the benchmark: copies `bytes` from pinned host memory into device memory `reps` times
+ * (a) with cudaMemcpyAsync and (b) with the library's recall kernel on a synthetic plan, and returns GB/s of each. */
+wnw_status_t wnw_measure_host_link(int32_t device, int64_t bytes, int32_t reps, double *memcpy_gbs, double *kernel_gbs);
+
+const char *wnw_status_string(wnw_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WNW_H_ */

@@ -1,0 +1,143 @@
+// Internal device-side view of a WnW cache and launch-argument structs shared by the kernels
+// and the host runtime.  Nothing here is part of the public ABI (see include/wnw.h).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace wnw {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int GR = 16;        // tokens per granule: one mma k16/n16 tile, the unit of loading and of score partials
+constexpr int MAX_TOPK = 8;   // upper bound on config topk
+constexpr int MAX_G = 16;     // query heads per KV head handled by one m16 tile
+
+constexpr int ROLE_ANCHOR = 0, ROLE_TIDAL = 1, ROLE_FIXED = 2;
+
+// device status bits (sticky)
+constexpr int STATUS_NO_VICTIM = 1;     // table update found no evictable slot
+constexpr int STATUS_BAD_TABLE = 2;     // slot/chunk id out of range
+constexpr int STATUS_NONFINITE = 4;     // non-finite chunk score
+
+struct WorkItem {  // one CTA of the attention kernel
+  int32_t i;       // index into the active-sequence list
+  int32_t h;       // KV head
+  int32_t g0, g1;  // granule range in the head's virtual key space [text capacity | audio]
+};
+struct HeadItems { int32_t first, count; };  // work items of one (active seq, KV head)
+
+struct LayerInfo {
+  int32_t n_anchor, n_tidal, n_fixed;
+  int32_t anchor_off;   // anchor heads in earlier layers
+  int32_t fixed_off;    // fixed heads in earlier layers
+  int32_t tid_prefix;   // tidal heads in earlier layers
+  int32_t src;          // layer whose scores rank this layer's chunks, -1 if it has no tidal head
+  int32_t upd_first, upd_count;  // range in upd_list: layers whose tables are updated in this layer's tail
+  long long pool_off;   // element offset of this layer's slots inside one sequence's pool
+};
+
+struct Geometry {
+  int32_t L, Hq, Hkv, d, g, nc, gpc, topk;
+  int32_t T_cap_pad, n_tg;         // text capacity (multiple of 16) and its granules
+  int32_t C_max, S_max, T_a_pad;   // chunk / slot capacity per sequence; audio capacity padded to whole chunks
+  int32_t A_tot, F_tot;            // anchor / fixed heads per sequence over all layers
+  int32_t max_batch;
+  long long text_seq_stride, anchor_seq_stride, pool_seq_stride, fixed_seq_stride;  // elements
+  float scale_log2;                // softmax scale * log2(e)
+};
+
+struct CacheView {
+  Geometry geo;
+  const uint8_t *roles;      // [L][Hkv]
+  const int16_t *role_idx;   // [L][Hkv] index among the heads of the same role in that layer
+  const LayerInfo *layers;   // [L]
+  const int32_t *upd_list;   // concatenated per-layer update lists
+  bf16 *text, *anchor, *pool, *fixed;
+  int32_t *text_len, *T_a, *C, *S;   // [B]
+  long long *steps;                  // [B]
+  int32_t *slot_chunk;               // [B][L][S_max]
+  int32_t *chunk_slot;               // [B][L][C_max]
+  long long *stamp;                  // [B][L][S_max]
+  float *score_sum;                  // [B][L][C_max]
+  int32_t *sel, *n_sel;              // [B][L][topk], [B][L]
+  int32_t *plan, *n_plan;            // [B][L][topk][2] (chunk, slot), [B][L]
+  int32_t *fixed_chunks, *fixed_n;   // [B][F_tot][S_max], [B][F_tot]
+  float *pre;                        // [B][L][Hkv][C_max]
+  unsigned long long *stats;         // [B][4] hits, misses, evictions, recall_bytes
+  bf16 **mirror;                     // [B] pinned host mirrors (device-visible addresses)
+  int32_t *status;
+};
+
+// ---- address helpers (element offsets; every row is d bf16) ----
+__host__ __device__ inline long long text_off(const Geometry &G, int b, int l, int h, int kv) {
+  return (long long)b * G.text_seq_stride + ((long long)(l * G.Hkv + h) * 2 + kv) * G.T_cap_pad * G.d;
+}
+__host__ __device__ inline long long anchor_off(const Geometry &G, long long seq_stride, int b, int head, int kv) {
+  return (long long)b * seq_stride + ((long long)head * 2 + kv) * G.T_a_pad * G.d;
+}
+__host__ __device__ inline long long pool_off(const Geometry &G, const LayerInfo &li, int b, int slot, int t_idx, int kv) {
+  return (long long)b * G.pool_seq_stride + li.pool_off + ((long long)(slot * li.n_tidal + t_idx) * 2 + kv) * G.nc * G.d;
+}
+__host__ __device__ inline long long fixed_off(const Geometry &G, const LayerInfo &li, int b, int f_idx, int kv) {
+  return (long long)b * G.fixed_seq_stride + ((long long)(li.fixed_off + f_idx) * 2 + kv) * G.S_max * G.nc * G.d;
+}
+__host__ __device__ inline long long mirror_off(const Geometry &G, const LayerInfo &li, int C_b, int c, int t_idx, int kv) {
+  return (((long long)C_b * li.tid_prefix + (long long)c * li.n_tidal + t_idx) * 2 + kv) * G.nc * G.d;
+}
+
+// ---- attention launch ----
+enum { ATTN_DECODE = 0, ATTN_FULL = 1, ATTN_PREFILL = 2 };
+
+struct AttnArgs {
+  int32_t mode;          // ATTN_*
+  int32_t layer;
+  int32_t n_active;
+  int32_t has_new;       // the text region holds one more row than text_len says
+  int32_t score_on;      // write per-granule softmax-mass partials for anchor-like heads
+  const int32_t *active; // [n_active] sequence ids
+  const WorkItem *items;
+  int32_t n_items;
+  const bf16 *q;         // [n_active][Hq][d]
+  // anchor-like source: decode -> cache anchor store; full -> same store, head = l*Hkv+h; prefill -> staging, head = h
+  const bf16 *anchor_base;
+  long long anchor_seq_stride;
+  int32_t anchor_head0;
+  // outputs
+  float *part_o;         // [n_items][g][d]
+  float2 *part_ml;       // [n_items][g]   (m in log2 units, l)
+  float2 *gran_em;       // [n_active][n_aq][n_ag_max]  (sum of 2^(s-m) over the granule, m at that time)
+  int32_t n_aq, n_ag_max;
+};
+
+struct TailArgs {
+  int32_t mode, layer, n_active, score_on;
+  const int32_t *active;
+  const HeadItems *head_items;  // [n_active][Hkv]
+  const float *part_o;
+  const float2 *part_ml;
+  const float2 *gran_em;
+  int32_t n_aq, n_ag_max;
+  float2 *head_mz;              // [n_active][Hq] final (M, Z) per query head
+  bf16 *out;                    // [n_active][Hq][d]
+  int32_t *seq_done;            // [n_active] completion counters (self-resetting)
+};
+
+// kernels' host launchers (defined in the .cu files)
+cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st);
+cudaError_t launch_tail(const CacheView &cv, const TailArgs &a, int max_count, cudaStream_t st);
+cudaError_t launch_append(const CacheView &cv, int layer, int n_active, const int32_t *active, const bf16 *k_new,
+                          const bf16 *v_new, cudaStream_t st);
+cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *active, int appended, cudaStream_t st);
+cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,
+                          int skip_copy, cudaStream_t st);
+cudaError_t launch_place_scatter(const CacheView &cv, int b, int layer, const bf16 *k, const bf16 *v, int n_tokens, int ab,
+                                 int ae, int T_t, int C_b, int S_b, bf16 *stage, cudaStream_t st);
+cudaError_t launch_prefill_select(const CacheView &cv, int b, int layer, const HeadItems *head_items, const float2 *part_ml,
+                                  const float2 *gran_em, int n_ag_max, cudaStream_t st);
+cudaError_t launch_place_gather(const CacheView &cv, int b, int layer, int full_mode, const bf16 *stage, int C_b,
+                                cudaStream_t st);
+cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
+int attn_warps();  // warps per attention CTA (granules per work item should be a multiple)
+
+}  // namespace wnw

@@ -1,0 +1,838 @@
+// Host runtime behind the C ABI of include/wnw.h: cache object, device stores, work lists, streams and events.
+// Every step of the path runs in the kernels of wnw_attn.cu / wnw_kernels.cu; this file only validates
+// arguments, sizes buffers and queues launches.  There is no CPU fallback.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/wnw.h"
+#include "wnw_internal.cuh"
+
+using namespace wnw;
+
+namespace {
+
+struct SeqHost {
+  int placed_layers = 0;
+  int T_a = 0, T_t = 0, C = 0, S = 0;
+  bf16 *mirror = nullptr;
+  size_t mirror_bytes = 0;
+};
+
+struct LayerWork {
+  int first_item = 0, n_items = 0, max_count = 0;  // range in the uploaded item array
+  int head_items_off = 0;                          // offset in the uploaded HeadItems array
+};
+
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+struct wnw_cache {
+  wnw_config_t cfg;
+  Geometry geo;
+  CacheView cv;
+  std::vector<uint8_t> roles;
+  std::vector<int16_t> role_idx;
+  std::vector<LayerInfo> layers;
+  std::vector<int32_t> upd_list;
+  std::vector<int> tail_of;  // layer -> layer whose tail updates its table, -1 if none
+  int tid_total = 0, n_sm = 148;
+  std::vector<SeqHost> seqs;
+  std::vector<void *> dev_allocs;
+  std::vector<bf16 *> mirror_ptrs;  // host copy of cv.mirror
+  bf16 *stage = nullptr;
+  int32_t *d_iota = nullptr, *d_active = nullptr;
+  // step state
+  std::vector<int> active;
+  bool in_step = false;
+  int next_layer = 0, appended = -1;
+  // work lists
+  std::vector<int> wl_active;
+  std::vector<int> wl_T_a;
+  std::vector<LayerWork> wl_layers;
+  WorkItem *d_items = nullptr;
+  HeadItems *d_head_items = nullptr;
+  size_t d_items_cap = 0, d_head_items_cap = 0;
+  int prefill_C = -1;
+  WorkItem *d_pf_items = nullptr;
+  HeadItems *d_pf_head_items = nullptr;
+  int pf_n_items = 0;
+  size_t pf_items_cap = 0;
+  // partial buffers
+  float *part_o = nullptr;
+  float2 *part_ml = nullptr, *gran_em = nullptr, *head_mz = nullptr;
+  int32_t *seq_done = nullptr;
+  int part_cap_items = 0, n_aq_max = 0, n_ag_max = 0;
+  // streams / events
+  cudaStream_t side = nullptr, last_stream = nullptr;
+  std::vector<cudaEvent_t> ev_layer_done, ev_recall_done;
+  std::vector<char> recall_recorded;
+  cudaEvent_t ev_place = nullptr, ev_step = nullptr;
+  bool place_recorded = false, step_recorded = false;
+  // timing
+  bool timing = false;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> t_used;
+  std::vector<cudaEvent_t> t_free;
+  cudaError_t last_cuda = cudaSuccess;
+};
+
+#define CK(expr)                                 \
+  do {                                           \
+    cudaError_t _e = (expr);                     \
+    if (_e != cudaSuccess) {                     \
+      c->last_cuda = _e;                         \
+      return _e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA; \
+    }                                            \
+  } while (0)
+
+static int slots_for(float budget, int C) {
+  if (C <= 0) return 0;
+  int S = (int)std::floor((double)budget * (double)C + 1e-6);
+  if (S < 1) S = 1;
+  if (S > C) S = C;
+  return S;
+}
+
+template <typename T>
+static wnw_status_t dev_alloc(wnw_cache *c, T **p, size_t count, bool zero = true) {
+  const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
+  CK(cudaMalloc((void **)p, bytes));
+  c->dev_allocs.push_back((void *)*p);
+  if (zero) CK(cudaMemset(*p, 0, bytes));
+  return WNW_OK;
+}
+template <typename T>
+static wnw_status_t dev_upload(wnw_cache *c, T **p, const std::vector<T> &v) {
+  wnw_status_t s = dev_alloc(c, p, v.size(), true);
+  if (s != WNW_OK) return s;
+  if (!v.empty()) CK(cudaMemcpy(*p, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice));
+  return WNW_OK;
+}
+
+static void destroy_impl(wnw_cache *c) {
+  DeviceGuard guard(c->cfg.device);
+  cudaDeviceSynchronize();
+  for (void *p : c->dev_allocs) cudaFree(p);
+  for (auto &s : c->seqs)
+    if (s.mirror) cudaFreeHost(s.mirror);
+  if (c->side) cudaStreamDestroy(c->side);
+  for (auto e : c->ev_layer_done) cudaEventDestroy(e);
+  for (auto e : c->ev_recall_done) cudaEventDestroy(e);
+  if (c->ev_place) cudaEventDestroy(c->ev_place);
+  if (c->ev_step) cudaEventDestroy(c->ev_step);
+  for (auto &p : c->t_used) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
+  for (auto e : c->t_free) cudaEventDestroy(e);
+  delete c;
+}
+
+extern "C" const char *wnw_status_string(wnw_status_t s) {
+  switch (s) {
+    case WNW_OK: return "ok";
+    case WNW_ERR_INVALID_ARG: return "invalid argument";
+    case WNW_ERR_STATE: return "call out of order for the cache's state";
+    case WNW_ERR_OOM_DEVICE: return "out of device memory";
+    case WNW_ERR_OOM_HOST: return "out of pinned host memory";
+    case WNW_ERR_CUDA: return "CUDA runtime error";
+    case WNW_ERR_CAPACITY: return "sequence capacity exceeded";
+    case WNW_ERR_TIMEOUT: return "timeout";
+    case WNW_ERR_UNSUPPORTED: return "unsupported shape";
+    case WNW_ERR_DEVICE_CHECK: return "device-side consistency check failed";
+  }
+  return "unknown status";
+}
+
+static wnw_status_t validate_config(const wnw_config_t *cfg) {
+  if (!cfg || !cfg->roles) return WNW_ERR_INVALID_ARG;
+  if (cfg->n_layers < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads % cfg->n_kv_heads) return WNW_ERR_INVALID_ARG;
+  if (cfg->max_batch < 1 || cfg->max_audio_tokens < 0 || cfg->max_text_tokens < 0) return WNW_ERR_INVALID_ARG;
+  if (cfg->max_audio_tokens + cfg->max_text_tokens < 1) return WNW_ERR_INVALID_ARG;
+  if (cfg->chunk_tokens < 1 || cfg->topk < 0 || cfg->topk > MAX_TOPK || cfg->evict_lag < 0) return WNW_ERR_INVALID_ARG;
+  if (!(cfg->budget > 0.f && cfg->budget <= 1.f)) return WNW_ERR_INVALID_ARG;
+  if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return WNW_ERR_INVALID_ARG;
+  if (cfg->mode != WNW_MODE_TIERED && cfg->mode != WNW_MODE_FULL) return WNW_ERR_INVALID_ARG;
+  if (cfg->recall_mode < WNW_RECALL_SIDE_STREAM || cfg->recall_mode > WNW_RECALL_SKIP) return WNW_ERR_INVALID_ARG;
+  if (cfg->device < 0) return WNW_ERR_INVALID_ARG;
+  bool any_anchor = false, any_tidal = false;
+  for (int i = 0; i < cfg->n_layers * cfg->n_kv_heads; ++i) {
+    if (cfg->roles[i] > WNW_ROLE_FIXED) return WNW_ERR_INVALID_ARG;
+    any_anchor |= cfg->roles[i] == WNW_ROLE_ANCHOR;
+    any_tidal |= cfg->roles[i] == WNW_ROLE_TIDAL;
+  }
+  if (cfg->mode == WNW_MODE_TIERED && any_tidal && !any_anchor) return WNW_ERR_INVALID_ARG;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return WNW_ERR_UNSUPPORTED;
+  if (cfg->chunk_tokens % GR) return WNW_ERR_UNSUPPORTED;
+  if (cfg->n_q_heads / cfg->n_kv_heads > MAX_G) return WNW_ERR_UNSUPPORTED;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
+  if (!out) return WNW_ERR_INVALID_ARG;
+  wnw_status_t vs = validate_config(cfg);
+  if (vs != WNW_OK) return vs;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device >= n_dev) return WNW_ERR_CUDA;
+  wnw_cache *c = new (std::nothrow) wnw_cache();
+  if (!c) return WNW_ERR_OOM_HOST;
+  c->cfg = *cfg;
+  if (c->cfg.topk == 0) c->cfg.topk = 3;
+  DeviceGuard guard(cfg->device);
+  auto fail = [&](wnw_status_t s) { destroy_impl(c); return s; };
+#define CKC(call) do { wnw_status_t _s = (call); if (_s != WNW_OK) return fail(_s); } while (0)
+#define CKE(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { return fail(_e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA); } } while (0)
+  cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
+  const int L = cfg->n_layers, Hkv = cfg->n_kv_heads, d = cfg->head_dim, nc = cfg->chunk_tokens;
+  const bool full = cfg->mode == WNW_MODE_FULL;
+  c->roles.assign(cfg->roles, cfg->roles + (size_t)L * Hkv);
+  c->cfg.roles = nullptr;
+  Geometry &G = c->geo;
+  G.L = L; G.Hq = cfg->n_q_heads; G.Hkv = Hkv; G.d = d; G.g = cfg->n_q_heads / Hkv; G.nc = nc; G.gpc = nc / GR;
+  G.topk = c->cfg.topk;
+  G.T_cap_pad = (std::max(cfg->max_text_tokens, 1) + GR - 1) / GR * GR;
+  G.n_tg = G.T_cap_pad / GR;
+  G.C_max = (cfg->max_audio_tokens + nc - 1) / nc;
+  G.S_max = full ? 0 : slots_for(cfg->budget, G.C_max);
+  G.T_a_pad = std::max(G.C_max, 1) * nc;
+  G.max_batch = cfg->max_batch;
+  const double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / std::sqrt((double)d);
+  G.scale_log2 = (float)(scale * 1.4426950408889634);
+  // roles -> per-layer tables, score routing, update lists
+  c->role_idx.assign((size_t)L * Hkv, 0);
+  c->layers.assign(L, LayerInfo{});
+  int a_tot = 0, f_tot = 0, t_tot = 0;
+  long long pool_elems = 0;
+  for (int l = 0; l < L; ++l) {
+    LayerInfo &li = c->layers[l];
+    li.anchor_off = a_tot; li.fixed_off = f_tot; li.tid_prefix = t_tot; li.pool_off = pool_elems; li.src = -1;
+    for (int h = 0; h < Hkv; ++h) {
+      const int role = c->roles[l * Hkv + h];
+      int16_t &ri = c->role_idx[l * Hkv + h];
+      if (role == ROLE_ANCHOR) ri = (int16_t)li.n_anchor++;
+      else if (role == ROLE_TIDAL) ri = (int16_t)li.n_tidal++;
+      else ri = (int16_t)li.n_fixed++;
+    }
+    a_tot += li.n_anchor; f_tot += li.n_fixed; t_tot += li.n_tidal;
+    pool_elems += (long long)G.S_max * li.n_tidal * 2 * nc * d;
+  }
+  c->tid_total = t_tot;
+  c->tail_of.assign(L, -1);
+  std::vector<std::vector<int>> upd(L);
+  for (int l = 0; l < L; ++l) {
+    if (full || c->layers[l].n_tidal == 0) continue;
+    int best = -1;
+    for (int a = 0; a < L; ++a)
+      if (c->layers[a].n_anchor > 0 && (best < 0 || std::abs(a - l) < std::abs(best - l))) best = a;
+    c->layers[l].src = best;  // nearest anchor layer, ties to the lower one
+    const int x = std::max(l, best);  // the first point at which both layer l's attention and its source scores are done
+    c->tail_of[l] = x;
+    upd[x].push_back(l);
+  }
+  for (int l = 0; l < L; ++l) {
+    c->layers[l].upd_first = (int)c->upd_list.size();
+    c->layers[l].upd_count = (int)upd[l].size();
+    c->upd_list.insert(c->upd_list.end(), upd[l].begin(), upd[l].end());
+  }
+  G.A_tot = full ? L * Hkv : a_tot;
+  G.F_tot = full ? 0 : f_tot;
+  G.text_seq_stride = (long long)L * Hkv * 2 * G.T_cap_pad * d;
+  G.anchor_seq_stride = (long long)G.A_tot * 2 * G.T_a_pad * d;
+  G.pool_seq_stride = full ? 0 : pool_elems;
+  G.fixed_seq_stride = (long long)G.F_tot * 2 * G.S_max * nc * d;
+
+  CacheView &cv = c->cv;
+  memset(&cv, 0, sizeof(cv));
+  cv.geo = G;
+  const size_t B = (size_t)cfg->max_batch;
+  {
+    uint8_t *p; int16_t *q; LayerInfo *li; int32_t *ul;
+    CKC(dev_upload(c, &p, c->roles)); cv.roles = p;
+    CKC(dev_upload(c, &q, c->role_idx)); cv.role_idx = q;
+    CKC(dev_upload(c, &li, c->layers)); cv.layers = li;
+    CKC(dev_upload(c, &ul, c->upd_list)); cv.upd_list = ul;
+  }
+  CKC(dev_alloc(c, &cv.text, B * (size_t)G.text_seq_stride));
+  CKC(dev_alloc(c, &cv.anchor, B * (size_t)G.anchor_seq_stride));
+  CKC(dev_alloc(c, &cv.pool, B * (size_t)G.pool_seq_stride));
+  CKC(dev_alloc(c, &cv.fixed, B * (size_t)G.fixed_seq_stride));
+  CKC(dev_alloc(c, &c->stage, (size_t)Hkv * 2 * G.T_a_pad * d));
+  CKC(dev_alloc(c, &cv.text_len, B)); CKC(dev_alloc(c, &cv.T_a, B)); CKC(dev_alloc(c, &cv.C, B)); CKC(dev_alloc(c, &cv.S, B));
+  CKC(dev_alloc(c, &cv.steps, B));
+  CKC(dev_alloc(c, &cv.slot_chunk, B * L * std::max(G.S_max, 1)));
+  CKC(dev_alloc(c, &cv.chunk_slot, B * L * std::max(G.C_max, 1)));
+  CKC(dev_alloc(c, &cv.stamp, B * L * std::max(G.S_max, 1)));
+  CKC(dev_alloc(c, &cv.score_sum, B * L * std::max(G.C_max, 1)));
+  CKC(dev_alloc(c, &cv.sel, B * L * G.topk)); CKC(dev_alloc(c, &cv.n_sel, B * L));
+  CKC(dev_alloc(c, &cv.plan, B * L * G.topk * 2)); CKC(dev_alloc(c, &cv.n_plan, B * L));
+  CKC(dev_alloc(c, &cv.fixed_chunks, B * std::max(G.F_tot, 1) * std::max(G.S_max, 1)));
+  CKC(dev_alloc(c, &cv.fixed_n, B * std::max(G.F_tot, 1)));
+  CKC(dev_alloc(c, &cv.pre, B * L * Hkv * std::max(G.C_max, 1)));
+  CKC(dev_alloc(c, &cv.stats, B * 4));
+  CKC(dev_alloc(c, &cv.mirror, B));
+  CKC(dev_alloc(c, &cv.status, 1));
+  {
+    std::vector<int32_t> iota(B);
+    for (size_t i = 0; i < B; ++i) iota[i] = (int32_t)i;
+    CKC(dev_upload(c, &c->d_iota, iota));
+  }
+  CKC(dev_alloc(c, &c->d_active, B));
+  // partial buffers: the work-list builder keeps items <= target + heads
+  int n_aq = 0;
+  for (int l = 0; l < L; ++l) n_aq = std::max(n_aq, c->layers[l].n_anchor * G.g);
+  c->n_aq_max = std::max(n_aq, 1);
+  c->n_ag_max = std::max(G.C_max * G.gpc, 1);
+  c->part_cap_items = 2 * c->n_sm + (int)B * Hkv + 16;
+  CKC(dev_alloc(c, &c->part_o, (size_t)c->part_cap_items * G.g * d, false));
+  CKC(dev_alloc(c, &c->part_ml, (size_t)c->part_cap_items * G.g, false));
+  CKC(dev_alloc(c, &c->gran_em, std::max(B * (size_t)c->n_aq_max, (size_t)G.Hq) * c->n_ag_max, false));
+  CKC(dev_alloc(c, &c->head_mz, B * (size_t)G.Hq, false));
+  CKC(dev_alloc(c, &c->seq_done, B));
+  c->seqs.assign(B, SeqHost{});
+  c->mirror_ptrs.assign(B, nullptr);
+  CKE(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
+  c->ev_layer_done.resize(L); c->ev_recall_done.resize(L); c->recall_recorded.assign(L, 0);
+  for (int l = 0; l < L; ++l) {
+    CKE(cudaEventCreateWithFlags(&c->ev_layer_done[l], cudaEventDisableTiming));
+    CKE(cudaEventCreateWithFlags(&c->ev_recall_done[l], cudaEventDisableTiming));
+  }
+  CKE(cudaEventCreateWithFlags(&c->ev_place, cudaEventDisableTiming));
+  CKE(cudaEventCreateWithFlags(&c->ev_step, cudaEventDisableTiming));
+  CKE(cudaDeviceSynchronize());
+#undef CKC
+#undef CKE
+  *out = c;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_destroy(wnw_cache_t *c) {
+  if (!c) return WNW_ERR_INVALID_ARG;
+  destroy_impl(c);
+  return WNW_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Work lists: split every (sequence, KV head) granule space into CTA-sized items
+// ---------------------------------------------------------------------------------------------
+static int granules_per_item(const wnw_cache *c, long long total_granules) {
+  const int nw = attn_warps();
+  const long long target = 2ll * c->n_sm;
+  long long per = (total_granules + target - 1) / target;
+  per = (per + nw - 1) / nw * nw;
+  return (int)std::max<long long>(per, nw);
+}
+
+// Appends the items of one layer for the given sequences.  audio_granules(role, b) gives each head's audio part.
+static void build_layer_items(const wnw_cache *c, int layer, int mode, const std::vector<int> &seq_ids,
+                              std::vector<WorkItem> &items, std::vector<HeadItems> &heads, LayerWork &lw) {
+  const Geometry &G = c->geo;
+  std::vector<int> n_gran(seq_ids.size() * G.Hkv);
+  long long total = 0;
+  for (size_t i = 0; i < seq_ids.size(); ++i) {
+    const SeqHost &s = c->seqs[seq_ids[i]];
+    for (int h = 0; h < G.Hkv; ++h) {
+      const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
+      const int audio = (role == ROLE_ANCHOR ? s.C : s.S) * G.gpc;
+      n_gran[i * G.Hkv + h] = G.n_tg + audio;
+      total += G.n_tg + audio;
+    }
+  }
+  const int gpi = granules_per_item(c, total);
+  lw.first_item = (int)items.size();
+  lw.head_items_off = (int)heads.size();
+  lw.max_count = 0;
+  for (size_t i = 0; i < seq_ids.size(); ++i)
+    for (int h = 0; h < G.Hkv; ++h) {
+      const int n = n_gran[i * G.Hkv + h];
+      HeadItems hi{(int)items.size() - lw.first_item, 0};
+      for (int g0 = 0; g0 < n; g0 += gpi) {
+        items.push_back(WorkItem{(int)i, h, g0, std::min(n, g0 + gpi)});
+        ++hi.count;
+      }
+      heads.push_back(hi);
+      lw.max_count = std::max(lw.max_count, hi.count);
+    }
+  lw.n_items = (int)items.size() - lw.first_item;
+}
+
+static wnw_status_t ensure_worklists(wnw_cache *c) {
+  std::vector<int> T_a(c->active.size());
+  for (size_t i = 0; i < c->active.size(); ++i) T_a[i] = c->seqs[c->active[i]].T_a;
+  if (c->wl_active == c->active && c->wl_T_a == T_a && !c->wl_layers.empty()) return WNW_OK;
+  const Geometry &G = c->geo;
+  const int mode = c->cfg.mode == WNW_MODE_FULL ? ATTN_FULL : ATTN_DECODE;
+  std::vector<WorkItem> items;
+  std::vector<HeadItems> heads;
+  c->wl_layers.assign(G.L, LayerWork{});
+  for (int l = 0; l < G.L; ++l) {
+    build_layer_items(c, l, mode, c->active, items, heads, c->wl_layers[l]);
+    if (c->wl_layers[l].n_items > c->part_cap_items) return WNW_ERR_CAPACITY;
+  }
+  // the previous lists may still be read by queued kernels
+  CK(cudaDeviceSynchronize());
+  if (items.size() > c->d_items_cap) {
+    CK(cudaMalloc((void **)&c->d_items, items.size() * sizeof(WorkItem)));
+    c->dev_allocs.push_back(c->d_items);
+    c->d_items_cap = items.size();
+  }
+  if (heads.size() > c->d_head_items_cap) {
+    CK(cudaMalloc((void **)&c->d_head_items, heads.size() * sizeof(HeadItems)));
+    c->dev_allocs.push_back(c->d_head_items);
+    c->d_head_items_cap = heads.size();
+  }
+  CK(cudaMemcpy(c->d_items, items.data(), items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
+  CK(cudaMemcpy(c->d_head_items, heads.data(), heads.size() * sizeof(HeadItems), cudaMemcpyHostToDevice));
+  std::vector<int32_t> act(c->active.begin(), c->active.end());
+  CK(cudaMemcpy(c->d_active, act.data(), act.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+  c->wl_active = c->active;
+  c->wl_T_a = T_a;
+  return WNW_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Prefill placement
+// ---------------------------------------------------------------------------------------------
+extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                                          int32_t n_tokens, int32_t audio_begin, int32_t audio_end, const void *q_last_dev,
+                                          void *cuda_stream) {
+  if (!c || !k_dev || !v_dev) return WNW_ERR_INVALID_ARG;
+  const Geometry &G = c->geo;
+  if (seq < 0 || seq >= G.max_batch || layer < 0 || layer >= G.L || n_tokens < 1) return WNW_ERR_INVALID_ARG;
+  if (audio_begin < 0 || audio_end < audio_begin || audio_end > n_tokens) return WNW_ERR_INVALID_ARG;
+  if (c->in_step) return WNW_ERR_STATE;
+  const int T_a = audio_end - audio_begin, T_t = n_tokens - T_a;
+  if (T_a > c->cfg.max_audio_tokens || T_t > c->cfg.max_text_tokens) return WNW_ERR_CAPACITY;
+  const bool full = c->cfg.mode == WNW_MODE_FULL;
+  SeqHost &s = c->seqs[seq];
+  if (layer != 0 && (layer != s.placed_layers || T_a != s.T_a || T_t != s.T_t)) return WNW_ERR_STATE;
+  const int C_b = (T_a + G.nc - 1) / G.nc, S_b = full ? 0 : slots_for(c->cfg.budget, C_b);
+  if (!full && C_b > 0 && !q_last_dev) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (layer == 0) {
+    s.placed_layers = 0;
+    const size_t need = full ? 0 : (size_t)C_b * c->tid_total * 2 * G.nc * G.d * sizeof(bf16);
+    if (need != s.mirror_bytes) {
+      CK(cudaDeviceSynchronize());
+      if (s.mirror) cudaFreeHost(s.mirror);
+      s.mirror = nullptr; s.mirror_bytes = 0;
+      if (need) {
+        void *p = nullptr;
+        if (cudaHostAlloc(&p, need, cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess) {
+          cudaGetLastError();
+          return WNW_ERR_OOM_HOST;
+        }
+        void *dp = nullptr;
+        CK(cudaHostGetDevicePointer(&dp, p, 0));
+        s.mirror = (bf16 *)p; s.mirror_bytes = need;
+        c->mirror_ptrs[seq] = (bf16 *)dp;
+      } else {
+        c->mirror_ptrs[seq] = nullptr;
+      }
+      CK(cudaMemcpy(c->cv.mirror + seq, &c->mirror_ptrs[seq], sizeof(bf16 *), cudaMemcpyHostToDevice));
+    }
+    s.T_a = T_a; s.T_t = T_t; s.C = C_b; s.S = S_b;
+    c->wl_layers.clear();  // dims may have changed
+  }
+  // the staging buffer and the partial buffers are shared: order after earlier placements and steps
+  if (c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
+  if (c->step_recorded) CK(cudaStreamWaitEvent(st, c->ev_step, 0));
+  CK(launch_place_scatter(c->cv, seq, layer, (const bf16 *)k_dev, (const bf16 *)v_dev, n_tokens, audio_begin, audio_end, T_t,
+                          C_b, S_b, c->stage, st));
+  if (!full && C_b > 0) {
+    if (c->prefill_C != C_b) {
+      std::vector<WorkItem> items;
+      std::vector<HeadItems> heads;
+      LayerWork lw;
+      std::vector<int> one{seq};
+      build_layer_items(c, layer, ATTN_PREFILL, one, items, heads, lw);
+      if ((int)items.size() > c->part_cap_items) return WNW_ERR_CAPACITY;
+      if (items.size() > c->pf_items_cap) {
+        CK(cudaMalloc((void **)&c->d_pf_items, items.size() * sizeof(WorkItem)));
+        c->dev_allocs.push_back(c->d_pf_items);
+        c->pf_items_cap = items.size();
+      }
+      if (!c->d_pf_head_items) {
+        CK(cudaMalloc((void **)&c->d_pf_head_items, (size_t)G.Hkv * sizeof(HeadItems)));
+        c->dev_allocs.push_back(c->d_pf_head_items);
+      }
+      for (auto &it : items) it.i = 0;
+      CK(cudaMemcpyAsync(c->d_pf_items, items.data(), items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice, st));
+      CK(cudaMemcpyAsync(c->d_pf_head_items, heads.data(), heads.size() * sizeof(HeadItems), cudaMemcpyHostToDevice, st));
+      CK(cudaStreamSynchronize(st));  // the host vectors go out of scope
+      c->pf_n_items = (int)items.size();
+      c->prefill_C = C_b;
+    }
+    AttnArgs a{};
+    a.mode = ATTN_PREFILL; a.layer = layer; a.n_active = 1; a.has_new = 0; a.score_on = 1;
+    a.active = c->d_iota + seq; a.items = c->d_pf_items; a.n_items = c->pf_n_items;
+    a.q = (const bf16 *)q_last_dev;
+    a.anchor_base = c->stage; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
+    a.part_o = c->part_o; a.part_ml = c->part_ml; a.gran_em = c->gran_em; a.n_aq = G.Hq; a.n_ag_max = c->n_ag_max;
+    CK(launch_attn(c->cv, a, st));
+    CK(launch_prefill_select(c->cv, seq, layer, c->d_pf_head_items, c->part_ml, c->gran_em, c->n_ag_max, st));
+  }
+  CK(launch_place_gather(c->cv, seq, layer, full ? 1 : 0, c->stage, C_b, st));
+  CK(cudaEventRecord(c->ev_place, st));
+  c->place_recorded = true;
+  c->last_stream = st;
+  s.placed_layers = layer + 1;
+  return WNW_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Decode step
+// ---------------------------------------------------------------------------------------------
+extern "C" wnw_status_t wnw_step_begin(wnw_cache_t *c, const int32_t *active, int32_t n_active) {
+  if (!c || !active || n_active < 1 || n_active > c->geo.max_batch) return WNW_ERR_INVALID_ARG;
+  if (c->in_step) return WNW_ERR_STATE;
+  for (int i = 0; i < n_active; ++i) {
+    if (active[i] < 0 || active[i] >= c->geo.max_batch) return WNW_ERR_INVALID_ARG;
+    for (int j = 0; j < i; ++j)
+      if (active[j] == active[i]) return WNW_ERR_INVALID_ARG;
+    if (c->seqs[active[i]].placed_layers != c->geo.L) return WNW_ERR_STATE;
+  }
+  DeviceGuard guard(c->cfg.device);
+  c->active.assign(active, active + n_active);
+  wnw_status_t s = ensure_worklists(c);
+  if (s != WNW_OK) return s;
+  c->in_step = true; c->next_layer = 0; c->appended = -1;
+  return WNW_OK;
+}
+
+static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer, const void *q, const void *k_new,
+                                      const void *v_new, void *out, void *cuda_stream) {
+  if (!c || !q || !out || ((k_new == nullptr) != (v_new == nullptr))) return WNW_ERR_INVALID_ARG;
+  if (c->cfg.mode != want_mode) return WNW_ERR_STATE;
+  if (!c->in_step || layer != c->next_layer) return WNW_ERR_STATE;
+  const int has_new = k_new != nullptr;
+  if (c->appended >= 0 && c->appended != has_new) return WNW_ERR_STATE;
+  if (has_new)
+    for (int b : c->active)
+      if (c->seqs[b].T_t + 1 > c->cfg.max_text_tokens) return WNW_ERR_CAPACITY;
+  const Geometry &G = c->geo;
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int n_active = (int)c->active.size();
+  const bool tiered = want_mode == WNW_MODE_TIERED;
+  if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
+  // the recall that refreshed this layer's slots (issued in the previous step) must have landed
+  if (tiered && c->cfg.recall_mode == WNW_RECALL_SIDE_STREAM) {
+    const int x = c->tail_of[layer];
+    if (x >= 0 && c->recall_recorded[x]) CK(cudaStreamWaitEvent(st, c->ev_recall_done[x], 0));
+  }
+  if (has_new) CK(launch_append(c->cv, layer, n_active, c->d_active, (const bf16 *)k_new, (const bf16 *)v_new, st));
+  const LayerWork &lw = c->wl_layers[layer];
+  const LayerInfo &li = c->layers[layer];
+  AttnArgs a{};
+  a.mode = tiered ? ATTN_DECODE : ATTN_FULL; a.layer = layer; a.n_active = n_active; a.has_new = has_new;
+  a.score_on = tiered && li.n_anchor > 0;
+  a.active = c->d_active; a.items = c->d_items + lw.first_item; a.n_items = lw.n_items;
+  a.q = (const bf16 *)q;
+  a.anchor_base = c->cv.anchor; a.anchor_seq_stride = G.anchor_seq_stride;
+  a.anchor_head0 = tiered ? li.anchor_off : layer * G.Hkv;
+  a.part_o = c->part_o; a.part_ml = c->part_ml; a.gran_em = c->gran_em;
+  a.n_aq = std::max(li.n_anchor * G.g, 1); a.n_ag_max = c->n_ag_max;
+  cudaEvent_t t0 = nullptr, t1 = nullptr;
+  if (c->timing) {
+    for (cudaEvent_t *e : {&t0, &t1}) {
+      if (!c->t_free.empty()) { *e = c->t_free.back(); c->t_free.pop_back(); }
+      else CK(cudaEventCreate(e));
+    }
+    CK(cudaEventRecord(t0, st));
+  }
+  CK(launch_attn(c->cv, a, st));
+  if (c->timing) {
+    CK(cudaEventRecord(t1, st));
+    c->t_used.emplace_back(t0, t1);
+  }
+  TailArgs t{};
+  t.mode = a.mode; t.layer = layer; t.n_active = n_active; t.score_on = a.score_on;
+  t.active = c->d_active; t.head_items = c->d_head_items + lw.head_items_off;
+  t.part_o = c->part_o; t.part_ml = c->part_ml; t.gran_em = c->gran_em; t.n_aq = a.n_aq; t.n_ag_max = a.n_ag_max;
+  t.head_mz = c->head_mz; t.out = (bf16 *)out; t.seq_done = c->seq_done;
+  CK(launch_tail(c->cv, t, lw.max_count, st));
+  if (tiered && li.upd_count > 0) {
+    const int skip = c->cfg.recall_mode == WNW_RECALL_SKIP;
+    if (c->cfg.recall_mode == WNW_RECALL_SIDE_STREAM) {
+      CK(cudaEventRecord(c->ev_layer_done[layer], st));
+      CK(cudaStreamWaitEvent(c->side, c->ev_layer_done[layer], 0));
+      CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count, 0, c->side));
+      CK(cudaEventRecord(c->ev_recall_done[layer], c->side));
+      c->recall_recorded[layer] = 1;
+    } else {
+      CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count, skip, st));
+    }
+  }
+  c->appended = has_new;
+  c->next_layer = layer + 1;
+  c->last_stream = st;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_decode_layer(wnw_cache_t *c, int32_t layer, const void *q, const void *k_new, const void *v_new,
+                                         void *out, void *cuda_stream) {
+  return decode_layer_impl(c, WNW_MODE_TIERED, layer, q, k_new, v_new, out, cuda_stream);
+}
+extern "C" wnw_status_t wnw_decode_layer_full(wnw_cache_t *c, int32_t layer, const void *q, const void *k_new,
+                                              const void *v_new, void *out, void *cuda_stream) {
+  return decode_layer_impl(c, WNW_MODE_FULL, layer, q, k_new, v_new, out, cuda_stream);
+}
+
+extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
+  if (!c) return WNW_ERR_INVALID_ARG;
+  if (!c->in_step || c->next_layer != c->geo.L) return WNW_ERR_STATE;
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1, st));
+  CK(cudaEventRecord(c->ev_step, st));
+  c->step_recorded = true;
+  for (int b : c->active)
+    if (c->appended == 1) c->seqs[b].T_t += 1;
+  c->in_step = false;
+  c->last_stream = st;
+  return WNW_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Inspection
+// ---------------------------------------------------------------------------------------------
+static wnw_status_t drain(wnw_cache *c) {
+  CK(cudaStreamSynchronize(c->last_stream));
+  CK(cudaStreamSynchronize(c->side));
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_sync(wnw_cache_t *c) {
+  if (!c) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  wnw_status_t s = drain(c);
+  if (s != WNW_OK) return s;
+  int32_t st = 0;
+  CK(cudaMemcpy(&st, c->cv.status, sizeof(st), cudaMemcpyDeviceToHost));
+  return st ? WNW_ERR_DEVICE_CHECK : WNW_OK;
+}
+
+static wnw_status_t check_seq_layer(wnw_cache *c, int seq, int layer) {
+  if (!c) return WNW_ERR_INVALID_ARG;
+  if (seq < 0 || seq >= c->geo.max_batch || layer < 0 || layer >= c->geo.L) return WNW_ERR_INVALID_ARG;
+  if (c->seqs[seq].placed_layers <= layer) return WNW_ERR_STATE;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_seq_dims(wnw_cache_t *c, int32_t seq, int32_t *T_a, int32_t *T_t, int32_t *C, int32_t *S) {
+  if (!c || seq < 0 || seq >= c->geo.max_batch || !T_a || !T_t || !C || !S) return WNW_ERR_INVALID_ARG;
+  const SeqHost &s = c->seqs[seq];
+  if (s.placed_layers == 0) return WNW_ERR_STATE;
+  *T_a = s.T_a; *T_t = s.T_t; *C = s.C; *S = s.S;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_chunk_scores(wnw_cache_t *c, int32_t seq, int32_t layer, float *scores, int32_t *n) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!scores || !n) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  if ((s = drain(c)) != WNW_OK) return s;
+  const int C_b = c->seqs[seq].C;
+  if (C_b > 0)
+    CK(cudaMemcpy(scores, c->cv.score_sum + ((size_t)seq * c->geo.L + layer) * c->geo.C_max, C_b * sizeof(float),
+                  cudaMemcpyDeviceToHost));
+  *n = C_b;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_prefill_scores(wnw_cache_t *c, int32_t seq, int32_t layer, int32_t kv_head, float *scores,
+                                               int32_t *n) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!scores || !n || kv_head < 0 || kv_head >= c->geo.Hkv) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  if ((s = drain(c)) != WNW_OK) return s;
+  const int C_b = c->seqs[seq].C;
+  if (C_b > 0)
+    CK(cudaMemcpy(scores, c->cv.pre + (((size_t)seq * c->geo.L + layer) * c->geo.Hkv + kv_head) * c->geo.C_max,
+                  C_b * sizeof(float), cudaMemcpyDeviceToHost));
+  *n = C_b;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_selected(wnw_cache_t *c, int32_t seq, int32_t layer, int32_t *sel, int32_t *n_sel) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!sel || !n_sel) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  if ((s = drain(c)) != WNW_OK) return s;
+  const size_t bl = (size_t)seq * c->geo.L + layer;
+  int32_t n = 0;
+  CK(cudaMemcpy(&n, c->cv.n_sel + bl, sizeof(n), cudaMemcpyDeviceToHost));
+  if (n > 0) CK(cudaMemcpy(sel, c->cv.sel + bl * c->geo.topk, n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  *n_sel = n;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_residency(wnw_cache_t *c, int32_t seq, int32_t layer, int32_t *slot_chunk, int64_t *stamp,
+                                          int32_t *n_slots) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!slot_chunk || !n_slots) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  if ((s = drain(c)) != WNW_OK) return s;
+  const int S_b = c->seqs[seq].S;
+  const size_t off = ((size_t)seq * c->geo.L + layer) * std::max(c->geo.S_max, 1);
+  if (S_b > 0) {
+    CK(cudaMemcpy(slot_chunk, c->cv.slot_chunk + off, S_b * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (stamp) CK(cudaMemcpy(stamp, c->cv.stamp + off, S_b * sizeof(int64_t), cudaMemcpyDeviceToHost));
+  }
+  *n_slots = S_b;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_fixed_set(wnw_cache_t *c, int32_t seq, int32_t layer, int32_t kv_head, int32_t *chunks,
+                                          int32_t *n) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!chunks || !n || kv_head < 0 || kv_head >= c->geo.Hkv) return WNW_ERR_INVALID_ARG;
+  if (c->cfg.mode != WNW_MODE_TIERED || c->roles[layer * c->geo.Hkv + kv_head] != ROLE_FIXED) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  if ((s = drain(c)) != WNW_OK) return s;
+  const size_t fh = (size_t)seq * c->geo.F_tot + c->layers[layer].fixed_off + c->role_idx[layer * c->geo.Hkv + kv_head];
+  int32_t cnt = 0;
+  CK(cudaMemcpy(&cnt, c->cv.fixed_n + fh, sizeof(cnt), cudaMemcpyDeviceToHost));
+  if (cnt > 0) CK(cudaMemcpy(chunks, c->cv.fixed_chunks + fh * c->geo.S_max, cnt * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  *n = cnt;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_slot_kv(wnw_cache_t *c, int32_t seq, int32_t layer, int32_t kv_head, int32_t slot,
+                                        int32_t which, void *rows) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!rows || kv_head < 0 || kv_head >= c->geo.Hkv || which < 0 || which > 1) return WNW_ERR_INVALID_ARG;
+  if (c->cfg.mode != WNW_MODE_TIERED || c->roles[layer * c->geo.Hkv + kv_head] != ROLE_TIDAL) return WNW_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= c->seqs[seq].S) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  if ((s = drain(c)) != WNW_OK) return s;
+  const long long off = pool_off(c->geo, c->layers[layer], seq, slot, c->role_idx[layer * c->geo.Hkv + kv_head], which);
+  CK(cudaMemcpy(rows, c->cv.pool + off, (size_t)c->geo.nc * c->geo.d * sizeof(bf16), cudaMemcpyDeviceToHost));
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
+  if (!c || !out) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  wnw_status_t s = drain(c);
+  if (s != WNW_OK) return s;
+  const Geometry &G = c->geo;
+  const size_t B = (size_t)G.max_batch;
+  std::vector<unsigned long long> st(B * 4);
+  std::vector<long long> steps(B);
+  CK(cudaMemcpy(st.data(), c->cv.stats, st.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(steps.data(), c->cv.steps, B * sizeof(long long), cudaMemcpyDeviceToHost));
+  std::vector<int32_t> slot_chunk(B * G.L * std::max(G.S_max, 1)), fixed_n(B * std::max(G.F_tot, 1)),
+      fixed_chunks(B * std::max(G.F_tot, 1) * std::max(G.S_max, 1));
+  CK(cudaMemcpy(slot_chunk.data(), c->cv.slot_chunk, slot_chunk.size() * 4, cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(fixed_n.data(), c->cv.fixed_n, fixed_n.size() * 4, cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(fixed_chunks.data(), c->cv.fixed_chunks, fixed_chunks.size() * 4, cudaMemcpyDeviceToHost));
+  wnw_stats_t r{};
+  auto len_of = [&](const SeqHost &sq, int ch) { return std::min(G.nc, sq.T_a - ch * G.nc); };
+  for (size_t b = 0; b < B; ++b) {
+    const SeqHost &sq = c->seqs[b];
+    if (sq.placed_layers == 0) continue;
+    r.steps += steps[b];
+    r.hits += (int64_t)st[b * 4]; r.misses += (int64_t)st[b * 4 + 1]; r.evictions += (int64_t)st[b * 4 + 2];
+    r.recall_bytes += (int64_t)st[b * 4 + 3];
+    for (int l = 0; l < sq.placed_layers; ++l) {
+      const LayerInfo &li = c->layers[l];
+      r.full_audio_tokens += (int64_t)G.Hkv * sq.T_a;
+      if (c->cfg.mode == WNW_MODE_FULL) { r.resident_audio_tokens += (int64_t)G.Hkv * sq.T_a; continue; }
+      r.resident_audio_tokens += (int64_t)li.n_anchor * sq.T_a;
+      int64_t res = 0;
+      for (int j = 0; j < sq.S; ++j) {
+        const int ch = slot_chunk[(b * G.L + l) * std::max(G.S_max, 1) + j];
+        if (ch >= 0) res += len_of(sq, ch);
+      }
+      r.resident_audio_tokens += (int64_t)li.n_tidal * res;
+      r.host_audio_tokens += (int64_t)li.n_tidal * (sq.T_a - res);
+      for (int f = 0; f < li.n_fixed; ++f) {
+        const size_t fh = b * G.F_tot + li.fixed_off + f;
+        for (int j = 0; j < fixed_n[fh]; ++j) r.resident_audio_tokens += len_of(sq, fixed_chunks[fh * G.S_max + j]);
+      }
+    }
+  }
+  *out = r;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_set_kernel_timing(wnw_cache_t *c, int32_t enable) {
+  if (!c) return WNW_ERR_INVALID_ARG;
+  c->timing = enable != 0;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_kernel_time(wnw_cache_t *c, float *attn_ms, int32_t *attn_launches) {
+  if (!c || !attn_ms || !attn_launches) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(c->cfg.device);
+  wnw_status_t s = drain(c);
+  if (s != WNW_OK) return s;
+  float total = 0.f;
+  for (auto &p : c->t_used) {
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, p.first, p.second));
+    total += ms;
+    c->t_free.push_back(p.first); c->t_free.push_back(p.second);
+  }
+  *attn_ms = total;
+  *attn_launches = (int32_t)c->t_used.size();
+  c->t_used.clear();
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_measure_host_link(int32_t device, int64_t bytes, int32_t reps, double *memcpy_gbs, double *kernel_gbs) {
+  if (bytes < 4096 || reps < 1 || !memcpy_gbs || !kernel_gbs) return WNW_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  bytes = bytes / 16 * 16;
+  void *h = nullptr, *d = nullptr, *hd = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaStream_t st = nullptr;
+  wnw_status_t rc = WNW_OK;
+  float best_copy = 1e30f, best_kernel = 1e30f;
+  if (cudaHostAlloc(&h, bytes, cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess) { cudaGetLastError(); return WNW_ERR_OOM_HOST; }
+  memset(h, 1, bytes);
+  if (cudaMalloc(&d, bytes) != cudaSuccess) { cudaGetLastError(); cudaFreeHost(h); return WNW_ERR_OOM_DEVICE; }
+  if (cudaHostGetDevicePointer(&hd, h, 0) != cudaSuccess || cudaEventCreate(&e0) != cudaSuccess ||
+      cudaEventCreate(&e1) != cudaSuccess || cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess) {
+    rc = WNW_ERR_CUDA;
+  }
+  for (int r = 0; rc == WNW_OK && r < reps + 1; ++r) {
+    float ms = 0.f;
+    cudaEventRecord(e0, st);
+    cudaMemcpyAsync(d, h, bytes, cudaMemcpyHostToDevice, st);
+    cudaEventRecord(e1, st);
+    if (cudaStreamSynchronize(st) != cudaSuccess || cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc = WNW_ERR_CUDA; break; }
+    if (r > 0) best_copy = std::min(best_copy, ms);
+    cudaEventRecord(e0, st);
+    if (launch_copy_plan((const uint4 *)hd, (uint4 *)d, bytes / 16, 64, st) != cudaSuccess) { rc = WNW_ERR_CUDA; break; }
+    cudaEventRecord(e1, st);
+    if (cudaStreamSynchronize(st) != cudaSuccess || cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc = WNW_ERR_CUDA; break; }
+    if (r > 0) best_kernel = std::min(best_kernel, ms);
+  }
+  if (rc == WNW_OK) {
+    *memcpy_gbs = (double)bytes / (best_copy * 1e-3) / 1e9;
+    *kernel_gbs = (double)bytes / (best_kernel * 1e-3) / 1e9;
+  }
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (st) cudaStreamDestroy(st);
+  cudaFree(d);
+  cudaFreeHost(h);
+  return rc;
+}

@@ -1,0 +1,233 @@
+"""Lock-step parity driver: the CUDA path (through the C ABI binding) against the CPU oracle on the same seeded bits.
+
+Staged parity, because selected indices must match bit-exactly while the scores they derive from are floating point:
+  (i)   scores (decode chunk scores, prefill scores): |gpu - oracle| <= 1e-4 * |oracle| + 1e-8;
+  (ii)  the oracle's top-k and table update, run on the GPU's own fp32 scores and the GPU's previous table, must
+        reproduce the GPU's selection, table and stamps bit-exactly;
+  (iii) the oracle, selecting from its own fp64 scores, must agree as well; a disagreement is accepted only if the
+        ranking keys at the selection boundary are within 2e-4 relative (a near-tie), is counted, and the oracle then
+        adopts the GPU's table so the trajectories stay aligned.
+Attention outputs: max |gpu - oracle| <= 2e-2 (bf16 outputs of O(1) magnitude).
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import paper_2608_22704_b200 as wnw
+from helpers import bf16_bits_to_f64, make_oracle
+from oracle import wnw_oracle as wo
+from workloads import ROLE_ANCHOR, ROLE_FIXED, ROLE_TIDAL, Synth, Workload
+from workloads.synth import bf16_bits
+
+OUT_TOL = 2e-2
+SCORE_RTOL, SCORE_ATOL = 1e-4, 1e-8
+TIE_RTOL = 2e-4
+
+
+def chunk_lens(T_a, chunk):
+    C = -(-T_a // chunk)
+    return np.array([min(chunk, T_a - c * chunk) for c in range(C)], np.int32)
+
+
+def assert_scores_close(gpu, ref, what):
+    gpu = np.asarray(gpu, np.float64); ref = np.asarray(ref, np.float64)
+    err = np.abs(gpu - ref)
+    bound = SCORE_RTOL * np.abs(ref) + SCORE_ATOL
+    assert (err <= bound).all(), f"{what}: worst rel err {(err / np.maximum(np.abs(ref), 1e-30)).max():.3e}"
+
+
+def near_tie(scores64, lens, sel_a, sel_b):
+    """True if the two selections differ only across a near-tie of the ranking key."""
+    key = (np.asarray(scores64, np.float64) / lens)
+    diff = set(sel_a) ^ set(sel_b)
+    if not diff:   # same set, different order: the swapped ranks must be near-ties
+        diff = {a for a, b in zip(sel_a, sel_b) if a != b} | {b for a, b in zip(sel_a, sel_b) if a != b}
+    ks = key[sorted(diff)]
+    return (ks.max() - ks.min()) <= TIE_RTOL * max(ks.max(), 1e-30)
+
+
+class Lockstep:
+    def __init__(self, w: Workload, seed=0, device="cuda:0", recall_mode=0, gen_device=None, oracle_seqs=None):
+        self.w = w
+        self.dev = torch.device(device)
+        self.syn = Synth(w, seed=seed, device=gen_device or "cpu")
+        self.oracle_seqs = list(range(w.batch)) if oracle_seqs is None else list(oracle_seqs)
+        self.o = make_oracle(w)
+        self.h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max(max(w.audio_lens), 0),
+                                w.text_capacity, w.chunk, w.budget, w.roles, topk=w.topk, device=self.dev.index or 0,
+                                recall_mode=recall_mode)
+        self.kept = {}
+        self.near_ties = 0
+        self.max_out_err = 0.0
+        self.dec = {}
+        self.step = 0
+        self._steps = {}
+        self.expected_recall_bytes = 0
+
+    def close(self):
+        if self.h:
+            wnw.wnw_destroy(self.h); self.h = None
+        self.o.close()
+
+    # ------------------------------------------------------------------ prefill
+    def prefill(self, check_slots=True):
+        w = self.w
+        for b in range(w.batch):
+            for l in range(w.n_layers):
+                p = self.syn.prefill(b, l)
+                k, v, ql = (p[n].to(self.dev) for n in ("k", "v", "q_last"))
+                wnw.wnw_place_prefill(self.h, b, l, k, v, p["audio_begin"], p["audio_end"], ql)
+                if b in self.oracle_seqs:
+                    kb, vb = bf16_bits(p["k"]), bf16_bits(p["v"])
+                    self.o.place_prefill(b, l, kb, vb, p["audio_begin"], p["audio_end"], bf16_bits(p["q_last"]))
+                    self.kept[(b, l)] = (kb[p["audio_begin"]:p["audio_end"]], vb[p["audio_begin"]:p["audio_end"]])
+        wnw.wnw_sync(self.h)
+        for b in self.oracle_seqs:
+            T_a, T_t, C, S = wnw.wnw_get_seq_dims(self.h, b)
+            assert (T_a, T_t, C, S) == self.o.dims(b)
+            if C == 0:
+                continue
+            lens = chunk_lens(T_a, w.chunk)
+            for l in range(w.n_layers):
+                tid_sum = np.zeros(C, np.float32)
+                any_tid = False
+                for h in range(w.n_kv_heads):
+                    role = w.roles[l, h]
+                    if role == ROLE_ANCHOR:
+                        continue
+                    g_pre = wnw.wnw_get_prefill_scores(self.h, b, l, h)
+                    assert_scores_close(g_pre, self.o.prefill_scores(b, l, h), f"prefill scores b{b} l{l} h{h}")
+                    if role == ROLE_FIXED:
+                        g_set = wnw.wnw_get_fixed_set(self.h, b, l, h)
+                        assert g_set.tolist() == wo.topk(g_pre, lens, S).tolist(), f"fixed set (ii) b{b} l{l} h{h}"
+                        o_set = self.o.fixed_set(b, l, h)
+                        if g_set.tolist() != o_set.tolist():
+                            assert near_tie(self.o.prefill_scores(b, l, h), lens, g_set.tolist(), o_set.tolist())
+                            self.near_ties += 1
+                            self.o.set_fixed_set(b, l, h, g_set)
+                    else:
+                        tid_sum = (tid_sum + g_pre).astype(np.float32); any_tid = True
+                if any_tid:
+                    g_tab, g_stamp = wnw.wnw_get_residency(self.h, b, l)
+                    want = wo.topk(tid_sum, lens, S)
+                    assert g_tab.tolist() == want.tolist(), f"tidal table (ii) b{b} l{l}"
+                    assert g_stamp.tolist() == [-1 - r for r in range(S)]
+                    o_tab, o_stamp = self.o.residency(b, l)
+                    if g_tab.tolist() != o_tab.tolist():
+                        o_sum = sum(self.o.prefill_scores(b, l, h) for h in range(w.n_kv_heads) if w.roles[l, h] == ROLE_TIDAL)
+                        assert near_tie(o_sum, lens, g_tab.tolist(), o_tab.tolist())
+                        self.near_ties += 1
+                        self.o.set_residency(b, l, g_tab, g_stamp)
+                    if check_slots:
+                        self.check_slot_bytes(b, l)
+
+    def check_slot_bytes(self, b, l):
+        """Slot contents are an exact copy of the source K,V of the chunk the table says is there."""
+        w = self.w
+        tab, _ = wnw.wnw_get_residency(self.h, b, l)
+        T_a = w.audio_lens[b]
+        kb, vb = self.kept[(b, l)]
+        for h in range(w.n_kv_heads):
+            if w.roles[l, h] != ROLE_TIDAL:
+                continue
+            for j, c in enumerate(tab.tolist()):
+                if c < 0:
+                    continue
+                n = min(w.chunk, T_a - c * w.chunk)
+                for which, src in ((0, kb), (1, vb)):
+                    rows = wnw.wnw_get_slot_kv(self.h, b, l, h, j, which, w.chunk, w.head_dim)
+                    assert np.array_equal(rows[:n], src[c * w.chunk:c * w.chunk + n, h]), f"slot bytes b{b} l{l} h{h} slot{j}"
+
+    # ------------------------------------------------------------------ decode
+    def _dec(self, b, l):
+        if (b, l) not in self.dec:
+            self.dec[(b, l)] = self.syn.decode(b, l)
+        return self.dec[(b, l)]
+
+    def decode_step(self, t=None, append=True, active=None, check_slots=False):
+        w = self.w
+        t = self.step if t is None else t
+        active = list(range(w.batch)) if active is None else list(active)
+        o_active = [b for b in active if b in self.oracle_seqs]
+        prev_tab = {(b, l): wnw.wnw_get_residency(self.h, b, l) for b in o_active for l in range(w.n_layers)
+                    if (w.roles[l] == ROLE_TIDAL).any()}
+        steps_before = {b: self._steps.get(b, 0) for b in active}
+        wnw.wnw_step_begin(self.h, active)
+        if o_active:
+            self.o.step_begin(o_active)
+        outs = []
+        for l in range(w.n_layers):
+            q = torch.stack([self._dec(b, l)["q"][t] for b in active]).to(self.dev)
+            kn = torch.stack([self._dec(b, l)["k_new"][t] for b in active]).to(self.dev) if append else None
+            vn = torch.stack([self._dec(b, l)["v_new"][t] for b in active]).to(self.dev) if append else None
+            out = torch.empty_like(q)
+            wnw.wnw_decode_layer(self.h, l, q, kn, vn, out)
+            outs.append((q, kn, vn, out))
+            if o_active:
+                idx = [active.index(b) for b in o_active]
+                qb = bf16_bits(q.cpu())[idx]
+                knb = bf16_bits(kn.cpu())[idx] if append else None
+                vnb = bf16_bits(vn.cpu())[idx] if append else None
+                ref = self.o.decode_layer(l, qb, knb, vnb)
+                got = bf16_bits_to_f64(bf16_bits(out.cpu()))[idx]
+                err = np.abs(got - ref).max()
+                self.max_out_err = max(self.max_out_err, float(err))
+                assert err <= OUT_TOL, f"attention output step {t} layer {l}: max abs err {err:.4f}"
+        wnw.wnw_step_end(self.h)
+        wnw.wnw_sync(self.h)
+        if o_active:
+            self.o.step_end()
+        for b in o_active:
+            T_a, _, C, S = self.o.dims(b)
+            if C == 0:
+                continue
+            lens = chunk_lens(T_a, w.chunk)
+            g_scores = {}
+            for l in range(w.n_layers):
+                if (w.roles[l] == ROLE_ANCHOR).any():
+                    g_scores[l] = wnw.wnw_get_chunk_scores(self.h, b, l)
+                    assert_scores_close(g_scores[l], self.o.chunk_scores(b, l), f"chunk scores step {t} b{b} l{l}")
+            for l in range(w.n_layers):
+                if not (w.roles[l] == ROLE_TIDAL).any():
+                    continue
+                src = self.o.score_source(l)
+                k = min(w.topk, S)
+                g_sel = wnw.wnw_get_selected(self.h, b, l)
+                g_tab, g_stamp = wnw.wnw_get_residency(self.h, b, l)
+                # (ii) oracle logic on GPU scores and the GPU's previous table
+                want_sel = wo.topk(g_scores[src], lens, k)
+                assert g_sel.tolist() == want_sel.tolist(), f"selection (ii) step {t} b{b} l{l}"
+                tab, stamp = prev_tab[(b, l)][0].copy(), prev_tab[(b, l)][1].copy()
+                plan, _ = wo.table_update(tab, stamp, want_sel, steps_before[b], w.topk)
+                n_tid = int((w.roles[l] == ROLE_TIDAL).sum())
+                self.expected_recall_bytes += len(plan) * n_tid * 2 * w.chunk * w.head_dim * 2
+                assert g_tab.tolist() == tab.tolist(), f"table (ii) step {t} b{b} l{l}"
+                assert g_stamp.tolist() == stamp.tolist(), f"stamps (ii) step {t} b{b} l{l}"
+                # (iii) oracle on its own scores
+                o_sel = self.o.selected(b, l)
+                o_tab, o_stamp = self.o.residency(b, l)
+                if o_sel.tolist() != g_sel.tolist() or o_tab.tolist() != g_tab.tolist() or o_stamp.tolist() != g_stamp.tolist():
+                    assert near_tie(self.o.chunk_scores(b, src), lens, g_sel.tolist(), o_sel.tolist()), \
+                        f"selection differs beyond a near-tie, step {t} b{b} l{l}: gpu {g_sel} oracle {o_sel}"
+                    self.near_ties += 1
+                    self.o.set_residency(b, l, g_tab, g_stamp)
+                if check_slots:
+                    self.check_slot_bytes(b, l)
+        for b in active:
+            self._steps[b] = steps_before[b] + 1
+        self.step = t + 1
+        return outs
+
+    def check_stats(self):
+        """Hit/miss/eviction counters agree with the oracle's when the oracle follows every sequence."""
+        if sorted(self.oracle_seqs) != list(range(self.w.batch)) or self.near_ties:
+            return
+        g = wnw.wnw_get_stats(self.h)
+        o = {"hits": 0, "misses": 0, "evictions": 0}
+        for b in range(self.w.batch):
+            s = self.o.stats(b)
+            for k in o:
+                o[k] += s[k]
+        assert (g["hits"], g["misses"], g["evictions"]) == (o["hits"], o["misses"], o["evictions"])
+        assert g["recall_bytes"] == self.expected_recall_bytes
