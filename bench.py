@@ -1,0 +1,492 @@
+#!/usr/bin/env python
+"""Benchmark of the WnW decode hot path on B200.
+
+One "step" is one generated token: the whole hot path (text append, anchor attention with fused chunk scores,
+split merge, top-k selection, residency update, recall, tidal and fixed sparse attention) for every layer of the
+stack, through the C ABI.  Workload at one GPU: the 3B Voxtral-shaped stack of the configuration list (30 layers,
+32 q / 8 KV heads, head_dim 128, 3000 audio + 64 text tokens, chunk 64, 20 % audio budget, batch 1), synthetic
+seeded inputs.  With N GPUs every rank serves its own sequence (no data-path collective): weak scaling.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1|cfg3]
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from workloads import ROLE_ANCHOR, ROLE_FIXED, ROLE_TIDAL, Synth, config1, config3
+from workloads.synth import bf16_bits
+
+METRIC = "wnw_decode_tokens_per_s_at_20pct_audio_budget"
+UNIT = "tokens/s"
+L2_FLUSH_BYTES = 512 << 20
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def make_workload(name: str, n_steps: int, seed: int):
+    if name == "cfg1":
+        w = config1(seed=0, n_steps=n_steps)
+    elif name == "cfg3":
+        w = config3(seed=0, n_steps=n_steps)
+    else:
+        raise SystemExit(f"unknown workload {name}")
+    return w
+
+
+# ------------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.gpu)], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [x for x in sm if x > 0.5 * max(sm)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------- job state
+class Job:
+    """Caches, resident inputs and launch helpers of one rank."""
+
+    def __init__(self, w, seed, device, wnw):
+        self.w, self.dev, self.wnw = w, device, wnw
+        self.syn = Synth(w, seed=seed, device=str(device))
+        self.B = w.batch
+        self.caches = {}
+        L, n = w.n_layers, w.n_steps
+        # decode inputs resident in HBM: [step][layer][B][...] so one step is one contiguous slab
+        self.q = torch.empty((n, L, self.B, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=device)
+        self.kn = torch.empty((n, L, self.B, w.n_kv_heads, w.head_dim), dtype=torch.bfloat16, device=device)
+        self.vn = torch.empty_like(self.kn)
+        for b in range(self.B):
+            for l in range(L):
+                d = self.syn.decode(b, l)
+                self.q[:, l, b] = d["q"]; self.kn[:, l, b] = d["k_new"]; self.vn[:, l, b] = d["v_new"]
+        self.out = torch.zeros((L, self.B, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=device)
+        self.flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+
+    def create(self, key, mode, recall_mode=0):
+        w, wnw = self.w, self.wnw
+        h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, self.B, max(w.audio_lens), w.text_capacity,
+                           w.chunk, w.budget, w.roles, topk=w.topk, device=self.dev.index or 0, mode=mode,
+                           recall_mode=recall_mode)
+        self.caches[key] = h
+        return h
+
+    def place_all(self, keys, keep_host=None):
+        """Generates each (seq, layer) prefill once on the device and places it into every cache in `keys`."""
+        w, wnw = self.w, self.wnw
+        for b in range(self.B):
+            for l in range(w.n_layers):
+                p = self.syn.prefill(b, l)
+                for key in keys:
+                    wnw.wnw_place_prefill(self.caches[key], b, l, p["k"], p["v"], p["audio_begin"], p["audio_end"], p["q_last"])
+                if keep_host is not None and keep_host(b, l):
+                    keep_host.store[(b, l)] = (bf16_bits(p["k"]), bf16_bits(p["v"]), bf16_bits(p["q_last"]), p["audio_begin"],
+                                               p["audio_end"])
+                torch.cuda.synchronize(self.dev)
+        for key in keys:
+            wnw.wnw_sync(self.caches[key])
+
+    def flush_l2(self):
+        self.flush_buf.fill_(1)
+
+    def step(self, key, t, full=False, q=None, kn=None, vn=None, out=None):
+        wnw, h = self.wnw, self.caches[key]
+        q = self.q[t] if q is None else q
+        kn = self.kn[t] if kn is None else kn
+        vn = self.vn[t] if vn is None else vn
+        out = self.out if out is None else out
+        fn = wnw.wnw_decode_layer_full if full else wnw.wnw_decode_layer
+        wnw.wnw_step_begin(h, list(range(self.B)))
+        for l in range(self.w.n_layers):
+            fn(h, l, q[l], kn[l], vn[l], out[l])
+        wnw.wnw_step_end(h)
+
+    def timed_steps(self, key, t0, n, full=False, flush=True):
+        """Device time of n consecutive steps, L2 flushed (untimed) before each.  Returns per-step ms."""
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for i in range(n):
+            if flush:
+                self.flush_l2()
+            evs[i][0].record()
+            self.step(key, t0 + i, full=full)
+            evs[i][1].record()
+        torch.cuda.synchronize(self.dev)
+        return [a.elapsed_time(b) for a, b in evs]
+
+    def kv_bytes_of_step(self, key, full=False):
+        """Algorithmic K,V bytes one step reads: 4*d bytes per (KV head, visible token), summed over layers; from the
+        residency tables as they stand (the tables the next step's attention will use)."""
+        w, wnw, h = self.w, self.wnw, self.caches[key]
+        total = 0
+        per_layer = []
+        for l in range(w.n_layers):
+            lb = 0
+            for b in range(self.B):
+                T_a, T_t, C, S = wnw.wnw_get_seq_dims(h, b)
+                T_t += 1  # the appended token is visible to its own step
+                clen = lambda c: min(w.chunk, T_a - c * w.chunk)
+                if full:
+                    tok = w.n_kv_heads * (T_t + T_a)
+                else:
+                    roles = w.roles[l]
+                    tok = int((roles == ROLE_ANCHOR).sum()) * (T_t + T_a)
+                    n_tid = int((roles == ROLE_TIDAL).sum())
+                    if n_tid:
+                        tab, _ = wnw.wnw_get_residency(h, b, l)
+                        tok += n_tid * (T_t + sum(clen(c) for c in tab.tolist() if c >= 0))
+                    for hh in np.nonzero(roles == ROLE_FIXED)[0]:
+                        tok += T_t + sum(clen(c) for c in wnw.wnw_get_fixed_set(h, b, l, int(hh)).tolist())
+                lb += tok * 4 * w.head_dim
+            per_layer.append(lb)
+            total += lb
+        return total, per_layer
+
+    def destroy(self):
+        for h in self.caches.values():
+            self.wnw.wnw_destroy(h)
+        self.caches.clear()
+
+
+# ------------------------------------------------------------------------------------------------- oracle timing
+def time_oracle(w, store, syn_dec, n_layers_sample, n_steps, warm, seqs):
+    """Times the CPU oracle, as it stands, on the first `n_layers_sample` layers of the workload for `n_steps` decode
+    steps of the sequences in `seqs`; returns (seconds per sampled step, threads)."""
+    from oracle.wnw_oracle import Oracle
+    threads = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    Ls = n_layers_sample
+    o = Oracle(Ls, w.n_q_heads, w.n_kv_heads, w.head_dim, len(seqs), max(w.audio_lens), w.text_capacity, w.chunk, w.topk,
+               w.budget, w.roles[:Ls])
+    for i, b in enumerate(seqs):
+        for l in range(Ls):
+            kb, vb, qb, ab, ae = store[(b, l)]
+            o.place_prefill(i, l, kb, vb, ab, ae, qb)
+    times = []
+    for t in range(warm + n_steps):
+        t0 = time.perf_counter()
+        o.step_begin(list(range(len(seqs))))
+        for l in range(Ls):
+            q, kn, vn = syn_dec(t, l, seqs)
+            o.decode_layer(l, q, kn, vn)
+        o.step_end()
+        if t >= warm:
+            times.append(time.perf_counter() - t0)
+    o.close()
+    return sum(times) / len(times), threads
+
+
+# ------------------------------------------------------------------------------------------------- main arms
+def run_reference(args, rank, world):
+    """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    total = args.steps + args.warmup
+    w = make_workload(args.workload, max(total, 1), 0)
+    syn = Synth(w, seed=0, device="cpu")
+    threads = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    # bound the run: sample the first Ls layers of sequence 0 so that (K+W) steps stay within about two minutes
+    probe_layers = 1
+    store = {}
+    for l in range(probe_layers):
+        p = syn.prefill(0, l)
+        store[(0, l)] = (bf16_bits(p["k"]), bf16_bits(p["v"]), bf16_bits(p["q_last"]), p["audio_begin"], p["audio_end"])
+    dec = {}
+
+    def syn_dec(t, l, seqs):
+        if l not in dec:
+            d = syn.decode(0, l)
+            dec[l] = (bf16_bits(d["q"]), bf16_bits(d["k_new"]), bf16_bits(d["v_new"]))
+        q, kn, vn = dec[l]
+        return q[t][None], kn[t][None], vn[t][None]
+
+    per_layer_s, _ = time_oracle(w, store, syn_dec, 1, 2, 1, [0])
+    budget_s = 120.0
+    Ls = int(max(1, min(w.n_layers, budget_s / max(per_layer_s * total, 1e-9))))
+    for l in range(probe_layers, Ls):
+        p = syn.prefill(0, l)
+        store[(0, l)] = (bf16_bits(p["k"]), bf16_bits(p["v"]), bf16_bits(p["q_last"]), p["audio_begin"], p["audio_end"])
+    sec, threads = time_oracle(w, store, syn_dec, Ls, args.steps, args.warmup, [0])
+    ms_step = sec * (w.n_layers / Ls) * w.batch * 1e3
+    value = w.batch / (ms_step * 1e-3)
+    sample = (f"sequence 0, first {Ls} of {w.n_layers} layers, {args.steps} decode steps; time scaled by "
+              f"{w.n_layers}/{Ls} layers and x{w.batch} sequences")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": workload_config(w),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w):
+    return {"workload": w.name, "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads,
+            "head_dim": w.head_dim, "batch": w.batch, "audio_tokens": w.audio_lens if w.batch <= 4 else
+            {"min": min(w.audio_lens), "max": max(w.audio_lens), "mean": sum(w.audio_lens) / w.batch},
+            "text_tokens": w.n_text, "chunk": w.chunk, "audio_budget": w.budget, "topk": w.topk,
+            "l2": f"flushed between steps ({L2_FLUSH_BYTES >> 20} MiB write, untimed)"}
+
+
+def run_ours(args, rank, world, local_rank):
+    import paper_2608_22704_b200 as wnw
+    wnw.lib()  # fails loudly if the CUDA library is missing
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+    peak_gbs, peak_kind = load_peaks()
+    K, W = args.steps, args.warmup
+    R = args.roofline_steps
+    total = W + R + K
+    w = make_workload(args.workload, total, 0)
+    job = Job(w, seed=rank, device=dev, wnw=wnw)
+    job.create("wnw", wnw.WNW_MODE_TIERED)
+    job.create("full", wnw.WNW_MODE_FULL)
+    job.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
+
+    class Keep:
+        store = {}
+
+        def __call__(self, b, l):
+            return rank == 0 and b == 0 and l < args.oracle_layers
+    keep = Keep()
+    job.place_all(["wnw", "full", "skip"], keep_host=keep)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize(dev)
+
+    # ---- warm-up (all three caches take the same steps so their states stay comparable)
+    for t in range(W):
+        for key, full in (("wnw", False), ("full", True), ("skip", False)):
+            job.step(key, t, full=full)
+    torch.cuda.synchronize(dev)
+
+    # ---- roofline pass: attention-kernel launches bracketed by CUDA events inside the library
+    wnw.wnw_set_kernel_timing(job.caches["wnw"], True)
+    wnw.wnw_set_kernel_timing(job.caches["full"], True)
+    algo_bytes = algo_bytes_full = 0
+    for t in range(W, W + R):
+        b_step, _ = job.kv_bytes_of_step("wnw")
+        bf_step, _ = job.kv_bytes_of_step("full", full=True)
+        algo_bytes += b_step; algo_bytes_full += bf_step
+        job.flush_l2(); job.step("wnw", t)
+        job.flush_l2(); job.step("full", t, full=True)
+        job.step("skip", t)
+    attn_ms, attn_n = wnw.wnw_get_kernel_time(job.caches["wnw"])
+    full_ms, full_n = wnw.wnw_get_kernel_time(job.caches["full"])
+    wnw.wnw_set_kernel_timing(job.caches["wnw"], False)
+    wnw.wnw_set_kernel_timing(job.caches["full"], False)
+
+    # ---- headline: K steps, device time, L2 flushed between steps, clocks sampled
+    stats0 = wnw.wnw_get_stats(job.caches["wnw"])
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    barrier()
+    sampler.start()
+    wall0 = time.perf_counter()
+    per_step = job.timed_steps("wnw", W + R, K)
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop()
+    stats1 = wnw.wnw_get_stats(job.caches["wnw"])
+    ms_total = sum(per_step)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    ms_per_step = float(t.item()) / K
+    value = world * w.batch / (ms_per_step * 1e-3)
+
+    # ---- comparison: own full-cache kernel, and WnW with recall copies skipped (exposed recall time)
+    full_steps = job.timed_steps("full", W + R, K, full=True)
+    skip_steps = job.timed_steps("skip", W + R, K)
+    barrier()
+
+    # ---- end to end: inputs start in pinned host memory, outputs end there, copies inside the timed region
+    n_e2e = min(K, 64)
+    hq = job.q[W + R:W + R + n_e2e].cpu().pin_memory(); hkn = job.kn[W + R:W + R + n_e2e].cpu().pin_memory()
+    hvn = job.vn[W + R:W + R + n_e2e].cpu().pin_memory()
+    hout = torch.empty((n_e2e,) + tuple(job.out.shape), dtype=torch.bfloat16).pin_memory()
+    job.create("e2e", wnw.WNW_MODE_TIERED)
+    job.place_all(["e2e"])
+    for tt in range(W + R):
+        job.step("e2e", tt)
+    dq = torch.empty_like(job.q[0]); dkn = torch.empty_like(job.kn[0]); dvn = torch.empty_like(job.vn[0])
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_ms = 0.0
+    for i in range(n_e2e):
+        job.flush_l2()
+        e0.record()
+        dq.copy_(hq[i], non_blocking=True); dkn.copy_(hkn[i], non_blocking=True); dvn.copy_(hvn[i], non_blocking=True)
+        job.step("e2e", W + R + i, q=dq, kn=dkn, vn=dvn)
+        hout[i].copy_(job.out, non_blocking=True)
+        e1.record()
+        e1.synchronize()
+        e2e_ms += e0.elapsed_time(e1)
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    e2e_value = world * w.batch / (float(t.item()) / n_e2e * 1e-3)
+    h2d = (dq.numel() + dkn.numel() + dvn.numel()) * 2
+    d2h = job.out.numel() * 2
+
+    if rank != 0:
+        job.destroy()
+        return
+
+    # ---- host link
+    try:
+        link_copy, link_kernel = wnw.wnw_measure_host_link(dev.index or 0, 256 << 20, 5)
+    except Exception:
+        link_copy = link_kernel = None
+
+    # ---- CPU baseline: the oracle on a bounded sample
+    cpu = None
+    if args.oracle_layers > 0:
+        dec_host = {}
+
+        def syn_dec(tt, l, seqs):
+            if l not in dec_host:
+                dec_host[l] = (bf16_bits(job.q[:, l, 0].cpu()), bf16_bits(job.kn[:, l, 0].cpu()), bf16_bits(job.vn[:, l, 0].cpu()))
+            q, kn, vn = dec_host[l]
+            return q[tt][None], kn[tt][None], vn[tt][None]
+        Ls = args.oracle_layers
+        sec, threads = time_oracle(w, keep.store, syn_dec, Ls, args.oracle_steps, 1, [0])
+        ms_oracle = sec * (w.n_layers / Ls) * w.batch * 1e3
+        cpu = {"value": w.batch / (ms_oracle * 1e-3), "unit": UNIT, "cores": threads, "kind": "oracle",
+               "ms_per_step": ms_oracle,
+               "sample": f"sequence 0, first {Ls} of {w.n_layers} layers, {args.oracle_steps} decode steps; time scaled by "
+                         f"{w.n_layers}/{Ls} layers and x{w.batch} sequences"}
+
+    attn_us = attn_ms * 1e3 / max(attn_n, 1)
+    bytes_per_launch = algo_bytes / max(attn_n, 1)
+    achieved = bytes_per_launch / (attn_us * 1e-6) / 1e9 if attn_us > 0 else 0.0
+    full_us = full_ms * 1e3 / max(full_n, 1)
+    full_achieved = (algo_bytes_full / max(full_n, 1)) / (full_us * 1e-6) / 1e9 if full_us > 0 else 0.0
+    n_upd_layers = int(sum(1 for l in range(w.n_layers) if (w.roles[l] == ROLE_TIDAL).any()))
+    launches_per_step = w.n_layers * 3 + n_upd_layers + 1  # append + attention + tail per layer, recall per tidal layer, step end
+    recall_bytes_step = (stats1["recall_bytes"] - stats0["recall_bytes"]) / K
+    ms_full = sum(full_steps) / K
+    ms_skip = sum(skip_steps) / K
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "attn_traffic.json")
+    if os.path.exists(tpath):
+        try:
+            traffic = json.load(open(tpath)).get(w.name)
+        except Exception:
+            traffic = None
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(w),
+        "clocks": clocks, "gpu_launches": launches_per_step * K,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e},
+        "roofline": {"bound": "hbm", "kernel": "wnw_attn_kernel", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
+                     "frac": achieved / peak_gbs, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                     "bytes_per_launch": bytes_per_launch, "us_per_launch": attn_us, "launches": attn_n},
+        "cpu_baseline": cpu,
+        "full_cache": {"ms_per_step": ms_full, "tokens_per_s": w.batch / (ms_full * 1e-3), "attn_us_per_launch": full_us,
+                       "attn_GBps": full_achieved, "attn_frac": full_achieved / peak_gbs,
+                       "wnw_step_over_full_step": ms_per_step / ms_full},
+        "recall": {"bytes_per_step": recall_bytes_step, "hits": stats1["hits"] - stats0["hits"],
+                   "misses": stats1["misses"] - stats0["misses"], "link_memcpy_GBps": link_copy, "link_kernel_GBps": link_kernel,
+                   "ms_per_step_copies_skipped": ms_skip, "exposed_us_per_step": (ms_per_step - ms_skip) * 1e3},
+        "retention": {"r_gpu": stats1["resident_audio_tokens"] / max(stats1["full_audio_tokens"], 1),
+                      "r_gpu_cpu": (stats1["resident_audio_tokens"] + stats1["host_audio_tokens"]) / max(stats1["full_audio_tokens"], 1)},
+        "wall_s_timed_region": wall,
+    }
+    print(json.dumps(line), flush=True)
+    job.destroy()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3"])
+    ap.add_argument("--roofline-steps", type=int, default=16)
+    ap.add_argument("--oracle-layers", type=int, default=6, help="layers of sequence 0 the CPU baseline samples (0 = skip)")
+    ap.add_argument("--oracle-steps", type=int, default=4)
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    try:
+        run_ours(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
