@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from workloads import ROLE_ANCHOR, ROLE_FIXED, ROLE_TIDAL, Synth, config1, config3
+from workloads import ROLE_ANCHOR, ROLE_FIXED, ROLE_TIDAL, Synth, config1, config3, config4
 from workloads.synth import bf16_bits
 
 METRIC = "wnw_decode_tokens_per_s_at_20pct_audio_budget"
@@ -50,6 +50,9 @@ def make_workload(name: str, n_steps: int, seed: int):
         w = config1(seed=0, n_steps=n_steps)
     elif name == "cfg3":
         w = config3(seed=0, n_steps=n_steps)
+    elif name == "prof":   # small many-sequence case for profiler captures: config-1 heads, 4 layers, 16 x 7500 audio tokens
+        w = config4(seed=0, budget=0.2, chunk=64, batch=16, n_steps=n_steps)
+        w.n_layers = 4; w.roles = w.roles[:4]; w.jump_every = 0; w.sweep_steps = 128; w.name = "prof_4layers_b16_7500"
     else:
         raise SystemExit(f"unknown workload {name}")
     return w
@@ -296,6 +299,18 @@ def run_ours(args, rank, world, local_rank):
     w = make_workload(args.workload, total, 0)
     job = Job(w, seed=rank, device=dev, wnw=wnw)
     job.create("wnw", wnw.WNW_MODE_TIERED)
+    if args.quick:   # profiler mode: the WnW steps only, nothing else launched
+        job.place_all(["wnw"])
+        for t in range(W):
+            job.step("wnw", t)
+        torch.cuda.synchronize(dev)
+        wnw.wnw_set_kernel_timing(job.caches["wnw"], True)
+        per_step = job.timed_steps("wnw", W, K, flush=not args.no_flush)
+        ms, n = wnw.wnw_get_kernel_time(job.caches["wnw"])
+        print(json.dumps({"quick": True, "workload": w.name, "ms_per_step": sum(per_step) / K, "steps": K,
+                          "attn_us_per_launch": ms * 1e3 / max(n, 1)}), flush=True)
+        job.destroy()
+        return
     job.create("full", wnw.WNW_MODE_FULL)
     job.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
 
@@ -465,7 +480,9 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3"])
+    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3", "prof"])
+    ap.add_argument("--quick", action="store_true", help="only the WnW steps (for profiler captures); prints a short line")
+    ap.add_argument("--no-flush", action="store_true", help="with --quick: do not flush L2 between steps")
     ap.add_argument("--roofline-steps", type=int, default=16)
     ap.add_argument("--oracle-layers", type=int, default=6, help="layers of sequence 0 the CPU baseline samples (0 = skip)")
     ap.add_argument("--oracle-steps", type=int, default=4)

@@ -11,14 +11,38 @@
 // memory and keeps a private online-softmax state; QK^T and PV run on mma.sync m16n8k16 with the g query
 // heads of the group padded to the 16 rows of the tile (bf16 in, fp32 accumulate).  Warps merge through
 // shared memory and the CTA writes one (m, l, o[g][d]) partial.
+//
+// The same launch also does the rest of the layer's step, with no further kernel and no host round trip:
+//   - the warp that owns the text granule of the token being generated reads that row from k_new/v_new and
+//     stores it into the text region (generated tokens are kept in full);
+//   - the CTA that finishes a head last merges the head's split partials into bf16 outputs (log-sum-exp) and
+//     publishes the head's final (max, denominator), which the selection kernel needs for the chunk scores.
+// Chunk scoring, selection and recall are not needed by whatever consumes the attention output next, so they run
+// in wnw_select_kernel / wnw_recall_kernel on a side stream (wnw_kernels.cu), off the critical path.
 #include "wnw_internal.cuh"
+#include "wnw_tail.cuh"
 
 namespace wnw {
 
-constexpr int NW = 4;      // warps per CTA
+constexpr int NW = 8;      // warps per CTA
 constexpr int NSTAGE = 3;  // granules in flight per warp
 
 int attn_warps() { return NW; }
+
+// Phase stamps for latency studies: compiled in only with -DWNW_PHASE_STAMPS (never in the product build).
+#ifdef WNW_PHASE_STAMPS
+__device__ long long g_stamps[8192 * 16];
+#define STAMP(k) do { if (threadIdx.x == 0 && blockIdx.x < 8192) g_stamps[blockIdx.x * 16 + (k)] = clock64(); } while (0)
+extern "C" int wnw_debug_read_stamps(long long *host, int n_ctas) {
+  return (int)cudaMemcpyFromSymbol(host, g_stamps, sizeof(long long) * 16 * n_ctas);
+}
+extern "C" int wnw_debug_clear_stamps() {
+  static long long zeros[8192 * 16];
+  return (int)cudaMemcpyToSymbol(g_stamps, zeros, sizeof(zeros));
+}
+#else
+#define STAMP(k) do { } while (0)
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes) {
@@ -53,7 +77,7 @@ struct GranDesc {
 
 // Maps granule j of a head's virtual key space [text capacity | audio] to memory.
 __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const AttnArgs &a, const LayerInfo &li, int b, int h,
-                                                   int role, int ridx, int j, int T_t, int T_a, int S_b) {
+                                                   int role, int ridx, int j, int T_t, int T_a) {
   const Geometry &G = cv.geo;
   GranDesc r;
   r.k = cv.text; r.valid = 0; r.score_idx = -1;
@@ -72,7 +96,6 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
     base = a.anchor_base + anchor_off(G, a.anchor_seq_stride, b, a.anchor_head0 + ridx, 0);
     store_row = ci * G.nc + off;
   } else if (role == ROLE_TIDAL) {
-    if (ci >= S_b) return r;
     c = cv.slot_chunk[((long long)b * G.L + a.layer) * G.S_max + ci];
     base = cv.pool + pool_off(G, li, b, ci, ridx, 0);
     store_row = off;
@@ -105,16 +128,13 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   constexpr int NQ = G16 ? 4 : 2;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr size_t SMEM_TOTAL = (size_t)NW * NSTAGE * 2 * GR * D * 2;
+  STAMP(0);
   const WorkItem it = a.items[blockIdx.x];
-  const int b = a.active[it.i];
+  const int b = it.b, role = it.role, ridx = it.ridx, T_a = it.T_a;
   const int g = G.g;
-  const LayerInfo li = cv.layers[a.layer];
-  int role = ROLE_ANCHOR, ridx = it.h;
-  if (a.mode == ATTN_DECODE) {
-    role = cv.roles[a.layer * G.Hkv + it.h];
-    ridx = cv.role_idx[a.layer * G.Hkv + it.h];
-  }
-  const int T_t = cv.text_len[b] + a.has_new, T_a = cv.T_a[b], S_b = cv.S[b];
+  const LayerInfo &li = a.li;
+  const int T_t = cv.text_len[b] + a.has_new;
   long long v_delta_audio;
   if (role == ROLE_ANCHOR) v_delta_audio = (long long)G.T_a_pad * G.d;
   else if (role == ROLE_TIDAL) v_delta_audio = (long long)G.nc * G.d;
@@ -156,7 +176,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     if (n < n_my) {
       if ((n & 31) == 0) {
         const int nn = n + lane;
-        if (nn < n_my) blk = decode_granule(cv, a, li, b, it.h, role, ridx, first + nn * NW, T_t, T_a, S_b);
+        if (nn < n_my) blk = decode_granule(cv, a, li, b, it.h, role, ridx, first + nn * NW, T_t, T_a);
         else { blk.valid = 0; blk.score_idx = -1; }
       }
       const int src_lane = n & 31;
@@ -167,8 +187,11 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       if (lane == 0) ring[warp][stage] = make_int2(valid, sidx);
       if (valid > 0) {
         const bf16 *k = reinterpret_cast<const bf16 *>(kp);
-        const bool is_text = first + n * NW < G.n_tg;
+        const int j = first + n * NW;
+        const bool is_text = j < G.n_tg;
         const bf16 *v = k + (is_text ? v_delta_text : v_delta_audio);
+        // the row of the token being generated comes from k_new/v_new and is stored into the text region here
+        const int new_row = (is_text && a.has_new) ? (T_t - 1) - j * GR : -1;
         const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB;
 #pragma unroll
         for (int x = 0; x < GR * PPR / 32; ++x) {
@@ -176,8 +199,16 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
           const int ok = row < valid;
           const int src_row = ok ? row : 0;
           const uint32_t dst = row * ROWB + ((pc ^ (row & 7)) << 4);
-          cp_async16(sK + dst, k + (long long)src_row * D + pc * 8, ok ? 16 : 0);
-          cp_async16(sV + dst, v + (long long)src_row * D + pc * 8, ok ? 16 : 0);
+          const bf16 *ks = k + (long long)src_row * D + pc * 8, *vs = v + (long long)src_row * D + pc * 8;
+          if (row == new_row) {
+            const long long noff = ((long long)it.i * G.Hkv + it.h) * D + pc * 8;
+            const uint4 kn = *reinterpret_cast<const uint4 *>(a.k_new + noff), vn = *reinterpret_cast<const uint4 *>(a.v_new + noff);
+            *reinterpret_cast<uint4 *>(const_cast<bf16 *>(ks)) = kn;
+            *reinterpret_cast<uint4 *>(const_cast<bf16 *>(vs)) = vn;
+            ks = a.k_new + noff; vs = a.v_new + noff;
+          }
+          cp_async16(sK + dst, ks, ok ? 16 : 0);
+          cp_async16(sV + dst, vs, ok ? 16 : 0);
         }
       }
     }
@@ -186,6 +217,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 
 #pragma unroll
   for (int n = 0; n < NSTAGE - 1; ++n) issue(n);
+  STAMP(1);
 
   for (int n = 0; n < n_my; ++n) {
     cp_async_wait<NSTAGE - 2>();
@@ -275,6 +307,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   }
   cp_async_wait<0>();
   __syncthreads();
+  STAMP(2);
 
   // ---- merge the warps' partial states through shared memory ----
   float2 *red_ml = reinterpret_cast<float2 *>(smem);                           // [NW][16]
@@ -308,6 +341,74 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     a.part_o[((long long)blockIdx.x * g + row) * D + col] = acc;
     if (col == 0) a.part_ml[(long long)blockIdx.x * g + row] = make_float2(M, L);
   }
+  STAMP(3);
+  if (a.mode == ATTN_PREFILL || a.debug_stop == 1) return;
+
+  // ---- the CTA that finishes this head last merges its split partials ----
+  __shared__ int s_flag;
+  const HeadItems hi = a.head_items[it.i * G.Hkv + it.h];
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int *ctr = a.head_done + it.i * G.Hkv + it.h;
+    const int prev = atomicAdd(ctr, 1);
+    s_flag = prev == hi.count - 1;
+    if (s_flag) *ctr = 0;
+  }
+  __syncthreads();
+  STAMP(4);
+  if (!s_flag) return;
+  __threadfence();
+  constexpr int NT = NW * 32;
+  {
+    // Each thread owns four output columns of one query head.  The partials of up to MB splits are fetched in one
+    // batch of independent loads (one L2 round trip); longer heads continue with an online log-sum-exp merge.
+    constexpr int MB = 16;
+    const int nvec = g * D / 4;
+    const float4 *po = reinterpret_cast<const float4 *>(a.part_o + (long long)hi.first * g * D);
+    const float2 *pml = a.part_ml + (long long)hi.first * g;
+    bf16 *ob = a.out + ((long long)it.i * G.Hq + (long long)it.h * g) * D;
+    for (int v = threadIdx.x; v < nvec; v += NT) {
+      const int row = v * 4 / D;
+      float M = -INFINITY, Z = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int n0 = 0; n0 < hi.count; n0 += MB) {
+        float2 ml[MB];
+        float4 x[MB];
+#pragma unroll
+        for (int j = 0; j < MB; ++j) {
+          if (n0 + j < hi.count) {
+            ml[j] = __ldcg(pml + (long long)(n0 + j) * g + row);
+            x[j] = __ldcg(po + (long long)(n0 + j) * nvec + v);
+          } else {
+            ml[j] = make_float2(-INFINITY, 0.f);
+            x[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
+        float Mb = M;
+#pragma unroll
+        for (int j = 0; j < MB; ++j) Mb = fmaxf(Mb, ml[j].x);
+        if (Mb > -INFINITY) {
+          const float sc0 = exp2f(M - Mb);  // M = -inf on the first batch -> 0
+          acc.x *= sc0; acc.y *= sc0; acc.z *= sc0; acc.w *= sc0; Z *= sc0;
+#pragma unroll
+          for (int j = 0; j < MB; ++j) {
+            const float w = exp2f(ml[j].x - Mb);  // empty split: m = -inf -> 0
+            acc.x += x[j].x * w; acc.y += x[j].y * w; acc.z += x[j].z * w; acc.w += x[j].w * w;
+            Z += ml[j].y * w;
+          }
+          M = Mb;
+        }
+      }
+      const float inv = Z > 0.f ? 1.f / Z : 0.f;
+      uint2 packed;
+      packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+      packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+      *reinterpret_cast<uint2 *>(ob + v * 4) = packed;
+      if (v % (D / 4) == 0) a.head_mz[(long long)it.i * G.Hq + it.h * g + row] = make_float2(M, Z);
+    }
+  }
+  STAMP(5);
 }
 
 template <int D, bool G16>

@@ -12,6 +12,8 @@ typedef __nv_bfloat16 bf16;
 constexpr int GR = 16;        // tokens per granule: one mma k16/n16 tile, the unit of loading and of score partials
 constexpr int MAX_TOPK = 8;   // upper bound on config topk
 constexpr int MAX_G = 16;     // query heads per KV head handled by one m16 tile
+constexpr int MAX_AQ = 128;   // anchor query heads of one layer
+constexpr int MAX_UPD_BY_VALUE = 8;  // update-list entries carried in kernel parameters; longer lists read the rest from memory
 
 constexpr int ROLE_ANCHOR = 0, ROLE_TIDAL = 1, ROLE_FIXED = 2;
 
@@ -20,10 +22,15 @@ constexpr int STATUS_NO_VICTIM = 1;     // table update found no evictable slot
 constexpr int STATUS_BAD_TABLE = 2;     // slot/chunk id out of range
 constexpr int STATUS_NONFINITE = 4;     // non-finite chunk score
 
-struct WorkItem {  // one CTA of the attention kernel
+struct WorkItem {  // one CTA of the attention kernel; everything static about it is precomputed on the host
   int32_t i;       // index into the active-sequence list
   int32_t h;       // KV head
   int32_t g0, g1;  // granule range in the head's virtual key space [text capacity | audio]
+  int32_t b;       // sequence id
+  int32_t role;    // ROLE_* the head plays in this launch
+  int32_t ridx;    // index among the heads of that role (anchor-like launches: the KV head)
+  int32_t T_a;     // audio tokens of the sequence
+  int32_t C, S;    // chunks and slots of the sequence
 };
 struct HeadItems { int32_t first, count; };  // work items of one (active seq, KV head)
 
@@ -86,48 +93,59 @@ __host__ __device__ inline long long mirror_off(const Geometry &G, const LayerIn
   return (((long long)C_b * li.tid_prefix + (long long)c * li.n_tidal + t_idx) * 2 + kv) * G.nc * G.d;
 }
 
+// shared-memory workspace of one table update in the selection kernel: keys[C] u64, stamp[S] i64, slot[S] i32, scores[C] f32
+__host__ __device__ inline size_t select_ws_bytes(int C, int S) {
+  return ((size_t)C * 8 + (size_t)S * 8 + (size_t)S * 4 + (size_t)C * 4 + 15) / 16 * 16;
+}
+
 // ---- attention launch ----
 enum { ATTN_DECODE = 0, ATTN_FULL = 1, ATTN_PREFILL = 2 };
 
 struct AttnArgs {
   int32_t mode;          // ATTN_*
   int32_t layer;
+  LayerInfo li;          // cv.layers[layer], by value (no global load on the critical path)
   int32_t n_active;
-  int32_t has_new;       // the text region holds one more row than text_len says
+  int32_t has_new;       // k_new/v_new hold one more text row per sequence (appended by this launch)
   int32_t score_on;      // write per-granule softmax-mass partials for anchor-like heads
+  int32_t debug_stop;    // timing experiments only: 1 = return after the split partials, 2 = after the head merge
   const int32_t *active; // [n_active] sequence ids
   const WorkItem *items;
   int32_t n_items;
+  const HeadItems *head_items;  // [n_active][Hkv] work items of each head (first is relative to `items`)
   const bf16 *q;         // [n_active][Hq][d]
+  const bf16 *k_new, *v_new;    // [n_active][Hkv][d] or null
   // anchor-like source: decode -> cache anchor store; full -> same store, head = l*Hkv+h; prefill -> staging, head = h
   const bf16 *anchor_base;
   long long anchor_seq_stride;
   int32_t anchor_head0;
-  // outputs
+  // split partials
   float *part_o;         // [n_items][g][d]
   float2 *part_ml;       // [n_items][g]   (m in log2 units, l)
   float2 *gran_em;       // [n_active][n_aq][n_ag_max]  (sum of 2^(s-m) over the granule, m at that time)
   int32_t n_aq, n_ag_max;
+  // fused head merge (decode and full modes)
+  int32_t *head_done;    // [n_active][Hkv] finished-item counters (self-resetting)
+  float2 *head_mz;       // [n_active][Hq] final (M, Z) per query head
+  bf16 *out;             // [n_active][Hq][d]
 };
 
-struct TailArgs {
-  int32_t mode, layer, n_active, score_on;
+// Selection launch (side stream): chunk scores of `layer` from its granule partials, then top-k, residency update
+// and recall plan for every layer in the update list.  Static data travels by value.
+struct SelectArgs {
+  int32_t layer, n_active, score_on;
+  LayerInfo li;
   const int32_t *active;
-  const HeadItems *head_items;  // [n_active][Hkv]
-  const float *part_o;
-  const float2 *part_ml;
-  const float2 *gran_em;
+  const float2 *gran_em;   // this layer's [n_active][n_aq][n_ag_max]
+  const float2 *head_mz;   // this layer's [n_active][Hq]
   int32_t n_aq, n_ag_max;
-  float2 *head_mz;              // [n_active][Hq] final (M, Z) per query head
-  bf16 *out;                    // [n_active][Hq][d]
-  int32_t *seq_done;            // [n_active] completion counters (self-resetting)
+  uint8_t aq_head[MAX_AQ]; // query-head index of anchor q-head slot aq (score order)
+  int16_t upd_layer[MAX_UPD_BY_VALUE], upd_src[MAX_UPD_BY_VALUE];
 };
 
 // kernels' host launchers (defined in the .cu files)
 cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st);
-cudaError_t launch_tail(const CacheView &cv, const TailArgs &a, int max_count, cudaStream_t st);
-cudaError_t launch_append(const CacheView &cv, int layer, int n_active, const int32_t *active, const bf16 *k_new,
-                          const bf16 *v_new, cudaStream_t st);
+cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, cudaStream_t st);
 cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *active, int appended, cudaStream_t st);
 cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,
                           int skip_copy, cudaStream_t st);

@@ -1,233 +1,122 @@
-// Tail (split merge, chunk-score finalize, top-k, residency update, recall plan), recall, text append,
-// step bookkeeping and prefill placement kernels (sm_100a).
+// Recall, step bookkeeping and prefill placement kernels (sm_100a).
 #include "wnw_internal.cuh"
+#include "wnw_tail.cuh"
 
 namespace wnw {
 
-__device__ __forceinline__ int chunk_len(const Geometry &G, int T_a, int c) {
-  int len = T_a - c * G.nc;
-  return len > G.nc ? G.nc : len;
-}
-
-__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    unsigned long long w = __shfl_xor_sync(0xffffffffu, v, o);
-    v = w > v ? w : v;
-  }
-  return v;
-}
-__device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    unsigned long long w = __shfl_xor_sync(0xffffffffu, v, o);
-    v = w < v ? w : v;
-  }
-  return v;
-}
-
-// Ranking key of "Dynamic Chunk Selection": the chunk MEAN as fp32 (IEEE division), ties to the lower chunk
-// index.  Scores are >= 0, so the float's bit pattern orders like the value.
-__device__ __forceinline__ unsigned long long rank_key(float score_sum, int len, int c) {
-  const float key = __fdiv_rn(score_sum, (float)len);
-  return ((unsigned long long)__float_as_uint(key) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)c);
-}
-
-// One warp: top-k of layer `lt` of sequence b from the scores of its source layer, then the residency update
-// (hit: refresh stamp; miss: lowest free slot, else least recently selected resident not selected now) and the
-// recall plan.  The new table is read by attention from the next step on.
-__device__ void select_and_update(const CacheView &cv, int b, int lt, int lane) {
+// ------------------------------------------------------------------------------------------------
+// Selection (side stream): grid (n_active), one CTA per sequence.  "Decode-Step Score Aggregation" summed per
+// chunk, then "Dynamic Chunk Selection" for every layer whose score source is complete with this layer.
+// ------------------------------------------------------------------------------------------------
+constexpr int SEL_WARPS = 8;
+__global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid_constant__ CacheView cv,
+                                                                    const __grid_constant__ SelectArgs a, int smem_total) {
+  extern __shared__ __align__(16) unsigned char smem[];
   const Geometry &G = cv.geo;
-  const LayerInfo li = cv.layers[lt];
+  constexpr int NT = SEL_WARPS * 32;
+  const int i = blockIdx.x, b = a.active[i];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const LayerInfo &li = a.li;
+  // per-sequence scalars: one batch of independent loads
   const int C_b = cv.C[b], S_b = cv.S[b], T_a = cv.T_a[b];
-  const long long bl = (long long)b * G.L + lt;
-  int k = G.topk < S_b ? G.topk : S_b;
-  if (li.src < 0 || C_b <= 0) k = 0;
-  int sel[MAX_TOPK];
-  const float *sc = cv.score_sum + ((long long)b * G.L + li.src) * G.C_max;
-  unsigned long long prev = ~0ull;
-  for (int r = 0; r < k; ++r) {
-    unsigned long long best = 0ull;
-    for (int c = lane; c < C_b; c += 32) {
-      const float s = __ldcg(sc + c);
-      const unsigned long long key = rank_key(s, chunk_len(G, T_a, c), c);
-      if (key < prev && key > best) best = key;
-    }
-    best = warp_max_u64(best);
-    sel[r] = (int)(0xFFFFFFFFu - (unsigned)(best & 0xFFFFFFFFull));
-    prev = best;
+  const long long step_b = cv.steps[b];
+  const int n_aq = a.n_aq;
+  const bool scored = li.n_anchor > 0 && a.score_on && C_b > 0;
+  const int n_ag = (T_a + GR - 1) / GR;  // granules that hold audio
+  // shared-memory layout: (M,Z) of the anchor q-heads | this layer's scores | per-warp update workspaces | granule partials
+  float2 *mz_s = reinterpret_cast<float2 *>(smem);
+  float *sc_s = reinterpret_cast<float *>(smem + ((size_t)n_aq * 8 + 15) / 16 * 16);
+  unsigned char *ws0 = reinterpret_cast<unsigned char *>(sc_s) + ((size_t)C_b * 4 + 15) / 16 * 16;
+  const size_t ws_bytes = select_ws_bytes(C_b, S_b);
+  const int n_par = li.upd_count < SEL_WARPS ? li.upd_count : SEL_WARPS;
+  float2 *em_s = reinterpret_cast<float2 *>(ws0 + (size_t)n_par * ws_bytes);
+  const long long em_room = ((long long)smem_total - (long long)(reinterpret_cast<unsigned char *>(em_s) - smem)) / 8;
+  int tile_c = 0;
+  if (scored) {
+    tile_c = (int)(em_room / ((long long)n_aq * G.gpc));
+    if (tile_c > C_b) tile_c = C_b;
   }
-  int *slot_chunk = cv.slot_chunk + bl * G.S_max;
-  int *chunk_slot = cv.chunk_slot + bl * G.C_max;
-  long long *stamp = cv.stamp + bl * G.S_max;
-  int *plan = cv.plan + bl * G.topk * 2;
-  const long long step = cv.steps[b];
-  int n_plan = 0, hits = 0, evictions = 0;
-  for (int r = 0; r < k; ++r) {
-    const int c = sel[r];
-    const long long st = step * G.topk + (G.topk - 1 - r);
-    int j = chunk_slot[c];
-    if (j >= 0) {
-      if (lane == 0) stamp[j] = st;
-      ++hits;
-      __syncwarp();
-      continue;
-    }
-    // lowest-index free slot
-    unsigned long long cand = ~0ull;
-    for (int s = lane; s < S_b; s += 32)
-      if (slot_chunk[s] < 0) { cand = (unsigned long long)s; break; }
-    cand = warp_min_u64(cand);
-    if (cand != ~0ull) {
-      j = (int)cand;
-    } else {  // victim: smallest stamp among residents that are not selected now (stamps are unique)
-      unsigned long long mykey = ~0ull;
-      int myslot = -1;
-      for (int s = lane; s < S_b; s += 32) {
-        const int rc = slot_chunk[s];
-        bool in_sel = false;
-        for (int q = 0; q < k; ++q) in_sel |= sel[q] == rc;
-        if (in_sel) continue;
-        const unsigned long long key = (unsigned long long)(stamp[s] + (1ll << 62));  // order-preserving bias
-        if (key < mykey) { mykey = key; myslot = s; }
-      }
-      const unsigned long long best = warp_min_u64(mykey);
-      if (best == ~0ull) {
-        if (lane == 0) atomicOr(cv.status, STATUS_NO_VICTIM);
-        break;
-      }
-      const unsigned owner = __ballot_sync(0xffffffffu, mykey == best);
-      j = __shfl_sync(0xffffffffu, myslot, __ffs(owner) - 1);
-    }
-    __syncwarp();
-    if (lane == 0) {
-      const int old = slot_chunk[j];
-      if (old >= 0) { chunk_slot[old] = -1; ++evictions; }
-      slot_chunk[j] = c;
-      chunk_slot[c] = j;
-      stamp[j] = st;
-      plan[2 * n_plan] = c;
-      plan[2 * n_plan + 1] = j;
-    }
-    ++n_plan;
-    __syncwarp();
+  if (em_room < 0 || (scored && tile_c < 1)) {  // beyond what the host sized the launch for
+    if (threadIdx.x == 0) atomicOr(cv.status, STATUS_BAD_TABLE);
+    return;
   }
-  if (lane == 0) {
-    for (int r = 0; r < k; ++r) cv.sel[bl * G.topk + r] = sel[r];
-    cv.n_sel[bl] = k;
-    cv.n_plan[bl] = n_plan;
-    if (k > 0) {
-      atomicAdd(cv.stats + (long long)b * 4 + 0, (unsigned long long)hits);
-      atomicAdd(cv.stats + (long long)b * 4 + 1, (unsigned long long)n_plan);
-      atomicAdd(cv.stats + (long long)b * 4 + 2, (unsigned long long)evictions);
+  auto stage_em = [&](int c0, int c1) {
+    const int span = (c1 - c0) * G.gpc, ag0 = c0 * G.gpc;
+    for (int idx = threadIdx.x; idx < n_aq * span; idx += NT) {
+      const int aq = idx / span, ag = ag0 + (idx - aq * span);
+      if (ag < n_ag) cp_async_small(em_s + idx, a.gran_em + ((long long)i * n_aq + aq) * a.n_ag_max + ag, 8);
+      else em_s[idx] = make_float2(0.f, 0.f);
     }
+  };
+  auto upd_of = [&](int u, int &lt, int &src) {
+    if (u < MAX_UPD_BY_VALUE) { lt = a.upd_layer[u]; src = a.upd_src[u]; }
+    else { lt = cv.upd_list[li.upd_first + u]; src = cv.layers[lt].src; }
+  };
+  // one batch of copies: (M,Z), the first tile of granule partials, the tables of the first round of updates
+  if (scored) {
+    if (threadIdx.x < n_aq) cp_async_small(mz_s + threadIdx.x, a.head_mz + (long long)i * G.Hq + a.aq_head[threadIdx.x], 8);
+    stage_em(0, tile_c);
   }
-}
-
-// grid (Hkv, n_active).  Merges the split partials of one (sequence, KV head) into bf16 outputs; the CTA that
-// finishes a sequence last finalizes this layer's chunk scores and runs selection for every layer whose score
-// source is now complete.
-__global__ void __launch_bounds__(256) wnw_tail_kernel(const __grid_constant__ CacheView cv,
-                                                       const __grid_constant__ TailArgs a) {
-  extern __shared__ float sm_w[];  // [count][g] weights, then [count][g] l
-  __shared__ float sM[MAX_G], sZ[MAX_G];
-  __shared__ int s_last;
-  const Geometry &G = cv.geo;
-  const int h = blockIdx.x, i = blockIdx.y, b = a.active[i];
-  const int g = G.g, D = G.d, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const HeadItems hi = a.head_items[i * G.Hkv + h];
-  float *sm_l = sm_w + hi.count * g;
-  for (int idx = tid; idx < hi.count * g; idx += blockDim.x) {
-    const float2 ml = __ldcg(a.part_ml + (long long)hi.first * g + idx);
-    sm_w[idx] = ml.x;
-    sm_l[idx] = ml.y;
+  if (warp < n_par) {
+    int lt, src;
+    upd_of(warp, lt, src);
+    select_stage(cv, b, lt, src, scored && src == a.layer, C_b, S_b, lane, select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b));
   }
+  cp_async_commit_wait_all();
   __syncthreads();
-  for (int row = warp; row < g; row += 8) {
-    float M = -INFINITY;
-    for (int n = lane; n < hi.count; n += 32) M = fmaxf(M, sm_w[n * g + row]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    float Z = 0.f;
-    for (int n = lane; n < hi.count; n += 32) {
-      const float w = M > -INFINITY ? exp2f(sm_w[n * g + row] - M) : 0.f;
-      sm_w[n * g + row] = w;
-      Z += sm_l[n * g + row] * w;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, o);
-    if (lane == 0) {
-      sM[row] = M; sZ[row] = Z;
-      a.head_mz[(long long)i * G.Hq + h * g + row] = make_float2(M, Z);
-    }
-  }
-  __syncthreads();
-  if (a.out != nullptr) {
-    for (int idx = tid; idx < g * D; idx += blockDim.x) {
-      const int row = idx / D, col = idx - row * D;
-      float acc = 0.f;
-      const float *po = a.part_o + ((long long)hi.first * g + row) * D + col;
-      for (int n = 0; n < hi.count; ++n) acc += __ldcg(po + (long long)n * g * D) * sm_w[n * g + row];
-      const float Z = sZ[row];
-      a.out[((long long)i * G.Hq + h * g + row) * D + col] = __float2bfloat16_rn(Z > 0.f ? acc / Z : 0.f);
-    }
-  }
-  if (a.mode != ATTN_DECODE) return;
-
-  // ---- last CTA of this sequence: scores, selection, table update ----
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int prev = atomicAdd(a.seq_done + i, 1);
-    s_last = prev == G.Hkv - 1;
-    if (s_last) a.seq_done[i] = 0;
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  const LayerInfo li = cv.layers[a.layer];
-  const int C_b = cv.C[b], T_a = cv.T_a[b];
-  if (li.n_anchor > 0 && a.score_on) {
+  if (scored) {
+    // score_sum[c] = sum over anchor q-heads (head order) of (sum over the chunk's granules of e * 2^(m - M)) / Z
     float *dst = cv.score_sum + ((long long)b * G.L + a.layer) * G.C_max;
-    for (int c = tid; c < C_b; c += blockDim.x) {
-      float total = 0.f;
-      int aidx = 0;
-      for (int hh = 0; hh < G.Hkv; ++hh) {
-        if (cv.roles[a.layer * G.Hkv + hh] != ROLE_ANCHOR) continue;
-        for (int r = 0; r < g; ++r) {
-          const float2 mz = __ldcg(a.head_mz + (long long)i * G.Hq + hh * g + r);
-          const float2 *ge = a.gran_em + ((long long)i * a.n_aq + (long long)aidx * g + r) * a.n_ag_max + (long long)c * G.gpc;
+    for (int c0 = 0; c0 < C_b; c0 += tile_c) {
+      const int c1 = c0 + tile_c < C_b ? c0 + tile_c : C_b, span = (c1 - c0) * G.gpc;
+      if (c0 > 0) {
+        stage_em(c0, c1);
+        cp_async_commit_wait_all();
+        __syncthreads();
+      }
+      for (int c = c0 + threadIdx.x; c < c1; c += NT) {
+        float total = 0.f;
+        for (int aq = 0; aq < n_aq; ++aq) {
+          const float2 mz = mz_s[aq];
+          const float2 *p = em_s + (size_t)aq * span + (size_t)(c - c0) * G.gpc;
           float sum_h = 0.f;
-          for (int gi = 0; gi < G.gpc; ++gi) {
-            if (c * G.nc + gi * GR >= T_a) break;
-            const float2 em = __ldcg(ge + gi);
-            sum_h += em.x * exp2f(em.y - mz.x);
-          }
+          for (int gi = 0; gi < G.gpc; ++gi) sum_h += p[gi].x * exp2f(p[gi].y - mz.x);
           total += mz.y > 0.f ? sum_h / mz.y : 0.f;
         }
-        ++aidx;
+        if (!(total >= 0.f) || isinf(total)) atomicOr(cv.status, STATUS_NONFINITE);
+        dst[c] = total;
+        sc_s[c] = total;
       }
-      if (!(total >= 0.f) || isinf(total)) atomicOr(cv.status, STATUS_NONFINITE);
-      dst[c] = total;
+      __syncthreads();
     }
   }
-  __syncthreads();
-  for (int u = warp; u < li.upd_count; u += 8) select_and_update(cv, b, cv.upd_list[li.upd_first + u], lane);
+  if (warp < n_par) {
+    const SelectWs w = select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b);
+    for (int u = warp; u < li.upd_count; u += n_par) {
+      int lt, src;
+      upd_of(u, lt, src);
+      const bool local = scored && src == a.layer;
+      if (u >= n_par) {  // later rounds stage their own tables
+        __syncwarp();
+        select_stage(cv, b, lt, src, local, C_b, S_b, lane, w);
+        cp_async_commit_wait_all();
+        __syncwarp();
+      }
+      select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, local ? sc_s : w.sc, w);
+    }
+  }
 }
 
-// max_count: the largest number of work items of any (sequence, KV head) in this launch (sizes shared memory).
-cudaError_t launch_tail(const CacheView &cv, const TailArgs &a, int max_count, cudaStream_t st) {
-  const size_t smem = (size_t)max_count * cv.geo.g * 2 * sizeof(float);
-  if (smem > 200 * 1024) return cudaErrorInvalidValue;
-  if (smem > 48 * 1024) {
+cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, cudaStream_t st) {
+  if (smem_bytes > 48 * 1024) {
     static size_t configured = 0;
-    if (smem > configured) {
-      cudaError_t e = cudaFuncSetAttribute(wnw_tail_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (smem_bytes > configured) {
+      cudaError_t e = cudaFuncSetAttribute(wnw_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
       if (e != cudaSuccess) return e;
-      configured = smem;
+      configured = smem_bytes;
     }
   }
-  wnw_tail_kernel<<<dim3(cv.geo.Hkv, a.n_active), 256, smem, st>>>(cv, a);
+  wnw_select_kernel<<<a.n_active, SEL_WARPS * 32, smem_bytes, st>>>(cv, a, (int)smem_bytes);
   return cudaGetLastError();
 }
 
@@ -302,32 +191,8 @@ cudaError_t launch_copy_plan(const uint4 *src, uint4 *dst, long long n_vec, int 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Text append and step bookkeeping
+// Step bookkeeping
 // ------------------------------------------------------------------------------------------------
-__global__ void wnw_append_kernel(const __grid_constant__ CacheView cv, int layer, const int32_t *active, const bf16 *k_new,
-                                  const bf16 *v_new) {
-  const Geometry &G = cv.geo;
-  const int i = blockIdx.x, b = active[i];
-  const int row = cv.text_len[b];
-  if (row >= G.T_cap_pad) {
-    if (threadIdx.x == 0) atomicOr(cv.status, STATUS_BAD_TABLE);
-    return;
-  }
-  const int vec_per_head = G.d / 8;
-  for (int idx = threadIdx.x; idx < G.Hkv * vec_per_head * 2; idx += blockDim.x) {
-    const int kv = idx / (G.Hkv * vec_per_head), rem = idx - kv * G.Hkv * vec_per_head;
-    const int h = rem / vec_per_head, v = rem - h * vec_per_head;
-    const bf16 *src = (kv ? v_new : k_new) + ((long long)i * G.Hkv + h) * G.d + v * 8;
-    bf16 *dst = cv.text + text_off(G, b, layer, h, kv) + (long long)row * G.d + v * 8;
-    *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
-  }
-}
-cudaError_t launch_append(const CacheView &cv, int layer, int n_active, const int32_t *active, const bf16 *k_new,
-                          const bf16 *v_new, cudaStream_t st) {
-  wnw_append_kernel<<<n_active, 128, 0, st>>>(cv, layer, active, k_new, v_new);
-  return cudaGetLastError();
-}
-
 __global__ void wnw_step_end_kernel(const __grid_constant__ CacheView cv, int n_active, const int32_t *active, int appended) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_active) return;

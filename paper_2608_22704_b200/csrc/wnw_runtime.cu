@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -64,7 +65,7 @@ struct wnw_cache {
   WorkItem *d_items = nullptr;
   HeadItems *d_head_items = nullptr;
   size_t d_items_cap = 0, d_head_items_cap = 0;
-  int prefill_C = -1;
+  int prefill_seq = -1, prefill_T_a = -1;
   WorkItem *d_pf_items = nullptr;
   HeadItems *d_pf_head_items = nullptr;
   int pf_n_items = 0;
@@ -72,12 +73,17 @@ struct wnw_cache {
   // partial buffers
   float *part_o = nullptr;
   float2 *part_ml = nullptr, *gran_em = nullptr, *head_mz = nullptr;
-  int32_t *seq_done = nullptr;
+  int32_t *head_done = nullptr;
+  float2 *pf_gran_em = nullptr;
   int part_cap_items = 0, n_aq_max = 0, n_ag_max = 0;
   // streams / events
   cudaStream_t side = nullptr, last_stream = nullptr;
-  std::vector<cudaEvent_t> ev_layer_done, ev_recall_done;
-  std::vector<char> recall_recorded;
+  std::vector<cudaEvent_t> ev_layer_done, ev_side_done;
+  std::vector<char> side_recorded;
+  std::vector<size_t> sel_smem;   // dynamic shared memory of each layer's selection launch
+  size_t gran_em_layer_stride = 0;
+  bool step_capturing = false;
+  int last_side_layer = -1;
   cudaEvent_t ev_place = nullptr, ev_step = nullptr;
   bool place_recorded = false, step_recorded = false;
   // timing
@@ -128,7 +134,7 @@ static void destroy_impl(wnw_cache *c) {
     if (s.mirror) cudaFreeHost(s.mirror);
   if (c->side) cudaStreamDestroy(c->side);
   for (auto e : c->ev_layer_done) cudaEventDestroy(e);
-  for (auto e : c->ev_recall_done) cudaEventDestroy(e);
+  for (auto e : c->ev_side_done) cudaEventDestroy(e);
   if (c->ev_place) cudaEventDestroy(c->ev_place);
   if (c->ev_step) cudaEventDestroy(c->ev_step);
   for (auto &p : c->t_used) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
@@ -172,7 +178,7 @@ static wnw_status_t validate_config(const wnw_config_t *cfg) {
   if (cfg->mode == WNW_MODE_TIERED && any_tidal && !any_anchor) return WNW_ERR_INVALID_ARG;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return WNW_ERR_UNSUPPORTED;
   if (cfg->chunk_tokens % GR) return WNW_ERR_UNSUPPORTED;
-  if (cfg->n_q_heads / cfg->n_kv_heads > MAX_G) return WNW_ERR_UNSUPPORTED;
+  if (cfg->n_q_heads / cfg->n_kv_heads > MAX_G || cfg->n_q_heads > MAX_AQ || cfg->n_layers > 32767) return WNW_ERR_UNSUPPORTED;
   return WNW_OK;
 }
 
@@ -293,16 +299,31 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   c->part_cap_items = 2 * c->n_sm + (int)B * Hkv + 16;
   CKC(dev_alloc(c, &c->part_o, (size_t)c->part_cap_items * G.g * d, false));
   CKC(dev_alloc(c, &c->part_ml, (size_t)c->part_cap_items * G.g, false));
-  CKC(dev_alloc(c, &c->gran_em, std::max(B * (size_t)c->n_aq_max, (size_t)G.Hq) * c->n_ag_max, false));
-  CKC(dev_alloc(c, &c->head_mz, B * (size_t)G.Hq, false));
-  CKC(dev_alloc(c, &c->seq_done, B));
+  // granule partials and final (M,Z) are per layer: the side-stream selection of layer l reads them while the
+  // caller's stream already runs later layers
+  c->gran_em_layer_stride = B * (size_t)c->n_aq_max * c->n_ag_max;
+  CKC(dev_alloc(c, &c->gran_em, full ? 1 : (size_t)L * c->gran_em_layer_stride, false));
+  CKC(dev_alloc(c, &c->pf_gran_em, full ? 1 : (size_t)G.Hq * c->n_ag_max, false));
+  CKC(dev_alloc(c, &c->head_mz, (size_t)L * B * G.Hq, false));
+  c->sel_smem.assign(L, 0);
+  for (int l = 0; l < L && !full; ++l) {
+    const LayerInfo &li = c->layers[l];
+    const size_t n_aq_l = (size_t)std::max(li.n_anchor * G.g, 1);
+    const size_t fixed_part = (n_aq_l * 8 + 15) / 16 * 16 + ((size_t)G.C_max * 4 + 15) / 16 * 16 +
+                              (size_t)std::min(li.upd_count, 8) * select_ws_bytes(G.C_max, G.S_max);
+    const size_t per_chunk = li.n_anchor > 0 ? n_aq_l * G.gpc * 8 : 0;
+    const size_t cap = 200 * 1024;
+    if (fixed_part + per_chunk > cap) return fail(WNW_ERR_UNSUPPORTED);  // chunk tables too large for one CTA
+    c->sel_smem[l] = std::min(cap, fixed_part + per_chunk * std::max(G.C_max, 1)) + 16;
+  }
+  CKC(dev_alloc(c, &c->head_done, B * Hkv));
   c->seqs.assign(B, SeqHost{});
   c->mirror_ptrs.assign(B, nullptr);
   CKE(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
-  c->ev_layer_done.resize(L); c->ev_recall_done.resize(L); c->recall_recorded.assign(L, 0);
+  c->ev_layer_done.resize(L); c->ev_side_done.resize(L); c->side_recorded.assign(L, 0);
   for (int l = 0; l < L; ++l) {
     CKE(cudaEventCreateWithFlags(&c->ev_layer_done[l], cudaEventDisableTiming));
-    CKE(cudaEventCreateWithFlags(&c->ev_recall_done[l], cudaEventDisableTiming));
+    CKE(cudaEventCreateWithFlags(&c->ev_side_done[l], cudaEventDisableTiming));
   }
   CKE(cudaEventCreateWithFlags(&c->ev_place, cudaEventDisableTiming));
   CKE(cudaEventCreateWithFlags(&c->ev_step, cudaEventDisableTiming));
@@ -322,12 +343,17 @@ extern "C" wnw_status_t wnw_destroy(wnw_cache_t *c) {
 // ---------------------------------------------------------------------------------------------
 // Work lists: split every (sequence, KV head) granule space into CTA-sized items
 // ---------------------------------------------------------------------------------------------
-static int granules_per_item(const wnw_cache *c, long long total_granules) {
+// Granules per work item: enough items to fill the machine twice over, but never shorter than `min_gpi`
+// granules, because every item costs one partial in the merge that follows.
+static int granules_per_item(const wnw_cache *c, long long total_granules, int longest_head) {
   const int nw = attn_warps();
+  int min_gpi = nw;
+  if (const char *e = getenv("WNW_MIN_GRANULES_PER_ITEM")) min_gpi = std::max(nw, atoi(e) / nw * nw);
   const long long target = 2ll * c->n_sm;
   long long per = (total_granules + target - 1) / target;
+  per = std::max<long long>(per, (longest_head + 31) / 32);  // at most ~32 splits per head: the merge reads every split
   per = (per + nw - 1) / nw * nw;
-  return (int)std::max<long long>(per, nw);
+  return (int)std::max<long long>(per, min_gpi);
 }
 
 // Appends the items of one layer for the given sequences.  audio_granules(role, b) gives each head's audio part.
@@ -336,6 +362,7 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   const Geometry &G = c->geo;
   std::vector<int> n_gran(seq_ids.size() * G.Hkv);
   long long total = 0;
+  int longest = 0;
   for (size_t i = 0; i < seq_ids.size(); ++i) {
     const SeqHost &s = c->seqs[seq_ids[i]];
     for (int h = 0; h < G.Hkv; ++h) {
@@ -343,9 +370,10 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       const int audio = (role == ROLE_ANCHOR ? s.C : s.S) * G.gpc;
       n_gran[i * G.Hkv + h] = G.n_tg + audio;
       total += G.n_tg + audio;
+      longest = std::max(longest, G.n_tg + audio);
     }
   }
-  const int gpi = granules_per_item(c, total);
+  const int gpi = granules_per_item(c, total, longest);
   lw.first_item = (int)items.size();
   lw.head_items_off = (int)heads.size();
   lw.max_count = 0;
@@ -353,8 +381,11 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
     for (int h = 0; h < G.Hkv; ++h) {
       const int n = n_gran[i * G.Hkv + h];
       HeadItems hi{(int)items.size() - lw.first_item, 0};
+      const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
+      const int ridx = mode == ATTN_DECODE ? c->role_idx[layer * G.Hkv + h] : h;
       for (int g0 = 0; g0 < n; g0 += gpi) {
-        items.push_back(WorkItem{(int)i, h, g0, std::min(n, g0 + gpi)});
+        items.push_back(WorkItem{(int)i, h, g0, std::min(n, g0 + gpi), seq_ids[i], role, ridx, c->seqs[seq_ids[i]].T_a, c->seqs[seq_ids[i]].C,
+                                 c->seqs[seq_ids[i]].S});
         ++hi.count;
       }
       heads.push_back(hi);
@@ -448,7 +479,7 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
   CK(launch_place_scatter(c->cv, seq, layer, (const bf16 *)k_dev, (const bf16 *)v_dev, n_tokens, audio_begin, audio_end, T_t,
                           C_b, S_b, c->stage, st));
   if (!full && C_b > 0) {
-    if (c->prefill_C != C_b) {
+    if (c->prefill_seq != seq || c->prefill_T_a != T_a) {
       std::vector<WorkItem> items;
       std::vector<HeadItems> heads;
       LayerWork lw;
@@ -469,16 +500,16 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
       CK(cudaMemcpyAsync(c->d_pf_head_items, heads.data(), heads.size() * sizeof(HeadItems), cudaMemcpyHostToDevice, st));
       CK(cudaStreamSynchronize(st));  // the host vectors go out of scope
       c->pf_n_items = (int)items.size();
-      c->prefill_C = C_b;
+      c->prefill_seq = seq; c->prefill_T_a = T_a;
     }
     AttnArgs a{};
-    a.mode = ATTN_PREFILL; a.layer = layer; a.n_active = 1; a.has_new = 0; a.score_on = 1;
-    a.active = c->d_iota + seq; a.items = c->d_pf_items; a.n_items = c->pf_n_items;
+    a.mode = ATTN_PREFILL; a.layer = layer; a.li = c->layers[layer]; a.n_active = 1; a.has_new = 0; a.score_on = 1;
+    a.active = c->d_iota + seq; a.items = c->d_pf_items; a.n_items = c->pf_n_items; a.head_items = c->d_pf_head_items;
     a.q = (const bf16 *)q_last_dev;
     a.anchor_base = c->stage; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
-    a.part_o = c->part_o; a.part_ml = c->part_ml; a.gran_em = c->gran_em; a.n_aq = G.Hq; a.n_ag_max = c->n_ag_max;
+    a.part_o = c->part_o; a.part_ml = c->part_ml; a.gran_em = c->pf_gran_em; a.n_aq = G.Hq; a.n_ag_max = c->n_ag_max;
     CK(launch_attn(c->cv, a, st));
-    CK(launch_prefill_select(c->cv, seq, layer, c->d_pf_head_items, c->part_ml, c->gran_em, c->n_ag_max, st));
+    CK(launch_prefill_select(c->cv, seq, layer, c->d_pf_head_items, c->part_ml, c->pf_gran_em, c->n_ag_max, st));
   }
   CK(launch_place_gather(c->cv, seq, layer, full ? 1 : 0, c->stage, C_b, st));
   CK(cudaEventRecord(c->ev_place, st));
@@ -504,8 +535,14 @@ extern "C" wnw_status_t wnw_step_begin(wnw_cache_t *c, const int32_t *active, in
   c->active.assign(active, active + n_active);
   wnw_status_t s = ensure_worklists(c);
   if (s != WNW_OK) return s;
-  c->in_step = true; c->next_layer = 0; c->appended = -1;
+  c->in_step = true; c->next_layer = 0; c->appended = -1; c->last_side_layer = -1;
   return WNW_OK;
+}
+
+static bool stream_is_capturing(cudaStream_t st) {
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) { cudaGetLastError(); return false; }
+  return cs != cudaStreamCaptureStatusNone;
 }
 
 static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer, const void *q, const void *k_new,
@@ -523,26 +560,40 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const int n_active = (int)c->active.size();
   const bool tiered = want_mode == WNW_MODE_TIERED;
-  if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
-  // the recall that refreshed this layer's slots (issued in the previous step) must have landed
-  if (tiered && c->cfg.recall_mode == WNW_RECALL_SIDE_STREAM) {
-    const int x = c->tail_of[layer];
-    if (x >= 0 && c->recall_recorded[x]) CK(cudaStreamWaitEvent(st, c->ev_recall_done[x], 0));
+  // Inside a stream capture the step is one graph: cross-step ordering comes from the join in wnw_step_end, and
+  // events recorded outside the capture must not be waited on.
+  const bool capturing = stream_is_capturing(st);
+  if (layer == 0) c->step_capturing = capturing;
+  else if (capturing != c->step_capturing) return WNW_ERR_STATE;
+  if (!capturing) {
+    if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
+    // side-stream work of the previous step that this layer depends on must have landed: the selection kernel that
+    // read this layer's partial buffers, and the recall that refreshed this layer's slots
+    if (tiered && c->cfg.recall_mode != WNW_RECALL_INLINE) {
+      if (c->side_recorded[layer]) CK(cudaStreamWaitEvent(st, c->ev_side_done[layer], 0));
+      const int x = c->tail_of[layer];
+      if (x >= 0 && x != layer && c->side_recorded[x]) CK(cudaStreamWaitEvent(st, c->ev_side_done[x], 0));
+    }
   }
-  if (has_new) CK(launch_append(c->cv, layer, n_active, c->d_active, (const bf16 *)k_new, (const bf16 *)v_new, st));
   const LayerWork &lw = c->wl_layers[layer];
   const LayerInfo &li = c->layers[layer];
+  float2 *gran_em_l = c->gran_em + (size_t)layer * c->gran_em_layer_stride;
+  float2 *head_mz_l = c->head_mz + (size_t)layer * G.max_batch * G.Hq;
   AttnArgs a{};
-  a.mode = tiered ? ATTN_DECODE : ATTN_FULL; a.layer = layer; a.n_active = n_active; a.has_new = has_new;
+  a.mode = tiered ? ATTN_DECODE : ATTN_FULL; a.layer = layer; a.li = li; a.n_active = n_active; a.has_new = has_new;
   a.score_on = tiered && li.n_anchor > 0;
+  if (const char *e = getenv("WNW_DEBUG_STOP")) a.debug_stop = atoi(e);  // timing experiments only; breaks results
   a.active = c->d_active; a.items = c->d_items + lw.first_item; a.n_items = lw.n_items;
-  a.q = (const bf16 *)q;
+  a.head_items = c->d_head_items + lw.head_items_off;
+  a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
+  a.head_done = c->head_done; a.head_mz = head_mz_l; a.out = (bf16 *)out;
   a.anchor_base = c->cv.anchor; a.anchor_seq_stride = G.anchor_seq_stride;
   a.anchor_head0 = tiered ? li.anchor_off : layer * G.Hkv;
-  a.part_o = c->part_o; a.part_ml = c->part_ml; a.gran_em = c->gran_em;
+  a.part_o = c->part_o; a.part_ml = c->part_ml; a.gran_em = gran_em_l;
   a.n_aq = std::max(li.n_anchor * G.g, 1); a.n_ag_max = c->n_ag_max;
   cudaEvent_t t0 = nullptr, t1 = nullptr;
-  if (c->timing) {
+  const bool timing = c->timing && !capturing;
+  if (timing) {
     for (cudaEvent_t *e : {&t0, &t1}) {
       if (!c->t_free.empty()) { *e = c->t_free.back(); c->t_free.pop_back(); }
       else CK(cudaEventCreate(e));
@@ -550,26 +601,37 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     CK(cudaEventRecord(t0, st));
   }
   CK(launch_attn(c->cv, a, st));
-  if (c->timing) {
+  if (timing) {
     CK(cudaEventRecord(t1, st));
     c->t_used.emplace_back(t0, t1);
   }
-  TailArgs t{};
-  t.mode = a.mode; t.layer = layer; t.n_active = n_active; t.score_on = a.score_on;
-  t.active = c->d_active; t.head_items = c->d_head_items + lw.head_items_off;
-  t.part_o = c->part_o; t.part_ml = c->part_ml; t.gran_em = c->gran_em; t.n_aq = a.n_aq; t.n_ag_max = a.n_ag_max;
-  t.head_mz = c->head_mz; t.out = (bf16 *)out; t.seq_done = c->seq_done;
-  CK(launch_tail(c->cv, t, lw.max_count, st));
-  if (tiered && li.upd_count > 0) {
-    const int skip = c->cfg.recall_mode == WNW_RECALL_SKIP;
-    if (c->cfg.recall_mode == WNW_RECALL_SIDE_STREAM) {
+  // chunk scores, selection, recall: on the side stream, overlapping whatever follows on the caller's stream
+  if (tiered && (li.n_anchor > 0 || li.upd_count > 0)) {
+    SelectArgs sa{};
+    sa.layer = layer; sa.n_active = n_active; sa.score_on = a.score_on; sa.li = li; sa.active = c->d_active;
+    sa.gran_em = gran_em_l; sa.head_mz = head_mz_l; sa.n_aq = a.n_aq; sa.n_ag_max = a.n_ag_max;
+    int aq = 0;
+    for (int h = 0; h < G.Hkv; ++h)
+      if (c->roles[layer * G.Hkv + h] == ROLE_ANCHOR)
+        for (int r = 0; r < G.g; ++r) sa.aq_head[aq++] = (uint8_t)(h * G.g + r);
+    for (int u = 0; u < li.upd_count && u < MAX_UPD_BY_VALUE; ++u) {
+      sa.upd_layer[u] = (int16_t)c->upd_list[li.upd_first + u];
+      sa.upd_src[u] = (int16_t)c->layers[sa.upd_layer[u]].src;
+    }
+    const bool inline_mode = c->cfg.recall_mode == WNW_RECALL_INLINE;
+    cudaStream_t ss = inline_mode ? st : c->side;
+    if (!inline_mode) {
       CK(cudaEventRecord(c->ev_layer_done[layer], st));
-      CK(cudaStreamWaitEvent(c->side, c->ev_layer_done[layer], 0));
-      CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count, 0, c->side));
-      CK(cudaEventRecord(c->ev_recall_done[layer], c->side));
-      c->recall_recorded[layer] = 1;
-    } else {
-      CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count, skip, st));
+      CK(cudaStreamWaitEvent(ss, c->ev_layer_done[layer], 0));
+    }
+    CK(launch_select(c->cv, sa, c->sel_smem[layer], ss));
+    if (li.upd_count > 0)
+      CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count,
+                       c->cfg.recall_mode == WNW_RECALL_SKIP, ss));
+    if (!inline_mode) {
+      CK(cudaEventRecord(c->ev_side_done[layer], ss));
+      c->side_recorded[layer] = 1;
+      c->last_side_layer = layer;
     }
   }
   c->appended = has_new;
@@ -592,9 +654,15 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
   if (!c->in_step || c->next_layer != c->geo.L) return WNW_ERR_STATE;
   DeviceGuard guard(c->cfg.device);
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  const bool capturing = stream_is_capturing(st);
+  if (capturing != c->step_capturing) return WNW_ERR_STATE;
+  if (capturing && c->last_side_layer >= 0 && c->cfg.recall_mode != WNW_RECALL_INLINE)
+    CK(cudaStreamWaitEvent(st, c->ev_side_done[c->last_side_layer], 0));  // join the forked side stream into the graph
   CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1, st));
-  CK(cudaEventRecord(c->ev_step, st));
-  c->step_recorded = true;
+  if (!capturing) {
+    CK(cudaEventRecord(c->ev_step, st));
+    c->step_recorded = true;
+  }
   for (int b : c->active)
     if (c->appended == 1) c->seqs[b].T_t += 1;
   c->in_step = false;
