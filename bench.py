@@ -114,16 +114,25 @@ class Job:
         self.B = w.batch
         self.caches = {}
         L, n = w.n_layers, w.n_steps
-        # decode inputs resident in HBM: [step][layer][B][...] so one step is one contiguous slab
-        self.q = torch.empty((n, L, self.B, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=device)
-        self.kn = torch.empty((n, L, self.B, w.n_kv_heads, w.head_dim), dtype=torch.bfloat16, device=device)
-        self.vn = torch.empty_like(self.kn)
+        # decode inputs resident in HBM; one step is one contiguous slab [q of all layers | k_new | v_new]
+        nq, nk = L * self.B * w.n_q_heads * w.head_dim, L * self.B * w.n_kv_heads * w.head_dim
+        self.slab = torch.empty((n, nq + 2 * nk), dtype=torch.bfloat16, device=device)
+        self.q = self.slab[:, :nq].view(n, L, self.B, w.n_q_heads, w.head_dim)
+        self.kn = self.slab[:, nq:nq + nk].view(n, L, self.B, w.n_kv_heads, w.head_dim)
+        self.vn = self.slab[:, nq + nk:].view(n, L, self.B, w.n_kv_heads, w.head_dim)
         for b in range(self.B):
             for l in range(L):
                 d = self.syn.decode(b, l)
                 self.q[:, l, b] = d["q"]; self.kn[:, l, b] = d["k_new"]; self.vn[:, l, b] = d["v_new"]
+        # static buffers a captured step reads from / writes to (a producer kernel would fill them in a real decoder)
+        self.sslab = torch.zeros(nq + 2 * nk, dtype=torch.bfloat16, device=device)
+        self.sq = self.sslab[:nq].view(L, self.B, w.n_q_heads, w.head_dim)
+        self.skn = self.sslab[nq:nq + nk].view(L, self.B, w.n_kv_heads, w.head_dim)
+        self.svn = self.sslab[nq + nk:].view(L, self.B, w.n_kv_heads, w.head_dim)
         self.out = torch.zeros((L, self.B, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=device)
         self.flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+        self.stream = torch.cuda.Stream(device=device)
+        self.captured = set()
 
     def create(self, key, mode, recall_mode=0):
         w, wnw = self.w, self.wnw
@@ -163,15 +172,40 @@ class Job:
             fn(h, l, q[l], kn[l], vn[l], out[l])
         wnw.wnw_step_end(h)
 
-    def timed_steps(self, key, t0, n, full=False, flush=True):
-        """Device time of n consecutive steps, L2 flushed (untimed) before each.  Returns per-step ms."""
+    def capture(self, key, full=False):
+        """Captures one step of cache `key` on the job's stream as a CUDA graph that reads the static buffers."""
+        wnw, h = self.wnw, self.caches[key]
+        torch.cuda.synchronize(self.dev)
+        wnw.wnw_graph_begin(h, list(range(self.B)), self.stream)
+        fn = wnw.wnw_decode_layer_full if full else wnw.wnw_decode_layer
+        wnw.wnw_step_begin(h, list(range(self.B)))
+        for l in range(self.w.n_layers):
+            fn(h, l, self.sq[l], self.skn[l], self.svn[l], self.out[l], stream=self.stream)
+        wnw.wnw_step_end(h, stream=self.stream)
+        wnw.wnw_graph_end(h, self.stream)
+        self.captured.add(key)
+
+    def graph_step(self, key, t, src=None):
+        """One replayed step: the step's inputs are copied into the static buffers (one copy), then one graph launch."""
+        self.sslab.copy_(self.slab[t] if src is None else src, non_blocking=True)
+        self.wnw.wnw_graph_launch(self.caches[key], self.stream)
+
+    def timed_steps(self, key, t0, n, full=False, flush=True, graph=True):
+        """Device time of n consecutive steps, L2 flushed (untimed) before each.  Returns per-step ms.
+        graph=True replays the captured step; otherwise the layers are issued eagerly."""
+        if graph and key not in self.captured:
+            self.capture(key, full=full)
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
-        for i in range(n):
-            if flush:
-                self.flush_l2()
-            evs[i][0].record()
-            self.step(key, t0 + i, full=full)
-            evs[i][1].record()
+        with torch.cuda.stream(self.stream):
+            for i in range(n):
+                if flush:
+                    self.flush_l2()
+                evs[i][0].record()
+                if graph:
+                    self.graph_step(key, t0 + i)
+                else:
+                    self.step(key, t0 + i, full=full)
+                evs[i][1].record()
         torch.cuda.synchronize(self.dev)
         return [a.elapsed_time(b) for a, b in evs]
 
@@ -305,7 +339,7 @@ def run_ours(args, rank, world, local_rank):
             job.step("wnw", t)
         torch.cuda.synchronize(dev)
         wnw.wnw_set_kernel_timing(job.caches["wnw"], True)
-        per_step = job.timed_steps("wnw", W, K, flush=not args.no_flush)
+        per_step = job.timed_steps("wnw", W, K, flush=not args.no_flush, graph=not args.eager)
         ms, n = wnw.wnw_get_kernel_time(job.caches["wnw"])
         print(json.dumps({"quick": True, "workload": w.name, "ms_per_step": sum(per_step) / K, "steps": K,
                           "attn_us_per_launch": ms * 1e3 / max(n, 1)}), flush=True)
@@ -359,7 +393,7 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     sampler.start()
     wall0 = time.perf_counter()
-    per_step = job.timed_steps("wnw", W + R, K)
+    per_step = job.timed_steps("wnw", W + R, K, graph=not args.eager)
     barrier()
     wall = time.perf_counter() - wall0
     clocks = sampler.stop()
@@ -372,37 +406,41 @@ def run_ours(args, rank, world, local_rank):
     value = world * w.batch / (ms_per_step * 1e-3)
 
     # ---- comparison: own full-cache kernel, and WnW with recall copies skipped (exposed recall time)
-    full_steps = job.timed_steps("full", W + R, K, full=True)
-    skip_steps = job.timed_steps("skip", W + R, K)
+    full_steps = job.timed_steps("full", W + R, K, full=True, graph=not args.eager)
+    skip_steps = job.timed_steps("skip", W + R, K, graph=not args.eager)
     barrier()
 
     # ---- end to end: inputs start in pinned host memory, outputs end there, copies inside the timed region
     n_e2e = min(K, 64)
-    hq = job.q[W + R:W + R + n_e2e].cpu().pin_memory(); hkn = job.kn[W + R:W + R + n_e2e].cpu().pin_memory()
-    hvn = job.vn[W + R:W + R + n_e2e].cpu().pin_memory()
+    hslab = job.slab[W + R:W + R + n_e2e].cpu().pin_memory()
     hout = torch.empty((n_e2e,) + tuple(job.out.shape), dtype=torch.bfloat16).pin_memory()
     job.create("e2e", wnw.WNW_MODE_TIERED)
     job.place_all(["e2e"])
     for tt in range(W + R):
         job.step("e2e", tt)
-    dq = torch.empty_like(job.q[0]); dkn = torch.empty_like(job.kn[0]); dvn = torch.empty_like(job.vn[0])
     torch.cuda.synchronize(dev)
+    if not args.eager:
+        job.capture("e2e")
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2e_ms = 0.0
-    for i in range(n_e2e):
-        job.flush_l2()
-        e0.record()
-        dq.copy_(hq[i], non_blocking=True); dkn.copy_(hkn[i], non_blocking=True); dvn.copy_(hvn[i], non_blocking=True)
-        job.step("e2e", W + R + i, q=dq, kn=dkn, vn=dvn)
-        hout[i].copy_(job.out, non_blocking=True)
-        e1.record()
-        e1.synchronize()
-        e2e_ms += e0.elapsed_time(e1)
+    with torch.cuda.stream(job.stream):
+        for i in range(n_e2e):
+            job.flush_l2()
+            e0.record()
+            if args.eager:
+                job.sslab.copy_(hslab[i], non_blocking=True)
+                job.step("e2e", W + R + i, q=job.sq, kn=job.skn, vn=job.svn)
+            else:
+                job.graph_step("e2e", W + R + i, src=hslab[i])      # host -> device copy of the step's inputs, then the step
+            hout[i].copy_(job.out, non_blocking=True)               # device -> host read of the step's outputs
+            e1.record()
+            e1.synchronize()
+            e2e_ms += e0.elapsed_time(e1)
     t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
     if world > 1:
         torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
     e2e_value = world * w.batch / (float(t.item()) / n_e2e * 1e-3)
-    h2d = (dq.numel() + dkn.numel() + dvn.numel()) * 2
+    h2d = job.sslab.numel() * 2
     d2h = job.out.numel() * 2
 
     if rank != 0:
@@ -439,7 +477,10 @@ def run_ours(args, rank, world, local_rank):
     full_us = full_ms * 1e3 / max(full_n, 1)
     full_achieved = (algo_bytes_full / max(full_n, 1)) / (full_us * 1e-6) / 1e9 if full_us > 0 else 0.0
     n_upd_layers = int(sum(1 for l in range(w.n_layers) if (w.roles[l] == ROLE_TIDAL).any()))
-    launches_per_step = w.n_layers * 3 + n_upd_layers + 1  # append + attention + tail per layer, recall per tidal layer, step end
+    n_side_layers = int(sum(1 for l in range(w.n_layers) if (w.roles[l] == ROLE_TIDAL).any() or (w.roles[l] == ROLE_ANCHOR).any()))
+    # per step: one attention kernel per layer, one selection kernel per layer with anchors or a table to update,
+    # one recall kernel per layer with a table to update, one step-end kernel
+    launches_per_step = w.n_layers + n_side_layers + n_upd_layers + 1
     recall_bytes_step = (stats1["recall_bytes"] - stats0["recall_bytes"]) / K
     ms_full = sum(full_steps) / K
     ms_skip = sum(skip_steps) / K
@@ -453,7 +494,7 @@ def run_ours(args, rank, world, local_rank):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(w),
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(w), launch="eager" if args.eager else "cuda graph replay of the step"),
         "clocks": clocks, "gpu_launches": launches_per_step * K,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e},
         "roofline": {"bound": "hbm", "kernel": "wnw_attn_kernel", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
@@ -483,6 +524,7 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3", "prof"])
     ap.add_argument("--quick", action="store_true", help="only the WnW steps (for profiler captures); prints a short line")
     ap.add_argument("--no-flush", action="store_true", help="with --quick: do not flush L2 between steps")
+    ap.add_argument("--eager", action="store_true", help="issue every layer eagerly instead of replaying a captured step")
     ap.add_argument("--roofline-steps", type=int, default=16)
     ap.add_argument("--oracle-layers", type=int, default=6, help="layers of sequence 0 the CPU baseline samples (0 = skip)")
     ap.add_argument("--oracle-steps", type=int, default=4)

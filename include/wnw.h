@@ -152,6 +152,20 @@ wnw_status_t wnw_decode_layer_full(wnw_cache_t *cache, int32_t layer, const void
 /* Close the step: per-sequence step counters and text lengths advance.  All layers must have been called. */
 wnw_status_t wnw_step_end(wnw_cache_t *cache, void *cuda_stream);
 
+/* CUDA-graph replay of a decode step (launch overhead of a whole step collapses into one graph launch).
+ * wnw_graph_begin prepares the work lists for the given sequences (HOST array, as in wnw_step_begin) and starts
+ * capturing on cuda_stream; the caller then issues ONE ordinary step for those sequences on that stream
+ * (wnw_step_begin, wnw_decode_layer[_full] for every layer, wnw_step_end) using buffers it will keep at the same
+ * addresses; wnw_graph_end finishes the capture.  Nothing executes during capture and the cache's state does not
+ * advance.  Each wnw_graph_launch then runs one step for the captured set of sequences with whatever the buffers
+ * hold at that time, and advances the cache exactly like an eager step (text length, step counters).  The capture
+ * includes the side-stream selection and recall work and joins it before the step ends.  Eager steps and graph
+ * launches may be mixed.  A new capture replaces the previous graph.  Re-placing a sequence or changing the active
+ * set requires a new capture.  cuda_stream must not be the default (NULL) stream. */
+wnw_status_t wnw_graph_begin(wnw_cache_t *cache, const int32_t *active_seqs_host, int32_t n_active, void *cuda_stream);
+wnw_status_t wnw_graph_end(wnw_cache_t *cache, void *cuda_stream);
+wnw_status_t wnw_graph_launch(wnw_cache_t *cache, void *cuda_stream);
+
 /* Inspection.  Each call drains the cache's streams first.  Out-buffers are HOST memory owned by the caller.
  *   chunk_scores : score_sum of the last completed step, [C] floats (anchor layers only)
  *   prefill_scores: pre[c] of one non-anchor KV-head, [C] floats

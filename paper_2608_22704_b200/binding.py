@@ -51,6 +51,9 @@ _SIGNATURES = {
     "wnw_decode_layer": [_vp, _i32, _vp, _vp, _vp, _vp, _vp],
     "wnw_decode_layer_full": [_vp, _i32, _vp, _vp, _vp, _vp, _vp],
     "wnw_step_end": [_vp, _vp],
+    "wnw_graph_begin": [_vp, C.POINTER(_i32), _i32, _vp],
+    "wnw_graph_end": [_vp, _vp],
+    "wnw_graph_launch": [_vp, _vp],
     "wnw_get_chunk_scores": [_vp, _i32, _i32, C.POINTER(C.c_float), C.POINTER(_i32)],
     "wnw_get_prefill_scores": [_vp, _i32, _i32, _i32, C.POINTER(C.c_float), C.POINTER(_i32)],
     "wnw_get_selected": [_vp, _i32, _i32, C.POINTER(_i32), C.POINTER(_i32)],
@@ -153,6 +156,19 @@ def wnw_decode_layer_full(cache, layer, q, k_new, v_new, out, stream=None):
 
 def wnw_step_end(cache, stream=None):
     _ck(lib().wnw_step_end(cache, _stream(stream)), "wnw_step_end")
+
+
+def wnw_graph_begin(cache, active: Sequence[int], stream=None):
+    a = (C.c_int32 * len(active))(*active)
+    _ck(lib().wnw_graph_begin(cache, a, len(active), _stream(stream)), "wnw_graph_begin")
+
+
+def wnw_graph_end(cache, stream=None):
+    _ck(lib().wnw_graph_end(cache, _stream(stream)), "wnw_graph_end")
+
+
+def wnw_graph_launch(cache, stream=None):
+    _ck(lib().wnw_graph_launch(cache, _stream(stream)), "wnw_graph_launch")
 
 
 def wnw_sync(cache):

@@ -414,14 +414,22 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 template <int D, bool G16>
 static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
   const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(wnw_attn_kernel<D, G16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
   wnw_attn_kernel<D, G16><<<a.n_items, NW * 32, smem, st>>>(cv, a);
   return cudaGetLastError();
+}
+
+template <int D, bool G16>
+static cudaError_t configure_t() {
+  return cudaFuncSetAttribute(wnw_attn_kernel<D, G16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)((size_t)NW * NSTAGE * 2 * GR * D * 2));
+}
+// Opt-in shared-memory sizes, set once per device at cache creation (never during a stream capture).
+cudaError_t configure_attn_kernels() {
+  cudaError_t e;
+  if ((e = configure_t<128, true>()) != cudaSuccess) return e;
+  if ((e = configure_t<128, false>()) != cudaSuccess) return e;
+  if ((e = configure_t<64, true>()) != cudaSuccess) return e;
+  return configure_t<64, false>();
 }
 
 cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {

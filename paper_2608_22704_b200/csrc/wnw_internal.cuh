@@ -156,6 +156,9 @@ cudaError_t launch_prefill_select(const CacheView &cv, int b, int layer, const H
 cudaError_t launch_place_gather(const CacheView &cv, int b, int layer, int full_mode, const bf16 *stage, int C_b,
                                 cudaStream_t st);
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
+cudaError_t configure_attn_kernels();
+cudaError_t configure_select_kernel();
+constexpr int SELECT_SMEM_CAP = 200 * 1024;  // dynamic shared memory the selection kernel may be launched with
 int attn_warps();  // warps per attention CTA (granules per work item should be a multiple)
 
 }  // namespace wnw

@@ -107,15 +107,11 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
   }
 }
 
+cudaError_t configure_select_kernel() {
+  return cudaFuncSetAttribute(wnw_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM_CAP);
+}
+
 cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, cudaStream_t st) {
-  if (smem_bytes > 48 * 1024) {
-    static size_t configured = 0;
-    if (smem_bytes > configured) {
-      cudaError_t e = cudaFuncSetAttribute(wnw_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-      if (e != cudaSuccess) return e;
-      configured = smem_bytes;
-    }
-  }
   wnw_select_kernel<<<a.n_active, SEL_WARPS * 32, smem_bytes, st>>>(cv, a, (int)smem_bytes);
   return cudaGetLastError();
 }

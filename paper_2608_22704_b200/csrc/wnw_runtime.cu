@@ -79,10 +79,17 @@ struct wnw_cache {
   // streams / events
   cudaStream_t side = nullptr, last_stream = nullptr;
   std::vector<cudaEvent_t> ev_layer_done, ev_side_done;
+  std::vector<cudaEvent_t> ev_layer_done_cap, ev_side_done_cap;  // used only inside a stream capture
   std::vector<char> side_recorded;
   std::vector<size_t> sel_smem;   // dynamic shared memory of each layer's selection launch
   size_t gran_em_layer_stride = 0;
   bool step_capturing = false;
+  // captured step
+  bool graph_capturing = false;
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t graph_exec = nullptr;
+  std::vector<int> graph_active, graph_prepared;
+  int graph_appended = 0;
   int last_side_layer = -1;
   cudaEvent_t ev_place = nullptr, ev_step = nullptr;
   bool place_recorded = false, step_recorded = false;
@@ -135,8 +142,12 @@ static void destroy_impl(wnw_cache *c) {
   if (c->side) cudaStreamDestroy(c->side);
   for (auto e : c->ev_layer_done) cudaEventDestroy(e);
   for (auto e : c->ev_side_done) cudaEventDestroy(e);
+  for (auto e : c->ev_layer_done_cap) cudaEventDestroy(e);
+  for (auto e : c->ev_side_done_cap) cudaEventDestroy(e);
   if (c->ev_place) cudaEventDestroy(c->ev_place);
   if (c->ev_step) cudaEventDestroy(c->ev_step);
+  if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+  if (c->graph) cudaGraphDestroy(c->graph);
   for (auto &p : c->t_used) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
   for (auto e : c->t_free) cudaEventDestroy(e);
   delete c;
@@ -197,6 +208,8 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
 #define CKC(call) do { wnw_status_t _s = (call); if (_s != WNW_OK) return fail(_s); } while (0)
 #define CKE(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { return fail(_e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA); } } while (0)
   cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
+  CKE(configure_attn_kernels());
+  CKE(configure_select_kernel());
   const int L = cfg->n_layers, Hkv = cfg->n_kv_heads, d = cfg->head_dim, nc = cfg->chunk_tokens;
   const bool full = cfg->mode == WNW_MODE_FULL;
   c->roles.assign(cfg->roles, cfg->roles + (size_t)L * Hkv);
@@ -312,7 +325,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     const size_t fixed_part = (n_aq_l * 8 + 15) / 16 * 16 + ((size_t)G.C_max * 4 + 15) / 16 * 16 +
                               (size_t)std::min(li.upd_count, 8) * select_ws_bytes(G.C_max, G.S_max);
     const size_t per_chunk = li.n_anchor > 0 ? n_aq_l * G.gpc * 8 : 0;
-    const size_t cap = 200 * 1024;
+    const size_t cap = SELECT_SMEM_CAP - 16;
     if (fixed_part + per_chunk > cap) return fail(WNW_ERR_UNSUPPORTED);  // chunk tables too large for one CTA
     c->sel_smem[l] = std::min(cap, fixed_part + per_chunk * std::max(G.C_max, 1)) + 16;
   }
@@ -321,9 +334,12 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   c->mirror_ptrs.assign(B, nullptr);
   CKE(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
   c->ev_layer_done.resize(L); c->ev_side_done.resize(L); c->side_recorded.assign(L, 0);
+  c->ev_layer_done_cap.resize(L); c->ev_side_done_cap.resize(L);
   for (int l = 0; l < L; ++l) {
     CKE(cudaEventCreateWithFlags(&c->ev_layer_done[l], cudaEventDisableTiming));
     CKE(cudaEventCreateWithFlags(&c->ev_side_done[l], cudaEventDisableTiming));
+    CKE(cudaEventCreateWithFlags(&c->ev_layer_done_cap[l], cudaEventDisableTiming));
+    CKE(cudaEventCreateWithFlags(&c->ev_side_done_cap[l], cudaEventDisableTiming));
   }
   CKE(cudaEventCreateWithFlags(&c->ev_place, cudaEventDisableTiming));
   CKE(cudaEventCreateWithFlags(&c->ev_step, cudaEventDisableTiming));
@@ -532,7 +548,9 @@ extern "C" wnw_status_t wnw_step_begin(wnw_cache_t *c, const int32_t *active, in
     if (c->seqs[active[i]].placed_layers != c->geo.L) return WNW_ERR_STATE;
   }
   DeviceGuard guard(c->cfg.device);
-  c->active.assign(active, active + n_active);
+  std::vector<int> want(active, active + n_active);
+  if (c->graph_capturing && want != c->graph_prepared) return WNW_ERR_STATE;  // not the set the capture was prepared for
+  c->active = want;
   wnw_status_t s = ensure_worklists(c);
   if (s != WNW_OK) return s;
   c->in_step = true; c->next_layer = 0; c->appended = -1; c->last_side_layer = -1;
@@ -620,17 +638,19 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     }
     const bool inline_mode = c->cfg.recall_mode == WNW_RECALL_INLINE;
     cudaStream_t ss = inline_mode ? st : c->side;
+    cudaEvent_t ev_l = capturing ? c->ev_layer_done_cap[layer] : c->ev_layer_done[layer];
+    cudaEvent_t ev_s = capturing ? c->ev_side_done_cap[layer] : c->ev_side_done[layer];
     if (!inline_mode) {
-      CK(cudaEventRecord(c->ev_layer_done[layer], st));
-      CK(cudaStreamWaitEvent(ss, c->ev_layer_done[layer], 0));
+      CK(cudaEventRecord(ev_l, st));
+      CK(cudaStreamWaitEvent(ss, ev_l, 0));
     }
     CK(launch_select(c->cv, sa, c->sel_smem[layer], ss));
     if (li.upd_count > 0)
       CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count,
                        c->cfg.recall_mode == WNW_RECALL_SKIP, ss));
     if (!inline_mode) {
-      CK(cudaEventRecord(c->ev_side_done[layer], ss));
-      c->side_recorded[layer] = 1;
+      CK(cudaEventRecord(ev_s, ss));
+      if (!capturing) c->side_recorded[layer] = 1;
       c->last_side_layer = layer;
     }
   }
@@ -657,15 +677,91 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
   const bool capturing = stream_is_capturing(st);
   if (capturing != c->step_capturing) return WNW_ERR_STATE;
   if (capturing && c->last_side_layer >= 0 && c->cfg.recall_mode != WNW_RECALL_INLINE)
-    CK(cudaStreamWaitEvent(st, c->ev_side_done[c->last_side_layer], 0));  // join the forked side stream into the graph
+    CK(cudaStreamWaitEvent(st, c->ev_side_done_cap[c->last_side_layer], 0));  // join the forked side stream into the graph
   CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1, st));
   if (!capturing) {
     CK(cudaEventRecord(c->ev_step, st));
     c->step_recorded = true;
   }
-  for (int b : c->active)
-    if (c->appended == 1) c->seqs[b].T_t += 1;
+  if (!capturing) {
+    for (int b : c->active)
+      if (c->appended == 1) c->seqs[b].T_t += 1;
+  } else if (c->graph_capturing) {
+    c->graph_active = c->active;
+    c->graph_appended = c->appended == 1;
+  }
   c->in_step = false;
+  c->last_stream = st;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_graph_begin(wnw_cache_t *c, const int32_t *active, int32_t n_active, void *cuda_stream) {
+  if (!c || !active || n_active < 1 || n_active > c->geo.max_batch) return WNW_ERR_INVALID_ARG;
+  if (c->in_step || c->graph_capturing) return WNW_ERR_STATE;
+  if (!cuda_stream) return WNW_ERR_INVALID_ARG;  // the legacy default stream cannot be captured
+  for (int i = 0; i < n_active; ++i) {
+    if (active[i] < 0 || active[i] >= c->geo.max_batch) return WNW_ERR_INVALID_ARG;
+    for (int j = 0; j < i; ++j)
+      if (active[j] == active[i]) return WNW_ERR_INVALID_ARG;
+    if (c->seqs[active[i]].placed_layers != c->geo.L) return WNW_ERR_STATE;
+  }
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  // work lists are built and uploaded now: nothing may allocate or synchronise once the capture has begun
+  c->active.assign(active, active + n_active);
+  {
+    wnw_status_t ws = ensure_worklists(c);
+    if (ws != WNW_OK) return ws;
+  }
+  c->graph_prepared = c->active;
+  // everything queued so far must be ordered before the first replay: drain now, the capture cannot wait on it
+  CK(cudaStreamSynchronize(c->side));
+  if (c->last_stream != st) CK(cudaStreamSynchronize(c->last_stream));
+  CK(cudaStreamSynchronize(st));
+  CK(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+  c->graph_capturing = true;
+  c->graph_active.clear();
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_graph_end(wnw_cache_t *c, void *cuda_stream) {
+  if (!c) return WNW_ERR_INVALID_ARG;
+  if (!c->graph_capturing) return WNW_ERR_STATE;
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  c->graph_capturing = false;
+  cudaGraph_t g = nullptr;
+  cudaError_t e = cudaStreamEndCapture(st, &g);
+  const bool complete = !c->in_step && !c->graph_active.empty();
+  c->in_step = false;
+  if (e != cudaSuccess || !g) { c->last_cuda = e; cudaGetLastError(); return WNW_ERR_CUDA; }
+  if (!complete) { cudaGraphDestroy(g); return WNW_ERR_STATE; }  // the capture must hold exactly one whole step
+  if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
+  if (c->graph) { cudaGraphDestroy(c->graph); c->graph = nullptr; }
+  c->graph = g;
+  CK(cudaGraphInstantiate(&c->graph_exec, g, 0));
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_graph_launch(wnw_cache_t *c, void *cuda_stream) {
+  if (!c) return WNW_ERR_INVALID_ARG;
+  if (!c->graph_exec || c->in_step || c->graph_capturing) return WNW_ERR_STATE;
+  for (int b : c->graph_active) {
+    if (c->seqs[b].placed_layers != c->geo.L) return WNW_ERR_STATE;
+    if (c->graph_appended && c->seqs[b].T_t + 1 > c->cfg.max_text_tokens) return WNW_ERR_CAPACITY;
+  }
+  if (c->wl_active != c->graph_active) return WNW_ERR_STATE;  // the work lists the graph points at were rebuilt
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
+  // side-stream work of earlier eager steps touches the tables and slots the graph reads
+  for (int l = 0; l < c->geo.L; ++l)
+    if (c->side_recorded[l]) { CK(cudaStreamWaitEvent(st, c->ev_side_done[l], 0)); c->side_recorded[l] = 0; }
+  CK(cudaGraphLaunch(c->graph_exec, st));
+  CK(cudaEventRecord(c->ev_step, st));
+  c->step_recorded = true;
+  for (int b : c->graph_active)
+    if (c->graph_appended) c->seqs[b].T_t += 1;
   c->last_stream = st;
   return WNW_OK;
 }

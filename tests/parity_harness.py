@@ -145,7 +145,9 @@ class Lockstep:
             self.dec[(b, l)] = self.syn.decode(b, l)
         return self.dec[(b, l)]
 
-    def decode_step(self, t=None, append=True, active=None, check_slots=False):
+    def decode_step(self, t=None, append=True, active=None, check_slots=False, graph=False):
+        """One lock-step decode step.  graph=True replays a captured CUDA graph of the step (captured on first use)
+        from static input buffers instead of issuing the layers eagerly."""
         w = self.w
         t = self.step if t is None else t
         active = list(range(w.batch)) if active is None else list(active)
@@ -153,16 +155,44 @@ class Lockstep:
         prev_tab = {(b, l): wnw.wnw_get_residency(self.h, b, l) for b in o_active for l in range(w.n_layers)
                     if (w.roles[l] == ROLE_TIDAL).any()}
         steps_before = {b: self._steps.get(b, 0) for b in active}
-        wnw.wnw_step_begin(self.h, active)
         if o_active:
             self.o.step_begin(o_active)
         outs = []
+        qs = [torch.stack([self._dec(b, l)["q"][t] for b in active]).to(self.dev) for l in range(w.n_layers)]
+        kns = [torch.stack([self._dec(b, l)["k_new"][t] for b in active]).to(self.dev) if append else None for l in range(w.n_layers)]
+        vns = [torch.stack([self._dec(b, l)["v_new"][t] for b in active]).to(self.dev) if append else None for l in range(w.n_layers)]
+        if graph:
+            if getattr(self, "_graph", None) is None:
+                self._gstream = torch.cuda.Stream(device=self.dev)
+                self._gq = [torch.empty_like(x) for x in qs]
+                self._gkn = [torch.empty_like(x) if x is not None else None for x in kns]
+                self._gvn = [torch.empty_like(x) if x is not None else None for x in vns]
+                self._gout = [torch.empty_like(x) for x in qs]
+                torch.cuda.synchronize(self.dev)
+                wnw.wnw_graph_begin(self.h, active, self._gstream)
+                wnw.wnw_step_begin(self.h, active)
+                for l in range(w.n_layers):
+                    wnw.wnw_decode_layer(self.h, l, self._gq[l], self._gkn[l], self._gvn[l], self._gout[l], stream=self._gstream)
+                wnw.wnw_step_end(self.h, stream=self._gstream)
+                wnw.wnw_graph_end(self.h, self._gstream)
+                self._graph = True
+            with torch.cuda.stream(self._gstream):
+                for l in range(w.n_layers):
+                    self._gq[l].copy_(qs[l])
+                    if append:
+                        self._gkn[l].copy_(kns[l]); self._gvn[l].copy_(vns[l])
+            self._gstream.wait_stream(torch.cuda.current_stream(self.dev))
+            wnw.wnw_graph_launch(self.h, self._gstream)
+            self._gstream.synchronize()
+        else:
+            wnw.wnw_step_begin(self.h, active)
         for l in range(w.n_layers):
-            q = torch.stack([self._dec(b, l)["q"][t] for b in active]).to(self.dev)
-            kn = torch.stack([self._dec(b, l)["k_new"][t] for b in active]).to(self.dev) if append else None
-            vn = torch.stack([self._dec(b, l)["v_new"][t] for b in active]).to(self.dev) if append else None
-            out = torch.empty_like(q)
-            wnw.wnw_decode_layer(self.h, l, q, kn, vn, out)
+            q, kn, vn = qs[l], kns[l], vns[l]
+            if graph:
+                out = self._gout[l]
+            else:
+                out = torch.empty_like(q)
+                wnw.wnw_decode_layer(self.h, l, q, kn, vn, out)
             outs.append((q, kn, vn, out))
             if o_active:
                 idx = [active.index(b) for b in o_active]
@@ -174,7 +204,8 @@ class Lockstep:
                 err = np.abs(got - ref).max()
                 self.max_out_err = max(self.max_out_err, float(err))
                 assert err <= OUT_TOL, f"attention output step {t} layer {l}: max abs err {err:.4f}"
-        wnw.wnw_step_end(self.h)
+        if not graph:
+            wnw.wnw_step_end(self.h)
         wnw.wnw_sync(self.h)
         if o_active:
             self.o.step_end()

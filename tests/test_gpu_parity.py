@@ -84,6 +84,39 @@ def test_jumping_focus_turnover():
     _run(w, seed=6)
 
 
+def test_graph_replay_matches_oracle():
+    """A captured step replayed as a CUDA graph (side-stream selection and recall inside the graph) stays in
+    lock-step with the oracle, also when eager steps are mixed in."""
+    from parity_harness import Lockstep
+    w = tiny_custom(n_layers=3, n_q_heads=8, n_kv_heads=4, head_dim=128, n_text=8, audio_lens=(640, 300), chunk=32, budget=0.2,
+                    n_steps=12, roles=[[A, T, T, F], [T, F, T, F], [A, T, F, T]], region=32, jump_every=3)
+    ls = Lockstep(w, seed=8)
+    try:
+        ls.prefill()
+        ls.decode_step(0, check_slots=True)                       # eager
+        for t in range(1, 7):
+            ls.decode_step(t, graph=True, check_slots=True)       # replay
+        ls.decode_step(7, check_slots=True)                       # eager again
+        for t in range(8, 12):
+            ls.decode_step(t, graph=True, check_slots=True)
+        ls.check_stats()
+    finally:
+        ls.close()
+
+
+def test_config0_graph_replay_all_steps():
+    from parity_harness import Lockstep
+    ls = Lockstep(config0())
+    try:
+        ls.prefill()
+        for t in range(16):
+            ls.decode_step(t, graph=True, check_slots=True)
+        ls.check_stats()
+        assert ls.near_ties == 0
+    finally:
+        ls.close()
+
+
 def test_config1_first_steps():
     """3B Voxtral-shaped stack (30 layers, 32q/8kv, d=128, 3000 audio tokens, chunk 64), first decode steps."""
     w = config1(n_steps=3)
