@@ -19,6 +19,8 @@
 //     publishes the head's final (max, denominator), which the selection kernel needs for the chunk scores.
 // Chunk scoring, selection and recall are not needed by whatever consumes the attention output next, so they run
 // in wnw_select_kernel / wnw_recall_kernel on a side stream (wnw_kernels.cu), off the critical path.
+#include <cstring>
+
 #include "wnw_internal.cuh"
 #include "wnw_tail.cuh"
 
@@ -70,55 +72,52 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 struct GranDesc {
-  const bf16 *k;   // first K row of the granule (V row = k + v_delta)
-  int valid;       // visible tokens in the granule, 0 = nothing to do
+  const bf16 *k;   // first K row of the granule (V row = k + v_delta); always a mapped address
+  int meta;        // >= 0: visible tokens, known statically; -1: text granule, needs the text length; -2: needs `cid`
+  int cid;         // chunk id held by the slot / compact position (filled by a load that is not waited on here)
+  int off;         // token offset of the granule inside its chunk
   int score_idx;   // audio granule index for score partials, -1 = none
 };
 
-// Maps granule j of a head's virtual key space [text capacity | audio] to memory.
-__device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const AttnArgs &a, const LayerInfo &li, int b, int h,
-                                                   int role, int ridx, int j, int T_t, int T_a) {
+// Maps granule j of a head's virtual key space [text capacity | audio] to memory WITHOUT waiting on any global load:
+// the address of every granule is static; what may be unknown yet is how many of its 16 rows are visible.
+__device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const AttnArgs &a, const LayerInfo &li,
+                                                   const WorkItem &it, int j) {
   const Geometry &G = cv.geo;
   GranDesc r;
-  r.k = cv.text; r.valid = 0; r.score_idx = -1;
+  r.cid = -1; r.off = 0; r.score_idx = -1;
   if (j < G.n_tg) {
-    const int tok0 = j * GR, v = T_t - tok0;
-    if (v <= 0) return r;
-    r.valid = v < GR ? v : GR;
-    r.k = cv.text + text_off(G, b, a.layer, h, 0) + (long long)tok0 * G.d;
+    const int tok0 = j * GR;
+    r.k = cv.text + text_off(G, it.b, a.layer, it.h, 0) + (long long)tok0 * G.d;
+    r.meta = tok0 + GR <= it.T_hint ? GR : -1;
     return r;
   }
   const int ag = j - G.n_tg, ci = ag / G.gpc, off = (ag - ci * G.gpc) * GR;
-  int c, store_row;
-  const bf16 *base;
-  if (role == ROLE_ANCHOR) {
-    c = ci;
-    base = a.anchor_base + anchor_off(G, a.anchor_seq_stride, b, a.anchor_head0 + ridx, 0);
-    store_row = ci * G.nc + off;
-  } else if (role == ROLE_TIDAL) {
-    c = cv.slot_chunk[((long long)b * G.L + a.layer) * G.S_max + ci];
-    base = cv.pool + pool_off(G, li, b, ci, ridx, 0);
-    store_row = off;
+  r.off = off;
+  if (it.role == ROLE_ANCHOR) {
+    r.k = a.anchor_base + anchor_off(G, a.anchor_seq_stride, it.b, a.anchor_head0 + it.ridx, 0) + (long long)(ci * G.nc + off) * G.d;
+    int len = it.T_a - ci * G.nc;
+    if (len > G.nc) len = G.nc;
+    len -= off;
+    r.meta = len <= 0 ? 0 : (len < GR ? len : GR);
+    if (a.score_on) r.score_idx = ag;
+  } else if (it.role == ROLE_TIDAL) {
+    r.k = cv.pool + pool_off(G, li, it.b, ci, it.ridx, 0) + (long long)off * G.d;
+    r.cid = cv.slot_chunk[((long long)it.b * G.L + a.layer) * G.S_max + ci];
+    r.meta = -2;
   } else {
-    const long long fh = (long long)b * G.F_tot + li.fixed_off + ridx;
-    c = ci < cv.fixed_n[fh] ? cv.fixed_chunks[fh * G.S_max + ci] : -1;
-    base = cv.fixed + fixed_off(G, li, b, ridx, 0);
-    store_row = ci * G.nc + off;
+    const long long fh = (long long)it.b * G.F_tot + li.fixed_off + it.ridx;
+    r.k = cv.fixed + fixed_off(G, li, it.b, it.ridx, 0) + (long long)(ci * G.nc + off) * G.d;
+    r.cid = cv.fixed_chunks[fh * G.S_max + ci];
+    r.meta = -2;
   }
-  if (c < 0) return r;
-  int len = T_a - c * G.nc;
-  if (len > G.nc) len = G.nc;
-  len -= off;
-  if (len <= 0) return r;
-  r.valid = len < GR ? len : GR;
-  r.k = base + (long long)store_row * G.d;
-  if (role == ROLE_ANCHOR && a.score_on) r.score_idx = ag;
   return r;
 }
 
 template <int D, bool G16>
 __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant__ CacheView cv,
-                                                           const __grid_constant__ AttnArgs a) {
+                                                           const __grid_constant__ AttnArgs a,
+                                                           const __grid_constant__ InlineItems inl) {
   extern __shared__ __align__(128) unsigned char smem[];
   const Geometry &G = cv.geo;
   constexpr int ROWB = D * 2;             // bytes per K or V row
@@ -130,11 +129,15 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr size_t SMEM_TOTAL = (size_t)NW * NSTAGE * 2 * GR * D * 2;
   STAMP(0);
-  const WorkItem it = a.items[blockIdx.x];
+  // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
+  const WorkItem it = a.n_items <= INLINE_ITEMS_MAX ? inl.it[blockIdx.x] : a.items[blockIdx.x];
   const int b = it.b, role = it.role, ridx = it.ridx, T_a = it.T_a;
   const int g = G.g;
   const LayerInfo &li = a.li;
   const int T_t = cv.text_len[b] + a.has_new;
+#ifdef WNW_PHASE_STAMPS
+  if (it.g0 >= 0) STAMP(10);
+#endif
   long long v_delta_audio;
   if (role == ROLE_ANCHOR) v_delta_audio = (long long)G.T_a_pad * G.d;
   else if (role == ROLE_TIDAL) v_delta_audio = (long long)G.nc * G.d;
@@ -161,6 +164,9 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     }
   }
 
+#ifdef WNW_PHASE_STAMPS
+  if (my_base != 0) STAMP(11);
+#endif
   float o[D / 8][4];
 #pragma unroll
   for (int t = 0; t < D / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
@@ -170,33 +176,53 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   const int n_my = first < it.g1 ? (it.g1 - first + NW - 1) / NW : 0;
 
   GranDesc blk;  // descriptor this lane decoded for the current block of 32 granules
-  blk.k = cv.text; blk.valid = 0; blk.score_idx = -1;
+  blk.k = cv.text; blk.meta = 0; blk.cid = -1; blk.off = 0; blk.score_idx = -1;
 
-  auto issue = [&](int n) {
+  // Visible rows of a granule once its metadata has arrived.
+  auto visible = [&](int meta, int cid, int off, int j) -> int {
+    if (meta >= 0) return meta;
+    int len;
+    if (meta == -1) len = T_t - j * GR;
+    else {
+      if (cid < 0) return 0;
+      len = T_a - cid * G.nc;
+      if (len > G.nc) len = G.nc;
+      len -= off;
+    }
+    return len <= 0 ? 0 : (len < GR ? len : GR);
+  };
+  // Queues the copies of granule n.  Granules with a static address are fetched before anyone knows how many of
+  // their rows are visible (the stores hold finite data everywhere, masked columns get probability 0); only text
+  // granules beyond the host's lower bound wait for the text length.
+  auto issue_copy = [&](int n) {
     if (n < n_my) {
       if ((n & 31) == 0) {
         const int nn = n + lane;
-        if (nn < n_my) blk = decode_granule(cv, a, li, b, it.h, role, ridx, first + nn * NW, T_t, T_a);
-        else { blk.valid = 0; blk.score_idx = -1; }
+        if (nn < n_my) blk = decode_granule(cv, a, li, it, first + nn * NW);
+        else { blk.meta = 0; blk.cid = -1; blk.score_idx = -1; }
+#ifdef WNW_PHASE_STAMPS
+        if (n == 0 && blk.k != nullptr) STAMP(12);
+#endif
       }
       const int src_lane = n & 31;
-      const int valid = __shfl_sync(0xffffffffu, blk.valid, src_lane);
-      const int sidx = __shfl_sync(0xffffffffu, blk.score_idx, src_lane);
+      const int meta = __shfl_sync(0xffffffffu, blk.meta, src_lane);
       const unsigned long long kp = __shfl_sync(0xffffffffu, (unsigned long long)blk.k, src_lane);
-      const int stage = n % NSTAGE;
-      if (lane == 0) ring[warp][stage] = make_int2(valid, sidx);
-      if (valid > 0) {
+      const int j = first + n * NW;
+      const bool is_text = j < G.n_tg;
+      int rows = meta;                                   // static count
+      if (meta == -2) rows = GR;                         // speculative: the whole granule
+      else if (meta == -1) rows = visible(-1, 0, 0, j);  // waits for the text length
+      if (rows > 0) {
         const bf16 *k = reinterpret_cast<const bf16 *>(kp);
-        const int j = first + n * NW;
-        const bool is_text = j < G.n_tg;
         const bf16 *v = k + (is_text ? v_delta_text : v_delta_audio);
         // the row of the token being generated comes from k_new/v_new and is stored into the text region here
-        const int new_row = (is_text && a.has_new) ? (T_t - 1) - j * GR : -1;
+        const int new_row = (meta == -1 && a.has_new) ? (T_t - 1) - j * GR : -1;
+        const int stage = n % NSTAGE;
         const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB;
 #pragma unroll
         for (int x = 0; x < GR * PPR / 32; ++x) {
           const int p = lane + 32 * x, row = p / PPR, pc = p % PPR;
-          const int ok = row < valid;
+          const int ok = row < rows;
           const int src_row = ok ? row : 0;
           const uint32_t dst = row * ROWB + ((pc ^ (row & 7)) << 4);
           const bf16 *ks = k + (long long)src_row * D + pc * 8, *vs = v + (long long)src_row * D + pc * 8;
@@ -214,10 +240,21 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     }
     cp_async_commit();
   };
+  // Publishes (visible rows, score index) of granule n for the compute step; may wait for the metadata loads.
+  auto issue_meta = [&](int n) {
+    if (n < n_my) {
+      const int src_lane = n & 31;
+      const int valid = __shfl_sync(0xffffffffu, visible(blk.meta, blk.cid, blk.off, first + (n - src_lane + lane) * NW), src_lane);
+      const int sidx = __shfl_sync(0xffffffffu, blk.score_idx, src_lane);
+      if (lane == 0) ring[warp][n % NSTAGE] = make_int2(valid, sidx);
+    }
+  };
 
 #pragma unroll
-  for (int n = 0; n < NSTAGE - 1; ++n) issue(n);
+  for (int n = 0; n < NSTAGE - 1; ++n) issue_copy(n);
   STAMP(1);
+#pragma unroll
+  for (int n = 0; n < NSTAGE - 1; ++n) issue_meta(n);
 
   for (int n = 0; n < n_my; ++n) {
     cp_async_wait<NSTAGE - 2>();
@@ -303,11 +340,19 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       }
     }
     __syncwarp();
-    issue(n + NSTAGE - 1);
+    issue_copy(n + NSTAGE - 1);
+    issue_meta(n + NSTAGE - 1);
   }
   cp_async_wait<0>();
   __syncthreads();
   STAMP(2);
+
+  // Programmatic dependent launch.  Everything below writes scratch that alternates by layer parity, so the
+  // previous layer's kernel must have completed (wait); after that the next layer's kernel may be scheduled and
+  // stream its K/V while this one merges (launch_dependents).  Because every CTA waits before it releases the
+  // next kernel, at most two layer kernels ever overlap and two scratch parities are enough.
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
 
   // ---- merge the warps' partial states through shared memory ----
   float2 *red_ml = reinterpret_cast<float2 *>(smem);                           // [NW][16]
@@ -323,30 +368,40 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       *reinterpret_cast<float2 *>(red_o + ((size_t)warp * g + r0 + 8) * D + t * 8 + cq) = make_float2(o[t][2], o[t][3]);
   }
   __syncthreads();
-  for (int idx = threadIdx.x; idx < g * D; idx += NW * 32) {
-    const int row = idx / D, col = idx - row * D;
+  // A head served by a single CTA is finished here (bf16 output, final max and denominator); otherwise the CTA
+  // leaves one partial in global memory.  The prefill scoring pass always leaves partials.
+  const HeadItems hi = a.head_items[it.i * G.Hkv + it.h];
+  const bool direct = hi.count == 1 && a.mode != ATTN_PREFILL;
+  for (int pr = threadIdx.x; pr < g * D / 2; pr += NW * 32) {
+    const int idx = pr * 2, row = idx / D;
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < NW; ++w) M = fmaxf(M, red_ml[w * 16 + row].x);
-    float acc = 0.f, L = 0.f;
+    float a0 = 0.f, a1 = 0.f, L = 0.f;
     if (M > -INFINITY) {
 #pragma unroll
       for (int w = 0; w < NW; ++w) {
         const float2 ml = red_ml[w * 16 + row];
         const float f = exp2f(ml.x - M);   // a warp without work has m = -inf -> factor 0
-        acc += red_o[((size_t)w * g + row) * D + col] * f;
+        const float2 x = *reinterpret_cast<const float2 *>(red_o + ((size_t)w * g + row) * D + (idx - row * D));
+        a0 += x.x * f; a1 += x.y * f;
         L += ml.y * f;
       }
     }
-    a.part_o[((long long)blockIdx.x * g + row) * D + col] = acc;
-    if (col == 0) a.part_ml[(long long)blockIdx.x * g + row] = make_float2(M, L);
+    if (direct) {
+      const float inv = L > 0.f ? 1.f / L : 0.f;
+      *reinterpret_cast<uint32_t *>(a.out + ((long long)it.i * G.Hq + (long long)it.h * g) * D + idx) = pack_bf16(a0 * inv, a1 * inv);
+      if (idx % D == 0) a.head_mz[(long long)it.i * G.Hq + it.h * g + row] = make_float2(M, L);
+    } else {
+      *reinterpret_cast<float2 *>(a.part_o + (long long)blockIdx.x * g * D + idx) = make_float2(a0, a1);
+      if (idx % D == 0) a.part_ml[(long long)blockIdx.x * g + row] = make_float2(M, L);
+    }
   }
   STAMP(3);
-  if (a.mode == ATTN_PREFILL || a.debug_stop == 1) return;
+  if (direct || a.mode == ATTN_PREFILL || a.debug_stop == 1) return;
 
   // ---- the CTA that finishes this head last merges its split partials ----
   __shared__ int s_flag;
-  const HeadItems hi = a.head_items[it.i * G.Hkv + it.h];
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -414,8 +469,21 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 template <int D, bool G16>
 static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
   const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2;
-  wnw_attn_kernel<D, G16><<<a.n_items, NW * 32, smem, st>>>(cv, a);
-  return cudaGetLastError();
+  InlineItems inl;
+  if (a.n_items <= INLINE_ITEMS_MAX && a.items_host) memcpy(inl.it, a.items_host, sizeof(WorkItem) * a.n_items);
+  else if (a.n_items <= INLINE_ITEMS_MAX) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)a.n_items, 1, 1);
+  cfg.blockDim = dim3(NW * 32, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  if (a.pdl) {  // let this launch begin before the previous kernel in the stream has drained (see griddepcontrol above)
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, wnw_attn_kernel<D, G16>, cv, a, inl);
 }
 
 template <int D, bool G16>

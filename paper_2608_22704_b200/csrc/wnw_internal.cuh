@@ -31,8 +31,11 @@ struct WorkItem {  // one CTA of the attention kernel; everything static about i
   int32_t ridx;    // index among the heads of that role (anchor-like launches: the KV head)
   int32_t T_a;     // audio tokens of the sequence
   int32_t C, S;    // chunks and slots of the sequence
+  int32_t T_hint;  // text rows known to exist when the list was built (a lower bound: text only grows)
 };
-struct HeadItems { int32_t first, count; };  // work items of one (active seq, KV head)
+constexpr int INLINE_ITEMS_MAX = 96;  // launches with at most this many items carry them in kernel parameters
+struct InlineItems { WorkItem it[INLINE_ITEMS_MAX]; };
+struct HeadItems { int32_t first, count; };  // work items (= split partials) of one (active seq, KV head)
 
 struct LayerInfo {
   int32_t n_anchor, n_tidal, n_fixed;
@@ -110,8 +113,10 @@ struct AttnArgs {
   int32_t score_on;      // write per-granule softmax-mass partials for anchor-like heads
   int32_t debug_stop;    // timing experiments only: 1 = return after the split partials, 2 = after the head merge
   const int32_t *active; // [n_active] sequence ids
-  const WorkItem *items;
+  const WorkItem *items;         // device copy of the items
+  const WorkItem *items_host;    // host copy (the launcher inlines short lists into the kernel parameters)
   int32_t n_items;
+  int32_t pdl;                   // launch with programmatic stream serialization (previous stream op is a layer kernel)
   const HeadItems *head_items;  // [n_active][Hkv] work items of each head (first is relative to `items`)
   const bf16 *q;         // [n_active][Hq][d]
   const bf16 *k_new, *v_new;    // [n_active][Hkv][d] or null

@@ -63,6 +63,7 @@ struct wnw_cache {
   std::vector<int> wl_T_a;
   std::vector<LayerWork> wl_layers;
   WorkItem *d_items = nullptr;
+  std::vector<WorkItem> h_items, h_pf_items;  // host copies (short lists are inlined into kernel parameters)
   HeadItems *d_head_items = nullptr;
   size_t d_items_cap = 0, d_head_items_cap = 0;
   int prefill_seq = -1, prefill_T_a = -1;
@@ -77,20 +78,23 @@ struct wnw_cache {
   float2 *pf_gran_em = nullptr;
   int part_cap_items = 0, n_aq_max = 0, n_ag_max = 0;
   // streams / events
-  cudaStream_t side = nullptr, last_stream = nullptr;
+  static constexpr int N_SIDE = 4;  // layers alternate between side streams so selection + recall keep pace with attention
+  cudaStream_t side[N_SIDE] = {nullptr, nullptr, nullptr, nullptr}, last_stream = nullptr;
   std::vector<cudaEvent_t> ev_layer_done, ev_side_done;
   std::vector<cudaEvent_t> ev_layer_done_cap, ev_side_done_cap;  // used only inside a stream capture
   std::vector<char> side_recorded;
   std::vector<size_t> sel_smem;   // dynamic shared memory of each layer's selection launch
   size_t gran_em_layer_stride = 0;
   bool step_capturing = false;
+  bool pdl_enabled = true;
   // captured step
   bool graph_capturing = false;
   cudaGraph_t graph = nullptr;
   cudaGraphExec_t graph_exec = nullptr;
   std::vector<int> graph_active, graph_prepared;
+  long long wl_epoch = 0, graph_epoch = -1;  // work-list generation the graph was captured against
   int graph_appended = 0;
-  int last_side_layer = -1;
+  int last_side_layer[N_SIDE] = {-1, -1, -1, -1};
   cudaEvent_t ev_place = nullptr, ev_step = nullptr;
   bool place_recorded = false, step_recorded = false;
   // timing
@@ -139,7 +143,8 @@ static void destroy_impl(wnw_cache *c) {
   for (void *p : c->dev_allocs) cudaFree(p);
   for (auto &s : c->seqs)
     if (s.mirror) cudaFreeHost(s.mirror);
-  if (c->side) cudaStreamDestroy(c->side);
+  for (auto sd : c->side)
+    if (sd) cudaStreamDestroy(sd);
   for (auto e : c->ev_layer_done) cudaEventDestroy(e);
   for (auto e : c->ev_side_done) cudaEventDestroy(e);
   for (auto e : c->ev_layer_done_cap) cudaEventDestroy(e);
@@ -208,6 +213,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
 #define CKC(call) do { wnw_status_t _s = (call); if (_s != WNW_OK) return fail(_s); } while (0)
 #define CKE(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { return fail(_e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA); } } while (0)
   cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
+  if (const char *e = getenv("WNW_PDL")) c->pdl_enabled = atoi(e) != 0;
   CKE(configure_attn_kernels());
   CKE(configure_select_kernel());
   const int L = cfg->n_layers, Hkv = cfg->n_kv_heads, d = cfg->head_dim, nc = cfg->chunk_tokens;
@@ -310,8 +316,9 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   c->n_aq_max = std::max(n_aq, 1);
   c->n_ag_max = std::max(G.C_max * G.gpc, 1);
   c->part_cap_items = 2 * c->n_sm + (int)B * Hkv + 16;
-  CKC(dev_alloc(c, &c->part_o, (size_t)c->part_cap_items * G.g * d, false));
-  CKC(dev_alloc(c, &c->part_ml, (size_t)c->part_cap_items * G.g, false));
+  // split partials and head counters alternate by layer parity: two consecutive layer kernels may overlap
+  CKC(dev_alloc(c, &c->part_o, 2 * (size_t)c->part_cap_items * G.g * d, false));
+  CKC(dev_alloc(c, &c->part_ml, 2 * (size_t)c->part_cap_items * G.g, false));
   // granule partials and final (M,Z) are per layer: the side-stream selection of layer l reads them while the
   // caller's stream already runs later layers
   c->gran_em_layer_stride = B * (size_t)c->n_aq_max * c->n_ag_max;
@@ -329,10 +336,10 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     if (fixed_part + per_chunk > cap) return fail(WNW_ERR_UNSUPPORTED);  // chunk tables too large for one CTA
     c->sel_smem[l] = std::min(cap, fixed_part + per_chunk * std::max(G.C_max, 1)) + 16;
   }
-  CKC(dev_alloc(c, &c->head_done, B * Hkv));
+  CKC(dev_alloc(c, &c->head_done, 2 * B * Hkv));
   c->seqs.assign(B, SeqHost{});
   c->mirror_ptrs.assign(B, nullptr);
-  CKE(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
+  for (auto &sd : c->side) CKE(cudaStreamCreateWithFlags(&sd, cudaStreamNonBlocking));
   c->ev_layer_done.resize(L); c->ev_side_done.resize(L); c->side_recorded.assign(L, 0);
   c->ev_layer_done_cap.resize(L); c->ev_side_done_cap.resize(L);
   for (int l = 0; l < L; ++l) {
@@ -359,20 +366,20 @@ extern "C" wnw_status_t wnw_destroy(wnw_cache_t *c) {
 // ---------------------------------------------------------------------------------------------
 // Work lists: split every (sequence, KV head) granule space into CTA-sized items
 // ---------------------------------------------------------------------------------------------
-// Granules per work item: enough items to fill the machine twice over, but never shorter than `min_gpi`
-// granules, because every item costs one partial in the merge that follows.
+// Granules per work item: enough items to fill the machine about twice over, never shorter than one granule per
+// warp, and a head is cut into at most ~32 pieces because the merge that follows reads every piece.
 static int granules_per_item(const wnw_cache *c, long long total_granules, int longest_head) {
   const int nw = attn_warps();
   int min_gpi = nw;
   if (const char *e = getenv("WNW_MIN_GRANULES_PER_ITEM")) min_gpi = std::max(nw, atoi(e) / nw * nw);
   const long long target = 2ll * c->n_sm;
   long long per = (total_granules + target - 1) / target;
-  per = std::max<long long>(per, (longest_head + 31) / 32);  // at most ~32 splits per head: the merge reads every split
+  per = std::max<long long>(per, (longest_head + 31) / 32);
   per = (per + nw - 1) / nw * nw;
   return (int)std::max<long long>(per, min_gpi);
 }
 
-// Appends the items of one layer for the given sequences.  audio_granules(role, b) gives each head's audio part.
+// Appends the items of one layer for the given sequences.
 static void build_layer_items(const wnw_cache *c, int layer, int mode, const std::vector<int> &seq_ids,
                               std::vector<WorkItem> &items, std::vector<HeadItems> &heads, LayerWork &lw) {
   const Geometry &G = c->geo;
@@ -396,13 +403,14 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   for (size_t i = 0; i < seq_ids.size(); ++i)
     for (int h = 0; h < G.Hkv; ++h) {
       const int n = n_gran[i * G.Hkv + h];
-      HeadItems hi{(int)items.size() - lw.first_item, 0};
+      const SeqHost &sq = c->seqs[seq_ids[i]];
       const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
       const int ridx = mode == ATTN_DECODE ? c->role_idx[layer * G.Hkv + h] : h;
-      for (int g0 = 0; g0 < n; g0 += gpi) {
-        items.push_back(WorkItem{(int)i, h, g0, std::min(n, g0 + gpi), seq_ids[i], role, ridx, c->seqs[seq_ids[i]].T_a, c->seqs[seq_ids[i]].C,
-                                 c->seqs[seq_ids[i]].S});
-        ++hi.count;
+      const int n_cta = std::max(1, (n + gpi - 1) / gpi);
+      HeadItems hi{(int)items.size() - lw.first_item, n_cta};
+      for (int x = 0; x < n_cta; ++x) {  // even contiguous ranges
+        const int g0 = (int)((long long)n * x / n_cta), g1 = (int)((long long)n * (x + 1) / n_cta);
+        items.push_back(WorkItem{(int)i, h, g0, g1, seq_ids[i], role, ridx, sq.T_a, sq.C, sq.S, sq.T_t});
       }
       heads.push_back(hi);
       lw.max_count = std::max(lw.max_count, hi.count);
@@ -439,6 +447,8 @@ static wnw_status_t ensure_worklists(wnw_cache *c) {
   CK(cudaMemcpy(c->d_head_items, heads.data(), heads.size() * sizeof(HeadItems), cudaMemcpyHostToDevice));
   std::vector<int32_t> act(c->active.begin(), c->active.end());
   CK(cudaMemcpy(c->d_active, act.data(), act.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+  c->h_items = items;
+  ++c->wl_epoch;
   c->wl_active = c->active;
   c->wl_T_a = T_a;
   return WNW_OK;
@@ -516,11 +526,13 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
       CK(cudaMemcpyAsync(c->d_pf_head_items, heads.data(), heads.size() * sizeof(HeadItems), cudaMemcpyHostToDevice, st));
       CK(cudaStreamSynchronize(st));  // the host vectors go out of scope
       c->pf_n_items = (int)items.size();
+      c->h_pf_items = items;
       c->prefill_seq = seq; c->prefill_T_a = T_a;
     }
     AttnArgs a{};
     a.mode = ATTN_PREFILL; a.layer = layer; a.li = c->layers[layer]; a.n_active = 1; a.has_new = 0; a.score_on = 1;
-    a.active = c->d_iota + seq; a.items = c->d_pf_items; a.n_items = c->pf_n_items; a.head_items = c->d_pf_head_items;
+    a.active = c->d_iota + seq; a.items = c->d_pf_items; a.items_host = c->h_pf_items.data(); a.n_items = c->pf_n_items;
+    a.head_items = c->d_pf_head_items;
     a.q = (const bf16 *)q_last_dev;
     a.anchor_base = c->stage; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
     a.part_o = c->part_o; a.part_ml = c->part_ml; a.gran_em = c->pf_gran_em; a.n_aq = G.Hq; a.n_ag_max = c->n_ag_max;
@@ -553,7 +565,8 @@ extern "C" wnw_status_t wnw_step_begin(wnw_cache_t *c, const int32_t *active, in
   c->active = want;
   wnw_status_t s = ensure_worklists(c);
   if (s != WNW_OK) return s;
-  c->in_step = true; c->next_layer = 0; c->appended = -1; c->last_side_layer = -1;
+  c->in_step = true; c->next_layer = 0; c->appended = -1;
+  for (int &ls : c->last_side_layer) ls = -1;
   return WNW_OK;
 }
 
@@ -601,13 +614,18 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   a.mode = tiered ? ATTN_DECODE : ATTN_FULL; a.layer = layer; a.li = li; a.n_active = n_active; a.has_new = has_new;
   a.score_on = tiered && li.n_anchor > 0;
   if (const char *e = getenv("WNW_DEBUG_STOP")) a.debug_stop = atoi(e);  // timing experiments only; breaks results
-  a.active = c->d_active; a.items = c->d_items + lw.first_item; a.n_items = lw.n_items;
+  a.active = c->d_active; a.items = c->d_items + lw.first_item; a.items_host = c->h_items.data() + lw.first_item;
+  a.n_items = lw.n_items;
   a.head_items = c->d_head_items + lw.head_items_off;
   a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
-  a.head_done = c->head_done; a.head_mz = head_mz_l; a.out = (bf16 *)out;
+  const size_t par = (size_t)(layer & 1);
+  a.head_done = c->head_done + par * G.max_batch * G.Hkv; a.head_mz = head_mz_l; a.out = (bf16 *)out;
   a.anchor_base = c->cv.anchor; a.anchor_seq_stride = G.anchor_seq_stride;
   a.anchor_head0 = tiered ? li.anchor_off : layer * G.Hkv;
-  a.part_o = c->part_o; a.part_ml = c->part_ml; a.gran_em = gran_em_l;
+  a.part_o = c->part_o + par * c->part_cap_items * G.g * G.d; a.part_ml = c->part_ml + par * c->part_cap_items * G.g;
+  a.gran_em = gran_em_l;
+  // overlap with the previous layer's kernel when that is what precedes this launch in the stream
+  a.pdl = layer > 0 && c->pdl_enabled;
   a.n_aq = std::max(li.n_anchor * G.g, 1); a.n_ag_max = c->n_ag_max;
   cudaEvent_t t0 = nullptr, t1 = nullptr;
   const bool timing = c->timing && !capturing;
@@ -637,12 +655,19 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
       sa.upd_src[u] = (int16_t)c->layers[sa.upd_layer[u]].src;
     }
     const bool inline_mode = c->cfg.recall_mode == WNW_RECALL_INLINE;
-    cudaStream_t ss = inline_mode ? st : c->side;
+    const int si = layer % wnw_cache::N_SIDE;
+    cudaStream_t ss = inline_mode ? st : c->side[si];
     cudaEvent_t ev_l = capturing ? c->ev_layer_done_cap[layer] : c->ev_layer_done[layer];
     cudaEvent_t ev_s = capturing ? c->ev_side_done_cap[layer] : c->ev_side_done[layer];
     if (!inline_mode) {
       CK(cudaEventRecord(ev_l, st));
       CK(cudaStreamWaitEvent(ss, ev_l, 0));
+      // a routed layer ranks by scores that an earlier layer's selection kernel wrote, maybe on the other side stream
+      for (int u = 0; u < li.upd_count; ++u) {
+        const int src = c->layers[c->upd_list[li.upd_first + u]].src;
+        if (src >= 0 && src != layer && src % wnw_cache::N_SIDE != si)
+          CK(cudaStreamWaitEvent(ss, capturing ? c->ev_side_done_cap[src] : c->ev_side_done[src], 0));
+      }
     }
     CK(launch_select(c->cv, sa, c->sel_smem[layer], ss));
     if (li.upd_count > 0)
@@ -651,7 +676,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     if (!inline_mode) {
       CK(cudaEventRecord(ev_s, ss));
       if (!capturing) c->side_recorded[layer] = 1;
-      c->last_side_layer = layer;
+      c->last_side_layer[si] = layer;
     }
   }
   c->appended = has_new;
@@ -676,8 +701,9 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const bool capturing = stream_is_capturing(st);
   if (capturing != c->step_capturing) return WNW_ERR_STATE;
-  if (capturing && c->last_side_layer >= 0 && c->cfg.recall_mode != WNW_RECALL_INLINE)
-    CK(cudaStreamWaitEvent(st, c->ev_side_done_cap[c->last_side_layer], 0));  // join the forked side stream into the graph
+  if (capturing && c->cfg.recall_mode != WNW_RECALL_INLINE)
+    for (int ls : c->last_side_layer)  // join the forked side streams into the graph
+      if (ls >= 0) CK(cudaStreamWaitEvent(st, c->ev_side_done_cap[ls], 0));
   CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1, st));
   if (!capturing) {
     CK(cudaEventRecord(c->ev_step, st));
@@ -715,7 +741,7 @@ extern "C" wnw_status_t wnw_graph_begin(wnw_cache_t *c, const int32_t *active, i
   }
   c->graph_prepared = c->active;
   // everything queued so far must be ordered before the first replay: drain now, the capture cannot wait on it
-  CK(cudaStreamSynchronize(c->side));
+  for (auto sd : c->side) CK(cudaStreamSynchronize(sd));
   if (c->last_stream != st) CK(cudaStreamSynchronize(c->last_stream));
   CK(cudaStreamSynchronize(st));
   CK(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
@@ -740,6 +766,7 @@ extern "C" wnw_status_t wnw_graph_end(wnw_cache_t *c, void *cuda_stream) {
   if (c->graph) { cudaGraphDestroy(c->graph); c->graph = nullptr; }
   c->graph = g;
   CK(cudaGraphInstantiate(&c->graph_exec, g, 0));
+  c->graph_epoch = c->wl_epoch;
   return WNW_OK;
 }
 
@@ -750,7 +777,8 @@ extern "C" wnw_status_t wnw_graph_launch(wnw_cache_t *c, void *cuda_stream) {
     if (c->seqs[b].placed_layers != c->geo.L) return WNW_ERR_STATE;
     if (c->graph_appended && c->seqs[b].T_t + 1 > c->cfg.max_text_tokens) return WNW_ERR_CAPACITY;
   }
-  if (c->wl_active != c->graph_active) return WNW_ERR_STATE;  // the work lists the graph points at were rebuilt
+  if (c->wl_active != c->graph_active || c->wl_layers.empty() || c->wl_epoch != c->graph_epoch)
+    return WNW_ERR_STATE;  // the work lists the graph points at were rebuilt or invalidated
   DeviceGuard guard(c->cfg.device);
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
@@ -771,7 +799,7 @@ extern "C" wnw_status_t wnw_graph_launch(wnw_cache_t *c, void *cuda_stream) {
 // ---------------------------------------------------------------------------------------------
 static wnw_status_t drain(wnw_cache *c) {
   CK(cudaStreamSynchronize(c->last_stream));
-  CK(cudaStreamSynchronize(c->side));
+  for (auto sd : c->side) CK(cudaStreamSynchronize(sd));
   return WNW_OK;
 }
 
