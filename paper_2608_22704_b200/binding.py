@@ -66,6 +66,7 @@ _SIGNATURES = {
     "wnw_get_kernel_time": [_vp, C.POINTER(C.c_float), C.POINTER(_i32)],
     "wnw_sync": [_vp],
     "wnw_measure_host_link": [_i32, C.c_int64, _i32, C.POINTER(C.c_double), C.POINTER(C.c_double)],
+    "wnw_attend_static": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, C.c_float, _i32, _vp],
 }
 
 
@@ -249,3 +250,12 @@ def wnw_measure_host_link(device=0, nbytes=256 << 20, reps=5):
     a, b = C.c_double(), C.c_double()
     _ck(lib().wnw_measure_host_link(device, nbytes, reps, C.byref(a), C.byref(b)), "wnw_measure_host_link")
     return a.value, b.value
+
+
+def wnw_attend_static(kv, n_tokens, q, out, softmax_scale=0.0, stream=None):
+    """Full attention of one query token over kv [n_kv_heads, 2, padded_tokens, head_dim] (bf16 CUDA tensor) with no
+    allocation inside the library; q, out: [n_q_heads, head_dim] bf16 CUDA tensors."""
+    n_kv, two, padded, d = kv.shape
+    assert two == 2
+    _ck(lib().wnw_attend_static(_ptr(kv), n_tokens, padded, _ptr(q), _ptr(out), q.shape[0], n_kv, d, softmax_scale,
+                                kv.device.index or 0, _stream(stream)), "wnw_attend_static")
