@@ -7,8 +7,8 @@
 //   tidal heads  : text + the chunks resident in the slot pool (gather by slot table);
 //   fixed heads  : text + the compacted prefill subset.
 // A CTA takes one work item = a granule range of one (sequence, KV head).  Each of its warps streams its
-// own granules (16 tokens x d, K and V) through a private cp.async pipeline into XOR-swizzled shared
-// memory and keeps a private online-softmax state; QK^T and PV run on mma.sync m16n8k16 with the g query
+// own granules (16 tokens x d, K and V) through a private TMA pipeline (cp.async.bulk.tensor, 128-byte
+// swizzle, one mbarrier per stage, issued by one elected lane) and keeps a private online-softmax state; QK^T and PV run on mma.sync m16n8k16 with the g query
 // heads of the group padded to the 16 rows of the tile (bf16 in, fp32 accumulate).  Warps merge through
 // shared memory and the CTA writes one (m, l, o[g][d]) partial.
 //
@@ -47,12 +47,32 @@ extern "C" int wnw_debug_clear_stamps() {
 #endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+// ---- mbarrier + TMA (no cluster multicast anywhere: every CTA fetches its own tiles) ----
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+// Bounded wait: gives up after about a second of SM clocks and reports it instead of hanging.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity))
+    if (clock64() - t0 > 2000000000ll) return false;
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -72,7 +92,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 struct GranDesc {
-  const bf16 *k;   // first K row of the granule (V row = k + v_delta); always a mapped address
+  int row;         // first K row of the granule in its store's 2-D view [rows][d] (V row = row + v_delta)
   int meta;        // >= 0: visible tokens, known statically; -1: text granule, needs the text length; -2: needs `cid`
   int cid;         // chunk id held by the slot / compact position (filled by a load that is not waited on here)
   int off;         // token offset of the granule inside its chunk
@@ -80,7 +100,7 @@ struct GranDesc {
 };
 
 // Maps granule j of a head's virtual key space [text capacity | audio] to memory WITHOUT waiting on any global load:
-// the address of every granule is static; what may be unknown yet is how many of its 16 rows are visible.
+// the row of every granule is static; what may be unknown yet is how many of its 16 rows are visible.
 __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const AttnArgs &a, const LayerInfo &li,
                                                    const WorkItem &it, int j) {
   const Geometry &G = cv.geo;
@@ -88,26 +108,26 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
   r.cid = -1; r.off = 0; r.score_idx = -1;
   if (j < G.n_tg) {
     const int tok0 = j * GR;
-    r.k = cv.text + text_off(G, it.b, a.layer, it.h, 0) + (long long)tok0 * G.d;
+    r.row = (int)(text_off(G, it.b, a.layer, it.h, 0) / G.d) + tok0;
     r.meta = tok0 + GR <= it.T_hint ? GR : -1;
     return r;
   }
   const int ag = j - G.n_tg, ci = ag / G.gpc, off = (ag - ci * G.gpc) * GR;
   r.off = off;
   if (it.role == ROLE_ANCHOR) {
-    r.k = a.anchor_base + anchor_off(G, a.anchor_seq_stride, it.b, a.anchor_head0 + it.ridx, 0) + (long long)(ci * G.nc + off) * G.d;
+    r.row = (int)(anchor_off(G, a.anchor_seq_stride, it.b, a.anchor_head0 + it.ridx, 0) / G.d) + ci * G.nc + off;
     int len = it.T_a - ci * G.nc;
     if (len > G.nc) len = G.nc;
     len -= off;
     r.meta = len <= 0 ? 0 : (len < GR ? len : GR);
     if (a.score_on) r.score_idx = ag;
   } else if (it.role == ROLE_TIDAL) {
-    r.k = cv.pool + pool_off(G, li, it.b, ci, it.ridx, 0) + (long long)off * G.d;
+    r.row = (int)(pool_off(G, li, it.b, ci, it.ridx, 0) / G.d) + off;
     r.cid = cv.slot_chunk[((long long)it.b * G.L + a.layer) * G.S_max + ci];
     r.meta = -2;
   } else {
     const long long fh = (long long)it.b * G.F_tot + li.fixed_off + it.ridx;
-    r.k = cv.fixed + fixed_off(G, li, it.b, it.ridx, 0) + (long long)(ci * G.nc + off) * G.d;
+    r.row = (int)(fixed_off(G, li, it.b, it.ridx, 0) / G.d) + ci * G.nc + off;
     r.cid = cv.fixed_chunks[fh * G.S_max + ci];
     r.meta = -2;
   }
@@ -117,17 +137,20 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
 template <int D, bool G16>
 __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant__ CacheView cv,
                                                            const __grid_constant__ AttnArgs a,
-                                                           const __grid_constant__ InlineItems inl) {
-  extern __shared__ __align__(128) unsigned char smem[];
+                                                           const __grid_constant__ InlineItems inl,
+                                                           const __grid_constant__ TmaMaps maps) {
+  extern __shared__ unsigned char smem_raw[];
+  // TMA boxes with the 128-byte swizzle must start on a 1024-byte boundary of the shared window
+  unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const Geometry &G = cv.geo;
-  constexpr int ROWB = D * 2;             // bytes per K or V row
-  constexpr int TILEB = GR * ROWB;        // bytes per K (or V) granule
+  constexpr int HALVES = D / 64;          // a K (or V) granule is HALVES boxes of 16 rows x 128 bytes
+  constexpr int HALFB = GR * 128;         // bytes per box
+  constexpr int TILEB = HALVES * HALFB;   // bytes per K (or V) granule
   constexpr int PPR = D / 8;              // 16-byte pieces per row
   constexpr int KK = D / 16;              // k16 steps of QK^T; also pairs of n8 tiles of PV
   constexpr int NQ = G16 ? 4 : 2;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr size_t SMEM_TOTAL = (size_t)NW * NSTAGE * 2 * GR * D * 2;
   STAMP(0);
   // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
   const WorkItem it = a.n_items <= INLINE_ITEMS_MAX ? inl.it[blockIdx.x] : a.items[blockIdx.x];
@@ -138,45 +161,29 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 #ifdef WNW_PHASE_STAMPS
   if (it.g0 >= 0) STAMP(10);
 #endif
-  long long v_delta_audio;
-  if (role == ROLE_ANCHOR) v_delta_audio = (long long)G.T_a_pad * G.d;
-  else if (role == ROLE_TIDAL) v_delta_audio = (long long)G.nc * G.d;
-  else v_delta_audio = (long long)G.S_max * G.nc * G.d;
-  const long long v_delta_text = (long long)G.T_cap_pad * G.d;
+  int v_delta_audio;  // rows between a granule's K and V rows
+  const CUtensorMap *map_audio;
+  if (role == ROLE_ANCHOR) { v_delta_audio = G.T_a_pad; map_audio = &maps.anchor; }
+  else if (role == ROLE_TIDAL) { v_delta_audio = G.nc; map_audio = &maps.pool; }
+  else { v_delta_audio = G.S_max * G.nc; map_audio = &maps.fixed; }
+  const int v_delta_text = G.T_cap_pad;
 
-  __shared__ int2 ring[NW][NSTAGE];
-  unsigned char *my_smem = smem + (size_t)warp * NSTAGE * 2 * TILEB;
-  const uint32_t my_base = smem_u32(my_smem);
-
-  // ---- Q fragments (rows >= g are zero padding) ----
-  const int r0 = lane >> 2, cq = (lane & 3) * 2;
-  uint32_t qa[KK][NQ];
-  {
-    const bf16 *qb = a.q + ((long long)it.i * G.Hq + (long long)it.h * g) * D;
+  __shared__ int2 ring[NW][NSTAGE];                              // per stage: visible rows | loaded << 8, score index
+  __shared__ __align__(8) unsigned long long bars[NW][NSTAGE];   // one mbarrier per stage, producer = consumer = this warp
+  const uint32_t my_base = smem_u32(smem + (size_t)warp * NSTAGE * 2 * TILEB);
+  if (lane == 0) {
 #pragma unroll
-    for (int kk = 0; kk < KK; ++kk) {
-      qa[kk][0] = r0 < g ? *reinterpret_cast<const uint32_t *>(qb + r0 * D + kk * 16 + cq) : 0u;
-      qa[kk][1] = r0 < g ? *reinterpret_cast<const uint32_t *>(qb + r0 * D + kk * 16 + 8 + cq) : 0u;
-      if (G16) {
-        qa[kk][2] = r0 + 8 < g ? *reinterpret_cast<const uint32_t *>(qb + (r0 + 8) * D + kk * 16 + cq) : 0u;
-        qa[kk][3] = r0 + 8 < g ? *reinterpret_cast<const uint32_t *>(qb + (r0 + 8) * D + kk * 16 + 8 + cq) : 0u;
-      }
-    }
+    for (int st = 0; st < NSTAGE; ++st) mbar_init(smem_u32(&bars[warp][st]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    fence_proxy_async();
   }
-
-#ifdef WNW_PHASE_STAMPS
-  if (my_base != 0) STAMP(11);
-#endif
-  float o[D / 8][4];
-#pragma unroll
-  for (int t = 0; t < D / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  __syncwarp();
 
   const int first = it.g0 + warp;
   const int n_my = first < it.g1 ? (it.g1 - first + NW - 1) / NW : 0;
 
   GranDesc blk;  // descriptor this lane decoded for the current block of 32 granules
-  blk.k = cv.text; blk.meta = 0; blk.cid = -1; blk.off = 0; blk.score_idx = -1;
+  blk.row = 0; blk.meta = 0; blk.cid = -1; blk.off = 0; blk.score_idx = -1;
 
   // Visible rows of a granule once its metadata has arrived.
   auto visible = [&](int meta, int cid, int off, int j) -> int {
@@ -191,96 +198,128 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     }
     return len <= 0 ? 0 : (len < GR ? len : GR);
   };
-  // Queues the copies of granule n.  Granules with a static address are fetched before anyone knows how many of
-  // their rows are visible (the stores hold finite data everywhere, masked columns get probability 0); only text
-  // granules beyond the host's lower bound wait for the text length.
-  auto issue_copy = [&](int n) {
-    if (n < n_my) {
-      if ((n & 31) == 0) {
-        const int nn = n + lane;
-        if (nn < n_my) blk = decode_granule(cv, a, li, it, first + nn * NW);
-        else { blk.meta = 0; blk.cid = -1; blk.score_idx = -1; }
+  // Queues the TMA copies of granule n (K and V, all 16 rows).  Granules with a static row are fetched before anyone
+  // knows how many of their rows are visible (the stores hold finite data everywhere; masked columns get probability
+  // 0); only text granules beyond the host's lower bound wait for the text length.  Returns whether a copy was queued.
+  auto issue_copy = [&](int n) -> bool {
+    if (n >= n_my) return false;
+    if ((n & 31) == 0) {
+      const int nn = n + lane;
+      if (nn < n_my) blk = decode_granule(cv, a, li, it, first + nn * NW);
+      else { blk.meta = 0; blk.cid = -1; blk.score_idx = -1; }
 #ifdef WNW_PHASE_STAMPS
-        if (n == 0 && blk.k != nullptr) STAMP(12);
+      if (n == 0 && blk.row >= 0) STAMP(12);
 #endif
-      }
-      const int src_lane = n & 31;
-      const int meta = __shfl_sync(0xffffffffu, blk.meta, src_lane);
-      const unsigned long long kp = __shfl_sync(0xffffffffu, (unsigned long long)blk.k, src_lane);
-      const int j = first + n * NW;
-      const bool is_text = j < G.n_tg;
-      int rows = meta;                                   // static count
-      if (meta == -2) rows = GR;                         // speculative: the whole granule
-      else if (meta == -1) rows = visible(-1, 0, 0, j);  // waits for the text length
-      if (rows > 0) {
-        const bf16 *k = reinterpret_cast<const bf16 *>(kp);
-        const bf16 *v = k + (is_text ? v_delta_text : v_delta_audio);
-        // the row of the token being generated comes from k_new/v_new and is stored into the text region here
-        const int new_row = (meta == -1 && a.has_new) ? (T_t - 1) - j * GR : -1;
-        const int stage = n % NSTAGE;
-        const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB;
+    }
+    const int src_lane = n & 31;
+    const int meta = __shfl_sync(0xffffffffu, blk.meta, src_lane);
+    const int row = __shfl_sync(0xffffffffu, blk.row, src_lane);
+    const int j = first + n * NW;
+    const bool is_text = j < G.n_tg;
+    bool load = meta != 0;
+    if (meta == -1) load = visible(-1, 0, 0, j) > 0;  // waits for the text length
+    if (load && lane == 0) {
+      const int stage = n % NSTAGE;
+      const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB, bar = smem_u32(&bars[warp][stage]);
+      const CUtensorMap *map = is_text ? &maps.text : map_audio;
+      const int vrow = row + (is_text ? v_delta_text : v_delta_audio);
+      fence_proxy_async();  // the stage was last read through the generic proxy (ldmatrix)
+      mbar_expect_tx(bar, 2 * TILEB);
 #pragma unroll
-        for (int x = 0; x < GR * PPR / 32; ++x) {
-          const int p = lane + 32 * x, row = p / PPR, pc = p % PPR;
-          const int ok = row < rows;
-          const int src_row = ok ? row : 0;
-          const uint32_t dst = row * ROWB + ((pc ^ (row & 7)) << 4);
-          const bf16 *ks = k + (long long)src_row * D + pc * 8, *vs = v + (long long)src_row * D + pc * 8;
-          if (row == new_row) {
-            const long long noff = ((long long)it.i * G.Hkv + it.h) * D + pc * 8;
-            const uint4 kn = *reinterpret_cast<const uint4 *>(a.k_new + noff), vn = *reinterpret_cast<const uint4 *>(a.v_new + noff);
-            *reinterpret_cast<uint4 *>(const_cast<bf16 *>(ks)) = kn;
-            *reinterpret_cast<uint4 *>(const_cast<bf16 *>(vs)) = vn;
-            ks = a.k_new + noff; vs = a.v_new + noff;
-          }
-          cp_async16(sK + dst, ks, ok ? 16 : 0);
-          cp_async16(sV + dst, vs, ok ? 16 : 0);
-        }
+      for (int hf = 0; hf < HALVES; ++hf) {
+        tma_load_2d(sK + hf * HALFB, map, hf * 64, row, bar);
+        tma_load_2d(sV + hf * HALFB, map, hf * 64, vrow, bar);
       }
     }
-    cp_async_commit();
+    return load;
   };
-  // Publishes (visible rows, score index) of granule n for the compute step; may wait for the metadata loads.
-  auto issue_meta = [&](int n) {
+  // Publishes (visible rows, loaded, score index) of granule n for the compute step; may wait for the metadata loads.
+  auto issue_meta = [&](int n, bool loaded) {
     if (n < n_my) {
       const int src_lane = n & 31;
       const int valid = __shfl_sync(0xffffffffu, visible(blk.meta, blk.cid, blk.off, first + (n - src_lane + lane) * NW), src_lane);
       const int sidx = __shfl_sync(0xffffffffu, blk.score_idx, src_lane);
-      if (lane == 0) ring[warp][n % NSTAGE] = make_int2(valid, sidx);
+      if (lane == 0) ring[warp][n % NSTAGE] = make_int2(valid | (loaded ? 256 : 0), sidx);
     }
   };
 
+  bool pro_loaded[NSTAGE - 1];
 #pragma unroll
-  for (int n = 0; n < NSTAGE - 1; ++n) issue_copy(n);
+  for (int n = 0; n < NSTAGE - 1; ++n) pro_loaded[n] = issue_copy(n);
   STAMP(1);
+
+  // ---- Q fragments (rows >= g are zero padding); loaded after the first K/V copies are in flight ----
+  const int r0 = lane >> 2, cq = (lane & 3) * 2;
+  uint32_t qa[KK][NQ];
+  {
+    const bf16 *qb = a.q + ((long long)it.i * G.Hq + (long long)it.h * g) * D;
 #pragma unroll
-  for (int n = 0; n < NSTAGE - 1; ++n) issue_meta(n);
+    for (int kk = 0; kk < KK; ++kk) {
+      qa[kk][0] = r0 < g ? *reinterpret_cast<const uint32_t *>(qb + r0 * D + kk * 16 + cq) : 0u;
+      qa[kk][1] = r0 < g ? *reinterpret_cast<const uint32_t *>(qb + r0 * D + kk * 16 + 8 + cq) : 0u;
+      if (G16) {
+        qa[kk][2] = r0 + 8 < g ? *reinterpret_cast<const uint32_t *>(qb + (r0 + 8) * D + kk * 16 + cq) : 0u;
+        qa[kk][3] = r0 + 8 < g ? *reinterpret_cast<const uint32_t *>(qb + (r0 + 8) * D + kk * 16 + 8 + cq) : 0u;
+      }
+    }
+  }
+#pragma unroll
+  for (int n = 0; n < NSTAGE - 1; ++n) issue_meta(n, pro_loaded[n]);
+
+  float o[D / 8][4];
+#pragma unroll
+  for (int t = 0; t < D / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  uint32_t phase_bits = 0;   // parity of each stage's barrier
+  bool timed_out = false;
 
   for (int n = 0; n < n_my; ++n) {
-    cp_async_wait<NSTAGE - 2>();
     __syncwarp();
     const int stage = n % NSTAGE;
     const int2 rg = ring[warp][stage];
-    const int valid = rg.x;
-    if (valid > 0) {
+    const int valid = rg.x & 255;
+    if (rg.x & 256) {  // a copy was queued for this stage: wait for its bytes (bounded)
+      if (!mbar_wait(smem_u32(&bars[warp][stage]), (phase_bits >> stage) & 1u)) { timed_out = true; break; }
+      phase_bits ^= 1u << stage;
+    }
+    if (valid > 0 && !timed_out) {
       const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB;
+      // the row of the token being generated: take it from k_new/v_new and store it into the text region
+      const int j = first + n * NW;
+      if (a.has_new && j < G.n_tg && (T_t - 1) / GR == j) {
+        const int nr = (T_t - 1) - j * GR;
+        if (lane < 2 * PPR) {
+          const int kv = lane / PPR, pc = lane - kv * PPR;
+          const long long noff = ((long long)it.i * G.Hkv + it.h) * D + pc * 8;
+          const uint4 val = *reinterpret_cast<const uint4 *>((kv ? a.v_new : a.k_new) + noff);
+          *reinterpret_cast<uint4 *>(cv.text + text_off(G, b, a.layer, it.h, kv) + (long long)(T_t - 1) * D + pc * 8) = val;
+          const uint32_t dst = (kv ? sV : sK) + (pc >> 3) * HALFB + nr * 128 + (((pc & 7) ^ (nr & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(dst), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+        }
+        __syncwarp();
+      }
       float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+      float s2[4] = {0.f, 0.f, 0.f, 0.f}, s3[4] = {0.f, 0.f, 0.f, 0.f};   // odd k-steps: shorter dependent mma chains
       {
         const int mtx = lane >> 3, row = ((mtx >> 1) << 3) + (lane & 7);
-        const uint32_t rowaddr = sK + row * ROWB;
+        const uint32_t rowaddr = sK + row * 128;
 #pragma unroll
         for (int kk = 0; kk < KK; ++kk) {
           uint32_t bk[4];
           const int piece = 2 * kk + (mtx & 1);
-          ldsm_x4(bk, rowaddr + ((piece ^ (row & 7)) << 4));
+          ldsm_x4(bk, rowaddr + (kk >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4));
+          float (&t0)[4] = (kk & 1) ? s2 : s0;
+          float (&t1)[4] = (kk & 1) ? s3 : s1;
           if (G16) {
-            mma16816(s0, qa[kk][0], qa[kk][2], qa[kk][1], qa[kk][3], bk[0], bk[1]);
-            mma16816(s1, qa[kk][0], qa[kk][2], qa[kk][1], qa[kk][3], bk[2], bk[3]);
+            mma16816(t0, qa[kk][0], qa[kk][2], qa[kk][1], qa[kk][3], bk[0], bk[1]);
+            mma16816(t1, qa[kk][0], qa[kk][2], qa[kk][1], qa[kk][3], bk[2], bk[3]);
           } else {
-            mma16816(s0, qa[kk][0], 0u, qa[kk][1], 0u, bk[0], bk[1]);
-            mma16816(s1, qa[kk][0], 0u, qa[kk][1], 0u, bk[2], bk[3]);
+            mma16816(t0, qa[kk][0], 0u, qa[kk][1], 0u, bk[0], bk[1]);
+            mma16816(t1, qa[kk][0], 0u, qa[kk][1], 0u, bk[2], bk[3]);
           }
         }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { s0[e] += s2[e]; s1[e] += s3[e]; }
       }
       // ---- online softmax in log2 units, fp32; columns = tokens cq, cq+1, 8+cq, 9+cq ----
       const float sc = G.scale_log2;
@@ -328,22 +367,24 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       }
       {
         const int mtx = lane >> 3, row = ((mtx & 1) << 3) + (lane & 7);
-        const uint32_t rowaddr = sV + row * ROWB;
+        const uint32_t rowaddr = sV + row * 128;
 #pragma unroll
         for (int t2 = 0; t2 < KK; ++t2) {
           uint32_t bv[4];
           const int piece = 2 * t2 + (mtx >> 1);
-          ldsm_x4_t(bv, rowaddr + ((piece ^ (row & 7)) << 4));
+          ldsm_x4_t(bv, rowaddr + (t2 >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4));
           mma16816(o[2 * t2], pa0, pa1, pa2, pa3, bv[0], bv[1]);
           mma16816(o[2 * t2 + 1], pa0, pa1, pa2, pa3, bv[2], bv[3]);
         }
       }
     }
     __syncwarp();
-    issue_copy(n + NSTAGE - 1);
-    issue_meta(n + NSTAGE - 1);
+    {
+      const bool ld = issue_copy(n + NSTAGE - 1);
+      issue_meta(n + NSTAGE - 1, ld);
+    }
   }
-  cp_async_wait<0>();
+  if (timed_out && lane == 0) atomicOr(cv.status, STATUS_TIMEOUT);
   __syncthreads();
   STAMP(2);
 
@@ -468,7 +509,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 
 template <int D, bool G16>
 static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
-  const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2;
+  const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024;  // + slack to align the stages to the swizzle atom
+  if (!a.maps) return cudaErrorInvalidValue;
   InlineItems inl;
   if (a.n_items <= INLINE_ITEMS_MAX && a.items_host) memcpy(inl.it, a.items_host, sizeof(WorkItem) * a.n_items);
   else if (a.n_items <= INLINE_ITEMS_MAX) return cudaErrorInvalidValue;
@@ -483,13 +525,40 @@ static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
   }
-  return cudaLaunchKernelEx(&cfg, wnw_attn_kernel<D, G16>, cv, a, inl);
+  return cudaLaunchKernelEx(&cfg, wnw_attn_kernel<D, G16>, cv, a, inl, *a.maps);
+}
+
+// ---- TMA descriptors ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d) {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {  // the driver entry point is looked up at run time: the library does not link against libcuda
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess || !p ||
+        qres != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    fn = (EncodeTiledFn)p;
+  }
+  if (rows < 1) rows = 1;
+  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)d * 2};          // bytes between rows
+  const cuuint32_t box[2] = {64, (cuuint32_t)GR};              // 128 bytes x 16 rows
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int D, bool G16>
 static cudaError_t configure_t() {
   return cudaFuncSetAttribute(wnw_attn_kernel<D, G16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)((size_t)NW * NSTAGE * 2 * GR * D * 2));
+                              (int)((size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024));
 }
 // Opt-in shared-memory sizes, set once per device at cache creation (never during a stream capture).
 cudaError_t configure_attn_kernels() {

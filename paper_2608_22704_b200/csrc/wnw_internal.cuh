@@ -1,6 +1,7 @@
 // Internal device-side view of a WnW cache and launch-argument structs shared by the kernels
 // and the host runtime.  Nothing here is part of the public ABI (see include/wnw.h).
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -21,6 +22,7 @@ constexpr int ROLE_ANCHOR = 0, ROLE_TIDAL = 1, ROLE_FIXED = 2;
 constexpr int STATUS_NO_VICTIM = 1;     // table update found no evictable slot
 constexpr int STATUS_BAD_TABLE = 2;     // slot/chunk id out of range
 constexpr int STATUS_NONFINITE = 4;     // non-finite chunk score
+constexpr int STATUS_TIMEOUT = 8;       // a bounded wait on a TMA barrier gave up
 
 struct WorkItem {  // one CTA of the attention kernel; everything static about it is precomputed on the host
   int32_t i;       // index into the active-sequence list
@@ -104,6 +106,10 @@ __host__ __device__ inline size_t select_ws_bytes(int C, int S) {
 // ---- attention launch ----
 enum { ATTN_DECODE = 0, ATTN_FULL = 1, ATTN_PREFILL = 2 };
 
+// TMA descriptors of the K/V stores, each viewed as a 2-D bf16 tensor [rows][d] with 16 x 64-element boxes and the
+// 128-byte swizzle.  `anchor` is whichever store plays the contiguous full-audio role in the launch.
+struct TmaMaps { CUtensorMap text, anchor, pool, fixed; };
+
 struct AttnArgs {
   int32_t mode;          // ATTN_*
   int32_t layer;
@@ -115,6 +121,7 @@ struct AttnArgs {
   const int32_t *active; // [n_active] sequence ids
   const WorkItem *items;         // device copy of the items
   const WorkItem *items_host;    // host copy (the launcher inlines short lists into the kernel parameters)
+  const TmaMaps *maps;           // host pointer; passed to the kernel by value
   int32_t n_items;
   int32_t pdl;                   // launch with programmatic stream serialization (previous stream op is a layer kernel)
   const HeadItems *head_items;  // [n_active][Hkv] work items of each head (first is relative to `items`)
@@ -162,6 +169,8 @@ cudaError_t launch_place_gather(const CacheView &cv, int b, int layer, int full_
                                 cudaStream_t st);
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
 cudaError_t configure_attn_kernels();
+// Encodes the descriptor of one store: base (device), rows, head_dim.  Returns false if the driver refuses.
+bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d);
 cudaError_t configure_select_kernel();
 constexpr int SELECT_SMEM_CAP = 200 * 1024;  // dynamic shared memory the selection kernel may be launched with
 int attn_warps();  // warps per attention CTA (granules per work item should be a multiple)

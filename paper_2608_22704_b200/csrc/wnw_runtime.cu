@@ -53,6 +53,7 @@ struct wnw_cache {
   std::vector<void *> dev_allocs;
   std::vector<bf16 *> mirror_ptrs;  // host copy of cv.mirror
   bf16 *stage = nullptr;
+  TmaMaps maps_decode, maps_prefill;  // TMA descriptors: cache stores; prefill scoring reads the staging copy as `anchor`
   int32_t *d_iota = nullptr, *d_active = nullptr;
   // step state
   std::vector<int> active;
@@ -337,6 +338,19 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     c->sel_smem[l] = std::min(cap, fixed_part + per_chunk * std::max(G.C_max, 1)) + 16;
   }
   CKC(dev_alloc(c, &c->head_done, 2 * B * Hkv));
+  {
+    const unsigned long long r_text = B * (unsigned long long)G.text_seq_stride / d, r_anchor = B * (unsigned long long)G.anchor_seq_stride / d,
+                             r_pool = B * (unsigned long long)G.pool_seq_stride / d, r_fixed = B * (unsigned long long)G.fixed_seq_stride / d,
+                             r_stage = (unsigned long long)Hkv * 2 * G.T_a_pad;
+    if (std::max({r_text, r_anchor, r_pool, r_fixed}) >= (1ull << 31)) return fail(WNW_ERR_UNSUPPORTED);  // rows are 32-bit TMA coordinates
+    bool ok = encode_store_map(&c->maps_decode.text, cv.text, r_text, d);
+    ok = ok && encode_store_map(&c->maps_decode.anchor, cv.anchor, r_anchor, d);
+    ok = ok && encode_store_map(&c->maps_decode.pool, r_pool ? (void *)cv.pool : (void *)cv.text, r_pool ? r_pool : r_text, d);
+    ok = ok && encode_store_map(&c->maps_decode.fixed, r_fixed ? (void *)cv.fixed : (void *)cv.text, r_fixed ? r_fixed : r_text, d);
+    c->maps_prefill = c->maps_decode;
+    ok = ok && encode_store_map(&c->maps_prefill.anchor, c->stage, r_stage, d);
+    if (!ok) return fail(WNW_ERR_CUDA);
+  }
   c->seqs.assign(B, SeqHost{});
   c->mirror_ptrs.assign(B, nullptr);
   for (auto &sd : c->side) CKE(cudaStreamCreateWithFlags(&sd, cudaStreamNonBlocking));
@@ -531,7 +545,7 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
     }
     AttnArgs a{};
     a.mode = ATTN_PREFILL; a.layer = layer; a.li = c->layers[layer]; a.n_active = 1; a.has_new = 0; a.score_on = 1;
-    a.active = c->d_iota + seq; a.items = c->d_pf_items; a.items_host = c->h_pf_items.data(); a.n_items = c->pf_n_items;
+    a.active = c->d_iota + seq; a.items = c->d_pf_items; a.items_host = c->h_pf_items.data(); a.n_items = c->pf_n_items; a.maps = &c->maps_prefill;
     a.head_items = c->d_pf_head_items;
     a.q = (const bf16 *)q_last_dev;
     a.anchor_base = c->stage; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
@@ -615,7 +629,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   a.score_on = tiered && li.n_anchor > 0;
   if (const char *e = getenv("WNW_DEBUG_STOP")) a.debug_stop = atoi(e);  // timing experiments only; breaks results
   a.active = c->d_active; a.items = c->d_items + lw.first_item; a.items_host = c->h_items.data() + lw.first_item;
-  a.n_items = lw.n_items;
+  a.n_items = lw.n_items; a.maps = &c->maps_decode;
   a.head_items = c->d_head_items + lw.head_items_off;
   a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
   const size_t par = (size_t)(layer & 1);

@@ -113,7 +113,12 @@ extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, 
   if (cudaMemcpyAsync(scr + OFF_HEAD_ITEMS, heads.data(), heads.size() * sizeof(HeadItems), cudaMemcpyHostToDevice, st) !=
       cudaSuccess) { cudaGetLastError(); return WNW_ERR_CUDA; }
 
+  // descriptor of the caller's buffer (a host-side encode, no allocation); every role points at it
+  TmaMaps maps;
+  if (!encode_store_map(&maps.anchor, kv_dev, (unsigned long long)n_kv_heads * 2 * padded_tokens, head_dim)) return WNW_ERR_CUDA;
+  maps.text = maps.pool = maps.fixed = maps.anchor;
   AttnArgs a{};
+  a.maps = &maps;
   a.mode = ATTN_FULL; a.layer = 0; a.n_active = 1; a.has_new = 0; a.score_on = 0;
   a.items = nullptr; a.items_host = items.data(); a.n_items = (int)items.size(); a.pdl = 0;
   a.head_items = reinterpret_cast<const HeadItems *>(scr + OFF_HEAD_ITEMS);
