@@ -332,14 +332,14 @@ def run_ours(args, rank, world, local_rank):
     total = W + R + K
     w = make_workload(args.workload, total, 0)
     job = Job(w, seed=rank, device=dev, wnw=wnw)
-    job.create("wnw", wnw.WNW_MODE_TIERED)
+    job.create("wnw", wnw.WNW_MODE_FULL if args.quick_full else wnw.WNW_MODE_TIERED, recall_mode=args.recall_mode)
     if args.quick:   # profiler mode: the WnW steps only, nothing else launched
         job.place_all(["wnw"])
         for t in range(W):
-            job.step("wnw", t)
+            job.step("wnw", t, full=args.quick_full)
         torch.cuda.synchronize(dev)
         wnw.wnw_set_kernel_timing(job.caches["wnw"], True)
-        per_step = job.timed_steps("wnw", W, K, flush=not args.no_flush, graph=not args.eager)
+        per_step = job.timed_steps("wnw", W, K, full=args.quick_full, flush=not args.no_flush, graph=not args.eager)
         ms, n = wnw.wnw_get_kernel_time(job.caches["wnw"])
         print(json.dumps({"quick": True, "workload": w.name, "ms_per_step": sum(per_step) / K, "steps": K,
                           "attn_us_per_launch": ms * 1e3 / max(n, 1)}), flush=True)
@@ -524,6 +524,8 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3", "prof"])
     ap.add_argument("--quick", action="store_true", help="only the WnW steps (for profiler captures); prints a short line")
     ap.add_argument("--no-flush", action="store_true", help="with --quick: do not flush L2 between steps")
+    ap.add_argument("--recall-mode", type=int, default=0, help="with --quick: 0 side stream, 1 inline, 2 copies skipped")
+    ap.add_argument("--quick-full", action="store_true", help="with --quick: time the full-cache comparison path instead")
     ap.add_argument("--eager", action="store_true", help="issue every layer eagerly instead of replaying a captured step")
     ap.add_argument("--roofline-steps", type=int, default=16)
     ap.add_argument("--oracle-layers", type=int, default=6, help="layers of sequence 0 the CPU baseline samples (0 = skip)")

@@ -26,10 +26,12 @@
 
 namespace wnw {
 
-constexpr int NW = 8;      // warps per CTA
+constexpr int NW_LAT = 8;  // warps per CTA when the launch fits one wave (latency regime): 1 CTA per SM
+constexpr int NW_THR = 8;  // warps per CTA otherwise (throughput regime).  A 4-warp, 2-CTAs-per-SM variant measured no faster (CTAs of
+                           // a wave run their prologue, streaming and merge phases in lock-step), so both regimes use 8 warps.
 constexpr int NSTAGE = 3;  // granules in flight per warp
 
-int attn_warps() { return NW; }
+int attn_warps(bool throughput) { return throughput ? NW_THR : NW_LAT; }
 
 // Phase stamps for latency studies: compiled in only with -DWNW_PHASE_STAMPS (never in the product build).
 #ifdef WNW_PHASE_STAMPS
@@ -134,7 +136,7 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
   return r;
 }
 
-template <int D, bool G16>
+template <int D, bool G16, int NW>
 __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant__ CacheView cv,
                                                            const __grid_constant__ AttnArgs a,
                                                            const __grid_constant__ InlineItems inl,
@@ -507,7 +509,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   STAMP(5);
 }
 
-template <int D, bool G16>
+template <int D, bool G16, int NW>
 static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
   const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024;  // + slack to align the stages to the swizzle atom
   if (!a.maps) return cudaErrorInvalidValue;
@@ -525,7 +527,7 @@ static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
   }
-  return cudaLaunchKernelEx(&cfg, wnw_attn_kernel<D, G16>, cv, a, inl, *a.maps);
+  return cudaLaunchKernelEx(&cfg, wnw_attn_kernel<D, G16, NW>, cv, a, inl, *a.maps);
 }
 
 // ---- TMA descriptors ----
@@ -555,25 +557,34 @@ bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long row
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool G16>
+template <int D, bool G16, int NW>
 static cudaError_t configure_t() {
-  return cudaFuncSetAttribute(wnw_attn_kernel<D, G16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  return cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)((size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024));
 }
 // Opt-in shared-memory sizes, set once per device at cache creation (never during a stream capture).
 cudaError_t configure_attn_kernels() {
   cudaError_t e;
-  if ((e = configure_t<128, true>()) != cudaSuccess) return e;
-  if ((e = configure_t<128, false>()) != cudaSuccess) return e;
-  if ((e = configure_t<64, true>()) != cudaSuccess) return e;
-  return configure_t<64, false>();
+  if ((e = configure_t<128, true, NW_LAT>()) != cudaSuccess) return e;
+  if ((e = configure_t<128, false, NW_LAT>()) != cudaSuccess) return e;
+  if ((e = configure_t<64, true, NW_LAT>()) != cudaSuccess) return e;
+  if ((e = configure_t<64, false, NW_LAT>()) != cudaSuccess) return e;
+  if ((e = configure_t<128, true, NW_THR>()) != cudaSuccess) return e;
+  if ((e = configure_t<128, false, NW_THR>()) != cudaSuccess) return e;
+  if ((e = configure_t<64, true, NW_THR>()) != cudaSuccess) return e;
+  return configure_t<64, false, NW_THR>();
 }
 
 cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
   if (a.n_items <= 0) return cudaSuccess;
   const bool g16 = cv.geo.g > 8;
-  if (cv.geo.d == 128) return g16 ? launch_t<128, true>(cv, a, st) : launch_t<128, false>(cv, a, st);
-  if (cv.geo.d == 64) return g16 ? launch_t<64, true>(cv, a, st) : launch_t<64, false>(cv, a, st);
+  if (a.throughput) {
+    if (cv.geo.d == 128) return g16 ? launch_t<128, true, NW_THR>(cv, a, st) : launch_t<128, false, NW_THR>(cv, a, st);
+    if (cv.geo.d == 64) return g16 ? launch_t<64, true, NW_THR>(cv, a, st) : launch_t<64, false, NW_THR>(cv, a, st);
+  } else {
+    if (cv.geo.d == 128) return g16 ? launch_t<128, true, NW_LAT>(cv, a, st) : launch_t<128, false, NW_LAT>(cv, a, st);
+    if (cv.geo.d == 64) return g16 ? launch_t<64, true, NW_LAT>(cv, a, st) : launch_t<64, false, NW_LAT>(cv, a, st);
+  }
   return cudaErrorInvalidValue;
 }
 

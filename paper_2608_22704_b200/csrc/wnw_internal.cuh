@@ -123,6 +123,7 @@ struct AttnArgs {
   const WorkItem *items_host;    // host copy (the launcher inlines short lists into the kernel parameters)
   const TmaMaps *maps;           // host pointer; passed to the kernel by value
   int32_t n_items;
+  int32_t throughput;            // items were cut for the 4-warp, 2-CTAs-per-SM variant (more than one wave of work)
   int32_t pdl;                   // launch with programmatic stream serialization (previous stream op is a layer kernel)
   const HeadItems *head_items;  // [n_active][Hkv] work items of each head (first is relative to `items`)
   const bf16 *q;         // [n_active][Hq][d]
@@ -173,6 +174,6 @@ cudaError_t configure_attn_kernels();
 bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d);
 cudaError_t configure_select_kernel();
 constexpr int SELECT_SMEM_CAP = 200 * 1024;  // dynamic shared memory the selection kernel may be launched with
-int attn_warps();  // warps per attention CTA (granules per work item should be a multiple)
+int attn_warps(bool throughput);  // warps per attention CTA in the latency / throughput variant
 
 }  // namespace wnw

@@ -25,6 +25,7 @@ struct SeqHost {
 
 struct LayerWork {
   int first_item = 0, n_items = 0, max_count = 0;  // range in the uploaded item array
+  bool throughput = false;                         // which kernel variant the items were cut for
   int head_items_off = 0;                          // offset in the uploaded HeadItems array
 };
 
@@ -71,6 +72,7 @@ struct wnw_cache {
   WorkItem *d_pf_items = nullptr;
   HeadItems *d_pf_head_items = nullptr;
   int pf_n_items = 0;
+  bool pf_throughput = false;
   size_t pf_items_cap = 0;
   // partial buffers
   float *part_o = nullptr;
@@ -316,7 +318,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   for (int l = 0; l < L; ++l) n_aq = std::max(n_aq, c->layers[l].n_anchor * G.g);
   c->n_aq_max = std::max(n_aq, 1);
   c->n_ag_max = std::max(G.C_max * G.gpc, 1);
-  c->part_cap_items = 2 * c->n_sm + (int)B * Hkv + 16;
+  c->part_cap_items = 10 * c->n_sm + 2 * (int)B * Hkv + 64;
   // split partials and head counters alternate by layer parity: two consecutive layer kernels may overlap
   CKC(dev_alloc(c, &c->part_o, 2 * (size_t)c->part_cap_items * G.g * d, false));
   CKC(dev_alloc(c, &c->part_ml, 2 * (size_t)c->part_cap_items * G.g, false));
@@ -382,15 +384,32 @@ extern "C" wnw_status_t wnw_destroy(wnw_cache_t *c) {
 // ---------------------------------------------------------------------------------------------
 // Granules per work item: enough items to fill the machine about twice over, never shorter than one granule per
 // warp, and a head is cut into at most ~32 pieces because the merge that follows reads every piece.
-static int granules_per_item(const wnw_cache *c, long long total_granules, int longest_head) {
-  const int nw = attn_warps();
+// Little work (fits one wave of CTAs): smallest useful items, so every byte is in flight at once.  Otherwise items are
+// sized for about two CTAs per SM per `wave`: every item costs a prologue and a merge, so fewer, longer items win.
+static int granules_per_item(const wnw_cache *c, long long total_granules, int longest_head, int n_heads, bool *throughput) {
+  int nw = attn_warps(false);
   int min_gpi = nw;
   if (const char *e = getenv("WNW_MIN_GRANULES_PER_ITEM")) min_gpi = std::max(nw, atoi(e) / nw * nw);
-  const long long target = 2ll * c->n_sm;
+  long long items_lat = 0;
+  {
+    long long per = std::max<long long>(min_gpi, (longest_head + 31) / 32);
+    per = (per + nw - 1) / nw * nw;
+    items_lat = (total_granules + per - 1) / per + n_heads;
+  }
+  *throughput = items_lat > c->n_sm;
+  if (const char *e = getenv("WNW_THROUGHPUT")) *throughput = atoi(e) != 0;
+  if (!*throughput) {
+    long long per = std::max<long long>(min_gpi, (longest_head + 31) / 32);
+    return (int)((per + nw - 1) / nw * nw);
+  }
+  nw = attn_warps(true);
+  int waves = 1;
+  if (const char *e = getenv("WNW_WAVES")) waves = std::max(1, atoi(e));
+  const long long target = 2ll * c->n_sm * waves;
   long long per = (total_granules + target - 1) / target;
   per = std::max<long long>(per, (longest_head + 31) / 32);
-  per = (per + nw - 1) / nw * nw;
-  return (int)std::max<long long>(per, min_gpi);
+  per = std::max<long long>(per, 2 * nw);          // at least two granules per warp: the per-CTA overhead must amortise
+  return (int)((per + nw - 1) / nw * nw);
 }
 
 // Appends the items of one layer for the given sequences.
@@ -410,7 +429,9 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       longest = std::max(longest, G.n_tg + audio);
     }
   }
-  const int gpi = granules_per_item(c, total, longest);
+  bool throughput = false;
+  const int gpi = granules_per_item(c, total, longest, (int)seq_ids.size() * G.Hkv, &throughput);
+  lw.throughput = throughput;
   lw.first_item = (int)items.size();
   lw.head_items_off = (int)heads.size();
   lw.max_count = 0;
@@ -540,12 +561,13 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
       CK(cudaMemcpyAsync(c->d_pf_head_items, heads.data(), heads.size() * sizeof(HeadItems), cudaMemcpyHostToDevice, st));
       CK(cudaStreamSynchronize(st));  // the host vectors go out of scope
       c->pf_n_items = (int)items.size();
+      c->pf_throughput = lw.throughput;
       c->h_pf_items = items;
       c->prefill_seq = seq; c->prefill_T_a = T_a;
     }
     AttnArgs a{};
     a.mode = ATTN_PREFILL; a.layer = layer; a.li = c->layers[layer]; a.n_active = 1; a.has_new = 0; a.score_on = 1;
-    a.active = c->d_iota + seq; a.items = c->d_pf_items; a.items_host = c->h_pf_items.data(); a.n_items = c->pf_n_items; a.maps = &c->maps_prefill;
+    a.active = c->d_iota + seq; a.items = c->d_pf_items; a.items_host = c->h_pf_items.data(); a.n_items = c->pf_n_items; a.maps = &c->maps_prefill; a.throughput = c->pf_throughput;
     a.head_items = c->d_pf_head_items;
     a.q = (const bf16 *)q_last_dev;
     a.anchor_base = c->stage; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
@@ -629,7 +651,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   a.score_on = tiered && li.n_anchor > 0;
   if (const char *e = getenv("WNW_DEBUG_STOP")) a.debug_stop = atoi(e);  // timing experiments only; breaks results
   a.active = c->d_active; a.items = c->d_items + lw.first_item; a.items_host = c->h_items.data() + lw.first_item;
-  a.n_items = lw.n_items; a.maps = &c->maps_decode;
+  a.n_items = lw.n_items; a.maps = &c->maps_decode; a.throughput = lw.throughput;
   a.head_items = c->d_head_items + lw.head_items_off;
   a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
   const size_t par = (size_t)(layer & 1);

@@ -77,7 +77,7 @@ extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, 
   cudaStream_t st = (cudaStream_t)cuda_stream;
 
   // split every head's granules over at most ST_MAX_ITEMS CTAs in total
-  const int nw = attn_warps();
+  const int nw = attn_warps(false);
   const int n_gran = (n_tokens + GR - 1) / GR;
   const int per_head_max = ST_MAX_ITEMS / n_kv_heads;
   if (per_head_max < 1) return WNW_ERR_CAPACITY;
