@@ -58,6 +58,28 @@ def make_workload(name: str, n_steps: int, seed: int):
     return w
 
 
+# ------------------------------------------------------------------------------------------------- multi-rank helpers
+def shard_plan(world: int, batch_per_rank: int) -> dict:
+    """The path shards by sequence: every rank serves its own sequences on its own GPU with no data-path collective,
+    so the whole job is `world` independent replicas of the per-rank workload (weak scaling)."""
+    return {"scaling": "weak", "sequences_per_rank": batch_per_rank, "total_sequences": world * batch_per_rank,
+            "collective": None}
+
+
+def dist_max(x: float, device, world: int) -> float:
+    """Max over ranks of a device-timed duration (the only cross-rank exchange; not on the data path)."""
+    if world <= 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world: int, batch_per_rank: int, ms_per_step_max: float) -> float:
+    """All ranks step together; the job emits world * batch tokens per step, paced by the slowest rank."""
+    return world * batch_per_rank / (ms_per_step_max * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------------- clocks
 class ClockSampler:
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -398,12 +420,8 @@ def run_ours(args, rank, world, local_rank):
     wall = time.perf_counter() - wall0
     clocks = sampler.stop()
     stats1 = wnw.wnw_get_stats(job.caches["wnw"])
-    ms_total = sum(per_step)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    ms_per_step = float(t.item()) / K
-    value = world * w.batch / (ms_per_step * 1e-3)
+    ms_per_step = dist_max(sum(per_step), dev, world) / K
+    value = whole_job_tokens_per_s(world, w.batch, ms_per_step)
 
     # ---- comparison: own full-cache kernel, and WnW with recall copies skipped (exposed recall time)
     full_steps = job.timed_steps("full", W + R, K, full=True, graph=not args.eager)
@@ -436,10 +454,7 @@ def run_ours(args, rank, world, local_rank):
             e1.record()
             e1.synchronize()
             e2e_ms += e0.elapsed_time(e1)
-    t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    e2e_value = world * w.batch / (float(t.item()) / n_e2e * 1e-3)
+    e2e_value = whole_job_tokens_per_s(world, w.batch, dist_max(e2e_ms, dev, world) / n_e2e)
     h2d = job.sslab.numel() * 2
     d2h = job.out.numel() * 2
 

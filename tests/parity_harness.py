@@ -78,6 +78,8 @@ class Lockstep:
                 p = self.syn.prefill(b, l)
                 k, v, ql = (p[n].to(self.dev) for n in ("k", "v", "q_last"))
                 wnw.wnw_place_prefill(self.h, b, l, k, v, p["audio_begin"], p["audio_end"], ql)
+                if self.syn.device.type == "cuda":
+                    torch.cuda.synchronize(self.dev)   # the generator's buffers are released right after
                 if b in self.oracle_seqs:
                     kb, vb = bf16_bits(p["k"]), bf16_bits(p["v"])
                     self.o.place_prefill(b, l, kb, vb, p["audio_begin"], p["audio_end"], bf16_bits(p["q_last"]))

@@ -1,0 +1,39 @@
+"""GPU parity at the full sizes of the batched configurations, in the launch configuration the benchmark times
+(captured step replayed as a CUDA graph).  The oracle follows a sample of the sequences; inputs are generated on the
+device and the sampled sequences' bits are copied to the host for the oracle.  (Needs a B200.)"""
+import numpy as np
+import pytest
+import torch
+
+from workloads import config3, config4
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(w, oracle_seqs, n_steps, graph=True):
+    from parity_harness import Lockstep
+    ls = Lockstep(w, seed=0, gen_device="cuda:0", oracle_seqs=oracle_seqs)
+    try:
+        ls.prefill(check_slots=False)
+        for t in range(n_steps):
+            ls.decode_step(t, graph=graph, check_slots=(t == n_steps - 1))
+        return ls.near_ties
+    finally:
+        ls.close()
+
+
+def test_config3_batch32_ragged_sampled_sequences():
+    """Batched serving: config-1 shapes at batch 32, audio lengths U{2000..7500}; the oracle follows the shortest and
+    the longest sequence through prefill placement and three decode steps."""
+    w = config3(n_steps=3)
+    lens = np.array(w.audio_lens)
+    _run(w, oracle_seqs=sorted({int(lens.argmin()), int(lens.argmax())}), n_steps=3)
+
+
+@pytest.mark.parametrize("budget,chunk", [(0.1, 16), (0.4, 256)])
+def test_config4_recall_stress_corners(budget, chunk):
+    """Recall stress: batch 8 x 7500 audio tokens, focus jumping every 4 steps; corners of the budget x chunk grid
+    (469 chunks of 16 tokens / 30 chunks of 256 tokens).  Five steps cover one jump; the last step also checks that
+    every resident slot holds the exact bytes of its chunk."""
+    w = config4(budget=budget, chunk=chunk, n_steps=5)
+    _run(w, oracle_seqs=[3], n_steps=5)
