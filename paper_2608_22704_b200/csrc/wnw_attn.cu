@@ -44,8 +44,20 @@ extern "C" int wnw_debug_clear_stamps() {
   static long long zeros[8192 * 16];
   return (int)cudaMemcpyToSymbol(g_stamps, zeros, sizeof(zeros));
 }
+__device__ unsigned long long g_ktime[4 * 64 * 4];   // [step % 4][layer][start_min, trigger_max, end_max, unused], nanoseconds
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define KSTAMP_MIN(slot, k) do { if (threadIdx.x == 0) atomicMin(&g_ktime[(slot) * 4 + (k)], gtime()); } while (0)
+#define KSTAMP_MAX(slot, k) do { if (threadIdx.x == 0) atomicMax(&g_ktime[(slot) * 4 + (k)], gtime()); } while (0)
+extern "C" int wnw_debug_read_ktime(unsigned long long *host) { return (int)cudaMemcpyFromSymbol(host, g_ktime, sizeof(g_ktime)); }
+extern "C" int wnw_debug_init_ktime() {
+  static unsigned long long init[4 * 64 * 4];
+  for (int i = 0; i < 4 * 64 * 4; ++i) init[i] = (i % 4 == 0) ? ~0ull : 0ull;
+  return (int)cudaMemcpyToSymbol(g_ktime, init, sizeof(init));
+}
 #else
 #define STAMP(k) do { } while (0)
+#define KSTAMP_MIN(slot, k) do { } while (0)
+#define KSTAMP_MAX(slot, k) do { } while (0)
 #endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -162,7 +174,20 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   const int T_t = cv.text_len[b] + a.has_new;
 #ifdef WNW_PHASE_STAMPS
   if (it.g0 >= 0) STAMP(10);
+  const int kslot = (int)((cv.steps[b] & 3) * 64 + a.layer);
+  KSTAMP_MIN(kslot, 0);
 #endif
+  // Programmatic dependent launch: the next layer's kernel may be scheduled right away.  A layer kernel touches only
+  // its own layer's stores, partial buffers, counters and outputs, so consecutive layer kernels are independent and
+  // may overlap as deeply as free SMs allow.  What later stream work relies on is that a completed kernel implies
+  // that all earlier ones completed: one CTA waits for the predecessor right before it exits (pdl_finish).
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+  auto pdl_finish = [&]() {
+    if (blockIdx.x == 0) {
+      asm volatile("griddepcontrol.wait;\n" ::: "memory");
+      KSTAMP_MAX(kslot, 1);
+    }
+  };
   int v_delta_audio;  // rows between a granule's K and V rows
   const CUtensorMap *map_audio;
   if (role == ROLE_ANCHOR) { v_delta_audio = G.T_a_pad; map_audio = &maps.anchor; }
@@ -390,13 +415,6 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   __syncthreads();
   STAMP(2);
 
-  // Programmatic dependent launch.  Everything below writes scratch that alternates by layer parity, so the
-  // previous layer's kernel must have completed (wait); after that the next layer's kernel may be scheduled and
-  // stream its K/V while this one merges (launch_dependents).  Because every CTA waits before it releases the
-  // next kernel, at most two layer kernels ever overlap and two scratch parities are enough.
-  asm volatile("griddepcontrol.wait;\n" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
-
   // ---- merge the warps' partial states through shared memory ----
   float2 *red_ml = reinterpret_cast<float2 *>(smem);                           // [NW][16]
   float *red_o = reinterpret_cast<float *>(smem + NW * 16 * sizeof(float2));   // [NW][g][D]
@@ -441,7 +459,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     }
   }
   STAMP(3);
-  if (direct || a.mode == ATTN_PREFILL || a.debug_stop == 1) return;
+  KSTAMP_MAX(kslot, 2);
+  if (direct || a.mode == ATTN_PREFILL || a.debug_stop == 1) { pdl_finish(); return; }
 
   // ---- the CTA that finishes this head last merges its split partials ----
   __shared__ int s_flag;
@@ -507,6 +526,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     }
   }
   STAMP(5);
+  KSTAMP_MAX(kslot, 2);
+  pdl_finish();
 }
 
 template <int D, bool G16, int NW>

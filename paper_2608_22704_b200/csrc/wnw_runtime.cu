@@ -26,6 +26,7 @@ struct SeqHost {
 struct LayerWork {
   int first_item = 0, n_items = 0, max_count = 0;  // range in the uploaded item array
   bool throughput = false;                         // which kernel variant the items were cut for
+  size_t part_off = 0;                             // first partial of this layer in the partial buffers (in items)
   int head_items_off = 0;                          // offset in the uploaded HeadItems array
 };
 
@@ -78,7 +79,9 @@ struct wnw_cache {
   float *part_o = nullptr;
   float2 *part_ml = nullptr, *gran_em = nullptr, *head_mz = nullptr;
   int32_t *head_done = nullptr;
-  float2 *pf_gran_em = nullptr;
+  float2 *pf_gran_em = nullptr, *pf_part_ml = nullptr;
+  float *pf_part_o = nullptr;
+  size_t part_cap_total = 0;
   int part_cap_items = 0, n_aq_max = 0, n_ag_max = 0;
   // streams / events
   static constexpr int N_SIDE = 4;  // layers alternate between side streams so selection + recall keep pace with attention
@@ -90,6 +93,7 @@ struct wnw_cache {
   size_t gran_em_layer_stride = 0;
   bool step_capturing = false;
   bool pdl_enabled = true;
+  int direct_max_granules = 64;   // heads up to this many granules (text capacity included) are not split in the latency regime
   // captured step
   bool graph_capturing = false;
   cudaGraph_t graph = nullptr;
@@ -217,6 +221,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
 #define CKE(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { return fail(_e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA); } } while (0)
   cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
   if (const char *e = getenv("WNW_PDL")) c->pdl_enabled = atoi(e) != 0;
+  if (const char *e = getenv("WNW_DIRECT_MAX_GRANULES")) c->direct_max_granules = atoi(e);
   CKE(configure_attn_kernels());
   CKE(configure_select_kernel());
   const int L = cfg->n_layers, Hkv = cfg->n_kv_heads, d = cfg->head_dim, nc = cfg->chunk_tokens;
@@ -319,9 +324,10 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   c->n_aq_max = std::max(n_aq, 1);
   c->n_ag_max = std::max(G.C_max * G.gpc, 1);
   c->part_cap_items = 10 * c->n_sm + 2 * (int)B * Hkv + 64;
-  // split partials and head counters alternate by layer parity: two consecutive layer kernels may overlap
-  CKC(dev_alloc(c, &c->part_o, 2 * (size_t)c->part_cap_items * G.g * d, false));
-  CKC(dev_alloc(c, &c->part_ml, 2 * (size_t)c->part_cap_items * G.g, false));
+  // split partials of the prefill scoring pass; the decode layers get one region each (sized with the work lists),
+  // because consecutive layer kernels overlap
+  CKC(dev_alloc(c, &c->pf_part_o, (size_t)c->part_cap_items * G.g * d, false));
+  CKC(dev_alloc(c, &c->pf_part_ml, (size_t)c->part_cap_items * G.g, false));
   // granule partials and final (M,Z) are per layer: the side-stream selection of layer l reads them while the
   // caller's stream already runs later layers
   c->gran_em_layer_stride = B * (size_t)c->n_aq_max * c->n_ag_max;
@@ -339,7 +345,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     if (fixed_part + per_chunk > cap) return fail(WNW_ERR_UNSUPPORTED);  // chunk tables too large for one CTA
     c->sel_smem[l] = std::min(cap, fixed_part + per_chunk * std::max(G.C_max, 1)) + 16;
   }
-  CKC(dev_alloc(c, &c->head_done, 2 * B * Hkv));
+  CKC(dev_alloc(c, &c->head_done, (size_t)L * B * Hkv));
   {
     const unsigned long long r_text = B * (unsigned long long)G.text_seq_stride / d, r_anchor = B * (unsigned long long)G.anchor_seq_stride / d,
                              r_pool = B * (unsigned long long)G.pool_seq_stride / d, r_fixed = B * (unsigned long long)G.fixed_seq_stride / d,
@@ -441,7 +447,9 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       const SeqHost &sq = c->seqs[seq_ids[i]];
       const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
       const int ridx = mode == ATTN_DECODE ? c->role_idx[layer * G.Hkv + h] : h;
-      const int n_cta = std::max(1, (n + gpi - 1) / gpi);
+      // latency regime: a short head stays in one CTA, which then writes the output itself (no partial, no merge)
+      int n_cta = std::max(1, (n + gpi - 1) / gpi);
+      if (!throughput && n <= c->direct_max_granules) n_cta = 1;
       HeadItems hi{(int)items.size() - lw.first_item, n_cta};
       for (int x = 0; x < n_cta; ++x) {  // even contiguous ranges
         const int g0 = (int)((long long)n * x / n_cta), g1 = (int)((long long)n * (x + 1) / n_cta);
@@ -462,12 +470,22 @@ static wnw_status_t ensure_worklists(wnw_cache *c) {
   std::vector<WorkItem> items;
   std::vector<HeadItems> heads;
   c->wl_layers.assign(G.L, LayerWork{});
+  size_t part_total = 0;
   for (int l = 0; l < G.L; ++l) {
     build_layer_items(c, l, mode, c->active, items, heads, c->wl_layers[l]);
-    if (c->wl_layers[l].n_items > c->part_cap_items) return WNW_ERR_CAPACITY;
+    c->wl_layers[l].part_off = part_total;
+    part_total += (size_t)c->wl_layers[l].n_items;
   }
   // the previous lists may still be read by queued kernels
   CK(cudaDeviceSynchronize());
+  if (part_total > c->part_cap_total) {  // one partial region per layer
+    float *po = nullptr; float2 *pm = nullptr;
+    CK(cudaMalloc((void **)&po, part_total * G.g * G.d * sizeof(float)));
+    c->dev_allocs.push_back(po);
+    CK(cudaMalloc((void **)&pm, part_total * G.g * sizeof(float2)));
+    c->dev_allocs.push_back(pm);
+    c->part_o = po; c->part_ml = pm; c->part_cap_total = part_total;
+  }
   if (items.size() > c->d_items_cap) {
     CK(cudaMalloc((void **)&c->d_items, items.size() * sizeof(WorkItem)));
     c->dev_allocs.push_back(c->d_items);
@@ -571,9 +589,9 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
     a.head_items = c->d_pf_head_items;
     a.q = (const bf16 *)q_last_dev;
     a.anchor_base = c->stage; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
-    a.part_o = c->part_o; a.part_ml = c->part_ml; a.gran_em = c->pf_gran_em; a.n_aq = G.Hq; a.n_ag_max = c->n_ag_max;
+    a.part_o = c->pf_part_o; a.part_ml = c->pf_part_ml; a.gran_em = c->pf_gran_em; a.n_aq = G.Hq; a.n_ag_max = c->n_ag_max;
     CK(launch_attn(c->cv, a, st));
-    CK(launch_prefill_select(c->cv, seq, layer, c->d_pf_head_items, c->part_ml, c->pf_gran_em, c->n_ag_max, st));
+    CK(launch_prefill_select(c->cv, seq, layer, c->d_pf_head_items, c->pf_part_ml, c->pf_gran_em, c->n_ag_max, st));
   }
   CK(launch_place_gather(c->cv, seq, layer, full ? 1 : 0, c->stage, C_b, st));
   CK(cudaEventRecord(c->ev_place, st));
@@ -654,11 +672,10 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   a.n_items = lw.n_items; a.maps = &c->maps_decode; a.throughput = lw.throughput;
   a.head_items = c->d_head_items + lw.head_items_off;
   a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
-  const size_t par = (size_t)(layer & 1);
-  a.head_done = c->head_done + par * G.max_batch * G.Hkv; a.head_mz = head_mz_l; a.out = (bf16 *)out;
+  a.head_done = c->head_done + (size_t)layer * G.max_batch * G.Hkv; a.head_mz = head_mz_l; a.out = (bf16 *)out;
   a.anchor_base = c->cv.anchor; a.anchor_seq_stride = G.anchor_seq_stride;
   a.anchor_head0 = tiered ? li.anchor_off : layer * G.Hkv;
-  a.part_o = c->part_o + par * c->part_cap_items * G.g * G.d; a.part_ml = c->part_ml + par * c->part_cap_items * G.g;
+  a.part_o = c->part_o + lw.part_off * G.g * G.d; a.part_ml = c->part_ml + lw.part_off * G.g;
   a.gran_em = gran_em_l;
   // overlap with the previous layer's kernel when that is what precedes this launch in the stream
   a.pdl = layer > 0 && c->pdl_enabled;
