@@ -84,8 +84,8 @@ struct wnw_cache {
   size_t part_cap_total = 0;
   int part_cap_items = 0, n_aq_max = 0, n_ag_max = 0;
   // streams / events
-  static constexpr int N_SIDE = 4;  // layers alternate between side streams so selection + recall keep pace with attention
-  cudaStream_t side[N_SIDE] = {nullptr, nullptr, nullptr, nullptr}, last_stream = nullptr;
+  static constexpr int N_SIDE = 8;  // layers alternate between side streams so selection + recall keep pace with attention
+  cudaStream_t side[N_SIDE] = {}, last_stream = nullptr;
   std::vector<cudaEvent_t> ev_layer_done, ev_side_done;
   std::vector<cudaEvent_t> ev_layer_done_cap, ev_side_done_cap;  // used only inside a stream capture
   std::vector<char> side_recorded;
@@ -101,7 +101,7 @@ struct wnw_cache {
   std::vector<int> graph_active, graph_prepared;
   long long wl_epoch = 0, graph_epoch = -1;  // work-list generation the graph was captured against
   int graph_appended = 0;
-  int last_side_layer[N_SIDE] = {-1, -1, -1, -1};
+  int last_side_layer[N_SIDE] = {-1, -1, -1, -1, -1, -1, -1, -1};
   cudaEvent_t ev_place = nullptr, ev_step = nullptr;
   bool place_recorded = false, step_recorded = false;
   // timing
