@@ -363,8 +363,12 @@ def run_ours(args, rank, world, local_rank):
         wnw.wnw_set_kernel_timing(job.caches["wnw"], True)
         per_step = job.timed_steps("wnw", W, K, full=args.quick_full, flush=not args.no_flush, graph=not args.eager)
         ms, n = wnw.wnw_get_kernel_time(job.caches["wnw"])
-        print(json.dumps({"quick": True, "workload": w.name, "ms_per_step": sum(per_step) / K, "steps": K,
-                          "attn_us_per_launch": ms * 1e3 / max(n, 1)}), flush=True)
+        kv_bytes, _ = job.kv_bytes_of_step("wnw", full=args.quick_full)
+        ms_step = sum(per_step) / K
+        print(json.dumps({"quick": True, "workload": w.name, "ms_per_step": ms_step, "steps": K,
+                          "attn_us_per_launch": ms * 1e3 / max(n, 1), "kv_GB_per_step": kv_bytes / 1e9,
+                          "kv_GBps": kv_bytes / (ms_step * 1e-3) / 1e9, "frac_of_peak": kv_bytes / (ms_step * 1e-3) / 1e9 / peak_gbs}),
+              flush=True)
         job.destroy()
         return
     job.create("full", wnw.WNW_MODE_FULL)

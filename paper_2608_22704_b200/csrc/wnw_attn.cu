@@ -166,37 +166,23 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   STAMP(0);
-  // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
-  const WorkItem it = a.n_items <= INLINE_ITEMS_MAX ? inl.it[blockIdx.x] : a.items[blockIdx.x];
-  const int b = it.b, role = it.role, ridx = it.ridx, T_a = it.T_a;
-  const int g = G.g;
-  const LayerInfo &li = a.li;
-  const int T_t = cv.text_len[b] + a.has_new;
-#ifdef WNW_PHASE_STAMPS
-  if (it.g0 >= 0) STAMP(10);
-  const int kslot = (int)((cv.steps[b] & 3) * 64 + a.layer);
-  KSTAMP_MIN(kslot, 0);
-#endif
   // Programmatic dependent launch: the next layer's kernel may be scheduled right away.  A layer kernel touches only
   // its own layer's stores, partial buffers, counters and outputs, so consecutive layer kernels are independent and
   // may overlap as deeply as free SMs allow.  What later stream work relies on is that a completed kernel implies
   // that all earlier ones completed: one CTA waits for the predecessor right before it exits (pdl_finish).
   asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+#ifdef WNW_PHASE_STAMPS
+  int kslot = 0;
+#endif
   auto pdl_finish = [&]() {
     if (blockIdx.x == 0) {
       asm volatile("griddepcontrol.wait;\n" ::: "memory");
       KSTAMP_MAX(kslot, 1);
     }
   };
-  int v_delta_audio;  // rows between a granule's K and V rows
-  const CUtensorMap *map_audio;
-  if (role == ROLE_ANCHOR) { v_delta_audio = G.T_a_pad; map_audio = &maps.anchor; }
-  else if (role == ROLE_TIDAL) { v_delta_audio = G.nc; map_audio = &maps.pool; }
-  else { v_delta_audio = G.S_max * G.nc; map_audio = &maps.fixed; }
-  const int v_delta_text = G.T_cap_pad;
-
   __shared__ int2 ring[NW][NSTAGE];                              // per stage: visible rows | loaded << 8, score index
   __shared__ __align__(8) unsigned long long bars[NW][NSTAGE];   // one mbarrier per stage, producer = consumer = this warp
+  __shared__ int s_flag;
   const uint32_t my_base = smem_u32(smem + (size_t)warp * NSTAGE * 2 * TILEB);
   if (lane == 0) {
 #pragma unroll
@@ -205,6 +191,33 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     fence_proxy_async();
   }
   __syncwarp();
+  uint32_t phase_bits = 0;   // parity of each stage's barrier (carried across the CTA's work items)
+  bool timed_out = false;
+  const int g = G.g;
+  const LayerInfo &li = a.li;
+
+  // One work item per CTA when the launch fits the machine; otherwise a persistent CTA per SM walks the items the
+  // host assigned to it (balanced by size), so no SM idles through a partial last wave.
+  int q_begin = blockIdx.x, q_end = blockIdx.x + 1;
+  if (a.cta_ranges) { q_begin = a.cta_ranges[blockIdx.x]; q_end = a.cta_ranges[blockIdx.x + 1]; }
+  for (int qi = q_begin; qi < q_end; ++qi) {
+  const int item_idx = a.cta_ranges ? a.order[qi] : qi;
+  if (qi > q_begin) __syncthreads();  // the previous item's merge is done with shared memory
+  // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
+  const WorkItem it = a.n_items <= INLINE_ITEMS_MAX ? inl.it[item_idx] : a.items[item_idx];
+  const int b = it.b, role = it.role, ridx = it.ridx, T_a = it.T_a;
+  const int T_t = cv.text_len[b] + a.has_new;
+#ifdef WNW_PHASE_STAMPS
+  if (it.g0 >= 0) STAMP(10);
+  kslot = (int)((cv.steps[b] & 3) * 64 + a.layer);
+  KSTAMP_MIN(kslot, 0);
+#endif
+  int v_delta_audio;  // rows between a granule's K and V rows
+  const CUtensorMap *map_audio;
+  if (role == ROLE_ANCHOR) { v_delta_audio = G.T_a_pad; map_audio = &maps.anchor; }
+  else if (role == ROLE_TIDAL) { v_delta_audio = G.nc; map_audio = &maps.pool; }
+  else { v_delta_audio = G.S_max * G.nc; map_audio = &maps.fixed; }
+  const int v_delta_text = G.T_cap_pad;
 
   const int first = it.g0 + warp;
   const int n_my = first < it.g1 ? (it.g1 - first + NW - 1) / NW : 0;
@@ -297,8 +310,6 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 #pragma unroll
   for (int t = 0; t < D / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-  uint32_t phase_bits = 0;   // parity of each stage's barrier
-  bool timed_out = false;
 
   for (int n = 0; n < n_my; ++n) {
     __syncwarp();
@@ -454,16 +465,15 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       *reinterpret_cast<uint32_t *>(a.out + ((long long)it.i * G.Hq + (long long)it.h * g) * D + idx) = pack_bf16(a0 * inv, a1 * inv);
       if (idx % D == 0) a.head_mz[(long long)it.i * G.Hq + it.h * g + row] = make_float2(M, L);
     } else {
-      *reinterpret_cast<float2 *>(a.part_o + (long long)blockIdx.x * g * D + idx) = make_float2(a0, a1);
-      if (idx % D == 0) a.part_ml[(long long)blockIdx.x * g + row] = make_float2(M, L);
+      *reinterpret_cast<float2 *>(a.part_o + (long long)item_idx * g * D + idx) = make_float2(a0, a1);
+      if (idx % D == 0) a.part_ml[(long long)item_idx * g + row] = make_float2(M, L);
     }
   }
   STAMP(3);
   KSTAMP_MAX(kslot, 2);
-  if (direct || a.mode == ATTN_PREFILL || a.debug_stop == 1) { pdl_finish(); return; }
+  if (direct || a.mode == ATTN_PREFILL || a.debug_stop == 1) continue;
 
   // ---- the CTA that finishes this head last merges its split partials ----
-  __shared__ int s_flag;
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -474,7 +484,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   }
   __syncthreads();
   STAMP(4);
-  if (!s_flag) return;
+  if (!s_flag) continue;
   __threadfence();
   constexpr int NT = NW * 32;
   {
@@ -527,6 +537,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   }
   STAMP(5);
   KSTAMP_MAX(kslot, 2);
+  }  // work items of this CTA
   pdl_finish();
 }
 
@@ -538,7 +549,7 @@ static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t
   if (a.n_items <= INLINE_ITEMS_MAX && a.items_host) memcpy(inl.it, a.items_host, sizeof(WorkItem) * a.n_items);
   else if (a.n_items <= INLINE_ITEMS_MAX) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)a.n_items, 1, 1);
+  cfg.gridDim = dim3((unsigned)(a.cta_ranges ? a.n_ctas : a.n_items), 1, 1);
   cfg.blockDim = dim3(NW * 32, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;

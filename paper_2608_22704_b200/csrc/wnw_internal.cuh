@@ -123,6 +123,9 @@ struct AttnArgs {
   const WorkItem *items_host;    // host copy (the launcher inlines short lists into the kernel parameters)
   const TmaMaps *maps;           // host pointer; passed to the kernel by value
   int32_t n_items;
+  const int32_t *order;          // persistent schedule (throughput regime), else null: order[cta_ranges[c] .. cta_ranges[c+1]) are
+  const int32_t *cta_ranges;     //   the item indices CTA c processes; n_ctas CTAs are launched
+  int32_t n_ctas;
   int32_t throughput;            // items were cut for the 4-warp, 2-CTAs-per-SM variant (more than one wave of work)
   int32_t pdl;                   // launch with programmatic stream serialization (previous stream op is a layer kernel)
   const HeadItems *head_items;  // [n_active][Hkv] work items of each head (first is relative to `items`)

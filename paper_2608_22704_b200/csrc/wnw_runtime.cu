@@ -27,6 +27,7 @@ struct LayerWork {
   int first_item = 0, n_items = 0, max_count = 0;  // range in the uploaded item array
   bool throughput = false;                         // which kernel variant the items were cut for
   size_t part_off = 0;                             // first partial of this layer in the partial buffers (in items)
+  int n_ctas = 0, order_off = 0, ranges_off = 0;   // persistent schedule (throughput regime): offsets into the uploaded arrays
   int head_items_off = 0;                          // offset in the uploaded HeadItems array
 };
 
@@ -66,6 +67,9 @@ struct wnw_cache {
   std::vector<int> wl_T_a;
   std::vector<LayerWork> wl_layers;
   WorkItem *d_items = nullptr;
+  int32_t *d_sched = nullptr, *d_pf_sched = nullptr;  // persistent schedules: [order of all layers | ranges of all layers]
+  size_t d_sched_cap = 0, sched_ranges_base = 0, pf_sched_cap = 0, pf_ranges_base = 0;
+  int pf_n_ctas = 0;
   std::vector<WorkItem> h_items, h_pf_items;  // host copies (short lists are inlined into kernel parameters)
   HeadItems *d_head_items = nullptr;
   size_t d_items_cap = 0, d_head_items_cap = 0;
@@ -420,7 +424,8 @@ static int granules_per_item(const wnw_cache *c, long long total_granules, int l
 
 // Appends the items of one layer for the given sequences.
 static void build_layer_items(const wnw_cache *c, int layer, int mode, const std::vector<int> &seq_ids,
-                              std::vector<WorkItem> &items, std::vector<HeadItems> &heads, LayerWork &lw) {
+                              std::vector<WorkItem> &items, std::vector<HeadItems> &heads, LayerWork &lw,
+                              std::vector<int32_t> &order, std::vector<int32_t> &ranges) {
   const Geometry &G = c->geo;
   std::vector<int> n_gran(seq_ids.size() * G.Hkv);
   long long total = 0;
@@ -459,6 +464,32 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       lw.max_count = std::max(lw.max_count, hi.count);
     }
   lw.n_items = (int)items.size() - lw.first_item;
+  lw.n_ctas = 0;
+  if (throughput) {
+    // Persistent schedule: one CTA per SM; items go, longest first, to the CTA with the least work so far.  Every
+    // item also costs a prologue and a merge, counted as a few granules' worth.
+    const int P = std::min(c->n_sm, lw.n_items);
+    std::vector<int> idx(lw.n_items);
+    for (int i = 0; i < lw.n_items; ++i) idx[i] = i;
+    auto weight = [&](int i) { const WorkItem &w = items[lw.first_item + i]; return (w.g1 - w.g0) + 6; };
+    std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return weight(x) > weight(y); });
+    std::vector<long long> load(P, 0);
+    std::vector<std::vector<int>> mine(P);
+    for (int i : idx) {
+      const int cta = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+      mine[cta].push_back(i);
+      load[cta] += weight(i);
+    }
+    lw.order_off = (int)order.size();
+    lw.ranges_off = (int)ranges.size();
+    lw.n_ctas = P;
+    int pos = 0;
+    for (int cta = 0; cta < P; ++cta) {
+      ranges.push_back(pos);
+      for (int i : mine[cta]) { order.push_back(i); ++pos; }
+    }
+    ranges.push_back(pos);
+  }
 }
 
 static wnw_status_t ensure_worklists(wnw_cache *c) {
@@ -469,10 +500,11 @@ static wnw_status_t ensure_worklists(wnw_cache *c) {
   const int mode = c->cfg.mode == WNW_MODE_FULL ? ATTN_FULL : ATTN_DECODE;
   std::vector<WorkItem> items;
   std::vector<HeadItems> heads;
+  std::vector<int32_t> order, ranges;
   c->wl_layers.assign(G.L, LayerWork{});
   size_t part_total = 0;
   for (int l = 0; l < G.L; ++l) {
-    build_layer_items(c, l, mode, c->active, items, heads, c->wl_layers[l]);
+    build_layer_items(c, l, mode, c->active, items, heads, c->wl_layers[l], order, ranges);
     c->wl_layers[l].part_off = part_total;
     part_total += (size_t)c->wl_layers[l].n_items;
   }
@@ -496,6 +528,16 @@ static wnw_status_t ensure_worklists(wnw_cache *c) {
     c->dev_allocs.push_back(c->d_head_items);
     c->d_head_items_cap = heads.size();
   }
+  if (order.size() + ranges.size() > c->d_sched_cap) {
+    CK(cudaMalloc((void **)&c->d_sched, (order.size() + ranges.size()) * sizeof(int32_t)));
+    c->dev_allocs.push_back(c->d_sched);
+    c->d_sched_cap = order.size() + ranges.size();
+  }
+  if (!order.empty()) {
+    CK(cudaMemcpy(c->d_sched, order.data(), order.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(c->d_sched + order.size(), ranges.data(), ranges.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+  }
+  c->sched_ranges_base = order.size();
   CK(cudaMemcpy(c->d_items, items.data(), items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
   CK(cudaMemcpy(c->d_head_items, heads.data(), heads.size() * sizeof(HeadItems), cudaMemcpyHostToDevice));
   std::vector<int32_t> act(c->active.begin(), c->active.end());
@@ -563,7 +605,19 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
       std::vector<HeadItems> heads;
       LayerWork lw;
       std::vector<int> one{seq};
-      build_layer_items(c, layer, ATTN_PREFILL, one, items, heads, lw);
+      std::vector<int32_t> order, ranges;
+      build_layer_items(c, layer, ATTN_PREFILL, one, items, heads, lw, order, ranges);
+      if (order.size() + ranges.size() > c->pf_sched_cap) {
+        CK(cudaMalloc((void **)&c->d_pf_sched, (order.size() + ranges.size()) * sizeof(int32_t)));
+        c->dev_allocs.push_back(c->d_pf_sched);
+        c->pf_sched_cap = order.size() + ranges.size();
+      }
+      if (!order.empty()) {
+        CK(cudaMemcpyAsync(c->d_pf_sched, order.data(), order.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+        CK(cudaMemcpyAsync(c->d_pf_sched + order.size(), ranges.data(), ranges.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+      }
+      c->pf_ranges_base = order.size();
+      c->pf_n_ctas = lw.n_ctas;
       if ((int)items.size() > c->part_cap_items) return WNW_ERR_CAPACITY;
       if (items.size() > c->pf_items_cap) {
         CK(cudaMalloc((void **)&c->d_pf_items, items.size() * sizeof(WorkItem)));
@@ -586,6 +640,7 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
     AttnArgs a{};
     a.mode = ATTN_PREFILL; a.layer = layer; a.li = c->layers[layer]; a.n_active = 1; a.has_new = 0; a.score_on = 1;
     a.active = c->d_iota + seq; a.items = c->d_pf_items; a.items_host = c->h_pf_items.data(); a.n_items = c->pf_n_items; a.maps = &c->maps_prefill; a.throughput = c->pf_throughput;
+    if (c->pf_n_ctas > 0) { a.order = c->d_pf_sched; a.cta_ranges = c->d_pf_sched + c->pf_ranges_base; a.n_ctas = c->pf_n_ctas; }
     a.head_items = c->d_pf_head_items;
     a.q = (const bf16 *)q_last_dev;
     a.anchor_base = c->stage; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
@@ -670,6 +725,9 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   if (const char *e = getenv("WNW_DEBUG_STOP")) a.debug_stop = atoi(e);  // timing experiments only; breaks results
   a.active = c->d_active; a.items = c->d_items + lw.first_item; a.items_host = c->h_items.data() + lw.first_item;
   a.n_items = lw.n_items; a.maps = &c->maps_decode; a.throughput = lw.throughput;
+  if (lw.n_ctas > 0) {
+    a.order = c->d_sched + lw.order_off; a.cta_ranges = c->d_sched + c->sched_ranges_base + lw.ranges_off; a.n_ctas = lw.n_ctas;
+  }
   a.head_items = c->d_head_items + lw.head_items_off;
   a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
   a.head_done = c->head_done + (size_t)layer * G.max_batch * G.Hkv; a.head_mz = head_mz_l; a.out = (bf16 *)out;
