@@ -50,9 +50,10 @@ def make_workload(name: str, n_steps: int, seed: int):
         w = config1(seed=0, n_steps=n_steps)
     elif name == "cfg3":
         w = config3(seed=0, n_steps=n_steps)
-    elif name == "prof":   # small many-sequence case for profiler captures: config-1 heads, 4 layers, 16 x 7500 audio tokens
+    elif name in ("prof", "hbm"):   # many long sequences, config-1 heads: 4 layers (profiler captures) or 12 layers (HBM-bound case)
+        n_l = 4 if name == "prof" else 12
         w = config4(seed=0, budget=0.2, chunk=64, batch=16, n_steps=n_steps)
-        w.n_layers = 4; w.roles = w.roles[:4]; w.jump_every = 0; w.sweep_steps = 128; w.name = "prof_4layers_b16_7500"
+        w.n_layers = n_l; w.roles = w.roles[:n_l]; w.jump_every = 0; w.sweep_steps = 128; w.name = f"{name}_{n_l}layers_b16_7500"
     else:
         raise SystemExit(f"unknown workload {name}")
     return w
@@ -490,6 +491,36 @@ def run_ours(args, rank, world, local_rank):
                "sample": f"sequence 0, first {Ls} of {w.n_layers} layers, {args.oracle_steps} decode steps; time scaled by "
                          f"{w.n_layers}/{Ls} layers and x{w.batch} sequences"}
 
+    # ---- the HBM-bound regime, in the same run: many long sequences (config-1 heads, 12 layers, 16 x 7500 audio tokens).
+    # Whole-step time of the replayed graph over the algorithmic K,V bytes; recall copies skipped for the WnW figure so
+    # that the host link does not enter (the normal mode is reported beside it).
+    hbm_case = None
+    if not args.no_hbm_case:
+        job.destroy()
+        torch.cuda.empty_cache()
+        wp = make_workload("hbm", 16, 0)
+        jp = Job(wp, seed=0, device=dev, wnw=wnw)
+        jp.create("wnw", wnw.WNW_MODE_TIERED)
+        jp.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
+        jp.create("full", wnw.WNW_MODE_FULL)
+        jp.place_all(["wnw", "skip", "full"])
+        res = {}
+        for key, full in (("wnw", False), ("skip", False), ("full", True)):
+            for tt in range(3):
+                jp.step(key, tt, full=full)
+            torch.cuda.synchronize(dev)
+            nb, _ = jp.kv_bytes_of_step(key, full=full)
+            ms = sum(jp.timed_steps(key, 3, 10, full=full)) / 10
+            res[key] = (nb, ms)
+        hbm_case = {"workload": wp.name, "layers": wp.n_layers, "batch": wp.batch,
+                    "wnw_copies_skipped": {"GB_per_step": res["skip"][0] / 1e9, "ms_per_step": res["skip"][1],
+                                           "GBps": res["skip"][0] / res["skip"][1] / 1e6, "frac": res["skip"][0] / res["skip"][1] / 1e6 / peak_gbs},
+                    "wnw_with_recall": {"ms_per_step": res["wnw"][1], "GBps": res["wnw"][0] / res["wnw"][1] / 1e6},
+                    "full_cache": {"GB_per_step": res["full"][0] / 1e9, "ms_per_step": res["full"][1],
+                                   "GBps": res["full"][0] / res["full"][1] / 1e6, "frac": res["full"][0] / res["full"][1] / 1e6 / peak_gbs},
+                    "note": "whole replayed step over algorithmic K,V bytes; peak = measured copy bandwidth (read+write)"}
+        jp.destroy()
+
     attn_us = attn_ms * 1e3 / max(attn_n, 1)
     bytes_per_launch = algo_bytes / max(attn_n, 1)
     achieved = bytes_per_launch / (attn_us * 1e-6) / 1e9 if attn_us > 0 else 0.0
@@ -534,12 +565,13 @@ def run_ours(args, rank, world, local_rank):
         "recall": {"bytes_per_step": recall_bytes_step, "hits": stats1["hits"] - stats0["hits"],
                    "misses": stats1["misses"] - stats0["misses"], "link_memcpy_GBps": link_copy, "link_kernel_GBps": link_kernel,
                    "ms_per_step_copies_skipped": ms_skip, "exposed_us_per_step": (ms_per_step - ms_skip) * 1e3},
+        "hbm_bound_case": hbm_case,
         "retention": {"r_gpu": stats1["resident_audio_tokens"] / max(stats1["full_audio_tokens"], 1),
                       "r_gpu_cpu": (stats1["resident_audio_tokens"] + stats1["host_audio_tokens"]) / max(stats1["full_audio_tokens"], 1)},
         "wall_s_timed_region": wall,
     }
     print(json.dumps(line), flush=True)
-    job.destroy()
+    job.destroy()   # no-op if the caches were already released
 
 
 def main():
@@ -548,7 +580,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3", "prof"])
+    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3", "prof", "hbm"])
+    ap.add_argument("--no-hbm-case", action="store_true", help="skip the extra many-sequence measurement")
     ap.add_argument("--quick", action="store_true", help="only the WnW steps (for profiler captures); prints a short line")
     ap.add_argument("--no-flush", action="store_true", help="with --quick: do not flush L2 between steps")
     ap.add_argument("--recall-mode", type=int, default=0, help="with --quick: 0 side stream, 1 inline, 2 copies skipped")
