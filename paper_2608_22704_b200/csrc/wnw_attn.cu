@@ -27,8 +27,8 @@
 namespace wnw {
 
 constexpr int NW_LAT = 8;  // warps per CTA when the launch fits one wave (latency regime): 1 CTA per SM
-constexpr int NW_THR = 8;  // warps per CTA otherwise (throughput regime).  A 4-warp, 2-CTAs-per-SM variant measured no faster (CTAs of
-                           // a wave run their prologue, streaming and merge phases in lock-step), so both regimes use 8 warps.
+constexpr int NW_THR = 4;  // warps per CTA otherwise (throughput regime): two persistent CTAs per SM, whose phases drift apart,
+                           // so one CTA's prologue and merge overlap the other's streaming
 constexpr int NSTAGE = 3;  // granules in flight per warp
 
 int attn_warps(bool throughput) { return throughput ? NW_THR : NW_LAT; }

@@ -468,7 +468,9 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   if (throughput) {
     // Persistent schedule: one CTA per SM; items go, longest first, to the CTA with the least work so far.  Every
     // item also costs a prologue and a merge, counted as a few granules' worth.
-    const int P = std::min(c->n_sm, lw.n_items);
+    int per_sm = 2;  // persistent CTAs per SM (4 warps, 96 KB of shared memory each)
+    if (const char *e = getenv("WNW_CTAS_PER_SM")) per_sm = std::max(1, atoi(e));
+    const int P = std::min(per_sm * c->n_sm, lw.n_items);
     std::vector<int> idx(lw.n_items);
     for (int i = 0; i < lw.n_items; ++i) idx[i] = i;
     auto weight = [&](int i) { const WorkItem &w = items[lw.first_item + i]; return (w.g1 - w.g0) + 6; };
