@@ -471,7 +471,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   }
   STAMP(3);
   KSTAMP_MAX(kslot, 2);
-  if (direct || a.mode == ATTN_PREFILL || a.debug_stop == 1) continue;
+  if (direct || a.mode == ATTN_PREFILL) continue;
 
   // ---- the CTA that finishes this head last merges its split partials ----
   __threadfence();

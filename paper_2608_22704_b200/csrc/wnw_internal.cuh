@@ -117,7 +117,6 @@ struct AttnArgs {
   int32_t n_active;
   int32_t has_new;       // k_new/v_new hold one more text row per sequence (appended by this launch)
   int32_t score_on;      // write per-granule softmax-mass partials for anchor-like heads
-  int32_t debug_stop;    // timing experiments only: 1 = return after the split partials, 2 = after the head merge
   const int32_t *active; // [n_active] sequence ids
   const WorkItem *items;         // device copy of the items
   const WorkItem *items_host;    // host copy (the launcher inlines short lists into the kernel parameters)

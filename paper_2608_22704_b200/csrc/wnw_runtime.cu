@@ -724,7 +724,6 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   AttnArgs a{};
   a.mode = tiered ? ATTN_DECODE : ATTN_FULL; a.layer = layer; a.li = li; a.n_active = n_active; a.has_new = has_new;
   a.score_on = tiered && li.n_anchor > 0;
-  if (const char *e = getenv("WNW_DEBUG_STOP")) a.debug_stop = atoi(e);  // timing experiments only; breaks results
   a.active = c->d_active; a.items = c->d_items + lw.first_item; a.items_host = c->h_items.data() + lw.first_item;
   a.n_items = lw.n_items; a.maps = &c->maps_decode; a.throughput = lw.throughput;
   if (lw.n_ctas > 0) {

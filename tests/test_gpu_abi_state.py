@@ -1,0 +1,108 @@
+"""Call-order and capacity errors of the C ABI on a real device: every misuse returns a status, nothing faults (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from workloads import ROLE_ANCHOR, ROLE_FIXED, ROLE_TIDAL, Synth, tiny_custom
+
+pytestmark = pytest.mark.gpu
+
+
+def _mk(wnw, w, **kw):
+    return wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max(w.audio_lens), w.text_capacity,
+                          w.chunk, w.budget, w.roles, topk=w.topk, **kw)
+
+
+def _place(wnw, h, syn, b, layers):
+    for l in layers:
+        p = syn.prefill(b, l)
+        dev = torch.device("cuda:0")
+        wnw.wnw_place_prefill(h, b, l, p["k"].to(dev), p["v"].to(dev), p["audio_begin"], p["audio_end"], p["q_last"].to(dev))
+
+
+def test_call_order_and_capacity_errors():
+    import paper_2608_22704_b200 as wnw
+    dev = torch.device("cuda:0")
+    w = tiny_custom(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, n_text=4, audio_lens=(64, 64), chunk=16, n_steps=2)
+    syn = Synth(w, seed=1)
+    h = _mk(wnw, w)
+    try:
+        q = torch.zeros((1, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+        kn = torch.zeros((1, w.n_kv_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+        out = torch.zeros_like(q)
+
+        def expect(status, fn, *a, **k):
+            with pytest.raises(wnw.WnwError) as e:
+                fn(*a, **k)
+            assert e.value.status == status, e.value
+
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_step_begin, h, [0])                       # decode before prefill
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_get_seq_dims, h, 0)
+        _place(wnw, h, syn, 0, [0])
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_step_begin, h, [0])                       # only one of two layers placed
+        p = syn.prefill(0, 0)
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_place_prefill, h, 0, 1, p["k"][:-1].to(dev), p["v"][:-1].to(dev), p["audio_begin"],
+               p["audio_end"] - 1, p["q_last"].to(dev))                            # token counts differ from layer 0
+        _place(wnw, h, syn, 0, [1])
+        expect(wnw.WNW_ERR_INVALID_ARG, wnw.wnw_step_begin, h, [0, 0])              # duplicate sequence
+        expect(wnw.WNW_ERR_INVALID_ARG, wnw.wnw_step_begin, h, [5])
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_decode_layer, h, 0, q, kn, kn, out)       # no step open
+        wnw.wnw_step_begin(h, [0])
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_step_begin, h, [0])                       # step already open
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_decode_layer, h, 1, q, kn, kn, out)       # layers out of order
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_decode_layer_full, h, 0, q, kn, kn, out)  # tiered cache, full-cache entry point
+        expect(wnw.WNW_ERR_INVALID_ARG, wnw.wnw_decode_layer, h, 0, q, kn, None, out)
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_step_end, h)                              # not all layers done
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_place_prefill, h, 1, 0, p["k"].to(dev), p["v"].to(dev), p["audio_begin"],
+               p["audio_end"], p["q_last"].to(dev))                                # placement inside a step
+        wnw.wnw_decode_layer(h, 0, q, kn, kn, out)
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_decode_layer, h, 1, q, None, None, out)   # append in layer 0 but not in layer 1
+        wnw.wnw_decode_layer(h, 1, q, kn, kn, out)
+        wnw.wnw_step_end(h)
+        wnw.wnw_step_begin(h, [0]); wnw.wnw_decode_layer(h, 0, q, kn, kn, out); wnw.wnw_decode_layer(h, 1, q, kn, kn, out)
+        wnw.wnw_step_end(h)                                                        # text capacity (4 + 2 steps) is now full
+        wnw.wnw_step_begin(h, [0])
+        expect(wnw.WNW_ERR_CAPACITY, wnw.wnw_decode_layer, h, 0, q, kn, kn, out)
+        wnw.wnw_decode_layer(h, 0, q, None, None, out)                             # attending without appending still works
+        wnw.wnw_decode_layer(h, 1, q, None, None, out)
+        wnw.wnw_step_end(h)
+        wnw.wnw_sync(h)                                                            # no sticky device-side error
+        assert wnw.wnw_get_seq_dims(h, 0)[1] == 6
+        big = torch.zeros((200, w.n_kv_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+        expect(wnw.WNW_ERR_CAPACITY, wnw.wnw_place_prefill, h, 1, 0, big, big, 10, 190, p["q_last"].to(dev))   # audio > capacity
+        expect(wnw.WNW_ERR_INVALID_ARG, wnw.wnw_graph_begin, h, [0], None)          # the default stream cannot be captured
+        expect(wnw.WNW_ERR_STATE, wnw.wnw_graph_launch, h, torch.cuda.Stream())     # nothing captured yet
+    finally:
+        wnw.wnw_destroy(h)
+
+
+def test_replacing_a_sequence_invalidates_the_captured_graph():
+    import paper_2608_22704_b200 as wnw
+    dev = torch.device("cuda:0")
+    w = tiny_custom(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, n_text=4, audio_lens=(64,), chunk=16, n_steps=8)
+    syn = Synth(w, seed=2)
+    h = _mk(wnw, w)
+    try:
+        _place(wnw, h, syn, 0, [0, 1])
+        st = torch.cuda.Stream()
+        q = torch.zeros((1, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+        kn = torch.zeros((1, w.n_kv_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+        out = torch.zeros_like(q)
+        torch.cuda.synchronize()
+        wnw.wnw_graph_begin(h, [0], st)
+        wnw.wnw_step_begin(h, [0])
+        for l in range(2):
+            wnw.wnw_decode_layer(h, l, q, kn, kn, out, stream=st)
+        wnw.wnw_step_end(h, stream=st)
+        wnw.wnw_graph_end(h, st)
+        assert wnw.wnw_get_seq_dims(h, 0)[1] == 4                                  # capture ran nothing
+        wnw.wnw_graph_launch(h, st); wnw.wnw_graph_launch(h, st)
+        wnw.wnw_sync(h)
+        assert wnw.wnw_get_seq_dims(h, 0)[1] == 6
+        assert wnw.wnw_get_stats(h)["steps"] == 2
+        _place(wnw, h, syn, 0, [0, 1])                                             # re-place: work lists are rebuilt
+        with pytest.raises(wnw.WnwError) as e:
+            wnw.wnw_graph_launch(h, st)
+        assert e.value.status == wnw.WNW_ERR_STATE
+    finally:
+        wnw.wnw_destroy(h)
