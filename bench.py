@@ -344,12 +344,51 @@ def workload_config(w):
             "l2": f"flushed between steps ({L2_FLUSH_BYTES >> 20} MiB write, untimed)"}
 
 
+def run_recall_sweep(args, wnw, dev):
+    """Recall-stress grid (config-1 shapes, batch 8, 7500 audio tokens, focus jumping every 4 steps):
+    budget x chunk; per point the step time with recall, with recall copies skipped, the bytes recalled per step,
+    the sustained recall rate and the measured host-link bandwidth."""
+    link_copy, link_kernel = wnw.wnw_measure_host_link(dev.index or 0, 256 << 20, 5)
+    K, W = args.steps if args.steps != 200 else 48, max(args.warmup, 4)
+    points = []
+    for budget in (0.1, 0.2, 0.4):
+        for chunk in (16, 64, 256):
+            w = config4(seed=0, budget=budget, chunk=chunk, batch=8, n_steps=W + K)
+            job = Job(w, seed=0, device=dev, wnw=wnw)
+            job.create("wnw", wnw.WNW_MODE_TIERED)
+            job.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
+            job.place_all(["wnw", "skip"])
+            for t in range(W):
+                job.step("wnw", t); job.step("skip", t)
+            torch.cuda.synchronize(dev)
+            s0 = wnw.wnw_get_stats(job.caches["wnw"])
+            ms = sum(job.timed_steps("wnw", W, K)) / K
+            s1 = wnw.wnw_get_stats(job.caches["wnw"])
+            ms_skip = sum(job.timed_steps("skip", W, K)) / K
+            rb = (s1["recall_bytes"] - s0["recall_bytes"]) / K
+            T_a, _, C, S = wnw.wnw_get_seq_dims(job.caches["wnw"], 0)
+            points.append({"budget": budget, "chunk": chunk, "chunks": C, "slots": S, "step_us": ms * 1e3,
+                           "step_us_copies_skipped": ms_skip * 1e3, "exposed_recall_us": (ms - ms_skip) * 1e3,
+                           "recall_MB_per_step": rb / 1e6, "misses_per_step": (s1["misses"] - s0["misses"]) / K,
+                           "sustained_recall_GBps": rb / (ms * 1e-3) / 1e9,
+                           "sustained_over_link": rb / (ms * 1e-3) / 1e9 / link_kernel})
+            job.destroy()
+            del job
+            torch.cuda.empty_cache()
+    print(json.dumps({"workload": "cfg4_recall_stress_sweep", "batch": 8, "audio_tokens": 7500, "steps": K, "warmup": W,
+                      "link_memcpy_GBps": link_copy, "link_kernel_GBps": link_kernel, "points": points}), flush=True)
+
+
 def run_ours(args, rank, world, local_rank):
     import paper_2608_22704_b200 as wnw
     wnw.lib()  # fails loudly if the CUDA library is missing
     dev = torch.device(f"cuda:{local_rank}")
     torch.cuda.set_device(dev)
     peak_gbs, peak_kind = load_peaks()
+    if args.workload == "cfg4":
+        if rank == 0:
+            run_recall_sweep(args, wnw, dev)
+        return
     K, W = args.steps, args.warmup
     R = args.roofline_steps
     total = W + R + K
@@ -580,7 +619,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3", "prof", "hbm"])
+    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3", "cfg4", "prof", "hbm"])
     ap.add_argument("--no-hbm-case", action="store_true", help="skip the extra many-sequence measurement")
     ap.add_argument("--quick", action="store_true", help="only the WnW steps (for profiler captures); prints a short line")
     ap.add_argument("--no-flush", action="store_true", help="with --quick: do not flush L2 between steps")
