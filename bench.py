@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from workloads import ROLE_ANCHOR, ROLE_FIXED, ROLE_TIDAL, Synth, config1, config3, config4
+from workloads import ROLE_ANCHOR, ROLE_FIXED, ROLE_TIDAL, Synth, config1, config2, config3, config4
 from workloads.synth import bf16_bits
 
 METRIC = "wnw_decode_tokens_per_s_at_20pct_audio_budget"
@@ -48,6 +48,8 @@ def load_peaks():
 def make_workload(name: str, n_steps: int, seed: int):
     if name == "cfg1":
         w = config1(seed=0, n_steps=n_steps)
+    elif name == "cfg2":
+        w = config2(seed=0, n_steps=n_steps)
     elif name == "cfg3":
         w = config3(seed=0, n_steps=n_steps)
     elif name in ("prof", "hbm"):   # many long sequences, config-1 heads: 4 layers (profiler captures) or 12 layers (HBM-bound case)
@@ -619,7 +621,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg3", "cfg4", "prof", "hbm"])
+    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg2", "cfg3", "cfg4", "prof", "hbm"])
     ap.add_argument("--no-hbm-case", action="store_true", help="skip the extra many-sequence measurement")
     ap.add_argument("--quick", action="store_true", help="only the WnW steps (for profiler captures); prints a short line")
     ap.add_argument("--no-flush", action="store_true", help="with --quick: do not flush L2 between steps")

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from workloads import config3, config4
+from workloads import config1, config3, config4
 
 pytestmark = pytest.mark.gpu
 
@@ -37,3 +37,22 @@ def test_config4_recall_stress_corners(budget, chunk):
     every resident slot holds the exact bytes of its chunk."""
     w = config4(budget=budget, chunk=chunk, n_steps=5)
     _run(w, oracle_seqs=[3], n_steps=5)
+
+
+def test_config1_sixty_four_steps_graph_replay():
+    """3B Voxtral-shaped stack, 64 of the 256 decode steps (a quarter of the clip: the focus leaves the prefill set, chunks
+    are recalled and evicted in every layer), replayed as a CUDA graph with overlapping layer kernels; the oracle follows
+    every step.  Counters (hits, misses, evictions, recalled bytes) must agree at the end."""
+    from parity_harness import Lockstep
+    w = config1(n_steps=64)
+    ls = Lockstep(w, seed=0, gen_device="cuda:0")
+    try:
+        ls.prefill(check_slots=False)
+        for t in range(64):
+            ls.decode_step(t, graph=True, check_slots=(t % 16 == 15))
+        ls.check_stats()
+        assert ls.near_ties == 0
+        st = ls.o.stats(0)
+        assert st["misses"] > 100 and st["evictions"] > 100      # the sweep really exercises recall and eviction
+    finally:
+        ls.close()
