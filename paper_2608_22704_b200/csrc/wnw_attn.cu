@@ -212,6 +212,22 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   kslot = (int)((cv.steps[b] & 3) * 64 + a.layer);
   KSTAMP_MIN(kslot, 0);
 #endif
+  if (a.wait_epoch && role == ROLE_TIDAL) {
+    // Replayed steps: the recall that refreshed this layer's slots ran outside the captured graph, possibly still
+    // overlapping this step.  Bounded acquire-wait on the layer's epoch word before any slot is read.
+    if (lane == 0) {
+      const int expect = *a.expect_epoch;
+      int seen;
+      const long long t0 = clock64();
+      for (;;) {
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];\n" : "=r"(seen) : "l"(a.wait_epoch) : "memory");
+        if (seen >= expect) break;
+        if (clock64() - t0 > 2000000000ll) { timed_out = true; break; }
+      }
+      asm volatile("fence.proxy.async.global;\n" ::: "memory");  // the slots are read by TMA (async proxy)
+    }
+    timed_out = __shfl_sync(0xffffffffu, (int)timed_out, 0) != 0;
+  }
   int v_delta_audio;  // rows between a granule's K and V rows
   const CUtensorMap *map_audio;
   if (role == ROLE_ANCHOR) { v_delta_audio = G.T_a_pad; map_audio = &maps.anchor; }

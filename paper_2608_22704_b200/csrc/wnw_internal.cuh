@@ -126,6 +126,8 @@ struct AttnArgs {
   const int32_t *cta_ranges;     //   the item indices CTA c processes; n_ctas CTAs are launched
   int32_t n_ctas;
   int32_t throughput;            // items were cut for the 4-warp, 2-CTAs-per-SM variant (more than one wave of work)
+  const int32_t *wait_epoch;     // replayed steps: tidal CTAs wait until *wait_epoch >= *expect_epoch (this layer's recall of the
+  const int32_t *expect_epoch;   //   previous step, which runs outside the captured graph, has landed); null otherwise
   int32_t pdl;                   // launch with programmatic stream serialization (previous stream op is a layer kernel)
   const HeadItems *head_items;  // [n_active][Hkv] work items of each head (first is relative to `items`)
   const bf16 *q;         // [n_active][Hq][d]
@@ -158,12 +160,20 @@ struct SelectArgs {
   int16_t upd_layer[MAX_UPD_BY_VALUE], upd_src[MAX_UPD_BY_VALUE];
 };
 
+// Completion signalling of a recall launch that runs outside the captured step (all null for in-step launches).
+struct RecallSignal {
+  int32_t *epoch_words;       // [L] epoch of the last completed recall of each layer's table
+  int32_t *counters;          // [L] finished-CTA counters (self-resetting)
+  const int32_t *step_epoch;  // epoch to publish: the number of replayed steps that have ended
+};
+
 // kernels' host launchers (defined in the .cu files)
 cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st);
 cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, cudaStream_t st);
-cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *active, int appended, cudaStream_t st);
+cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *active, int appended, int32_t *bump_epoch,
+                            cudaStream_t st);
 cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,
-                          int skip_copy, cudaStream_t st);
+                          int skip_copy, RecallSignal sig, cudaStream_t st);
 cudaError_t launch_place_scatter(const CacheView &cv, int b, int layer, const bf16 *k, const bf16 *v, int n_tokens, int ab,
                                  int ae, int T_t, int C_b, int S_b, bf16 *stage, cudaStream_t st);
 cudaError_t launch_prefill_select(const CacheView &cv, int b, int layer, const HeadItems *head_items, const float2 *part_ml,

@@ -117,49 +117,67 @@ cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_
 }
 
 // ------------------------------------------------------------------------------------------------
-// Recall: copies every planned chunk block pinned host -> slot pool.  grid (ctas, topk, n_active * n_layers).
+// Recall: copies every planned chunk block pinned host -> slot pool.  grid (ctas, topk, n_layers * n_active), earlier
+// layers first.  With `sig` set (replayed steps, where this kernel runs outside the captured graph and overlaps the
+// next step) the last CTA of every layer publishes the layer's recall epoch, which the next step's tidal CTAs acquire.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) wnw_recall_kernel(const __grid_constant__ CacheView cv, int n_active,
                                                          const int32_t *active, const int32_t *layers, int n_layers,
-                                                         int skip_copy) {
+                                                         int skip_copy, RecallSignal sig) {
   const Geometry &G = cv.geo;
-  const int i = blockIdx.z / n_layers, l = layers[blockIdx.z % n_layers], r = blockIdx.y;
+  const int l = layers[blockIdx.z / n_active], i = blockIdx.z % n_active, r = blockIdx.y;
   const int b = active[i];
   const long long bl = (long long)b * G.L + l;
-  if (r >= cv.n_plan[bl]) return;
-  const LayerInfo li = cv.layers[l];
-  const int c = cv.plan[(bl * G.topk + r) * 2], slot = cv.plan[(bl * G.topk + r) * 2 + 1];
-  const long long n_vec = (long long)li.n_tidal * 2 * G.nc * G.d / 8;  // 16-byte vectors per chunk block
-  if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(cv.stats + (long long)b * 4 + 3, (unsigned long long)n_vec * 16ull);
-  if (skip_copy) return;
-  if (c < 0 || c >= cv.C[b] || slot < 0 || slot >= cv.S[b]) {
-    if (threadIdx.x == 0) atomicOr(cv.status, STATUS_BAD_TABLE);
-    return;
-  }
-  const uint4 *src = reinterpret_cast<const uint4 *>(cv.mirror[b] + mirror_off(G, li, cv.C[b], c, 0, 0));
-  uint4 *dst = reinterpret_cast<uint4 *>(cv.pool + pool_off(G, li, b, slot, 0, 0));
-  constexpr int U = 8;
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; v0 < n_vec; v0 += stride * U) {
-    uint4 t[U];
+  if (r < cv.n_plan[bl]) {
+    const LayerInfo li = cv.layers[l];
+    const int c = cv.plan[(bl * G.topk + r) * 2], slot = cv.plan[(bl * G.topk + r) * 2 + 1];
+    const long long n_vec = (long long)li.n_tidal * 2 * G.nc * G.d / 8;  // 16-byte vectors per chunk block
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(cv.stats + (long long)b * 4 + 3, (unsigned long long)n_vec * 16ull);
+    if (!skip_copy) {
+      if (c < 0 || c >= cv.C[b] || slot < 0 || slot >= cv.S[b]) {
+        if (threadIdx.x == 0) atomicOr(cv.status, STATUS_BAD_TABLE);
+      } else {
+        const uint4 *src = reinterpret_cast<const uint4 *>(cv.mirror[b] + mirror_off(G, li, cv.C[b], c, 0, 0));
+        uint4 *dst = reinterpret_cast<uint4 *>(cv.pool + pool_off(G, li, b, slot, 0, 0));
+        constexpr int U = 8;
+        const long long stride = (long long)gridDim.x * blockDim.x;
+        for (long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; v0 < n_vec; v0 += stride * U) {
+          uint4 t[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const long long v = v0 + u * stride;
-      if (v < n_vec) t[u] = __ldcs(src + v);
+          for (int u = 0; u < U; ++u) {
+            const long long v = v0 + u * stride;
+            if (v < n_vec) t[u] = __ldcs(src + v);
+          }
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            const long long v = v0 + u * stride;
+            if (v < n_vec) dst[v] = t[u];
+          }
+        }
+      }
     }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const long long v = v0 + u * stride;
-      if (v < n_vec) dst[v] = t[u];
+  }
+  if (sig.epoch_words) {  // completion of this layer's recall: counted per CTA, published by the last one
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const int total = gridDim.x * gridDim.y * n_active;
+      const int prev = atomicAdd(sig.counters + l, 1);
+      if (prev == total - 1) {
+        sig.counters[l] = 0;
+        __threadfence();
+        const int epoch = *sig.step_epoch;
+        asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(sig.epoch_words + l), "r"(epoch) : "memory");
+      }
     }
   }
 }
 
 cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,
-                          int skip_copy, cudaStream_t st) {
+                          int skip_copy, RecallSignal sig, cudaStream_t st) {
   if (n_layers <= 0 || n_active <= 0) return cudaSuccess;
   wnw_recall_kernel<<<dim3(8, cv.geo.topk, n_active * n_layers), 256, 0, st>>>(cv, n_active, active, layers_dev, n_layers,
-                                                                            skip_copy);
+                                                                            skip_copy, sig);
   return cudaGetLastError();
 }
 
@@ -189,15 +207,18 @@ cudaError_t launch_copy_plan(const uint4 *src, uint4 *dst, long long n_vec, int 
 // ------------------------------------------------------------------------------------------------
 // Step bookkeeping
 // ------------------------------------------------------------------------------------------------
-__global__ void wnw_step_end_kernel(const __grid_constant__ CacheView cv, int n_active, const int32_t *active, int appended) {
+__global__ void wnw_step_end_kernel(const __grid_constant__ CacheView cv, int n_active, const int32_t *active, int appended,
+                                    int32_t *bump_epoch) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i == 0 && bump_epoch) *bump_epoch += 1;  // replayed steps: the recall of this step will publish this epoch
   if (i >= n_active) return;
   const int b = active[i];
   cv.steps[b] += 1;
   if (appended) cv.text_len[b] += 1;
 }
-cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *active, int appended, cudaStream_t st) {
-  wnw_step_end_kernel<<<(n_active + 127) / 128, 128, 0, st>>>(cv, n_active, active, appended);
+cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *active, int appended, int32_t *bump_epoch,
+                            cudaStream_t st) {
+  wnw_step_end_kernel<<<(n_active + 127) / 128, 128, 0, st>>>(cv, n_active, active, appended, bump_epoch);
   return cudaGetLastError();
 }
 

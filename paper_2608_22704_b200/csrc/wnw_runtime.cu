@@ -97,6 +97,11 @@ struct wnw_cache {
   size_t gran_em_layer_stride = 0;
   bool step_capturing = false;
   bool pdl_enabled = true;
+  // replayed steps: one recall launch per step outside the captured graph, overlapping the next step
+  int32_t *d_recall_epoch = nullptr, *d_recall_ctr = nullptr, *d_step_epoch = nullptr;
+  int external_recall_mode = -1;   // -1 automatic, 0 never, 1 always
+  bool cap_external_recall = false, graph_external_recall = false, recall_all_pending = false;
+  cudaEvent_t ev_graph_done = nullptr, ev_recall_all = nullptr;
   int direct_max_granules = 64;   // heads up to this many granules (text capacity included) are not split in the latency regime
   // captured step
   bool graph_capturing = false;
@@ -162,6 +167,8 @@ static void destroy_impl(wnw_cache *c) {
   for (auto e : c->ev_side_done_cap) cudaEventDestroy(e);
   if (c->ev_place) cudaEventDestroy(c->ev_place);
   if (c->ev_step) cudaEventDestroy(c->ev_step);
+  if (c->ev_graph_done) cudaEventDestroy(c->ev_graph_done);
+  if (c->ev_recall_all) cudaEventDestroy(c->ev_recall_all);
   if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
   if (c->graph) cudaGraphDestroy(c->graph);
   for (auto &p : c->t_used) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
@@ -225,6 +232,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
 #define CKE(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { return fail(_e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA); } } while (0)
   cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
   if (const char *e = getenv("WNW_PDL")) c->pdl_enabled = atoi(e) != 0;
+  if (const char *e = getenv("WNW_EXTERNAL_RECALL")) c->external_recall_mode = atoi(e);
   if (const char *e = getenv("WNW_DIRECT_MAX_GRANULES")) c->direct_max_granules = atoi(e);
   CKE(configure_attn_kernels());
   CKE(configure_select_kernel());
@@ -376,6 +384,11 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   }
   CKE(cudaEventCreateWithFlags(&c->ev_place, cudaEventDisableTiming));
   CKE(cudaEventCreateWithFlags(&c->ev_step, cudaEventDisableTiming));
+  CKE(cudaEventCreateWithFlags(&c->ev_graph_done, cudaEventDisableTiming));
+  CKE(cudaEventCreateWithFlags(&c->ev_recall_all, cudaEventDisableTiming));
+  CKC(dev_alloc(c, &c->d_recall_epoch, (size_t)L));
+  CKC(dev_alloc(c, &c->d_recall_ctr, (size_t)L));
+  CKC(dev_alloc(c, &c->d_step_epoch, 1));
   CKE(cudaDeviceSynchronize());
 #undef CKC
 #undef CKE
@@ -599,6 +612,7 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
   // the staging buffer and the partial buffers are shared: order after earlier placements and steps
   if (c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
   if (c->step_recorded) CK(cudaStreamWaitEvent(st, c->ev_step, 0));
+  if (c->recall_all_pending) CK(cudaStreamWaitEvent(st, c->ev_recall_all, 0));
   CK(launch_place_scatter(c->cv, seq, layer, (const bf16 *)k_dev, (const bf16 *)v_dev, n_tokens, audio_begin, audio_end, T_t,
                           C_b, S_b, c->stage, st));
   if (!full && C_b > 0) {
@@ -707,8 +721,21 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   const bool capturing = stream_is_capturing(st);
   if (layer == 0) c->step_capturing = capturing;
   else if (capturing != c->step_capturing) return WNW_ERR_STATE;
+  if (layer == 0) {
+    // Replayed steps of small launches (latency regime) take their recall out of the captured graph, so that it can
+    // overlap the next replay.  In the throughput regime the persistent attention CTAs would sit on their SMs while
+    // they wait for it, so recall stays inside the step there.
+    bool small = true;
+    for (const LayerWork &w : c->wl_layers) small = small && !w.throughput;
+    c->cap_external_recall = capturing && c->graph_capturing && tiered && c->cfg.recall_mode != WNW_RECALL_INLINE &&
+                             (c->external_recall_mode == 1 || (c->external_recall_mode < 0 && small));
+  }
   if (!capturing) {
     if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
+    if (layer == 0 && c->recall_all_pending) {  // the recall launch that followed the last replayed step
+      CK(cudaStreamWaitEvent(st, c->ev_recall_all, 0));
+      c->recall_all_pending = false;
+    }
     // side-stream work of the previous step that this layer depends on must have landed: the selection kernel that
     // read this layer's partial buffers, and the recall that refreshed this layer's slots
     if (tiered && c->cfg.recall_mode != WNW_RECALL_INLINE) {
@@ -736,6 +763,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   a.anchor_head0 = tiered ? li.anchor_off : layer * G.Hkv;
   a.part_o = c->part_o + lw.part_off * G.g * G.d; a.part_ml = c->part_ml + lw.part_off * G.g;
   a.gran_em = gran_em_l;
+  if (c->cap_external_recall && li.n_tidal > 0) { a.wait_epoch = c->d_recall_epoch + layer; a.expect_epoch = c->d_step_epoch; }
   // overlap with the previous layer's kernel when that is what precedes this launch in the stream
   a.pdl = layer > 0 && c->pdl_enabled;
   a.n_aq = std::max(li.n_anchor * G.g, 1); a.n_ag_max = c->n_ag_max;
@@ -782,9 +810,9 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
       }
     }
     CK(launch_select(c->cv, sa, c->sel_smem[layer], ss));
-    if (li.upd_count > 0)
+    if (li.upd_count > 0 && !c->cap_external_recall)
       CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count,
-                       c->cfg.recall_mode == WNW_RECALL_SKIP, ss));
+                       c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{nullptr, nullptr, nullptr}, ss));
     if (!inline_mode) {
       CK(cudaEventRecord(ev_s, ss));
       if (!capturing) c->side_recorded[layer] = 1;
@@ -816,7 +844,8 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
   if (capturing && c->cfg.recall_mode != WNW_RECALL_INLINE)
     for (int ls : c->last_side_layer)  // join the forked side streams into the graph
       if (ls >= 0) CK(cudaStreamWaitEvent(st, c->ev_side_done_cap[ls], 0));
-  CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1, st));
+  CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1,
+                     (capturing && c->cap_external_recall) ? c->d_step_epoch : nullptr, st));
   if (!capturing) {
     CK(cudaEventRecord(c->ev_step, st));
     c->step_recorded = true;
@@ -879,6 +908,8 @@ extern "C" wnw_status_t wnw_graph_end(wnw_cache_t *c, void *cuda_stream) {
   c->graph = g;
   CK(cudaGraphInstantiate(&c->graph_exec, g, 0));
   c->graph_epoch = c->wl_epoch;
+  c->graph_external_recall = c->cap_external_recall;
+  c->cap_external_recall = false;
   return WNW_OK;
 }
 
@@ -898,6 +929,17 @@ extern "C" wnw_status_t wnw_graph_launch(wnw_cache_t *c, void *cuda_stream) {
   for (int l = 0; l < c->geo.L; ++l)
     if (c->side_recorded[l]) { CK(cudaStreamWaitEvent(st, c->ev_side_done[l], 0)); c->side_recorded[l] = 0; }
   CK(cudaGraphLaunch(c->graph_exec, st));
+  if (c->graph_external_recall && !c->upd_list.empty()) {
+    // This step's recall, for every layer's table at once, outside the graph: it overlaps the next replay, whose tidal
+    // CTAs wait on the per-layer epoch words it publishes.
+    CK(cudaEventRecord(c->ev_graph_done, st));
+    CK(cudaStreamWaitEvent(c->side[0], c->ev_graph_done, 0));
+    CK(launch_recall(c->cv, (int)c->graph_active.size(), c->d_active, c->cv.upd_list, (int)c->upd_list.size(),
+                     c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{c->d_recall_epoch, c->d_recall_ctr, c->d_step_epoch},
+                     c->side[0]));
+    CK(cudaEventRecord(c->ev_recall_all, c->side[0]));
+    c->recall_all_pending = true;
+  }
   CK(cudaEventRecord(c->ev_step, st));
   c->step_recorded = true;
   for (int b : c->graph_active)
