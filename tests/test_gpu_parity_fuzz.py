@@ -1,0 +1,45 @@
+"""Randomised small configurations: roles, group size, head_dim, chunk, budget, batch, ragged lengths, routing, eager and
+graph replay mixed.  Every case runs the full lock-step parity check against the oracle (needs a B200)."""
+import numpy as np
+import pytest
+
+from workloads import ROLE_ANCHOR, ROLE_FIXED, ROLE_TIDAL, tiny_custom
+
+pytestmark = pytest.mark.gpu
+
+
+def _draw(seed):
+    rs = np.random.RandomState(1000 + seed)
+    n_layers = int(rs.randint(1, 6))
+    hkv = int(rs.choice([1, 2, 4, 8]))
+    g = int(rs.choice([1, 2, 4, 8, 16]))
+    while hkv * g > 128:
+        g //= 2
+    d = int(rs.choice([64, 128]))
+    chunk = int(rs.choice([16, 32, 64]))
+    batch = int(rs.randint(1, 4))
+    lens = [int(rs.randint(0, 12) * chunk + rs.randint(0, chunk)) for _ in range(batch)]
+    if sum(lens) == 0:
+        lens[0] = chunk * 3 + 5
+    roles = rs.choice([ROLE_ANCHOR, ROLE_TIDAL, ROLE_FIXED], size=(n_layers, hkv), p=[0.25, 0.45, 0.3]).astype(np.uint8)
+    if not (roles == ROLE_ANCHOR).any():
+        roles[rs.randint(n_layers), rs.randint(hkv)] = ROLE_ANCHOR
+    return tiny_custom(n_layers=n_layers, n_q_heads=hkv * g, n_kv_heads=hkv, head_dim=d, n_text=int(rs.randint(0, 40)),
+                       audio_lens=tuple(lens), chunk=chunk, budget=float(rs.choice([0.1, 0.25, 0.5, 1.0])), n_steps=6,
+                       roles=roles, topk=int(rs.randint(1, 5)), region=chunk, jump_every=int(rs.choice([0, 2])),
+                       name=f"fuzz{seed}"), rs
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_configuration(seed):
+    from parity_harness import Lockstep
+    w, rs = _draw(seed)
+    ls = Lockstep(w, seed=seed)
+    try:
+        ls.prefill()
+        use_graph = bool(seed % 2)
+        for t in range(w.n_steps):
+            ls.decode_step(t, append=True, graph=use_graph and t not in (0, 3), check_slots=True)
+        ls.check_stats()
+    finally:
+        ls.close()
