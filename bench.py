@@ -35,6 +35,7 @@ from workloads.synth import bf16_bits
 METRIC = "wnw_decode_tokens_per_s_at_20pct_audio_budget"
 UNIT = "tokens/s"
 L2_FLUSH_BYTES = 512 << 20
+SWEEP_STEPS_OVERRIDE = 0
 
 
 def load_peaks():
@@ -58,6 +59,9 @@ def make_workload(name: str, n_steps: int, seed: int):
         w.n_layers = n_l; w.roles = w.roles[:n_l]; w.jump_every = 0; w.sweep_steps = 128; w.name = f"{name}_{n_l}layers_b16_7500"
     else:
         raise SystemExit(f"unknown workload {name}")
+    if SWEEP_STEPS_OVERRIDE:
+        w.sweep_steps = SWEEP_STEPS_OVERRIDE   # slower or faster drift of the decode focus through the clip
+        w.name += f"_sweep{SWEEP_STEPS_OVERRIDE}"
     return w
 
 
@@ -631,7 +635,12 @@ def main():
     ap.add_argument("--roofline-steps", type=int, default=16)
     ap.add_argument("--oracle-layers", type=int, default=6, help="layers of sequence 0 the CPU baseline samples (0 = skip)")
     ap.add_argument("--oracle-steps", type=int, default=4)
+    ap.add_argument("--sweep-steps", type=int, default=0,
+                    help="decode steps for one sweep of the focus through the clip (0: the workload's own; e.g. 1200 on cfg3 is "
+                         "about 4 audio tokens per generated token, a speech-like rate)")
     args = ap.parse_args()
+    global SWEEP_STEPS_OVERRIDE
+    SWEEP_STEPS_OVERRIDE = args.sweep_steps
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     rank = int(os.environ.get("RANK", "0"))

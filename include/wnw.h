@@ -76,7 +76,7 @@ typedef struct {
   int32_t max_batch;                       /* sequences the cache can hold */
   int32_t max_audio_tokens;                /* per sequence */
   int32_t max_text_tokens;                 /* per sequence, prompt text + every decode append */
-  int32_t chunk_tokens;                    /* n_c; multiple of 16 */
+  int32_t chunk_tokens;                    /* n_c >= 1 (e.g. ceil(4 s * 12.5 tok/s) = 50, "Chunk Structure"); stored padded to 16 rows */
   int32_t topk;                            /* k, chunks selected per step; 0 -> 3 (the paper's k) */
   int32_t evict_lag;                       /* the paper's delta; accepted, reserved (fixed pool evicts least-recent) */
   float budget;                            /* (0,1]; see S above */
@@ -100,7 +100,7 @@ typedef struct {
 /* Create a cache: head roles from the offline triage, GPU budget, capacities.
  * Allocates all device stores up front; pinned host mirrors are allocated per
  * sequence at prefill.  Rejects: tidal heads with no anchor anywhere, head_dim
- * not in {64,128}, chunk_tokens not a multiple of 16, budget outside (0,1],
+ * not in {64,128}, budget outside (0,1],
  * group > 16.  ("Three-Way Classification"; Eq. 1 budget; "Chunk Structure".) */
 wnw_status_t wnw_create(const wnw_config_t *cfg_host, wnw_cache_t **out);
 

@@ -129,7 +129,7 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
   const int ag = j - G.n_tg, ci = ag / G.gpc, off = (ag - ci * G.gpc) * GR;
   r.off = off;
   if (it.role == ROLE_ANCHOR) {
-    r.row = (int)(anchor_off(G, a.anchor_seq_stride, it.b, a.anchor_head0 + it.ridx, 0) / G.d) + ci * G.nc + off;
+    r.row = (int)(anchor_off(G, a.anchor_seq_stride, it.b, a.anchor_head0 + it.ridx, 0) / G.d) + ci * G.ncp + off;
     int len = it.T_a - ci * G.nc;
     if (len > G.nc) len = G.nc;
     len -= off;
@@ -141,7 +141,7 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
     r.meta = -2;
   } else {
     const long long fh = (long long)it.b * G.F_tot + li.fixed_off + it.ridx;
-    r.row = (int)(fixed_off(G, li, it.b, it.ridx, 0) / G.d) + ci * G.nc + off;
+    r.row = (int)(fixed_off(G, li, it.b, it.ridx, 0) / G.d) + ci * G.ncp + off;
     r.cid = cv.fixed_chunks[fh * G.S_max + ci];
     r.meta = -2;
   }
@@ -231,8 +231,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   int v_delta_audio;  // rows between a granule's K and V rows
   const CUtensorMap *map_audio;
   if (role == ROLE_ANCHOR) { v_delta_audio = G.T_a_pad; map_audio = &maps.anchor; }
-  else if (role == ROLE_TIDAL) { v_delta_audio = G.nc; map_audio = &maps.pool; }
-  else { v_delta_audio = G.S_max * G.nc; map_audio = &maps.fixed; }
+  else if (role == ROLE_TIDAL) { v_delta_audio = G.ncp; map_audio = &maps.pool; }
+  else { v_delta_audio = G.S_max * G.ncp; map_audio = &maps.fixed; }
   const int v_delta_text = G.T_cap_pad;
 
   const int first = it.g0 + warp;

@@ -50,7 +50,8 @@ struct LayerInfo {
 };
 
 struct Geometry {
-  int32_t L, Hq, Hkv, d, g, nc, gpc, topk;
+  int32_t L, Hq, Hkv, d, g, nc, gpc, topk;  // nc: audio tokens per chunk; gpc: 16-token granules per stored chunk
+  int32_t ncp;                              // rows a chunk occupies in every store: nc rounded up to whole granules
   int32_t T_cap_pad, n_tg;         // text capacity (multiple of 16) and its granules
   int32_t C_max, S_max, T_a_pad;   // chunk / slot capacity per sequence; audio capacity padded to whole chunks
   int32_t A_tot, F_tot;            // anchor / fixed heads per sequence over all layers
@@ -89,13 +90,13 @@ __host__ __device__ inline long long anchor_off(const Geometry &G, long long seq
   return (long long)b * seq_stride + ((long long)head * 2 + kv) * G.T_a_pad * G.d;
 }
 __host__ __device__ inline long long pool_off(const Geometry &G, const LayerInfo &li, int b, int slot, int t_idx, int kv) {
-  return (long long)b * G.pool_seq_stride + li.pool_off + ((long long)(slot * li.n_tidal + t_idx) * 2 + kv) * G.nc * G.d;
+  return (long long)b * G.pool_seq_stride + li.pool_off + ((long long)(slot * li.n_tidal + t_idx) * 2 + kv) * G.ncp * G.d;
 }
 __host__ __device__ inline long long fixed_off(const Geometry &G, const LayerInfo &li, int b, int f_idx, int kv) {
-  return (long long)b * G.fixed_seq_stride + ((long long)(li.fixed_off + f_idx) * 2 + kv) * G.S_max * G.nc * G.d;
+  return (long long)b * G.fixed_seq_stride + ((long long)(li.fixed_off + f_idx) * 2 + kv) * G.S_max * G.ncp * G.d;
 }
 __host__ __device__ inline long long mirror_off(const Geometry &G, const LayerInfo &li, int C_b, int c, int t_idx, int kv) {
-  return (((long long)C_b * li.tid_prefix + (long long)c * li.n_tidal + t_idx) * 2 + kv) * G.nc * G.d;
+  return (((long long)C_b * li.tid_prefix + (long long)c * li.n_tidal + t_idx) * 2 + kv) * G.ncp * G.d;
 }
 
 // shared-memory workspace of one table update in the selection kernel: keys[C] u64, stamp[S] i64, slot[S] i32, scores[C] f32

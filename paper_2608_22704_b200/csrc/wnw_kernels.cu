@@ -22,7 +22,6 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
   const long long step_b = cv.steps[b];
   const int n_aq = a.n_aq;
   const bool scored = li.n_anchor > 0 && a.score_on && C_b > 0;
-  const int n_ag = (T_a + GR - 1) / GR;  // granules that hold audio
   // shared-memory layout: (M,Z) of the anchor q-heads | this layer's scores | per-warp update workspaces | granule partials
   float2 *mz_s = reinterpret_cast<float2 *>(smem);
   float *sc_s = reinterpret_cast<float *>(smem + ((size_t)n_aq * 8 + 15) / 16 * 16);
@@ -44,7 +43,8 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
     const int span = (c1 - c0) * G.gpc, ag0 = c0 * G.gpc;
     for (int idx = threadIdx.x; idx < n_aq * span; idx += NT) {
       const int aq = idx / span, ag = ag0 + (idx - aq * span);
-      if (ag < n_ag) cp_async_small(em_s + idx, a.gran_em + ((long long)i * n_aq + aq) * a.n_ag_max + ag, 8);
+      const int cc = ag / G.gpc, gi = ag - cc * G.gpc;   // a granule holds audio iff it starts inside its chunk's tokens
+      if (gi * GR < chunk_len(G, T_a, cc)) cp_async_small(em_s + idx, a.gran_em + ((long long)i * n_aq + aq) * a.n_ag_max + ag, 8);
       else em_s[idx] = make_float2(0.f, 0.f);
     }
   };
@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(256) wnw_recall_kernel(const __grid_constant__
   if (r < cv.n_plan[bl]) {
     const LayerInfo li = cv.layers[l];
     const int c = cv.plan[(bl * G.topk + r) * 2], slot = cv.plan[(bl * G.topk + r) * 2 + 1];
-    const long long n_vec = (long long)li.n_tidal * 2 * G.nc * G.d / 8;  // 16-byte vectors per chunk block
+    const long long n_vec = (long long)li.n_tidal * 2 * G.ncp * G.d / 8;  // 16-byte vectors per chunk block
     if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(cv.stats + (long long)b * 4 + 3, (unsigned long long)n_vec * 16ull);
     if (!skip_copy) {
       if (c < 0 || c >= cv.C[b] || slot < 0 || slot >= cv.S[b]) {
@@ -248,22 +248,20 @@ __global__ void __launch_bounds__(256) wnw_place_scatter_kernel(const __grid_con
     const LayerInfo li = cv.layers[layer];
     for (int f = threadIdx.x; f < li.n_fixed; f += blockDim.x) cv.fixed_n[(long long)b * G.F_tot + li.fixed_off + f] = 0;
   }
-  const int rows_total = n_tokens + (C_b * G.nc - T_a);  // real tokens, then staging pad rows
-  const long long work = (long long)rows_total * G.Hkv * 2 * vec_per_row;
+  const long long work = (long long)n_tokens * G.Hkv * 2 * vec_per_row;   // the staging copy was zeroed by the caller
   for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < work; idx += (long long)gridDim.x * blockDim.x) {
     const int vv = (int)(idx % vec_per_row);
     long long t = idx / vec_per_row;
     const int kv = (int)(t % 2); t /= 2;
     const int h = (int)(t % G.Hkv);
     const int tok = (int)(t / G.Hkv);
-    uint4 val = make_uint4(0, 0, 0, 0);
+    const uint4 val = *reinterpret_cast<const uint4 *>((kv ? v : k) + ((long long)tok * G.Hkv + h) * G.d + vv * 8);
     bf16 *dst;
-    if (tok < n_tokens) {
-      val = *reinterpret_cast<const uint4 *>((kv ? v : k) + ((long long)tok * G.Hkv + h) * G.d + vv * 8);
-      if (tok >= ab && tok < ae) dst = stage + anchor_off(G, 0, 0, h, kv) + (long long)(tok - ab) * G.d + vv * 8;
-      else dst = cv.text + text_off(G, b, layer, h, kv) + (long long)(tok < ab ? tok : tok - T_a) * G.d + vv * 8;
+    if (tok >= ab && tok < ae) {  // audio token tau sits in row (tau / nc) * ncp + tau % nc: every chunk starts on a granule
+      const int tau = tok - ab, cc = tau / G.nc;
+      dst = stage + anchor_off(G, 0, 0, h, kv) + (long long)(cc * G.ncp + (tau - cc * G.nc)) * G.d + vv * 8;
     } else {
-      dst = stage + anchor_off(G, 0, 0, h, kv) + (long long)(T_a + (tok - n_tokens)) * G.d + vv * 8;
+      dst = cv.text + text_off(G, b, layer, h, kv) + (long long)(tok < ab ? tok : tok - T_a) * G.d + vv * 8;
     }
     *reinterpret_cast<uint4 *>(dst) = val;
   }
@@ -314,7 +312,7 @@ __global__ void __launch_bounds__(512) wnw_prefill_select_kernel(const __grid_co
         const float2 *ge = gran_em + (long long)hq * n_ag_max + (long long)c * G.gpc;
         float sum_h = 0.f;
         for (int gi = 0; gi < G.gpc; ++gi) {
-          if (c * G.nc + gi * GR >= T_a) break;
+          if (gi * GR >= chunk_len(G, T_a, c)) break;
           sum_h += ge[gi].x * exp2f(ge[gi].y - sM[hq]);
         }
         total += sZ[hq] > 0.f ? sum_h / sZ[hq] : 0.f;
@@ -375,18 +373,18 @@ __global__ void __launch_bounds__(128) wnw_place_gather_kernel(const __grid_cons
   const long long bl = (long long)b * G.L + layer;
   const int role = full_mode ? ROLE_ANCHOR : cv.roles[layer * G.Hkv + h];
   const int ridx = full_mode ? h : cv.role_idx[layer * G.Hkv + h];
-  const int vec_per_chunk = G.nc * G.d / 8;
+  const int vec_per_chunk = G.ncp * G.d / 8;
   bf16 *dst0[2] = {nullptr, nullptr}, *dst1[2] = {nullptr, nullptr};
   if (role == ROLE_ANCHOR) {
     const int head = full_mode ? layer * G.Hkv + h : li.anchor_off + ridx;
-    for (int kv = 0; kv < 2; ++kv) dst0[kv] = cv.anchor + anchor_off(G, G.anchor_seq_stride, b, head, kv) + (long long)c * G.nc * G.d;
+    for (int kv = 0; kv < 2; ++kv) dst0[kv] = cv.anchor + anchor_off(G, G.anchor_seq_stride, b, head, kv) + (long long)c * G.ncp * G.d;
   } else if (role == ROLE_FIXED) {
     const long long fh = (long long)b * G.F_tot + li.fixed_off + ridx;
     int pos = -1;
     for (int s = 0; s < cv.fixed_n[fh]; ++s)
       if (cv.fixed_chunks[fh * G.S_max + s] == c) pos = s;
     if (pos < 0) return;
-    for (int kv = 0; kv < 2; ++kv) dst0[kv] = cv.fixed + fixed_off(G, li, b, ridx, kv) + (long long)pos * G.nc * G.d;
+    for (int kv = 0; kv < 2; ++kv) dst0[kv] = cv.fixed + fixed_off(G, li, b, ridx, kv) + (long long)pos * G.ncp * G.d;
   } else {
     const int slot = cv.chunk_slot[bl * G.C_max + c];
     for (int kv = 0; kv < 2; ++kv) {
@@ -395,7 +393,7 @@ __global__ void __launch_bounds__(128) wnw_place_gather_kernel(const __grid_cons
     }
   }
   for (int kv = 0; kv < 2; ++kv) {
-    const uint4 *src = reinterpret_cast<const uint4 *>(stage + anchor_off(G, 0, 0, h, kv) + (long long)c * G.nc * G.d);
+    const uint4 *src = reinterpret_cast<const uint4 *>(stage + anchor_off(G, 0, 0, h, kv) + (long long)c * G.ncp * G.d);
     uint4 *d0 = reinterpret_cast<uint4 *>(dst0[kv]), *d1 = reinterpret_cast<uint4 *>(dst1[kv]);
     for (int v = threadIdx.x; v < vec_per_chunk; v += blockDim.x) {
       const uint4 val = src[v];  // staging pad rows are zero

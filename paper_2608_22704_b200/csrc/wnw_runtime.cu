@@ -211,7 +211,6 @@ static wnw_status_t validate_config(const wnw_config_t *cfg) {
   }
   if (cfg->mode == WNW_MODE_TIERED && any_tidal && !any_anchor) return WNW_ERR_INVALID_ARG;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return WNW_ERR_UNSUPPORTED;
-  if (cfg->chunk_tokens % GR) return WNW_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > MAX_G || cfg->n_q_heads > MAX_AQ || cfg->n_layers > 32767) return WNW_ERR_UNSUPPORTED;
   return WNW_OK;
 }
@@ -241,13 +240,13 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   c->roles.assign(cfg->roles, cfg->roles + (size_t)L * Hkv);
   c->cfg.roles = nullptr;
   Geometry &G = c->geo;
-  G.L = L; G.Hq = cfg->n_q_heads; G.Hkv = Hkv; G.d = d; G.g = cfg->n_q_heads / Hkv; G.nc = nc; G.gpc = nc / GR;
+  G.L = L; G.Hq = cfg->n_q_heads; G.Hkv = Hkv; G.d = d; G.g = cfg->n_q_heads / Hkv; G.nc = nc; G.ncp = (nc + GR - 1) / GR * GR; G.gpc = G.ncp / GR;
   G.topk = c->cfg.topk;
   G.T_cap_pad = (std::max(cfg->max_text_tokens, 1) + GR - 1) / GR * GR;
   G.n_tg = G.T_cap_pad / GR;
   G.C_max = (cfg->max_audio_tokens + nc - 1) / nc;
   G.S_max = full ? 0 : slots_for(cfg->budget, G.C_max);
-  G.T_a_pad = std::max(G.C_max, 1) * nc;
+  G.T_a_pad = std::max(G.C_max, 1) * G.ncp;
   G.max_batch = cfg->max_batch;
   const double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / std::sqrt((double)d);
   G.scale_log2 = (float)(scale * 1.4426950408889634);
@@ -267,7 +266,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
       else ri = (int16_t)li.n_fixed++;
     }
     a_tot += li.n_anchor; f_tot += li.n_fixed; t_tot += li.n_tidal;
-    pool_elems += (long long)G.S_max * li.n_tidal * 2 * nc * d;
+    pool_elems += (long long)G.S_max * li.n_tidal * 2 * G.ncp * d;
   }
   c->tid_total = t_tot;
   c->tail_of.assign(L, -1);
@@ -292,7 +291,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   G.text_seq_stride = (long long)L * Hkv * 2 * G.T_cap_pad * d;
   G.anchor_seq_stride = (long long)G.A_tot * 2 * G.T_a_pad * d;
   G.pool_seq_stride = full ? 0 : pool_elems;
-  G.fixed_seq_stride = (long long)G.F_tot * 2 * G.S_max * nc * d;
+  G.fixed_seq_stride = (long long)G.F_tot * 2 * G.S_max * G.ncp * d;
 
   CacheView &cv = c->cv;
   memset(&cv, 0, sizeof(cv));
@@ -586,7 +585,7 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (layer == 0) {
     s.placed_layers = 0;
-    const size_t need = full ? 0 : (size_t)C_b * c->tid_total * 2 * G.nc * G.d * sizeof(bf16);
+    const size_t need = full ? 0 : (size_t)C_b * c->tid_total * 2 * G.ncp * G.d * sizeof(bf16);
     if (need != s.mirror_bytes) {
       CK(cudaDeviceSynchronize());
       if (s.mirror) cudaFreeHost(s.mirror);
@@ -613,6 +612,8 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
   if (c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
   if (c->step_recorded) CK(cudaStreamWaitEvent(st, c->ev_step, 0));
   if (c->recall_all_pending) CK(cudaStreamWaitEvent(st, c->ev_recall_all, 0));
+  // chunks start on granule boundaries in every store; the rows between a chunk's last token and the next chunk are zero
+  CK(cudaMemsetAsync(c->stage, 0, (size_t)G.Hkv * 2 * G.T_a_pad * G.d * sizeof(bf16), st));
   CK(launch_place_scatter(c->cv, seq, layer, (const bf16 *)k_dev, (const bf16 *)v_dev, n_tokens, audio_begin, audio_end, T_t,
                           C_b, S_b, c->stage, st));
   if (!full && C_b > 0) {

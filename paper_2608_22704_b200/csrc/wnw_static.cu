@@ -99,7 +99,7 @@ extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, 
   memset(&cv, 0, sizeof(cv));
   Geometry &G = cv.geo;
   G.L = 1; G.Hq = n_q_heads; G.Hkv = n_kv_heads; G.d = head_dim; G.g = n_q_heads / n_kv_heads;
-  G.nc = GR; G.gpc = 1; G.topk = 0;
+  G.nc = GR; G.ncp = GR; G.gpc = 1; G.topk = 0;
   G.T_cap_pad = GR; G.n_tg = 0;                        // no text region: every key comes from kv_dev
   G.C_max = padded_tokens / GR; G.S_max = 0; G.T_a_pad = padded_tokens;
   G.max_batch = 1;

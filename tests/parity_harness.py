@@ -234,7 +234,7 @@ class Lockstep:
                 tab, stamp = prev_tab[(b, l)][0].copy(), prev_tab[(b, l)][1].copy()
                 plan, _ = wo.table_update(tab, stamp, want_sel, steps_before[b], w.topk)
                 n_tid = int((w.roles[l] == ROLE_TIDAL).sum())
-                self.expected_recall_bytes += len(plan) * n_tid * 2 * w.chunk * w.head_dim * 2
+                self.expected_recall_bytes += len(plan) * n_tid * 2 * (-(-w.chunk // 16) * 16) * w.head_dim * 2   # blocks are stored padded to 16 rows
                 assert g_tab.tolist() == tab.tolist(), f"table (ii) step {t} b{b} l{l}"
                 assert g_stamp.tolist() == stamp.tolist(), f"stamps (ii) step {t} b{b} l{l}"
                 # (iii) oracle on its own scores

@@ -37,7 +37,7 @@ def test_status_strings():
     (dict(budget=0.0), wnw.WNW_ERR_INVALID_ARG),
     (dict(budget=1.5), wnw.WNW_ERR_INVALID_ARG),
     (dict(head_dim=96), wnw.WNW_ERR_UNSUPPORTED),
-    (dict(chunk_tokens=50), wnw.WNW_ERR_UNSUPPORTED),
+    (dict(chunk_tokens=0), wnw.WNW_ERR_INVALID_ARG),
     (dict(n_q_heads=7), wnw.WNW_ERR_INVALID_ARG),
     (dict(n_q_heads=4 * 32), wnw.WNW_ERR_UNSUPPORTED),
     (dict(topk=99), wnw.WNW_ERR_INVALID_ARG),

@@ -44,6 +44,10 @@ def test_config0_without_append():
     (200, 16, 64, 32, 2),     # g = 16 (both row halves of the mma tile)
     (48, 16, 128, 2, 2),      # g = 1
     (1000, 256, 128, 8, 4),   # chunk spans many granules
+    (3000 // 4, 50, 128, 8, 2),    # the paper's n_c = ceil(4 s * 12.5 tok/s) = 50: chunks stored padded to 64 rows
+    (1500, 100, 128, 16, 2),       # n_c = ceil(4 s * 25 tok/s) = 100, g = 8
+    (333, 25, 64, 4, 2),           # n_s = 25 tokens
+    (77, 7, 64, 2, 2),             # smaller than a granule
 ])
 def test_small_shapes(audio_len, chunk, d, hq, hkv):
     roles = [[A, T] + [F, T][: hkv - 2], [T, F] + [A, T][: hkv - 2], [A, F] + [T, T][: hkv - 2]]

@@ -16,7 +16,7 @@ def _draw(seed):
     while hkv * g > 128:
         g //= 2
     d = int(rs.choice([64, 128]))
-    chunk = int(rs.choice([16, 32, 64]))
+    chunk = int(rs.choice([16, 32, 64, 25, 50, 40, 9]))
     batch = int(rs.randint(1, 4))
     lens = [int(rs.randint(0, 12) * chunk + rs.randint(0, chunk)) for _ in range(batch)]
     if sum(lens) == 0:

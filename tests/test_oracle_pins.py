@@ -347,3 +347,32 @@ def test_selection_used_from_next_step():
     p2, _ = o.attention_row(0, 0, 2, q8[2])
     seen2 = set(np.nonzero(p2[T_t:].reshape(C, w.chunk).sum(axis=1))[0].tolist())
     assert seen2 == set(after.tolist())
+
+
+# ---------------------------------------------------------------- chunk geometry constants printed in the paper
+def test_paper_chunk_geometry_constants():
+    """W_c = 4 s, W_s = 2 s: 12.5 tok/s gives n_c = 50, n_s = 25; 25 tok/s gives 100 and 50 ("Chunk Structure")."""
+    from workloads import paper_chunk_geometry
+    assert paper_chunk_geometry(4, 2, 12.5) == (50, 25)
+    assert paper_chunk_geometry(4, 2, 25) == (100, 50)
+
+
+def test_oracle_accepts_the_papers_chunk_size():
+    """Chunks of 50 tokens (not a multiple of anything convenient): budget 1.0 still equals dense attention and the
+    chunk scores still sum to the anchor audio mass."""
+    w = tiny_custom(n_layers=1, n_q_heads=4, n_kv_heads=2, head_dim=64, n_text=3, audio_lens=(230,), chunk=50, budget=1.0,
+                    roles=[[ROLE_ANCHOR, ROLE_TIDAL]], n_steps=1)
+    syn = Synth(w, seed=4)
+    o = make_oracle(w)
+    kept = place_all(o, syn, keep=True)
+    assert o.dims(0)[2:] == (5, 5)
+    q = bf16_bits(syn.decode(0, 0)["q"][0])
+    mass = 0.0
+    for hq in (0, 1):
+        p, _ = o.attention_row(0, 0, hq, q[hq])
+        mass += p[3:].sum()
+    o.step_begin([0]); out = o.decode_layer(0, q[None]); o.step_end()
+    assert abs(o.chunk_scores(0, 0).sum() - mass) < 1e-12
+    K, V, _, ab, ae = kept[(0, 0)]
+    ref, _ = dense_attention(bf16_bits_to_f64(q[2]), K[:, 1], V[:, 1], 1 / math.sqrt(64))
+    assert np.abs(out[0, 2] - ref).max() < 1e-12

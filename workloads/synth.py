@@ -78,6 +78,12 @@ class Workload:
         return -(-self.audio_lens[seq] // self.chunk)
 
 
+def paper_chunk_geometry(window_s: float, stride_s: float, tokens_per_s: float):
+    """Tokens per chunk and per segment for a chunk window and stride in seconds at an audio frame rate
+    ("Chunk Structure": n_c = ceil(W_c r_tok), n_s = ceil(W_s r_tok))."""
+    return math.ceil(window_s * tokens_per_s), math.ceil(stride_s * tokens_per_s)
+
+
 def _mix(seed: int, tag: int, a: int = 0, b: int = 0) -> int:
     x = (seed + 1) * 0x9E3779B97F4A7C15 + tag * 0xBF58476D1CE4E5B9 + a * 0x94D049BB133111EB + b * 0xD6E8FEB86659FD93
     x ^= x >> 31
