@@ -137,7 +137,8 @@ class ClockSampler:
 class Job:
     """Caches, resident inputs and launch helpers of one rank."""
 
-    def __init__(self, w, seed, device, wnw):
+    def __init__(self, w, seed, device, wnw, score_scope=0):
+        self.score_scope = score_scope
         self.w, self.dev, self.wnw = w, device, wnw
         self.syn = Synth(w, seed=seed, device=str(device))
         self.B = w.batch
@@ -167,7 +168,7 @@ class Job:
         w, wnw = self.w, self.wnw
         h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, self.B, max(w.audio_lens), w.text_capacity,
                            w.chunk, w.budget, w.roles, topk=w.topk, device=self.dev.index or 0, mode=mode,
-                           recall_mode=recall_mode)
+                           recall_mode=recall_mode, score_scope=self.score_scope)
         self.caches[key] = h
         return h
 
@@ -399,7 +400,7 @@ def run_ours(args, rank, world, local_rank):
     R = args.roofline_steps
     total = W + R + K
     w = make_workload(args.workload, total, 0)
-    job = Job(w, seed=rank, device=dev, wnw=wnw)
+    job = Job(w, seed=rank, device=dev, wnw=wnw, score_scope=args.score_scope)
     job.create("wnw", wnw.WNW_MODE_FULL if args.quick_full else wnw.WNW_MODE_TIERED, recall_mode=args.recall_mode)
     if args.quick:   # profiler mode: the WnW steps only, nothing else launched
         job.place_all(["wnw"])
@@ -589,7 +590,8 @@ def run_ours(args, rank, world, local_rank):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(w), launch="eager" if args.eager else "cuda graph replay of the step"),
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(w), launch="eager" if args.eager else "cuda graph replay of the step",
+                                                                                score_scope="global" if args.score_scope else "per layer"),
         "clocks": clocks, "gpu_launches": launches_per_step * K,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e},
         # achieved: algorithmic K,V bytes of one launch / its duration, each launch bracketed by CUDA events on the launching
@@ -631,6 +633,8 @@ def main():
     ap.add_argument("--no-flush", action="store_true", help="with --quick: do not flush L2 between steps")
     ap.add_argument("--recall-mode", type=int, default=0, help="with --quick: 0 side stream, 1 inline, 2 copies skipped")
     ap.add_argument("--quick-full", action="store_true", help="with --quick: time the full-cache comparison path instead")
+    ap.add_argument("--score-scope", type=int, default=0, choices=[0, 1],
+                    help="0: every layer ranks by its own (or the nearest) anchor heads; 1: Eq. 2's sum over all anchor layers")
     ap.add_argument("--eager", action="store_true", help="issue every layer eagerly instead of replaying a captured step")
     ap.add_argument("--roofline-steps", type=int, default=16)
     ap.add_argument("--oracle-layers", type=int, default=6, help="layers of sequence 0 the CPU baseline samples (0 = skip)")

@@ -64,6 +64,12 @@ enum { WNW_ROLE_ANCHOR = 0, WNW_ROLE_TIDAL = 1, WNW_ROLE_FIXED = 2 };
  * wnw_decode_layer_full; roles are ignored for storage in that mode. */
 enum { WNW_MODE_TIERED = 0, WNW_MODE_FULL = 1 };
 
+/* Which anchor heads rank a tidal layer's chunks.
+ *   PER_LAYER  the layer's own anchor heads, else those of the nearest layer that has some (ties to the lower layer)
+ *   GLOBAL     Eq. 2 as printed: one accumulator over ALL anchor (layer, q-head) pairs of the step, added in layer
+ *              order; every tidal layer takes the same selection, made once the last layer of the step has run */
+enum { WNW_SCOPE_PER_LAYER = 0, WNW_SCOPE_GLOBAL = 1 };
+
 /* How recall copies are issued (for measurement; results are identical for 0 and 1):
  *   0  side stream, overlapped with the following layers (default)
  *   1  on the caller's stream right after the layer (the paper's naive schedule, Limitations section)
@@ -85,6 +91,7 @@ typedef struct {
   int32_t device;                          /* CUDA ordinal */
   int32_t mode;                            /* WNW_MODE_* */
   int32_t recall_mode;                     /* WNW_RECALL_* */
+  int32_t score_scope;                     /* WNW_SCOPE_* */
 } wnw_config_t;
 
 typedef struct {

@@ -33,8 +33,10 @@
  *     c of the softmax weight; the ranking key is the chunk MEAN,
  *     (float)score_sum[c] / (float)len_c, compared as float, ties to the lower
  *     chunk index;
- *   - a layer without anchor heads ranks by the scores of the nearest layer
- *     that has one (ties to the lower layer);
+ *   - score scope PER_LAYER: a layer without anchor heads ranks by the scores
+ *     of the nearest layer that has one (ties to the lower layer); score scope
+ *     GLOBAL (Eq. 2 as printed): every tidal layer ranks by the sum of the
+ *     scores of ALL anchor layers of the step, added in layer order;
  *   - a selection made at step s is used by tidal attention at step s+1;
  *   - slots S = max(1, floor((double)budget * C + 1e-6)), capped at C;
  *   - stamps: a chunk selected with rank r at step s gets s*topk + (topk-1-r);
@@ -74,6 +76,7 @@ typedef struct {
 
 typedef struct {
   int L, Hq, Hkv, d, g, chunk, topk, max_batch, max_audio, max_text;
+  int scope;      /* 0: per layer with nearest-anchor routing; 1: global sum over all anchor layers */
   double budget, scale;
   uint8_t *roles; /* [L][Hkv] */
   int *src;       /* [L] score source layer, -1 if the layer has no tidal heads or no source */
@@ -194,15 +197,16 @@ void wnwo_destroy(Oracle *o) {
 }
 
 int wnwo_create(int L, int Hq, int Hkv, int d, int max_batch, int max_audio, int max_text, int chunk, int topk,
-                double budget, double scale, const uint8_t *roles, Oracle **out) {
+                double budget, double scale, const uint8_t *roles, int scope, Oracle **out) {
   if (!out || !roles || L < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv || d < 1 || max_batch < 1 || chunk < 1 || topk < 1)
     return WNWO_ERR_ARG;
-  if (!(budget > 0.0 && budget <= 1.0)) return WNWO_ERR_ARG;
+  if (!(budget > 0.0 && budget <= 1.0) || scope < 0 || scope > 1) return WNWO_ERR_ARG;
   Oracle *o = (Oracle *)calloc(1, sizeof(Oracle));
   if (!o) return WNWO_ERR_OOM;
   o->L = L; o->Hq = Hq; o->Hkv = Hkv; o->d = d; o->g = Hq / Hkv; o->chunk = chunk; o->topk = topk;
   o->max_batch = max_batch; o->max_audio = max_audio; o->max_text = max_text;
   o->budget = budget;
+  o->scope = scope;
   o->scale = scale > 0.0 ? scale : 1.0 / sqrt((double)d); /* Eq. 2: q K^T / sqrt(d) */
   o->roles = (uint8_t *)malloc((size_t)L * Hkv);
   o->src = (int *)malloc(sizeof(int) * L);
@@ -486,10 +490,15 @@ int wnwo_step_end(Oracle *o) {
       int *pc = (int *)malloc(sizeof(int) * o->topk), *ps = (int *)malloc(sizeof(int) * o->topk),
           *ev = (int *)malloc(sizeof(int) * o->topk);
       for (int c = 0; c < C; ++c) lens[c] = chunk_len(o, s, c);
+      double *glob = (double *)calloc((size_t)C, sizeof(double));
+      if (o->scope == 1) /* Eq. 2: one accumulator over all anchor (layer, q-head) pairs of the step */
+        for (int a = 0; a < o->L; ++a)
+          if (layer_has(o, a, ROLE_ANCHOR))
+            for (int c = 0; c < C; ++c) glob[c] += s->score_sum[(size_t)a * C + c];
       for (int l = 0; l < o->L; ++l) {
         s->n_sel[l] = 0;
         if (o->src[l] < 0) continue;
-        const double *sc = s->score_sum + (size_t)o->src[l] * C;
+        const double *sc = o->scope == 1 ? glob : s->score_sum + (size_t)o->src[l] * C;
         for (int c = 0; c < C; ++c) sf[c] = (float)sc[c];
         int k = o->topk < S ? o->topk : S;
         k = wnwo_topk(sf, lens, C, k, s->sel + (size_t)l * o->topk);
@@ -500,7 +509,7 @@ int wnwo_step_end(Oracle *o) {
         s->hits += hits; s->misses += n;
         for (int j = 0; j < n; ++j) s->evictions += ev[j] >= 0;
       }
-      free(lens); free(sf); free(pc); free(ps); free(ev);
+      free(lens); free(sf); free(pc); free(ps); free(ev); free(glob);
     }
     s->steps += 1;
     if (o->appended == 1) s->T_t += 1;

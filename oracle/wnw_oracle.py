@@ -41,7 +41,7 @@ def lib():
     global _lib
     if _lib is None:
         _lib = C.CDLL(build())
-        _lib.wnwo_create.argtypes = [C.c_int] * 9 + [C.c_double, C.c_double, C.POINTER(C.c_uint8), C.POINTER(C.c_void_p)]
+        _lib.wnwo_create.argtypes = [C.c_int] * 9 + [C.c_double, C.c_double, C.POINTER(C.c_uint8), C.c_int, C.POINTER(C.c_void_p)]
         _lib.wnwo_destroy.argtypes = [C.c_void_p]
         _lib.wnwo_destroy.restype = None
         _lib.wnwo_score_source.argtypes = [C.c_void_p, C.c_int]
@@ -105,7 +105,7 @@ class Oracle:
     """The stateful decode-step oracle.  Arrays in/out are numpy; bf16 values travel as uint16 bit patterns."""
 
     def __init__(self, n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
-                 chunk_tokens, topk, budget, roles, softmax_scale=0.0):
+                 chunk_tokens, topk, budget, roles, softmax_scale=0.0, score_scope=0):
         self.L, self.Hq, self.Hkv, self.d = n_layers, n_q_heads, n_kv_heads, head_dim
         self.topk_cfg = topk
         roles = np.ascontiguousarray(roles, dtype=np.uint8).reshape(-1)
@@ -114,7 +114,8 @@ class Oracle:
         # budget is a float32 field in the library's config; mirror that rounding here
         _check(lib().wnwo_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
                                  chunk_tokens, topk, float(np.float32(budget)), float(softmax_scale),
-                                 _p(roles, C.c_uint8), C.byref(h)), "create")
+                                 _p(roles, C.c_uint8), score_scope, C.byref(h)), "create")
+        self.score_scope = score_scope
         self._h = h
         self._n_active = 0
 

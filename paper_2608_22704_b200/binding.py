@@ -20,6 +20,7 @@ WNW_ERR_CAPACITY, WNW_ERR_TIMEOUT, WNW_ERR_UNSUPPORTED, WNW_ERR_DEVICE_CHECK = 6
 WNW_ROLE_ANCHOR, WNW_ROLE_TIDAL, WNW_ROLE_FIXED = 0, 1, 2
 WNW_MODE_TIERED, WNW_MODE_FULL = 0, 1
 WNW_RECALL_SIDE_STREAM, WNW_RECALL_INLINE, WNW_RECALL_SKIP = 0, 1, 2
+WNW_SCOPE_PER_LAYER, WNW_SCOPE_GLOBAL = 0, 1
 
 
 class wnw_config_t(C.Structure):
@@ -27,7 +28,7 @@ class wnw_config_t(C.Structure):
                 ("max_batch", C.c_int32), ("max_audio_tokens", C.c_int32), ("max_text_tokens", C.c_int32),
                 ("chunk_tokens", C.c_int32), ("topk", C.c_int32), ("evict_lag", C.c_int32), ("budget", C.c_float),
                 ("softmax_scale", C.c_float), ("roles", C.POINTER(C.c_uint8)), ("device", C.c_int32), ("mode", C.c_int32),
-                ("recall_mode", C.c_int32)]
+                ("recall_mode", C.c_int32), ("score_scope", C.c_int32)]
 
 
 class wnw_stats_t(C.Structure):
@@ -120,11 +121,11 @@ def _stream(stream) -> Optional[int]:
 
 def wnw_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens, chunk_tokens,
                budget, roles, topk=3, evict_lag=3, softmax_scale=0.0, device=0, mode=WNW_MODE_TIERED,
-               recall_mode=WNW_RECALL_SIDE_STREAM) -> int:
+               recall_mode=WNW_RECALL_SIDE_STREAM, score_scope=WNW_SCOPE_PER_LAYER) -> int:
     roles = np.ascontiguousarray(roles, dtype=np.uint8).reshape(-1)
     cfg = wnw_config_t(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
                        chunk_tokens, topk, evict_lag, budget, softmax_scale,
-                       roles.ctypes.data_as(C.POINTER(C.c_uint8)), device, mode, recall_mode)
+                       roles.ctypes.data_as(C.POINTER(C.c_uint8)), device, mode, recall_mode, score_scope)
     if roles.size != n_layers * n_kv_heads:
         raise WnwError(WNW_ERR_INVALID_ARG, "wnw_create (roles size)")
     h = _vp()

@@ -66,6 +66,9 @@ struct CacheView {
   const int16_t *role_idx;   // [L][Hkv] index among the heads of the same role in that layer
   const LayerInfo *layers;   // [L]
   const int32_t *upd_list;   // concatenated per-layer update lists
+  const int32_t *anchor_layers;  // layers that have anchor heads, ascending
+  int32_t n_anchor_layers;
+  int32_t scope_global;          // tidal layers rank by the sum over all anchor layers (src = -2 in their LayerInfo)
   bf16 *text, *anchor, *pool, *fixed;
   int32_t *text_len, *T_a, *C, *S;   // [B]
   long long *steps;                  // [B]

@@ -25,7 +25,8 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
   // shared-memory layout: (M,Z) of the anchor q-heads | this layer's scores | per-warp update workspaces | granule partials
   float2 *mz_s = reinterpret_cast<float2 *>(smem);
   float *sc_s = reinterpret_cast<float *>(smem + ((size_t)n_aq * 8 + 15) / 16 * 16);
-  unsigned char *ws0 = reinterpret_cast<unsigned char *>(sc_s) + ((size_t)C_b * 4 + 15) / 16 * 16;
+  float *glob_s = sc_s + (C_b + 3) / 4 * 4;   // global scope: sum of all anchor layers' scores
+  unsigned char *ws0 = reinterpret_cast<unsigned char *>(glob_s) + ((size_t)C_b * 4 + 15) / 16 * 16;
   const size_t ws_bytes = select_ws_bytes(C_b, S_b);
   const int n_par = li.upd_count < SEL_WARPS ? li.upd_count : SEL_WARPS;
   float2 *em_s = reinterpret_cast<float2 *>(ws0 + (size_t)n_par * ws_bytes);
@@ -90,19 +91,31 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
       __syncthreads();
     }
   }
+  if (cv.scope_global && li.upd_count > 0) {
+    // Eq. 2 as printed: one accumulator over all anchor layers of the step, added in layer order
+    for (int c = threadIdx.x; c < C_b; c += NT) {
+      float gsum = 0.f;
+      for (int x = 0; x < cv.n_anchor_layers; ++x) {
+        const int al = cv.anchor_layers[x];
+        gsum += (al == a.layer && scored) ? sc_s[c] : __ldcg(cv.score_sum + ((long long)b * G.L + al) * G.C_max + c);
+      }
+      glob_s[c] = gsum;
+    }
+    __syncthreads();
+  }
   if (warp < n_par) {
     const SelectWs w = select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b);
     for (int u = warp; u < li.upd_count; u += n_par) {
       int lt, src;
       upd_of(u, lt, src);
-      const bool local = scored && src == a.layer;
+      const bool local = (scored && src == a.layer) || src == -2;
       if (u >= n_par) {  // later rounds stage their own tables
         __syncwarp();
         select_stage(cv, b, lt, src, local, C_b, S_b, lane, w);
         cp_async_commit_wait_all();
         __syncwarp();
       }
-      select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, local ? sc_s : w.sc, w);
+      select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, src == -2 ? glob_s : (local ? sc_s : w.sc), w);
     }
   }
 }

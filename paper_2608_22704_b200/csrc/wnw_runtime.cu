@@ -49,7 +49,7 @@ struct wnw_cache {
   std::vector<uint8_t> roles;
   std::vector<int16_t> role_idx;
   std::vector<LayerInfo> layers;
-  std::vector<int32_t> upd_list;
+  std::vector<int32_t> upd_list, anchor_layers;
   std::vector<int> tail_of;  // layer -> layer whose tail updates its table, -1 if none
   int tid_total = 0, n_sm = 148;
   std::vector<SeqHost> seqs;
@@ -201,6 +201,7 @@ static wnw_status_t validate_config(const wnw_config_t *cfg) {
   if (!(cfg->budget > 0.f && cfg->budget <= 1.f)) return WNW_ERR_INVALID_ARG;
   if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return WNW_ERR_INVALID_ARG;
   if (cfg->mode != WNW_MODE_TIERED && cfg->mode != WNW_MODE_FULL) return WNW_ERR_INVALID_ARG;
+  if (cfg->score_scope != WNW_SCOPE_PER_LAYER && cfg->score_scope != WNW_SCOPE_GLOBAL) return WNW_ERR_INVALID_ARG;
   if (cfg->recall_mode < WNW_RECALL_SIDE_STREAM || cfg->recall_mode > WNW_RECALL_SKIP) return WNW_ERR_INVALID_ARG;
   if (cfg->device < 0) return WNW_ERR_INVALID_ARG;
   bool any_anchor = false, any_tidal = false;
@@ -276,8 +277,9 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     int best = -1;
     for (int a = 0; a < L; ++a)
       if (c->layers[a].n_anchor > 0 && (best < 0 || std::abs(a - l) < std::abs(best - l))) best = a;
-    c->layers[l].src = best;  // nearest anchor layer, ties to the lower one
-    const int x = std::max(l, best);  // the first point at which both layer l's attention and its source scores are done
+    const bool global = cfg->score_scope == WNW_SCOPE_GLOBAL;
+    c->layers[l].src = (global && best >= 0) ? -2 : best;  // nearest anchor layer, ties to the lower one; -2: the global accumulator
+    const int x = global ? L - 1 : std::max(l, best);  // first point at which layer l's attention and its scores are done
     c->tail_of[l] = x;
     upd[x].push_back(l);
   }
@@ -303,6 +305,12 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     CKC(dev_upload(c, &q, c->role_idx)); cv.role_idx = q;
     CKC(dev_upload(c, &li, c->layers)); cv.layers = li;
     CKC(dev_upload(c, &ul, c->upd_list)); cv.upd_list = ul;
+    for (int l = 0; l < L; ++l)
+      if (c->layers[l].n_anchor > 0) c->anchor_layers.push_back(l);
+    int32_t *al;
+    CKC(dev_upload(c, &al, c->anchor_layers)); cv.anchor_layers = al;
+    cv.n_anchor_layers = (int32_t)c->anchor_layers.size();
+    cv.scope_global = !full && cfg->score_scope == WNW_SCOPE_GLOBAL;
   }
   CKC(dev_alloc(c, &cv.text, B * (size_t)G.text_seq_stride));
   CKC(dev_alloc(c, &cv.anchor, B * (size_t)G.anchor_seq_stride));
@@ -349,7 +357,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   for (int l = 0; l < L && !full; ++l) {
     const LayerInfo &li = c->layers[l];
     const size_t n_aq_l = (size_t)std::max(li.n_anchor * G.g, 1);
-    const size_t fixed_part = (n_aq_l * 8 + 15) / 16 * 16 + ((size_t)G.C_max * 4 + 15) / 16 * 16 +
+    const size_t fixed_part = (n_aq_l * 8 + 15) / 16 * 16 + 2 * (((size_t)G.C_max * 4 + 15) / 16 * 16) + 16 +
                               (size_t)std::min(li.upd_count, 8) * select_ws_bytes(G.C_max, G.S_max);
     const size_t per_chunk = li.n_anchor > 0 ? n_aq_l * G.gpc * 8 : 0;
     const size_t cap = SELECT_SMEM_CAP - 16;
@@ -809,6 +817,10 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
         if (src >= 0 && src != layer && src % wnw_cache::N_SIDE != si)
           CK(cudaStreamWaitEvent(ss, capturing ? c->ev_side_done_cap[src] : c->ev_side_done[src], 0));
       }
+      if (c->cv.scope_global && li.upd_count > 0)  // the global accumulator needs every anchor layer's scores of this step
+        for (int al : c->anchor_layers)
+          if (al != layer && al % wnw_cache::N_SIDE != si)
+            CK(cudaStreamWaitEvent(ss, capturing ? c->ev_side_done_cap[al] : c->ev_side_done[al], 0));
     }
     CK(launch_select(c->cv, sa, c->sel_smem[layer], ss));
     if (li.upd_count > 0 && !c->cap_external_recall)

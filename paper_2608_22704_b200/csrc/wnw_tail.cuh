@@ -89,7 +89,7 @@ __device__ __forceinline__ void select_and_update(const CacheView &cv, int b, in
   const Geometry &G = cv.geo;
   const long long bl = (long long)b * G.L + lt;
   int k = G.topk < S_b ? G.topk : S_b;
-  if (src < 0 || C_b <= 0) k = 0;
+  if (src == -1 || C_b <= 0) k = 0;   // -1: nothing to rank by; -2: the global accumulator
   int *slot_chunk = cv.slot_chunk + bl * G.S_max;
   int *chunk_slot = cv.chunk_slot + bl * G.C_max;
   long long *stamp = cv.stamp + bl * G.S_max;

@@ -376,3 +376,30 @@ def test_oracle_accepts_the_papers_chunk_size():
     K, V, _, ab, ae = kept[(0, 0)]
     ref, _ = dense_attention(bf16_bits_to_f64(q[2]), K[:, 1], V[:, 1], 1 / math.sqrt(64))
     assert np.abs(out[0, 2] - ref).max() < 1e-12
+
+
+# ---------------------------------------------------------------- global aggregation (Eq. 2 as printed)
+def test_global_scope_sums_all_anchor_layers_and_shares_one_selection():
+    """Score scope GLOBAL: every tidal layer selects from the sum of all anchor layers' chunk scores of the step."""
+    A, T, F = ROLE_ANCHOR, ROLE_TIDAL, ROLE_FIXED
+    w = tiny_custom(n_layers=4, n_q_heads=4, n_kv_heads=2, n_text=4, audio_lens=(160,), chunk=16, budget=0.4,
+                    roles=[[A, T], [T, F], [A, T], [T, T]], n_steps=3)
+    syn = Synth(w, seed=7)
+    o = make_oracle(w, score_scope=1); place_all(o, syn)
+    dec = {l: syn.decode(0, l) for l in range(4)}
+    for t in range(3):
+        o.step_begin([0])
+        for l in range(4):
+            o.decode_layer(l, bf16_bits(dec[l]["q"][t])[None])
+        o.step_end()
+        glob = o.chunk_scores(0, 0) + o.chunk_scores(0, 2)
+        want = _brute_rank(glob.astype(np.float32), np.full(10, 16))[:3]
+        for l in range(4):
+            assert o.selected(0, l).tolist() == want
+    # per-layer scope on the same inputs routes layer 1 to layer 0 and layer 3 to layer 2 instead
+    o2 = make_oracle(w, score_scope=0); place_all(o2, syn)
+    o2.step_begin([0])
+    for l in range(4):
+        o2.decode_layer(l, bf16_bits(dec[l]["q"][0])[None])
+    o2.step_end()
+    assert o2.selected(0, 3).tolist() == _brute_rank(o2.chunk_scores(0, 2).astype(np.float32), np.full(10, 16))[:3]
