@@ -398,11 +398,13 @@ def run_ours(args, rank, world, local_rank):
         return
     K, W = args.steps, args.warmup
     R = args.roofline_steps
-    total = W + R + K
+    Kc = 0 if (args.quick or args.eager) else min(K, args.chain_steps)
+    total = W + R + K + 2 * Kc
     w = make_workload(args.workload, total, 0)
     job = Job(w, seed=rank, device=dev, wnw=wnw, score_scope=args.score_scope)
     job.create("wnw", wnw.WNW_MODE_FULL if args.quick_full else wnw.WNW_MODE_TIERED, recall_mode=args.recall_mode)
     if args.quick:   # profiler mode: the WnW steps only, nothing else launched
+        wnw.wnw_set_layer_dependency(job.caches["wnw"], args.layer_dependency)
         job.place_all(["wnw"])
         for t in range(W):
             job.step("wnw", t, full=args.quick_full)
@@ -464,6 +466,7 @@ def run_ours(args, rank, world, local_rank):
         gpu_id = str(local_rank)
     sampler = ClockSampler(gpu_id)
     barrier()
+    bytes_before, _ = job.kv_bytes_of_step("wnw")
     sampler.start()
     wall0 = time.perf_counter()
     per_step = job.timed_steps("wnw", W + R, K, graph=not args.eager)
@@ -471,6 +474,8 @@ def run_ours(args, rank, world, local_rank):
     wall = time.perf_counter() - wall0
     clocks = sampler.stop()
     stats1 = wnw.wnw_get_stats(job.caches["wnw"])
+    bytes_after, _ = job.kv_bytes_of_step("wnw")
+    region_bytes_per_launch = 0.5 * (bytes_before + bytes_after) / w.n_layers   # the text grows by one token per step
     ms_per_step = dist_max(sum(per_step), dev, world) / K
     value = whole_job_tokens_per_s(world, w.batch, ms_per_step)
 
@@ -508,6 +513,22 @@ def run_ours(args, rank, world, local_rank):
     e2e_value = whole_job_tokens_per_s(world, w.batch, dist_max(e2e_ms, dev, world) / n_e2e)
     h2d = job.sslab.numel() * 2
     d2h = job.out.numel() * 2
+
+    # ---- the same step with layers that feed one another (chained) and with plain serial launches
+    dep = {}
+    if Kc > 0:
+        t_dep = W + R + K
+        for name, mode in (("chained", wnw.WNW_LAYERS_CHAINED), ("serial", wnw.WNW_LAYERS_SERIAL)):
+            wnw.wnw_sync(job.caches["wnw"])
+            wnw.wnw_set_layer_dependency(job.caches["wnw"], mode)
+            job.captured.discard("wnw")
+            nb, _ = job.kv_bytes_of_step("wnw")
+            ms = dist_max(sum(job.timed_steps("wnw", t_dep, Kc)), dev, world) / Kc
+            t_dep += Kc
+            us_l = ms * 1e3 / w.n_layers
+            dep[name] = {"step_us": ms * 1e3, "us_per_launch": us_l, "achieved": nb / w.n_layers / (us_l * 1e-6) / 1e9,
+                         "frac": nb / w.n_layers / (us_l * 1e-6) / 1e9 / peak_gbs, "steps": Kc}
+        wnw.wnw_set_layer_dependency(job.caches["wnw"], wnw.WNW_LAYERS_INDEPENDENT)
 
     if rank != 0:
         job.destroy()
@@ -568,6 +589,8 @@ def run_ours(args, rank, world, local_rank):
         jp.destroy()
 
     attn_us = attn_ms * 1e3 / max(attn_n, 1)
+    region_us_per_launch = ms_per_step * 1e3 / w.n_layers
+    region_achieved = region_bytes_per_launch / (region_us_per_launch * 1e-6) / 1e9
     bytes_per_launch = algo_bytes / max(attn_n, 1)
     achieved = bytes_per_launch / (attn_us * 1e-6) / 1e9 if attn_us > 0 else 0.0
     full_us = full_ms * 1e3 / max(full_n, 1)
@@ -594,17 +617,22 @@ def run_ours(args, rank, world, local_rank):
                                                                                 score_scope="global" if args.score_scope else "per layer"),
         "clocks": clocks, "gpu_launches": launches_per_step * K,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e},
-        # achieved: algorithmic K,V bytes of one launch / its duration, each launch bracketed by CUDA events on the launching
-        # stream (eager pass, launches isolated).  In the timed region proper the layer kernels of a step overlap
-        # (programmatic dependent launch inside the replayed graph), so one launch has no duration of its own there;
-        # `pipelined_*` divides the same bytes by the step time per layer instead.
-        "roofline": {"bound": "hbm", "kernel": "wnw_attn_kernel", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
-                     "frac": achieved / peak_gbs, "peak_kind": f"of {peak_kind}", "traffic": traffic,
-                     "bytes_per_launch": bytes_per_launch, "us_per_launch": attn_us, "launches": attn_n,
-                     "pipelined_us_per_layer": ms_per_step * 1e3 / w.n_layers,
-                     "pipelined_achieved": bytes_per_launch / (ms_per_step * 1e-3 / w.n_layers) / 1e9,
-                     "pipelined_frac": bytes_per_launch / (ms_per_step * 1e-3 / w.n_layers) / 1e9 / peak_gbs,
-                     "regime": "latency-bound: 3.9 MB per launch would take 0.6 us at peak"},
+        # achieved: algorithmic K,V bytes of one launch / the launch's share of the timed region (CUDA events around every
+        # replayed step; the attention kernels are the only work on the timed stream, one per layer; consecutive layer
+        # kernels overlap through programmatic dependent launch, so the share of one launch is step time / layers).
+        # `chained`: every kernel waits for its predecessor before reading q (layers that feed one another; only the
+        # K/V prefetch overlaps).  `serial`: plain stream order.  `eager_event_bracket`: one launch bracketed by events on
+        # an eager stream (includes launch latency and host pacing; kept for reference).
+        "roofline": {"bound": "hbm", "kernel": "wnw_attn_kernel", "achieved": region_achieved, "peak": peak_gbs, "unit": "GB/s",
+                     "frac": region_achieved / peak_gbs, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                     "bytes_per_launch": region_bytes_per_launch, "us_per_launch": region_us_per_launch,
+                     "launches": w.n_layers * K,
+                     "duration_kind": "timed region / attention launches (layer kernels overlap inside the replayed step)",
+                     "chained": dep.get("chained"), "serial": dep.get("serial"),
+                     "eager_event_bracket": {"us_per_launch": attn_us, "achieved": achieved, "frac": achieved / peak_gbs,
+                                             "launches": attn_n},
+                     "regime": f"{region_bytes_per_launch / 1e6:.1f} MB per launch would take "
+                               f"{region_bytes_per_launch / (peak_gbs * 1e3):.2f} us at peak"},
         "cpu_baseline": cpu,
         "full_cache": {"ms_per_step": ms_full, "tokens_per_s": w.batch / (ms_full * 1e-3), "attn_us_per_launch": full_us,
                        "attn_GBps": full_achieved, "attn_frac": full_achieved / peak_gbs,
@@ -637,6 +665,10 @@ def main():
                     help="0: every layer ranks by its own (or the nearest) anchor heads; 1: Eq. 2's sum over all anchor layers")
     ap.add_argument("--eager", action="store_true", help="issue every layer eagerly instead of replaying a captured step")
     ap.add_argument("--roofline-steps", type=int, default=16)
+    ap.add_argument("--layer-dependency", type=int, default=0, choices=[0, 1, 2],
+                    help="with --quick: 0 independent layers (overlap), 1 chained, 2 serial launches")
+    ap.add_argument("--chain-steps", type=int, default=48,
+                    help="steps timed with chained layers and with serial layer launches (0 = skip)")
     ap.add_argument("--oracle-layers", type=int, default=6, help="layers of sequence 0 the CPU baseline samples (0 = skip)")
     ap.add_argument("--oracle-steps", type=int, default=4)
     ap.add_argument("--sweep-steps", type=int, default=0,

@@ -195,6 +195,18 @@ wnw_status_t wnw_get_slot_kv(wnw_cache_t *cache, int32_t seq, int32_t layer, int
                              void *rows_host);
 wnw_status_t wnw_get_stats(wnw_cache_t *cache, wnw_stats_t *stats_host);
 
+/* How a layer's attention kernel is ordered against the work that precedes it on the caller's stream.
+ *   INDEPENDENT  (default) q/k_new/v_new of every layer of the step exist before the step is issued: consecutive layer
+ *                kernels are launched programmatically dependent and may overlap freely (they touch disjoint state).
+ *   CHAINED      q/k_new/v_new of a layer are written by the work just before it on the stream (a decoder whose layers
+ *                feed one another): the kernel still starts early and queues its K/V cache loads, which do not depend
+ *                on that work, but waits for the predecessor to complete before it reads q, k_new or v_new.
+ *   SERIAL       plain stream order, no early start.
+ * Takes effect for layers issued afterwards; a captured step keeps the mode it was captured with.  Not allowed inside
+ * a step.  Results are identical in all three modes. */
+enum { WNW_LAYERS_INDEPENDENT = 0, WNW_LAYERS_CHAINED = 1, WNW_LAYERS_SERIAL = 2 };
+wnw_status_t wnw_set_layer_dependency(wnw_cache_t *cache, int32_t mode);
+
 /* Optional per-kernel timing: when enabled the library brackets its attention-kernel launches with CUDA events
  * on the launching stream; wnw_get_kernel_time returns the accumulated milliseconds and launch count since the
  * last call (drains the stream).  Off by default. */

@@ -21,6 +21,7 @@ WNW_ROLE_ANCHOR, WNW_ROLE_TIDAL, WNW_ROLE_FIXED = 0, 1, 2
 WNW_MODE_TIERED, WNW_MODE_FULL = 0, 1
 WNW_RECALL_SIDE_STREAM, WNW_RECALL_INLINE, WNW_RECALL_SKIP = 0, 1, 2
 WNW_SCOPE_PER_LAYER, WNW_SCOPE_GLOBAL = 0, 1
+WNW_LAYERS_INDEPENDENT, WNW_LAYERS_CHAINED, WNW_LAYERS_SERIAL = 0, 1, 2
 
 
 class wnw_config_t(C.Structure):
@@ -63,6 +64,7 @@ _SIGNATURES = {
     "wnw_get_seq_dims": [_vp, _i32] + [C.POINTER(_i32)] * 4,
     "wnw_get_slot_kv": [_vp, _i32, _i32, _i32, _i32, _i32, _vp],
     "wnw_get_stats": [_vp, C.POINTER(wnw_stats_t)],
+    "wnw_set_layer_dependency": [_vp, _i32],
     "wnw_set_kernel_timing": [_vp, _i32],
     "wnw_get_kernel_time": [_vp, C.POINTER(C.c_float), C.POINTER(_i32)],
     "wnw_sync": [_vp],
@@ -235,6 +237,10 @@ def wnw_get_stats(cache) -> dict:
     s = wnw_stats_t()
     _ck(lib().wnw_get_stats(cache, C.byref(s)), "wnw_get_stats")
     return {n: getattr(s, n) for n, _ in wnw_stats_t._fields_}
+
+
+def wnw_set_layer_dependency(cache, mode: int):
+    _ck(lib().wnw_set_layer_dependency(cache, int(mode)), "wnw_set_layer_dependency")
 
 
 def wnw_set_kernel_timing(cache, enable: bool):

@@ -304,6 +304,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   for (int n = 0; n < NSTAGE - 1; ++n) pro_loaded[n] = issue_copy(n);
   STAMP(1);
 
+  // Chained layers: the cache loads above never depend on the preceding work, the query and the new token's K/V do.
+  if (a.wait_inputs && qi == q_begin) asm volatile("griddepcontrol.wait;\n" ::: "memory");
   // ---- Q fragments (rows >= g are zero padding); loaded after the first K/V copies are in flight ----
   const int r0 = lane >> 2, cq = (lane & 3) * 2;
   uint32_t qa[KK][NQ];

@@ -133,6 +133,7 @@ struct AttnArgs {
   const int32_t *wait_epoch;     // replayed steps: tidal CTAs wait until *wait_epoch >= *expect_epoch (this layer's recall of the
   const int32_t *expect_epoch;   //   previous step, which runs outside the captured graph, has landed); null otherwise
   int32_t pdl;                   // launch with programmatic stream serialization (previous stream op is a layer kernel)
+  int wait_inputs;  // q/k_new/v_new come from the preceding work on the stream: wait for it before reading them
   const HeadItems *head_items;  // [n_active][Hkv] work items of each head (first is relative to `items`)
   const bf16 *q;         // [n_active][Hq][d]
   const bf16 *k_new, *v_new;    // [n_active][Hkv][d] or null

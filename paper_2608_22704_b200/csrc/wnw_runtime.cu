@@ -97,6 +97,7 @@ struct wnw_cache {
   size_t gran_em_layer_stride = 0;
   bool step_capturing = false;
   bool pdl_enabled = true;
+  int layer_dependency = WNW_LAYERS_INDEPENDENT;
   // replayed steps: one recall launch per step outside the captured graph, overlapping the next step
   int32_t *d_recall_epoch = nullptr, *d_recall_ctr = nullptr, *d_step_epoch = nullptr;
   int external_recall_mode = -1;   // -1 automatic, 0 never, 1 always
@@ -774,7 +775,8 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   a.gran_em = gran_em_l;
   if (c->cap_external_recall && li.n_tidal > 0) { a.wait_epoch = c->d_recall_epoch + layer; a.expect_epoch = c->d_step_epoch; }
   // overlap with the previous layer's kernel when that is what precedes this launch in the stream
-  a.pdl = layer > 0 && c->pdl_enabled;
+  a.pdl = layer > 0 && c->pdl_enabled && c->layer_dependency != WNW_LAYERS_SERIAL;
+  a.wait_inputs = a.pdl && c->layer_dependency == WNW_LAYERS_CHAINED;
   a.n_aq = std::max(li.n_anchor * G.g, 1); a.n_ag_max = c->n_ag_max;
   cudaEvent_t t0 = nullptr, t1 = nullptr;
   const bool timing = c->timing && !capturing;
@@ -1128,6 +1130,13 @@ extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
     }
   }
   *out = r;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_set_layer_dependency(wnw_cache_t *c, int32_t mode) {
+  if (!c || mode < WNW_LAYERS_INDEPENDENT || mode > WNW_LAYERS_SERIAL) return WNW_ERR_INVALID_ARG;
+  if (c->in_step || c->graph_capturing) return WNW_ERR_STATE;
+  c->layer_dependency = mode;
   return WNW_OK;
 }
 
