@@ -57,6 +57,11 @@ def make_workload(name: str, n_steps: int, seed: int):
         n_l = 4 if name == "prof" else 12
         w = config4(seed=0, budget=0.2, chunk=64, batch=16, n_steps=n_steps)
         w.n_layers = n_l; w.roles = w.roles[:n_l]; w.jump_every = 0; w.sweep_steps = 128; w.name = f"{name}_{n_l}layers_b16_7500"
+    elif name.startswith("b") and "x" in name:   # b<batch>x<audio tokens>: config-1 heads, 12 layers (regime studies)
+        nb, na = name[1:].split("x")
+        w = config4(seed=0, budget=0.2, chunk=64, batch=int(nb), n_steps=n_steps)
+        w.audio_lens = [int(na)] * int(nb)
+        w.n_layers = 12; w.roles = w.roles[:12]; w.jump_every = 0; w.sweep_steps = 256; w.name = f"cfg1heads_12layers_{name}"
     else:
         raise SystemExit(f"unknown workload {name}")
     if SWEEP_STEPS_OVERRIDE:
@@ -655,7 +660,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "cfg2", "cfg3", "cfg4", "prof", "hbm"])
+    ap.add_argument("--workload", default="cfg1",
+                    help="cfg1 | cfg2 | cfg3 | cfg4 (recall sweep) | prof | hbm | b<batch>x<audio tokens> (config-1 heads, 12 layers)")
     ap.add_argument("--no-hbm-case", action="store_true", help="skip the extra many-sequence measurement")
     ap.add_argument("--quick", action="store_true", help="only the WnW steps (for profiler captures); prints a short line")
     ap.add_argument("--no-flush", action="store_true", help="with --quick: do not flush L2 between steps")

@@ -33,6 +33,7 @@ constexpr int NSTAGE = 3;  // granules in flight per warp
 
 int attn_warps(bool throughput) { return throughput ? NW_THR : NW_LAT; }
 
+
 // Phase stamps for latency studies: compiled in only with -DWNW_PHASE_STAMPS (never in the product build).
 #ifdef WNW_PHASE_STAMPS
 __device__ long long g_stamps[8192 * 16];
@@ -200,68 +201,70 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   // host assigned to it (balanced by size), so no SM idles through a partial last wave.
   int q_begin = blockIdx.x, q_end = blockIdx.x + 1;
   if (a.cta_ranges) { q_begin = a.cta_ranges[blockIdx.x]; q_end = a.cta_ranges[blockIdx.x + 1]; }
-  for (int qi = q_begin; qi < q_end; ++qi) {
-  const int item_idx = a.cta_ranges ? a.order[qi] : qi;
-  if (qi > q_begin) __syncthreads();  // the previous item's merge is done with shared memory
-  // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
-  const WorkItem it = a.n_items <= INLINE_ITEMS_MAX ? inl.it[item_idx] : a.items[item_idx];
-  const int b = it.b, role = it.role, ridx = it.ridx, T_a = it.T_a;
-  const int T_t = cv.text_len[b] + a.has_new;
-#ifdef WNW_PHASE_STAMPS
-  if (it.g0 >= 0) STAMP(10);
-  kslot = (int)((cv.steps[b] & 3) * 64 + a.layer);
-  KSTAMP_MIN(kslot, 0);
-#endif
-  if (a.wait_epoch && role == ROLE_TIDAL) {
-    // Replayed steps: the recall that refreshed this layer's slots ran outside the captured graph, possibly still
-    // overlapping this step.  Bounded acquire-wait on the layer's epoch word before any slot is read.
-    if (lane == 0) {
-      const int expect = *a.expect_epoch;
-      int seen;
-      const long long t0 = clock64();
-      for (;;) {
-        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];\n" : "=r"(seen) : "l"(a.wait_epoch) : "memory");
-        if (seen >= expect) break;
-        if (clock64() - t0 > 2000000000ll) { timed_out = true; break; }
+
+  // What a warp needs to address the granules of one work item.
+  struct Ctx {
+    WorkItem it;
+    int item_idx, T_t, v_delta_audio, first, n_my;
+    const CUtensorMap *map_audio;
+  };
+  auto load_ctx = [&](Ctx &c, int qi) {
+    c.item_idx = a.cta_ranges ? a.order[qi] : qi;
+    // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
+    c.it = a.n_items <= INLINE_ITEMS_MAX ? inl.it[c.item_idx] : a.items[c.item_idx];
+    c.T_t = cv.text_len[c.it.b] + a.has_new;
+    if (c.it.role == ROLE_ANCHOR) { c.v_delta_audio = G.T_a_pad; c.map_audio = &maps.anchor; }       // rows between a
+    else if (c.it.role == ROLE_TIDAL) { c.v_delta_audio = G.ncp; c.map_audio = &maps.pool; }          // granule's K and
+    else { c.v_delta_audio = G.S_max * G.ncp; c.map_audio = &maps.fixed; }                            // V rows
+    c.first = c.it.g0 + warp;
+    c.n_my = c.first < c.it.g1 ? (c.it.g1 - c.first + NW - 1) / NW : 0;
+    if (a.wait_epoch && c.it.role == ROLE_TIDAL) {
+      // Replayed steps: the recall that refreshed this layer's slots ran outside the captured graph, possibly still
+      // overlapping this step.  Bounded acquire-wait on the layer's epoch word before any slot is read.
+      if (lane == 0) {
+        const int expect = *a.expect_epoch;
+        int seen;
+        const long long t0 = clock64();
+        for (;;) {
+          asm volatile("ld.acquire.gpu.global.s32 %0, [%1];\n" : "=r"(seen) : "l"(a.wait_epoch) : "memory");
+          if (seen >= expect) break;
+          if (clock64() - t0 > 2000000000ll) { timed_out = true; break; }
+        }
+        asm volatile("fence.proxy.async.global;\n" ::: "memory");  // the slots are read by TMA (async proxy)
       }
-      asm volatile("fence.proxy.async.global;\n" ::: "memory");  // the slots are read by TMA (async proxy)
+      timed_out = __shfl_sync(0xffffffffu, (int)timed_out, 0) != 0;
     }
-    timed_out = __shfl_sync(0xffffffffu, (int)timed_out, 0) != 0;
-  }
-  int v_delta_audio;  // rows between a granule's K and V rows
-  const CUtensorMap *map_audio;
-  if (role == ROLE_ANCHOR) { v_delta_audio = G.T_a_pad; map_audio = &maps.anchor; }
-  else if (role == ROLE_TIDAL) { v_delta_audio = G.ncp; map_audio = &maps.pool; }
-  else { v_delta_audio = G.S_max * G.ncp; map_audio = &maps.fixed; }
+  };
   const int v_delta_text = G.T_cap_pad;
 
-  const int first = it.g0 + warp;
-  const int n_my = first < it.g1 ? (it.g1 - first + NW - 1) / NW : 0;
-
-  GranDesc blk;  // descriptor this lane decoded for the current block of 32 granules
+  // ---- producer side of the per-warp pipeline: (prod, p_n) is the next granule to fetch, seq_p its stage sequence ----
+  Ctx prod;
+  int p_n = 0;
+  uint32_t seq_p = 0, seq_c = 0;
+  GranDesc blk;  // descriptor this lane decoded for the producer's current block of 32 granules
   blk.row = 0; blk.meta = 0; blk.cid = -1; blk.off = 0; blk.score_idx = -1;
 
   // Visible rows of a granule once its metadata has arrived.
-  auto visible = [&](int meta, int cid, int off, int j) -> int {
+  auto visible = [&](const Ctx &c, int meta, int cid, int off, int j) -> int {
     if (meta >= 0) return meta;
     int len;
-    if (meta == -1) len = T_t - j * GR;
+    if (meta == -1) len = c.T_t - j * GR;
     else {
       if (cid < 0) return 0;
-      len = T_a - cid * G.nc;
+      len = c.it.T_a - cid * G.nc;
       if (len > G.nc) len = G.nc;
       len -= off;
     }
     return len <= 0 ? 0 : (len < GR ? len : GR);
   };
-  // Queues the TMA copies of granule n (K and V, all 16 rows).  Granules with a static row are fetched before anyone
-  // knows how many of their rows are visible (the stores hold finite data everywhere; masked columns get probability
-  // 0); only text granules beyond the host's lower bound wait for the text length.  Returns whether a copy was queued.
-  auto issue_copy = [&](int n) -> bool {
-    if (n >= n_my) return false;
+  // Queues the TMA copies of granule n of item c (K and V, all 16 rows) into stage seq % NSTAGE.  Granules with a static
+  // row are fetched before anyone knows how many of their rows are visible (the stores hold finite data everywhere;
+  // masked columns get probability 0); only text granules beyond the host's lower bound wait for the text length.
+  // Returns whether a copy was queued.
+  auto issue_copy = [&](const Ctx &c, int n, uint32_t seq) -> bool {
     if ((n & 31) == 0) {
       const int nn = n + lane;
-      if (nn < n_my) blk = decode_granule(cv, a, li, it, first + nn * NW);
+      if (nn < c.n_my) blk = decode_granule(cv, a, li, c.it, c.first + nn * NW);
       else { blk.meta = 0; blk.cid = -1; blk.score_idx = -1; }
 #ifdef WNW_PHASE_STAMPS
       if (n == 0 && blk.row >= 0) STAMP(12);
@@ -270,15 +273,15 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     const int src_lane = n & 31;
     const int meta = __shfl_sync(0xffffffffu, blk.meta, src_lane);
     const int row = __shfl_sync(0xffffffffu, blk.row, src_lane);
-    const int j = first + n * NW;
+    const int j = c.first + n * NW;
     const bool is_text = j < G.n_tg;
     bool load = meta != 0;
-    if (meta == -1) load = visible(-1, 0, 0, j) > 0;  // waits for the text length
+    if (meta == -1) load = visible(c, -1, 0, 0, j) > 0;  // waits for the text length
     if (load && lane == 0) {
-      const int stage = n % NSTAGE;
+      const int stage = (int)(seq % NSTAGE);
       const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB, bar = smem_u32(&bars[warp][stage]);
-      const CUtensorMap *map = is_text ? &maps.text : map_audio;
-      const int vrow = row + (is_text ? v_delta_text : v_delta_audio);
+      const CUtensorMap *map = is_text ? &maps.text : c.map_audio;
+      const int vrow = row + (is_text ? v_delta_text : c.v_delta_audio);
       fence_proxy_async();  // the stage was last read through the generic proxy (ldmatrix)
       mbar_expect_tx(bar, 2 * TILEB);
 #pragma unroll
@@ -289,19 +292,42 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     }
     return load;
   };
-  // Publishes (visible rows, loaded, score index) of granule n for the compute step; may wait for the metadata loads.
-  auto issue_meta = [&](int n, bool loaded) {
-    if (n < n_my) {
-      const int src_lane = n & 31;
-      const int valid = __shfl_sync(0xffffffffu, visible(blk.meta, blk.cid, blk.off, first + (n - src_lane + lane) * NW), src_lane);
-      const int sidx = __shfl_sync(0xffffffffu, blk.score_idx, src_lane);
-      if (lane == 0) ring[warp][n % NSTAGE] = make_int2(valid | (loaded ? 256 : 0), sidx);
-    }
+  // Publishes (visible rows, loaded, score index) of granule n of item c for the compute step; may wait for the
+  // metadata loads.
+  auto issue_meta = [&](const Ctx &c, int n, uint32_t seq, bool loaded) {
+    const int src_lane = n & 31;
+    const int valid = __shfl_sync(0xffffffffu, visible(c, blk.meta, blk.cid, blk.off, c.first + (n - src_lane + lane) * NW), src_lane);
+    const int sidx = __shfl_sync(0xffffffffu, blk.score_idx, src_lane);
+    if (lane == 0) ring[warp][seq % NSTAGE] = make_int2(valid | (loaded ? 256 : 0), sidx);
+  };
+  // Fetches the producer's next granule of the current work item, if this warp has one left.
+  auto produce = [&]() {
+    if (p_n >= prod.n_my) return;
+    const bool ld = issue_copy(prod, p_n, seq_p);
+    issue_meta(prod, p_n, seq_p, ld);
+    ++p_n; ++seq_p;
   };
 
+  for (int qi = q_begin; qi < q_end; ++qi) {
+  // the merge below reuses the stages as scratch: the previous item's merge must be done
+  if (qi > q_begin) __syncthreads();
+  p_n = 0;
+  load_ctx(prod, qi);
+  const WorkItem &it = prod.it;
+  const int item_idx = prod.item_idx;
+  const int b = it.b, ridx = it.ridx, T_t = prod.T_t;
+  const int first = prod.first, n_my = prod.n_my;
+#ifdef WNW_PHASE_STAMPS
+  if (it.g0 >= 0) STAMP(10);
+  kslot = (int)((cv.steps[b] & 3) * 64 + a.layer);
+  KSTAMP_MIN(kslot, 0);
+#endif
+  // the first copies go out before anything else is read; their metadata follows the Q loads
   bool pro_loaded[NSTAGE - 1];
+  int n_pro = 0;
 #pragma unroll
-  for (int n = 0; n < NSTAGE - 1; ++n) pro_loaded[n] = issue_copy(n);
+  for (int n = 0; n < NSTAGE - 1; ++n)
+    if (n < n_my) { pro_loaded[n] = issue_copy(prod, n, seq_p + n); n_pro = n + 1; }
   STAMP(1);
 
   // Chained layers: the cache loads above never depend on the preceding work, the query and the new token's K/V do.
@@ -322,16 +348,18 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     }
   }
 #pragma unroll
-  for (int n = 0; n < NSTAGE - 1; ++n) issue_meta(n, pro_loaded[n]);
+  for (int n = 0; n < NSTAGE - 1; ++n)
+    if (n < n_pro) issue_meta(prod, n, seq_p + n, pro_loaded[n]);
+  p_n = n_pro; seq_p += n_pro;
 
   float o[D / 8][4];
 #pragma unroll
   for (int t = 0; t < D / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
-  for (int n = 0; n < n_my; ++n) {
+  for (int n = 0; n < n_my; ++n, ++seq_c) {
     __syncwarp();
-    const int stage = n % NSTAGE;
+    const int stage = (int)(seq_c % NSTAGE);
     const int2 rg = ring[warp][stage];
     const int valid = rg.x & 255;
     if (rg.x & 256) {  // a copy was queued for this stage: wait for its bytes (bounded)
@@ -339,6 +367,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       phase_bits ^= 1u << stage;
     }
     if (valid > 0 && !timed_out) {
+
       const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB;
       // the row of the token being generated: take it from k_new/v_new and store it into the text region
       const int j = first + n * NW;
@@ -435,17 +464,14 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       }
     }
     __syncwarp();
-    {
-      const bool ld = issue_copy(n + NSTAGE - 1);
-      issue_meta(n + NSTAGE - 1, ld);
-    }
+    produce();
   }
   if (timed_out && lane == 0) atomicOr(cv.status, STATUS_TIMEOUT);
   __syncthreads();
   STAMP(2);
 
   // ---- merge the warps' partial states through shared memory ----
-  float2 *red_ml = reinterpret_cast<float2 *>(smem);                           // [NW][16]
+  float2 *red_ml = reinterpret_cast<float2 *>(smem);                           // [NW][16]  (the stages are idle by now)
   float *red_o = reinterpret_cast<float *>(smem + NW * 16 * sizeof(float2));   // [NW][g][D]
   if ((lane & 3) == 0) {
     red_ml[warp * 16 + r0] = make_float2(m0, l0);
@@ -556,6 +582,14 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   STAMP(5);
   KSTAMP_MAX(kslot, 2);
   }  // work items of this CTA
+  // after a timeout copies may still be in flight towards this CTA's shared memory: bounded wait before it is released
+  for (; seq_c < seq_p; ++seq_c) {
+    const int stage = (int)(seq_c % NSTAGE);
+    if (ring[warp][stage].x & 256) {
+      mbar_wait(smem_u32(&bars[warp][stage]), (phase_bits >> stage) & 1u);
+      phase_bits ^= 1u << stage;
+    }
+  }
   pdl_finish();
 }
 

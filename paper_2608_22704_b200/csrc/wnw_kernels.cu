@@ -134,7 +134,9 @@ cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_
 // layers first.  With `sig` set (replayed steps, where this kernel runs outside the captured graph and overlaps the
 // next step) the last CTA of every layer publishes the layer's recall epoch, which the next step's tidal CTAs acquire.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) wnw_recall_kernel(const __grid_constant__ CacheView cv, int n_active,
+// At most 40 registers per thread, so that a recall CTA fits beside a resident attention CTA instead of waiting for a
+// free SM (the link needs little in flight: four 16-byte loads per thread).
+__global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constant__ CacheView cv, int n_active,
                                                          const int32_t *active, const int32_t *layers, int n_layers,
                                                          int skip_copy, RecallSignal sig) {
   const Geometry &G = cv.geo;
@@ -142,7 +144,7 @@ __global__ void __launch_bounds__(256) wnw_recall_kernel(const __grid_constant__
   const int b = active[i];
   const long long bl = (long long)b * G.L + l;
   if (r < cv.n_plan[bl]) {
-    const LayerInfo li = cv.layers[l];
+    const LayerInfo &li = cv.layers[l];
     const int c = cv.plan[(bl * G.topk + r) * 2], slot = cv.plan[(bl * G.topk + r) * 2 + 1];
     const long long n_vec = (long long)li.n_tidal * 2 * G.ncp * G.d / 8;  // 16-byte vectors per chunk block
     if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(cv.stats + (long long)b * 4 + 3, (unsigned long long)n_vec * 16ull);
@@ -152,19 +154,19 @@ __global__ void __launch_bounds__(256) wnw_recall_kernel(const __grid_constant__
       } else {
         const uint4 *src = reinterpret_cast<const uint4 *>(cv.mirror[b] + mirror_off(G, li, cv.C[b], c, 0, 0));
         uint4 *dst = reinterpret_cast<uint4 *>(cv.pool + pool_off(G, li, b, slot, 0, 0));
-        constexpr int U = 8;
-        const long long stride = (long long)gridDim.x * blockDim.x;
-        for (long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; v0 < n_vec; v0 += stride * U) {
+        constexpr int U = 4;
+        const int stride = gridDim.x * blockDim.x, n = (int)n_vec;   // a chunk block is far below 2^31 vectors
+        for (int v0 = blockIdx.x * blockDim.x + threadIdx.x; v0 < n; v0 += stride * U) {
           uint4 t[U];
 #pragma unroll
           for (int u = 0; u < U; ++u) {
-            const long long v = v0 + u * stride;
-            if (v < n_vec) t[u] = __ldcs(src + v);
+            const int v = v0 + u * stride;
+            if (v < n) t[u] = __ldcs(src + v);
           }
 #pragma unroll
           for (int u = 0; u < U; ++u) {
-            const long long v = v0 + u * stride;
-            if (v < n_vec) dst[v] = t[u];
+            const int v = v0 + u * stride;
+            if (v < n) dst[v] = t[u];
           }
         }
       }

@@ -10,10 +10,12 @@ from workloads import config1, config3, config4
 pytestmark = pytest.mark.gpu
 
 
-def _run(w, oracle_seqs, n_steps, graph=True):
+def _run(w, oracle_seqs, n_steps, graph=True, layer_dependency=0):
+    import paper_2608_22704_b200 as wnw
     from parity_harness import Lockstep
     ls = Lockstep(w, seed=0, gen_device="cuda:0", oracle_seqs=oracle_seqs)
     try:
+        wnw.wnw_set_layer_dependency(ls.h, layer_dependency)
         ls.prefill(check_slots=False)
         for t in range(n_steps):
             ls.decode_step(t, graph=graph, check_slots=(t == n_steps - 1))
@@ -22,12 +24,14 @@ def _run(w, oracle_seqs, n_steps, graph=True):
         ls.close()
 
 
-def test_config3_batch32_ragged_sampled_sequences():
+@pytest.mark.parametrize("layer_dependency", [0, 1])
+def test_config3_batch32_ragged_sampled_sequences(layer_dependency):
     """Batched serving: config-1 shapes at batch 32, audio lengths U{2000..7500}; the oracle follows the shortest and
-    the longest sequence through prefill placement and three decode steps."""
+    the longest sequence through prefill placement and three decode steps.  Independent layers run as one-shot CTAs
+    (mostly one per head); chained layers run as persistent CTAs over the host-balanced schedule."""
     w = config3(n_steps=3)
     lens = np.array(w.audio_lens)
-    _run(w, oracle_seqs=sorted({int(lens.argmin()), int(lens.argmax())}), n_steps=3)
+    _run(w, oracle_seqs=sorted({int(lens.argmin()), int(lens.argmax())}), n_steps=3, layer_dependency=layer_dependency)
 
 
 @pytest.mark.parametrize("budget,chunk", [(0.1, 16), (0.4, 256)])
@@ -37,6 +41,7 @@ def test_config4_recall_stress_corners(budget, chunk):
     every resident slot holds the exact bytes of its chunk."""
     w = config4(budget=budget, chunk=chunk, n_steps=5)
     _run(w, oracle_seqs=[3], n_steps=5)
+    _run(w, oracle_seqs=[5], n_steps=2, layer_dependency=2)
 
 
 def test_config1_sixty_four_steps_graph_replay():
