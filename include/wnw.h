@@ -207,6 +207,10 @@ wnw_status_t wnw_get_stats(wnw_cache_t *cache, wnw_stats_t *stats_host);
 enum { WNW_LAYERS_INDEPENDENT = 0, WNW_LAYERS_CHAINED = 1, WNW_LAYERS_SERIAL = 2 };
 wnw_status_t wnw_set_layer_dependency(wnw_cache_t *cache, int32_t mode);
 
+/* Kernels this cache has launched on the decode path since creation, replayed captured steps included:
+ * counts[0] attention, [1] selection, [2] recall, [3] step-end.  Host counters, no synchronisation. */
+wnw_status_t wnw_get_launch_counts(wnw_cache_t *cache, int64_t counts[4]);
+
 /* Optional per-kernel timing: when enabled the library brackets its attention-kernel launches with CUDA events
  * on the launching stream; wnw_get_kernel_time returns the accumulated milliseconds and launch count since the
  * last call (drains the stream).  Off by default. */

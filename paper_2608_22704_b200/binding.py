@@ -65,6 +65,7 @@ _SIGNATURES = {
     "wnw_get_slot_kv": [_vp, _i32, _i32, _i32, _i32, _i32, _vp],
     "wnw_get_stats": [_vp, C.POINTER(wnw_stats_t)],
     "wnw_set_layer_dependency": [_vp, _i32],
+    "wnw_get_launch_counts": [_vp, C.POINTER(C.c_int64)],
     "wnw_set_kernel_timing": [_vp, _i32],
     "wnw_get_kernel_time": [_vp, C.POINTER(C.c_float), C.POINTER(_i32)],
     "wnw_sync": [_vp],
@@ -237,6 +238,13 @@ def wnw_get_stats(cache) -> dict:
     s = wnw_stats_t()
     _ck(lib().wnw_get_stats(cache, C.byref(s)), "wnw_get_stats")
     return {n: getattr(s, n) for n, _ in wnw_stats_t._fields_}
+
+
+def wnw_get_launch_counts(cache):
+    """(attention, selection, recall, step-end) kernels launched so far, replayed steps included."""
+    arr = (C.c_int64 * 4)()
+    _ck(lib().wnw_get_launch_counts(cache, arr), "wnw_get_launch_counts")
+    return tuple(int(x) for x in arr)
 
 
 def wnw_set_layer_dependency(cache, mode: int):

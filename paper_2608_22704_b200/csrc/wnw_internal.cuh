@@ -163,6 +163,12 @@ struct SelectArgs {
   int32_t n_aq, n_ag_max;
   uint8_t aq_head[MAX_AQ]; // query-head index of anchor q-head slot aq (score order)
   int16_t upd_layer[MAX_UPD_BY_VALUE], upd_src[MAX_UPD_BY_VALUE];
+  // Captured steps: the selection CTA that finishes last in the step also does the step's bookkeeping (step counters,
+  // text lengths, recall epoch), which saves the dependent launch of a kernel of its own at the end of every step.
+  int32_t fold_total;      // selection CTAs in the step (0: the step-end kernel runs instead)
+  int32_t fold_appended;   // the step appended a text token
+  int32_t *fold_counter;   // finished selection CTAs (self-resetting)
+  int32_t *fold_bump_epoch;
 };
 
 // Completion signalling of a recall launch that runs outside the captured step (all null for in-step launches).

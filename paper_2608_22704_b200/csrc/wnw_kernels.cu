@@ -36,8 +36,30 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
     tile_c = (int)(em_room / ((long long)n_aq * G.gpc));
     if (tile_c > C_b) tile_c = C_b;
   }
+  __shared__ int s_last;
+  // Every CTA passes here exactly once, also on the error path: the last one of the step closes the step.
+  auto close_step = [&]() {
+    if (a.fold_total <= 0) return;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      __threadfence();
+      const int prev = atomicAdd(a.fold_counter, 1);
+      s_last = prev == a.fold_total - 1;
+      if (s_last) *a.fold_counter = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int j = threadIdx.x; j < a.n_active; j += NT) {
+      const int bj = a.active[j];
+      cv.steps[bj] += 1;
+      if (a.fold_appended) cv.text_len[bj] += 1;
+    }
+    if (threadIdx.x == 0 && a.fold_bump_epoch) *a.fold_bump_epoch += 1;
+  };
   if (em_room < 0 || (scored && tile_c < 1)) {  // beyond what the host sized the launch for
     if (threadIdx.x == 0) atomicOr(cv.status, STATUS_BAD_TABLE);
+    close_step();
     return;
   }
   auto stage_em = [&](int c0, int c1) {
@@ -118,6 +140,7 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
       select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, src == -2 ? glob_s : (local ? sc_s : w.sc), w);
     }
   }
+  close_step();
 }
 
 cudaError_t configure_select_kernel() {

@@ -97,6 +97,11 @@ struct wnw_cache {
   size_t gran_em_layer_stride = 0;
   bool step_capturing = false;
   bool pdl_enabled = true;
+  bool fold_enabled = true, cap_fold = false;   // captured steps: the last selection CTA closes the step
+  int n_side_layers = 0;
+  int32_t *d_fold_ctr = nullptr;
+  long long launches[4] = {0, 0, 0, 0}, cap_launches[4] = {0, 0, 0, 0};  // attention, selection, recall, step-end kernels
+  void count_launch(int kind, int n, bool capturing) { (capturing ? cap_launches : launches)[kind] += n; }
   int layer_dependency = WNW_LAYERS_INDEPENDENT;
   // replayed steps: one recall launch per step outside the captured graph, overlapping the next step
   int32_t *d_recall_epoch = nullptr, *d_recall_ctr = nullptr, *d_step_epoch = nullptr;
@@ -235,6 +240,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
 #define CKE(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { return fail(_e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA); } } while (0)
   cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
   if (const char *e = getenv("WNW_PDL")) c->pdl_enabled = atoi(e) != 0;
+  if (const char *e = getenv("WNW_FOLD_STEP_END")) c->fold_enabled = atoi(e) != 0;
   if (const char *e = getenv("WNW_EXTERNAL_RECALL")) c->external_recall_mode = atoi(e);
   if (const char *e = getenv("WNW_DIRECT_MAX_GRANULES")) c->direct_max_granules = atoi(e);
   CKE(configure_attn_kernels());
@@ -400,6 +406,9 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   CKC(dev_alloc(c, &c->d_recall_epoch, (size_t)L));
   CKC(dev_alloc(c, &c->d_recall_ctr, (size_t)L));
   CKC(dev_alloc(c, &c->d_step_epoch, 1));
+  CKC(dev_alloc(c, &c->d_fold_ctr, 1));
+  for (int l = 0; l < L; ++l)
+    if (!full && (c->layers[l].n_anchor > 0 || c->layers[l].upd_count > 0)) ++c->n_side_layers;
   CKE(cudaDeviceSynchronize());
 #undef CKC
 #undef CKE
@@ -751,6 +760,11 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     // they wait for it, so recall stays inside the step there.
     bool small = true;   // no launch can fill the machine with CTAs that wait
     for (const LayerWork &w : c->wl_layers) small = small && !w.throughput && w.n_items <= c->n_sm / 2;
+    // the selection kernel of the last layer starts after every attention kernel of the step has completed, so the
+    // selection CTA that finishes last in the step may update what those kernels read
+    const LayerInfo &last = c->layers[G.L - 1];
+    c->cap_fold = c->fold_enabled && capturing && c->graph_capturing && tiered && c->cfg.recall_mode != WNW_RECALL_INLINE &&
+                  (last.n_anchor > 0 || last.upd_count > 0);
     c->cap_external_recall = capturing && c->graph_capturing && tiered && c->cfg.recall_mode != WNW_RECALL_INLINE &&
                              (c->external_recall_mode == 1 || (c->external_recall_mode < 0 && small));
   }
@@ -802,6 +816,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     CK(cudaEventRecord(t0, st));
   }
   CK(launch_attn(c->cv, a, st));
+  c->count_launch(0, 1, capturing);
   if (timing) {
     CK(cudaEventRecord(t1, st));
     c->t_used.emplace_back(t0, t1);
@@ -815,6 +830,10 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     SelectArgs sa{};
     sa.layer = layer; sa.n_active = n_active; sa.score_on = a.score_on; sa.li = li; sa.active = c->d_active;
     sa.gran_em = gran_em_l; sa.head_mz = head_mz_l; sa.n_aq = a.n_aq; sa.n_ag_max = a.n_ag_max;
+    if (c->cap_fold) {
+      sa.fold_total = c->n_side_layers * n_active; sa.fold_appended = has_new; sa.fold_counter = c->d_fold_ctr;
+      sa.fold_bump_epoch = c->cap_external_recall ? c->d_step_epoch : nullptr;
+    }
     int aq = 0;
     for (int h = 0; h < G.Hkv; ++h)
       if (c->roles[layer * G.Hkv + h] == ROLE_ANCHOR)
@@ -840,9 +859,12 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
             CK(cudaStreamWaitEvent(ss, capturing ? c->ev_side_done_cap[al] : c->ev_side_done[al], 0));
     }
     CK(launch_select(c->cv, sa, c->sel_smem[layer], ss));
-    if (li.upd_count > 0 && !c->cap_external_recall)
+    c->count_launch(1, 1, capturing);
+    if (li.upd_count > 0 && !c->cap_external_recall) {
       CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count,
                        c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{nullptr, nullptr, nullptr}, ss));
+      c->count_launch(2, 1, capturing);
+    }
     if (!inline_mode) {
       CK(cudaEventRecord(ev_s, ss));
       if (!capturing) c->side_recorded[layer] = 1;
@@ -875,8 +897,11 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
     for (int ls : c->last_side_layer)  // join the forked side streams into the graph
       if (ls >= 0) CK(cudaStreamWaitEvent(st, c->ev_side_done_cap[ls], 0));
 
-  CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1,
-                     (capturing && c->cap_external_recall) ? c->d_step_epoch : nullptr, st));
+  if (!(capturing && c->cap_fold)) {
+    CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1,
+                       (capturing && c->cap_external_recall) ? c->d_step_epoch : nullptr, st));
+    c->count_launch(3, 1, capturing);
+  }
   if (!capturing) {
     CK(cudaEventRecord(c->ev_step, st));
     c->step_recorded = true;
@@ -916,6 +941,7 @@ extern "C" wnw_status_t wnw_graph_begin(wnw_cache_t *c, const int32_t *active, i
   for (auto sd : c->side) CK(cudaStreamSynchronize(sd));
   if (c->last_stream != st) CK(cudaStreamSynchronize(c->last_stream));
   CK(cudaStreamSynchronize(st));
+  for (long long &x : c->cap_launches) x = 0;
   CK(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
   c->graph_capturing = true;
   c->graph_active.clear();
@@ -960,6 +986,7 @@ extern "C" wnw_status_t wnw_graph_launch(wnw_cache_t *c, void *cuda_stream) {
   for (int l = 0; l < c->geo.L; ++l)
     if (c->side_recorded[l]) { CK(cudaStreamWaitEvent(st, c->ev_side_done[l], 0)); c->side_recorded[l] = 0; }
   CK(cudaGraphLaunch(c->graph_exec, st));
+  for (int k = 0; k < 4; ++k) c->launches[k] += c->cap_launches[k];  // the kernels of the captured step
   if (c->graph_external_recall && !c->upd_list.empty()) {
     // This step's recall, for every layer's table at once, outside the graph: it overlaps the next replay, whose tidal
     // CTAs wait on the per-layer epoch words it publishes.
@@ -968,6 +995,7 @@ extern "C" wnw_status_t wnw_graph_launch(wnw_cache_t *c, void *cuda_stream) {
     CK(launch_recall(c->cv, (int)c->graph_active.size(), c->d_active, c->cv.upd_list, (int)c->upd_list.size(),
                      c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{c->d_recall_epoch, c->d_recall_ctr, c->d_step_epoch},
                      c->side[0]));
+    c->count_launch(2, 1, false);
     CK(cudaEventRecord(c->ev_recall_all, c->side[0]));
     c->recall_all_pending = true;
   }
@@ -1146,6 +1174,12 @@ extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
     }
   }
   *out = r;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_launch_counts(wnw_cache_t *c, int64_t *counts) {
+  if (!c || !counts) return WNW_ERR_INVALID_ARG;
+  for (int k = 0; k < 4; ++k) counts[k] = c->launches[k];
   return WNW_OK;
 }
 
