@@ -169,12 +169,18 @@ struct SelectArgs {
   int32_t fold_appended;   // the step appended a text token
   int32_t *fold_counter;   // finished selection CTAs (self-resetting)
   int32_t *fold_bump_epoch;
+  // Recall outside the captured step: a layer whose tables need no copy in this step (for any sequence) gets its recall
+  // epoch published right here, so the next step's tidal CTAs do not wait for the recall launch at all.
+  int32_t *epoch_words;        // [L] or null
+  int32_t *empty_ctr;          // [L] sequences with an empty plan (reset by whoever publishes the layer's epoch)
+  const int32_t *step_epoch;
 };
 
 // Completion signalling of a recall launch that runs outside the captured step (all null for in-step launches).
 struct RecallSignal {
   int32_t *epoch_words;       // [L] epoch of the last completed recall of each layer's table
   int32_t *counters;          // [L] finished-CTA counters (self-resetting)
+  int32_t *empty_ctr;         // [L] the selection kernels' empty-plan counters, reset here
   const int32_t *step_epoch;  // epoch to publish: the number of replayed steps that have ended
 };
 

@@ -137,7 +137,16 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
         cp_async_commit_wait_all();
         __syncwarp();
       }
-      select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, src == -2 ? glob_s : (local ? sc_s : w.sc), w);
+      const int n_copies = select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, src == -2 ? glob_s : (local ? sc_s : w.sc), w);
+      if (a.epoch_words && n_copies == 0 && lane == 0) {
+        const int prev = atomicAdd(a.empty_ctr + lt, 1);
+        if (prev == a.n_active - 1) {   // nothing to recall for this layer in this step: its slots are current
+          a.empty_ctr[lt] = 0;
+          __threadfence();
+          const int epoch = *a.step_epoch + 1;   // the step's own bump comes after every selection CTA has finished
+          asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(a.epoch_words + lt), "r"(epoch) : "memory");
+        }
+      }
     }
   }
   close_step();
@@ -153,33 +162,43 @@ cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_
 }
 
 // ------------------------------------------------------------------------------------------------
-// Recall: copies every planned chunk block pinned host -> slot pool.  grid (ctas, topk, n_layers * n_active), earlier
-// layers first.  With `sig` set (replayed steps, where this kernel runs outside the captured graph and overlaps the
-// next step) the last CTA of every layer publishes the layer's recall epoch, which the next step's tidal CTAs acquire.
+// Recall: copies every planned chunk block pinned host -> slot pool.  A NARROW kernel: RECALL_CTAS CTAs in up to
+// RECALL_GROUPS groups; group g walks the layers g, g + groups, ... (earlier layers first), every CTA of the group taking
+// its stripe of each block, so several layers' transfers are in flight at once.  The host link needs little in flight
+// (32 CTAs x 256 threads x four 16-byte loads = 512 KB); CTAs that wait on the link must not sit on the SMs the
+// attention kernels need (40 registers, one CTA per SM, fits beside a resident attention CTA).
+// With `sig` set (replayed steps, where this kernel runs outside the captured graph and overlaps the next step) the
+// CTA that finishes a layer last publishes the layer's recall epoch, which the next step's tidal CTAs acquire.
 // ------------------------------------------------------------------------------------------------
-// At most 40 registers per thread, so that a recall CTA fits beside a resident attention CTA instead of waiting for a
-// free SM (the link needs little in flight: four 16-byte loads per thread).
+constexpr int RECALL_CTAS = 32, RECALL_GROUPS = 8;
 __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constant__ CacheView cv, int n_active,
-                                                         const int32_t *active, const int32_t *layers, int n_layers,
-                                                         int skip_copy, RecallSignal sig) {
+                                                            const int32_t *active, const int32_t *layers, int n_layers,
+                                                            int n_groups, int skip_copy, RecallSignal sig) {
   const Geometry &G = cv.geo;
-  const int l = layers[blockIdx.z / n_active], i = blockIdx.z % n_active, r = blockIdx.y;
-  const int b = active[i];
-  const long long bl = (long long)b * G.L + l;
-  if (r < cv.n_plan[bl]) {
+  constexpr int U = 4;
+  const int cpg = gridDim.x / n_groups, grp = blockIdx.x / cpg, rank = blockIdx.x - grp * cpg;
+  const int stride = cpg * blockDim.x;
+  for (int x = grp; x < n_layers; x += n_groups) {
+    const int l = layers[x];
     const LayerInfo &li = cv.layers[l];
-    const int c = cv.plan[(bl * G.topk + r) * 2], slot = cv.plan[(bl * G.topk + r) * 2 + 1];
-    const long long n_vec = (long long)li.n_tidal * 2 * G.ncp * G.d / 8;  // 16-byte vectors per chunk block
-    if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(cv.stats + (long long)b * 4 + 3, (unsigned long long)n_vec * 16ull);
-    if (!skip_copy) {
-      if (c < 0 || c >= cv.C[b] || slot < 0 || slot >= cv.S[b]) {
-        if (threadIdx.x == 0) atomicOr(cv.status, STATUS_BAD_TABLE);
-      } else {
+    const int n = li.n_tidal * 2 * G.ncp * G.d / 8;  // 16-byte vectors per chunk block (far below 2^31)
+    bool copies = false;                             // uniform over the whole grid: the plans do not change under this kernel
+    for (int i = 0; i < n_active; ++i) {
+      const int b = active[i];
+      const long long bl = (long long)b * G.L + l;
+      const int n_plan = cv.n_plan[bl];
+      for (int r = 0; r < n_plan && r < G.topk; ++r) {
+        const int c = cv.plan[(bl * G.topk + r) * 2], slot = cv.plan[(bl * G.topk + r) * 2 + 1];
+        if (rank == 0 && threadIdx.x == 0) atomicAdd(cv.stats + (long long)b * 4 + 3, (unsigned long long)n * 16ull);
+        if (skip_copy) continue;
+        copies = true;
+        if (c < 0 || c >= cv.C[b] || slot < 0 || slot >= cv.S[b]) {
+          if (threadIdx.x == 0) atomicOr(cv.status, STATUS_BAD_TABLE);
+          continue;
+        }
         const uint4 *src = reinterpret_cast<const uint4 *>(cv.mirror[b] + mirror_off(G, li, cv.C[b], c, 0, 0));
         uint4 *dst = reinterpret_cast<uint4 *>(cv.pool + pool_off(G, li, b, slot, 0, 0));
-        constexpr int U = 4;
-        const int stride = gridDim.x * blockDim.x, n = (int)n_vec;   // a chunk block is far below 2^31 vectors
-        for (int v0 = blockIdx.x * blockDim.x + threadIdx.x; v0 < n; v0 += stride * U) {
+        for (int v0 = rank * blockDim.x + threadIdx.x; v0 < n; v0 += stride * U) {
           uint4 t[U];
 #pragma unroll
           for (int u = 0; u < U; ++u) {
@@ -194,18 +213,25 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
         }
       }
     }
-  }
-  if (sig.epoch_words) {  // completion of this layer's recall: counted per CTA, published by the last one
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      const int total = gridDim.x * gridDim.y * n_active;
-      const int prev = atomicAdd(sig.counters + l, 1);
-      if (prev == total - 1) {
-        sig.counters[l] = 0;
-        __threadfence();
+    if (sig.epoch_words && !copies) {
+      // nothing was written for this layer: its epoch goes out at once, without the round of fences and counting
+      if (rank == 0 && threadIdx.x == 0) {
+        sig.empty_ctr[l] = 0;
         const int epoch = *sig.step_epoch;
         asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(sig.epoch_words + l), "r"(epoch) : "memory");
+      }
+    } else if (sig.epoch_words) {  // completion of this layer's recall: counted per CTA, published by the last one
+      __threadfence();
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        const int prev = atomicAdd(sig.counters + l, 1);
+        if (prev == cpg - 1) {
+          sig.counters[l] = 0;
+          sig.empty_ctr[l] = 0;
+          __threadfence();
+          const int epoch = *sig.step_epoch;
+          asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(sig.epoch_words + l), "r"(epoch) : "memory");
+        }
       }
     }
   }
@@ -214,14 +240,14 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
 cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,
                           int skip_copy, RecallSignal sig, cudaStream_t st) {
   if (n_layers <= 0 || n_active <= 0) return cudaSuccess;
-  wnw_recall_kernel<<<dim3(8, cv.geo.topk, n_active * n_layers), 256, 0, st>>>(cv, n_active, active, layers_dev, n_layers,
-                                                                            skip_copy, sig);
+  const int groups = n_layers < RECALL_GROUPS ? n_layers : RECALL_GROUPS;   // few layers: all CTAs on each block
+  wnw_recall_kernel<<<RECALL_CTAS / groups * groups, 256, 0, st>>>(cv, n_active, active, layers_dev, n_layers, groups, skip_copy, sig);
   return cudaGetLastError();
 }
 
 // Plain host-mapped -> device copy with the recall kernel's access pattern (link probe).
 __global__ void __launch_bounds__(256) wnw_copy_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, long long n_vec) {
-  constexpr int U = 8;
+  constexpr int U = 4;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long v0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; v0 < n_vec; v0 += stride * U) {
     uint4 t[U];

@@ -99,7 +99,7 @@ struct wnw_cache {
   bool pdl_enabled = true;
   bool fold_enabled = true, cap_fold = false;   // captured steps: the last selection CTA closes the step
   int n_side_layers = 0;
-  int32_t *d_fold_ctr = nullptr;
+  int32_t *d_fold_ctr = nullptr, *d_empty_ctr = nullptr;
   long long launches[4] = {0, 0, 0, 0}, cap_launches[4] = {0, 0, 0, 0};  // attention, selection, recall, step-end kernels
   void count_launch(int kind, int n, bool capturing) { (capturing ? cap_launches : launches)[kind] += n; }
   int layer_dependency = WNW_LAYERS_INDEPENDENT;
@@ -407,6 +407,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   CKC(dev_alloc(c, &c->d_recall_ctr, (size_t)L));
   CKC(dev_alloc(c, &c->d_step_epoch, 1));
   CKC(dev_alloc(c, &c->d_fold_ctr, 1));
+  CKC(dev_alloc(c, &c->d_empty_ctr, (size_t)L));
   for (int l = 0; l < L; ++l)
     if (!full && (c->layers[l].n_anchor > 0 || c->layers[l].upd_count > 0)) ++c->n_side_layers;
   CKE(cudaDeviceSynchronize());
@@ -834,6 +835,9 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
       sa.fold_total = c->n_side_layers * n_active; sa.fold_appended = has_new; sa.fold_counter = c->d_fold_ctr;
       sa.fold_bump_epoch = c->cap_external_recall ? c->d_step_epoch : nullptr;
     }
+    if (c->cap_external_recall && c->cap_fold) {   // the epoch arithmetic relies on the bump coming after every selection
+      sa.epoch_words = c->d_recall_epoch; sa.empty_ctr = c->d_empty_ctr; sa.step_epoch = c->d_step_epoch;
+    }
     int aq = 0;
     for (int h = 0; h < G.Hkv; ++h)
       if (c->roles[layer * G.Hkv + h] == ROLE_ANCHOR)
@@ -862,7 +866,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     c->count_launch(1, 1, capturing);
     if (li.upd_count > 0 && !c->cap_external_recall) {
       CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count,
-                       c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{nullptr, nullptr, nullptr}, ss));
+                       c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{nullptr, nullptr, nullptr, nullptr}, ss));
       c->count_launch(2, 1, capturing);
     }
     if (!inline_mode) {
@@ -993,7 +997,7 @@ extern "C" wnw_status_t wnw_graph_launch(wnw_cache_t *c, void *cuda_stream) {
     CK(cudaEventRecord(c->ev_graph_done, st));
     CK(cudaStreamWaitEvent(c->side[0], c->ev_graph_done, 0));
     CK(launch_recall(c->cv, (int)c->graph_active.size(), c->d_active, c->cv.upd_list, (int)c->upd_list.size(),
-                     c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{c->d_recall_epoch, c->d_recall_ctr, c->d_step_epoch},
+                     c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{c->d_recall_epoch, c->d_recall_ctr, c->d_empty_ctr, c->d_step_epoch},
                      c->side[0]));
     c->count_launch(2, 1, false);
     CK(cudaEventRecord(c->ev_recall_all, c->side[0]));
@@ -1239,7 +1243,7 @@ extern "C" wnw_status_t wnw_measure_host_link(int32_t device, int64_t bytes, int
     if (cudaStreamSynchronize(st) != cudaSuccess || cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc = WNW_ERR_CUDA; break; }
     if (r > 0) best_copy = std::min(best_copy, ms);
     cudaEventRecord(e0, st);
-    if (launch_copy_plan((const uint4 *)hd, (uint4 *)d, bytes / 16, 64, st) != cudaSuccess) { rc = WNW_ERR_CUDA; break; }
+    if (launch_copy_plan((const uint4 *)hd, (uint4 *)d, bytes / 16, 32, st) != cudaSuccess) { rc = WNW_ERR_CUDA; break; }
     cudaEventRecord(e1, st);
     if (cudaStreamSynchronize(st) != cudaSuccess || cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc = WNW_ERR_CUDA; break; }
     if (r > 0) best_kernel = std::min(best_kernel, ms);

@@ -84,7 +84,8 @@ __device__ __forceinline__ void select_stage(const CacheView &cv, int b, int lt,
 // Stage 2 (one warp): top-k of layer `lt` from scores `sc` (shared memory), then the residency update (hit:
 // refresh stamp; miss: lowest free slot, else least recently selected resident not selected now) and the recall
 // plan.  Works on the staged table; global memory only receives stores.
-__device__ __forceinline__ void select_and_update(const CacheView &cv, int b, int lt, int src, int C_b, int S_b, int T_a,
+// Returns the number of planned copies (uniform over the warp).
+__device__ __forceinline__ int select_and_update(const CacheView &cv, int b, int lt, int src, int C_b, int S_b, int T_a,
                                                   long long step, int lane, const float *sc, const SelectWs &w) {
   const Geometry &G = cv.geo;
   const long long bl = (long long)b * G.L + lt;
@@ -170,6 +171,7 @@ __device__ __forceinline__ void select_and_update(const CacheView &cv, int b, in
       atomicAdd(cv.stats + (long long)b * 4 + 2, (unsigned long long)evictions);
     }
   }
+  return n_plan;
 }
 
 }  // namespace wnw
