@@ -40,7 +40,16 @@
  *   - a selection made at step s is used by tidal attention at step s+1;
  *   - slots S = max(1, floor((double)budget * C + 1e-6)), capped at C;
  *   - stamps: a chunk selected with rank r at step s gets s*topk + (topk-1-r);
- *     prefill gives rank r the stamp -1-r.
+ *     prefill gives rank r the stamp -1-r;
+ *   - residency SEGMENT_LAG (Chunk Structure + Dynamic Chunk Selection as printed):
+ *     the storage unit (`chunk` tokens) is a SEGMENT; a chunk is two consecutive
+ *     segments, so adjacent chunks share one; chunk j = segments {j, j+1}, ranked
+ *     by the mean over its tokens, (float)(sum_j + sum_{j+1}) / (len_j + len_{j+1});
+ *     the segments placed at prefill stay resident for good (slots [0, S_base));
+ *     the segments of the selected chunks that are not resident are fetched into
+ *     dynamic slots [S_base, S); a fetched segment left unselected for delta
+ *     consecutive steps is dropped (its stamp = the step it was last selected in).
+ *     D = S - S_base = 2*topk*(delta+1) dynamic slots always suffice.
  */
 #include <math.h>
 #include <stdint.h>
@@ -59,7 +68,8 @@
 typedef struct {
   int placed_layers;   /* how many layers have been placed */
   int T_a, T_t, T_cap; /* audio tokens, current text tokens, text capacity */
-  int C, S;            /* chunks, slots */
+  int C, S;            /* chunks (segments in SEGMENT_LAG), slots of the tidal table */
+  int S_base;          /* slots filled at prefill; = S with the hard budget; fixed heads keep S_base chunks */
   long long steps;     /* decode steps this sequence took part in */
   uint16_t **audK, **audV; /* [L] -> [Hkv][T_a][d]   full audio K,V of every head */
   uint16_t **txtK, **txtV; /* [L] -> [Hkv][T_cap][d] */
@@ -77,6 +87,8 @@ typedef struct {
 typedef struct {
   int L, Hq, Hkv, d, g, chunk, topk, max_batch, max_audio, max_text;
   int scope;      /* 0: per layer with nearest-anchor routing; 1: global sum over all anchor layers */
+  int residency;  /* 0: hard budget (fixed pool, least-recently-selected eviction); 1: SEGMENT_LAG */
+  int delta;      /* eviction lag of SEGMENT_LAG */
   double budget, scale;
   uint8_t *roles; /* [L][Hkv] */
   int *src;       /* [L] score source layer, -1 if the layer has no tidal heads or no source */
@@ -175,6 +187,76 @@ int wnwo_table_update(int *slot_chunk, long long *stamp, int S, const int *sel, 
   return n_plan;
 }
 
+/* Dynamic Chunk Selection over OVERLAPPING chunks (Chunk Structure): chunk j is segments j and j+1 (a clip of one
+ * segment has the single chunk {0}).  seg_sum as float, lens = tokens per segment.  Writes the k best chunks in rank
+ * order to sel_chunks and their segments, in that order without repeats, to segs; returns the number of segments. */
+int wnwo_select_segments(const float *seg_sum, const int *lens, int n_seg, int k, int *sel_chunks, int *n_sel, int *segs) {
+  const int n_ch = n_seg > 1 ? n_seg - 1 : n_seg;
+  if (k > n_ch) k = n_ch;
+  float *ch_sum = (float *)malloc(sizeof(float) * (size_t)(n_ch > 0 ? n_ch : 1));
+  int *ch_len = (int *)malloc(sizeof(int) * (size_t)(n_ch > 0 ? n_ch : 1));
+  if (!ch_sum || !ch_len) { free(ch_sum); free(ch_len); return -1; }
+  for (int j = 0; j < n_ch; ++j) {
+    ch_sum[j] = n_seg > 1 ? seg_sum[j] + seg_sum[j + 1] : seg_sum[j]; /* float add: the decision precision */
+    ch_len[j] = n_seg > 1 ? lens[j] + lens[j + 1] : lens[j];
+  }
+  k = wnwo_topk(ch_sum, ch_len, n_ch, k, sel_chunks);
+  free(ch_sum); free(ch_len);
+  if (k < 0) return -1;
+  int n = 0;
+  for (int r = 0; r < k; ++r)
+    for (int e = 0; e < (n_seg > 1 ? 2 : 1); ++e) {
+      int g = sel_chunks[r] + e, seen = 0;
+      for (int i = 0; i < n; ++i) seen |= segs[i] == g;
+      if (!seen) segs[n++] = g;
+    }
+  if (n_sel) *n_sel = k;
+  return n;
+}
+
+/* Chunk swap with a permanent base and lag-delta release (Dynamic Chunk Selection).  Slots [0, S_base) never change.
+ * segs: the selected segments of this step, in order.  A selected segment that is resident is a hit (a dynamic one gets
+ * stamp = step); then every dynamic slot whose segment was not selected now and has step - stamp >= delta is released;
+ * then the misses take the lowest free dynamic slots in order.  released[] receives the dropped segments.
+ * Returns the number of misses (plan entries), -1 if no free slot was left (cannot happen when S - S_base >= 2k(delta+1)). */
+int wnwo_lag_update(int *slot_seg, long long *stamp, int S_base, int S, const int *segs, int n, long long step, int delta,
+                    int *plan_seg, int *plan_slot, int *released, int *n_released, int *n_hits) {
+  int hits = 0, n_rel = 0, n_plan = 0;
+  unsigned char *miss = (unsigned char *)calloc((size_t)(n > 0 ? n : 1), 1);
+  if (!miss) return -1;
+  for (int i = 0; i < n; ++i) {
+    int j = -1;
+    for (int x = 0; x < S; ++x)
+      if (slot_seg[x] == segs[i]) j = x;
+    if (j < 0) { miss[i] = 1; continue; }
+    ++hits;
+    if (j >= S_base) stamp[j] = step;
+  }
+  for (int x = S_base; x < S; ++x) {
+    if (slot_seg[x] < 0 || stamp[x] == step) continue; /* free, or selected in this step */
+    if (step - stamp[x] >= (long long)delta) {
+      released[n_rel++] = slot_seg[x];
+      slot_seg[x] = -1;
+    }
+  }
+  for (int i = 0; i < n; ++i) {
+    if (!miss[i]) continue;
+    int j = -1;
+    for (int x = S_base; x < S && j < 0; ++x)
+      if (slot_seg[x] < 0) j = x;
+    if (j < 0) { free(miss); return -1; }
+    slot_seg[j] = segs[i];
+    stamp[j] = step;
+    plan_seg[n_plan] = segs[i];
+    plan_slot[n_plan] = j;
+    ++n_plan;
+  }
+  free(miss);
+  if (n_released) *n_released = n_rel;
+  if (n_hits) *n_hits = hits;
+  return n_plan;
+}
+
 /* ------------------------------------------------------------------ */
 /* Life cycle                                                           */
 /* ------------------------------------------------------------------ */
@@ -197,16 +279,19 @@ void wnwo_destroy(Oracle *o) {
 }
 
 int wnwo_create(int L, int Hq, int Hkv, int d, int max_batch, int max_audio, int max_text, int chunk, int topk,
-                double budget, double scale, const uint8_t *roles, int scope, Oracle **out) {
+                double budget, double scale, const uint8_t *roles, int scope, int residency, int delta, Oracle **out) {
   if (!out || !roles || L < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv || d < 1 || max_batch < 1 || chunk < 1 || topk < 1)
     return WNWO_ERR_ARG;
-  if (!(budget > 0.0 && budget <= 1.0) || scope < 0 || scope > 1) return WNWO_ERR_ARG;
+  if (!(budget > 0.0 && budget <= 1.0) || scope < 0 || scope > 1 || residency < 0 || residency > 1 || delta < 0)
+    return WNWO_ERR_ARG;
   Oracle *o = (Oracle *)calloc(1, sizeof(Oracle));
   if (!o) return WNWO_ERR_OOM;
   o->L = L; o->Hq = Hq; o->Hkv = Hkv; o->d = d; o->g = Hq / Hkv; o->chunk = chunk; o->topk = topk;
   o->max_batch = max_batch; o->max_audio = max_audio; o->max_text = max_text;
   o->budget = budget;
   o->scope = scope;
+  o->residency = residency;
+  o->delta = delta;
   o->scale = scale > 0.0 ? scale : 1.0 / sqrt((double)d); /* Eq. 2: q K^T / sqrt(d) */
   o->roles = (uint8_t *)malloc((size_t)L * Hkv);
   o->src = (int *)malloc(sizeof(int) * L);
@@ -245,6 +330,12 @@ static int alloc_seq(Oracle *o, Seq *s, int T_a, int T_t) {
   int S = (int)floor(o->budget * (double)s->C + 1e-6);
   if (S < 1) S = 1;
   if (S > s->C) S = s->C;
+  s->S_base = S;
+  if (o->residency == 1) { /* dynamic slots for everything selected within the last delta+1 steps */
+    int D = 2 * o->topk * (o->delta + 1);
+    if (D > s->C - S) D = s->C - S;
+    S += D;
+  }
   s->S = S;
   size_t nS = (size_t)(S > 0 ? S : 1), nC = (size_t)(s->C > 0 ? s->C : 1);
   s->audK = (uint16_t **)calloc((size_t)L, sizeof(void *)); s->audV = (uint16_t **)calloc((size_t)L, sizeof(void *));
@@ -393,7 +484,7 @@ int wnwo_place_prefill(Oracle *o, int seq, int layer, const uint16_t *k, const u
     if (role == ROLE_FIXED) { /* its own top-S chunks, frozen */
       for (int c = 0; c < C; ++c) keyf[c] = (float)pre[c];
       int *F = s->fixed_set + ((size_t)layer * Hkv + h) * S;
-      s->fixed_n[layer * Hkv + h] = wnwo_topk(keyf, lens, C, S, F);
+      s->fixed_n[layer * Hkv + h] = wnwo_topk(keyf, lens, C, s->S_base, F);
     } else {
       for (int c = 0; c < C; ++c) tid[c] += pre[c]; /* summed in head order */
       ++n_tid;
@@ -402,7 +493,7 @@ int wnwo_place_prefill(Oracle *o, int seq, int layer, const uint16_t *k, const u
   if (n_tid > 0) { /* one table for the layer's tidal heads: rank r -> slot r, stamp -1-r */
     for (int c = 0; c < C; ++c) keyf[c] = (float)tid[c];
     int *tmp = (int *)malloc(sizeof(int) * S);
-    int n = wnwo_topk(keyf, lens, C, S, tmp);
+    int n = wnwo_topk(keyf, lens, C, s->S_base, tmp);
     for (int r = 0; r < n; ++r) {
       s->slot_chunk[(size_t)layer * S + r] = tmp[r];
       s->stamp[(size_t)layer * S + r] = -1 - (long long)r;
@@ -495,11 +586,22 @@ int wnwo_step_end(Oracle *o) {
         for (int a = 0; a < o->L; ++a)
           if (layer_has(o, a, ROLE_ANCHOR))
             for (int c = 0; c < C; ++c) glob[c] += s->score_sum[(size_t)a * C + c];
+      int *segs = (int *)malloc(sizeof(int) * 2 * o->topk), *rel = (int *)malloc(sizeof(int) * (size_t)(S > 0 ? S : 1));
+      int *pg = (int *)malloc(sizeof(int) * 2 * o->topk), *pj = (int *)malloc(sizeof(int) * 2 * o->topk);
       for (int l = 0; l < o->L; ++l) {
         s->n_sel[l] = 0;
         if (o->src[l] < 0) continue;
         const double *sc = o->scope == 1 ? glob : s->score_sum + (size_t)o->src[l] * C;
         for (int c = 0; c < C; ++c) sf[c] = (float)sc[c];
+        if (o->residency == 1) { /* overlapping chunks, permanent base, lag-delta release */
+          int n_sel = 0, n_rel = 0, hits = 0;
+          int n_seg = wnwo_select_segments(sf, lens, C, o->topk, s->sel + (size_t)l * o->topk, &n_sel, segs);
+          s->n_sel[l] = n_sel;
+          int n = wnwo_lag_update(s->slot_chunk + (size_t)l * S, s->stamp + (size_t)l * S, s->S_base, S, segs, n_seg, s->steps,
+                                  o->delta, pg, pj, rel, &n_rel, &hits);
+          s->hits += hits; s->misses += n; s->evictions += n_rel;
+          continue;
+        }
         int k = o->topk < S ? o->topk : S;
         k = wnwo_topk(sf, lens, C, k, s->sel + (size_t)l * o->topk);
         s->n_sel[l] = k;
@@ -509,7 +611,7 @@ int wnwo_step_end(Oracle *o) {
         s->hits += hits; s->misses += n;
         for (int j = 0; j < n; ++j) s->evictions += ev[j] >= 0;
       }
-      free(lens); free(sf); free(pc); free(ps); free(ev); free(glob);
+      free(lens); free(sf); free(pc); free(ps); free(ev); free(glob); free(segs); free(rel); free(pg); free(pj);
     }
     s->steps += 1;
     if (o->appended == 1) s->T_t += 1;
@@ -526,6 +628,11 @@ int wnwo_get_dims(const Oracle *o, int seq, int *T_a, int *T_t, int *C, int *S) 
   if (!o || seq < 0 || seq >= o->max_batch || o->seq[seq].placed_layers == 0) return WNWO_ERR_STATE;
   const Seq *s = &o->seq[seq];
   *T_a = s->T_a; *T_t = s->T_t; *C = s->C; *S = s->S;
+  return WNWO_OK;
+}
+int wnwo_get_base_slots(const Oracle *o, int seq, int *S_base) {
+  if (!o || seq < 0 || seq >= o->max_batch || o->seq[seq].placed_layers == 0) return WNWO_ERR_STATE;
+  *S_base = o->seq[seq].S_base;
   return WNWO_OK;
 }
 int wnwo_get_chunk_scores(const Oracle *o, int seq, int layer, double *scores) {

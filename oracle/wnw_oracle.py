@@ -41,7 +41,8 @@ def lib():
     global _lib
     if _lib is None:
         _lib = C.CDLL(build())
-        _lib.wnwo_create.argtypes = [C.c_int] * 9 + [C.c_double, C.c_double, C.POINTER(C.c_uint8), C.c_int, C.POINTER(C.c_void_p)]
+        _lib.wnwo_create.argtypes = [C.c_int] * 9 + [C.c_double, C.c_double, C.POINTER(C.c_uint8), C.c_int, C.c_int, C.c_int,
+                                     C.POINTER(C.c_void_p)]
         _lib.wnwo_destroy.argtypes = [C.c_void_p]
         _lib.wnwo_destroy.restype = None
         _lib.wnwo_score_source.argtypes = [C.c_void_p, C.c_int]
@@ -62,6 +63,12 @@ def lib():
         _lib.wnwo_get_stats.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_longlong)] * 3
         _lib.wnwo_attention_row.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_uint16),
                                             C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        _lib.wnwo_get_base_slots.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int)]
+        _lib.wnwo_select_segments.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int), C.c_int, C.c_int, C.POINTER(C.c_int),
+                                              C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        _lib.wnwo_lag_update.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_longlong), C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int,
+                                         C.c_longlong, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
+                                         C.POINTER(C.c_int), C.POINTER(C.c_int)]
         _lib.wnwo_topk.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int), C.c_int, C.c_int, C.POINTER(C.c_int)]
         _lib.wnwo_table_update.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_longlong), C.c_int, C.POINTER(C.c_int), C.c_int,
                                            C.c_longlong, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
@@ -101,11 +108,40 @@ def table_update(slot_chunk: np.ndarray, stamp: np.ndarray, sel: Sequence[int], 
     return [(int(pc[i]), int(ps[i]), int(ev[i])) for i in range(n)], hits.value
 
 
+def select_segments(seg_sum: np.ndarray, lens: np.ndarray, k: int):
+    """Overlapping chunks (chunk j = segments j, j+1): the k best chunks in rank order and their segments, in that order
+    without repeats.  Returns (chunks, segments)."""
+    s = np.ascontiguousarray(seg_sum, dtype=np.float32)
+    ln = np.ascontiguousarray(lens, dtype=np.int32)
+    ch = np.full(max(k, 1), -1, dtype=np.int32)
+    sg = np.full(max(2 * k, 1), -1, dtype=np.int32)
+    n_sel = C.c_int(0)
+    n = lib().wnwo_select_segments(_p(s, C.c_float), _p(ln, C.c_int), len(s), k, _p(ch, C.c_int), C.byref(n_sel), _p(sg, C.c_int))
+    if n < 0:
+        raise OracleError("select_segments failed")
+    return ch[:n_sel.value].copy(), sg[:n].copy()
+
+
+def lag_update(slot_seg: np.ndarray, stamp: np.ndarray, s_base: int, segs: Sequence[int], step: int, delta: int):
+    """Apply one segment swap with permanent base slots [0, s_base) and lag-delta release, in place.
+    Returns (plan [(segment, slot)], released segments, n_hits)."""
+    assert slot_seg.dtype == np.int32 and stamp.dtype == np.int64
+    segs = np.ascontiguousarray(segs, dtype=np.int32)
+    n = len(segs)
+    pg = np.zeros(max(n, 1), np.int32); pj = np.zeros(max(n, 1), np.int32); rel = np.zeros(max(len(slot_seg), 1), np.int32)
+    n_rel, hits = C.c_int(0), C.c_int(0)
+    m = lib().wnwo_lag_update(_p(slot_seg, C.c_int), _p(stamp, C.c_longlong), s_base, len(slot_seg), _p(segs, C.c_int), n, step,
+                              delta, _p(pg, C.c_int), _p(pj, C.c_int), _p(rel, C.c_int), C.byref(n_rel), C.byref(hits))
+    if m < 0:
+        raise OracleError("lag_update: no free dynamic slot")
+    return [(int(pg[i]), int(pj[i])) for i in range(m)], [int(x) for x in rel[:n_rel.value]], hits.value
+
+
 class Oracle:
     """The stateful decode-step oracle.  Arrays in/out are numpy; bf16 values travel as uint16 bit patterns."""
 
     def __init__(self, n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
-                 chunk_tokens, topk, budget, roles, softmax_scale=0.0, score_scope=0):
+                 chunk_tokens, topk, budget, roles, softmax_scale=0.0, score_scope=0, residency=0, evict_lag=3):
         self.L, self.Hq, self.Hkv, self.d = n_layers, n_q_heads, n_kv_heads, head_dim
         self.topk_cfg = topk
         roles = np.ascontiguousarray(roles, dtype=np.uint8).reshape(-1)
@@ -114,7 +150,8 @@ class Oracle:
         # budget is a float32 field in the library's config; mirror that rounding here
         _check(lib().wnwo_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
                                  chunk_tokens, topk, float(np.float32(budget)), float(softmax_scale),
-                                 _p(roles, C.c_uint8), score_scope, C.byref(h)), "create")
+                                 _p(roles, C.c_uint8), score_scope, residency, evict_lag, C.byref(h)), "create")
+        self.residency_mode, self.evict_lag = residency, evict_lag
         self.score_scope = score_scope
         self._h = h
         self._n_active = 0
@@ -129,6 +166,12 @@ class Oracle:
             self.close()
         except Exception:
             pass
+
+    def base_slots(self, seq: int) -> int:
+        """Slots of the tidal tables that were filled at prefill (all of them under the hard budget)."""
+        v = C.c_int(0)
+        _check(lib().wnwo_get_base_slots(self._h, seq, C.byref(v)), "get_base_slots")
+        return v.value
 
     def score_source(self, layer: int) -> int:
         return lib().wnwo_score_source(self._h, layer)

@@ -31,10 +31,12 @@ def dense_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float, m
     return p @ V, p
 
 
-def make_oracle(w: Workload, budget: float | None = None, max_batch: int | None = None, score_scope: int = 0):
+def make_oracle(w: Workload, budget: float | None = None, max_batch: int | None = None, score_scope: int = 0,
+                residency: int = 0, evict_lag: int = 3):
     from oracle.wnw_oracle import Oracle
     return Oracle(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, max_batch or w.batch, max(max(w.audio_lens), 1),
-                  w.text_capacity, w.chunk, w.topk, w.budget if budget is None else budget, w.roles, score_scope=score_scope)
+                  w.text_capacity, w.chunk, w.topk, w.budget if budget is None else budget, w.roles, score_scope=score_scope,
+                  residency=residency, evict_lag=evict_lag)
 
 
 def place_all(oracle, syn: Synth, keep: bool = False):

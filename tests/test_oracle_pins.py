@@ -403,3 +403,65 @@ def test_global_scope_sums_all_anchor_layers_and_shares_one_selection():
         o2.decode_layer(l, bf16_bits(dec[l]["q"][0])[None])
     o2.step_end()
     assert o2.selected(0, 3).tolist() == _brute_rank(o2.chunk_scores(0, 2).astype(np.float32), np.full(10, 16))[:3]
+
+
+def test_segment_lag_residency_end_to_end():
+    """Residency SEGMENT_LAG (Chunk Structure + Dynamic Chunk Selection as printed): the paper's n_s = 25-token segments,
+    chunks of two segments; the prefill segments stay for good; a fetched segment is dropped after delta unselected
+    steps.  Checked through the whole oracle: dims, permanent base, selection from the overlapping-chunk means, the
+    dynamic set against the window model, and tidal attention against dense attention masked by the table."""
+    A, T, F = ROLE_ANCHOR, ROLE_TIDAL, ROLE_FIXED
+    delta, k = 2, 2
+    w = tiny_custom(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, n_text=5, audio_lens=(610,), chunk=25, budget=0.2,
+                    roles=[[A, T], [T, F]], n_steps=12, topk=k, region=25, jump_every=3)
+    syn = Synth(w, seed=13)
+    o = make_oracle(w, residency=1, evict_lag=delta)
+    kept = place_all(o, syn, keep=True)
+    T_a, T_t0, C, S = o.dims(0)
+    s_base = o.base_slots(0)
+    assert C == 25 and s_base == 5 and S == s_base + 2 * k * (delta + 1)      # 610 tokens = 24 segments of 25 + one of 10
+    lens = np.array([25] * 24 + [10])
+    base = {l: o.residency(0, l)[0][:s_base].copy() for l in range(2)}
+    assert all((o.residency(0, l)[0][s_base:] == -1).all() for l in range(2))
+    assert len(o.fixed_set(0, 1, 1)) == s_base                                 # fixed heads keep the base amount only
+    dec = {l: syn.decode(0, l) for l in range(2)}
+    scale = 1 / math.sqrt(w.head_dim)
+    history = {0: [], 1: []}
+    moved = 0
+    for t in range(w.n_steps):
+        tables = {l: o.residency(0, l)[0].copy() for l in range(2)}
+        o.step_begin([0])
+        for l in range(2):
+            q = bf16_bits(dec[l]["q"][t])
+            out = o.decode_layer(l, q[None])
+            h = 1 if l == 0 else 0                                             # the tidal head of the layer
+            tK, tV, aK, aV = _split(kept, 0, l, h)
+            vis = np.zeros(C, bool); vis[[c for c in tables[l] if c >= 0]] = True
+            mask = np.concatenate([np.ones(len(tK), bool), np.repeat(vis, w.chunk)[:T_a]])
+            for hq in range(h * 2, h * 2 + 2):
+                ref, _ = dense_attention(bf16_bits_to_f64(q[hq]), np.concatenate([tK, aK]), np.concatenate([tV, aV]), scale, mask)
+                assert np.abs(out[0, hq] - ref).max() < 1e-12
+        o.step_end()
+        sums = o.chunk_scores(0, 0).astype(np.float32)                         # layer 1 routes to layer 0
+        keys = (sums[:-1] + sums[1:]) / (lens[:-1] + lens[1:]).astype(np.float32)
+        want_chunks = sorted(range(C - 1), key=lambda j: (-float(keys[j]), j))[:k]
+        for l in range(2):
+            assert o.selected(0, l).tolist() == want_chunks
+            segs = set()
+            for j in want_chunks:
+                segs |= {j, j + 1}
+            history[l].append(segs)
+            tab = o.residency(0, l)[0]
+            assert tab[:s_base].tolist() == base[l].tolist()
+            window = set().union(*history[l][-delta:]) - set(base[l].tolist())
+            assert set(int(x) for x in tab[s_base:] if x >= 0) == window
+            moved += len(window)
+    assert moved > 0
+    st = o.stats(0)
+    assert st["misses"] > 0 and st["evictions"] > 0
+
+
+def test_segment_lag_rejects_negative_lag():
+    w = config0()
+    with pytest.raises(wo.OracleError):
+        make_oracle(w, residency=1, evict_lag=-1)

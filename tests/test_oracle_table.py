@@ -2,6 +2,7 @@
 import os
 
 import numpy as np
+import pytest
 from hypothesis import given, settings, strategies as st
 
 from oracle import wnw_oracle as wo
@@ -84,3 +85,91 @@ def test_table_update_matches_set_model(data):
         assert (stamp[changed] > last_stamp[changed]).all()         # stamps only grow
         assert len(set(stamp[slot >= 0].tolist())) == len(res)      # and stay unique among residents
         last_stamp = stamp.copy()
+
+
+# ------------------------------------------------------------------ overlapping chunks, permanent base, lag-delta release
+def _parse_lag_trace():
+    rows = []
+    for line in open(os.path.join(os.path.dirname(GOLDEN), "lag_update_trace.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        step, chunk, table, stamps, fetched, released, hits = [x.strip() for x in line.split("|")]
+        rows.append(dict(step=int(step), chunk=int(chunk), table=[int(x) for x in table.split()],
+                         stamps=[None if x == "x" else int(x) for x in stamps.split()],
+                         fetched=[] if fetched == "-" else [tuple(int(y) for y in x.split("->")) for x in fetched.split()],
+                         released=[] if released == "-" else [int(x) for x in released.split()], hits=int(hits)))
+    return rows
+
+
+def test_lag_update_follows_the_hand_worked_trace():
+    """Dynamic Chunk Selection with a permanent prefill base and lag-delta release, against a trace worked by hand."""
+    tab = np.array([0, 4, -1, -1, -1, -1], np.int32)
+    stamp = np.array([-1, -2, 0, 0, 0, 0], np.int64)
+    for row in _parse_lag_trace():
+        segs = [row["chunk"], row["chunk"] + 1]
+        plan, released, hits = wo.lag_update(tab, stamp, 2, segs, row["step"], 2)
+        assert tab.tolist() == row["table"], row
+        assert plan == row["fetched"], row
+        assert sorted(released) == sorted(row["released"]), row
+        assert hits == row["hits"], row
+        for j, want in enumerate(row["stamps"]):
+            if want is not None:
+                assert stamp[2 + j] == want, row
+
+
+def test_select_segments_overlapping_chunks_against_brute_force():
+    """Chunk j = segments j, j+1 ranked by the mean over its tokens (float32), ties to the lower chunk; the segment list
+    is the chunks' segments in rank order without repeats."""
+    rng = np.random.default_rng(5)
+    for trial in range(200):
+        n_seg = int(rng.integers(1, 12))
+        k = int(rng.integers(1, 5))
+        sums = rng.random(n_seg).astype(np.float32)
+        if trial % 5 == 0:
+            sums[:] = np.float32(0.25)          # all ties
+        lens = np.full(n_seg, 25, np.int32)
+        lens[-1] = int(rng.integers(1, 26))     # ragged last segment
+        ch, sg = wo.select_segments(sums, lens, k)
+        n_ch = n_seg - 1 if n_seg > 1 else 1
+        keys = [(np.float32(sums[j] + sums[j + 1]) / np.float32(lens[j] + lens[j + 1])) if n_seg > 1 else sums[0] / np.float32(lens[0])
+                for j in range(n_ch)]
+        order = sorted(range(n_ch), key=lambda j: (-float(keys[j]), j))[:min(k, n_ch)]
+        assert ch.tolist() == order
+        want = []
+        for j in order:
+            for g in ((j, j + 1) if n_seg > 1 else (j,)):
+                if g not in want:
+                    want.append(g)
+        assert sg.tolist() == want
+
+
+@pytest.mark.parametrize("delta", [0, 1, 3])
+def test_lag_update_equals_the_window_set_model(delta):
+    """Independent model: after step s the dynamic set is exactly the union of the segments selected in the last
+    max(delta, 1) steps, minus the base; the plan is what was selected now and was not resident before; the pool of
+    2*k*(delta+1) dynamic slots never overflows; base slots never change."""
+    rng = np.random.default_rng(11 + delta)
+    n_seg, k, s_base = 40, 3, 8
+    D = 2 * k * (delta + 1)
+    base = rng.choice(n_seg, s_base, replace=False).astype(np.int32)
+    tab = np.concatenate([base, np.full(D, -1, np.int32)]).astype(np.int32)
+    stamp = np.zeros(s_base + D, np.int64)
+    history = []
+    for step in range(60):
+        chunks = rng.choice(n_seg - 1, k, replace=False) if step % 7 else np.array([3, 4, 5])   # overlapping chunks too
+        segs = []
+        for j in chunks:
+            for g in (int(j), int(j) + 1):
+                if g not in segs:
+                    segs.append(g)
+        before = set(int(x) for x in tab if x >= 0)
+        plan, released, hits = wo.lag_update(tab, stamp, s_base, segs, step, delta)
+        history.append(set(segs))
+        window = set().union(*history[-max(delta, 1):]) - set(base.tolist())
+        assert set(int(x) for x in tab[s_base:] if x >= 0) == window
+        assert tab[:s_base].tolist() == base.tolist()
+        assert [g for g, _ in plan] == [g for g in segs if g not in before]
+        assert hits == len([g for g in segs if g in before])
+        assert set(released) == (before - set(base.tolist())) - window
+        assert len(set(int(x) for x in tab if x >= 0)) == int((tab >= 0).sum())     # no segment twice
