@@ -142,8 +142,9 @@ class ClockSampler:
 class Job:
     """Caches, resident inputs and launch helpers of one rank."""
 
-    def __init__(self, w, seed, device, wnw, score_scope=0):
+    def __init__(self, w, seed, device, wnw, score_scope=0, residency=0, evict_lag=3):
         self.score_scope = score_scope
+        self.residency, self.evict_lag = residency, evict_lag
         self.w, self.dev, self.wnw = w, device, wnw
         self.syn = Synth(w, seed=seed, device=str(device))
         self.B = w.batch
@@ -174,7 +175,8 @@ class Job:
         w, wnw = self.w, self.wnw
         h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, self.B, max(w.audio_lens), w.text_capacity,
                            w.chunk, w.budget, w.roles, topk=w.topk, device=self.dev.index or 0, mode=mode,
-                           recall_mode=recall_mode, score_scope=self.score_scope)
+                           recall_mode=recall_mode, score_scope=self.score_scope, residency=self.residency,
+                           evict_lag=self.evict_lag)
         self.caches[key] = h
         return h
 
@@ -440,7 +442,10 @@ def run_ours(args, rank, world, local_rank):
     Kb = 0 if (args.quick or args.eager) else min(K, args.back_to_back_steps)
     total = W + R + K + Kb + 2 * Kc
     w = make_workload(args.workload, total, 0)
-    job = Job(w, seed=rank, device=dev, wnw=wnw, score_scope=args.score_scope)
+    if args.segment_tokens > 0:
+        w.chunk = args.segment_tokens
+        w.name += f"_seg{args.segment_tokens}"
+    job = Job(w, seed=rank, device=dev, wnw=wnw, score_scope=args.score_scope, residency=args.residency, evict_lag=args.evict_lag)
     job.create("wnw", wnw.WNW_MODE_FULL if args.quick_full else wnw.WNW_MODE_TIERED, recall_mode=args.recall_mode)
     if args.quick:   # profiler mode: the WnW steps only, nothing else launched
         wnw.wnw_set_layer_dependency(job.caches["wnw"], args.layer_dependency)
@@ -662,7 +667,8 @@ def run_ours(args, rank, world, local_rank):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(w), launch="eager" if args.eager else "cuda graph replay of the step",
-                                                                                score_scope="global" if args.score_scope else "per layer"),
+                                                                                score_scope="global" if args.score_scope else "per layer",
+                                                                                residency="segment lag" if args.residency else "hard budget"),
         "clocks": clocks, "gpu_launches": int(sum(region_launches)),
         "launches": {"attention": region_launches[0], "selection": region_launches[1], "recall": region_launches[2],
                      "step_end": region_launches[3], "layers_per_attention_launch": w.n_layers / attn_per_step},
@@ -718,6 +724,10 @@ def main():
     ap.add_argument("--quick-full", action="store_true", help="with --quick: time the full-cache comparison path instead")
     ap.add_argument("--score-scope", type=int, default=0, choices=[0, 1],
                     help="0: every layer ranks by its own (or the nearest) anchor heads; 1: Eq. 2's sum over all anchor layers")
+    ap.add_argument("--residency", type=int, default=0, choices=[0, 1],
+                    help="0: hard budget (fixed slot pool); 1: SEGMENT_LAG (overlapping two-segment chunks, lag release)")
+    ap.add_argument("--evict-lag", type=int, default=3, help="delta of SEGMENT_LAG")
+    ap.add_argument("--segment-tokens", type=int, default=0, help="override the workload's chunk_tokens (e.g. the paper's 25 / 50)")
     ap.add_argument("--eager", action="store_true", help="issue every layer eagerly instead of replaying a captured step")
     ap.add_argument("--roofline-steps", type=int, default=16)
     ap.add_argument("--layer-dependency", type=int, default=0, choices=[0, 1, 2],

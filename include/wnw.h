@@ -70,6 +70,19 @@ enum { WNW_MODE_TIERED = 0, WNW_MODE_FULL = 1 };
  *              order; every tidal layer takes the same selection, made once the last layer of the step has run */
 enum { WNW_SCOPE_PER_LAYER = 0, WNW_SCOPE_GLOBAL = 1 };
 
+/* How the tidal tables evolve ("Chunk Structure", "Dynamic Chunk Selection").
+ *   HARD_BUDGET  a fixed pool of S = max(1, floor(budget*C)) slots per (sequence, layer); non-overlapping chunks of
+ *                chunk_tokens; a miss takes a free slot, else evicts the least recently selected chunk that is not
+ *                selected now.  evict_lag is not used.
+ *   SEGMENT_LAG  the paper's form: chunk_tokens is the SEGMENT length n_s; a chunk is two consecutive segments, so
+ *                adjacent chunks share one (chunk j = segments j, j+1; ranked by the mean over its tokens; wnw_get_selected
+ *                returns chunk indices).  The S_base = max(1, floor(budget*C)) segments placed at prefill stay resident
+ *                for good; the missing segments of the selected chunks are fetched into 2*topk*(evict_lag+1) further
+ *                slots (never short), and a fetched segment left unselected for evict_lag consecutive steps is dropped
+ *                (its host copy persists).  Fixed heads keep S_base segments.  wnw_get_seq_dims reports all slots;
+ *                wnw_get_base_slots the permanent ones. */
+enum { WNW_RESIDENCY_HARD_BUDGET = 0, WNW_RESIDENCY_SEGMENT_LAG = 1 };
+
 /* How recall copies are issued (for measurement; results are identical for 0 and 1):
  *   0  side stream, overlapped with the following layers (default)
  *   1  on the caller's stream right after the layer (the paper's naive schedule, Limitations section)
@@ -92,6 +105,7 @@ typedef struct {
   int32_t mode;                            /* WNW_MODE_* */
   int32_t recall_mode;                     /* WNW_RECALL_* */
   int32_t score_scope;                     /* WNW_SCOPE_* */
+  int32_t residency;                       /* WNW_RESIDENCY_* */
 } wnw_config_t;
 
 typedef struct {
@@ -191,6 +205,8 @@ wnw_status_t wnw_get_fixed_set(wnw_cache_t *cache, int32_t seq, int32_t layer, i
                                int32_t *n);
 wnw_status_t wnw_get_seq_dims(wnw_cache_t *cache, int32_t seq, int32_t *audio_tokens, int32_t *text_tokens,
                               int32_t *n_chunks, int32_t *n_slots);
+/* Slots of the sequence's tidal tables that hold the prefill placement (all of them under HARD_BUDGET). */
+wnw_status_t wnw_get_base_slots(wnw_cache_t *cache, int32_t seq, int32_t *S_base);
 wnw_status_t wnw_get_slot_kv(wnw_cache_t *cache, int32_t seq, int32_t layer, int32_t kv_head, int32_t slot, int32_t which,
                              void *rows_host);
 wnw_status_t wnw_get_stats(wnw_cache_t *cache, wnw_stats_t *stats_host);

@@ -22,6 +22,7 @@ WNW_MODE_TIERED, WNW_MODE_FULL = 0, 1
 WNW_RECALL_SIDE_STREAM, WNW_RECALL_INLINE, WNW_RECALL_SKIP = 0, 1, 2
 WNW_SCOPE_PER_LAYER, WNW_SCOPE_GLOBAL = 0, 1
 WNW_LAYERS_INDEPENDENT, WNW_LAYERS_CHAINED, WNW_LAYERS_SERIAL = 0, 1, 2
+WNW_RESIDENCY_HARD_BUDGET, WNW_RESIDENCY_SEGMENT_LAG = 0, 1
 
 
 class wnw_config_t(C.Structure):
@@ -29,7 +30,7 @@ class wnw_config_t(C.Structure):
                 ("max_batch", C.c_int32), ("max_audio_tokens", C.c_int32), ("max_text_tokens", C.c_int32),
                 ("chunk_tokens", C.c_int32), ("topk", C.c_int32), ("evict_lag", C.c_int32), ("budget", C.c_float),
                 ("softmax_scale", C.c_float), ("roles", C.POINTER(C.c_uint8)), ("device", C.c_int32), ("mode", C.c_int32),
-                ("recall_mode", C.c_int32), ("score_scope", C.c_int32)]
+                ("recall_mode", C.c_int32), ("score_scope", C.c_int32), ("residency", C.c_int32)]
 
 
 class wnw_stats_t(C.Structure):
@@ -66,6 +67,7 @@ _SIGNATURES = {
     "wnw_get_stats": [_vp, C.POINTER(wnw_stats_t)],
     "wnw_set_layer_dependency": [_vp, _i32],
     "wnw_get_launch_counts": [_vp, C.POINTER(C.c_int64)],
+    "wnw_get_base_slots": [_vp, _i32, C.POINTER(_i32)],
     "wnw_set_kernel_timing": [_vp, _i32],
     "wnw_get_kernel_time": [_vp, C.POINTER(C.c_float), C.POINTER(_i32)],
     "wnw_sync": [_vp],
@@ -124,11 +126,11 @@ def _stream(stream) -> Optional[int]:
 
 def wnw_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens, chunk_tokens,
                budget, roles, topk=3, evict_lag=3, softmax_scale=0.0, device=0, mode=WNW_MODE_TIERED,
-               recall_mode=WNW_RECALL_SIDE_STREAM, score_scope=WNW_SCOPE_PER_LAYER) -> int:
+               recall_mode=WNW_RECALL_SIDE_STREAM, score_scope=WNW_SCOPE_PER_LAYER, residency=WNW_RESIDENCY_HARD_BUDGET) -> int:
     roles = np.ascontiguousarray(roles, dtype=np.uint8).reshape(-1)
     cfg = wnw_config_t(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
                        chunk_tokens, topk, evict_lag, budget, softmax_scale,
-                       roles.ctypes.data_as(C.POINTER(C.c_uint8)), device, mode, recall_mode, score_scope)
+                       roles.ctypes.data_as(C.POINTER(C.c_uint8)), device, mode, recall_mode, score_scope, residency)
     if roles.size != n_layers * n_kv_heads:
         raise WnwError(WNW_ERR_INVALID_ARG, "wnw_create (roles size)")
     h = _vp()
@@ -184,6 +186,12 @@ def wnw_get_seq_dims(cache, seq):
     v = [_i32() for _ in range(4)]
     _ck(lib().wnw_get_seq_dims(cache, seq, *[C.byref(x) for x in v]), "wnw_get_seq_dims")
     return tuple(x.value for x in v)  # T_a, T_t, C, S
+
+
+def wnw_get_base_slots(cache, seq) -> int:
+    v = _i32()
+    _ck(lib().wnw_get_base_slots(cache, seq, C.byref(v)), "wnw_get_base_slots")
+    return v.value
 
 
 def wnw_get_chunk_scores(cache, seq, layer) -> np.ndarray:

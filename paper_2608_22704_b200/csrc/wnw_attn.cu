@@ -108,7 +108,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 struct GranDesc {
   int row;         // first K row of the granule in its store's 2-D view [rows][d] (V row = row + v_delta)
-  int meta;        // >= 0: visible tokens, known statically; -1: text granule, needs the text length; -2: needs `cid`
+  int meta;        // >= 0: visible tokens, known statically; -1: text granule, needs the text length; -2: needs `cid`;
+                   // -3: needs `cid` and is not fetched at all when the slot is empty
   int cid;         // chunk id held by the slot / compact position (filled by a load that is not waited on here)
   int off;         // token offset of the granule inside its chunk
   int score_idx;   // audio granule index for score partials, -1 = none
@@ -139,7 +140,7 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
   } else if (it.role == ROLE_TIDAL) {
     r.row = (int)(pool_off(G, li, it.b, ci, it.ridx, 0) / G.d) + off;
     r.cid = cv.slot_chunk[((long long)it.b * G.L + a.layer) * G.S_max + ci];
-    r.meta = -2;
+    r.meta = ci < it.S ? -2 : -3;   // beyond the permanent slots a slot may be empty: its rows are fetched only if it is not
   } else {
     const long long fh = (long long)it.b * G.F_tot + li.fixed_off + it.ridx;
     r.row = (int)(fixed_off(G, li, it.b, it.ridx, 0) / G.d) + ci * G.ncp + off;
@@ -277,6 +278,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     const bool is_text = j < G.n_tg;
     bool load = meta != 0;
     if (meta == -1) load = visible(c, -1, 0, 0, j) > 0;  // waits for the text length
+    if (meta == -3) load = __shfl_sync(0xffffffffu, blk.cid, src_lane) >= 0;  // waits for the table entry
     if (load && lane == 0) {
       const int stage = (int)(seq % NSTAGE);
       const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB, bar = smem_u32(&bars[warp][stage]);

@@ -32,7 +32,7 @@ struct WorkItem {  // one CTA of the attention kernel; everything static about i
   int32_t role;    // ROLE_* the head plays in this launch
   int32_t ridx;    // index among the heads of that role (anchor-like launches: the KV head)
   int32_t T_a;     // audio tokens of the sequence
-  int32_t C, S;    // chunks and slots of the sequence
+  int32_t C, S;    // chunks of the sequence; its PERMANENT slots (tidal slots from S on may be empty)
   int32_t T_hint;  // text rows known to exist when the list was built (a lower bound: text only grows)
 };
 constexpr int INLINE_ITEMS_MAX = 96;  // launches with at most this many items carry them in kernel parameters
@@ -55,6 +55,7 @@ struct Geometry {
   int32_t T_cap_pad, n_tg;         // text capacity (multiple of 16) and its granules
   int32_t C_max, S_max, T_a_pad;   // chunk / slot capacity per sequence; audio capacity padded to whole chunks
   int32_t A_tot, F_tot;            // anchor / fixed heads per sequence over all layers
+  int32_t lag_mode, delta, plan_cap;  // SEGMENT_LAG residency; its eviction lag; plan entries per (sequence, layer)
   int32_t max_batch;
   long long text_seq_stride, anchor_seq_stride, pool_seq_stride, fixed_seq_stride;  // elements
   float scale_log2;                // softmax scale * log2(e)
@@ -70,14 +71,15 @@ struct CacheView {
   int32_t n_anchor_layers;
   int32_t scope_global;          // tidal layers rank by the sum over all anchor layers (src = -2 in their LayerInfo)
   bf16 *text, *anchor, *pool, *fixed;
-  int32_t *text_len, *T_a, *C, *S;   // [B]
+  int32_t *text_len, *T_a, *C, *S;   // [B]  (S: all slots of a tidal table)
+  int32_t *S_base;                   // [B] slots filled at prefill (= S under the hard budget); what fixed heads keep
   long long *steps;                  // [B]
   int32_t *slot_chunk;               // [B][L][S_max]
   int32_t *chunk_slot;               // [B][L][C_max]
   long long *stamp;                  // [B][L][S_max]
   float *score_sum;                  // [B][L][C_max]
   int32_t *sel, *n_sel;              // [B][L][topk], [B][L]
-  int32_t *plan, *n_plan;            // [B][L][topk][2] (chunk, slot), [B][L]
+  int32_t *plan, *n_plan;            // [B][L][plan_cap][2] (chunk, slot), [B][L]
   int32_t *fixed_chunks, *fixed_n;   // [B][F_tot][S_max], [B][F_tot]
   float *pre;                        // [B][L][Hkv][C_max]
   unsigned long long *stats;         // [B][4] hits, misses, evictions, recall_bytes
@@ -192,7 +194,7 @@ cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *ac
 cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,
                           int skip_copy, RecallSignal sig, cudaStream_t st);
 cudaError_t launch_place_scatter(const CacheView &cv, int b, int layer, const bf16 *k, const bf16 *v, int n_tokens, int ab,
-                                 int ae, int T_t, int C_b, int S_b, bf16 *stage, cudaStream_t st);
+                                 int ae, int T_t, int C_b, int S_b, int S_base, bf16 *stage, cudaStream_t st);
 cudaError_t launch_prefill_select(const CacheView &cv, int b, int layer, const HeadItems *head_items, const float2 *part_ml,
                                   const float2 *gran_em, int n_ag_max, cudaStream_t st);
 cudaError_t launch_place_gather(const CacheView &cv, int b, int layer, int full_mode, const bf16 *stage, int C_b,

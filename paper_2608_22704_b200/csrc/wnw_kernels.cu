@@ -137,7 +137,9 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
         cp_async_commit_wait_all();
         __syncwarp();
       }
-      const int n_copies = select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, src == -2 ? glob_s : (local ? sc_s : w.sc), w);
+      const float *rank_by = src == -2 ? glob_s : (local ? sc_s : w.sc);
+      const int n_copies = G.lag_mode ? select_and_update_lag(cv, b, lt, src, C_b, S_b, cv.S_base[b], T_a, step_b, lane, rank_by, w)
+                                      : select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, rank_by, w);
       if (a.epoch_words && n_copies == 0 && lane == 0) {
         const int prev = atomicAdd(a.empty_ctr + lt, 1);
         if (prev == a.n_active - 1) {   // nothing to recall for this layer in this step: its slots are current
@@ -187,8 +189,8 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
       const int b = active[i];
       const long long bl = (long long)b * G.L + l;
       const int n_plan = cv.n_plan[bl];
-      for (int r = 0; r < n_plan && r < G.topk; ++r) {
-        const int c = cv.plan[(bl * G.topk + r) * 2], slot = cv.plan[(bl * G.topk + r) * 2 + 1];
+      for (int r = 0; r < n_plan && r < G.plan_cap; ++r) {
+        const int c = cv.plan[(bl * G.plan_cap + r) * 2], slot = cv.plan[(bl * G.plan_cap + r) * 2 + 1];
         if (rank == 0 && threadIdx.x == 0) atomicAdd(cv.stats + (long long)b * 4 + 3, (unsigned long long)n * 16ull);
         if (skip_copy) continue;
         copies = true;
@@ -294,13 +296,13 @@ cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *ac
 // (anchor layout [Hkv][K|V][T_a_pad][d]), zero-pads the staging tail, and resets the layer's tables.
 __global__ void __launch_bounds__(256) wnw_place_scatter_kernel(const __grid_constant__ CacheView cv, int b, int layer,
                                                                 const bf16 *k, const bf16 *v, int n_tokens, int ab, int ae,
-                                                                int T_t, int C_b, int S_b, bf16 *stage) {
+                                                                int T_t, int C_b, int S_b, int S_base, bf16 *stage) {
   const Geometry &G = cv.geo;
   const int T_a = ae - ab, vec_per_row = G.d / 8;
   const long long bl = (long long)b * G.L + layer;
   if (blockIdx.x == 0) {
     if (threadIdx.x == 0) {
-      cv.text_len[b] = T_t; cv.T_a[b] = T_a; cv.C[b] = C_b; cv.S[b] = S_b;
+      cv.text_len[b] = T_t; cv.T_a[b] = T_a; cv.C[b] = C_b; cv.S[b] = S_b; cv.S_base[b] = S_base;
       cv.n_sel[bl] = 0; cv.n_plan[bl] = 0;
       if (layer == 0) {
         cv.steps[b] = 0;
@@ -331,8 +333,8 @@ __global__ void __launch_bounds__(256) wnw_place_scatter_kernel(const __grid_con
   }
 }
 cudaError_t launch_place_scatter(const CacheView &cv, int b, int layer, const bf16 *k, const bf16 *v, int n_tokens, int ab,
-                                 int ae, int T_t, int C_b, int S_b, bf16 *stage, cudaStream_t st) {
-  wnw_place_scatter_kernel<<<296, 256, 0, st>>>(cv, b, layer, k, v, n_tokens, ab, ae, T_t, C_b, S_b, stage);
+                                 int ae, int T_t, int C_b, int S_b, int S_base, bf16 *stage, cudaStream_t st) {
+  wnw_place_scatter_kernel<<<296, 256, 0, st>>>(cv, b, layer, k, v, n_tokens, ab, ae, T_t, C_b, S_b, S_base, stage);
   return cudaGetLastError();
 }
 
@@ -344,7 +346,7 @@ __global__ void __launch_bounds__(512) wnw_prefill_select_kernel(const __grid_co
   extern __shared__ float sm[];  // [Hq] M, [Hq] Z, [C_max] keys (as u64 pairs)
   const Geometry &G = cv.geo;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarp = blockDim.x >> 5;
-  const int g = G.g, C_b = cv.C[b], S_b = cv.S[b], T_a = cv.T_a[b];
+  const int g = G.g, C_b = cv.C[b], S_b = cv.S_base[b], T_a = cv.T_a[b];   // the prefill placement fills the permanent slots
   float *sM = sm, *sZ = sm + G.Hq;
   unsigned long long *skey = reinterpret_cast<unsigned long long *>(sm + 2 * G.Hq + (2 * G.Hq & 1));
   const LayerInfo li = cv.layers[layer];

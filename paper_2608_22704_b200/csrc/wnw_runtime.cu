@@ -18,7 +18,7 @@ namespace {
 
 struct SeqHost {
   int placed_layers = 0;
-  int T_a = 0, T_t = 0, C = 0, S = 0;
+  int T_a = 0, T_t = 0, C = 0, S = 0, S_base = 0;   // S: all slots of a tidal table; S_base: the permanent ones
   bf16 *mirror = nullptr;
   size_t mirror_bytes = 0;
 };
@@ -143,6 +143,13 @@ static int slots_for(float budget, int C) {
   if (S > C) S = C;
   return S;
 }
+// All slots of a tidal table: under SEGMENT_LAG the permanent ones plus room for everything selected within the last
+// evict_lag + 1 steps (two segments per chunk), so a miss always finds a free slot.
+static int slots_total(const wnw_config_t &cfg, int C) {
+  const int base = slots_for(cfg.budget, C);
+  if (cfg.residency != WNW_RESIDENCY_SEGMENT_LAG || C <= 0) return base;
+  return base + std::min(2 * cfg.topk * (cfg.evict_lag + 1), C - base);
+}
 
 template <typename T>
 static wnw_status_t dev_alloc(wnw_cache *c, T **p, size_t count, bool zero = true) {
@@ -210,6 +217,7 @@ static wnw_status_t validate_config(const wnw_config_t *cfg) {
   if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return WNW_ERR_INVALID_ARG;
   if (cfg->mode != WNW_MODE_TIERED && cfg->mode != WNW_MODE_FULL) return WNW_ERR_INVALID_ARG;
   if (cfg->score_scope != WNW_SCOPE_PER_LAYER && cfg->score_scope != WNW_SCOPE_GLOBAL) return WNW_ERR_INVALID_ARG;
+  if (cfg->residency != WNW_RESIDENCY_HARD_BUDGET && cfg->residency != WNW_RESIDENCY_SEGMENT_LAG) return WNW_ERR_INVALID_ARG;
   if (cfg->recall_mode < WNW_RECALL_SIDE_STREAM || cfg->recall_mode > WNW_RECALL_SKIP) return WNW_ERR_INVALID_ARG;
   if (cfg->device < 0) return WNW_ERR_INVALID_ARG;
   bool any_anchor = false, any_tidal = false;
@@ -255,7 +263,10 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   G.T_cap_pad = (std::max(cfg->max_text_tokens, 1) + GR - 1) / GR * GR;
   G.n_tg = G.T_cap_pad / GR;
   G.C_max = (cfg->max_audio_tokens + nc - 1) / nc;
-  G.S_max = full ? 0 : slots_for(cfg->budget, G.C_max);
+  G.S_max = full ? 0 : slots_total(c->cfg, G.C_max);
+  G.lag_mode = !full && c->cfg.residency == WNW_RESIDENCY_SEGMENT_LAG;
+  G.delta = c->cfg.evict_lag;
+  G.plan_cap = G.lag_mode ? 2 * G.topk : G.topk;
   G.T_a_pad = std::max(G.C_max, 1) * G.ncp;
   G.max_batch = cfg->max_batch;
   const double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / std::sqrt((double)d);
@@ -327,13 +338,14 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   CKC(dev_alloc(c, &cv.fixed, B * (size_t)G.fixed_seq_stride));
   CKC(dev_alloc(c, &c->stage, (size_t)Hkv * 2 * G.T_a_pad * d));
   CKC(dev_alloc(c, &cv.text_len, B)); CKC(dev_alloc(c, &cv.T_a, B)); CKC(dev_alloc(c, &cv.C, B)); CKC(dev_alloc(c, &cv.S, B));
+  CKC(dev_alloc(c, &cv.S_base, B));
   CKC(dev_alloc(c, &cv.steps, B));
   CKC(dev_alloc(c, &cv.slot_chunk, B * L * std::max(G.S_max, 1)));
   CKC(dev_alloc(c, &cv.chunk_slot, B * L * std::max(G.C_max, 1)));
   CKC(dev_alloc(c, &cv.stamp, B * L * std::max(G.S_max, 1)));
   CKC(dev_alloc(c, &cv.score_sum, B * L * std::max(G.C_max, 1)));
   CKC(dev_alloc(c, &cv.sel, B * L * G.topk)); CKC(dev_alloc(c, &cv.n_sel, B * L));
-  CKC(dev_alloc(c, &cv.plan, B * L * G.topk * 2)); CKC(dev_alloc(c, &cv.n_plan, B * L));
+  CKC(dev_alloc(c, &cv.plan, B * L * G.plan_cap * 2)); CKC(dev_alloc(c, &cv.n_plan, B * L));
   CKC(dev_alloc(c, &cv.fixed_chunks, B * std::max(G.F_tot, 1) * std::max(G.S_max, 1)));
   CKC(dev_alloc(c, &cv.fixed_n, B * std::max(G.F_tot, 1)));
   CKC(dev_alloc(c, &cv.pre, B * L * Hkv * std::max(G.C_max, 1)));
@@ -470,17 +482,21 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
                               std::vector<WorkItem> &items, std::vector<HeadItems> &heads, LayerWork &lw,
                               std::vector<int32_t> &order, std::vector<int32_t> &ranges) {
   const Geometry &G = c->geo;
-  std::vector<int> n_gran(seq_ids.size() * G.Hkv);
+  // n_gran: the head's whole virtual key space (what the items must cover); n_work: the granules expected to hold data
+  // (what the items are sized by): the dynamic slots of a SEGMENT_LAG table are about half empty and cost nothing then
+  std::vector<int> n_gran(seq_ids.size() * G.Hkv), n_work(seq_ids.size() * G.Hkv);
   long long total = 0;
   int longest = 0;
   for (size_t i = 0; i < seq_ids.size(); ++i) {
     const SeqHost &s = c->seqs[seq_ids[i]];
     for (int h = 0; h < G.Hkv; ++h) {
       const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
-      const int audio = (role == ROLE_ANCHOR ? s.C : s.S) * G.gpc;
+      const int audio = (role == ROLE_ANCHOR ? s.C : role == ROLE_TIDAL ? s.S : s.S_base) * G.gpc;
       n_gran[i * G.Hkv + h] = G.n_tg + audio;
-      total += G.n_tg + audio;
-      longest = std::max(longest, G.n_tg + audio);
+      const int work = G.n_tg + audio - (role == ROLE_TIDAL ? (s.S - s.S_base) * G.gpc / 2 : 0);
+      n_work[i * G.Hkv + h] = work;
+      total += work;
+      longest = std::max(longest, work);
     }
   }
   bool throughput = false;
@@ -498,12 +514,13 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
       const int ridx = mode == ATTN_DECODE ? c->role_idx[layer * G.Hkv + h] : h;
       // latency regime: a short head stays in one CTA, which then writes the output itself (no partial, no merge)
-      int n_cta = std::max(1, (n + gpi - 1) / gpi);
-      if (!throughput && n <= c->direct_max_granules) n_cta = 1;
+      const int nw_ = n_work[i * G.Hkv + h];
+      int n_cta = std::max(1, (nw_ + gpi - 1) / gpi);
+      if (!throughput && nw_ <= c->direct_max_granules) n_cta = 1;
       HeadItems hi{(int)items.size() - lw.first_item, n_cta};
       for (int x = 0; x < n_cta; ++x) {  // even contiguous ranges
         const int g0 = (int)((long long)n * x / n_cta), g1 = (int)((long long)n * (x + 1) / n_cta);
-        items.push_back(WorkItem{(int)i, h, g0, g1, seq_ids[i], role, ridx, sq.T_a, sq.C, sq.S, sq.T_t});
+        items.push_back(WorkItem{(int)i, h, g0, g1, seq_ids[i], role, ridx, sq.T_a, sq.C, sq.S_base, sq.T_t});
       }
       heads.push_back(hi);
       lw.max_count = std::max(lw.max_count, hi.count);
@@ -612,7 +629,8 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
   const bool full = c->cfg.mode == WNW_MODE_FULL;
   SeqHost &s = c->seqs[seq];
   if (layer != 0 && (layer != s.placed_layers || T_a != s.T_a || T_t != s.T_t)) return WNW_ERR_STATE;
-  const int C_b = (T_a + G.nc - 1) / G.nc, S_b = full ? 0 : slots_for(c->cfg.budget, C_b);
+  const int C_b = (T_a + G.nc - 1) / G.nc, S_b = full ? 0 : slots_total(c->cfg, C_b);
+  const int S_base_b = full ? 0 : slots_for(c->cfg.budget, C_b);
   if (!full && C_b > 0 && !q_last_dev) return WNW_ERR_INVALID_ARG;
   DeviceGuard guard(c->cfg.device);
   cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -638,7 +656,7 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
       }
       CK(cudaMemcpy(c->cv.mirror + seq, &c->mirror_ptrs[seq], sizeof(bf16 *), cudaMemcpyHostToDevice));
     }
-    s.T_a = T_a; s.T_t = T_t; s.C = C_b; s.S = S_b;
+    s.T_a = T_a; s.T_t = T_t; s.C = C_b; s.S = S_b; s.S_base = S_base_b;
     c->wl_layers.clear();  // dims may have changed
   }
   // the staging buffer and the partial buffers are shared: order after earlier placements and steps
@@ -648,7 +666,7 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
   // chunks start on granule boundaries in every store; the rows between a chunk's last token and the next chunk are zero
   CK(cudaMemsetAsync(c->stage, 0, (size_t)G.Hkv * 2 * G.T_a_pad * G.d * sizeof(bf16), st));
   CK(launch_place_scatter(c->cv, seq, layer, (const bf16 *)k_dev, (const bf16 *)v_dev, n_tokens, audio_begin, audio_end, T_t,
-                          C_b, S_b, c->stage, st));
+                          C_b, S_b, S_base_b, c->stage, st));
   if (!full && C_b > 0) {
     if (c->prefill_seq != seq || c->prefill_T_a != T_a) {
       std::vector<WorkItem> items;
@@ -1178,6 +1196,13 @@ extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
     }
   }
   *out = r;
+  return WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_get_base_slots(wnw_cache_t *c, int32_t seq, int32_t *S_base) {
+  if (!c || !S_base || seq < 0 || seq >= c->geo.max_batch) return WNW_ERR_INVALID_ARG;
+  if (c->seqs[seq].placed_layers == 0) return WNW_ERR_STATE;
+  *S_base = c->seqs[seq].S_base;
   return WNW_OK;
 }
 

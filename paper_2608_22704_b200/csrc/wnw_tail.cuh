@@ -109,7 +109,7 @@ __device__ __forceinline__ int select_and_update(const CacheView &cv, int b, int
     sel[r] = (int)(0xFFFFFFFFu - (unsigned)(best & 0xFFFFFFFFull));
     prev = best;
   }
-  int *plan = cv.plan + bl * G.topk * 2;
+  int *plan = cv.plan + bl * G.plan_cap * 2;
   int n_plan = 0, hits = 0, evictions = 0;
   for (int r = 0; r < k; ++r) {
     const int c = sel[r];
@@ -169,6 +169,111 @@ __device__ __forceinline__ int select_and_update(const CacheView &cv, int b, int
       atomicAdd(cv.stats + (long long)b * 4 + 0, (unsigned long long)hits);
       atomicAdd(cv.stats + (long long)b * 4 + 1, (unsigned long long)n_plan);
       atomicAdd(cv.stats + (long long)b * 4 + 2, (unsigned long long)evictions);
+    }
+  }
+  return n_plan;
+}
+
+// SEGMENT_LAG residency (one warp): chunk j = segments j, j+1 ranked by the mean over its tokens; the segments of the k
+// best chunks, in rank order without repeats, are this step's selection.  Slots [0, S_base) never change.  A selected
+// segment that is resident is a hit (a dynamic one gets stamp = step); then every dynamic slot not selected now with
+// step - stamp >= delta is released; then the misses take the lowest free dynamic slots in order and are planned.
+// Returns the number of planned copies (uniform over the warp).
+__device__ __forceinline__ int select_and_update_lag(const CacheView &cv, int b, int lt, int src, int C_b, int S_b, int S_base,
+                                                      int T_a, long long step, int lane, const float *sc, const SelectWs &w) {
+  const Geometry &G = cv.geo;
+  const long long bl = (long long)b * G.L + lt;
+  const int n_ch = C_b > 1 ? C_b - 1 : C_b;
+  int k = G.topk < n_ch ? G.topk : n_ch;
+  if (src == -1 || C_b <= 0) k = 0;
+  int *slot_chunk = cv.slot_chunk + bl * G.S_max;
+  int *chunk_slot = cv.chunk_slot + bl * G.C_max;
+  long long *stamp = cv.stamp + bl * G.S_max;
+  if (k > 0)
+    for (int j = lane; j < n_ch; j += 32) {
+      const float sum = C_b > 1 ? __fadd_rn(sc[j], sc[j + 1]) : sc[j];
+      const int len = chunk_len(G, T_a, j) + (C_b > 1 ? chunk_len(G, T_a, j + 1) : 0);
+      w.keys[j] = rank_key(sum, len, j);
+    }
+  __syncwarp();
+  int sel[MAX_TOPK];
+  unsigned long long prev = ~0ull;
+  for (int r = 0; r < k; ++r) {
+    unsigned long long best = 0ull;
+    for (int j = lane; j < n_ch; j += 32) {
+      const unsigned long long key = w.keys[j];
+      if (key < prev && key > best) best = key;
+    }
+    best = warp_max_u64(best);
+    sel[r] = (int)(0xFFFFFFFFu - (unsigned)(best & 0xFFFFFFFFull));
+    prev = best;
+  }
+  int segs[2 * MAX_TOPK];
+  int n_seg = 0;
+  for (int r = 0; r < k; ++r)
+    for (int e = 0; e < (C_b > 1 ? 2 : 1); ++e) {
+      const int g = sel[r] + e;
+      bool seen = false;
+      for (int i = 0; i < n_seg; ++i) seen |= segs[i] == g;
+      if (!seen) segs[n_seg++] = g;
+    }
+  // hits
+  unsigned miss = 0;
+  int hits = 0;
+  for (int i = 0; i < n_seg; ++i) {
+    int j = -1;
+    for (int s = lane; s < S_b; s += 32)
+      if (w.slot[s] == segs[i]) j = s;
+    const unsigned hit_mask = __ballot_sync(0xffffffffu, j >= 0);
+    if (!hit_mask) { miss |= 1u << i; continue; }
+    j = __shfl_sync(0xffffffffu, j, __ffs(hit_mask) - 1);
+    ++hits;
+    if (j >= S_base && lane == 0) { w.stamp[j] = step; stamp[j] = step; }
+  }
+  __syncwarp();
+  // release what has gone unselected for delta steps
+  int released = 0;
+  for (int s0 = S_base; s0 < S_b; s0 += 32) {
+    const int s = s0 + lane;
+    bool drop = false;
+    if (s < S_b) {
+      const int rc = w.slot[s];
+      drop = rc >= 0 && w.stamp[s] != step && step - w.stamp[s] >= (long long)G.delta;
+      if (drop) { w.slot[s] = -1; slot_chunk[s] = -1; chunk_slot[rc] = -1; }
+    }
+    released += __popc(__ballot_sync(0xffffffffu, drop));
+  }
+  __syncwarp();
+  // misses, in order, into the lowest free dynamic slots
+  int *plan = cv.plan + bl * G.plan_cap * 2;
+  int n_plan = 0;
+  for (int i = 0; i < n_seg; ++i) {
+    if (!(miss >> i & 1u)) continue;
+    int free_j = 0x7fffffff;
+    for (int s = S_base + lane; s < S_b; s += 32)
+      if (w.slot[s] < 0 && s < free_j) free_j = s;
+    free_j = __reduce_min_sync(0xffffffffu, free_j);
+    if (free_j == 0x7fffffff) {   // cannot happen: 2k(delta+1) dynamic slots always suffice
+      if (lane == 0) atomicOr(cv.status, STATUS_NO_VICTIM);
+      break;
+    }
+    if (lane == 0) {
+      w.slot[free_j] = segs[i]; w.stamp[free_j] = step;
+      slot_chunk[free_j] = segs[i]; chunk_slot[segs[i]] = free_j; stamp[free_j] = step;
+      plan[2 * n_plan] = segs[i];
+      plan[2 * n_plan + 1] = free_j;
+    }
+    ++n_plan;
+    __syncwarp();
+  }
+  if (lane == 0) {
+    for (int r = 0; r < k; ++r) cv.sel[bl * G.topk + r] = sel[r];
+    cv.n_sel[bl] = k;
+    cv.n_plan[bl] = n_plan;
+    if (k > 0) {
+      atomicAdd(cv.stats + (long long)b * 4 + 0, (unsigned long long)hits);
+      atomicAdd(cv.stats + (long long)b * 4 + 1, (unsigned long long)n_plan);
+      atomicAdd(cv.stats + (long long)b * 4 + 2, (unsigned long long)released);
     }
   }
   return n_plan;

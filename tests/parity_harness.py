@@ -49,16 +49,17 @@ def near_tie(scores64, lens, sel_a, sel_b):
 
 class Lockstep:
     def __init__(self, w: Workload, seed=0, device="cuda:0", recall_mode=0, gen_device=None, oracle_seqs=None,
-                 score_scope=0):
+                 score_scope=0, residency=0, evict_lag=3):
         self.w = w
         self.dev = torch.device(device)
         self.syn = Synth(w, seed=seed, device=gen_device or "cpu")
         self.oracle_seqs = list(range(w.batch)) if oracle_seqs is None else list(oracle_seqs)
         self.scope = score_scope
-        self.o = make_oracle(w, score_scope=score_scope)
+        self.residency, self.evict_lag = residency, evict_lag
+        self.o = make_oracle(w, score_scope=score_scope, residency=residency, evict_lag=evict_lag)
         self.h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max(max(w.audio_lens), 0),
                                 w.text_capacity, w.chunk, w.budget, w.roles, topk=w.topk, device=self.dev.index or 0,
-                                recall_mode=recall_mode, score_scope=score_scope)
+                                recall_mode=recall_mode, score_scope=score_scope, residency=residency, evict_lag=evict_lag)
         self.kept = {}
         self.near_ties = 0
         self.max_out_err = 0.0
@@ -93,6 +94,8 @@ class Lockstep:
             if C == 0:
                 continue
             lens = chunk_lens(T_a, w.chunk)
+            S_all, S = S, wnw.wnw_get_base_slots(self.h, b)      # the prefill placement fills the permanent slots
+            assert S == self.o.base_slots(b)
             for l in range(w.n_layers):
                 tid_sum = np.zeros(C, np.float32)
                 any_tid = False
@@ -115,12 +118,12 @@ class Lockstep:
                 if any_tid:
                     g_tab, g_stamp = wnw.wnw_get_residency(self.h, b, l)
                     want = wo.topk(tid_sum, lens, S)
-                    assert g_tab.tolist() == want.tolist(), f"tidal table (ii) b{b} l{l}"
-                    assert g_stamp.tolist() == [-1 - r for r in range(S)]
+                    assert g_tab.tolist() == want.tolist() + [-1] * (S_all - S), f"tidal table (ii) b{b} l{l}"
+                    assert g_stamp.tolist() == [-1 - r for r in range(S)] + [0] * (S_all - S)
                     o_tab, o_stamp = self.o.residency(b, l)
                     if g_tab.tolist() != o_tab.tolist():
                         o_sum = sum(self.o.prefill_scores(b, l, h) for h in range(w.n_kv_heads) if w.roles[l, h] == ROLE_TIDAL)
-                        assert near_tie(o_sum, lens, g_tab.tolist(), o_tab.tolist())
+                        assert near_tie(o_sum, lens, g_tab[:S].tolist(), o_tab[:S].tolist())
                         self.near_ties += 1
                         self.o.set_residency(b, l, g_tab, g_stamp)
                     if check_slots:
@@ -244,10 +247,17 @@ class Lockstep:
                 g_sel = wnw.wnw_get_selected(self.h, b, l)
                 g_tab, g_stamp = wnw.wnw_get_residency(self.h, b, l)
                 # (ii) oracle logic on GPU scores and the GPU's previous table
-                want_sel = wo.topk(rank_g, lens, k)
-                assert g_sel.tolist() == want_sel.tolist(), f"selection (ii) step {t} b{b} l{l}"
                 tab, stamp = prev_tab[(b, l)][0].copy(), prev_tab[(b, l)][1].copy()
-                plan, _ = wo.table_update(tab, stamp, want_sel, steps_before[b], w.topk)
+                if self.residency == 1:   # overlapping chunks, permanent base, lag-delta release
+                    want_sel, segs = wo.select_segments(rank_g, lens, w.topk)
+                    assert g_sel.tolist() == want_sel.tolist(), f"selection (ii) step {t} b{b} l{l}"
+                    plan, _, _ = wo.lag_update(tab, stamp, wnw.wnw_get_base_slots(self.h, b), segs, steps_before[b], self.evict_lag)
+                    if C > 1:                  # the ranking the near-tie check looks at: chunk sums and lengths
+                        rank_o, lens_tie = rank_o[:-1] + rank_o[1:], lens[:-1] + lens[1:]
+                else:
+                    want_sel = wo.topk(rank_g, lens, k)
+                    assert g_sel.tolist() == want_sel.tolist(), f"selection (ii) step {t} b{b} l{l}"
+                    plan, _ = wo.table_update(tab, stamp, want_sel, steps_before[b], w.topk)
                 n_tid = int((w.roles[l] == ROLE_TIDAL).sum())
                 self.expected_recall_bytes += len(plan) * n_tid * 2 * (-(-w.chunk // 16) * 16) * w.head_dim * 2   # blocks are stored padded to 16 rows
                 assert g_tab.tolist() == tab.tolist(), f"table (ii) step {t} b{b} l{l}"
@@ -256,7 +266,7 @@ class Lockstep:
                 o_sel = self.o.selected(b, l)
                 o_tab, o_stamp = self.o.residency(b, l)
                 if o_sel.tolist() != g_sel.tolist() or o_tab.tolist() != g_tab.tolist() or o_stamp.tolist() != g_stamp.tolist():
-                    assert near_tie(rank_o, lens, g_sel.tolist(), o_sel.tolist()), \
+                    assert near_tie(rank_o, lens_tie if self.residency == 1 and C > 1 else lens, g_sel.tolist(), o_sel.tolist()), \
                         f"selection differs beyond a near-tie, step {t} b{b} l{l}: gpu {g_sel} oracle {o_sel}"
                     self.near_ties += 1
                     self.o.set_residency(b, l, g_tab, g_stamp)
