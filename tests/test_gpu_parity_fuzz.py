@@ -43,3 +43,22 @@ def test_random_configuration(seed):
         ls.check_stats()
     finally:
         ls.close()
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_configuration_segment_lag(seed):
+    """The same random shapes under SEGMENT_LAG residency with a random eviction lag, score scope and layer ordering."""
+    import paper_2608_22704_b200 as wnw
+    from parity_harness import Lockstep
+    w, rs = _draw(seed)
+    delta = int(rs.randint(0, 4))
+    ls = Lockstep(w, seed=seed, residency=wnw.WNW_RESIDENCY_SEGMENT_LAG, evict_lag=delta, score_scope=int(rs.randint(0, 2)))
+    try:
+        wnw.wnw_set_layer_dependency(ls.h, int(rs.randint(0, 3)))
+        ls.prefill()
+        use_graph = bool(seed % 2)
+        for t in range(w.n_steps):
+            ls.decode_step(t, append=True, graph=use_graph and t not in (0, 3), check_slots=True)
+        ls.check_stats()
+    finally:
+        ls.close()
