@@ -317,6 +317,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   load_ctx(prod, qi);
   const WorkItem &it = prod.it;
   const int item_idx = prod.item_idx;
+  if (cv.step_snap && it.h == 0 && it.g0 == 0 && threadIdx.x == 0 && a.mode != ATTN_PREFILL)   // (no cache state behind the
+    cv.step_snap[(long long)it.b * G.L + a.layer] = cv.steps[it.b];                            //  allocation-free entry)
   const int b = it.b, ridx = it.ridx, T_t = prod.T_t;
   const int first = prod.first, n_my = prod.n_my;
 #ifdef WNW_PHASE_STAMPS

@@ -74,6 +74,8 @@ struct CacheView {
   int32_t *text_len, *T_a, *C, *S;   // [B]  (S: all slots of a tidal table)
   int32_t *S_base;                   // [B] slots filled at prefill (= S under the hard budget); what fixed heads keep
   long long *steps;                  // [B]
+  long long *step_snap;              // [B][L] the step index as the layer's attention kernel saw it: what the layer's
+                                     // selection kernel stamps with (the step-end update may overtake that kernel)
   int32_t *slot_chunk;               // [B][L][S_max]
   int32_t *chunk_slot;               // [B][L][C_max]
   long long *stamp;                  // [B][L][S_max]
@@ -183,7 +185,8 @@ struct RecallSignal {
   int32_t *epoch_words;       // [L] epoch of the last completed recall of each layer's table
   int32_t *counters;          // [L] finished-CTA counters (self-resetting)
   int32_t *empty_ctr;         // [L] the selection kernels' empty-plan counters, reset here
-  const int32_t *step_epoch;  // epoch to publish: the number of replayed steps that have ended
+  int32_t publish_epoch;      // epoch to publish: the number of replayed steps that have ended with this one (the host counts
+                              // them; the device word may already be further when this kernel runs late)
 };
 
 // kernels' host launchers (defined in the .cu files)

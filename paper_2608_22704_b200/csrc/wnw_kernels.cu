@@ -19,7 +19,8 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
   const LayerInfo &li = a.li;
   // per-sequence scalars: one batch of independent loads
   const int C_b = cv.C[b], S_b = cv.S[b], T_a = cv.T_a[b];
-  const long long step_b = cv.steps[b];
+  const long long step_b = cv.step_snap[(long long)b * G.L + a.layer];   // not cv.steps: an eager step's bookkeeping kernel
+                                                                         // follows the attention kernel, not this one
   const int n_aq = a.n_aq;
   const bool scored = li.n_anchor > 0 && a.score_on && C_b > 0;
   // shared-memory layout: (M,Z) of the anchor q-heads | this layer's scores | per-warp update workspaces | granule partials
@@ -182,6 +183,13 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
   const int stride = cpg * blockDim.x;
   for (int x = grp; x < n_layers; x += n_groups) {
     const int l = layers[x];
+    if (sig.epoch_words) {
+      // Already published for this step (by the selection kernel: no sequence planned a copy for this layer).  Its
+      // plans must not be read then: the next step's selection may be rewriting them by now.
+      int seen;
+      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];\n" : "=r"(seen) : "l"(sig.epoch_words + l) : "memory");
+      if (seen >= sig.publish_epoch) continue;
+    }
     const LayerInfo &li = cv.layers[l];
     const int n = li.n_tidal * 2 * G.ncp * G.d / 8;  // 16-byte vectors per chunk block (far below 2^31)
     bool copies = false;                             // uniform over the whole grid: the plans do not change under this kernel
@@ -219,8 +227,7 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
       // nothing was written for this layer: its epoch goes out at once, without the round of fences and counting
       if (rank == 0 && threadIdx.x == 0) {
         sig.empty_ctr[l] = 0;
-        const int epoch = *sig.step_epoch;
-        asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(sig.epoch_words + l), "r"(epoch) : "memory");
+        asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(sig.epoch_words + l), "r"(sig.publish_epoch) : "memory");
       }
     } else if (sig.epoch_words) {  // completion of this layer's recall: counted per CTA, published by the last one
       __threadfence();
@@ -231,8 +238,7 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
           sig.counters[l] = 0;
           sig.empty_ctr[l] = 0;
           __threadfence();
-          const int epoch = *sig.step_epoch;
-          asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(sig.epoch_words + l), "r"(epoch) : "memory");
+          asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(sig.epoch_words + l), "r"(sig.publish_epoch) : "memory");
         }
       }
     }

@@ -100,6 +100,7 @@ struct wnw_cache {
   bool fold_enabled = true, cap_fold = false;   // captured steps: the last selection CTA closes the step
   int n_side_layers = 0;
   int32_t *d_fold_ctr = nullptr, *d_empty_ctr = nullptr;
+  int32_t host_epoch = 0;   // replayed steps with out-of-graph recall so far = the value of the device's step epoch after them
   long long launches[4] = {0, 0, 0, 0}, cap_launches[4] = {0, 0, 0, 0};  // attention, selection, recall, step-end kernels
   void count_launch(int kind, int n, bool capturing) { (capturing ? cap_launches : launches)[kind] += n; }
   int layer_dependency = WNW_LAYERS_INDEPENDENT;
@@ -340,6 +341,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   CKC(dev_alloc(c, &cv.text_len, B)); CKC(dev_alloc(c, &cv.T_a, B)); CKC(dev_alloc(c, &cv.C, B)); CKC(dev_alloc(c, &cv.S, B));
   CKC(dev_alloc(c, &cv.S_base, B));
   CKC(dev_alloc(c, &cv.steps, B));
+  CKC(dev_alloc(c, &cv.step_snap, B * L));
   CKC(dev_alloc(c, &cv.slot_chunk, B * L * std::max(G.S_max, 1)));
   CKC(dev_alloc(c, &cv.chunk_slot, B * L * std::max(G.C_max, 1)));
   CKC(dev_alloc(c, &cv.stamp, B * L * std::max(G.S_max, 1)));
@@ -884,7 +886,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     c->count_launch(1, 1, capturing);
     if (li.upd_count > 0 && !c->cap_external_recall) {
       CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count,
-                       c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{nullptr, nullptr, nullptr, nullptr}, ss));
+                       c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{nullptr, nullptr, nullptr, 0}, ss));
       c->count_launch(2, 1, capturing);
     }
     if (!inline_mode) {
@@ -1010,12 +1012,13 @@ extern "C" wnw_status_t wnw_graph_launch(wnw_cache_t *c, void *cuda_stream) {
   CK(cudaGraphLaunch(c->graph_exec, st));
   for (int k = 0; k < 4; ++k) c->launches[k] += c->cap_launches[k];  // the kernels of the captured step
   if (c->graph_external_recall && !c->upd_list.empty()) {
+    ++c->host_epoch;
     // This step's recall, for every layer's table at once, outside the graph: it overlaps the next replay, whose tidal
     // CTAs wait on the per-layer epoch words it publishes.
     CK(cudaEventRecord(c->ev_graph_done, st));
     CK(cudaStreamWaitEvent(c->side[0], c->ev_graph_done, 0));
     CK(launch_recall(c->cv, (int)c->graph_active.size(), c->d_active, c->cv.upd_list, (int)c->upd_list.size(),
-                     c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{c->d_recall_epoch, c->d_recall_ctr, c->d_empty_ctr, c->d_step_epoch},
+                     c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{c->d_recall_epoch, c->d_recall_ctr, c->d_empty_ctr, c->host_epoch},
                      c->side[0]));
     c->count_launch(2, 1, false);
     CK(cudaEventRecord(c->ev_recall_all, c->side[0]));

@@ -11,11 +11,11 @@ from workloads import ROLE_ANCHOR, ROLE_TIDAL, Synth, config1, config4
 pytestmark = pytest.mark.gpu
 
 
-def _run(w, drained, n_steps, dependency=0, score_scope=0):
+def _run(w, drained, n_steps, dependency=0, score_scope=0, eager_steps=(), residency=0):
     dev = torch.device("cuda:0")
     syn = Synth(w, seed=3, device="cuda:0")
     h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max(w.audio_lens), w.text_capacity,
-                       w.chunk, w.budget, w.roles, topk=w.topk, score_scope=score_scope)
+                       w.chunk, w.budget, w.roles, topk=w.topk, score_scope=score_scope, residency=residency, evict_lag=2)
     try:
         wnw.wnw_set_layer_dependency(h, dependency)
         for b in range(w.batch):
@@ -45,7 +45,13 @@ def _run(w, drained, n_steps, dependency=0, score_scope=0):
         with torch.cuda.stream(st):
             for t in range(n_steps):
                 sq.copy_(q[t]); skn.copy_(kn[t]); svn.copy_(vn[t])
-                wnw.wnw_graph_launch(h, st)
+                if t in eager_steps:       # an eager step between replays, on the same stream, still without host sync
+                    wnw.wnw_step_begin(h, act)
+                    for l in range(w.n_layers):
+                        wnw.wnw_decode_layer(h, l, sq[l], skn[l], svn[l], out[l], stream=st)
+                    wnw.wnw_step_end(h, stream=st)
+                else:
+                    wnw.wnw_graph_launch(h, st)
                 outs.append(out.clone())
                 if drained:
                     wnw.wnw_sync(h)
@@ -60,7 +66,11 @@ def _run(w, drained, n_steps, dependency=0, score_scope=0):
 
 def _same(a, b):
     for t, (x, y) in enumerate(zip(a[0], b[0])):
-        assert torch.equal(x, y), f"outputs differ at step {t}"
+        if not torch.equal(x, y):
+            d = (x.float() - y.float()).abs()
+            where = [(l, b, h) for l in range(x.shape[0]) for b in range(x.shape[1]) for h in range(x.shape[2])
+                     if d[l, b, h].max() > 0]
+            raise AssertionError(f"outputs differ at step {t}: max abs {d.max().item():.4g}, (layer, seq, q head) {where[:12]}")
     for (t1, s1), (t2, s2) in zip(a[1], b[1]):
         assert np.array_equal(t1, t2) and np.array_equal(s1, s2)
     assert a[2] == b[2]
@@ -91,3 +101,19 @@ def test_undrained_replays_match_drained_chained_and_serial(dependency):
     w = config4(budget=0.2, chunk=64, batch=2, n_steps=8)
     w.n_layers = 6; w.roles = w.roles[:6]
     _same(_run(w, True, 8, dependency=dependency), _run(w, False, 8, dependency=dependency))
+
+
+@pytest.mark.parametrize("residency", [0, 1])
+def test_undrained_mix_of_eager_steps_and_replays(residency):
+    """Eager steps in between replays on the same stream, nothing drained: the eager step waits for the pending
+    out-of-graph recall, the next replay for the eager step's side streams."""
+    w = config4(budget=0.2, chunk=25 if residency else 64, batch=2, n_steps=12)
+    w.n_layers = 6; w.roles = w.roles[:6]
+    a = _run(w, True, 12, eager_steps=(3, 4, 8), residency=residency)
+    b = _run(w, False, 12, eager_steps=(3, 4, 8), residency=residency)
+    _same(a, b)
+    c = _run(w, False, 12, residency=residency)          # and the mix gives what pure replay gives
+    for t, (x, y) in enumerate(zip(a[0], c[0])):
+        assert torch.equal(x, y), (f"eager/replay mix differs from pure replay at step {t}: max abs "
+                                   f"{(x.float() - y.float()).abs().max().item():.4g}, layers "
+                                   f"{[l for l in range(w.n_layers) if not torch.equal(x[l], y[l])]}")
