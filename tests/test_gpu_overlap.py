@@ -117,3 +117,15 @@ def test_undrained_mix_of_eager_steps_and_replays(residency):
         assert torch.equal(x, y), (f"eager/replay mix differs from pure replay at step {t}: max abs "
                                    f"{(x.float() - y.float()).abs().max().item():.4g}, layers "
                                    f"{[l for l in range(w.n_layers) if not torch.equal(x[l], y[l])]}")
+
+
+@pytest.mark.parametrize("dependency,residency", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_undrained_replays_large_launches(dependency, residency):
+    """Launches too large for the out-of-graph recall (recall stays inside the captured step); chained layers run the
+    persistent schedule.  Eager steps mixed in."""
+    w = config4(budget=0.1, chunk=25 if residency else 64, batch=12, n_steps=8)
+    w.n_layers = 4; w.roles = w.roles[:4]
+    a = _run(w, True, 8, dependency=dependency, residency=residency, eager_steps=(2, 5))
+    b = _run(w, False, 8, dependency=dependency, residency=residency, eager_steps=(2, 5))
+    _same(a, b)
+    assert b[3][2] > 8      # recall launches per layer, not one per step
