@@ -191,7 +191,8 @@ struct RecallSignal {
 
 // kernels' host launchers (defined in the .cu files)
 cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st);
-cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, cudaStream_t st);
+// groups: CTAs per sequence (a layer that updates many tables, e.g. the last one under the global score scope)
+cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, int groups, cudaStream_t st);
 cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *active, int appended, int32_t *bump_epoch,
                             cudaStream_t st);
 cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,

@@ -81,9 +81,11 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
     if (threadIdx.x < n_aq) cp_async_small(mz_s + threadIdx.x, a.head_mz + (long long)i * G.Hq + a.aq_head[threadIdx.x], 8);
     stage_em(0, tile_c);
   }
-  if (warp < n_par) {
+  // the tables to update are dealt out over the CTAs of the sequence (grid y), then over the warps of a CTA
+  const int u_first = (int)blockIdx.y * n_par + warp, u_step = (int)gridDim.y * n_par;
+  if (warp < n_par && u_first < li.upd_count) {
     int lt, src;
-    upd_of(warp, lt, src);
+    upd_of(u_first, lt, src);
     select_stage(cv, b, lt, src, scored && src == a.layer, C_b, S_b, lane, select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b));
   }
   cp_async_commit_wait_all();
@@ -128,11 +130,11 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
   }
   if (warp < n_par) {
     const SelectWs w = select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b);
-    for (int u = warp; u < li.upd_count; u += n_par) {
+    for (int u = u_first; u < li.upd_count; u += u_step) {
       int lt, src;
       upd_of(u, lt, src);
       const bool local = (scored && src == a.layer) || src == -2;
-      if (u >= n_par) {  // later rounds stage their own tables
+      if (u != u_first) {  // later rounds stage their own tables
         __syncwarp();
         select_stage(cv, b, lt, src, local, C_b, S_b, lane, w);
         cp_async_commit_wait_all();
@@ -159,8 +161,8 @@ cudaError_t configure_select_kernel() {
   return cudaFuncSetAttribute(wnw_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM_CAP);
 }
 
-cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, cudaStream_t st) {
-  wnw_select_kernel<<<a.n_active, SEL_WARPS * 32, smem_bytes, st>>>(cv, a, (int)smem_bytes);
+cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, int groups, cudaStream_t st) {
+  wnw_select_kernel<<<dim3(a.n_active, groups), SEL_WARPS * 32, smem_bytes, st>>>(cv, a, (int)smem_bytes);
   return cudaGetLastError();
 }
 

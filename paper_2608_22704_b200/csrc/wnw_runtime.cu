@@ -98,7 +98,7 @@ struct wnw_cache {
   bool step_capturing = false;
   bool pdl_enabled = true;
   bool fold_enabled = true, cap_fold = false;   // captured steps: the last selection CTA closes the step
-  int n_side_layers = 0;
+  int n_side_layers = 0, n_select_ctas = 0;   // layers with a selection kernel; its CTAs per sequence over all layers
   int32_t *d_fold_ctr = nullptr, *d_empty_ctr = nullptr;
   int32_t host_epoch = 0;   // replayed steps with out-of-graph recall so far = the value of the device's step epoch after them
   long long launches[4] = {0, 0, 0, 0}, cap_launches[4] = {0, 0, 0, 0};  // attention, selection, recall, step-end kernels
@@ -136,6 +136,9 @@ struct wnw_cache {
       return _e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA; \
     }                                            \
   } while (0)
+
+// CTAs per sequence of a layer's selection kernel: one per eight tables to update.
+static int select_groups(const LayerInfo &li) { return std::max(1, std::min(8, (li.upd_count + 7) / 8)); }
 
 static int slots_for(float budget, int C) {
   if (C <= 0) return 0;
@@ -423,7 +426,10 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   CKC(dev_alloc(c, &c->d_fold_ctr, 1));
   CKC(dev_alloc(c, &c->d_empty_ctr, (size_t)L));
   for (int l = 0; l < L; ++l)
-    if (!full && (c->layers[l].n_anchor > 0 || c->layers[l].upd_count > 0)) ++c->n_side_layers;
+    if (!full && (c->layers[l].n_anchor > 0 || c->layers[l].upd_count > 0)) {
+      ++c->n_side_layers;
+      c->n_select_ctas += select_groups(c->layers[l]);
+    }
   CKE(cudaDeviceSynchronize());
 #undef CKC
 #undef CKE
@@ -852,7 +858,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     sa.layer = layer; sa.n_active = n_active; sa.score_on = a.score_on; sa.li = li; sa.active = c->d_active;
     sa.gran_em = gran_em_l; sa.head_mz = head_mz_l; sa.n_aq = a.n_aq; sa.n_ag_max = a.n_ag_max;
     if (c->cap_fold) {
-      sa.fold_total = c->n_side_layers * n_active; sa.fold_appended = has_new; sa.fold_counter = c->d_fold_ctr;
+      sa.fold_total = c->n_select_ctas * n_active; sa.fold_appended = has_new; sa.fold_counter = c->d_fold_ctr;
       sa.fold_bump_epoch = c->cap_external_recall ? c->d_step_epoch : nullptr;
     }
     if (c->cap_external_recall && c->cap_fold) {   // the epoch arithmetic relies on the bump coming after every selection
@@ -882,7 +888,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
           if (al != layer && al % wnw_cache::N_SIDE != si)
             CK(cudaStreamWaitEvent(ss, capturing ? c->ev_side_done_cap[al] : c->ev_side_done[al], 0));
     }
-    CK(launch_select(c->cv, sa, c->sel_smem[layer], ss));
+    CK(launch_select(c->cv, sa, c->sel_smem[layer], select_groups(li), ss));
     c->count_launch(1, 1, capturing);
     if (li.upd_count > 0 && !c->cap_external_recall) {
       CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count,
