@@ -524,7 +524,8 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       // latency regime: a short head stays in one CTA, which then writes the output itself (no partial, no merge)
       const int nw_ = n_work[i * G.Hkv + h];
       int n_cta = std::max(1, (nw_ + gpi - 1) / gpi);
-      if (!throughput && nw_ <= c->direct_max_granules) n_cta = 1;
+      // a short head stays in one CTA; twice as long when layers overlap (work per launch counts, not the kernel's span)
+      if (!throughput && nw_ <= (overlapped ? 2 : 1) * c->direct_max_granules) n_cta = 1;
       HeadItems hi{(int)items.size() - lw.first_item, n_cta};
       for (int x = 0; x < n_cta; ++x) {  // even contiguous ranges
         const int g0 = (int)((long long)n * x / n_cta), g1 = (int)((long long)n * (x + 1) / n_cta);
