@@ -61,3 +61,38 @@ def test_config1_sixty_four_steps_graph_replay():
         assert st["misses"] > 100 and st["evictions"] > 100      # the sweep really exercises recall and eviction
     finally:
         ls.close()
+
+
+@pytest.mark.parametrize("residency,seg,scope", [(0, 64, 0), (1, 50, 0), (1, 50, 1)])
+def test_config2_graph_replay(residency, seg, scope):
+    """3B Qwen-Omni-shaped stack at full size (36 layers, 16q/2kv, g = 8, 15000 audio tokens = a 10-minute clip, layers
+    without anchors routed to the nearest anchor layer) under graph replay: the contract's chunk-64 hard budget, and the
+    paper's form for this tokeniser rate (50-token segments, chunks of two, lag-3 release), per-layer and global scores."""
+    from parity_harness import Lockstep
+    from workloads import config2
+    w = config2(n_steps=6)
+    w.chunk = seg
+    ls = Lockstep(w, seed=0, gen_device="cuda:0", residency=residency, evict_lag=3, score_scope=scope)
+    try:
+        ls.prefill(check_slots=False)
+        for t in range(6):
+            ls.decode_step(t, graph=t >= 1, check_slots=(t == 5))
+        ls.check_stats()
+    finally:
+        ls.close()
+
+
+def test_config3_batch32_segment_lag_sampled_sequences():
+    """Batch 32 ragged in the paper's form (25-token segments, lag release): one CTA per head, recall inside the step."""
+    w = config3(n_steps=3)
+    w.chunk = 25
+    lens = np.array(w.audio_lens)
+    from parity_harness import Lockstep
+    ls = Lockstep(w, seed=0, gen_device="cuda:0", oracle_seqs=sorted({int(lens.argmin()), int(lens.argmax())}),
+                  residency=1, evict_lag=3)
+    try:
+        ls.prefill(check_slots=False)
+        for t in range(3):
+            ls.decode_step(t, graph=True, check_slots=(t == 2))
+    finally:
+        ls.close()
