@@ -456,7 +456,7 @@ extern "C" wnw_status_t wnw_destroy(wnw_cache_t *c) {
 // persistent schedule on the batched workloads: 77 % vs 71 % and 85 % vs 82 % of the copy bandwidth.
 //
 // Layers that wait for one another (chained or serial): the span of one kernel counts.  Little work (fits one wave of
-// CTAs): the smallest useful items, so every byte is in flight at once.  Otherwise persistent 4-warp CTAs, two per
+// CTAs): small items (two granules per warp), so nearly every byte is in flight at once and the merge stays short.  Otherwise persistent 4-warp CTAs, two per
 // SM, over items sized for about one item per CTA and placed longest-first by the host.
 static int granules_per_item(const wnw_cache *c, long long total_granules, int longest_head, int n_heads, bool overlapped,
                              bool *throughput) {
@@ -470,7 +470,7 @@ static int granules_per_item(const wnw_cache *c, long long total_granules, int l
     per = std::max<long long>(per, (total_granules + cap - 1) / cap);
     return (int)((per + nw - 1) / nw * nw);
   }
-  long long per = std::max<long long>(min_gpi, (longest_head + 31) / 32);
+  long long per = std::max<long long>(2 * min_gpi, (longest_head + 31) / 32);   // two granules per warp: fewer partials to merge
   per = (per + nw - 1) / nw * nw;
   *throughput = (total_granules + per - 1) / per + n_heads > c->n_sm;
   if (const char *e = getenv("WNW_THROUGHPUT")) *throughput = atoi(e) != 0;
@@ -524,8 +524,9 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       // latency regime: a short head stays in one CTA, which then writes the output itself (no partial, no merge)
       const int nw_ = n_work[i * G.Hkv + h];
       int n_cta = std::max(1, (nw_ + gpi - 1) / gpi);
-      // a short head stays in one CTA; twice as long when layers overlap (work per launch counts, not the kernel's span)
-      if (!throughput && nw_ <= (overlapped ? 2 : 1) * c->direct_max_granules) n_cta = 1;
+      // a short head stays in one CTA: up to 128 granules when layers overlap (work per launch counts), 32 when the
+      // kernel's span counts (measured, chained config 1: 298 -> 240 us per step against a threshold of 64)
+      if (!throughput && nw_ <= (overlapped ? 2 * c->direct_max_granules : c->direct_max_granules / 2)) n_cta = 1;
       HeadItems hi{(int)items.size() - lw.first_item, n_cta};
       for (int x = 0; x < n_cta; ++x) {  // even contiguous ranges
         const int g0 = (int)((long long)n * x / n_cta), g1 = (int)((long long)n * (x + 1) / n_cta);
