@@ -219,7 +219,8 @@ wnw_status_t wnw_get_stats(wnw_cache_t *cache, wnw_stats_t *stats_host);
  *                on that work, but waits for the predecessor to complete before it reads q, k_new or v_new.
  *   SERIAL       plain stream order, no early start.
  * Takes effect for layers issued afterwards; a captured step keeps the mode it was captured with.  Not allowed inside
- * a step.  Results are identical in all three modes. */
+ * a step.  The modes cut the work differently, so outputs agree up to the rounding order of the split merge; selections
+ * and tables are the same. */
 enum { WNW_LAYERS_INDEPENDENT = 0, WNW_LAYERS_CHAINED = 1, WNW_LAYERS_SERIAL = 2 };
 wnw_status_t wnw_set_layer_dependency(wnw_cache_t *cache, int32_t mode);
 
