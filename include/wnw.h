@@ -52,7 +52,7 @@ typedef enum {
   WNW_ERR_OOM_HOST = 4,   /* pinned host allocation failed */
   WNW_ERR_CUDA = 5,       /* a CUDA runtime call failed */
   WNW_ERR_CAPACITY = 6,   /* text or audio capacity exceeded */
-  WNW_ERR_TIMEOUT = 7,    /* reserved */
+  WNW_ERR_TIMEOUT = 7,    /* a bounded device-side wait ran out (sticky, reported by wnw_sync); the context stays usable */
   WNW_ERR_UNSUPPORTED = 8,/* shape outside what the kernels are built for */
   WNW_ERR_DEVICE_CHECK = 9/* a device-side consistency check failed (sticky) */
 } wnw_status_t;
@@ -223,6 +223,12 @@ wnw_status_t wnw_get_stats(wnw_cache_t *cache, wnw_stats_t *stats_host);
  * and tables are the same. */
 enum { WNW_LAYERS_INDEPENDENT = 0, WNW_LAYERS_CHAINED = 1, WNW_LAYERS_SERIAL = 2 };
 wnw_status_t wnw_set_layer_dependency(wnw_cache_t *cache, int32_t mode);
+
+/* Test hook for the bounded waits: adds `delta` to the device's step-epoch word, so that the tidal CTAs of the next
+ * replayed step wait for a recall epoch that nothing will publish.  Every such wait gives up after about a second of
+ * SM clocks, the kernel finishes on what it has and sets the sticky status that wnw_sync reports as WNW_ERR_TIMEOUT.
+ * The cache's results are meaningless afterwards; destroy it.  Not for production use. */
+wnw_status_t wnw_debug_advance_step_epoch(wnw_cache_t *cache, int32_t delta);
 
 /* Kernels this cache has launched on the decode path since creation, replayed captured steps included:
  * counts[0] attention, [1] selection, [2] recall, [3] step-end.  Host counters, no synchronisation. */

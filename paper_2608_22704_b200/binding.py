@@ -67,6 +67,7 @@ _SIGNATURES = {
     "wnw_get_stats": [_vp, C.POINTER(wnw_stats_t)],
     "wnw_set_layer_dependency": [_vp, _i32],
     "wnw_get_launch_counts": [_vp, C.POINTER(C.c_int64)],
+    "wnw_debug_advance_step_epoch": [_vp, _i32],
     "wnw_get_base_slots": [_vp, _i32, C.POINTER(_i32)],
     "wnw_set_kernel_timing": [_vp, _i32],
     "wnw_get_kernel_time": [_vp, C.POINTER(C.c_float), C.POINTER(_i32)],
@@ -246,6 +247,10 @@ def wnw_get_stats(cache) -> dict:
     s = wnw_stats_t()
     _ck(lib().wnw_get_stats(cache, C.byref(s)), "wnw_get_stats")
     return {n: getattr(s, n) for n, _ in wnw_stats_t._fields_}
+
+
+def wnw_debug_advance_step_epoch(cache, delta: int):
+    _ck(lib().wnw_debug_advance_step_epoch(cache, int(delta)), "wnw_debug_advance_step_epoch")
 
 
 def wnw_get_launch_counts(cache):

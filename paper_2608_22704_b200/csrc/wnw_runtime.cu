@@ -1056,7 +1056,21 @@ extern "C" wnw_status_t wnw_sync(wnw_cache_t *c) {
   if (s != WNW_OK) return s;
   int32_t st = 0;
   CK(cudaMemcpy(&st, c->cv.status, sizeof(st), cudaMemcpyDeviceToHost));
+  if (st & STATUS_TIMEOUT) return WNW_ERR_TIMEOUT;   // a bounded device-side wait ran out (sticky)
   return st ? WNW_ERR_DEVICE_CHECK : WNW_OK;
+}
+
+extern "C" wnw_status_t wnw_debug_advance_step_epoch(wnw_cache_t *c, int32_t delta) {
+  if (!c) return WNW_ERR_INVALID_ARG;
+  if (c->in_step || c->graph_capturing) return WNW_ERR_STATE;
+  DeviceGuard guard(c->cfg.device);
+  wnw_status_t s = drain(c);
+  if (s != WNW_OK) return s;
+  int32_t v = 0;
+  CK(cudaMemcpy(&v, c->d_step_epoch, sizeof(v), cudaMemcpyDeviceToHost));
+  v += delta;
+  CK(cudaMemcpy(c->d_step_epoch, &v, sizeof(v), cudaMemcpyHostToDevice));
+  return WNW_OK;
 }
 
 static wnw_status_t check_seq_layer(wnw_cache *c, int seq, int layer) {

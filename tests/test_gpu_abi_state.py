@@ -150,3 +150,64 @@ def test_layer_dependency_rejects_bad_mode():
         wnw.wnw_set_layer_dependency(h, 1)
     finally:
         wnw.wnw_destroy(h)
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """The tidal CTAs of a replayed step wait (bounded, about a second of SM clocks) for the recall epoch of the previous
+    step.  With the expected epoch pushed beyond anything that will be published the waits run out: the kernels finish,
+    wnw_sync reports WNW_ERR_TIMEOUT, nothing hangs, and the context stays usable."""
+    import time
+    import paper_2608_22704_b200 as wnw
+    dev = torch.device("cuda:0")
+    A, T, F = ROLE_ANCHOR, ROLE_TIDAL, ROLE_FIXED
+    w = tiny_custom(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, n_text=4, audio_lens=(200,), chunk=16, budget=0.25,
+                    n_steps=6, roles=[[A, T], [A, T]])
+    syn = Synth(w, seed=1)
+
+    def run(h, n_replays, skew_before=None):
+        _place(wnw, h, syn, 0, range(w.n_layers))
+        dec = [syn.decode(0, l) for l in range(w.n_layers)]
+        sq = torch.zeros((w.n_layers, 1, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+        skn = torch.zeros((w.n_layers, 1, w.n_kv_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+        svn, out = torch.zeros_like(skn), torch.zeros_like(sq)
+        st = torch.cuda.Stream(device=dev)
+        torch.cuda.synchronize()
+        wnw.wnw_graph_begin(h, [0], st)
+        wnw.wnw_step_begin(h, [0])
+        for l in range(w.n_layers):
+            wnw.wnw_decode_layer(h, l, sq[l], skn[l], svn[l], out[l], stream=st)
+        wnw.wnw_step_end(h, stream=st)
+        wnw.wnw_graph_end(h, st)
+        for t in range(n_replays):
+            if skew_before == t:
+                wnw.wnw_debug_advance_step_epoch(h, 3)
+            with torch.cuda.stream(st):
+                for l in range(w.n_layers):
+                    sq[l, 0].copy_(dec[l]["q"][t]); skn[l, 0].copy_(dec[l]["k_new"][t]); svn[l, 0].copy_(dec[l]["v_new"][t])
+                wnw.wnw_graph_launch(h, st)
+        return out
+
+    h = _mk(wnw, w)
+    try:
+        run(h, 2)
+        wnw.wnw_sync(h)                                  # healthy replays: no status
+    finally:
+        wnw.wnw_destroy(h)
+    h = _mk(wnw, w)
+    try:
+        t0 = time.perf_counter()
+        run(h, 3, skew_before=2)
+        with pytest.raises(wnw.WnwError) as e:
+            wnw.wnw_sync(h)
+        elapsed = time.perf_counter() - t0
+        assert e.value.status == wnw.WNW_ERR_TIMEOUT
+        assert 0.3 < elapsed < 30.0                      # the waits gave up by themselves
+    finally:
+        wnw.wnw_destroy(h)
+    h = _mk(wnw, w)                                      # the context is still good
+    try:
+        out = run(h, 2)
+        wnw.wnw_sync(h)
+        assert torch.isfinite(out.float()).all()
+    finally:
+        wnw.wnw_destroy(h)
