@@ -96,3 +96,29 @@ def test_config3_batch32_segment_lag_sampled_sequences():
             ls.decode_step(t, graph=True, check_slots=(t == 2))
     finally:
         ls.close()
+
+
+@pytest.mark.parametrize("residency,seg", [(0, 64), (1, 25)])
+def test_config1_whole_decode_graph_replay(residency, seg):
+    """The whole 256-step decode of the 4-minute clip (text 64 -> 320 tokens, one full sweep of the focus through the audio)
+    under graph replay, the oracle following every step: the contract's form and the paper's form."""
+    from parity_harness import Lockstep
+    w = config1(n_steps=256)
+    w.chunk = seg
+    ls = Lockstep(w, seed=0, gen_device="cuda:0", residency=residency, evict_lag=3)
+    try:
+        ls.prefill(check_slots=False)
+        for t in range(256):
+            ls.decode_step(t, graph=True, check_slots=(t % 64 == 63))
+        ls.check_stats()
+        assert ls.near_ties <= 2
+        st = ls.o.stats(0)
+        assert st["misses"] > 500 and st["evictions"] > 400
+        assert wnw_text_len(ls) == w.n_text + 256
+    finally:
+        ls.close()
+
+
+def wnw_text_len(ls):
+    import paper_2608_22704_b200 as wnw
+    return wnw.wnw_get_seq_dims(ls.h, 0)[1]
