@@ -26,8 +26,8 @@
 
 namespace wnw {
 
-constexpr int NW_LAT = 8;  // warps per CTA when the launch fits one wave (latency regime): 1 CTA per SM
-constexpr int NW_THR = 4;  // warps per CTA otherwise (throughput regime): two persistent CTAs per SM, whose phases drift apart,
+constexpr int NW_LAT = 8;  // warps of a one-shot CTA (one work item each): 1 CTA per SM
+constexpr int NW_THR = 4;  // warps of a persistent CTA (large launches of chained layers): two per SM, whose phases drift apart,
                            // so one CTA's prologue and merge overlap the other's streaming
 constexpr int NSTAGE = 3;  // granules in flight per warp
 

@@ -109,7 +109,8 @@ struct wnw_cache {
   int external_recall_mode = -1;   // -1 automatic, 0 never, 1 always
   bool cap_external_recall = false, graph_external_recall = false, recall_all_pending = false;
   cudaEvent_t ev_graph_done = nullptr, ev_recall_all = nullptr;
-  int direct_max_granules = 64;   // heads up to this many granules (text capacity included) are not split in the latency regime
+  int direct_max_granules = 64;   // scale of the one-CTA rule: a head of up to 2x (overlapping layers) or x/2 (chained layers)
+                                  // this many granules (text capacity included) is not split
   // captured step
   bool graph_capturing = false;
   cudaGraph_t graph = nullptr;
@@ -521,7 +522,7 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       const SeqHost &sq = c->seqs[seq_ids[i]];
       const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
       const int ridx = mode == ATTN_DECODE ? c->role_idx[layer * G.Hkv + h] : h;
-      // latency regime: a short head stays in one CTA, which then writes the output itself (no partial, no merge)
+      // one-shot CTAs: a short head stays in one CTA, which then writes the output itself (no partial, no merge)
       const int nw_ = n_work[i * G.Hkv + h];
       int n_cta = std::max(1, (nw_ + gpi - 1) / gpi);
       // a short head stays in one CTA: up to 128 granules when layers overlap (work per launch counts), 32 when the
@@ -784,9 +785,9 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   if (layer == 0) c->step_capturing = capturing;
   else if (capturing != c->step_capturing) return WNW_ERR_STATE;
   if (layer == 0) {
-    // Replayed steps of small launches (latency regime) take their recall out of the captured graph, so that it can
-    // overlap the next replay.  In the throughput regime the persistent attention CTAs would sit on their SMs while
-    // they wait for it, so recall stays inside the step there.
+    // Replayed steps of small launches take their recall out of the captured graph, so that it can overlap the next
+    // replay.  Where a launch could fill the machine, its attention CTAs would sit on their SMs while they wait for
+    // it, so recall stays inside the step there.
     bool small = true;   // no launch can fill the machine with CTAs that wait
     for (const LayerWork &w : c->wl_layers) small = small && !w.throughput && w.n_items <= c->n_sm / 2;
     // the selection kernel of the last layer starts after every attention kernel of the step has completed, so the
