@@ -160,6 +160,7 @@ struct AttnArgs {
 // and recall plan for every layer in the update list.  Static data travels by value.
 struct SelectArgs {
   int32_t layer, n_active, score_on;
+  int32_t do_score, do_update;   // which half of the work this launch does (both, unless the step splits them)
   LayerInfo li;
   const int32_t *active;
   const float2 *gran_em;   // this layer's [n_active][n_aq][n_ag_max]
@@ -193,6 +194,8 @@ struct RecallSignal {
 cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st);
 // groups: CTAs per sequence (a layer that updates many tables, e.g. the last one under the global score scope)
 cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, int groups, cudaStream_t st);
+cudaError_t launch_select_all(const CacheView &cv, const SelectArgs *layer_args_dev, const int4 *map_dev, int n_entries,
+                              const SelectArgs &step, size_t smem_bytes, cudaStream_t st);
 cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *active, int appended, int32_t *bump_epoch,
                             cudaStream_t st);
 cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,

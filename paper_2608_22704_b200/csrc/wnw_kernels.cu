@@ -9,12 +9,12 @@ namespace wnw {
 // chunk, then "Dynamic Chunk Selection" for every layer whose score source is complete with this layer.
 // ------------------------------------------------------------------------------------------------
 constexpr int SEL_WARPS = 8;
-__global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid_constant__ CacheView cv,
-                                                                    const __grid_constant__ SelectArgs a, int smem_total) {
-  extern __shared__ __align__(16) unsigned char smem[];
+// One CTA: sequence i of the active list, group `grp` of `n_grp` over the layer's update list.
+__device__ __forceinline__ void select_body(const CacheView &cv, const SelectArgs &a, int smem_total, unsigned char *smem,
+                                            int i, int grp, int n_grp) {
   const Geometry &G = cv.geo;
   constexpr int NT = SEL_WARPS * 32;
-  const int i = blockIdx.x, b = a.active[i];
+  const int b = a.active[i];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const LayerInfo &li = a.li;
   // per-sequence scalars: one batch of independent loads
@@ -22,14 +22,15 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
   const long long step_b = cv.step_snap[(long long)b * G.L + a.layer];   // not cv.steps: an eager step's bookkeeping kernel
                                                                          // follows the attention kernel, not this one
   const int n_aq = a.n_aq;
-  const bool scored = li.n_anchor > 0 && a.score_on && C_b > 0;
+  const bool scored = li.n_anchor > 0 && a.score_on && C_b > 0 && a.do_score;
   // shared-memory layout: (M,Z) of the anchor q-heads | this layer's scores | per-warp update workspaces | granule partials
   float2 *mz_s = reinterpret_cast<float2 *>(smem);
   float *sc_s = reinterpret_cast<float *>(smem + ((size_t)n_aq * 8 + 15) / 16 * 16);
   float *glob_s = sc_s + (C_b + 3) / 4 * 4;   // global scope: sum of all anchor layers' scores
   unsigned char *ws0 = reinterpret_cast<unsigned char *>(glob_s) + ((size_t)C_b * 4 + 15) / 16 * 16;
   const size_t ws_bytes = select_ws_bytes(C_b, S_b);
-  const int n_par = li.upd_count < SEL_WARPS ? li.upd_count : SEL_WARPS;
+  const int n_upd = a.do_update ? li.upd_count : 0;
+  const int n_par = n_upd < SEL_WARPS ? n_upd : SEL_WARPS;
   float2 *em_s = reinterpret_cast<float2 *>(ws0 + (size_t)n_par * ws_bytes);
   const long long em_room = ((long long)smem_total - (long long)(reinterpret_cast<unsigned char *>(em_s) - smem)) / 8;
   int tile_c = 0;
@@ -82,8 +83,8 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
     stage_em(0, tile_c);
   }
   // the tables to update are dealt out over the CTAs of the sequence (grid y), then over the warps of a CTA
-  const int u_first = (int)blockIdx.y * n_par + warp, u_step = (int)gridDim.y * n_par;
-  if (warp < n_par && u_first < li.upd_count) {
+  const int u_first = grp * n_par + warp, u_step = n_grp * n_par;
+  if (warp < n_par && u_first < n_upd) {
     int lt, src;
     upd_of(u_first, lt, src);
     select_stage(cv, b, lt, src, scored && src == a.layer, C_b, S_b, lane, select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b));
@@ -116,7 +117,7 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
       __syncthreads();
     }
   }
-  if (cv.scope_global && li.upd_count > 0) {
+  if (cv.scope_global && n_upd > 0) {
     // Eq. 2 as printed: one accumulator over all anchor layers of the step, added in layer order
     for (int c = threadIdx.x; c < C_b; c += NT) {
       float gsum = 0.f;
@@ -130,7 +131,7 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
   }
   if (warp < n_par) {
     const SelectWs w = select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b);
-    for (int u = u_first; u < li.upd_count; u += u_step) {
+    for (int u = u_first; u < n_upd; u += u_step) {
       int lt, src;
       upd_of(u, lt, src);
       const bool local = (scored && src == a.layer) || src == -2;
@@ -157,8 +158,52 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid
   close_step();
 }
 
+__global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid_constant__ CacheView cv,
+                                                                    const __grid_constant__ SelectArgs a, int smem_total) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  select_body(cv, a, smem_total, smem, blockIdx.x, blockIdx.y, gridDim.y);
+}
+
+// The selection work of SEVERAL layers in one launch (captured steps of small launches: a launch costs about a
+// microsecond of the step whatever stream it is on, so thirty per-layer launches are replaced by one or two at the end
+// of the step).  grid (n_active, entries of `map`): entry y = (layer, group, groups of that layer).  The layer's
+// static arguments come from device memory, what changes per step from `step` (only those fields are read from it).
+__global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_all_kernel(const __grid_constant__ CacheView cv,
+                                                                        const SelectArgs *__restrict__ layer_args,
+                                                                        const int4 *__restrict__ map,
+                                                                        const __grid_constant__ SelectArgs step, int smem_total) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  __shared__ SelectArgs a_s;
+  const int4 m = map[blockIdx.y];
+  {
+    const int *src = reinterpret_cast<const int *>(layer_args + m.x);
+    int *dst = reinterpret_cast<int *>(&a_s);
+    for (int x = threadIdx.x; x < (int)(sizeof(SelectArgs) / sizeof(int)); x += blockDim.x) dst[x] = src[x];
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    a_s.n_active = step.n_active; a_s.active = step.active;
+    a_s.do_score = step.do_score; a_s.do_update = step.do_update;
+    a_s.fold_total = step.fold_total; a_s.fold_appended = step.fold_appended;
+    a_s.fold_counter = step.fold_counter; a_s.fold_bump_epoch = step.fold_bump_epoch;
+    a_s.epoch_words = step.epoch_words; a_s.empty_ctr = step.empty_ctr; a_s.step_epoch = step.step_epoch;
+  }
+  __syncthreads();
+  select_body(cv, a_s, smem_total, smem, blockIdx.x, m.y, m.z);
+}
+
 cudaError_t configure_select_kernel() {
+  cudaError_t e = cudaFuncSetAttribute(wnw_select_all_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM_CAP);
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(wnw_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM_CAP);
+}
+
+cudaError_t launch_select_all(const CacheView &cv, const SelectArgs *layer_args_dev, const int4 *map_dev, int n_entries,
+                              const SelectArgs &step, size_t smem_bytes, cudaStream_t st) {
+  if (n_entries <= 0 || step.n_active <= 0) return cudaSuccess;
+  wnw_select_all_kernel<<<dim3(step.n_active, n_entries), SEL_WARPS * 32, smem_bytes, st>>>(cv, layer_args_dev, map_dev, step,
+                                                                                           (int)smem_bytes);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, int groups, cudaStream_t st) {

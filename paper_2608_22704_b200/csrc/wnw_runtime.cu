@@ -97,6 +97,13 @@ struct wnw_cache {
   size_t gran_em_layer_stride = 0;
   bool step_capturing = false;
   bool pdl_enabled = true;
+  // Captured steps of small launches: the selection work of all layers in one launch at the end of the step (two when a
+  // layer ranks by another layer's scores: first all scores, then all updates).
+  bool select_all_enabled = true, cap_select_all = false, select_single_ok = false;
+  SelectArgs *d_sel_args = nullptr;
+  int4 *d_sel_map = nullptr;
+  int sel_map_single[2] = {0, 0}, sel_map_score[2] = {0, 0}, sel_map_update[2] = {0, 0};   // offset, entries
+  size_t sel_all_smem = 0;
   bool fold_enabled = true, cap_fold = false;   // captured steps: the last selection CTA closes the step
   int n_side_layers = 0, n_select_ctas = 0;   // layers with a selection kernel; its CTAs per sequence over all layers
   int32_t *d_fold_ctr = nullptr, *d_empty_ctr = nullptr;
@@ -237,6 +244,8 @@ static wnw_status_t validate_config(const wnw_config_t *cfg) {
   return WNW_OK;
 }
 
+static SelectArgs static_select_args(const wnw_cache *c, int layer);
+
 extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   if (!out) return WNW_ERR_INVALID_ARG;
   wnw_status_t vs = validate_config(cfg);
@@ -254,6 +263,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
   if (const char *e = getenv("WNW_PDL")) c->pdl_enabled = atoi(e) != 0;
   if (const char *e = getenv("WNW_FOLD_STEP_END")) c->fold_enabled = atoi(e) != 0;
+  if (const char *e = getenv("WNW_SELECT_ALL")) c->select_all_enabled = atoi(e) != 0;
   if (const char *e = getenv("WNW_EXTERNAL_RECALL")) c->external_recall_mode = atoi(e);
   if (const char *e = getenv("WNW_DIRECT_MAX_GRANULES")) c->direct_max_granules = atoi(e);
   CKE(configure_attn_kernels());
@@ -426,6 +436,34 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   CKC(dev_alloc(c, &c->d_step_epoch, 1));
   CKC(dev_alloc(c, &c->d_fold_ctr, 1));
   CKC(dev_alloc(c, &c->d_empty_ctr, (size_t)L));
+  if (!full) {
+    std::vector<SelectArgs> sel_args(L);
+    std::vector<int4> sel_map;
+    c->select_single_ok = !c->cv.scope_global;
+    for (int l = 0; l < L; ++l) {
+      sel_args[l] = static_select_args(c, l);
+      c->sel_all_smem = std::max(c->sel_all_smem, c->sel_smem[l]);
+      for (int u = 0; u < c->layers[l].upd_count; ++u)   // a layer that ranks by another layer's scores needs them complete
+        if (c->layers[c->upd_list[c->layers[l].upd_first + u]].src != l) c->select_single_ok = false;
+    }
+    auto add = [&](int (&range)[2], auto pred) {
+      range[0] = (int)sel_map.size();
+      for (int l = 0; l < L; ++l)
+        if (pred(c->layers[l])) {
+          const int g = select_groups(c->layers[l]);
+          for (int y = 0; y < g; ++y) sel_map.push_back(make_int4(l, y, g, 0));
+        }
+      range[1] = (int)sel_map.size() - range[0];
+    };
+    add(c->sel_map_single, [](const LayerInfo &li) { return li.n_anchor > 0 || li.upd_count > 0; });
+    add(c->sel_map_update, [](const LayerInfo &li) { return li.upd_count > 0; });
+    c->sel_map_score[0] = (int)sel_map.size();
+    for (int l = 0; l < L; ++l)
+      if (c->layers[l].n_anchor > 0) sel_map.push_back(make_int4(l, 0, 1, 0));
+    c->sel_map_score[1] = (int)sel_map.size() - c->sel_map_score[0];
+    CKC(dev_upload(c, &c->d_sel_args, sel_args));
+    CKC(dev_upload(c, &c->d_sel_map, sel_map));
+  }
   for (int l = 0; l < L; ++l)
     if (!full && (c->layers[l].n_anchor > 0 || c->layers[l].upd_count > 0)) {
       ++c->n_side_layers;
@@ -764,6 +802,28 @@ static bool stream_is_capturing(cudaStream_t st) {
   return cs != cudaStreamCaptureStatusNone;
 }
 
+// What a layer's selection kernel needs that never changes: the layer, its anchor q-heads, its update list.
+static SelectArgs static_select_args(const wnw_cache *c, int layer) {
+  const Geometry &G = c->geo;
+  const LayerInfo &li = c->layers[layer];
+  SelectArgs sa{};
+  sa.layer = layer; sa.li = li; sa.active = c->d_active;
+  sa.score_on = c->cfg.mode == WNW_MODE_TIERED && li.n_anchor > 0;
+  sa.do_score = 1; sa.do_update = 1;
+  sa.gran_em = c->gran_em + (size_t)layer * c->gran_em_layer_stride;
+  sa.head_mz = c->head_mz + (size_t)layer * G.max_batch * G.Hq;
+  sa.n_aq = std::max(li.n_anchor * G.g, 1); sa.n_ag_max = c->n_ag_max;
+  int aq = 0;
+  for (int h = 0; h < G.Hkv; ++h)
+    if (c->roles[layer * G.Hkv + h] == ROLE_ANCHOR)
+      for (int r = 0; r < G.g; ++r) sa.aq_head[aq++] = (uint8_t)(h * G.g + r);
+  for (int u = 0; u < li.upd_count && u < MAX_UPD_BY_VALUE; ++u) {
+    sa.upd_layer[u] = (int16_t)c->upd_list[li.upd_first + u];
+    sa.upd_src[u] = (int16_t)c->layers[sa.upd_layer[u]].src;
+  }
+  return sa;
+}
+
 static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer, const void *q, const void *k_new,
                                       const void *v_new, void *out, void *cuda_stream) {
   if (!c || !q || !out || ((k_new == nullptr) != (v_new == nullptr))) return WNW_ERR_INVALID_ARG;
@@ -795,8 +855,14 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     const LayerInfo &last = c->layers[G.L - 1];
     c->cap_fold = c->fold_enabled && capturing && c->graph_capturing && tiered && c->cfg.recall_mode != WNW_RECALL_INLINE &&
                   (last.n_anchor > 0 || last.upd_count > 0);
+    c->cap_select_all = false;
     c->cap_external_recall = capturing && c->graph_capturing && tiered && c->cfg.recall_mode != WNW_RECALL_INLINE &&
                              (c->external_recall_mode == 1 || (c->external_recall_mode < 0 && small));
+    // With the recall outside the graph nothing inside it needs a layer's selection before the step ends: all of it
+    // goes into one launch (or two) behind the last attention kernel.
+    c->cap_select_all = c->select_all_enabled && c->cap_external_recall && c->fold_enabled && small &&
+                        (c->select_single_ok ? c->sel_map_single[1] : c->sel_map_update[1]) > 0;
+    if (c->cap_select_all) c->cap_fold = true;
   }
   if (!capturing) {
     if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
@@ -852,28 +918,20 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     c->t_used.emplace_back(t0, t1);
   }
   // chunk scores, selection, recall: on the side stream, overlapping whatever follows on the caller's stream
-  const bool side_work = tiered && (li.n_anchor > 0 || li.upd_count > 0);
+  // (captured steps of small launches do all of it in one or two launches at the end of the step instead)
+  const bool side_work = tiered && (li.n_anchor > 0 || li.upd_count > 0) && !c->cap_select_all;
   const bool inline_mode = c->cfg.recall_mode == WNW_RECALL_INLINE;
   cudaEvent_t ev_l = capturing ? c->ev_layer_done_cap[layer] : c->ev_layer_done[layer];
   if (side_work && !inline_mode) CK(cudaEventRecord(ev_l, st));
   if (side_work) {
-    SelectArgs sa{};
-    sa.layer = layer; sa.n_active = n_active; sa.score_on = a.score_on; sa.li = li; sa.active = c->d_active;
-    sa.gran_em = gran_em_l; sa.head_mz = head_mz_l; sa.n_aq = a.n_aq; sa.n_ag_max = a.n_ag_max;
+    SelectArgs sa = static_select_args(c, layer);
+    sa.n_active = n_active;
     if (c->cap_fold) {
       sa.fold_total = c->n_select_ctas * n_active; sa.fold_appended = has_new; sa.fold_counter = c->d_fold_ctr;
       sa.fold_bump_epoch = c->cap_external_recall ? c->d_step_epoch : nullptr;
     }
     if (c->cap_external_recall && c->cap_fold) {   // the epoch arithmetic relies on the bump coming after every selection
       sa.epoch_words = c->d_recall_epoch; sa.empty_ctr = c->d_empty_ctr; sa.step_epoch = c->d_step_epoch;
-    }
-    int aq = 0;
-    for (int h = 0; h < G.Hkv; ++h)
-      if (c->roles[layer * G.Hkv + h] == ROLE_ANCHOR)
-        for (int r = 0; r < G.g; ++r) sa.aq_head[aq++] = (uint8_t)(h * G.g + r);
-    for (int u = 0; u < li.upd_count && u < MAX_UPD_BY_VALUE; ++u) {
-      sa.upd_layer[u] = (int16_t)c->upd_list[li.upd_first + u];
-      sa.upd_src[u] = (int16_t)c->layers[sa.upd_layer[u]].src;
     }
     const int si = layer % wnw_cache::N_SIDE;
     cudaStream_t ss = inline_mode ? st : c->side[si];
@@ -930,6 +988,22 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
     for (int ls : c->last_side_layer)  // join the forked side streams into the graph
       if (ls >= 0) CK(cudaStreamWaitEvent(st, c->ev_side_done_cap[ls], 0));
 
+  if (capturing && c->cap_select_all) {
+    SelectArgs stp{};
+    stp.n_active = (int)c->active.size(); stp.active = c->d_active;
+    stp.epoch_words = c->d_recall_epoch; stp.empty_ctr = c->d_empty_ctr; stp.step_epoch = c->d_step_epoch;
+    if (!c->select_single_ok) {   // first every anchor layer's scores, then every table update
+      stp.do_score = 1; stp.do_update = 0;
+      CK(launch_select_all(c->cv, c->d_sel_args, c->d_sel_map + c->sel_map_score[0], c->sel_map_score[1], stp, c->sel_all_smem, st));
+      if (c->sel_map_score[1] > 0) c->count_launch(1, 1, true);
+    }
+    const int *range = c->select_single_ok ? c->sel_map_single : c->sel_map_update;
+    stp.do_score = c->select_single_ok ? 1 : 0; stp.do_update = 1;
+    stp.fold_total = range[1] * stp.n_active; stp.fold_appended = c->appended == 1;
+    stp.fold_counter = c->d_fold_ctr; stp.fold_bump_epoch = c->d_step_epoch;
+    CK(launch_select_all(c->cv, c->d_sel_args, c->d_sel_map + range[0], range[1], stp, c->sel_all_smem, st));
+    c->count_launch(1, 1, true);
+  }
   if (!(capturing && c->cap_fold)) {
     CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1,
                        (capturing && c->cap_external_recall) ? c->d_step_epoch : nullptr, st));
