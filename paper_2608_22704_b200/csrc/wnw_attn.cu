@@ -209,6 +209,25 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     int item_idx, T_t, v_delta_audio, first, n_my;
     const CUtensorMap *map_audio;
   };
+  // Replayed steps: the recall that refreshed this layer's slots ran outside the captured graph, possibly still
+  // overlapping this step.  Bounded acquire-wait on the layer's epoch word before the first SLOT granule of a tidal item
+  // is fetched; the text granules that precede it in the item go out first and hide the round trip.
+  bool epoch_pending = false;
+  auto wait_recall_epoch = [&]() {
+    if (lane == 0) {
+      const int expect = *a.expect_epoch;
+      int seen;
+      const long long t0 = clock64();
+      for (;;) {
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];\n" : "=r"(seen) : "l"(a.wait_epoch) : "memory");
+        if (seen >= expect) break;
+        if (clock64() - t0 > 2000000000ll) { timed_out = true; break; }
+      }
+      asm volatile("fence.proxy.async.global;\n" ::: "memory");  // the slots are read by TMA (async proxy)
+    }
+    timed_out = __shfl_sync(0xffffffffu, (int)timed_out, 0) != 0;
+    epoch_pending = false;
+  };
   auto load_ctx = [&](Ctx &c, int qi) {
     c.item_idx = a.cta_ranges ? a.order[qi] : qi;
     // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
@@ -219,22 +238,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     else { c.v_delta_audio = G.S_max * G.ncp; c.map_audio = &maps.fixed; }                            // V rows
     c.first = c.it.g0 + warp;
     c.n_my = c.first < c.it.g1 ? (c.it.g1 - c.first + NW - 1) / NW : 0;
-    if (a.wait_epoch && c.it.role == ROLE_TIDAL) {
-      // Replayed steps: the recall that refreshed this layer's slots ran outside the captured graph, possibly still
-      // overlapping this step.  Bounded acquire-wait on the layer's epoch word before any slot is read.
-      if (lane == 0) {
-        const int expect = *a.expect_epoch;
-        int seen;
-        const long long t0 = clock64();
-        for (;;) {
-          asm volatile("ld.acquire.gpu.global.s32 %0, [%1];\n" : "=r"(seen) : "l"(a.wait_epoch) : "memory");
-          if (seen >= expect) break;
-          if (clock64() - t0 > 2000000000ll) { timed_out = true; break; }
-        }
-        asm volatile("fence.proxy.async.global;\n" ::: "memory");  // the slots are read by TMA (async proxy)
-      }
-      timed_out = __shfl_sync(0xffffffffu, (int)timed_out, 0) != 0;
-    }
+    epoch_pending = a.wait_epoch != nullptr && c.it.role == ROLE_TIDAL;   // see wait_recall_epoch
   };
   const int v_delta_text = G.T_cap_pad;
 
@@ -276,6 +280,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     const int row = __shfl_sync(0xffffffffu, blk.row, src_lane);
     const int j = c.first + n * NW;
     const bool is_text = j < G.n_tg;
+    if (epoch_pending && !is_text) wait_recall_epoch();
     bool load = meta != 0;
     if (meta == -1) load = visible(c, -1, 0, 0, j) > 0;  // waits for the text length
     if (meta == -3) load = __shfl_sync(0xffffffffu, blk.cid, src_lane) >= 0;  // waits for the table entry
