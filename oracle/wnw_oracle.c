@@ -428,10 +428,12 @@ static void allowed_for(const Oracle *o, const Seq *s, int layer, int kvh, unsig
 /* ------------------------------------------------------------------ */
 
 /* k,v: [n_tokens][Hkv][d] bf16 bits; audio = [audio_begin, audio_end); q_last: [Hq][d]. */
-int wnwo_place_prefill(Oracle *o, int seq, int layer, const uint16_t *k, const uint16_t *v, int n_tokens,
-                       int audio_begin, int audio_end, const uint16_t *q_last) {
+/* q_text: [n_q][Hq][d], the text queries whose attention over the audio is aggregated ("Prefill Compression":
+ * p_prefill = sum over text queries of their attention weights); n_q = 1 with the last prefix query is the contract's form. */
+int wnwo_place_prefill_multi(Oracle *o, int seq, int layer, const uint16_t *k, const uint16_t *v, int n_tokens,
+                             int audio_begin, int audio_end, const uint16_t *q_last, int n_q) {
   if (!o || seq < 0 || seq >= o->max_batch || layer < 0 || layer >= o->L || !k || !v || n_tokens < 0) return WNWO_ERR_ARG;
-  if (audio_begin < 0 || audio_end < audio_begin || audio_end > n_tokens) return WNWO_ERR_ARG;
+  if (audio_begin < 0 || audio_end < audio_begin || audio_end > n_tokens || n_q < 1) return WNWO_ERR_ARG;
   const int T_a = audio_end - audio_begin, T_t = n_tokens - T_a, Hkv = o->Hkv, d = o->d;
   if (T_a > o->max_audio || T_t > o->max_text) return WNWO_ERR_ARG;
   Seq *s = &o->seq[seq];
@@ -479,8 +481,9 @@ int wnwo_place_prefill(Oracle *o, int seq, int layer, const uint16_t *k, const u
     for (int c = 0; c < C; ++c) pre[c] = 0.0;
     int role = o->roles[layer * Hkv + h];
     if (role == ROLE_ANCHOR) continue;
-    for (int j = 0; j < o->g; ++j)
-      attend(o, s, layer, h, q_last + (size_t)(h * o->g + j) * d, T_t, all, out, pre, NULL);
+    for (int qi = 0; qi < n_q; ++qi) /* summed over the text queries, query by query, q-heads in order */
+      for (int j = 0; j < o->g; ++j)
+        attend(o, s, layer, h, q_last + ((size_t)qi * o->Hq + (size_t)(h * o->g + j)) * d, T_t, all, out, pre, NULL);
     if (role == ROLE_FIXED) { /* its own top-S chunks, frozen */
       for (int c = 0; c < C; ++c) keyf[c] = (float)pre[c];
       int *F = s->fixed_set + ((size_t)layer * Hkv + h) * S;
@@ -502,6 +505,11 @@ int wnwo_place_prefill(Oracle *o, int seq, int layer, const uint16_t *k, const u
   }
   free(all); free(out); free(lens); free(keyf); free(tid);
   return WNWO_OK;
+}
+
+int wnwo_place_prefill(Oracle *o, int seq, int layer, const uint16_t *k, const uint16_t *v, int n_tokens,
+                       int audio_begin, int audio_end, const uint16_t *q_last) {
+  return wnwo_place_prefill_multi(o, seq, layer, k, v, n_tokens, audio_begin, audio_end, q_last, 1);
 }
 
 /* ------------------------------------------------------------------ */

@@ -48,6 +48,8 @@ def lib():
         _lib.wnwo_score_source.argtypes = [C.c_void_p, C.c_int]
         _lib.wnwo_place_prefill.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_uint16), C.POINTER(C.c_uint16),
                                             C.c_int, C.c_int, C.c_int, C.POINTER(C.c_uint16)]
+        _lib.wnwo_place_prefill_multi.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_uint16), C.POINTER(C.c_uint16),
+                                                  C.c_int, C.c_int, C.c_int, C.POINTER(C.c_uint16), C.c_int]
         _lib.wnwo_step_begin.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.c_int]
         _lib.wnwo_decode_layer.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_uint16), C.POINTER(C.c_uint16),
                                            C.POINTER(C.c_uint16), C.POINTER(C.c_double)]
@@ -180,9 +182,10 @@ class Oracle:
         k_bits, v_bits = _u16(k_bits), _u16(v_bits)
         n = k_bits.shape[0]
         assert k_bits.shape == v_bits.shape == (n, self.Hkv, self.d)
-        q = None if q_last_bits is None else _u16(q_last_bits)
-        _check(lib().wnwo_place_prefill(self._h, seq, layer, _p(k_bits, C.c_uint16), _p(v_bits, C.c_uint16), n, audio_begin,
-                                        audio_end, _p(q, C.c_uint16)), "place_prefill")
+        q = None if q_last_bits is None else _u16(q_last_bits)   # [Hq, d], or [n_q, Hq, d]: all the text queries
+        n_q = 1 if q is None or q.ndim == 2 else q.shape[0]
+        _check(lib().wnwo_place_prefill_multi(self._h, seq, layer, _p(k_bits, C.c_uint16), _p(v_bits, C.c_uint16), n, audio_begin,
+                                              audio_end, _p(q, C.c_uint16), n_q), "place_prefill")
 
     def step_begin(self, active: Sequence[int]):
         a = np.ascontiguousarray(active, dtype=np.int32)

@@ -465,3 +465,47 @@ def test_segment_lag_rejects_negative_lag():
     w = config0()
     with pytest.raises(wo.OracleError):
         make_oracle(w, residency=1, evict_lag=-1)
+
+
+def test_prefill_scores_summed_over_text_queries():
+    """"Prefill Compression": the prefill score aggregates the attention of ALL text queries.  With n_q queries the
+    oracle's per-head chunk scores equal numpy dense attention summed over queries and q-heads, and (linearity) the sum
+    of the scores the single-query form gives for each query alone; the placements are the top chunks of that sum."""
+    A, T, F = ROLE_ANCHOR, ROLE_TIDAL, ROLE_FIXED
+    w = tiny_custom(n_layers=1, n_q_heads=4, n_kv_heads=2, head_dim=64, n_text=6, audio_lens=(150,), chunk=16, budget=0.3,
+                    roles=[[T, F]], n_steps=1)
+    w.roles = np.array([[T, F]], np.uint8)
+    w.n_prefill_queries = 5
+    # a tidal head needs an anchor somewhere: add a second layer that has one
+    w = tiny_custom(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=64, n_text=6, audio_lens=(150,), chunk=16, budget=0.3,
+                    roles=[[T, F], [A, F]], n_steps=1)
+    w.n_prefill_queries = 5
+    syn = Synth(w, seed=9)
+    p = syn.prefill(0, 0)
+    kb, vb, qt = bf16_bits(p["k"]), bf16_bits(p["v"]), bf16_bits(p["q_text"])
+    assert qt.shape == (5, 4, 64)
+    o = make_oracle(w)
+    o.place_prefill(0, 0, kb, vb, p["audio_begin"], p["audio_end"], qt)
+    scale = 1 / math.sqrt(w.head_dim)
+    K, V = bf16_bits_to_f64(kb), bf16_bits_to_f64(vb)
+    C = 10
+    for h in range(2):
+        want = np.zeros(C)
+        for qi in range(5):
+            for r in range(2):
+                _, prob = dense_attention(bf16_bits_to_f64(qt[qi, h * 2 + r]), K[:, h], V[:, h], scale)
+                aud = prob[p["audio_begin"]:p["audio_end"]]
+                want += np.add.reduceat(aud, np.arange(0, 150, 16))
+        got = o.prefill_scores(0, 0, h)
+        assert np.abs(got - want).max() < 1e-12
+        single = np.zeros(C)
+        for qi in range(5):
+            o1 = make_oracle(w)
+            o1.place_prefill(0, 0, kb, vb, p["audio_begin"], p["audio_end"], qt[qi])
+            single += o1.prefill_scores(0, 0, h)
+            o1.close()
+        assert np.abs(got - single).max() < 1e-12
+    S = o.dims(0)[3]
+    lens = np.array([16] * 9 + [6])
+    assert o.fixed_set(0, 0, 1).tolist() == _brute_rank(o.prefill_scores(0, 0, 1).astype(np.float32), lens)[:S]
+    assert o.residency(0, 0)[0].tolist() == _brute_rank(o.prefill_scores(0, 0, 0).astype(np.float32), lens)[:S]

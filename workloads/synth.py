@@ -39,7 +39,7 @@ ROLE_ANCHOR = 0
 ROLE_TIDAL = 1
 ROLE_FIXED = 2
 
-_TAG_DIRS, _TAG_PREFILL, _TAG_DECODE, _TAG_CENTRE, _TAG_ROLES, _TAG_LENS = 1, 2, 3, 4, 5, 6
+_TAG_DIRS, _TAG_PREFILL, _TAG_DECODE, _TAG_CENTRE, _TAG_ROLES, _TAG_LENS, _TAG_PREFILL_Q = 1, 2, 3, 4, 5, 6, 7
 
 
 @dataclass
@@ -61,6 +61,7 @@ class Workload:
     region: int = 64            # audio tokens per region code
     jump_every: int = 0         # 0: drifting focus; n>0: focus jumps every n steps
     sweep_steps: int = 0        # steps for one sweep of the clip (0: n_steps)
+    n_prefill_queries: int = 1  # text queries whose attention ranks the audio at prefill (1: the last prefix query only)
 
     @property
     def batch(self) -> int:
@@ -220,9 +221,20 @@ class Synth:
         q_noise = self._randn(g, w.n_q_heads, w.head_dim)
         s_q = s.repeat_interleave(w.group, dim=0)                                # [Hq,d]
         q_last = q_noise + 2.0 * math.sqrt(w.head_dim) * s_q
-        return {"k": k.to(torch.bfloat16).contiguous(), "v": v.to(torch.bfloat16).contiguous(),
-                "q_last": q_last.to(torch.bfloat16).contiguous(),
-                "n_tokens": n, "audio_begin": w.n_text, "audio_end": n}
+        out = {"k": k.to(torch.bfloat16).contiguous(), "v": v.to(torch.bfloat16).contiguous(),
+               "q_last": q_last.to(torch.bfloat16).contiguous(),
+               "n_tokens": n, "audio_begin": w.n_text, "audio_end": n}
+        if w.n_prefill_queries > 1:
+            # earlier text queries: each leans on the sink and on one region of its own; the last one is q_last
+            gq = self._gen(_TAG_PREFILL_Q, seq, layer)
+            m = w.n_prefill_queries - 1
+            qn = self._randn(gq, m, w.n_q_heads, w.head_dim)
+            n_reg = max(self.n_regions(seq), 1)
+            reg = torch.randint(0, n_reg, (m,), generator=gq, device=self.device)
+            lean = e[:, reg, :].permute(1, 0, 2).repeat_interleave(w.group, dim=1) if T_a > 0 else torch.zeros_like(qn)
+            qn = qn + 1.0 * math.sqrt(w.head_dim) * s_q.unsqueeze(0) + 1.0 * math.sqrt(w.head_dim) * lean
+            out["q_text"] = torch.cat([qn, q_last.unsqueeze(0)], dim=0).to(torch.bfloat16).contiguous()
+        return out
 
     def decode(self, seq: int, layer: int) -> dict:
         """Decode inputs of every step: q [n_steps,Hq,d], k_new, v_new [n_steps,Hkv,d]."""
