@@ -142,6 +142,12 @@ wnw_status_t wnw_destroy(wnw_cache_t *cache);
 wnw_status_t wnw_place_prefill(wnw_cache_t *cache, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
                                int32_t n_tokens, int32_t audio_begin, int32_t audio_end, const void *q_last_dev,
                                void *cuda_stream);
+/* The same with the prefill score summed over SEVERAL text queries ("Prefill Compression": p_prefill is the attention
+ * from the text queries aggregated over them): q_text_dev is [n_queries][n_q_heads][head_dim] bf16, every query
+ * attends to the whole prefill key set; one scoring pass per query, added in query order. */
+wnw_status_t wnw_place_prefill_multi(wnw_cache_t *cache, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                                     int32_t n_tokens, int32_t audio_begin, int32_t audio_end, const void *q_text_dev,
+                                     int32_t n_queries, void *cuda_stream);
 
 /* Open a decode step for the given sequences (HOST array of distinct sequence ids, all fully placed).
  * The order of active_seqs_host is the batch order of q/k_new/v_new/out in wnw_decode_layer. */

@@ -50,6 +50,7 @@ _SIGNATURES = {
     "wnw_create": [C.POINTER(wnw_config_t), C.POINTER(_vp)],
     "wnw_destroy": [_vp],
     "wnw_place_prefill": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _vp],
+    "wnw_place_prefill_multi": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp],
     "wnw_step_begin": [_vp, C.POINTER(_i32), _i32],
     "wnw_decode_layer": [_vp, _i32, _vp, _vp, _vp, _vp, _vp],
     "wnw_decode_layer_full": [_vp, _i32, _vp, _vp, _vp, _vp, _vp],
@@ -144,8 +145,16 @@ def wnw_destroy(cache: int):
 
 
 def wnw_place_prefill(cache, seq, layer, k, v, audio_begin, audio_end, q_last=None, stream=None):
+    """q_last: [n_q_heads, head_dim] (the last prefix query) or [n_queries, n_q_heads, head_dim] (all text queries)."""
+    if q_last is not None and q_last.dim() == 3:
+        return wnw_place_prefill_multi(cache, seq, layer, k, v, audio_begin, audio_end, q_last, stream)
     _ck(lib().wnw_place_prefill(cache, seq, layer, _ptr(k), _ptr(v), k.shape[0], audio_begin, audio_end, _ptr(q_last),
                                 _stream(stream)), "wnw_place_prefill")
+
+
+def wnw_place_prefill_multi(cache, seq, layer, k, v, audio_begin, audio_end, q_text, stream=None):
+    _ck(lib().wnw_place_prefill_multi(cache, seq, layer, _ptr(k), _ptr(v), k.shape[0], audio_begin, audio_end, _ptr(q_text),
+                                      q_text.shape[0], _stream(stream)), "wnw_place_prefill_multi")
 
 
 def wnw_step_begin(cache, active: Sequence[int]):

@@ -203,7 +203,7 @@ cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *acti
 cudaError_t launch_place_scatter(const CacheView &cv, int b, int layer, const bf16 *k, const bf16 *v, int n_tokens, int ab,
                                  int ae, int T_t, int C_b, int S_b, int S_base, bf16 *stage, cudaStream_t st);
 cudaError_t launch_prefill_select(const CacheView &cv, int b, int layer, const HeadItems *head_items, const float2 *part_ml,
-                                  const float2 *gran_em, int n_ag_max, cudaStream_t st);
+                                  const float2 *gran_em, int n_ag_max, int first, int last, cudaStream_t st);
 cudaError_t launch_place_gather(const CacheView &cv, int b, int layer, int full_mode, const bf16 *stage, int C_b,
                                 cudaStream_t st);
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);

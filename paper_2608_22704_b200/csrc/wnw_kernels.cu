@@ -395,7 +395,7 @@ cudaError_t launch_place_scatter(const CacheView &cv, int b, int layer, const bf
 // own top-S sets and the tidal heads' shared top-S table (rank r -> slot r, stamp -1-r).
 __global__ void __launch_bounds__(512) wnw_prefill_select_kernel(const __grid_constant__ CacheView cv, int b, int layer,
                                                                  const HeadItems *head_items, const float2 *part_ml,
-                                                                 const float2 *gran_em, int n_ag_max) {
+                                                                 const float2 *gran_em, int n_ag_max, int first, int last) {
   extern __shared__ float sm[];  // [Hq] M, [Hq] Z, [C_max] keys (as u64 pairs)
   const Geometry &G = cv.geo;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarp = blockDim.x >> 5;
@@ -437,8 +437,10 @@ __global__ void __launch_bounds__(512) wnw_prefill_select_kernel(const __grid_co
         total += sZ[hq] > 0.f ? sum_h / sZ[hq] : 0.f;
       }
     }
-    pre[(long long)h * G.C_max + c] = total;
+    // summed over the text queries, one launch per query ("Prefill Compression": p_prefill = sum over text queries)
+    pre[(long long)h * G.C_max + c] = first ? total : pre[(long long)h * G.C_max + c] + total;
   }
+  if (!last) return;   // the placement follows the last query
   __syncthreads();
   // fixed heads: rank by counting
   for (int h = 0; h < G.Hkv; ++h) {
@@ -476,9 +478,9 @@ __global__ void __launch_bounds__(512) wnw_prefill_select_kernel(const __grid_co
   }
 }
 cudaError_t launch_prefill_select(const CacheView &cv, int b, int layer, const HeadItems *head_items, const float2 *part_ml,
-                                  const float2 *gran_em, int n_ag_max, cudaStream_t st) {
+                                  const float2 *gran_em, int n_ag_max, int first, int last, cudaStream_t st) {
   const size_t smem = (size_t)(2 * cv.geo.Hq + 2) * sizeof(float) + (size_t)cv.geo.C_max * sizeof(unsigned long long);
-  wnw_prefill_select_kernel<<<1, 512, smem, st>>>(cv, b, layer, head_items, part_ml, gran_em, n_ag_max);
+  wnw_prefill_select_kernel<<<1, 512, smem, st>>>(cv, b, layer, head_items, part_ml, gran_em, n_ag_max, first, last);
   return cudaGetLastError();
 }
 

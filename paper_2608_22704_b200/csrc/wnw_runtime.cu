@@ -668,7 +668,13 @@ static wnw_status_t ensure_worklists(wnw_cache *c) {
 extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
                                           int32_t n_tokens, int32_t audio_begin, int32_t audio_end, const void *q_last_dev,
                                           void *cuda_stream) {
-  if (!c || !k_dev || !v_dev) return WNW_ERR_INVALID_ARG;
+  return wnw_place_prefill_multi(c, seq, layer, k_dev, v_dev, n_tokens, audio_begin, audio_end, q_last_dev, 1, cuda_stream);
+}
+
+extern "C" wnw_status_t wnw_place_prefill_multi(wnw_cache_t *c, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                                                int32_t n_tokens, int32_t audio_begin, int32_t audio_end,
+                                                const void *q_last_dev, int32_t n_queries, void *cuda_stream) {
+  if (!c || !k_dev || !v_dev || n_queries < 1) return WNW_ERR_INVALID_ARG;
   const Geometry &G = c->geo;
   if (seq < 0 || seq >= G.max_batch || layer < 0 || layer >= G.L || n_tokens < 1) return WNW_ERR_INVALID_ARG;
   if (audio_begin < 0 || audio_end < audio_begin || audio_end > n_tokens) return WNW_ERR_INVALID_ARG;
@@ -759,11 +765,14 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
     a.active = c->d_iota + seq; a.items = c->d_pf_items; a.items_host = c->h_pf_items.data(); a.n_items = c->pf_n_items; a.maps = &c->maps_prefill; a.throughput = c->pf_throughput;
     if (c->pf_n_ctas > 0) { a.order = c->d_pf_sched; a.cta_ranges = c->d_pf_sched + c->pf_ranges_base; a.n_ctas = c->pf_n_ctas; }
     a.head_items = c->d_pf_head_items;
-    a.q = (const bf16 *)q_last_dev;
     a.anchor_base = c->stage; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
     a.part_o = c->pf_part_o; a.part_ml = c->pf_part_ml; a.gran_em = c->pf_gran_em; a.n_aq = G.Hq; a.n_ag_max = c->n_ag_max;
-    CK(launch_attn(c->cv, a, st));
-    CK(launch_prefill_select(c->cv, seq, layer, c->d_pf_head_items, c->pf_part_ml, c->pf_gran_em, c->n_ag_max, st));
+    for (int qi = 0; qi < n_queries; ++qi) {   // one scoring pass per text query; the scores add up, the last pass places
+      a.q = (const bf16 *)q_last_dev + (size_t)qi * G.Hq * G.d;
+      CK(launch_attn(c->cv, a, st));
+      CK(launch_prefill_select(c->cv, seq, layer, c->d_pf_head_items, c->pf_part_ml, c->pf_gran_em, c->n_ag_max, qi == 0,
+                               qi == n_queries - 1, st));
+    }
   }
   CK(launch_place_gather(c->cv, seq, layer, full ? 1 : 0, c->stage, C_b, st));
   CK(cudaEventRecord(c->ev_place, st));

@@ -79,13 +79,14 @@ class Lockstep:
         for b in range(w.batch):
             for l in range(w.n_layers):
                 p = self.syn.prefill(b, l)
-                k, v, ql = (p[n].to(self.dev) for n in ("k", "v", "q_last"))
+                qname = "q_text" if "q_text" in p else "q_last"     # all text queries when the workload has several
+                k, v, ql = (p[n].to(self.dev) for n in ("k", "v", qname))
                 wnw.wnw_place_prefill(self.h, b, l, k, v, p["audio_begin"], p["audio_end"], ql)
                 if self.syn.device.type == "cuda":
                     torch.cuda.synchronize(self.dev)   # the generator's buffers are released right after
                 if b in self.oracle_seqs:
                     kb, vb = bf16_bits(p["k"]), bf16_bits(p["v"])
-                    self.o.place_prefill(b, l, kb, vb, p["audio_begin"], p["audio_end"], bf16_bits(p["q_last"]))
+                    self.o.place_prefill(b, l, kb, vb, p["audio_begin"], p["audio_end"], bf16_bits(p[qname]))
                     self.kept[(b, l)] = (kb[p["audio_begin"]:p["audio_end"]], vb[p["audio_begin"]:p["audio_end"]])
         wnw.wnw_sync(self.h)
         for b in self.oracle_seqs:

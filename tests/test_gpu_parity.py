@@ -131,3 +131,21 @@ def test_config2_first_steps():
     """3B Qwen-Omni-shaped stack (36 layers, 16q/2kv, d=128, 15000 audio tokens), routed layers, first decode steps."""
     w = config2(n_steps=2)
     _run(w, check_slots=False)
+
+
+@pytest.mark.parametrize("n_q,audio_len,chunk,d,hq,hkv", [(5, 333, 32, 128, 8, 2), (17, 1000, 25, 64, 4, 2), (3, 77, 7, 64, 2, 2)])
+def test_prefill_scores_summed_over_text_queries(n_q, audio_len, chunk, d, hq, hkv):
+    """Prefill placement ranked by the attention of ALL text queries (one scoring pass per query, scores added), then
+    decode steps on top of that placement."""
+    roles = [[A, T], [T, F], [A, F]]
+    w = tiny_custom(n_layers=3, n_q_heads=hq, n_kv_heads=hkv, head_dim=d, n_text=7, audio_lens=(audio_len, audio_len // 2),
+                    chunk=chunk, budget=0.3, n_steps=4, roles=roles, region=max(16, chunk))
+    w.n_prefill_queries = n_q
+    _run(w, seed=13)
+
+
+def test_prefill_scores_summed_over_text_queries_config1_shape():
+    w = config1(n_steps=2)
+    w.n_layers = 4; w.roles = w.roles[:4]
+    w.n_prefill_queries = 8
+    _run(w, check_slots=False)
