@@ -32,6 +32,12 @@ constexpr int NW_THR = 4;  // warps of a persistent CTA (large launches of chain
 constexpr int NSTAGE = 3;  // granules in flight per warp
 
 int attn_warps(bool throughput) { return throughput ? NW_THR : NW_LAT; }
+// Merge scratch of a CTA when it sits behind the stages instead of aliasing them: (m, l) and o of every warp.
+static size_t attn_scratch_bytes(int nw, int g, int d) { return (size_t)nw * 128 + (size_t)nw * g * d * 4; }
+// One-shot 8-warp CTAs can keep it there while everything fits the 227 KB a CTA may have.
+bool attn_xpref_fits(int g, int d) {
+  return (size_t)NW_LAT * NSTAGE * 2 * GR * d * 2 + 1024 + attn_scratch_bytes(NW_LAT, g, d) + 512 <= 227 * 1024;
+}
 
 
 // Phase stamps for latency studies: compiled in only with -DWNW_PHASE_STAMPS (never in the product build).
@@ -197,6 +203,10 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   bool timed_out = false;
   const int g = G.g;
   const LayerInfo &li = a.li;
+  // A CTA that serves several work items (short heads packed together) keeps its copy pipeline running across them:
+  // while one item is merged, the first granules of the next are already in flight.  Its merge scratch then sits
+  // behind the stages instead of aliasing them.
+  const bool xpref = a.xpref != 0;
 
   // One work item per CTA when the launch fits the machine; otherwise a persistent CTA per SM walks the items the
   // host assigned to it (balanced by size), so no SM idles through a partial last wave.
@@ -228,7 +238,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     timed_out = __shfl_sync(0xffffffffu, (int)timed_out, 0) != 0;
     epoch_pending = false;
   };
-  auto load_ctx = [&](Ctx &c, int qi) {
+  auto load_ctx = [&](Ctx &c, int qi, bool for_loads) {
     c.item_idx = a.cta_ranges ? a.order[qi] : qi;
     // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
     c.it = a.n_items <= INLINE_ITEMS_MAX ? inl.it[c.item_idx] : a.items[c.item_idx];
@@ -238,7 +248,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     else { c.v_delta_audio = G.S_max * G.ncp; c.map_audio = &maps.fixed; }                            // V rows
     c.first = c.it.g0 + warp;
     c.n_my = c.first < c.it.g1 ? (c.it.g1 - c.first + NW - 1) / NW : 0;
-    epoch_pending = a.wait_epoch != nullptr && c.it.role == ROLE_TIDAL;   // see wait_recall_epoch
+    if (for_loads) epoch_pending = a.wait_epoch != nullptr && c.it.role == ROLE_TIDAL;   // see wait_recall_epoch
   };
   const int v_delta_text = G.T_cap_pad;
 
@@ -307,25 +317,39 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     const int sidx = __shfl_sync(0xffffffffu, blk.score_idx, src_lane);
     if (lane == 0) ring[warp][seq % NSTAGE] = make_int2(valid | (loaded ? 256 : 0), sidx);
   };
-  // Fetches the producer's next granule of the current work item, if this warp has one left.
+  // Fetches the producer's next granule, moving on to the CTA's next work item when this warp has none left in the
+  // current one (only when the pipeline runs across items).
+  int p_qi = q_begin;
   auto produce = [&]() {
-    if (p_n >= prod.n_my) return;
+    while (p_n >= prod.n_my) {
+      if (!xpref || p_qi + 1 >= q_end) return;
+      ++p_qi;
+      load_ctx(prod, p_qi, true);
+      p_n = 0;
+    }
     const bool ld = issue_copy(prod, p_n, seq_p);
     issue_meta(prod, p_n, seq_p, ld);
     ++p_n; ++seq_p;
   };
 
   for (int qi = q_begin; qi < q_end; ++qi) {
-  // the merge below reuses the stages as scratch: the previous item's merge must be done
-  if (qi > q_begin) __syncthreads();
-  p_n = 0;
-  load_ctx(prod, qi);
-  const WorkItem &it = prod.it;
-  const int item_idx = prod.item_idx;
+  // without a scratch region of its own the merge below reuses the stages: the previous item's merge must be done
+  if (qi > q_begin && !xpref) __syncthreads();
+  const bool arm = !xpref || qi == q_begin;   // (re)start the pipeline at this item
+  Ctx cc;
+  if (arm) {
+    p_qi = qi; p_n = 0;
+    load_ctx(prod, qi, true);
+    cc = prod;
+  } else {
+    load_ctx(cc, qi, false);
+  }
+  const WorkItem &it = cc.it;
+  const int item_idx = cc.item_idx;
   if (cv.step_snap && it.h == 0 && it.g0 == 0 && threadIdx.x == 0 && a.mode != ATTN_PREFILL)   // (no cache state behind the
     cv.step_snap[(long long)it.b * G.L + a.layer] = cv.steps[it.b];                            //  allocation-free entry)
-  const int b = it.b, ridx = it.ridx, T_t = prod.T_t;
-  const int first = prod.first, n_my = prod.n_my;
+  const int b = it.b, ridx = it.ridx, T_t = cc.T_t;
+  const int first = cc.first, n_my = cc.n_my;
 #ifdef WNW_PHASE_STAMPS
   if (it.g0 >= 0) STAMP(10);
   kslot = (int)((cv.steps[b] & 3) * 64 + a.layer);
@@ -334,9 +358,11 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   // the first copies go out before anything else is read; their metadata follows the Q loads
   bool pro_loaded[NSTAGE - 1];
   int n_pro = 0;
+  if (arm) {
 #pragma unroll
-  for (int n = 0; n < NSTAGE - 1; ++n)
-    if (n < n_my) { pro_loaded[n] = issue_copy(prod, n, seq_p + n); n_pro = n + 1; }
+    for (int n = 0; n < NSTAGE - 1; ++n)
+      if (n < n_my) { pro_loaded[n] = issue_copy(prod, n, seq_p + n); n_pro = n + 1; }
+  }
   STAMP(1);
 
   // Chained layers: the cache loads above never depend on the preceding work, the query and the new token's K/V do.
@@ -356,10 +382,14 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       }
     }
   }
+  if (arm) {
 #pragma unroll
-  for (int n = 0; n < NSTAGE - 1; ++n)
-    if (n < n_pro) issue_meta(prod, n, seq_p + n, pro_loaded[n]);
-  p_n = n_pro; seq_p += n_pro;
+    for (int n = 0; n < NSTAGE - 1; ++n)
+      if (n < n_pro) issue_meta(prod, n, seq_p + n, pro_loaded[n]);
+    p_n = n_pro; seq_p += n_pro;
+    if (xpref)   // an item shorter than the pipeline: top up from the items that follow
+      for (int n = n_pro; n < NSTAGE - 1; ++n) produce();
+  }
 
   float o[D / 8][4];
 #pragma unroll
@@ -480,8 +510,11 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   STAMP(2);
 
   // ---- merge the warps' partial states through shared memory ----
-  float2 *red_ml = reinterpret_cast<float2 *>(smem);                           // [NW][16]  (the stages are idle by now)
-  float *red_o = reinterpret_cast<float *>(smem + NW * 16 * sizeof(float2));   // [NW][g][D]
+  // scratch: behind the stages when the pipeline runs across items (copies of the next item are landing in them),
+  // otherwise the stages themselves, which are idle by now
+  unsigned char *scratch = xpref ? smem + (size_t)NW * NSTAGE * 2 * TILEB : smem;
+  float2 *red_ml = reinterpret_cast<float2 *>(scratch);                           // [NW][16]
+  float *red_o = reinterpret_cast<float *>(scratch + NW * 16 * sizeof(float2));   // [NW][g][D]
   if ((lane & 3) == 0) {
     red_ml[warp * 16 + r0] = make_float2(m0, l0);
     red_ml[warp * 16 + r0 + 8] = make_float2(G16 ? m1 : -INFINITY, G16 ? l1 : 0.f);
@@ -604,7 +637,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 
 template <int D, bool G16, int NW>
 static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
-  const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024;  // + slack to align the stages to the swizzle atom
+  // stages + slack to align them to the swizzle atom + the merge scratch when it does not alias the stages
+  const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024 + (a.xpref ? attn_scratch_bytes(NW, cv.geo.g, D) : 0);
   if (!a.maps) return cudaErrorInvalidValue;
   InlineItems inl;
   if (a.n_items <= INLINE_ITEMS_MAX && a.items_host) memcpy(inl.it, a.items_host, sizeof(WorkItem) * a.n_items);
@@ -652,8 +686,9 @@ bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long row
 
 template <int D, bool G16, int NW>
 static cudaError_t configure_t() {
+  const size_t want = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024 + attn_scratch_bytes(NW, G16 ? 16 : 8, D);
   return cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)((size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024));
+                              (int)std::min<size_t>(want, 226 * 1024));
 }
 // Opt-in shared-memory sizes, set once per device at cache creation (never during a stream capture).
 cudaError_t configure_attn_kernels() {

@@ -137,6 +137,7 @@ struct AttnArgs {
   const int32_t *wait_epoch;     // replayed steps: tidal CTAs wait until *wait_epoch >= *expect_epoch (this layer's recall of the
   const int32_t *expect_epoch;   //   previous step, which runs outside the captured graph, has landed); null otherwise
   int32_t pdl;                   // launch with programmatic stream serialization (previous stream op is a layer kernel)
+  int xpref;        // the CTAs serve several work items each and keep their copy pipeline running across them
   int wait_inputs;  // q/k_new/v_new come from the preceding work on the stream: wait for it before reading them
   const HeadItems *head_items;  // [n_active][Hkv] work items of each head (first is relative to `items`)
   const bf16 *q;         // [n_active][Hq][d]
@@ -212,6 +213,7 @@ cudaError_t configure_attn_kernels();
 bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d);
 cudaError_t configure_select_kernel();
 constexpr int SELECT_SMEM_CAP = 200 * 1024;  // dynamic shared memory the selection kernel may be launched with
+bool attn_xpref_fits(int g, int d);  // a one-shot CTA can hold its merge scratch behind the copy stages
 int attn_warps(bool throughput);  // warps per attention CTA in the latency / throughput variant
 
 }  // namespace wnw
