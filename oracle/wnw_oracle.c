@@ -50,6 +50,12 @@
  *     dynamic slots [S_base, S); a fetched segment left unselected for delta
  *     consecutive steps is dropped (its stamp = the step it was last selected in).
  *     D = S - S_base = 2*topk*(delta+1) dynamic slots always suffice.
+ *   - token-granular prefill compression of FIXED heads (wnwo_place_prefill_tokens; "Prefill Compression" as
+ *     printed, Eq. 1 for the per-head retention): p_prefill[tau] = sum over the text queries and the head's q-heads
+ *     of the softmax weight of tau; the ranking key is (float)p_prefill[tau], ties to the earlier position; every
+ *     segment of `seg` tokens keeps its floor((double)retention * length) best positions (variant 1: the same total
+ *     from the whole head); the head then attends to [text | kept positions].  Tidal tables stay chunk-granular.
+ *     Pinned in tests/test_oracle_tokens.py against numpy sorts, a separate numpy softmax and hand-worked cases.
  */
 #include <math.h>
 #include <stdint.h>
@@ -77,6 +83,8 @@ typedef struct {
   long long *stamp;        /* [L][S] */
   int *fixed_set;          /* [L][Hkv][S] */
   int *fixed_n;            /* [L][Hkv] */
+  unsigned char **tok_mask; /* [L][Hkv] -> [T_a] kept positions of a fixed head placed token by token; NULL = chunk form */
+  double **tok_score;       /* [L][Hkv] -> [T_a] p_prefill of every audio position (token placement only) */
   double *score_sum;       /* [L][C]  this step's scores (anchor layers) */
   double *pre;             /* [L][Hkv][C] prefill scores */
   int *sel;                /* [L][topk] */
@@ -265,6 +273,9 @@ static void free_seq(Oracle *o, Seq *s) {
   if (s->audK)
     for (int l = 0; l < o->L; ++l) { free(s->audK[l]); free(s->audV[l]); free(s->txtK[l]); free(s->txtV[l]); }
   free(s->audK); free(s->audV); free(s->txtK); free(s->txtV);
+  if (s->tok_mask) for (int i = 0; i < o->L * o->Hkv; ++i) free(s->tok_mask[i]);
+  if (s->tok_score) for (int i = 0; i < o->L * o->Hkv; ++i) free(s->tok_score[i]);
+  free(s->tok_mask); free(s->tok_score);
   free(s->slot_chunk); free(s->stamp); free(s->fixed_set); free(s->fixed_n);
   free(s->score_sum); free(s->pre); free(s->sel); free(s->n_sel);
   memset(s, 0, sizeof(*s));
@@ -344,11 +355,14 @@ static int alloc_seq(Oracle *o, Seq *s, int T_a, int T_t) {
   s->stamp = (long long *)calloc((size_t)L * nS, sizeof(long long));
   s->fixed_set = (int *)malloc(sizeof(int) * L * Hkv * nS);
   s->fixed_n = (int *)calloc((size_t)L * Hkv, sizeof(int));
+  s->tok_mask = (unsigned char **)calloc((size_t)L * Hkv, sizeof(void *));
+  s->tok_score = (double **)calloc((size_t)L * Hkv, sizeof(void *));
   s->score_sum = (double *)calloc((size_t)L * nC, sizeof(double));
   s->pre = (double *)calloc((size_t)L * Hkv * nC, sizeof(double));
   s->sel = (int *)malloc(sizeof(int) * L * o->topk);
   s->n_sel = (int *)calloc((size_t)L, sizeof(int));
   if (!s->audK || !s->audV || !s->txtK || !s->txtV || !s->slot_chunk || !s->stamp || !s->fixed_set || !s->fixed_n ||
+      !s->tok_mask || !s->tok_score ||
       !s->score_sum || !s->pre || !s->sel || !s->n_sel)
     return WNWO_ERR_OOM;
   for (size_t i = 0; i < (size_t)L * nS; ++i) s->slot_chunk[i] = -1;
@@ -373,6 +387,8 @@ static int alloc_seq(Oracle *o, Seq *s, int T_a, int T_t) {
  * the whole probability row [T_t + T_a] (text first), zeros where masked. */
 static void attend(const Oracle *o, const Seq *s, int layer, int kvh, const uint16_t *q, int T_t,
                    const unsigned char *allowed, double *out, double *chunk_mass, double *p_row) {
+  /* a fixed head placed token by token sees exactly its kept positions */
+  const unsigned char *tok = s->tok_mask ? s->tok_mask[layer * o->Hkv + kvh] : NULL;
   const int d = o->d, T_a = s->T_a;
   const uint16_t *tK = s->txtK[layer] + (size_t)kvh * s->T_cap * d, *tV = s->txtV[layer] + (size_t)kvh * s->T_cap * d;
   const uint16_t *aK = s->audK[layer] + (size_t)kvh * T_a * d, *aV = s->audV[layer] + (size_t)kvh * T_a * d;
@@ -383,7 +399,7 @@ static void attend(const Oracle *o, const Seq *s, int layer, int kvh, const uint
     const uint16_t *krow;
     int vis;
     if (i < T_t) { krow = tK + (size_t)i * d; vis = 1; }
-    else { int tau = i - T_t; krow = aK + (size_t)tau * d; vis = allowed[tau / o->chunk] != 0; }
+    else { int tau = i - T_t; krow = aK + (size_t)tau * d; vis = tok ? tok[tau] != 0 : allowed[tau / o->chunk] != 0; }
     if (!vis) { logit[i] = -INFINITY; continue; }
     double acc = 0.0;
     for (int x = 0; x < d; ++x) acc += bf16_to_double(q[x]) * bf16_to_double(krow[x]);
@@ -504,6 +520,120 @@ int wnwo_place_prefill_multi(Oracle *o, int seq, int layer, const uint16_t *k, c
     free(tmp);
   }
   free(all); free(out); free(lens); free(keyf); free(tid);
+  return WNWO_OK;
+}
+
+/* Eq. 1: the fraction of audio positions a tidal or fixed head keeps on the GPU, from its normalised importance
+ * s_tilde in [0,1] and the scale lambda. */
+void wnwo_retention_schedule(const double *s_tilde, int n, double lambda, double *retention) {
+  for (int i = 0; i < n; ++i) {
+    double r = s_tilde[i] * lambda;
+    retention[i] = r < 1.0 ? r : 1.0;
+  }
+}
+
+/* Positions a fixed head keeps ("Prefill Compression"): key[tau] = p_prefill of position tau.
+ * variant 0: inside every segment of seg tokens (the last one may be shorter) the floor(retention * length) positions
+ *            with the largest key; variant 1 (the ablation's global top-k): the same total number of positions, taken
+ *            from the whole head with no per-segment quota.  Equal keys: the earlier position first.
+ * kept: ascending positions; returns their number, or a negated error code. */
+int wnwo_select_tokens(const float *key, int T_a, int seg, float retention, int variant, int *kept) {
+  if (!key || !kept || T_a < 0 || seg < 1 || !(retention >= 0.0f && retention <= 1.0f)) return -WNWO_ERR_ARG;
+  unsigned char *keep = (unsigned char *)calloc((size_t)(T_a > 0 ? T_a : 1), 1);
+  if (!keep) return -WNWO_ERR_OOM;
+  int total = 0;
+  for (int lo = 0; lo < T_a; lo += seg) {
+    int len = T_a - lo < seg ? T_a - lo : seg;
+    int m = (int)floor((double)retention * (double)len);
+    total += m;
+    if (variant == 0)
+      for (int r = 0; r < m; ++r) { /* the r-th largest of the segment among those not taken yet */
+        int best = -1;
+        for (int t = lo; t < lo + len; ++t)
+          if (!keep[t] && (best < 0 || key[t] > key[best])) best = t;
+        keep[best] = 1;
+      }
+  }
+  if (variant != 0)
+    for (int r = 0; r < total; ++r) {
+      int best = -1;
+      for (int t = 0; t < T_a; ++t)
+        if (!keep[t] && (best < 0 || key[t] > key[best])) best = t;
+      keep[best] = 1;
+    }
+  int n = 0;
+  for (int t = 0; t < T_a; ++t)
+    if (keep[t]) kept[n++] = t;
+  free(keep);
+  return n;
+}
+
+/* Prefill placement with the fixed heads compressed token by token ("Prefill Compression"): anchor heads keep all
+ * audio positions, the tidal table is filled as in wnwo_place_prefill_multi, and every fixed head h keeps the positions
+ * wnwo_select_tokens picks from p_prefill[tau] = sum over the text queries and the head's q-heads of the attention
+ * weight of tau (softmax over the whole prefix), with its own retention[h] (Eq. 1). */
+int wnwo_place_prefill_tokens(Oracle *o, int seq, int layer, const uint16_t *k, const uint16_t *v, int n_tokens,
+                              int audio_begin, int audio_end, const uint16_t *q_text, int n_q, const float *retention,
+                              int seg, int variant) {
+  if (!retention || seg < 1) return WNWO_ERR_ARG;
+  int rc = wnwo_place_prefill_multi(o, seq, layer, k, v, n_tokens, audio_begin, audio_end, q_text, n_q);
+  if (rc) return rc;
+  Seq *s = &o->seq[seq];
+  const int T_a = s->T_a, T_t = s->T_t, Hkv = o->Hkv, d = o->d;
+  if (s->C == 0) return WNWO_OK;
+  unsigned char *all = (unsigned char *)malloc((size_t)s->C);
+  double *out = (double *)malloc(sizeof(double) * d), *row = (double *)malloc(sizeof(double) * (size_t)(T_t + T_a));
+  float *keyf = (float *)malloc(sizeof(float) * T_a);
+  int *kept = (int *)malloc(sizeof(int) * T_a);
+  memset(all, 1, (size_t)s->C);
+  for (int h = 0; h < Hkv; ++h) {
+    if (o->roles[layer * Hkv + h] != ROLE_FIXED) continue;
+    if (!(retention[h] >= 0.0f && retention[h] <= 1.0f)) { rc = WNWO_ERR_ARG; break; }
+    const int idx = layer * Hkv + h;
+    free(s->tok_mask[idx]); s->tok_mask[idx] = NULL; /* the scoring below sees every position */
+    free(s->tok_score[idx]);
+    double *p = s->tok_score[idx] = (double *)calloc((size_t)T_a, sizeof(double));
+    for (int qi = 0; qi < n_q; ++qi)
+      for (int j = 0; j < o->g; ++j) {
+        attend(o, s, layer, h, q_text + ((size_t)qi * o->Hq + (size_t)(h * o->g + j)) * d, T_t, all, out, NULL, row);
+        for (int t = 0; t < T_a; ++t) p[t] += row[T_t + t];
+      }
+    for (int t = 0; t < T_a; ++t) keyf[t] = (float)p[t];
+    int n = wnwo_select_tokens(keyf, T_a, seg, retention[h], variant, kept);
+    unsigned char *mask = (unsigned char *)calloc((size_t)T_a, 1);
+    for (int i = 0; i < n; ++i) mask[kept[i]] = 1;
+    s->tok_mask[idx] = mask;
+  }
+  free(all); free(out); free(row); free(keyf); free(kept);
+  return rc;
+}
+
+int wnwo_get_token_scores(const Oracle *o, int seq, int layer, int kvh, double *out) {
+  const Seq *s = &o->seq[seq];
+  const double *p = s->tok_score ? s->tok_score[layer * o->Hkv + kvh] : NULL;
+  if (!p) return WNWO_ERR_STATE;
+  memcpy(out, p, sizeof(double) * s->T_a);
+  return WNWO_OK;
+}
+/* kept positions of a fixed head placed token by token, ascending; returns their number (-1: chunk form) */
+int wnwo_get_fixed_tokens(const Oracle *o, int seq, int layer, int kvh, int *pos) {
+  const Seq *s = &o->seq[seq];
+  const unsigned char *m = s->tok_mask ? s->tok_mask[layer * o->Hkv + kvh] : NULL;
+  if (!m) return -1;
+  int n = 0;
+  for (int t = 0; t < s->T_a; ++t)
+    if (m[t]) pos[n++] = t;
+  return n;
+}
+int wnwo_set_fixed_tokens(Oracle *o, int seq, int layer, int kvh, const int *pos, int n) {
+  Seq *s = &o->seq[seq];
+  unsigned char *m = s->tok_mask ? s->tok_mask[layer * o->Hkv + kvh] : NULL;
+  if (!m) return WNWO_ERR_STATE;
+  memset(m, 0, (size_t)s->T_a);
+  for (int i = 0; i < n; ++i) {
+    if (pos[i] < 0 || pos[i] >= s->T_a) return WNWO_ERR_ARG;
+    m[pos[i]] = 1;
+  }
   return WNWO_OK;
 }
 

@@ -71,6 +71,15 @@ def lib():
         _lib.wnwo_lag_update.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_longlong), C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int,
                                          C.c_longlong, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
                                          C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        _lib.wnwo_retention_schedule.argtypes = [C.POINTER(C.c_double), C.c_int, C.c_double, C.POINTER(C.c_double)]
+        _lib.wnwo_retention_schedule.restype = None
+        _lib.wnwo_select_tokens.argtypes = [C.POINTER(C.c_float), C.c_int, C.c_int, C.c_float, C.c_int, C.POINTER(C.c_int)]
+        _lib.wnwo_place_prefill_tokens.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_uint16), C.POINTER(C.c_uint16),
+                                                   C.c_int, C.c_int, C.c_int, C.POINTER(C.c_uint16), C.c_int,
+                                                   C.POINTER(C.c_float), C.c_int, C.c_int]
+        _lib.wnwo_get_token_scores.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_double)]
+        _lib.wnwo_get_fixed_tokens.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
+        _lib.wnwo_set_fixed_tokens.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int]
         _lib.wnwo_topk.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int), C.c_int, C.c_int, C.POINTER(C.c_int)]
         _lib.wnwo_table_update.argtypes = [C.POINTER(C.c_int), C.POINTER(C.c_longlong), C.c_int, C.POINTER(C.c_int), C.c_int,
                                            C.c_longlong, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
@@ -108,6 +117,24 @@ def table_update(slot_chunk: np.ndarray, stamp: np.ndarray, sel: Sequence[int], 
     if n < 0:
         raise OracleError("table_update: no victim (S < k?)")
     return [(int(pc[i]), int(ps[i]), int(ev[i])) for i in range(n)], hits.value
+
+
+def retention_schedule(s_tilde, lam: float) -> np.ndarray:
+    """Eq. 1: retention_i = min(s_tilde_i * lambda, 1)."""
+    st = np.ascontiguousarray(s_tilde, np.float64)
+    out = np.zeros(len(st), np.float64)
+    lib().wnwo_retention_schedule(_p(st, C.c_double), len(st), float(lam), _p(out, C.c_double))
+    return out
+
+
+def select_tokens(key: np.ndarray, seg: int, retention: float, variant: int = 0) -> np.ndarray:
+    """Kept positions of a fixed head ("Prefill Compression"): per-segment top floor(retention * n_s) (variant 0) or the
+    same total taken from the whole head (variant 1, the ablation's global top-k)."""
+    kf = np.ascontiguousarray(key, np.float32)
+    out = np.zeros(max(len(kf), 1), np.int32)
+    n = lib().wnwo_select_tokens(_p(kf, C.c_float), len(kf), int(seg), float(retention), int(variant), _p(out, C.c_int))
+    _check(-min(n, 0), "select_tokens")
+    return out[:n].copy()
 
 
 def select_segments(seg_sum: np.ndarray, lens: np.ndarray, k: int):
@@ -186,6 +213,29 @@ class Oracle:
         n_q = 1 if q is None or q.ndim == 2 else q.shape[0]
         _check(lib().wnwo_place_prefill_multi(self._h, seq, layer, _p(k_bits, C.c_uint16), _p(v_bits, C.c_uint16), n, audio_begin,
                                               audio_end, _p(q, C.c_uint16), n_q), "place_prefill")
+
+    def place_prefill_tokens(self, seq, layer, k_bits, v_bits, audio_begin, audio_end, q_text_bits, retention, seg, variant=0):
+        k = _u16(k_bits); v = _u16(v_bits); q = _u16(q_text_bits)
+        n_q = q.size // (self.Hq * self.d)
+        r = np.ascontiguousarray(retention, np.float32)
+        assert len(r) == self.Hkv
+        _check(lib().wnwo_place_prefill_tokens(self._h, seq, layer, _p(k, C.c_uint16), _p(v, C.c_uint16), k.shape[0],
+                                               audio_begin, audio_end, _p(q, C.c_uint16), n_q, _p(r, C.c_float), int(seg),
+                                               int(variant)), "place_prefill_tokens")
+
+    def token_scores(self, seq, layer, kv_head) -> np.ndarray:
+        out = np.zeros(max(self.dims(seq)[0], 1), np.float64)
+        _check(lib().wnwo_get_token_scores(self._h, seq, layer, kv_head, _p(out, C.c_double)), "token_scores")
+        return out[:self.dims(seq)[0]]
+
+    def fixed_tokens(self, seq, layer, kv_head):
+        out = np.zeros(max(self.dims(seq)[0], 1), np.int32)
+        n = lib().wnwo_get_fixed_tokens(self._h, seq, layer, kv_head, _p(out, C.c_int))
+        return None if n < 0 else out[:n].copy()
+
+    def set_fixed_tokens(self, seq, layer, kv_head, pos):
+        a = np.ascontiguousarray(pos, np.int32)
+        _check(lib().wnwo_set_fixed_tokens(self._h, seq, layer, kv_head, _p(a, C.c_int), len(a)), "set_fixed_tokens")
 
     def step_begin(self, active: Sequence[int]):
         a = np.ascontiguousarray(active, dtype=np.int32)
