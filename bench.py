@@ -180,14 +180,19 @@ class Job:
         self.caches[key] = h
         return h
 
-    def place_all(self, keys, keep_host=None):
-        """Generates each (seq, layer) prefill once on the device and places it into every cache in `keys`."""
+    def place_all(self, keys, keep_host=None, token=None):
+        """Generates each (seq, layer) prefill once on the device and places it into every cache in `keys`.
+        token = (retention [n_layers][n_kv_heads], segment_tokens, variant): fixed heads compressed token by token."""
         w, wnw = self.w, self.wnw
         for b in range(self.B):
             for l in range(w.n_layers):
                 p = self.syn.prefill(b, l)
                 for key in keys:
-                    wnw.wnw_place_prefill(self.caches[key], b, l, p["k"], p["v"], p["audio_begin"], p["audio_end"], p["q_last"])
+                    if token is not None:
+                        wnw.wnw_place_prefill_tokens(self.caches[key], b, l, p["k"], p["v"], p["audio_begin"], p["audio_end"],
+                                                     p["q_last"][None], token[0][l], token[1], token[2])
+                    else:
+                        wnw.wnw_place_prefill(self.caches[key], b, l, p["k"], p["v"], p["audio_begin"], p["audio_end"], p["q_last"])
                 if keep_host is not None and keep_host(b, l):
                     keep_host.store[(b, l)] = (bf16_bits(p["k"]), bf16_bits(p["v"]), bf16_bits(p["q_last"]), p["audio_begin"],
                                                p["audio_end"])
@@ -659,7 +664,11 @@ def run_ours(args, rank, world, local_rank):
         jq = Job(wq, seed=0, device=dev, wnw=wnw, score_scope=wnw.WNW_SCOPE_GLOBAL, residency=wnw.WNW_RESIDENCY_SEGMENT_LAG, evict_lag=3)
         jq.create("wnw", wnw.WNW_MODE_TIERED)
         jq.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
-        jq.place_all(["wnw", "skip"])
+        # fixed heads: token-granular per-segment top-k with per-head retention from Eq. 1 (seeded importances in [0,1],
+        # lambda = 2 x budget, so the mean retention is the budget)
+        lam_q = 2.0 * wq.budget
+        ret_q = wnw.wnw_retention_schedule(np.random.RandomState(0).rand(wq.n_layers * wq.n_kv_heads), lam_q)
+        jq.place_all(["wnw", "skip"], token=(ret_q.reshape(wq.n_layers, wq.n_kv_heads), wq.chunk, 0))
         for tt in range(W):
             jq.step("wnw", tt); jq.step("skip", tt)
         torch.cuda.synchronize(dev)
@@ -671,7 +680,9 @@ def run_ours(args, rank, world, local_rank):
         st1 = wnw.wnw_get_stats(jq.caches["wnw"])
         T_a_q, _, C_q, S_q = wnw.wnw_get_seq_dims(jq.caches["wnw"], 0)
         paper_form = {"segment_tokens": wq.chunk, "segments": C_q, "slots": S_q, "base_slots": wnw.wnw_get_base_slots(jq.caches["wnw"], 0),
-                      "evict_lag": 3, "score_scope": "global", "step_us": ms_q * 1e3, "tokens_per_s": wq.batch / (ms_q * 1e-3),
+                      "evict_lag": 3, "score_scope": "global",
+                      "fixed_heads": f"token-granular, per segment top floor(retention*n_s); retention = min(s*{lam_q:g}, 1), s ~ U[0,1] seeded",
+                      "step_us": ms_q * 1e3, "tokens_per_s": wq.batch / (ms_q * 1e-3),
                       "back_to_back_step_us": ms_q_bb * 1e3, "back_to_back_exposed_recall_us": (ms_q_bb - ms_q_bb_skip) * 1e3,
                       "recall_bytes_per_step": (st1["recall_bytes"] - st0["recall_bytes"]) / (n_pf + n_bb),
                       "r_gpu": st1["resident_audio_tokens"] / max(st1["full_audio_tokens"], 1)}

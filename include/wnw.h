@@ -148,6 +148,39 @@ wnw_status_t wnw_place_prefill(wnw_cache_t *cache, int32_t seq, int32_t layer, c
 wnw_status_t wnw_place_prefill_multi(wnw_cache_t *cache, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
                                      int32_t n_tokens, int32_t audio_begin, int32_t audio_end, const void *q_text_dev,
                                      int32_t n_queries, void *cuda_stream);
+/* Prefill placement with the FIXED heads compressed token by token ("Prefill Compression", per-head retention from
+ * Eq. 1).  Anchor heads, tidal tables, slots and host mirrors are placed exactly as by wnw_place_prefill_multi.  Every
+ * fixed KV-head h of the layer then keeps, instead of whole chunks, single audio positions:
+ *   p[tau]      = sum over the n_queries text queries and the head's q-heads of the softmax weight of audio position tau
+ *                 (softmax over the whole prefix, fp32);
+ *   variant 0   : inside every segment of segment_tokens positions (the last may be shorter) the
+ *                 floor((double)retention[h] * length) positions with the largest p, the earlier position on equal p;
+ *   variant 1   : the same number of positions taken from the whole head with no per-segment quota (the paper's
+ *                 global top-k ablation of the prefill selection).
+ * The kept positions, in ascending order, fill the head's compact store; decode attends to [text | kept positions].
+ *   retention   : HOST pointer, [n_kv_heads] floats in [0,1]; entries of heads that are not fixed in this layer are
+ *                 ignored.  A head may keep at most S_max * chunk_tokens positions (the capacity of its store, S_max
+ *                 the slots of a tidal table at max_audio_tokens): WNW_ERR_CAPACITY otherwise, nothing placed.
+ * Scratch and the position lists are allocated by the first call (device memory; not allocation-free).  In FULL mode
+ * this is wnw_place_prefill_multi.  Errors as wnw_place_prefill; WNW_ERR_INVALID_ARG for a retention outside [0,1],
+ * segment_tokens < 1 or an unknown variant. */
+wnw_status_t wnw_place_prefill_tokens(wnw_cache_t *cache, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                                      int32_t n_tokens, int32_t audio_begin, int32_t audio_end, const void *q_text_dev,
+                                      int32_t n_queries, const float *retention, int32_t segment_tokens, int32_t variant,
+                                      void *cuda_stream);
+/* Eq. 1 on the host: retention[i] = min(s_tilde[i] * lambda, 1) for n heads; s_tilde in [0,1] (the normalised
+ * importance of a tidal or fixed head), lambda >= 0.  Host pointers. */
+wnw_status_t wnw_retention_schedule(const float *s_tilde, int32_t n, float lambda, float *retention);
+/* Introspection of a token placement (host pointers; both wait for queued work).
+ * wnw_get_token_scores: p[tau] of a fixed head, [T_a] floats, valid for the (seq, layer) of the most recent
+ * wnw_place_prefill_tokens call only (WNW_ERR_STATE otherwise).
+ * wnw_get_fixed_tokens: the kept positions of a fixed head in ascending order and their number; WNW_ERR_STATE if the
+ * head was placed chunk-wise (then wnw_get_fixed_set applies, which in turn returns WNW_ERR_STATE for a head placed
+ * token by token). */
+wnw_status_t wnw_get_token_scores(wnw_cache_t *cache, int32_t seq, int32_t layer, int32_t kv_head, float *scores,
+                                  int32_t capacity);
+wnw_status_t wnw_get_fixed_tokens(wnw_cache_t *cache, int32_t seq, int32_t layer, int32_t kv_head, int32_t *positions,
+                                  int32_t capacity, int32_t *n);
 
 /* Open a decode step for the given sequences (HOST array of distinct sequence ids, all fully placed).
  * The order of active_seqs_host is the batch order of q/k_new/v_new/out in wnw_decode_layer. */

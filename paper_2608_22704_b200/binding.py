@@ -51,6 +51,10 @@ _SIGNATURES = {
     "wnw_destroy": [_vp],
     "wnw_place_prefill": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _vp],
     "wnw_place_prefill_multi": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp],
+    "wnw_place_prefill_tokens": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _i32, C.POINTER(C.c_float), _i32, _i32, _vp],
+    "wnw_retention_schedule": [C.POINTER(C.c_float), _i32, C.c_float, C.POINTER(C.c_float)],
+    "wnw_get_token_scores": [_vp, _i32, _i32, _i32, C.POINTER(C.c_float), _i32],
+    "wnw_get_fixed_tokens": [_vp, _i32, _i32, _i32, C.POINTER(_i32), _i32, C.POINTER(_i32)],
     "wnw_step_begin": [_vp, C.POINTER(_i32), _i32],
     "wnw_decode_layer": [_vp, _i32, _vp, _vp, _vp, _vp, _vp],
     "wnw_decode_layer_full": [_vp, _i32, _vp, _vp, _vp, _vp, _vp],
@@ -157,6 +161,22 @@ def wnw_place_prefill_multi(cache, seq, layer, k, v, audio_begin, audio_end, q_t
                                       q_text.shape[0], _stream(stream)), "wnw_place_prefill_multi")
 
 
+def wnw_place_prefill_tokens(cache, seq, layer, k, v, audio_begin, audio_end, q_text, retention, segment_tokens, variant=0,
+                             stream=None):
+    r = np.ascontiguousarray(retention, np.float32)
+    _ck(lib().wnw_place_prefill_tokens(cache, seq, layer, _ptr(k), _ptr(v), k.shape[0], audio_begin, audio_end, _ptr(q_text),
+                                       q_text.shape[0] if q_text.dim() == 3 else 1, r.ctypes.data_as(C.POINTER(C.c_float)),
+                                       segment_tokens, variant, _stream(stream)), "wnw_place_prefill_tokens")
+
+
+def wnw_retention_schedule(s_tilde, lam: float) -> np.ndarray:
+    s = np.ascontiguousarray(s_tilde, np.float32)
+    out = np.zeros(len(s), np.float32)
+    _ck(lib().wnw_retention_schedule(s.ctypes.data_as(C.POINTER(C.c_float)), len(s), float(lam),
+                                     out.ctypes.data_as(C.POINTER(C.c_float))), "wnw_retention_schedule")
+    return out
+
+
 def wnw_step_begin(cache, active: Sequence[int]):
     a = (C.c_int32 * len(active))(*active)
     _ck(lib().wnw_step_begin(cache, a, len(active)), "wnw_step_begin")
@@ -243,6 +263,23 @@ def wnw_get_fixed_set(cache, seq, layer, kv_head) -> np.ndarray:
     out = np.full(max(S, 1), -1, np.int32)
     n = _i32()
     _ck(lib().wnw_get_fixed_set(cache, seq, layer, kv_head, out.ctypes.data_as(C.POINTER(_i32)), C.byref(n)), "wnw_get_fixed_set")
+    return out[:n.value].copy()
+
+
+def wnw_get_token_scores(cache, seq, layer, kv_head) -> np.ndarray:
+    T_a = wnw_get_seq_dims(cache, seq)[0]
+    out = np.zeros(max(T_a, 1), np.float32)
+    _ck(lib().wnw_get_token_scores(cache, seq, layer, kv_head, out.ctypes.data_as(C.POINTER(C.c_float)), len(out)),
+        "wnw_get_token_scores")
+    return out[:T_a].copy()
+
+
+def wnw_get_fixed_tokens(cache, seq, layer, kv_head) -> np.ndarray:
+    T_a = wnw_get_seq_dims(cache, seq)[0]
+    out = np.full(max(T_a, 1), -1, np.int32)
+    n = _i32()
+    _ck(lib().wnw_get_fixed_tokens(cache, seq, layer, kv_head, out.ctypes.data_as(C.POINTER(_i32)), len(out), C.byref(n)),
+        "wnw_get_fixed_tokens")
     return out[:n.value].copy()
 
 

@@ -265,9 +265,12 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     int len;
     if (meta == -1) len = c.T_t - j * GR;
     else {
-      if (cid < 0) return 0;
-      len = c.it.T_a - cid * G.nc;
-      if (len > G.nc) len = G.nc;
+      if (cid == -1) return 0;
+      if (cid < -1) len = -cid - 2;   // a block of a token-compacted fixed head: the entry carries its row count
+      else {
+        len = c.it.T_a - cid * G.nc;
+        if (len > G.nc) len = G.nc;
+      }
       len -= off;
     }
     return len <= 0 ? 0 : (len < GR ? len : GR);

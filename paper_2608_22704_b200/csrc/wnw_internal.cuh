@@ -207,6 +207,11 @@ cudaError_t launch_prefill_select(const CacheView &cv, int b, int layer, const H
                                   const float2 *gran_em, int n_ag_max, int first, int last, cudaStream_t st);
 cudaError_t launch_place_gather(const CacheView &cv, int b, int layer, int full_mode, const bf16 *stage, int C_b,
                                 cudaStream_t st);
+// token-granular compression of the layer's fixed heads (after the chunk-granular placement staged the prefix)
+cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_fixed, const bf16 *stage, const bf16 *q_text,
+                                  int n_q, int T_t, int T_a, int seg, const float *retention_dev, int variant, float *work,
+                                  float *p_tok, int32_t *flags, long long p_stride, int32_t *fixed_tok, int tok_cap,
+                                  int32_t *tok_n, cudaStream_t st);
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
 cudaError_t configure_attn_kernels();
 // Encodes the descriptor of one store: base (device), rows, head_dim.  Returns false if the driver refuses.

@@ -21,6 +21,7 @@ struct SeqHost {
   int T_a = 0, T_t = 0, C = 0, S = 0, S_base = 0;   // S: all slots of a tidal table; S_base: the permanent ones
   bf16 *mirror = nullptr;
   size_t mirror_bytes = 0;
+  std::vector<int> fixed_blocks;   // [L][Hkv] blocks of a token-compacted fixed head's store; empty or -1: S_base chunks
 };
 
 struct LayerWork {
@@ -131,6 +132,11 @@ struct wnw_cache {
 
   cudaEvent_t ev_place = nullptr, ev_step = nullptr;
   bool place_recorded = false, step_recorded = false;
+  // token-granular compression of fixed heads (allocated by the first wnw_place_prefill_tokens)
+  float *tok_work = nullptr, *tok_p = nullptr, *tok_ret = nullptr;
+  int32_t *tok_flags = nullptr, *fixed_tok = nullptr, *tok_n = nullptr;
+  int tok_cap = 0, tok_fixed_max = 0, tok_last_seq = -1, tok_last_layer = -1;
+  long long tok_p_stride = 0;
   // timing
   bool timing = false;
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> t_used;
@@ -541,7 +547,10 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
     const SeqHost &s = c->seqs[seq_ids[i]];
     for (int h = 0; h < G.Hkv; ++h) {
       const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
-      const int audio = (role == ROLE_ANCHOR ? s.C : role == ROLE_TIDAL ? s.S : s.S_base) * G.gpc;
+      int fixed_blocks = s.S_base;   // a token-compacted fixed head: the blocks its kept positions fill
+      if (role == ROLE_FIXED && !s.fixed_blocks.empty() && s.fixed_blocks[layer * G.Hkv + h] >= 0)
+        fixed_blocks = s.fixed_blocks[layer * G.Hkv + h];
+      const int audio = (role == ROLE_ANCHOR ? s.C : role == ROLE_TIDAL ? s.S : fixed_blocks) * G.gpc;
       n_gran[i * G.Hkv + h] = G.n_tg + audio;
       const int work = G.n_tg + audio - (role == ROLE_TIDAL ? (s.S - s.S_base) * G.gpc / 2 : 0);
       n_work[i * G.Hkv + h] = work;
@@ -748,6 +757,7 @@ extern "C" wnw_status_t wnw_place_prefill_multi(wnw_cache_t *c, int32_t seq, int
       CK(cudaMemcpy(c->cv.mirror + seq, &c->mirror_ptrs[seq], sizeof(bf16 *), cudaMemcpyHostToDevice));
     }
     s.T_a = T_a; s.T_t = T_t; s.C = C_b; s.S = S_b; s.S_base = S_base_b;
+    s.fixed_blocks.clear();
     c->wl_layers.clear();  // dims may have changed
   }
   // the staging buffer and the partial buffers are shared: order after earlier placements and steps
@@ -815,6 +825,116 @@ extern "C" wnw_status_t wnw_place_prefill_multi(wnw_cache_t *c, int32_t seq, int
   c->place_recorded = true;
   c->last_stream = st;
   s.placed_layers = layer + 1;
+  return WNW_OK;
+}
+
+static wnw_status_t check_seq_layer(wnw_cache *c, int seq, int layer);
+static wnw_status_t drain(wnw_cache *c);
+
+// Eq. 1 on the host: retention_i = min(s_tilde_i * lambda, 1).
+extern "C" wnw_status_t wnw_retention_schedule(const float *s_tilde, int32_t n, float lambda, float *retention) {
+  if (!s_tilde || !retention || n < 0 || !(lambda >= 0.f)) return WNW_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (!(s_tilde[i] >= 0.f && s_tilde[i] <= 1.f)) return WNW_ERR_INVALID_ARG;
+    retention[i] = std::min(s_tilde[i] * lambda, 1.0f);
+  }
+  return WNW_OK;
+}
+
+// positions a head keeps: sum over its segments of floor(retention * length), the arithmetic of the selection kernel
+static int kept_positions(int T_a, int seg, float retention) {
+  int n = 0;
+  for (int lo = 0; lo < T_a; lo += seg) n += (int)std::floor((double)retention * (double)std::min(seg, T_a - lo));
+  return n;
+}
+
+extern "C" wnw_status_t wnw_place_prefill_tokens(wnw_cache_t *c, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                                                 int32_t n_tokens, int32_t audio_begin, int32_t audio_end,
+                                                 const void *q_text_dev, int32_t n_queries, const float *retention,
+                                                 int32_t segment_tokens, int32_t variant, void *cuda_stream) {
+  if (!c || !retention || segment_tokens < 1 || variant < 0 || variant > 1) return WNW_ERR_INVALID_ARG;
+  const Geometry &G = c->geo;
+  if (layer < 0 || layer >= G.L || seq < 0 || seq >= G.max_batch) return WNW_ERR_INVALID_ARG;
+  if (audio_begin < 0 || audio_end < audio_begin || audio_end > n_tokens) return WNW_ERR_INVALID_ARG;
+  const bool full = c->cfg.mode == WNW_MODE_FULL;
+  const LayerInfo &li = c->layers[layer];
+  const int T_a = audio_end - audio_begin, n_fixed = full ? 0 : li.n_fixed;
+  const int tok_cap = G.S_max * G.nc;
+  std::vector<int> blocks(G.Hkv, -1);
+  for (int h = 0; h < G.Hkv && n_fixed > 0; ++h) {
+    if (c->roles[layer * G.Hkv + h] != ROLE_FIXED) continue;
+    if (!(retention[h] >= 0.f && retention[h] <= 1.f)) return WNW_ERR_INVALID_ARG;
+    const int n = kept_positions(T_a, segment_tokens, retention[h]);
+    if (n > tok_cap) return WNW_ERR_CAPACITY;   // the head's compact store holds S_max blocks of chunk_tokens rows
+    blocks[h] = (n + G.nc - 1) / G.nc;
+  }
+  wnw_status_t rc = wnw_place_prefill_multi(c, seq, layer, k_dev, v_dev, n_tokens, audio_begin, audio_end, q_text_dev, n_queries,
+                                            cuda_stream);
+  if (rc != WNW_OK || n_fixed == 0 || T_a == 0) return rc;
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  SeqHost &s = c->seqs[seq];
+  if (!c->fixed_tok) {
+    int fmax = 0;
+    for (const LayerInfo &x : c->layers) fmax = std::max(fmax, (int)x.n_fixed);
+    c->tok_fixed_max = fmax; c->tok_cap = tok_cap;
+    c->tok_p_stride = c->cfg.max_audio_tokens;
+    const size_t B = G.max_batch;
+    if ((rc = dev_alloc(c, &c->tok_work, (size_t)fmax * ((size_t)c->cfg.max_text_tokens + c->cfg.max_audio_tokens))) != WNW_OK) return rc;
+    if ((rc = dev_alloc(c, &c->tok_p, (size_t)fmax * c->tok_p_stride)) != WNW_OK) return rc;
+    if ((rc = dev_alloc(c, &c->tok_flags, (size_t)fmax * c->tok_p_stride)) != WNW_OK) return rc;
+    if ((rc = dev_alloc(c, &c->tok_ret, (size_t)G.Hkv)) != WNW_OK) return rc;
+    if ((rc = dev_alloc(c, &c->tok_n, B * std::max(G.F_tot, 1))) != WNW_OK) return rc;
+    if ((rc = dev_alloc(c, &c->fixed_tok, B * std::max(G.F_tot, 1) * (size_t)std::max(tok_cap, 1))) != WNW_OK) return rc;
+  }
+  // the scratch is shared with earlier placements on other streams: the chunk placement above already ordered this
+  // stream after them; the retention values travel through a pageable copy, complete on the host side at return
+  CK(cudaMemcpyAsync(c->tok_ret, retention, (size_t)G.Hkv * sizeof(float), cudaMemcpyHostToDevice, st));
+  CK(launch_token_compress(c->cv, seq, layer, n_fixed, c->stage, (const bf16 *)q_text_dev, n_queries, s.T_t, T_a, segment_tokens,
+                           c->tok_ret, variant, c->tok_work, c->tok_p, c->tok_flags, c->tok_p_stride, c->fixed_tok, c->tok_cap,
+                           c->tok_n, st));
+  CK(cudaEventRecord(c->ev_place, st));
+  if (s.fixed_blocks.empty()) s.fixed_blocks.assign((size_t)G.L * G.Hkv, -1);
+  for (int h = 0; h < G.Hkv; ++h) s.fixed_blocks[layer * G.Hkv + h] = blocks[h];
+  c->wl_layers.clear();
+  c->tok_last_seq = seq; c->tok_last_layer = layer;
+  return WNW_OK;
+}
+
+// per-position prefill scores of one fixed head from the most recent token placement
+extern "C" wnw_status_t wnw_get_token_scores(wnw_cache_t *c, int32_t seq, int32_t layer, int32_t kv_head, float *scores,
+                                             int32_t capacity) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!scores || kv_head < 0 || kv_head >= c->geo.Hkv) return WNW_ERR_INVALID_ARG;
+  if (c->cfg.mode != WNW_MODE_TIERED || c->roles[layer * c->geo.Hkv + kv_head] != ROLE_FIXED) return WNW_ERR_INVALID_ARG;
+  if (!c->tok_p || c->tok_last_seq != seq || c->tok_last_layer != layer) return WNW_ERR_STATE;
+  const int T_a = c->seqs[seq].T_a;
+  if (capacity < T_a) return WNW_ERR_CAPACITY;
+  DeviceGuard guard(c->cfg.device);
+  if ((s = drain(c)) != WNW_OK) return s;
+  const int f = c->role_idx[layer * c->geo.Hkv + kv_head];
+  if (T_a > 0) CK(cudaMemcpy(scores, c->tok_p + (size_t)f * c->tok_p_stride, (size_t)T_a * sizeof(float), cudaMemcpyDeviceToHost));
+  return WNW_OK;
+}
+
+// kept positions (ascending) of a fixed head placed by wnw_place_prefill_tokens
+extern "C" wnw_status_t wnw_get_fixed_tokens(wnw_cache_t *c, int32_t seq, int32_t layer, int32_t kv_head, int32_t *positions,
+                                             int32_t capacity, int32_t *n) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!positions || !n || kv_head < 0 || kv_head >= c->geo.Hkv) return WNW_ERR_INVALID_ARG;
+  if (c->cfg.mode != WNW_MODE_TIERED || c->roles[layer * c->geo.Hkv + kv_head] != ROLE_FIXED) return WNW_ERR_INVALID_ARG;
+  const SeqHost &sq = c->seqs[seq];
+  if (!c->fixed_tok || sq.fixed_blocks.empty() || sq.fixed_blocks[layer * c->geo.Hkv + kv_head] < 0) return WNW_ERR_STATE;
+  DeviceGuard guard(c->cfg.device);
+  if ((s = drain(c)) != WNW_OK) return s;
+  const size_t fh = (size_t)seq * c->geo.F_tot + c->layers[layer].fixed_off + c->role_idx[layer * c->geo.Hkv + kv_head];
+  int32_t cnt = 0;
+  CK(cudaMemcpy(&cnt, c->tok_n + fh, sizeof(cnt), cudaMemcpyDeviceToHost));
+  if (cnt > capacity) return WNW_ERR_CAPACITY;
+  if (cnt > 0) CK(cudaMemcpy(positions, c->fixed_tok + fh * c->tok_cap, (size_t)cnt * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  *n = cnt;
   return WNW_OK;
 }
 
@@ -1277,6 +1397,8 @@ extern "C" wnw_status_t wnw_get_fixed_set(wnw_cache_t *c, int32_t seq, int32_t l
   if (c->cfg.mode != WNW_MODE_TIERED || c->roles[layer * c->geo.Hkv + kv_head] != ROLE_FIXED) return WNW_ERR_INVALID_ARG;
   DeviceGuard guard(c->cfg.device);
   if ((s = drain(c)) != WNW_OK) return s;
+  const SeqHost &sq_ = c->seqs[seq];   // a token-compacted head keeps positions, not chunks: wnw_get_fixed_tokens
+  if (!sq_.fixed_blocks.empty() && sq_.fixed_blocks[layer * c->geo.Hkv + kv_head] >= 0) return WNW_ERR_STATE;
   const size_t fh = (size_t)seq * c->geo.F_tot + c->layers[layer].fixed_off + c->role_idx[layer * c->geo.Hkv + kv_head];
   int32_t cnt = 0;
   CK(cudaMemcpy(&cnt, c->cv.fixed_n + fh, sizeof(cnt), cudaMemcpyDeviceToHost));
@@ -1337,7 +1459,10 @@ extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
       r.host_audio_tokens += (int64_t)li.n_tidal * (sq.T_a - res);
       for (int f = 0; f < li.n_fixed; ++f) {
         const size_t fh = b * G.F_tot + li.fixed_off + f;
-        for (int j = 0; j < fixed_n[fh]; ++j) r.resident_audio_tokens += len_of(sq, fixed_chunks[fh * G.S_max + j]);
+        for (int j = 0; j < fixed_n[fh]; ++j) {   // entries below -1: blocks of a token-compacted head, -(2 + rows)
+          const int ch = fixed_chunks[fh * G.S_max + j];
+          r.resident_audio_tokens += ch < -1 ? -ch - 2 : len_of(sq, ch);
+        }
       }
     }
   }

@@ -49,8 +49,11 @@ def near_tie(scores64, lens, sel_a, sel_b):
 
 class Lockstep:
     def __init__(self, w: Workload, seed=0, device="cuda:0", recall_mode=0, gen_device=None, oracle_seqs=None,
-                 score_scope=0, residency=0, evict_lag=3):
+                 score_scope=0, residency=0, evict_lag=3, token_retention=None, token_seg=25, token_variant=0):
         self.w = w
+        # token-granular compression of fixed heads: retention [n_layers][n_kv_heads], segment size, variant
+        self.tok_ret = None if token_retention is None else np.asarray(token_retention, np.float32)
+        self.tok_seg, self.tok_variant = token_seg, token_variant
         self.dev = torch.device(device)
         self.syn = Synth(w, seed=seed, device=gen_device or "cpu")
         self.oracle_seqs = list(range(w.batch)) if oracle_seqs is None else list(oracle_seqs)
@@ -81,12 +84,23 @@ class Lockstep:
                 p = self.syn.prefill(b, l)
                 qname = "q_text" if "q_text" in p else "q_last"     # all text queries when the workload has several
                 k, v, ql = (p[n].to(self.dev) for n in ("k", "v", qname))
-                wnw.wnw_place_prefill(self.h, b, l, k, v, p["audio_begin"], p["audio_end"], ql)
+                if self.tok_ret is not None:
+                    if ql.dim() == 2:
+                        ql = ql[None]
+                    wnw.wnw_place_prefill_tokens(self.h, b, l, k, v, p["audio_begin"], p["audio_end"], ql, self.tok_ret[l],
+                                                 self.tok_seg, self.tok_variant)
+                else:
+                    wnw.wnw_place_prefill(self.h, b, l, k, v, p["audio_begin"], p["audio_end"], ql)
                 if self.syn.device.type == "cuda":
                     torch.cuda.synchronize(self.dev)   # the generator's buffers are released right after
                 if b in self.oracle_seqs:
                     kb, vb = bf16_bits(p["k"]), bf16_bits(p["v"])
-                    self.o.place_prefill(b, l, kb, vb, p["audio_begin"], p["audio_end"], bf16_bits(p[qname]))
+                    if self.tok_ret is not None:
+                        self.o.place_prefill_tokens(b, l, kb, vb, p["audio_begin"], p["audio_end"], bf16_bits(p[qname]),
+                                                    self.tok_ret[l], self.tok_seg, self.tok_variant)
+                        self.check_token_sets(b, l, p["audio_end"] - p["audio_begin"])
+                    else:
+                        self.o.place_prefill(b, l, kb, vb, p["audio_begin"], p["audio_end"], bf16_bits(p[qname]))
                     self.kept[(b, l)] = (kb[p["audio_begin"]:p["audio_end"]], vb[p["audio_begin"]:p["audio_end"]])
         wnw.wnw_sync(self.h)
         for b in self.oracle_seqs:
@@ -106,6 +120,8 @@ class Lockstep:
                         continue
                     g_pre = wnw.wnw_get_prefill_scores(self.h, b, l, h)
                     assert_scores_close(g_pre, self.o.prefill_scores(b, l, h), f"prefill scores b{b} l{l} h{h}")
+                    if role == ROLE_FIXED and self.tok_ret is not None:
+                        continue                                   # kept positions, checked right after the placement
                     if role == ROLE_FIXED:
                         g_set = wnw.wnw_get_fixed_set(self.h, b, l, h)
                         assert g_set.tolist() == wo.topk(g_pre, lens, S).tolist(), f"fixed set (ii) b{b} l{l} h{h}"
@@ -129,6 +145,35 @@ class Lockstep:
                         self.o.set_residency(b, l, g_tab, g_stamp)
                     if check_slots:
                         self.check_slot_bytes(b, l)
+
+    def check_token_sets(self, b, l, T_a):
+        """Token-compressed fixed heads of (b, l), right after their placement: (i) per-position scores close,
+        (ii) the oracle's selection on the GPU's fp32 scores reproduces the GPU's kept positions bit-exactly,
+        (iii) the oracle's own set agrees or differs only across near-ties (then it adopts the GPU's)."""
+        w = self.w
+        if T_a == 0:
+            return
+        for h in range(w.n_kv_heads):
+            if w.roles[l, h] != ROLE_FIXED:
+                continue
+            g_p = wnw.wnw_get_token_scores(self.h, b, l, h)
+            o_p = self.o.token_scores(b, l, h)
+            assert_scores_close(g_p, o_p, f"token scores b{b} l{l} h{h}")
+            g_pos = wnw.wnw_get_fixed_tokens(self.h, b, l, h)
+            want = wo.select_tokens(g_p, self.tok_seg, float(self.tok_ret[l, h]), self.tok_variant)
+            assert g_pos.tolist() == want.tolist(), f"kept positions (ii) b{b} l{l} h{h}"
+            o_pos = self.o.fixed_tokens(b, l, h)
+            if g_pos.tolist() != o_pos.tolist():
+                assert len(g_pos) == len(o_pos)
+                diff = sorted(set(g_pos.tolist()) ^ set(o_pos.tolist()))
+                groups = {}
+                for t in diff:
+                    groups.setdefault(t // self.tok_seg if self.tok_variant == 0 else 0, []).append(t)
+                for ts in groups.values():
+                    ks = o_p[ts]
+                    assert ks.max() - ks.min() <= TIE_RTOL * max(ks.max(), 1e-30), f"kept positions b{b} l{l} h{h}: {ts}"
+                self.near_ties += 1
+                self.o.set_fixed_tokens(b, l, h, g_pos)
 
     def check_slot_bytes(self, b, l):
         """Slot contents are an exact copy of the source K,V of the chunk the table says is there."""

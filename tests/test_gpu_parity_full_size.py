@@ -122,3 +122,25 @@ def test_config1_whole_decode_graph_replay(residency, seg):
 def wnw_text_len(ls):
     import paper_2608_22704_b200 as wnw
     return wnw.wnw_get_seq_dims(ls.h, 0)[1]
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+def test_config1_token_compressed_fixed_heads(variant):
+    """Config 1 with its fixed heads compressed token by token in the paper's geometry (segments of 25 tokens = 2 s at
+    12.5 tokens/s; per-head retention from Eq. 1 with seeded importances, lambda = 0.18, so a head keeps 0 to 4 positions
+    of every segment of its 3000 audio tokens), four text queries; 12 decode steps replayed as a CUDA graph."""
+    import paper_2608_22704_b200 as wnw
+    from parity_harness import Lockstep
+    w = config1(n_steps=12)
+    w.n_prefill_queries = 4
+    s_tilde = np.random.RandomState(7).rand(w.n_layers * w.n_kv_heads)
+    ret = wnw.wnw_retention_schedule(s_tilde, 0.18).reshape(w.n_layers, w.n_kv_heads)
+    ls = Lockstep(w, seed=2, gen_device="cuda:0", token_retention=ret, token_seg=25, token_variant=variant)
+    try:
+        ls.prefill(check_slots=False)
+        for t in range(12):
+            ls.decode_step(t, graph=True, check_slots=(t == 11))
+        ls.check_stats()
+        assert ls.max_out_err <= 2e-2
+    finally:
+        ls.close()
