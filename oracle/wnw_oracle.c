@@ -54,7 +54,11 @@
  *     printed, Eq. 1 for the per-head retention): p_prefill[tau] = sum over the text queries and the head's q-heads
  *     of the softmax weight of tau; the ranking key is (float)p_prefill[tau], ties to the earlier position; every
  *     segment of `seg` tokens keeps its floor((double)retention * length) best positions (variant 1: the same total
- *     from the whole head); the head then attends to [text | kept positions].  Tidal tables stay chunk-granular.
+ *     from the whole head); the head then attends to [text | kept positions].  Tidal tables stay chunk-granular,
+ *     except with residency 2 (SEGMENT_LAG with a token-granular base): no segment is permanent as a whole; every tidal
+ *     head keeps its own per-segment best positions for good (variant 0 only) and attends to [text | its kept
+ *     positions | all positions of the segments resident in the layer's dynamic slots]; a selected segment that is
+ *     not in a dynamic slot counts as a miss (its complement has to be fetched).
  *     Pinned in tests/test_oracle_tokens.py against numpy sorts, a separate numpy softmax and hand-worked cases.
  */
 #include <math.h>
@@ -95,7 +99,8 @@ typedef struct {
 typedef struct {
   int L, Hq, Hkv, d, g, chunk, topk, max_batch, max_audio, max_text;
   int scope;      /* 0: per layer with nearest-anchor routing; 1: global sum over all anchor layers */
-  int residency;  /* 0: hard budget (fixed pool, least-recently-selected eviction); 1: SEGMENT_LAG */
+  int residency;  /* 0: hard budget (fixed pool, least-recently-selected eviction); 1: SEGMENT_LAG; 2: SEGMENT_LAG with a
+                     token-granular permanent base (tidal heads keep their best positions of every segment) */
   int delta;      /* eviction lag of SEGMENT_LAG */
   double budget, scale;
   uint8_t *roles; /* [L][Hkv] */
@@ -293,7 +298,7 @@ int wnwo_create(int L, int Hq, int Hkv, int d, int max_batch, int max_audio, int
                 double budget, double scale, const uint8_t *roles, int scope, int residency, int delta, Oracle **out) {
   if (!out || !roles || L < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv || d < 1 || max_batch < 1 || chunk < 1 || topk < 1)
     return WNWO_ERR_ARG;
-  if (!(budget > 0.0 && budget <= 1.0) || scope < 0 || scope > 1 || residency < 0 || residency > 1 || delta < 0)
+  if (!(budget > 0.0 && budget <= 1.0) || scope < 0 || scope > 1 || residency < 0 || residency > 2 || delta < 0)
     return WNWO_ERR_ARG;
   Oracle *o = (Oracle *)calloc(1, sizeof(Oracle));
   if (!o) return WNWO_ERR_OOM;
@@ -341,8 +346,9 @@ static int alloc_seq(Oracle *o, Seq *s, int T_a, int T_t) {
   int S = (int)floor(o->budget * (double)s->C + 1e-6);
   if (S < 1) S = 1;
   if (S > s->C) S = s->C;
+  if (o->residency == 2) S = 0; /* no whole segment is permanent: the base is a set of positions per head */
   s->S_base = S;
-  if (o->residency == 1) { /* dynamic slots for everything selected within the last delta+1 steps */
+  if (o->residency >= 1) { /* dynamic slots for everything selected within the last delta+1 steps */
     int D = 2 * o->topk * (o->delta + 1);
     if (D > s->C - S) D = s->C - S;
     S += D;
@@ -387,8 +393,10 @@ static int alloc_seq(Oracle *o, Seq *s, int T_a, int T_t) {
  * the whole probability row [T_t + T_a] (text first), zeros where masked. */
 static void attend(const Oracle *o, const Seq *s, int layer, int kvh, const uint16_t *q, int T_t,
                    const unsigned char *allowed, double *out, double *chunk_mass, double *p_row) {
-  /* a fixed head placed token by token sees exactly its kept positions */
+  /* a fixed head placed token by token sees exactly its kept positions; a tidal head with a token-granular base sees
+   * its kept positions and every position of the segments resident in its layer's dynamic slots */
   const unsigned char *tok = s->tok_mask ? s->tok_mask[layer * o->Hkv + kvh] : NULL;
+  const int tidal_base = o->roles[layer * o->Hkv + kvh] == ROLE_TIDAL;
   const int d = o->d, T_a = s->T_a;
   const uint16_t *tK = s->txtK[layer] + (size_t)kvh * s->T_cap * d, *tV = s->txtV[layer] + (size_t)kvh * s->T_cap * d;
   const uint16_t *aK = s->audK[layer] + (size_t)kvh * T_a * d, *aV = s->audV[layer] + (size_t)kvh * T_a * d;
@@ -399,7 +407,7 @@ static void attend(const Oracle *o, const Seq *s, int layer, int kvh, const uint
     const uint16_t *krow;
     int vis;
     if (i < T_t) { krow = tK + (size_t)i * d; vis = 1; }
-    else { int tau = i - T_t; krow = aK + (size_t)tau * d; vis = tok ? tok[tau] != 0 : allowed[tau / o->chunk] != 0; }
+    else { int tau = i - T_t; krow = aK + (size_t)tau * d; vis = tok ? (tok[tau] != 0 || (tidal_base && allowed[tau / o->chunk] != 0)) : allowed[tau / o->chunk] != 0; }
     if (!vis) { logit[i] = -INFINITY; continue; }
     double acc = 0.0;
     for (int x = 0; x < d; ++x) acc += bf16_to_double(q[x]) * bf16_to_double(krow[x]);
@@ -446,8 +454,8 @@ static void allowed_for(const Oracle *o, const Seq *s, int layer, int kvh, unsig
 /* k,v: [n_tokens][Hkv][d] bf16 bits; audio = [audio_begin, audio_end); q_last: [Hq][d]. */
 /* q_text: [n_q][Hq][d], the text queries whose attention over the audio is aggregated ("Prefill Compression":
  * p_prefill = sum over text queries of their attention weights); n_q = 1 with the last prefix query is the contract's form. */
-int wnwo_place_prefill_multi(Oracle *o, int seq, int layer, const uint16_t *k, const uint16_t *v, int n_tokens,
-                             int audio_begin, int audio_end, const uint16_t *q_last, int n_q) {
+static int place_multi(Oracle *o, int seq, int layer, const uint16_t *k, const uint16_t *v, int n_tokens,
+                       int audio_begin, int audio_end, const uint16_t *q_last, int n_q) {
   if (!o || seq < 0 || seq >= o->max_batch || layer < 0 || layer >= o->L || !k || !v || n_tokens < 0) return WNWO_ERR_ARG;
   if (audio_begin < 0 || audio_end < audio_begin || audio_end > n_tokens || n_q < 1) return WNWO_ERR_ARG;
   const int T_a = audio_end - audio_begin, T_t = n_tokens - T_a, Hkv = o->Hkv, d = o->d;
@@ -523,6 +531,12 @@ int wnwo_place_prefill_multi(Oracle *o, int seq, int layer, const uint16_t *k, c
   return WNWO_OK;
 }
 
+int wnwo_place_prefill_multi(Oracle *o, int seq, int layer, const uint16_t *k, const uint16_t *v, int n_tokens,
+                             int audio_begin, int audio_end, const uint16_t *q_last, int n_q) {
+  if (o && o->residency == 2) return WNWO_ERR_STATE; /* a token-granular base is placed by wnwo_place_prefill_tokens */
+  return place_multi(o, seq, layer, k, v, n_tokens, audio_begin, audio_end, q_last, n_q);
+}
+
 /* Eq. 1: the fraction of audio positions a tidal or fixed head keeps on the GPU, from its normalised importance
  * s_tilde in [0,1] and the scale lambda. */
 void wnwo_retention_schedule(const double *s_tilde, int n, double lambda, double *retention) {
@@ -576,7 +590,8 @@ int wnwo_place_prefill_tokens(Oracle *o, int seq, int layer, const uint16_t *k, 
                               int audio_begin, int audio_end, const uint16_t *q_text, int n_q, const float *retention,
                               int seg, int variant) {
   if (!retention || seg < 1) return WNWO_ERR_ARG;
-  int rc = wnwo_place_prefill_multi(o, seq, layer, k, v, n_tokens, audio_begin, audio_end, q_text, n_q);
+  if (o && o->residency == 2 && variant != 0) return WNWO_ERR_ARG; /* tidal bases keep a per-segment quota */
+  int rc = place_multi(o, seq, layer, k, v, n_tokens, audio_begin, audio_end, q_text, n_q);
   if (rc) return rc;
   Seq *s = &o->seq[seq];
   const int T_a = s->T_a, T_t = s->T_t, Hkv = o->Hkv, d = o->d;
@@ -587,7 +602,8 @@ int wnwo_place_prefill_tokens(Oracle *o, int seq, int layer, const uint16_t *k, 
   int *kept = (int *)malloc(sizeof(int) * T_a);
   memset(all, 1, (size_t)s->C);
   for (int h = 0; h < Hkv; ++h) {
-    if (o->roles[layer * Hkv + h] != ROLE_FIXED) continue;
+    const int role = o->roles[layer * Hkv + h];
+    if (role != ROLE_FIXED && !(role == ROLE_TIDAL && o->residency == 2)) continue;
     if (!(retention[h] >= 0.0f && retention[h] <= 1.0f)) { rc = WNWO_ERR_ARG; break; }
     const int idx = layer * Hkv + h;
     free(s->tok_mask[idx]); s->tok_mask[idx] = NULL; /* the scoring below sees every position */
@@ -731,7 +747,7 @@ int wnwo_step_end(Oracle *o) {
         if (o->src[l] < 0) continue;
         const double *sc = o->scope == 1 ? glob : s->score_sum + (size_t)o->src[l] * C;
         for (int c = 0; c < C; ++c) sf[c] = (float)sc[c];
-        if (o->residency == 1) { /* overlapping chunks, permanent base, lag-delta release */
+        if (o->residency >= 1) { /* overlapping chunks, permanent base, lag-delta release */
           int n_sel = 0, n_rel = 0, hits = 0;
           int n_seg = wnwo_select_segments(sf, lens, C, o->topk, s->sel + (size_t)l * o->topk, &n_sel, segs);
           s->n_sel[l] = n_sel;

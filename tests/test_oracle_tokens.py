@@ -179,3 +179,90 @@ def test_full_retention_equals_dense_attention_and_setter_round_trip():
     T_t = o.dims(0)[1]
     assert sorted(np.nonzero(p_row[T_t:])[0].tolist()) == [3, 9, 77]
     assert abs(p_row.sum() - 1.0) < 1e-12
+
+
+# ---------------------------------------------------------------- tidal heads with a token-granular base (residency 2)
+def _lag_workload():
+    w = tiny_custom(n_layers=2, n_q_heads=6, n_kv_heads=3, head_dim=64, n_text=6, audio_lens=(210,), chunk=25, budget=0.3,
+                    roles=[[A, T, F], [T, T, A]], n_steps=6, topk=2, region=25, jump_every=2)
+    w.n_prefill_queries = 3
+    return w
+
+
+def test_token_base_tidal_heads_against_numpy():
+    """Residency 2: no segment is permanent as a whole; a tidal head sees [text | its kept positions | every position of the
+    segments in its layer's dynamic slots].  Checked against numpy attention over exactly that key set, with the table
+    advanced by the (separately pinned) lag update; retention 0 leaves a head with the fetched segments only, retention 1
+    makes it plain dense attention."""
+    w = _lag_workload()
+    syn = Synth(w, seed=11)
+    o = make_oracle(w, score_scope=1, residency=2, evict_lag=1)
+    seg = w.chunk
+    ret = np.array([[1.0, 0.3, 0.5], [0.0, 1.0, 1.0]], np.float32)
+    scale = 1 / math.sqrt(w.head_dim)
+    pre = {}
+    with pytest.raises(wo.OracleError):                     # the chunk-granular placement has no base to offer here
+        p = syn.prefill(0, 0)
+        o.place_prefill(0, 0, bf16_bits(p["k"]), bf16_bits(p["v"]), p["audio_begin"], p["audio_end"], bf16_bits(p["q_text"]))
+    for l in range(2):
+        p = syn.prefill(0, l)
+        kb, vb, qt = bf16_bits(p["k"]), bf16_bits(p["v"]), bf16_bits(p["q_text"])
+        with pytest.raises(wo.OracleError):                 # tidal bases keep a per-segment quota: no global variant
+            o.place_prefill_tokens(0, l, kb, vb, p["audio_begin"], p["audio_end"], qt, ret[l], seg, 1)
+        o.place_prefill_tokens(0, l, kb, vb, p["audio_begin"], p["audio_end"], qt, ret[l], seg, 0)
+        pre[l] = (bf16_bits_to_f64(kb), bf16_bits_to_f64(vb), qt, p["audio_begin"], p["audio_end"])
+    T_a, T_t, C, S = o.dims(0)
+    assert (C, S, o.base_slots(0)) == (9, 2 * 2 * 2, 0)      # D = 2*topk*(delta+1) dynamic slots, no permanent ones
+    kept = {}
+    for l in range(2):
+        K, V, qt, ab, ae = pre[l]
+        tab, _ = o.residency(0, l)
+        assert (tab == -1).all()                              # nothing fetched yet
+        for h in range(3):
+            if w.roles[l, h] == A:
+                continue
+            want = np.zeros(T_a)
+            for qi in range(3):
+                for r in range(2):
+                    _, prob = dense_attention(bf16_bits_to_f64(qt[qi, h * 2 + r]), K[:, h], V[:, h], scale)
+                    want += prob[ab:ae]
+            k32 = want.astype(np.float32).astype(np.float64)
+            exp = []
+            for lo in range(0, T_a, seg):
+                n = min(seg, T_a - lo)
+                m = int(math.floor(float(ret[l, h]) * n))
+                exp += sorted((lo + np.argsort(-k32[lo:lo + n], kind="stable")[:m]).tolist())
+            kept[(l, h)] = o.fixed_tokens(0, l, h)
+            assert kept[(l, h)].tolist() == exp
+    assert len(kept[(1, 0)]) == 0 and len(kept[(1, 1)]) == T_a
+    dec = {l: syn.decode(0, l) for l in range(2)}
+    extra = {l: ([], []) for l in range(2)}
+    seen_fetch = False
+    for t in range(w.n_steps):
+        tabs = {l: o.residency(0, l)[0] for l in range(2)}    # what attention of this step sees
+        o.step_begin([0])
+        for l in range(2):
+            q, kn, vn = (bf16_bits(dec[l][n][t]) for n in ("q", "k_new", "v_new"))
+            out = o.decode_layer(l, q[None], kn[None], vn[None])
+            extra[l][0].append(bf16_bits_to_f64(kn)); extra[l][1].append(bf16_bits_to_f64(vn))
+            K, V, _, ab, ae = pre[l]
+            text = [i for i in range(K.shape[0]) if not (ab <= i < ae)]
+            for h in range(3):
+                if w.roles[l, h] == A:
+                    continue
+                vis = set(kept[(l, h)].tolist())
+                if w.roles[l, h] == T:
+                    for c in tabs[l]:
+                        if c >= 0:
+                            vis |= set(range(c * seg, min((c + 1) * seg, T_a)))
+                            seen_fetch = True
+                rows = sorted(vis)
+                Kh = np.concatenate([K[text, h], np.stack([x[h] for x in extra[l][0]]), K[ab:ae, h][rows]])
+                Vh = np.concatenate([V[text, h], np.stack([x[h] for x in extra[l][1]]), V[ab:ae, h][rows]])
+                for r in range(2):
+                    ref, _ = dense_attention(bf16_bits_to_f64(q[h * 2 + r]), Kh, Vh, scale)
+                    assert np.abs(out[0, h * 2 + r] - ref).max() < 1e-12
+        o.step_end()
+    assert seen_fetch
+    st = o.stats(0)
+    assert st["misses"] > 0 and st["evictions"] > 0           # segments were fetched and released again
