@@ -661,11 +661,12 @@ def run_ours(args, rank, world, local_rank):
         n_pf, n_bb = 40, 32
         wq = make_workload(args.workload, W + n_pf + n_bb, 0)
         wq.chunk = 50 if args.workload == "cfg2" else 25
-        jq = Job(wq, seed=0, device=dev, wnw=wnw, score_scope=wnw.WNW_SCOPE_GLOBAL, residency=wnw.WNW_RESIDENCY_SEGMENT_LAG, evict_lag=3)
+        jq = Job(wq, seed=0, device=dev, wnw=wnw, score_scope=wnw.WNW_SCOPE_GLOBAL, residency=wnw.WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE,
+                 evict_lag=3)
         jq.create("wnw", wnw.WNW_MODE_TIERED)
         jq.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
-        # fixed heads: token-granular per-segment top-k with per-head retention from Eq. 1 (seeded importances in [0,1],
-        # lambda = 2 x budget, so the mean retention is the budget)
+        # tidal bases and fixed heads: token-granular per-segment top-k with per-head retention from Eq. 1 (seeded
+        # importances in [0,1], lambda = 2 x budget, so the mean retention is the budget)
         lam_q = 2.0 * wq.budget
         ret_q = wnw.wnw_retention_schedule(np.random.RandomState(0).rand(wq.n_layers * wq.n_kv_heads), lam_q)
         jq.place_all(["wnw", "skip"], token=(ret_q.reshape(wq.n_layers, wq.n_kv_heads), wq.chunk, 0))
@@ -681,7 +682,7 @@ def run_ours(args, rank, world, local_rank):
         T_a_q, _, C_q, S_q = wnw.wnw_get_seq_dims(jq.caches["wnw"], 0)
         paper_form = {"segment_tokens": wq.chunk, "segments": C_q, "slots": S_q, "base_slots": wnw.wnw_get_base_slots(jq.caches["wnw"], 0),
                       "evict_lag": 3, "score_scope": "global",
-                      "fixed_heads": f"token-granular, per segment top floor(retention*n_s); retention = min(s*{lam_q:g}, 1), s ~ U[0,1] seeded",
+                      "prefill_compression": f"token-granular for tidal bases and fixed heads: per segment top floor(retention*n_s); retention = min(s*{lam_q:g}, 1), s ~ U[0,1] seeded",
                       "step_us": ms_q * 1e3, "tokens_per_s": wq.batch / (ms_q * 1e-3),
                       "back_to_back_step_us": ms_q_bb * 1e3, "back_to_back_exposed_recall_us": (ms_q_bb - ms_q_bb_skip) * 1e3,
                       "recall_bytes_per_step": (st1["recall_bytes"] - st0["recall_bytes"]) / (n_pf + n_bb),

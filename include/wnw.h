@@ -80,8 +80,17 @@ enum { WNW_SCOPE_PER_LAYER = 0, WNW_SCOPE_GLOBAL = 1 };
  *                for good; the missing segments of the selected chunks are fetched into 2*topk*(evict_lag+1) further
  *                slots (never short), and a fetched segment left unselected for evict_lag consecutive steps is dropped
  *                (its host copy persists).  Fixed heads keep S_base segments.  wnw_get_seq_dims reports all slots;
- *                wnw_get_base_slots the permanent ones. */
-enum { WNW_RESIDENCY_HARD_BUDGET = 0, WNW_RESIDENCY_SEGMENT_LAG = 1 };
+ *                wnw_get_base_slots the permanent ones.
+ *   SEGMENT_LAG_TOKEN_BASE  SEGMENT_LAG with the permanent base kept token by token ("Prefill Compression" as printed):
+ *                no segment is permanent as a whole (wnw_get_base_slots = 0; a table has only the 2*topk*(evict_lag+1)
+ *                dynamic slots).  Every tidal head keeps for good, in a compact store of its own, its best
+ *                floor(retention*length) positions of every segment (by its own prefill score); the host mirror holds
+ *                each segment with the positions that are NOT in the base first, so a fetched segment contributes
+ *                exactly its complement.  A tidal head attends to [text | its kept positions | the complements of the
+ *                segments in the layer's dynamic slots].  Sequences must be placed with wnw_place_prefill_tokens
+ *                (segment_tokens = chunk_tokens, variant 0); wnw_place_prefill and _multi return WNW_ERR_STATE.
+ *                A compact store holds floor(budget*C)+2*topk*(evict_lag+1) blocks of chunk_tokens positions. */
+enum { WNW_RESIDENCY_HARD_BUDGET = 0, WNW_RESIDENCY_SEGMENT_LAG = 1, WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE = 2 };
 
 /* How recall copies are issued (for measurement; results are identical for 0 and 1):
  *   0  side stream, overlapped with the following layers (default)
@@ -158,9 +167,14 @@ wnw_status_t wnw_place_prefill_multi(wnw_cache_t *cache, int32_t seq, int32_t la
  *   variant 1   : the same number of positions taken from the whole head with no per-segment quota (the paper's
  *                 global top-k ablation of the prefill selection).
  * The kept positions, in ascending order, fill the head's compact store; decode attends to [text | kept positions].
- *   retention   : HOST pointer, [n_kv_heads] floats in [0,1]; entries of heads that are not fixed in this layer are
- *                 ignored.  A head may keep at most S_max * chunk_tokens positions (the capacity of its store, S_max
- *                 the slots of a tidal table at max_audio_tokens): WNW_ERR_CAPACITY otherwise, nothing placed.
+ *   retention   : HOST pointer, [n_kv_heads] floats in [0,1]; entries of heads that are not compressed in this layer
+ *                 (anchor heads; tidal heads unless the residency is SEGMENT_LAG_TOKEN_BASE) are ignored.  A head may
+ *                 keep at most as many positions as its compact store holds (the slots of a tidal table at
+ *                 max_audio_tokens, under the lag residencies the budget's share plus the dynamic slots, times
+ *                 chunk_tokens): WNW_ERR_CAPACITY otherwise, nothing placed.
+ * With the residency SEGMENT_LAG_TOKEN_BASE the layer's tidal heads are compressed the same way, each by its own
+ * scores (their tables start empty); then segment_tokens must equal chunk_tokens and variant must be 0
+ * (WNW_ERR_UNSUPPORTED otherwise).
  * Scratch and the position lists are allocated by the first call (device memory; not allocation-free).  In FULL mode
  * this is wnw_place_prefill_multi.  Errors as wnw_place_prefill; WNW_ERR_INVALID_ARG for a retention outside [0,1],
  * segment_tokens < 1 or an unknown variant. */

@@ -143,14 +143,23 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
     len -= off;
     r.meta = len <= 0 ? 0 : (len < GR ? len : GR);
     if (a.score_on) r.score_idx = ag;
+  } else if (it.role == ROLE_TIDAL && G.token_base && ci < it.S) {
+    // token-granular permanent base: the first it.S units of the head are blocks of its compact store
+    const int head = G.F_fix + li.tid_prefix + it.ridx;
+    r.row = (int)(compact_off(G, it.b, head, 0) / G.d) + ci * G.ncp + off;
+    r.cid = cv.fixed_chunks[((long long)it.b * G.F_tot + head) * G.FB + ci];
+    r.meta = -2;
+    r.score_idx = -2;               // marks the compact store (tensor map and K-to-V row distance differ from the pool's)
   } else if (it.role == ROLE_TIDAL) {
-    r.row = (int)(pool_off(G, li, it.b, ci, it.ridx, 0) / G.d) + off;
-    r.cid = cv.slot_chunk[((long long)it.b * G.L + a.layer) * G.S_max + ci];
-    r.meta = ci < it.S ? -2 : -3;   // beyond the permanent slots a slot may be empty: its rows are fetched only if it is not
+    const int slot = G.token_base ? ci - it.S : ci;
+    r.row = (int)(pool_off(G, li, it.b, slot, it.ridx, 0) / G.d) + off;
+    r.cid = cv.slot_chunk[((long long)it.b * G.L + a.layer) * G.S_max + slot];
+    // beyond the permanent slots a slot may be empty: its rows are fetched only if it is not
+    r.meta = (G.token_base || ci >= it.S) ? -3 : -2;
   } else {
     const long long fh = (long long)it.b * G.F_tot + li.fixed_off + it.ridx;
     r.row = (int)(fixed_off(G, li, it.b, it.ridx, 0) / G.d) + ci * G.ncp + off;
-    r.cid = cv.fixed_chunks[fh * G.S_max + ci];
+    r.cid = cv.fixed_chunks[fh * G.FB + ci];
     r.meta = -2;
   }
   return r;
@@ -217,6 +226,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   struct Ctx {
     WorkItem it;
     int item_idx, T_t, v_delta_audio, first, n_my;
+    int m_full, m_tail;   // token-granular base: positions of a full / of the last segment that live in the base already
     const CUtensorMap *map_audio;
   };
   // Replayed steps: the recall that refreshed this layer's slots ran outside the captured graph, possibly still
@@ -245,7 +255,12 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     c.T_t = cv.text_len[c.it.b] + a.has_new;
     if (c.it.role == ROLE_ANCHOR) { c.v_delta_audio = G.T_a_pad; c.map_audio = &maps.anchor; }       // rows between a
     else if (c.it.role == ROLE_TIDAL) { c.v_delta_audio = G.ncp; c.map_audio = &maps.pool; }          // granule's K and
-    else { c.v_delta_audio = G.S_max * G.ncp; c.map_audio = &maps.fixed; }                            // V rows
+    else { c.v_delta_audio = G.FB * G.ncp; c.map_audio = &maps.fixed; }                            // V rows
+    c.m_full = c.m_tail = 0;
+    if (G.token_base && c.it.role == ROLE_TIDAL) {
+      const int2 m = cv.tok_m[((long long)c.it.b * G.L + a.layer) * G.Hkv + c.it.h];
+      c.m_full = m.x; c.m_tail = m.y;
+    }
     c.first = c.it.g0 + warp;
     c.n_my = c.first < c.it.g1 ? (c.it.g1 - c.first + NW - 1) / NW : 0;
     if (for_loads) epoch_pending = a.wait_epoch != nullptr && c.it.role == ROLE_TIDAL;   // see wait_recall_epoch
@@ -269,7 +284,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       if (cid < -1) len = -cid - 2;   // a block of a token-compacted fixed head: the entry carries its row count
       else {
         len = c.it.T_a - cid * G.nc;
-        if (len > G.nc) len = G.nc;
+        if (len > G.nc) { len = G.nc; len -= c.m_full; }
+        else len -= c.m_tail;   // the last segment; a fetched segment holds its complement first (m = 0 without a token base)
       }
       len -= off;
     }
@@ -293,15 +309,17 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     const int row = __shfl_sync(0xffffffffu, blk.row, src_lane);
     const int j = c.first + n * NW;
     const bool is_text = j < G.n_tg;
-    if (epoch_pending && !is_text) wait_recall_epoch();
+    // a block of a tidal head's permanent token base: compact store, never touched by the recall
+    const bool base_blk = G.token_base && __shfl_sync(0xffffffffu, blk.score_idx, src_lane) == -2;
+    if (epoch_pending && !is_text && !base_blk) wait_recall_epoch();
     bool load = meta != 0;
     if (meta == -1) load = visible(c, -1, 0, 0, j) > 0;  // waits for the text length
     if (meta == -3) load = __shfl_sync(0xffffffffu, blk.cid, src_lane) >= 0;  // waits for the table entry
     if (load && lane == 0) {
       const int stage = (int)(seq % NSTAGE);
       const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB, bar = smem_u32(&bars[warp][stage]);
-      const CUtensorMap *map = is_text ? &maps.text : c.map_audio;
-      const int vrow = row + (is_text ? v_delta_text : c.v_delta_audio);
+      const CUtensorMap *map = is_text ? &maps.text : (base_blk ? &maps.fixed : c.map_audio);
+      const int vrow = row + (is_text ? v_delta_text : (base_blk ? G.FB * G.ncp : c.v_delta_audio));
       fence_proxy_async();  // the stage was last read through the generic proxy (ldmatrix)
       mbar_expect_tx(bar, 2 * TILEB);
 #pragma unroll

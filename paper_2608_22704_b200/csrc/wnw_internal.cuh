@@ -54,7 +54,10 @@ struct Geometry {
   int32_t ncp;                              // rows a chunk occupies in every store: nc rounded up to whole granules
   int32_t T_cap_pad, n_tg;         // text capacity (multiple of 16) and its granules
   int32_t C_max, S_max, T_a_pad;   // chunk / slot capacity per sequence; audio capacity padded to whole chunks
-  int32_t A_tot, F_tot;            // anchor / fixed heads per sequence over all layers
+  int32_t A_tot, F_tot;            // anchor heads / heads with a compact store per sequence over all layers
+  int32_t F_fix;                   // of those, the fixed heads (they come first); the rest are tidal heads' token bases
+  int32_t FB;                      // blocks of chunk_tokens rows a compact store holds
+  int32_t token_base;              // SEGMENT_LAG with a token-granular permanent base (no permanent slots)
   int32_t lag_mode, delta, plan_cap;  // SEGMENT_LAG residency; its eviction lag; plan entries per (sequence, layer)
   int32_t max_batch;
   long long text_seq_stride, anchor_seq_stride, pool_seq_stride, fixed_seq_stride;  // elements
@@ -82,7 +85,8 @@ struct CacheView {
   float *score_sum;                  // [B][L][C_max]
   int32_t *sel, *n_sel;              // [B][L][topk], [B][L]
   int32_t *plan, *n_plan;            // [B][L][plan_cap][2] (chunk, slot), [B][L]
-  int32_t *fixed_chunks, *fixed_n;   // [B][F_tot][S_max], [B][F_tot]
+  int32_t *fixed_chunks, *fixed_n;   // [B][F_tot][FB], [B][F_tot]
+  int2 *tok_m;                       // [B][L][Hkv] token-granular tidal base: kept positions of a full / the last segment
   float *pre;                        // [B][L][Hkv][C_max]
   unsigned long long *stats;         // [B][4] hits, misses, evictions, recall_bytes
   bf16 **mirror;                     // [B] pinned host mirrors (device-visible addresses)
@@ -100,7 +104,11 @@ __host__ __device__ inline long long pool_off(const Geometry &G, const LayerInfo
   return (long long)b * G.pool_seq_stride + li.pool_off + ((long long)(slot * li.n_tidal + t_idx) * 2 + kv) * G.ncp * G.d;
 }
 __host__ __device__ inline long long fixed_off(const Geometry &G, const LayerInfo &li, int b, int f_idx, int kv) {
-  return (long long)b * G.fixed_seq_stride + ((long long)(li.fixed_off + f_idx) * 2 + kv) * G.S_max * G.ncp * G.d;
+  return (long long)b * G.fixed_seq_stride + ((long long)(li.fixed_off + f_idx) * 2 + kv) * G.FB * G.ncp * G.d;
+}
+// compact store of a head by its index among the heads that have one (fixed heads first, then tidal token bases)
+__host__ __device__ inline long long compact_off(const Geometry &G, int b, int head, int kv) {
+  return (long long)b * G.fixed_seq_stride + ((long long)head * 2 + kv) * G.FB * G.ncp * G.d;
 }
 __host__ __device__ inline long long mirror_off(const Geometry &G, const LayerInfo &li, int C_b, int c, int t_idx, int kv) {
   return (((long long)C_b * li.tid_prefix + (long long)c * li.n_tidal + t_idx) * 2 + kv) * G.ncp * G.d;
@@ -208,10 +216,10 @@ cudaError_t launch_prefill_select(const CacheView &cv, int b, int layer, const H
 cudaError_t launch_place_gather(const CacheView &cv, int b, int layer, int full_mode, const bf16 *stage, int C_b,
                                 cudaStream_t st);
 // token-granular compression of the layer's fixed heads (after the chunk-granular placement staged the prefix)
-cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_fixed, const bf16 *stage, const bf16 *q_text,
-                                  int n_q, int T_t, int T_a, int seg, const float *retention_dev, int variant, float *work,
-                                  float *p_tok, int32_t *flags, long long p_stride, int32_t *fixed_tok, int tok_cap,
-                                  int32_t *tok_n, cudaStream_t st);
+cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_comp, int n_tidal_base, const bf16 *stage,
+                                  const bf16 *q_text, int n_q, int T_t, int T_a, int seg, const float *retention_dev,
+                                  int variant, float *work, float *p_tok, int32_t *flags, long long p_stride,
+                                  int32_t *fixed_tok, int tok_cap, int32_t *tok_n, cudaStream_t st);
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
 cudaError_t configure_attn_kernels();
 // Encodes the descriptor of one store: base (device), rows, head_dim.  Returns false if the driver refuses.

@@ -452,7 +452,7 @@ __global__ void __launch_bounds__(512) wnw_prefill_select_kernel(const __grid_co
       const unsigned long long me = skey[c];
       int rank = 0;
       for (int x = 0; x < C_b; ++x) rank += skey[x] > me;
-      if (rank < S_b) cv.fixed_chunks[fh * G.S_max + rank] = c;
+      if (rank < S_b) cv.fixed_chunks[fh * G.FB + rank] = c;
     }
     if (tid == 0) cv.fixed_n[fh] = S_b;
     __syncthreads();
@@ -503,7 +503,7 @@ __global__ void __launch_bounds__(128) wnw_place_gather_kernel(const __grid_cons
     const long long fh = (long long)b * G.F_tot + li.fixed_off + ridx;
     int pos = -1;
     for (int s = 0; s < cv.fixed_n[fh]; ++s)
-      if (cv.fixed_chunks[fh * G.S_max + s] == c) pos = s;
+      if (cv.fixed_chunks[fh * G.FB + s] == c) pos = s;
     if (pos < 0) return;
     for (int kv = 0; kv < 2; ++kv) dst0[kv] = cv.fixed + fixed_off(G, li, b, ridx, kv) + (long long)pos * G.ncp * G.d;
   } else {

@@ -21,7 +21,8 @@ struct SeqHost {
   int T_a = 0, T_t = 0, C = 0, S = 0, S_base = 0;   // S: all slots of a tidal table; S_base: the permanent ones
   bf16 *mirror = nullptr;
   size_t mirror_bytes = 0;
-  std::vector<int> fixed_blocks;   // [L][Hkv] blocks of a token-compacted fixed head's store; empty or -1: S_base chunks
+  std::vector<int> fixed_blocks;   // [L][Hkv] blocks of a token-compacted head's store; empty or -1: S_base chunks
+  std::vector<int2> tok_m;         // [L][Hkv] tidal token bases: kept positions of a full / of the last segment
 };
 
 struct LayerWork {
@@ -164,10 +165,22 @@ static int slots_for(float budget, int C) {
   return S;
 }
 // All slots of a tidal table: under SEGMENT_LAG the permanent ones plus room for everything selected within the last
-// evict_lag + 1 steps (two segments per chunk), so a miss always finds a free slot.
+// evict_lag + 1 steps (two segments per chunk), so a miss always finds a free slot.  With a token-granular base no
+// slot is permanent.
+static bool lag_residency(const wnw_config_t &cfg) { return cfg.residency != WNW_RESIDENCY_HARD_BUDGET; }
+static int base_slots_for(const wnw_config_t &cfg, int C) {
+  return cfg.residency == WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE ? 0 : slots_for(cfg.budget, C);
+}
 static int slots_total(const wnw_config_t &cfg, int C) {
+  const int base = base_slots_for(cfg, C);
+  if (!lag_residency(cfg) || C <= 0) return base;
+  return base + std::min(2 * cfg.topk * (cfg.evict_lag + 1), C - base);
+}
+// Blocks of chunk_tokens rows in a head's compact store (fixed heads; tidal token bases): the budget's share plus, under
+// the lag residencies, as many blocks again as a table has dynamic slots (per-head retentions spread around the budget).
+static int compact_blocks(const wnw_config_t &cfg, int C) {
   const int base = slots_for(cfg.budget, C);
-  if (cfg.residency != WNW_RESIDENCY_SEGMENT_LAG || C <= 0) return base;
+  if (!lag_residency(cfg) || C <= 0) return base;
   return base + std::min(2 * cfg.topk * (cfg.evict_lag + 1), C - base);
 }
 
@@ -237,7 +250,7 @@ static wnw_status_t validate_config(const wnw_config_t *cfg) {
   if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return WNW_ERR_INVALID_ARG;
   if (cfg->mode != WNW_MODE_TIERED && cfg->mode != WNW_MODE_FULL) return WNW_ERR_INVALID_ARG;
   if (cfg->score_scope != WNW_SCOPE_PER_LAYER && cfg->score_scope != WNW_SCOPE_GLOBAL) return WNW_ERR_INVALID_ARG;
-  if (cfg->residency != WNW_RESIDENCY_HARD_BUDGET && cfg->residency != WNW_RESIDENCY_SEGMENT_LAG) return WNW_ERR_INVALID_ARG;
+  if (cfg->residency < WNW_RESIDENCY_HARD_BUDGET || cfg->residency > WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE) return WNW_ERR_INVALID_ARG;
   if (cfg->recall_mode < WNW_RECALL_SIDE_STREAM || cfg->recall_mode > WNW_RECALL_SKIP) return WNW_ERR_INVALID_ARG;
   if (cfg->device < 0) return WNW_ERR_INVALID_ARG;
   bool any_anchor = false, any_tidal = false;
@@ -288,7 +301,9 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   G.n_tg = G.T_cap_pad / GR;
   G.C_max = (cfg->max_audio_tokens + nc - 1) / nc;
   G.S_max = full ? 0 : slots_total(c->cfg, G.C_max);
-  G.lag_mode = !full && c->cfg.residency == WNW_RESIDENCY_SEGMENT_LAG;
+  G.FB = full ? 0 : compact_blocks(c->cfg, G.C_max);
+  G.lag_mode = !full && lag_residency(c->cfg);
+  G.token_base = !full && c->cfg.residency == WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE;
   G.delta = c->cfg.evict_lag;
   G.plan_cap = G.lag_mode ? 2 * G.topk : G.topk;
   G.T_a_pad = std::max(G.C_max, 1) * G.ncp;
@@ -333,11 +348,12 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     c->upd_list.insert(c->upd_list.end(), upd[l].begin(), upd[l].end());
   }
   G.A_tot = full ? L * Hkv : a_tot;
-  G.F_tot = full ? 0 : f_tot;
+  G.F_fix = full ? 0 : f_tot;
+  G.F_tot = full ? 0 : f_tot + (G.token_base ? t_tot : 0);   // tidal heads keep their token base in a compact store too
   G.text_seq_stride = (long long)L * Hkv * 2 * G.T_cap_pad * d;
   G.anchor_seq_stride = (long long)G.A_tot * 2 * G.T_a_pad * d;
   G.pool_seq_stride = full ? 0 : pool_elems;
-  G.fixed_seq_stride = (long long)G.F_tot * 2 * G.S_max * G.ncp * d;
+  G.fixed_seq_stride = (long long)G.F_tot * 2 * G.FB * G.ncp * d;
 
   CacheView &cv = c->cv;
   memset(&cv, 0, sizeof(cv));
@@ -371,8 +387,9 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   CKC(dev_alloc(c, &cv.score_sum, B * L * std::max(G.C_max, 1)));
   CKC(dev_alloc(c, &cv.sel, B * L * G.topk)); CKC(dev_alloc(c, &cv.n_sel, B * L));
   CKC(dev_alloc(c, &cv.plan, B * L * G.plan_cap * 2)); CKC(dev_alloc(c, &cv.n_plan, B * L));
-  CKC(dev_alloc(c, &cv.fixed_chunks, B * std::max(G.F_tot, 1) * std::max(G.S_max, 1)));
+  CKC(dev_alloc(c, &cv.fixed_chunks, B * std::max(G.F_tot, 1) * std::max(G.FB, 1)));
   CKC(dev_alloc(c, &cv.fixed_n, B * std::max(G.F_tot, 1)));
+  CKC(dev_alloc(c, &cv.tok_m, G.token_base ? B * (size_t)L * Hkv : 1));
   CKC(dev_alloc(c, &cv.pre, B * L * Hkv * std::max(G.C_max, 1)));
   CKC(dev_alloc(c, &cv.stats, B * 4));
   CKC(dev_alloc(c, &cv.mirror, B));
@@ -547,10 +564,11 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
     const SeqHost &s = c->seqs[seq_ids[i]];
     for (int h = 0; h < G.Hkv; ++h) {
       const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
-      int fixed_blocks = s.S_base;   // a token-compacted fixed head: the blocks its kept positions fill
-      if (role == ROLE_FIXED && !s.fixed_blocks.empty() && s.fixed_blocks[layer * G.Hkv + h] >= 0)
-        fixed_blocks = s.fixed_blocks[layer * G.Hkv + h];
-      const int audio = (role == ROLE_ANCHOR ? s.C : role == ROLE_TIDAL ? s.S : fixed_blocks) * G.gpc;
+      int fixed_blocks = s.S_base;   // a token-compacted head: the blocks its kept positions fill
+      if (!s.fixed_blocks.empty() && s.fixed_blocks[layer * G.Hkv + h] >= 0) fixed_blocks = s.fixed_blocks[layer * G.Hkv + h];
+      // a tidal head with a token base: its blocks first, then the table's (all dynamic) slots
+      const int tidal_units = s.S + (G.token_base && mode == ATTN_DECODE ? fixed_blocks : 0);
+      const int audio = (role == ROLE_ANCHOR ? s.C : role == ROLE_TIDAL ? tidal_units : fixed_blocks) * G.gpc;
       n_gran[i * G.Hkv + h] = G.n_tg + audio;
       const int work = G.n_tg + audio - (role == ROLE_TIDAL ? (s.S - s.S_base) * G.gpc / 2 : 0);
       n_work[i * G.Hkv + h] = work;
@@ -581,7 +599,10 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       HeadItems hi{(int)items.size() - lw.first_item, n_cta};
       for (int x = 0; x < n_cta; ++x) {  // even contiguous ranges
         const int g0 = (int)((long long)n * x / n_cta), g1 = (int)((long long)n * (x + 1) / n_cta);
-        items.push_back(WorkItem{(int)i, h, g0, g1, seq_ids[i], role, ridx, sq.T_a, sq.C, sq.S_base, sq.T_t});
+        // S: the head's leading permanent units: slots of the table, or blocks of a tidal head's token base
+        const int perm = (G.token_base && role == ROLE_TIDAL && !sq.fixed_blocks.empty()) ? std::max(sq.fixed_blocks[layer * G.Hkv + h], 0)
+                                                                                         : sq.S_base;
+        items.push_back(WorkItem{(int)i, h, g0, g1, seq_ids[i], role, ridx, sq.T_a, sq.C, perm, sq.T_t});
       }
       heads.push_back(hi);
       lw.max_count = std::max(lw.max_count, hi.count);
@@ -716,9 +737,21 @@ extern "C" wnw_status_t wnw_place_prefill(wnw_cache_t *c, int32_t seq, int32_t l
   return wnw_place_prefill_multi(c, seq, layer, k_dev, v_dev, n_tokens, audio_begin, audio_end, q_last_dev, 1, cuda_stream);
 }
 
+static wnw_status_t place_multi(wnw_cache_t *c, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                                int32_t n_tokens, int32_t audio_begin, int32_t audio_end, const void *q_last_dev,
+                                int32_t n_queries, void *cuda_stream);
+
 extern "C" wnw_status_t wnw_place_prefill_multi(wnw_cache_t *c, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
                                                 int32_t n_tokens, int32_t audio_begin, int32_t audio_end,
                                                 const void *q_last_dev, int32_t n_queries, void *cuda_stream) {
+  // a token-granular base is placed by wnw_place_prefill_tokens only
+  if (c && c->geo.token_base) return WNW_ERR_STATE;
+  return place_multi(c, seq, layer, k_dev, v_dev, n_tokens, audio_begin, audio_end, q_last_dev, n_queries, cuda_stream);
+}
+
+static wnw_status_t place_multi(wnw_cache_t *c, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                                int32_t n_tokens, int32_t audio_begin, int32_t audio_end, const void *q_last_dev,
+                                int32_t n_queries, void *cuda_stream) {
   if (!c || !k_dev || !v_dev || n_queries < 1) return WNW_ERR_INVALID_ARG;
   const Geometry &G = c->geo;
   if (seq < 0 || seq >= G.max_batch || layer < 0 || layer >= G.L || n_tokens < 1) return WNW_ERR_INVALID_ARG;
@@ -730,7 +763,7 @@ extern "C" wnw_status_t wnw_place_prefill_multi(wnw_cache_t *c, int32_t seq, int
   SeqHost &s = c->seqs[seq];
   if (layer != 0 && (layer != s.placed_layers || T_a != s.T_a || T_t != s.T_t)) return WNW_ERR_STATE;
   const int C_b = (T_a + G.nc - 1) / G.nc, S_b = full ? 0 : slots_total(c->cfg, C_b);
-  const int S_base_b = full ? 0 : slots_for(c->cfg.budget, C_b);
+  const int S_base_b = full ? 0 : base_slots_for(c->cfg, C_b);
   if (!full && C_b > 0 && !q_last_dev) return WNW_ERR_INVALID_ARG;
   DeviceGuard guard(c->cfg.device);
   cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -757,7 +790,7 @@ extern "C" wnw_status_t wnw_place_prefill_multi(wnw_cache_t *c, int32_t seq, int
       CK(cudaMemcpy(c->cv.mirror + seq, &c->mirror_ptrs[seq], sizeof(bf16 *), cudaMemcpyHostToDevice));
     }
     s.T_a = T_a; s.T_t = T_t; s.C = C_b; s.S = S_b; s.S_base = S_base_b;
-    s.fixed_blocks.clear();
+    s.fixed_blocks.clear(); s.tok_m.clear();
     c->wl_layers.clear();  // dims may have changed
   }
   // the staging buffer and the partial buffers are shared: order after earlier placements and steps
@@ -858,25 +891,31 @@ extern "C" wnw_status_t wnw_place_prefill_tokens(wnw_cache_t *c, int32_t seq, in
   if (audio_begin < 0 || audio_end < audio_begin || audio_end > n_tokens) return WNW_ERR_INVALID_ARG;
   const bool full = c->cfg.mode == WNW_MODE_FULL;
   const LayerInfo &li = c->layers[layer];
-  const int T_a = audio_end - audio_begin, n_fixed = full ? 0 : li.n_fixed;
-  const int tok_cap = G.S_max * G.nc;
+  const int T_a = audio_end - audio_begin, n_tidal_base = G.token_base ? li.n_tidal : 0;
+  const int n_comp = full ? 0 : li.n_fixed + n_tidal_base;   // compressed heads: the fixed ones, then the tidal bases
+  if (n_tidal_base > 0 && (segment_tokens != G.nc || variant != 0)) return WNW_ERR_UNSUPPORTED;
+  const int tok_cap = G.FB * G.nc;
+  const int C_b = (T_a + G.nc - 1) / G.nc, tail_len = T_a - (C_b - 1) * G.nc;
   std::vector<int> blocks(G.Hkv, -1);
-  for (int h = 0; h < G.Hkv && n_fixed > 0; ++h) {
-    if (c->roles[layer * G.Hkv + h] != ROLE_FIXED) continue;
+  std::vector<int2> m_host(G.Hkv, make_int2(0, 0));
+  for (int h = 0; h < G.Hkv && n_comp > 0; ++h) {
+    const int role = c->roles[layer * G.Hkv + h];
+    if (role != ROLE_FIXED && !(role == ROLE_TIDAL && G.token_base)) continue;
     if (!(retention[h] >= 0.f && retention[h] <= 1.f)) return WNW_ERR_INVALID_ARG;
     const int n = kept_positions(T_a, segment_tokens, retention[h]);
-    if (n > tok_cap) return WNW_ERR_CAPACITY;   // the head's compact store holds S_max blocks of chunk_tokens rows
+    if (n > tok_cap) return WNW_ERR_CAPACITY;   // the head's compact store holds FB blocks of chunk_tokens rows
     blocks[h] = (n + G.nc - 1) / G.nc;
+    if (role == ROLE_TIDAL && T_a > 0)
+      m_host[h] = make_int2((int)std::floor((double)retention[h] * (double)G.nc), (int)std::floor((double)retention[h] * (double)tail_len));
   }
-  wnw_status_t rc = wnw_place_prefill_multi(c, seq, layer, k_dev, v_dev, n_tokens, audio_begin, audio_end, q_text_dev, n_queries,
-                                            cuda_stream);
-  if (rc != WNW_OK || n_fixed == 0 || T_a == 0) return rc;
+  wnw_status_t rc = place_multi(c, seq, layer, k_dev, v_dev, n_tokens, audio_begin, audio_end, q_text_dev, n_queries, cuda_stream);
+  if (rc != WNW_OK || n_comp == 0 || T_a == 0) return rc;
   DeviceGuard guard(c->cfg.device);
   cudaStream_t st = (cudaStream_t)cuda_stream;
   SeqHost &s = c->seqs[seq];
   if (!c->fixed_tok) {
     int fmax = 0;
-    for (const LayerInfo &x : c->layers) fmax = std::max(fmax, (int)x.n_fixed);
+    for (const LayerInfo &x : c->layers) fmax = std::max(fmax, (int)x.n_fixed + (G.token_base ? (int)x.n_tidal : 0));
     c->tok_fixed_max = fmax; c->tok_cap = tok_cap;
     c->tok_p_stride = c->cfg.max_audio_tokens;
     const size_t B = G.max_batch;
@@ -890,15 +929,30 @@ extern "C" wnw_status_t wnw_place_prefill_tokens(wnw_cache_t *c, int32_t seq, in
   // the scratch is shared with earlier placements on other streams: the chunk placement above already ordered this
   // stream after them; the retention values travel through a pageable copy, complete on the host side at return
   CK(cudaMemcpyAsync(c->tok_ret, retention, (size_t)G.Hkv * sizeof(float), cudaMemcpyHostToDevice, st));
-  CK(launch_token_compress(c->cv, seq, layer, n_fixed, c->stage, (const bf16 *)q_text_dev, n_queries, s.T_t, T_a, segment_tokens,
-                           c->tok_ret, variant, c->tok_work, c->tok_p, c->tok_flags, c->tok_p_stride, c->fixed_tok, c->tok_cap,
-                           c->tok_n, st));
+  if (n_tidal_base > 0)
+    CK(cudaMemcpyAsync(c->cv.tok_m + ((size_t)seq * G.L + layer) * G.Hkv, m_host.data(), (size_t)G.Hkv * sizeof(int2),
+                       cudaMemcpyHostToDevice, st));
+  CK(launch_token_compress(c->cv, seq, layer, n_comp, n_tidal_base, c->stage, (const bf16 *)q_text_dev, n_queries, s.T_t, T_a,
+                           segment_tokens, c->tok_ret, variant, c->tok_work, c->tok_p, c->tok_flags, c->tok_p_stride,
+                           c->fixed_tok, c->tok_cap, c->tok_n, st));
   CK(cudaEventRecord(c->ev_place, st));
   if (s.fixed_blocks.empty()) s.fixed_blocks.assign((size_t)G.L * G.Hkv, -1);
-  for (int h = 0; h < G.Hkv; ++h) s.fixed_blocks[layer * G.Hkv + h] = blocks[h];
+  if (s.tok_m.empty()) s.tok_m.assign((size_t)G.L * G.Hkv, make_int2(0, 0));
+  for (int h = 0; h < G.Hkv; ++h) { s.fixed_blocks[layer * G.Hkv + h] = blocks[h]; s.tok_m[layer * G.Hkv + h] = m_host[h]; }
   c->wl_layers.clear();
   c->tok_last_seq = seq; c->tok_last_layer = layer;
   return WNW_OK;
+}
+
+// Index of a head's compact store among the sequence's (fixed heads first, then tidal token bases), -1 if it has none;
+// x: its position among the layer's compressed heads.
+static int compact_head_of(const wnw_cache *c, int layer, int kv_head, int *x) {
+  const int role = c->roles[layer * c->geo.Hkv + kv_head], ridx = c->role_idx[layer * c->geo.Hkv + kv_head];
+  const LayerInfo &li = c->layers[layer];
+  if (c->cfg.mode != WNW_MODE_TIERED) return -1;
+  if (role == ROLE_FIXED) { if (x) *x = ridx; return li.fixed_off + ridx; }
+  if (role == ROLE_TIDAL && c->geo.token_base) { if (x) *x = li.n_fixed + ridx; return c->geo.F_fix + li.tid_prefix + ridx; }
+  return -1;
 }
 
 // per-position prefill scores of one fixed head from the most recent token placement
@@ -907,13 +961,13 @@ extern "C" wnw_status_t wnw_get_token_scores(wnw_cache_t *c, int32_t seq, int32_
   wnw_status_t s = check_seq_layer(c, seq, layer);
   if (s != WNW_OK) return s;
   if (!scores || kv_head < 0 || kv_head >= c->geo.Hkv) return WNW_ERR_INVALID_ARG;
-  if (c->cfg.mode != WNW_MODE_TIERED || c->roles[layer * c->geo.Hkv + kv_head] != ROLE_FIXED) return WNW_ERR_INVALID_ARG;
+  int f = 0;
+  if (compact_head_of(c, layer, kv_head, &f) < 0) return WNW_ERR_INVALID_ARG;
   if (!c->tok_p || c->tok_last_seq != seq || c->tok_last_layer != layer) return WNW_ERR_STATE;
   const int T_a = c->seqs[seq].T_a;
   if (capacity < T_a) return WNW_ERR_CAPACITY;
   DeviceGuard guard(c->cfg.device);
   if ((s = drain(c)) != WNW_OK) return s;
-  const int f = c->role_idx[layer * c->geo.Hkv + kv_head];
   if (T_a > 0) CK(cudaMemcpy(scores, c->tok_p + (size_t)f * c->tok_p_stride, (size_t)T_a * sizeof(float), cudaMemcpyDeviceToHost));
   return WNW_OK;
 }
@@ -924,12 +978,13 @@ extern "C" wnw_status_t wnw_get_fixed_tokens(wnw_cache_t *c, int32_t seq, int32_
   wnw_status_t s = check_seq_layer(c, seq, layer);
   if (s != WNW_OK) return s;
   if (!positions || !n || kv_head < 0 || kv_head >= c->geo.Hkv) return WNW_ERR_INVALID_ARG;
-  if (c->cfg.mode != WNW_MODE_TIERED || c->roles[layer * c->geo.Hkv + kv_head] != ROLE_FIXED) return WNW_ERR_INVALID_ARG;
+  const int head = compact_head_of(c, layer, kv_head, nullptr);
+  if (head < 0) return WNW_ERR_INVALID_ARG;
   const SeqHost &sq = c->seqs[seq];
   if (!c->fixed_tok || sq.fixed_blocks.empty() || sq.fixed_blocks[layer * c->geo.Hkv + kv_head] < 0) return WNW_ERR_STATE;
   DeviceGuard guard(c->cfg.device);
   if ((s = drain(c)) != WNW_OK) return s;
-  const size_t fh = (size_t)seq * c->geo.F_tot + c->layers[layer].fixed_off + c->role_idx[layer * c->geo.Hkv + kv_head];
+  const size_t fh = (size_t)seq * c->geo.F_tot + head;
   int32_t cnt = 0;
   CK(cudaMemcpy(&cnt, c->tok_n + fh, sizeof(cnt), cudaMemcpyDeviceToHost));
   if (cnt > capacity) return WNW_ERR_CAPACITY;
@@ -1402,7 +1457,7 @@ extern "C" wnw_status_t wnw_get_fixed_set(wnw_cache_t *c, int32_t seq, int32_t l
   const size_t fh = (size_t)seq * c->geo.F_tot + c->layers[layer].fixed_off + c->role_idx[layer * c->geo.Hkv + kv_head];
   int32_t cnt = 0;
   CK(cudaMemcpy(&cnt, c->cv.fixed_n + fh, sizeof(cnt), cudaMemcpyDeviceToHost));
-  if (cnt > 0) CK(cudaMemcpy(chunks, c->cv.fixed_chunks + fh * c->geo.S_max, cnt * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  if (cnt > 0) CK(cudaMemcpy(chunks, c->cv.fixed_chunks + fh * c->geo.FB, cnt * sizeof(int32_t), cudaMemcpyDeviceToHost));
   *n = cnt;
   return WNW_OK;
 }
@@ -1433,7 +1488,7 @@ extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
   CK(cudaMemcpy(st.data(), c->cv.stats, st.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
   CK(cudaMemcpy(steps.data(), c->cv.steps, B * sizeof(long long), cudaMemcpyDeviceToHost));
   std::vector<int32_t> slot_chunk(B * G.L * std::max(G.S_max, 1)), fixed_n(B * std::max(G.F_tot, 1)),
-      fixed_chunks(B * std::max(G.F_tot, 1) * std::max(G.S_max, 1));
+      fixed_chunks(B * std::max(G.F_tot, 1) * std::max(G.FB, 1));
   CK(cudaMemcpy(slot_chunk.data(), c->cv.slot_chunk, slot_chunk.size() * 4, cudaMemcpyDeviceToHost));
   CK(cudaMemcpy(fixed_n.data(), c->cv.fixed_n, fixed_n.size() * 4, cudaMemcpyDeviceToHost));
   CK(cudaMemcpy(fixed_chunks.data(), c->cv.fixed_chunks, fixed_chunks.size() * 4, cudaMemcpyDeviceToHost));
@@ -1455,12 +1510,28 @@ extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
         const int ch = slot_chunk[(b * G.L + l) * std::max(G.S_max, 1) + j];
         if (ch >= 0) res += len_of(sq, ch);
       }
-      r.resident_audio_tokens += (int64_t)li.n_tidal * res;
-      r.host_audio_tokens += (int64_t)li.n_tidal * (sq.T_a - res);
+      if (G.token_base) {   // per head: its kept positions plus the complements of the fetched segments
+        for (int h = 0; h < G.Hkv; ++h) {
+          if (c->roles[l * G.Hkv + h] != ROLE_TIDAL) continue;
+          const size_t fh = b * G.F_tot + G.F_fix + li.tid_prefix + c->role_idx[l * G.Hkv + h];
+          const int2 m = sq.tok_m.empty() ? make_int2(0, 0) : sq.tok_m[l * G.Hkv + h];
+          int64_t mine = 0;
+          for (int j = 0; j < fixed_n[fh]; ++j) mine += -fixed_chunks[fh * G.FB + j] - 2;
+          for (int j = 0; j < sq.S; ++j) {
+            const int ch = slot_chunk[(b * G.L + l) * std::max(G.S_max, 1) + j];
+            if (ch >= 0) mine += len_of(sq, ch) - (ch == sq.C - 1 ? m.y : m.x);
+          }
+          r.resident_audio_tokens += mine;
+          r.host_audio_tokens += sq.T_a - mine;
+        }
+      } else {
+        r.resident_audio_tokens += (int64_t)li.n_tidal * res;
+        r.host_audio_tokens += (int64_t)li.n_tidal * (sq.T_a - res);
+      }
       for (int f = 0; f < li.n_fixed; ++f) {
         const size_t fh = b * G.F_tot + li.fixed_off + f;
         for (int j = 0; j < fixed_n[fh]; ++j) {   // entries below -1: blocks of a token-compacted head, -(2 + rows)
-          const int ch = fixed_chunks[fh * G.S_max + j];
+          const int ch = fixed_chunks[fh * G.FB + j];
           r.resident_audio_tokens += ch < -1 ? -ch - 2 : len_of(sq, ch);
         }
       }

@@ -1,4 +1,5 @@
-// Token-granular prefill compression of fixed heads ("Prefill Compression"; retention per head from Eq. 1).
+// Token-granular prefill compression of fixed heads, and of tidal heads' permanent base ("Prefill Compression";
+// retention per head from Eq. 1).
 //
 // Runs once per (sequence, layer) at placement, after the chunk-granular placement has staged the prefix: the staging
 // buffer holds every head's audio K,V in the chunk-padded row layout and the text store holds the text rows.
@@ -19,10 +20,15 @@ namespace {
 
 constexpr int TOK_THREADS = 512;
 
-__device__ __forceinline__ int fixed_head_kv(const CacheView &cv, int layer, int f) {
+// Compressed head x of a layer: the fixed heads first, then (token-granular tidal bases) the tidal heads.  Returns the
+// KV-head, and in `head` its index among the sequence's compact stores.
+__device__ __forceinline__ int comp_head(const CacheView &cv, int layer, int x, int &head) {
   const Geometry &G = cv.geo;
+  const LayerInfo &li = cv.layers[layer];
+  const int role = x < li.n_fixed ? ROLE_FIXED : ROLE_TIDAL, idx = x < li.n_fixed ? x : x - li.n_fixed;
+  head = role == ROLE_FIXED ? li.fixed_off + idx : G.F_fix + li.tid_prefix + idx;
   for (int h = 0; h < G.Hkv; ++h)
-    if (cv.roles[layer * G.Hkv + h] == ROLE_FIXED && cv.role_idx[layer * G.Hkv + h] == f) return h;
+    if (cv.roles[layer * G.Hkv + h] == role && cv.role_idx[layer * G.Hkv + h] == idx) return h;
   return -1;
 }
 
@@ -56,7 +62,8 @@ __global__ void __launch_bounds__(TOK_THREADS) wnw_token_score_kernel(const __gr
   const Geometry &G = cv.geo;
   extern __shared__ float tok_smem[];
   float *qf = tok_smem, *red = tok_smem + G.d;
-  const int f = blockIdx.x, h = fixed_head_kv(cv, layer, f);
+  int head;
+  const int f = blockIdx.x, h = comp_head(cv, layer, f, head);
   if (h < 0) return;
   const int n = T_t + T_a, d = G.d, pieces = d / 8;
   float *lg = work + (long long)f * (T_t + T_a), *p = p_tok + (long long)f * p_stride;
@@ -108,10 +115,10 @@ __global__ void __launch_bounds__(TOK_THREADS) wnw_token_select_kernel(const __g
                                                                       int32_t *fixed_tok, int tok_cap, int32_t *tok_n) {
   const Geometry &G = cv.geo;
   __shared__ int counts[TOK_THREADS + 1];
-  const int f = blockIdx.x, h = fixed_head_kv(cv, layer, f);
+  int head;
+  const int f = blockIdx.x, h = comp_head(cv, layer, f, head);
   if (h < 0) return;
-  const LayerInfo li = cv.layers[layer];
-  const long long fh = (long long)b * G.F_tot + li.fixed_off + f;
+  const long long fh = (long long)b * G.F_tot + head;
   const float *key = p_tok + (long long)f * p_stride;
   int32_t *fl = flags + (long long)f * p_stride, *out = fixed_tok + fh * tok_cap;
   const double ret = (double)retention[h];
@@ -146,27 +153,27 @@ __global__ void __launch_bounds__(TOK_THREADS) wnw_token_select_kernel(const __g
   for (int t = t0; t < t1; ++t)
     if (fl[t]) out[at++] = t;
   const int n = counts[TOK_THREADS], n_blk = (n + G.nc - 1) / G.nc;
-  for (int s = threadIdx.x; s < G.S_max; s += TOK_THREADS)   // block s of the compact store holds min(nc, n - s*nc) rows
-    cv.fixed_chunks[fh * G.S_max + s] = s < n_blk ? -(2 + min(G.nc, n - s * G.nc)) : -1;
+  for (int s = threadIdx.x; s < G.FB; s += TOK_THREADS)   // block s of the compact store holds min(nc, n - s*nc) rows
+    cv.fixed_chunks[fh * G.FB + s] = s < n_blk ? -(2 + min(G.nc, n - s * G.nc)) : -1;
   if (threadIdx.x == 0) { cv.fixed_n[fh] = n_blk; tok_n[fh] = n; }
 }
 
-// grid (S_max, fixed heads of the layer); block 128.  Fills block blockIdx.x of the head's compact store.
+// grid (FB, fixed heads of the layer); block 128.  Fills block blockIdx.x of the head's compact store.
 __global__ void __launch_bounds__(128) wnw_token_gather_kernel(const __grid_constant__ CacheView cv, int b, int layer,
                                                                const bf16 *stage, const int32_t *fixed_tok, int tok_cap,
                                                                const int32_t *tok_n) {
   const Geometry &G = cv.geo;
-  const int blk = blockIdx.x, f = blockIdx.y, h = fixed_head_kv(cv, layer, f);
+  int head;
+  const int blk = blockIdx.x, f = blockIdx.y, h = comp_head(cv, layer, f, head);
   if (h < 0) return;
-  const LayerInfo li = cv.layers[layer];
-  const long long fh = (long long)b * G.F_tot + li.fixed_off + f;
+  const long long fh = (long long)b * G.F_tot + head;
   const int n = tok_n[fh];
   if (blk * G.nc >= n) return;
   const int pieces = G.d / 8;
   const int32_t *pos = fixed_tok + fh * tok_cap;
   for (int kv = 0; kv < 2; ++kv) {
     const uint4 *src = reinterpret_cast<const uint4 *>(stage + anchor_off(G, 0, 0, h, kv));
-    uint4 *dst = reinterpret_cast<uint4 *>(cv.fixed + fixed_off(G, li, b, f, kv) + (long long)blk * G.ncp * G.d);
+    uint4 *dst = reinterpret_cast<uint4 *>(cv.fixed + compact_off(G, b, head, kv) + (long long)blk * G.ncp * G.d);
     for (int v = threadIdx.x; v < G.ncp * pieces; v += blockDim.x) {
       const int r = v / pieces, x = v - r * pieces, i = blk * G.nc + r;
       uint4 val = make_uint4(0, 0, 0, 0);   // rows past the block's last token are zero
@@ -179,16 +186,56 @@ __global__ void __launch_bounds__(128) wnw_token_gather_kernel(const __grid_cons
   }
 }
 
-cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_fixed, const bf16 *stage, const bf16 *q_text,
-                                  int n_q, int T_t, int T_a, int seg, const float *retention_dev, int variant, float *work,
-                                  float *p_tok, int32_t *flags, long long p_stride, int32_t *fixed_tok, int tok_cap,
-                                  int32_t *tok_n, cudaStream_t st) {
-  if (n_fixed <= 0 || T_a <= 0) return cudaSuccess;
+// grid (segments, tidal heads of the layer); block 128.  Token-granular tidal base: rewrites segment blockIdx.x of the
+// head's host mirror with the positions that are NOT in the base first (ascending), the kept ones after them, so that
+// the first (length - kept) rows of a fetched segment are exactly its complement.
+__global__ void __launch_bounds__(128) wnw_token_mirror_kernel(const __grid_constant__ CacheView cv, int b, int layer,
+                                                               const bf16 *stage, const int32_t *flags, long long p_stride,
+                                                               int T_a) {
+  const Geometry &G = cv.geo;
+  extern __shared__ int mirror_dst[];   // [nc] destination row of every position of the segment
+  const LayerInfo li = cv.layers[layer];
+  const int c = blockIdx.x, t = blockIdx.y, x = li.n_fixed + t;
+  int head;
+  const int h = comp_head(cv, layer, x, head);
+  if (h < 0) return;
+  const int lo = c * G.nc, len = min(G.nc, T_a - lo);
+  const int32_t *fl = flags + (long long)x * p_stride + lo;
+  int n_out = 0;
+  for (int r = 0; r < len; ++r) n_out += fl[r] == 0;
+  for (int r = threadIdx.x; r < len; r += blockDim.x) {
+    int before_same = 0;
+    for (int q = 0; q < r; ++q) before_same += fl[q] == fl[r];
+    mirror_dst[r] = fl[r] ? n_out + before_same : before_same;
+  }
+  __syncthreads();
+  const int pieces = G.d / 8;
+  for (int kv = 0; kv < 2; ++kv) {
+    const uint4 *src = reinterpret_cast<const uint4 *>(stage + anchor_off(G, 0, 0, h, kv) + (long long)c * G.ncp * G.d);
+    uint4 *dst = reinterpret_cast<uint4 *>(cv.mirror[b] + mirror_off(G, li, cv.C[b], c, t, kv));
+    for (int v = threadIdx.x; v < len * pieces; v += blockDim.x) {
+      const int r = v / pieces, piece = v - r * pieces;
+      dst[(long long)mirror_dst[r] * pieces + piece] = src[v];
+    }
+  }
+}
+
+// n_comp: compressed heads of the layer (its fixed heads, then its tidal heads when they keep a token base)
+cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_comp, int n_tidal_base, const bf16 *stage,
+                                  const bf16 *q_text, int n_q, int T_t, int T_a, int seg, const float *retention_dev,
+                                  int variant, float *work, float *p_tok, int32_t *flags, long long p_stride,
+                                  int32_t *fixed_tok, int tok_cap, int32_t *tok_n, cudaStream_t st) {
+  if (n_comp <= 0 || T_a <= 0) return cudaSuccess;
   const size_t smem = (size_t)(cv.geo.d + TOK_THREADS / 32) * sizeof(float);
-  wnw_token_score_kernel<<<n_fixed, TOK_THREADS, smem, st>>>(cv, b, layer, stage, q_text, n_q, T_t, T_a, work, p_tok, p_stride);
-  wnw_token_select_kernel<<<n_fixed, TOK_THREADS, 0, st>>>(cv, b, layer, p_tok, p_stride, T_a, seg, retention_dev, variant, flags,
-                                                          fixed_tok, tok_cap, tok_n);
-  wnw_token_gather_kernel<<<dim3(cv.geo.S_max, n_fixed), 128, 0, st>>>(cv, b, layer, stage, fixed_tok, tok_cap, tok_n);
+  wnw_token_score_kernel<<<n_comp, TOK_THREADS, smem, st>>>(cv, b, layer, stage, q_text, n_q, T_t, T_a, work, p_tok, p_stride);
+  wnw_token_select_kernel<<<n_comp, TOK_THREADS, 0, st>>>(cv, b, layer, p_tok, p_stride, T_a, seg, retention_dev, variant, flags,
+                                                         fixed_tok, tok_cap, tok_n);
+  wnw_token_gather_kernel<<<dim3(cv.geo.FB, n_comp), 128, 0, st>>>(cv, b, layer, stage, fixed_tok, tok_cap, tok_n);
+  if (n_tidal_base > 0) {
+    const int C_b = (T_a + cv.geo.nc - 1) / cv.geo.nc;
+    wnw_token_mirror_kernel<<<dim3(C_b, n_tidal_base), 128, (size_t)cv.geo.nc * sizeof(int), st>>>(cv, b, layer, stage, flags,
+                                                                                                  p_stride, T_a);
+  }
   return cudaGetLastError();
 }
 

@@ -64,6 +64,7 @@ class Lockstep:
                                 w.text_capacity, w.chunk, w.budget, w.roles, topk=w.topk, device=self.dev.index or 0,
                                 recall_mode=recall_mode, score_scope=score_scope, residency=residency, evict_lag=evict_lag)
         self.kept = {}
+        self.tok_kept = {}
         self.near_ties = 0
         self.max_out_err = 0.0
         self.dec = {}
@@ -154,7 +155,7 @@ class Lockstep:
         if T_a == 0:
             return
         for h in range(w.n_kv_heads):
-            if w.roles[l, h] != ROLE_FIXED:
+            if w.roles[l, h] != ROLE_FIXED and not (w.roles[l, h] == ROLE_TIDAL and self.residency == 2):
                 continue
             g_p = wnw.wnw_get_token_scores(self.h, b, l, h)
             o_p = self.o.token_scores(b, l, h)
@@ -174,6 +175,7 @@ class Lockstep:
                     assert ks.max() - ks.min() <= TIE_RTOL * max(ks.max(), 1e-30), f"kept positions b{b} l{l} h{h}: {ts}"
                 self.near_ties += 1
                 self.o.set_fixed_tokens(b, l, h, g_pos)
+            self.tok_kept[(b, l, h)] = g_pos
 
     def check_slot_bytes(self, b, l):
         """Slot contents are an exact copy of the source K,V of the chunk the table says is there."""
@@ -188,9 +190,14 @@ class Lockstep:
                 if c < 0:
                     continue
                 n = min(w.chunk, T_a - c * w.chunk)
+                order = np.arange(n)
+                if self.residency == 2:       # token-granular base: the positions outside the base first, the kept ones after
+                    kept = set(self.tok_kept[(b, l, h)].tolist())
+                    inb = np.array([c * w.chunk + r in kept for r in range(n)])
+                    order = np.concatenate([np.nonzero(~inb)[0], np.nonzero(inb)[0]])
                 for which, src in ((0, kb), (1, vb)):
                     rows = wnw.wnw_get_slot_kv(self.h, b, l, h, j, which, w.chunk, w.head_dim)
-                    assert np.array_equal(rows[:n], src[c * w.chunk:c * w.chunk + n, h]), f"slot bytes b{b} l{l} h{h} slot{j}"
+                    assert np.array_equal(rows[:n], src[c * w.chunk:c * w.chunk + n, h][order]), f"slot bytes b{b} l{l} h{h} slot{j}"
 
     # ------------------------------------------------------------------ decode
     def _dec(self, b, l):
@@ -294,7 +301,7 @@ class Lockstep:
                 g_tab, g_stamp = wnw.wnw_get_residency(self.h, b, l)
                 # (ii) oracle logic on GPU scores and the GPU's previous table
                 tab, stamp = prev_tab[(b, l)][0].copy(), prev_tab[(b, l)][1].copy()
-                if self.residency == 1:   # overlapping chunks, permanent base, lag-delta release
+                if self.residency >= 1:   # overlapping chunks, permanent base, lag-delta release
                     want_sel, segs = wo.select_segments(rank_g, lens, w.topk)
                     assert g_sel.tolist() == want_sel.tolist(), f"selection (ii) step {t} b{b} l{l}"
                     plan, _, _ = wo.lag_update(tab, stamp, wnw.wnw_get_base_slots(self.h, b), segs, steps_before[b], self.evict_lag)
@@ -312,7 +319,7 @@ class Lockstep:
                 o_sel = self.o.selected(b, l)
                 o_tab, o_stamp = self.o.residency(b, l)
                 if o_sel.tolist() != g_sel.tolist() or o_tab.tolist() != g_tab.tolist() or o_stamp.tolist() != g_stamp.tolist():
-                    assert near_tie(rank_o, lens_tie if self.residency == 1 and C > 1 else lens, g_sel.tolist(), o_sel.tolist()), \
+                    assert near_tie(rank_o, lens_tie if self.residency >= 1 and C > 1 else lens, g_sel.tolist(), o_sel.tolist()), \
                         f"selection differs beyond a near-tie, step {t} b{b} l{l}: gpu {g_sel} oracle {o_sel}"
                     self.near_ties += 1
                     self.o.set_residency(b, l, g_tab, g_stamp)

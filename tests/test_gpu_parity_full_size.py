@@ -144,3 +144,28 @@ def test_config1_token_compressed_fixed_heads(variant):
         assert ls.max_out_err <= 2e-2
     finally:
         ls.close()
+
+
+def test_config1_paper_form_with_token_base():
+    """Config 1 in the paper's full form: 25-token segments, chunks of two segments, scores summed over all anchor layers,
+    lag-3 release, and a token-granular permanent base: every tidal and fixed head keeps its per-segment best positions
+    (per-head retention from Eq. 1, seeded importances, lambda = 0.36), tidal tables start empty and fetch complements.
+    24 decode steps replayed as a CUDA graph; counters must agree at the end."""
+    import paper_2608_22704_b200 as wnw
+    from parity_harness import Lockstep
+    w = config1(n_steps=24)
+    w.chunk = 25
+    w.n_prefill_queries = 2
+    s_tilde = np.random.RandomState(11).rand(w.n_layers * w.n_kv_heads)
+    ret = wnw.wnw_retention_schedule(s_tilde, 0.36).reshape(w.n_layers, w.n_kv_heads)
+    ls = Lockstep(w, seed=3, gen_device="cuda:0", score_scope=1, residency=2, evict_lag=3, token_retention=ret, token_seg=25)
+    try:
+        ls.prefill(check_slots=False)
+        for t in range(24):
+            ls.decode_step(t, graph=True, check_slots=(t % 8 == 7))
+        ls.check_stats()
+        assert ls.max_out_err <= 2e-2
+        st = wnw.wnw_get_stats(ls.h)
+        assert st["misses"] > 0
+    finally:
+        ls.close()

@@ -137,3 +137,103 @@ def test_retention_schedule_on_the_host():
     assert r.tolist() == [0.0, np.float32(0.1) * np.float32(1.5), 0.75, 1.0]
     with pytest.raises(wnw.WnwError):
         wnw.wnw_retention_schedule([0.5, 1.2], 1.0)
+
+
+# ---------------------------------------------------------------- tidal heads with a token-granular permanent base
+def _lag_workload(audio=(640, 300, 77), chunk=25, head_dim=128, n_steps=10):
+    w = tiny_custom(n_layers=3, n_q_heads=8, n_kv_heads=4, head_dim=head_dim, n_text=9, audio_lens=audio, chunk=chunk, budget=0.3,
+                    n_steps=n_steps, roles=[[A, T, F, T], [T, F, T, F], [A, T, T, T]], region=chunk, jump_every=3, topk=2)
+    w.n_prefill_queries = 3
+    return w
+
+
+RET_LAG = np.array([[1.0, 0.3, 0.45, 0.0], [0.5, 0.2, 0.08, 0.33], [1.0, 0.41, 0.25, 0.5]], np.float32)
+
+
+@pytest.mark.parametrize("scope", [0, 1])
+def test_token_base_tidal_heads_follow_the_oracle(scope):
+    """Residency SEGMENT_LAG_TOKEN_BASE: every tidal head keeps its own per-segment best positions for good (retention
+    0 to 0.5 per head), tables start empty, selected segments are fetched as complements (host mirror permuted) and
+    released after the lag; per-layer and global score scope; eager and replayed steps; slot bytes checked against the
+    permuted source rows."""
+    from parity_harness import Lockstep
+    w = _lag_workload()
+    ls = Lockstep(w, seed=31 + scope, score_scope=scope, residency=2, evict_lag=1, token_retention=RET_LAG, token_seg=25)
+    try:
+        ls.prefill()
+        for b in range(w.batch):
+            assert wnw.wnw_get_base_slots(ls.h, b) == 0
+            for l in range(w.n_layers):
+                tab, _ = wnw.wnw_get_residency(ls.h, b, l)
+                assert (tab == -1).all()
+        ls.decode_step(0, check_slots=True)
+        for t in range(1, 6):
+            ls.decode_step(t, graph=True, check_slots=True)
+        ls.decode_step(6, check_slots=True)
+        for t in range(7, 10):
+            ls.decode_step(t, graph=True, check_slots=(t == 9))
+        ls.check_stats()
+        assert ls.max_out_err <= 2e-2
+        st = wnw.wnw_get_stats(ls.h)
+        assert st["misses"] > 0 and st["evictions"] > 0
+        # r_GPU accounting: kept positions plus the complements of the fetched segments, per tidal head
+        want = 0
+        for b in range(w.batch):
+            T_a = w.audio_lens[b]
+            C = -(-T_a // 25)
+            for l in range(w.n_layers):
+                tab, _ = wnw.wnw_get_residency(ls.h, b, l)
+                for h in range(w.n_kv_heads):
+                    if w.roles[l, h] == A:
+                        want += T_a
+                        continue
+                    kept = wnw.wnw_get_fixed_tokens(ls.h, b, l, h)
+                    want += len(kept)
+                    if w.roles[l, h] == T:
+                        ks = set(kept.tolist())
+                        for c in tab:
+                            if c >= 0:
+                                want += sum(1 for p in range(c * 25, min((c + 1) * 25, T_a)) if p not in ks)
+        assert st["resident_audio_tokens"] == want
+    finally:
+        ls.close()
+
+
+def test_token_base_chunk_of_64_and_d64():
+    """Segments of 64 tokens (four granules per block), head_dim 64, a sequence whose last segment is short."""
+    from parity_harness import Lockstep
+    w = tiny_custom(n_layers=2, n_q_heads=8, n_kv_heads=2, head_dim=64, n_text=5, audio_lens=(1000, 130), chunk=64, budget=0.25,
+                    n_steps=6, roles=[[A, T], [T, F]], region=64, jump_every=2, topk=3)
+    ret = np.array([[1.0, 0.3], [0.17, 0.4]], np.float32)
+    ls = Lockstep(w, seed=4, residency=2, evict_lag=2, token_retention=ret, token_seg=64)
+    try:
+        ls.prefill()
+        for t in range(6):
+            ls.decode_step(t, graph=(t % 2 == 1), check_slots=True)
+        ls.check_stats()
+        assert ls.max_out_err <= 2e-2
+    finally:
+        ls.close()
+
+
+def test_token_base_placement_rules():
+    w = _lag_workload(audio=(640,))
+    h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, 1, 640, w.text_capacity, w.chunk, w.budget, w.roles,
+                       topk=w.topk, residency=wnw.WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE, evict_lag=1)
+    try:
+        p = Synth(w, seed=1).prefill(0, 0)
+        k, v, q = (p[n].cuda() for n in ("k", "v", "q_text"))
+        with pytest.raises(wnw.WnwError) as e:       # the chunk-granular placement has no base to offer
+            wnw.wnw_place_prefill(h, 0, 0, k, v, p["audio_begin"], p["audio_end"], q)
+        assert e.value.status == wnw.WNW_ERR_STATE
+        args = (h, 0, 0, k, v, p["audio_begin"], p["audio_end"], q, RET_LAG[0])
+        for seg, variant in ((50, 0), (25, 1)):      # the quota's segment is the storage segment; no global variant
+            with pytest.raises(wnw.WnwError) as e:
+                wnw.wnw_place_prefill_tokens(*args, seg, variant)
+            assert e.value.status == wnw.WNW_ERR_UNSUPPORTED
+        wnw.wnw_place_prefill_tokens(*args, 25, 0)
+        wnw.wnw_sync(h)
+        assert len(wnw.wnw_get_fixed_tokens(h, 0, 0, 1)) == 25 * 7 + 4       # floor(.3*25)=7, tail floor(.3*15)=4
+        assert len(wnw.wnw_get_fixed_tokens(h, 0, 0, 3)) == 0
+    finally:
+        wnw.wnw_destroy(h)
