@@ -123,6 +123,7 @@ struct GranDesc {
 
 // Maps granule j of a head's virtual key space [text capacity | audio] to memory WITHOUT waiting on any global load:
 // the row of every granule is static; what may be unknown yet is how many of its 16 rows are visible.
+template <bool TB>
 __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const AttnArgs &a, const LayerInfo &li,
                                                    const WorkItem &it, int j) {
   const Geometry &G = cv.geo;
@@ -143,7 +144,7 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
     len -= off;
     r.meta = len <= 0 ? 0 : (len < GR ? len : GR);
     if (a.score_on) r.score_idx = ag;
-  } else if (it.role == ROLE_TIDAL && G.token_base && ci < it.S) {
+  } else if (TB && it.role == ROLE_TIDAL && ci < it.S) {
     // token-granular permanent base: the first it.S units of the head are blocks of its compact store
     const int head = G.F_fix + li.tid_prefix + it.ridx;
     r.row = (int)(compact_off(G, it.b, head, 0) / G.d) + ci * G.ncp + off;
@@ -151,11 +152,11 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
     r.meta = -2;
     r.score_idx = -2;               // marks the compact store (tensor map and K-to-V row distance differ from the pool's)
   } else if (it.role == ROLE_TIDAL) {
-    const int slot = G.token_base ? ci - it.S : ci;
+    const int slot = TB ? ci - it.S : ci;
     r.row = (int)(pool_off(G, li, it.b, slot, it.ridx, 0) / G.d) + off;
     r.cid = cv.slot_chunk[((long long)it.b * G.L + a.layer) * G.S_max + slot];
     // beyond the permanent slots a slot may be empty: its rows are fetched only if it is not
-    r.meta = (G.token_base || ci >= it.S) ? -3 : -2;
+    r.meta = (TB || ci >= it.S) ? -3 : -2;
   } else {
     const long long fh = (long long)it.b * G.F_tot + li.fixed_off + it.ridx;
     r.row = (int)(fixed_off(G, li, it.b, it.ridx, 0) / G.d) + ci * G.ncp + off;
@@ -165,7 +166,8 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
   return r;
 }
 
-template <int D, bool G16, int NW>
+// TB: tidal heads keep a token-granular permanent base (their key space is [text | base blocks | dynamic slots])
+template <int D, bool G16, int NW, bool TB>
 __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant__ CacheView cv,
                                                            const __grid_constant__ AttnArgs a,
                                                            const __grid_constant__ InlineItems inl,
@@ -257,7 +259,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     else if (c.it.role == ROLE_TIDAL) { c.v_delta_audio = G.ncp; c.map_audio = &maps.pool; }          // granule's K and
     else { c.v_delta_audio = G.FB * G.ncp; c.map_audio = &maps.fixed; }                            // V rows
     c.m_full = c.m_tail = 0;
-    if (G.token_base && c.it.role == ROLE_TIDAL) {
+    if (TB && c.it.role == ROLE_TIDAL) {
       const int2 m = cv.tok_m[((long long)c.it.b * G.L + a.layer) * G.Hkv + c.it.h];
       c.m_full = m.x; c.m_tail = m.y;
     }
@@ -284,8 +286,9 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       if (cid < -1) len = -cid - 2;   // a block of a token-compacted fixed head: the entry carries its row count
       else {
         len = c.it.T_a - cid * G.nc;
-        if (len > G.nc) { len = G.nc; len -= c.m_full; }
-        else len -= c.m_tail;   // the last segment; a fetched segment holds its complement first (m = 0 without a token base)
+        if (len > G.nc) len = G.nc;
+        // token base: a fetched segment holds its complement first; the last segment has its own count
+        if (TB) len -= (c.it.T_a - cid * G.nc > G.nc) ? c.m_full : c.m_tail;
       }
       len -= off;
     }
@@ -298,7 +301,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   auto issue_copy = [&](const Ctx &c, int n, uint32_t seq) -> bool {
     if ((n & 31) == 0) {
       const int nn = n + lane;
-      if (nn < c.n_my) blk = decode_granule(cv, a, li, c.it, c.first + nn * NW);
+      if (nn < c.n_my) blk = decode_granule<TB>(cv, a, li, c.it, c.first + nn * NW);
       else { blk.meta = 0; blk.cid = -1; blk.score_idx = -1; }
 #ifdef WNW_PHASE_STAMPS
       if (n == 0 && blk.row >= 0) STAMP(12);
@@ -310,7 +313,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     const int j = c.first + n * NW;
     const bool is_text = j < G.n_tg;
     // a block of a tidal head's permanent token base: compact store, never touched by the recall
-    const bool base_blk = G.token_base && __shfl_sync(0xffffffffu, blk.score_idx, src_lane) == -2;
+    const bool base_blk = TB && __shfl_sync(0xffffffffu, blk.score_idx, src_lane) == -2;
     if (epoch_pending && !is_text && !base_blk) wait_recall_epoch();
     bool load = meta != 0;
     if (meta == -1) load = visible(c, -1, 0, 0, j) > 0;  // waits for the text length
@@ -656,8 +659,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   pdl_finish();
 }
 
-template <int D, bool G16, int NW>
-static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
+template <int D, bool G16, int NW, bool TB>
+static cudaError_t launch_tb(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
   // stages + slack to align them to the swizzle atom + the merge scratch when it does not alias the stages
   const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024 + (a.xpref ? attn_scratch_bytes(NW, cv.geo.g, D) : 0);
   if (!a.maps) return cudaErrorInvalidValue;
@@ -675,7 +678,11 @@ static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
   }
-  return cudaLaunchKernelEx(&cfg, wnw_attn_kernel<D, G16, NW>, cv, a, inl, *a.maps);
+  return cudaLaunchKernelEx(&cfg, wnw_attn_kernel<D, G16, NW, TB>, cv, a, inl, *a.maps);
+}
+template <int D, bool G16, int NW>
+static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
+  return cv.geo.token_base ? launch_tb<D, G16, NW, true>(cv, a, st) : launch_tb<D, G16, NW, false>(cv, a, st);
 }
 
 // ---- TMA descriptors ----
@@ -708,8 +715,10 @@ bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long row
 template <int D, bool G16, int NW>
 static cudaError_t configure_t() {
   const size_t want = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024 + attn_scratch_bytes(NW, G16 ? 16 : 8, D);
-  return cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)std::min<size_t>(want, 226 * 1024));
+  const int bytes = (int)std::min<size_t>(want, 226 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 // Opt-in shared-memory sizes, set once per device at cache creation (never during a stream capture).
 cudaError_t configure_attn_kernels() {
