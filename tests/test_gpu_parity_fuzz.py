@@ -62,3 +62,36 @@ def test_random_configuration_segment_lag(seed):
         ls.check_stats()
     finally:
         ls.close()
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_configuration_token_compression(seed):
+    """The same random shapes with token-granular prefill compression: fixed heads under every residency (random segment
+    size and variant), tidal heads' permanent base under SEGMENT_LAG_TOKEN_BASE; random per-head retention within what a
+    compact store holds, random number of text queries, eviction lag, score scope and layer ordering."""
+    import paper_2608_22704_b200 as wnw
+    from parity_harness import Lockstep
+    w, rs = _draw(seed)
+    residency = int(rs.choice([0, 1, 2, 2]))
+    delta = int(rs.randint(0, 4))
+    w.n_prefill_queries = int(rs.randint(1, 4))
+    T_max = max(w.audio_lens)
+    C = -(-T_max // w.chunk)
+    base = min(C, max(1, int(np.floor(float(np.float32(w.budget)) * C + 1e-6))))
+    blocks = base + (min(2 * w.topk * (delta + 1), C - base) if residency else 0)
+    r_max = min(1.0, 0.95 * blocks * w.chunk / max(T_max, 1))
+    ret = (rs.rand(w.n_layers, w.n_kv_heads) * r_max).astype(np.float32)
+    ret[rs.rand(w.n_layers, w.n_kv_heads) < 0.1] = 0.0
+    seg = w.chunk if residency == 2 else int(rs.choice([w.chunk, 25, 7]))
+    variant = 0 if residency == 2 else int(rs.randint(0, 2))
+    ls = Lockstep(w, seed=seed, residency=residency, evict_lag=delta, score_scope=int(rs.randint(0, 2)), token_retention=ret,
+                  token_seg=seg, token_variant=variant)
+    try:
+        wnw.wnw_set_layer_dependency(ls.h, int(rs.randint(0, 3)))
+        ls.prefill()
+        use_graph = bool(seed % 2)
+        for t in range(w.n_steps):
+            ls.decode_step(t, append=True, graph=use_graph and t not in (0, 3), check_slots=True)
+        ls.check_stats()
+    finally:
+        ls.close()
