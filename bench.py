@@ -142,6 +142,8 @@ class ClockSampler:
 class Job:
     """Caches, resident inputs and launch helpers of one rank."""
 
+    layer_dependency = 0   # WNW_LAYERS_*: how the layers of a step are issued (set from --layer-dependency)
+
     def __init__(self, w, seed, device, wnw, score_scope=0, residency=0, evict_lag=3):
         self.score_scope = score_scope
         self.residency, self.evict_lag = residency, evict_lag
@@ -171,12 +173,13 @@ class Job:
         self.stream = torch.cuda.Stream(device=device)
         self.captured = set()
 
-    def create(self, key, mode, recall_mode=0):
+    def create(self, key, mode, recall_mode=0, layer_dependency=None):
         w, wnw = self.w, self.wnw
         h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, self.B, max(w.audio_lens), w.text_capacity,
                            w.chunk, w.budget, w.roles, topk=w.topk, device=self.dev.index or 0, mode=mode,
                            recall_mode=recall_mode, score_scope=self.score_scope, residency=self.residency,
                            evict_lag=self.evict_lag)
+        wnw.wnw_set_layer_dependency(h, Job.layer_dependency if layer_dependency is None else layer_dependency)
         self.caches[key] = h
         return h
 
@@ -445,7 +448,7 @@ def run_ours(args, rank, world, local_rank):
     R = args.roofline_steps
     Kc = 0 if (args.quick or args.eager) else min(K, args.chain_steps)
     Kb = 0 if (args.quick or args.eager) else min(K, args.back_to_back_steps)
-    total = W + R + K + Kb + 2 * Kc
+    total = W + R + K + Kb + 2 * Kc   # + the chained and the serial runs
     w = make_workload(args.workload, total, 0)
     if args.segment_tokens > 0:
         w.chunk = args.segment_tokens
@@ -453,7 +456,6 @@ def run_ours(args, rank, world, local_rank):
     job = Job(w, seed=rank, device=dev, wnw=wnw, score_scope=args.score_scope, residency=args.residency, evict_lag=args.evict_lag)
     job.create("wnw", wnw.WNW_MODE_FULL if args.quick_full else wnw.WNW_MODE_TIERED, recall_mode=args.recall_mode)
     if args.quick:   # profiler mode: the WnW steps only, nothing else launched
-        wnw.wnw_set_layer_dependency(job.caches["wnw"], args.layer_dependency)
         job.place_all(["wnw"])
         for t in range(W):
             job.step("wnw", t, full=args.quick_full)
@@ -471,6 +473,13 @@ def run_ours(args, rank, world, local_rank):
         return
     job.create("full", wnw.WNW_MODE_FULL)
     job.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
+    # the other way to issue layers whose inputs are all resident before the step: one launch for all layers where the
+    # headline uses one per layer (or the reverse); same steps, same state
+    alt_dep = wnw.WNW_LAYERS_INDEPENDENT if Job.layer_dependency == wnw.WNW_LAYERS_BATCHED else wnw.WNW_LAYERS_BATCHED
+    alt_name = "per_layer_launches" if alt_dep == wnw.WNW_LAYERS_INDEPENDENT else "all_layers_one_launch"
+    alt_on = not args.eager and not args.no_alt_form
+    if alt_on:
+        job.create("alt", wnw.WNW_MODE_TIERED, layer_dependency=alt_dep)
 
     class Keep:
         store = {}
@@ -478,7 +487,7 @@ def run_ours(args, rank, world, local_rank):
         def __call__(self, b, l):
             return rank == 0 and b == 0 and l < args.oracle_layers
     keep = Keep()
-    job.place_all(["wnw", "full", "skip"], keep_host=keep)
+    job.place_all(["wnw", "full", "skip"] + (["alt"] if alt_on else []), keep_host=keep)
 
     def barrier():
         if world > 1:
@@ -487,7 +496,7 @@ def run_ours(args, rank, world, local_rank):
 
     # ---- warm-up (all three caches take the same steps so their states stay comparable)
     for t in range(W):
-        for key, full in (("wnw", False), ("full", True), ("skip", False)):
+        for key, full in (("wnw", False), ("full", True), ("skip", False)) + ((("alt", False),) if alt_on else ()):
             job.step(key, t, full=full)
     torch.cuda.synchronize(dev)
 
@@ -535,6 +544,14 @@ def run_ours(args, rank, world, local_rank):
     # ---- comparison: own full-cache kernel, and WnW with recall copies skipped (exposed recall time)
     full_steps = job.timed_steps("full", W + R, K, full=True, graph=not args.eager)
     skip_steps = job.timed_steps("skip", W + R, K, graph=not args.eager)
+    alt = None
+    if alt_on:
+        for t in range(W, W + R):
+            job.step("alt", t)
+        nb_alt, _ = job.kv_bytes_of_step("alt")
+        ms_alt = dist_max(sum(job.timed_steps("alt", W + R, K)), dev, world) / K
+        alt = {"step_us": ms_alt * 1e3, "achieved": nb_alt / (ms_alt * 1e-3) / 1e9, "frac": nb_alt / (ms_alt * 1e-3) / 1e9 / peak_gbs,
+               "steps": K}
     barrier()
     # ---- continuous decoding: the same steps back to back in one timed region (no flush gaps in which a recall could
     # finish for free); the difference to the run with copies skipped is the recall time that overlap cannot hide
@@ -542,6 +559,8 @@ def run_ours(args, rank, world, local_rank):
     if Kb > 0:
         ms_bb = dist_max(job.timed_region("wnw", W + R + K, Kb), dev, world)
         ms_bb_skip = dist_max(job.timed_region("skip", W + R + K, Kb), dev, world)
+        if alt is not None:
+            alt["back_to_back_step_us"] = dist_max(job.timed_region("alt", W + R + K, Kb), dev, world) * 1e3
         bb = {"steps": Kb, "ms_per_step": ms_bb, "ms_per_step_copies_skipped": ms_bb_skip,
               "exposed_recall_us_per_step": (ms_bb - ms_bb_skip) * 1e3, "tokens_per_s": whole_job_tokens_per_s(world, w.batch, ms_bb),
               "note": "K steps in one event bracket, no L2 flush between them (a step reads more than L2 holds only on the "
@@ -581,7 +600,8 @@ def run_ours(args, rank, world, local_rank):
     dep = {}
     if Kc > 0:
         t_dep = W + R + K + Kb
-        for name, mode in (("chained", wnw.WNW_LAYERS_CHAINED), ("serial", wnw.WNW_LAYERS_SERIAL)):
+        modes = [("chained", wnw.WNW_LAYERS_CHAINED), ("serial", wnw.WNW_LAYERS_SERIAL)]
+        for name, mode in modes:
             wnw.wnw_sync(job.caches["wnw"])
             wnw.wnw_set_layer_dependency(job.caches["wnw"], mode)
             job.captured.discard("wnw")
@@ -591,7 +611,9 @@ def run_ours(args, rank, world, local_rank):
             us_l = ms * 1e3 / w.n_layers          # one launch per layer in these modes
             dep[name] = {"step_us": ms * 1e3, "us_per_launch": us_l, "achieved": nb / w.n_layers / (us_l * 1e-6) / 1e9,
                          "frac": nb / w.n_layers / (us_l * 1e-6) / 1e9 / peak_gbs, "steps": Kc}
-        wnw.wnw_set_layer_dependency(job.caches["wnw"], wnw.WNW_LAYERS_INDEPENDENT)
+        wnw.wnw_sync(job.caches["wnw"])
+        wnw.wnw_set_layer_dependency(job.caches["wnw"], Job.layer_dependency)
+        job.captured.discard("wnw")
 
     if rank != 0:
         job.destroy()
@@ -711,14 +733,19 @@ def run_ours(args, rank, world, local_rank):
         "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(w), launch="eager" if args.eager else "cuda graph replay of the step",
                                                                                 score_scope="global" if args.score_scope else "per layer",
-                                                                                residency="segment lag" if args.residency else "hard budget"),
+                                                                                residency="segment lag" if args.residency else "hard budget",
+                                                                                layers={0: "one launch per layer, overlapping (inputs of every layer resident before the step)",
+                                                                                        1: "chained (a layer waits for its predecessor before it reads q)",
+                                                                                        2: "serial launches",
+                                                                                        3: "all layers in one launch (inputs of every layer resident before the step, outputs read after it)"}[args.layer_dependency]),
         "clocks": clocks, "gpu_launches": int(sum(region_launches)),
         "launches": {"attention": region_launches[0], "selection": region_launches[1], "recall": region_launches[2],
                      "step_end": region_launches[3], "layers_per_attention_launch": w.n_layers / attn_per_step},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e},
         # achieved: algorithmic K,V bytes of one launch / the launch's share of the timed region (CUDA events around every
-        # replayed step; the attention kernels are the only work on the timed stream, one per layer; consecutive layer
-        # kernels overlap through programmatic dependent launch, so the share of one launch is step time / layers).
+        # replayed step; the attention kernels are the only work on the timed stream).  With all layers in one launch
+        # (the default) that launch carries the step's bytes and its share is the step; with one launch per layer the
+        # consecutive kernels overlap through programmatic dependent launch and the share of one is step time / layers.
         # `chained`: every kernel waits for its predecessor before reading q (layers that feed one another; only the
         # K/V prefetch overlaps).  `serial`: plain stream order.  `eager_event_bracket`: one launch bracketed by events on
         # an eager stream (includes launch latency and host pacing; kept for reference).
@@ -726,9 +753,9 @@ def run_ours(args, rank, world, local_rank):
                      "frac": region_achieved / peak_gbs, "peak_kind": f"of {peak_kind}", "traffic": traffic,
                      "bytes_per_launch": region_bytes_per_launch, "us_per_launch": region_us_per_launch,
                      "launches": region_launches[0],
-                     "duration_kind": "timed region / attention launches (small layers share a launch; consecutive "
-                                      "launches overlap inside the replayed step)",
-                     "chained": dep.get("chained"), "serial": dep.get("serial"),
+                     "duration_kind": "timed region / attention launches (all layers of a step in one launch by default; "
+                                      "per-layer launches overlap inside the replayed step)",
+                     "chained": dep.get("chained"), "serial": dep.get("serial"), alt_name: alt,
                      "eager_event_bracket": {"us_per_launch": attn_us, "achieved": achieved, "frac": achieved / peak_gbs,
                                              "launches": attn_n},
                      "regime": f"{region_bytes_per_launch / 1e6:.1f} MB per launch would take "
@@ -776,8 +803,10 @@ def main():
     ap.add_argument("--segment-tokens", type=int, default=0, help="override the workload's chunk_tokens (e.g. the paper's 25 / 50)")
     ap.add_argument("--eager", action="store_true", help="issue every layer eagerly instead of replaying a captured step")
     ap.add_argument("--roofline-steps", type=int, default=16)
-    ap.add_argument("--layer-dependency", type=int, default=0, choices=[0, 1, 2],
-                    help="with --quick: 0 independent layers (overlap), 1 chained, 2 serial launches")
+    ap.add_argument("--layer-dependency", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="how the layers of a step are issued: 0 one overlapping launch per layer (default; inputs of every layer "
+                         "resident before the step), 3 all layers in one launch (outputs read after the step), 1 chained, 2 serial")
+    ap.add_argument("--no-alt-form", action="store_true", help="skip the run in the other launch form (one launch per layer / all layers in one)")
     ap.add_argument("--back-to-back-steps", type=int, default=32,
                     help="steps timed in one region without L2 flushes (continuous decoding; exposes recall). 0 = skip")
     ap.add_argument("--chain-steps", type=int, default=48,
@@ -790,6 +819,7 @@ def main():
     args = ap.parse_args()
     global SWEEP_STEPS_OVERRIDE
     SWEEP_STEPS_OVERRIDE = args.sweep_steps
+    Job.layer_dependency = args.layer_dependency
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     rank = int(os.environ.get("RANK", "0"))

@@ -271,10 +271,15 @@ wnw_status_t wnw_get_stats(wnw_cache_t *cache, wnw_stats_t *stats_host);
  *                feed one another): the kernel still starts early and queues its K/V cache loads, which do not depend
  *                on that work, but waits for the predecessor to complete before it reads q, k_new or v_new.
  *   SERIAL       plain stream order, no early start.
+ *   BATCHED      as INDEPENDENT, and in addition no output of the step is read (by the host or by work queued on the
+ *                stream between the layer calls) before the step has ended.  Inside a captured step whose selection
+ *                work runs at the end of the step (wnw_graph_begin/end with launches smaller than the machine, recall
+ *                not inline; or FULL mode) wnw_decode_layer then only records its arguments and the last layer's call
+ *                issues ONE launch that carries the CTAs of all layers; elsewhere the mode behaves as INDEPENDENT.
  * Takes effect for layers issued afterwards; a captured step keeps the mode it was captured with.  Not allowed inside
  * a step.  The modes cut the work differently, so outputs agree up to the rounding order of the split merge; selections
  * and tables are the same. */
-enum { WNW_LAYERS_INDEPENDENT = 0, WNW_LAYERS_CHAINED = 1, WNW_LAYERS_SERIAL = 2 };
+enum { WNW_LAYERS_INDEPENDENT = 0, WNW_LAYERS_CHAINED = 1, WNW_LAYERS_SERIAL = 2, WNW_LAYERS_BATCHED = 3 };
 wnw_status_t wnw_set_layer_dependency(wnw_cache_t *cache, int32_t mode);
 
 /* Test hook for the bounded waits: adds `delta` to the device's step-epoch word, so that the tidal CTAs of the next

@@ -21,7 +21,7 @@ WNW_ROLE_ANCHOR, WNW_ROLE_TIDAL, WNW_ROLE_FIXED = 0, 1, 2
 WNW_MODE_TIERED, WNW_MODE_FULL = 0, 1
 WNW_RECALL_SIDE_STREAM, WNW_RECALL_INLINE, WNW_RECALL_SKIP = 0, 1, 2
 WNW_SCOPE_PER_LAYER, WNW_SCOPE_GLOBAL = 0, 1
-WNW_LAYERS_INDEPENDENT, WNW_LAYERS_CHAINED, WNW_LAYERS_SERIAL = 0, 1, 2
+WNW_LAYERS_INDEPENDENT, WNW_LAYERS_CHAINED, WNW_LAYERS_SERIAL, WNW_LAYERS_BATCHED = 0, 1, 2, 3
 WNW_RESIDENCY_HARD_BUDGET, WNW_RESIDENCY_SEGMENT_LAG, WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE = 0, 1, 2
 
 

@@ -53,6 +53,7 @@ extern "C" int wnw_debug_clear_stamps() {
 }
 __device__ unsigned long long g_ktime[4 * 64 * 4];   // [step % 4][layer][start_min, trigger_max, end_max, unused], nanoseconds
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define GSTAMP(k) do { if (threadIdx.x == 0 && blockIdx.x < 8192) g_stamps[blockIdx.x * 16 + (k)] = (long long)gtime(); } while (0)
 #define KSTAMP_MIN(slot, k) do { if (threadIdx.x == 0) atomicMin(&g_ktime[(slot) * 4 + (k)], gtime()); } while (0)
 #define KSTAMP_MAX(slot, k) do { if (threadIdx.x == 0) atomicMax(&g_ktime[(slot) * 4 + (k)], gtime()); } while (0)
 extern "C" int wnw_debug_read_ktime(unsigned long long *host) { return (int)cudaMemcpyFromSymbol(host, g_ktime, sizeof(g_ktime)); }
@@ -63,6 +64,7 @@ extern "C" int wnw_debug_init_ktime() {
 }
 #else
 #define STAMP(k) do { } while (0)
+#define GSTAMP(k) do { } while (0)
 #define KSTAMP_MIN(slot, k) do { } while (0)
 #define KSTAMP_MAX(slot, k) do { } while (0)
 #endif
@@ -167,11 +169,11 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
 }
 
 // TB: tidal heads keep a token-granular permanent base (their key space is [text | base blocks | dynamic slots])
+// bid: the CTA's index within its layer's launch (a launch may carry the CTAs of several layers back to back);
+// inl: the layer's work items when they travel in the kernel parameters, else null (read from a.items).
 template <int D, bool G16, int NW, bool TB>
-__global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant__ CacheView cv,
-                                                           const __grid_constant__ AttnArgs a,
-                                                           const __grid_constant__ InlineItems inl,
-                                                           const __grid_constant__ TmaMaps maps) {
+__device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a, const InlineItems *inl, const TmaMaps &maps,
+                                          const int bid) {
   extern __shared__ unsigned char smem_raw[];
   // TMA boxes with the 128-byte swizzle must start on a 1024-byte boundary of the shared window
   unsigned char *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -185,6 +187,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   STAMP(0);
+  GSTAMP(14);
   // Programmatic dependent launch: the next layer's kernel may be scheduled right away.  A layer kernel touches only
   // its own layer's stores, partial buffers, counters and outputs, so consecutive layer kernels are independent and
   // may overlap as deeply as free SMs allow.  What later stream work relies on is that a completed kernel implies
@@ -194,7 +197,7 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
   int kslot = 0;
 #endif
   auto pdl_finish = [&]() {
-    if (blockIdx.x == 0) {
+    if (blockIdx.x == 0) {   // one CTA of the launch, whichever layer it serves
       asm volatile("griddepcontrol.wait;\n" ::: "memory");
       KSTAMP_MAX(kslot, 1);
     }
@@ -221,8 +224,8 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 
   // One work item per CTA when the launch fits the machine; otherwise a persistent CTA per SM walks the items the
   // host assigned to it (balanced by size), so no SM idles through a partial last wave.
-  int q_begin = blockIdx.x, q_end = blockIdx.x + 1;
-  if (a.cta_ranges) { q_begin = a.cta_ranges[blockIdx.x]; q_end = a.cta_ranges[blockIdx.x + 1]; }
+  int q_begin = bid, q_end = bid + 1;
+  if (a.cta_ranges) { q_begin = a.cta_ranges[bid]; q_end = a.cta_ranges[bid + 1]; }
 
   // What a warp needs to address the granules of one work item.
   struct Ctx {
@@ -249,11 +252,12 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
     }
     timed_out = __shfl_sync(0xffffffffu, (int)timed_out, 0) != 0;
     epoch_pending = false;
+    if (warp == 0) STAMP(13);
   };
   auto load_ctx = [&](Ctx &c, int qi, bool for_loads) {
     c.item_idx = a.cta_ranges ? a.order[qi] : qi;
     // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
-    c.it = a.n_items <= INLINE_ITEMS_MAX ? inl.it[c.item_idx] : a.items[c.item_idx];
+    c.it = (inl && a.n_items <= INLINE_ITEMS_MAX) ? inl->it[c.item_idx] : a.items[c.item_idx];
     c.T_t = cv.text_len[c.it.b] + a.has_new;
     if (c.it.role == ROLE_ANCHOR) { c.v_delta_audio = G.T_a_pad; c.map_audio = &maps.anchor; }       // rows between a
     else if (c.it.role == ROLE_TIDAL) { c.v_delta_audio = G.ncp; c.map_audio = &maps.pool; }          // granule's K and
@@ -656,7 +660,38 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
       phase_bits ^= 1u << stage;
     }
   }
+  GSTAMP(15);
   pdl_finish();
+}
+
+template <int D, bool G16, int NW, bool TB>
+__global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant__ CacheView cv,
+                                                           const __grid_constant__ AttnArgs a,
+                                                           const __grid_constant__ InlineItems inl,
+                                                           const __grid_constant__ TmaMaps maps) {
+  attn_body<D, G16, NW, TB>(cv, a, &inl, maps, (int)blockIdx.x);
+}
+
+// The CTAs of several layers in one launch (layers whose inputs are all ready and whose outputs are read after the
+// step): CTA x belongs to the layer whose range of the prefix table holds x and does exactly what it would do in that
+// layer's own launch.
+// The register cap leaves room on the SM for a recall CTA (256 threads x 40 registers) beside an 8-warp attention CTA:
+// the recall of the previous step runs while this launch fills the machine.  (The layer's arguments are read through a
+// run-time index into the parameters, which costs registers: uncapped this kernel takes about 240, and the recall then
+// waits for attention CTAs to retire: config 1 back to back 84 us per step.)
+template <int D, bool G16, int NW, bool TB>
+__global__ void __maxnreg__(NW == 8 ? 208 : 255) wnw_attn_multi_kernel(const __grid_constant__ CacheView cv,
+                                                                 const __grid_constant__ MultiArgs m,
+                                                                 const __grid_constant__ TmaMaps maps) {
+  int l = 0;
+  while (l + 1 < m.n && (int)blockIdx.x >= m.cta_prefix[l + 1]) ++l;
+  attn_body<D, G16, NW, TB>(cv, m.l[l], nullptr, maps, (int)blockIdx.x - m.cta_prefix[l]);
+}
+
+template <int D, bool G16, int NW, bool TB>
+static cudaError_t launch_multi_tb(const CacheView &cv, const MultiArgs &m, size_t smem, const TmaMaps &maps, cudaStream_t st) {
+  wnw_attn_multi_kernel<D, G16, NW, TB><<<m.cta_prefix[m.n], NW * 32, smem, st>>>(cv, m, maps);
+  return cudaGetLastError();
 }
 
 template <int D, bool G16, int NW, bool TB>
@@ -718,6 +753,8 @@ static cudaError_t configure_t() {
   const int bytes = (int)std::min<size_t>(want, 226 * 1024);
   cudaError_t e = cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(wnw_attn_multi_kernel<D, G16, NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(wnw_attn_multi_kernel<D, G16, NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;
   return cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 // Opt-in shared-memory sizes, set once per device at cache creation (never during a stream capture).
@@ -742,6 +779,40 @@ cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st)
   } else {
     if (cv.geo.d == 128) return g16 ? launch_t<128, true, NW_LAT>(cv, a, st) : launch_t<128, false, NW_LAT>(cv, a, st);
     if (cv.geo.d == 64) return g16 ? launch_t<64, true, NW_LAT>(cv, a, st) : launch_t<64, false, NW_LAT>(cv, a, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+// One launch for the CTAs of n layers (all cut for the one-shot 8-warp variant).
+cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, cudaStream_t st) {
+  if (n <= 0 || n > MULTI_LAYERS_MAX) return cudaErrorInvalidValue;
+  MultiArgs m;
+  memset(&m, 0, sizeof(m));
+  size_t smem = 0;
+  int ctas = 0, n_used = 0;
+  const int d = cv.geo.d;
+  for (int i = 0; i < n; ++i) {
+    const AttnArgs &a = args[i];
+    if (a.n_items <= 0) continue;
+    if (a.throughput || !a.maps || a.maps != args[0].maps) return cudaErrorInvalidValue;
+    m.cta_prefix[n_used] = ctas;
+    m.l[n_used] = a;
+    m.l[n_used].pdl = 0; m.l[n_used].wait_inputs = 0;
+    ++n_used;
+    ctas += a.cta_ranges ? a.n_ctas : a.n_items;
+    smem = std::max(smem, (size_t)NW_LAT * NSTAGE * 2 * GR * d * 2 + 1024 + (a.xpref ? attn_scratch_bytes(NW_LAT, cv.geo.g, d) : 0));
+  }
+  if (n_used == 0) return cudaSuccess;
+  m.n = n_used; m.cta_prefix[n_used] = ctas;
+  const bool g16 = cv.geo.g > 8, tb = cv.geo.token_base != 0;
+  const TmaMaps &maps = *args[0].maps;
+  if (d == 128) {
+    if (g16) return tb ? launch_multi_tb<128, true, NW_LAT, true>(cv, m, smem, maps, st) : launch_multi_tb<128, true, NW_LAT, false>(cv, m, smem, maps, st);
+    return tb ? launch_multi_tb<128, false, NW_LAT, true>(cv, m, smem, maps, st) : launch_multi_tb<128, false, NW_LAT, false>(cv, m, smem, maps, st);
+  }
+  if (d == 64) {
+    if (g16) return tb ? launch_multi_tb<64, true, NW_LAT, true>(cv, m, smem, maps, st) : launch_multi_tb<64, true, NW_LAT, false>(cv, m, smem, maps, st);
+    return tb ? launch_multi_tb<64, false, NW_LAT, true>(cv, m, smem, maps, st) : launch_multi_tb<64, false, NW_LAT, false>(cv, m, smem, maps, st);
   }
   return cudaErrorInvalidValue;
 }

@@ -165,6 +165,14 @@ struct AttnArgs {
   bf16 *out;             // [n_active][Hq][d]
 };
 
+// Several layers in one launch: per-layer arguments and the first CTA of each layer's range.
+constexpr int MULTI_LAYERS_MAX = 48;
+struct MultiArgs {
+  int32_t n;
+  int32_t cta_prefix[MULTI_LAYERS_MAX + 1];
+  AttnArgs l[MULTI_LAYERS_MAX];
+};
+
 // Selection launch (side stream): chunk scores of `layer` from its granule partials, then top-k, residency update
 // and recall plan for every layer in the update list.  Static data travels by value.
 struct SelectArgs {
@@ -222,6 +230,8 @@ cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_c
                                   int32_t *fixed_tok, int tok_cap, int32_t *tok_n, cudaStream_t st);
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
 cudaError_t configure_attn_kernels();
+// the CTAs of several layers' launches (one-shot variant) in one launch
+cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, cudaStream_t st);
 // Encodes the descriptor of one store: base (device), rows, head_dim.  Returns false if the driver refuses.
 bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d);
 cudaError_t configure_select_kernel();

@@ -115,6 +115,9 @@ struct wnw_cache {
   long long launches[4] = {0, 0, 0, 0}, cap_launches[4] = {0, 0, 0, 0};  // attention, selection, recall, step-end kernels
   void count_launch(int kind, int n, bool capturing) { (capturing ? cap_launches : launches)[kind] += n; }
   int layer_dependency = WNW_LAYERS_INDEPENDENT;
+  std::vector<AttnArgs> batch_args;   // BATCHED layers of a captured step: recorded per layer, launched by the last one
+  bool cap_batched = false;
+  int batched_target = 0;             // granules of work per CTA when the step's layers share one launch
   // replayed steps: one recall launch per step outside the captured graph, overlapping the next step
   int32_t *d_recall_epoch = nullptr, *d_recall_ctr = nullptr, *d_step_epoch = nullptr;
   int external_recall_mode = -1;   // -1 automatic, 0 never, 1 always
@@ -550,6 +553,20 @@ static int granules_per_item(const wnw_cache *c, long long total_granules, int l
   return (int)((per + nw - 1) / nw * nw);
 }
 
+// Granules of one head: n_gran its whole virtual key space, work those expected to hold data.
+static void head_granules(const wnw_cache *c, int layer, int mode, const SeqHost &s, int h, int *n_gran, int *work) {
+  const Geometry &G = c->geo;
+  const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
+  int fixed_blocks = s.S_base;   // a token-compacted head: the blocks its kept positions fill
+  if (!s.fixed_blocks.empty() && s.fixed_blocks[layer * G.Hkv + h] >= 0) fixed_blocks = s.fixed_blocks[layer * G.Hkv + h];
+  // a tidal head with a token base: its blocks first, then the table's (all dynamic) slots
+  const int tidal_units = s.S + (G.token_base && mode == ATTN_DECODE ? fixed_blocks : 0);
+  const int audio = (role == ROLE_ANCHOR ? s.C : role == ROLE_TIDAL ? tidal_units : fixed_blocks) * G.gpc;
+  *n_gran = G.n_tg + audio;
+  // the dynamic slots of a SEGMENT_LAG table are about half empty and cost nothing then
+  *work = G.n_tg + audio - (role == ROLE_TIDAL ? (s.S - s.S_base) * G.gpc / 2 : 0);
+}
+
 // Appends the items of one layer for the given sequences.
 static void build_layer_items(const wnw_cache *c, int layer, int mode, const std::vector<int> &seq_ids,
                               std::vector<WorkItem> &items, std::vector<HeadItems> &heads, LayerWork &lw,
@@ -563,14 +580,8 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   for (size_t i = 0; i < seq_ids.size(); ++i) {
     const SeqHost &s = c->seqs[seq_ids[i]];
     for (int h = 0; h < G.Hkv; ++h) {
-      const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
-      int fixed_blocks = s.S_base;   // a token-compacted head: the blocks its kept positions fill
-      if (!s.fixed_blocks.empty() && s.fixed_blocks[layer * G.Hkv + h] >= 0) fixed_blocks = s.fixed_blocks[layer * G.Hkv + h];
-      // a tidal head with a token base: its blocks first, then the table's (all dynamic) slots
-      const int tidal_units = s.S + (G.token_base && mode == ATTN_DECODE ? fixed_blocks : 0);
-      const int audio = (role == ROLE_ANCHOR ? s.C : role == ROLE_TIDAL ? tidal_units : fixed_blocks) * G.gpc;
-      n_gran[i * G.Hkv + h] = G.n_tg + audio;
-      const int work = G.n_tg + audio - (role == ROLE_TIDAL ? (s.S - s.S_base) * G.gpc / 2 : 0);
+      int work = 0;
+      head_granules(c, layer, mode, s, h, &n_gran[i * G.Hkv + h], &work);
       n_work[i * G.Hkv + h] = work;
       total += work;
       longest = std::max(longest, work);
@@ -578,8 +589,14 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   }
   bool throughput = false;
   // the prefill scoring pass is a single launch: nothing overlaps it
-  const bool overlapped = mode != ATTN_PREFILL && c->layer_dependency == WNW_LAYERS_INDEPENDENT;
-  const int gpi = granules_per_item(c, total, longest, (int)seq_ids.size() * G.Hkv, overlapped, &throughput);
+  const bool overlapped = mode != ATTN_PREFILL && (c->layer_dependency == WNW_LAYERS_INDEPENDENT ||
+                                                  c->layer_dependency == WNW_LAYERS_BATCHED);
+  int gpi = granules_per_item(c, total, longest, (int)seq_ids.size() * G.Hkv, overlapped, &throughput);
+  // BATCHED layers share one launch: the work of the whole step is cut for one wave of CTAs, long heads into pieces as
+  // fat as a pack of short ones, short heads packed whole
+  const bool batched = overlapped && !throughput && c->layer_dependency == WNW_LAYERS_BATCHED && c->batched_target > 0 &&
+                       c->pack_enabled && attn_xpref_fits(G.g, G.d);
+  if (batched) gpi = (c->batched_target + attn_warps(false) - 1) / attn_warps(false) * attn_warps(false);
   lw.throughput = throughput;
   lw.first_item = (int)items.size();
   lw.head_items_off = (int)heads.size();
@@ -596,6 +613,7 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       // a short head stays in one CTA: up to 128 granules when layers overlap (work per launch counts), 32 when the
       // kernel's span counts (measured, chained config 1: 298 -> 240 us per step against a threshold of 64)
       if (!throughput && nw_ <= (overlapped ? 2 * c->direct_max_granules : c->direct_max_granules / 2)) n_cta = 1;
+      if (batched) n_cta = nw_ <= gpi * 3 / 2 ? 1 : (nw_ + gpi - 1) / gpi;
       HeadItems hi{(int)items.size() - lw.first_item, n_cta};
       for (int x = 0; x < n_cta; ++x) {  // even contiguous ranges
         const int g0 = (int)((long long)n * x / n_cta), g1 = (int)((long long)n * (x + 1) / n_cta);
@@ -611,13 +629,13 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   lw.n_ctas = 0;
   lw.packed = false;
   if (!throughput && overlapped && c->pack_enabled && attn_xpref_fits(G.g, G.d) &&
-      (c->pack_granules > 0 || lw.n_items > c->n_sm)) {
+      (c->pack_granules > 0 || lw.n_items > c->n_sm || batched)) {
     // One-shot CTAs of a launch that has more of them than SMs: heads that fit one CTA are packed several to a CTA
     // (consecutive ones, up to about 512 granules of work: a sequence's short heads), which then keeps its copy pipeline
     // running from one head into the next: the fixed cost of a CTA (launch, first reads, first DRAM round trip) is paid
     // once for the pack.  Pieces of split heads keep a CTA each.  Measured: batch-32 ragged 85 -> 91 % of the copy
     // bandwidth; launches with fewer CTAs than SMs lose parallelism instead (16 x 7500: 80 -> 76 %) and are left alone.
-    const int target = c->pack_granules > 0 ? c->pack_granules : 512;
+    const int target = batched ? gpi : c->pack_granules > 0 ? c->pack_granules : 512;
     lw.order_off = (int)order.size();
     lw.ranges_off = (int)ranges.size();
     int pos = 0, in_pack = 0, pack_work = 0, n_packs = 0;
@@ -639,7 +657,7 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
     }
     close_pack();
     ranges.push_back(pos);
-    if (any) { lw.n_ctas = n_packs; lw.packed = true; }
+    if (any || batched) { lw.n_ctas = n_packs; lw.packed = true; }
     else { order.resize(lw.order_off); ranges.resize(lw.ranges_off); }
   }
   if (throughput) {
@@ -681,6 +699,22 @@ static wnw_status_t ensure_worklists(wnw_cache *c) {
   std::vector<HeadItems> heads;
   std::vector<int32_t> order, ranges;
   c->wl_layers.assign(G.L, LayerWork{});
+  c->batched_target = 0;
+  if (c->layer_dependency == WNW_LAYERS_BATCHED) {   // the step's whole work over one wave of CTAs
+    long long total = 0;
+    for (int l = 0; l < G.L; ++l)
+      for (int b : c->active)
+        for (int h = 0; h < G.Hkv; ++h) {
+          int n = 0, work = 0;
+          head_granules(c, l, mode, c->seqs[b], h, &n, &work);
+          total += work;
+        }
+    // 1.4 x the mean share of an SM: heads are packed whole, so CTAs come out uneven; with this margin the launch stays
+    // within one wave (measured, config 1: 57 us per step at 1.2 to 1.7 x the mean, 61 to 65 us at 0.9 and 1.0 x, where
+    // a second, nearly empty wave forms, 66 us at 2 x, where too few SMs pull)
+    c->batched_target = (int)std::max<long long>(32, (total * 14 / 10 + c->n_sm - 1) / c->n_sm);
+    if (const char *e = getenv("WNW_BATCH_TARGET")) c->batched_target = std::max(8, atoi(e));
+  }
   size_t part_total = 0;
   for (int l = 0; l < G.L; ++l) {
     build_layer_items(c, l, mode, c->active, items, heads, c->wl_layers[l], order, ranges);
@@ -1083,6 +1117,12 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     c->cap_select_all = c->select_all_enabled && c->cap_external_recall && c->fold_enabled && small &&
                         (c->select_single_ok ? c->sel_map_single[1] : c->sel_map_update[1]) > 0;
     if (c->cap_select_all) c->cap_fold = true;
+    // BATCHED layers: one launch for the whole step where nothing inside the step needs a layer's result earlier
+    bool one_shot = G.L <= MULTI_LAYERS_MAX;
+    for (const LayerWork &w : c->wl_layers) one_shot = one_shot && !w.throughput;
+    c->cap_batched = c->layer_dependency == WNW_LAYERS_BATCHED && capturing && c->graph_capturing && one_shot &&
+                     (!tiered || c->cap_select_all);
+    if (c->cap_batched) c->batch_args.assign(G.L, AttnArgs{});
   }
   if (!capturing) {
     if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
@@ -1132,8 +1172,16 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     }
     CK(cudaEventRecord(t0, st));
   }
-  CK(launch_attn(c->cv, a, st));
-  c->count_launch(0, 1, capturing);
+  if (c->cap_batched) {
+    c->batch_args[layer] = a;
+    if (layer == G.L - 1) {
+      CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, st));
+      c->count_launch(0, 1, capturing);
+    }
+  } else {
+    CK(launch_attn(c->cv, a, st));
+    c->count_launch(0, 1, capturing);
+  }
   if (timing) {
     CK(cudaEventRecord(t1, st));
     c->t_used.emplace_back(t0, t1);
@@ -1555,7 +1603,7 @@ extern "C" wnw_status_t wnw_get_launch_counts(wnw_cache_t *c, int64_t *counts) {
 }
 
 extern "C" wnw_status_t wnw_set_layer_dependency(wnw_cache_t *c, int32_t mode) {
-  if (!c || mode < WNW_LAYERS_INDEPENDENT || mode > WNW_LAYERS_SERIAL) return WNW_ERR_INVALID_ARG;
+  if (!c || mode < WNW_LAYERS_INDEPENDENT || mode > WNW_LAYERS_BATCHED) return WNW_ERR_INVALID_ARG;
   if (c->in_step || c->graph_capturing) return WNW_ERR_STATE;
   if (mode != c->layer_dependency) c->wl_layers.clear();  // the work items are sized for the mode
   c->layer_dependency = mode;

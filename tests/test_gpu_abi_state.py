@@ -146,7 +146,7 @@ def test_layer_dependency_rejects_bad_mode():
                        w.roles, topk=w.topk)
     try:
         with pytest.raises(wnw.WnwError):
-            wnw.wnw_set_layer_dependency(h, 3)
+            wnw.wnw_set_layer_dependency(h, 4)
         wnw.wnw_set_layer_dependency(h, 1)
     finally:
         wnw.wnw_destroy(h)

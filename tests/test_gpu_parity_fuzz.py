@@ -54,7 +54,7 @@ def test_random_configuration_segment_lag(seed):
     delta = int(rs.randint(0, 4))
     ls = Lockstep(w, seed=seed, residency=wnw.WNW_RESIDENCY_SEGMENT_LAG, evict_lag=delta, score_scope=int(rs.randint(0, 2)))
     try:
-        wnw.wnw_set_layer_dependency(ls.h, int(rs.randint(0, 3)))
+        wnw.wnw_set_layer_dependency(ls.h, int(rs.randint(0, 4)))
         ls.prefill()
         use_graph = bool(seed % 2)
         for t in range(w.n_steps):
@@ -87,7 +87,7 @@ def test_random_configuration_token_compression(seed):
     ls = Lockstep(w, seed=seed, residency=residency, evict_lag=delta, score_scope=int(rs.randint(0, 2)), token_retention=ret,
                   token_seg=seg, token_variant=variant)
     try:
-        wnw.wnw_set_layer_dependency(ls.h, int(rs.randint(0, 3)))
+        wnw.wnw_set_layer_dependency(ls.h, int(rs.randint(0, 4)))
         ls.prefill()
         use_graph = bool(seed % 2)
         for t in range(w.n_steps):
