@@ -88,7 +88,7 @@ enum { WNW_SCOPE_PER_LAYER = 0, WNW_SCOPE_GLOBAL = 1 };
  *                each segment with the positions that are NOT in the base first, so a fetched segment contributes
  *                exactly its complement.  A tidal head attends to [text | its kept positions | the complements of the
  *                segments in the layer's dynamic slots].  Sequences must be placed with wnw_place_prefill_tokens
- *                (segment_tokens = chunk_tokens, variant 0); wnw_place_prefill and _multi return WNW_ERR_STATE.
+ *                (segment_tokens = chunk_tokens); wnw_place_prefill and _multi return WNW_ERR_STATE.
  *                A compact store holds floor(budget*C)+2*topk*(evict_lag+1) blocks of chunk_tokens positions. */
 enum { WNW_RESIDENCY_HARD_BUDGET = 0, WNW_RESIDENCY_SEGMENT_LAG = 1, WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE = 2 };
 
@@ -173,8 +173,9 @@ wnw_status_t wnw_place_prefill_multi(wnw_cache_t *cache, int32_t seq, int32_t la
  *                 max_audio_tokens, under the lag residencies the budget's share plus the dynamic slots, times
  *                 chunk_tokens): WNW_ERR_CAPACITY otherwise, nothing placed.
  * With the residency SEGMENT_LAG_TOKEN_BASE the layer's tidal heads are compressed the same way, each by its own
- * scores (their tables start empty); then segment_tokens must equal chunk_tokens and variant must be 0
- * (WNW_ERR_UNSUPPORTED otherwise).
+ * scores (their tables start empty); then segment_tokens must equal chunk_tokens (WNW_ERR_UNSUPPORTED otherwise).
+ * With variant 1 a head's base holds a different number of positions in every segment; a fetched segment then
+ * contributes its length minus that number (kept per head and segment on the device).
  * Scratch and the position lists are allocated by the first call (device memory; not allocation-free).  In FULL mode
  * this is wnw_place_prefill_multi.  Errors as wnw_place_prefill; WNW_ERR_INVALID_ARG for a retention outside [0,1],
  * segment_tokens < 1 or an unknown variant. */

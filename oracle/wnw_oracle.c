@@ -56,7 +56,7 @@
  *     segment of `seg` tokens keeps its floor((double)retention * length) best positions (variant 1: the same total
  *     from the whole head); the head then attends to [text | kept positions].  Tidal tables stay chunk-granular,
  *     except with residency 2 (SEGMENT_LAG with a token-granular base): no segment is permanent as a whole; every tidal
- *     head keeps its own per-segment best positions for good (variant 0 only) and attends to [text | its kept
+ *     head keeps its own best positions for good (either variant) and attends to [text | its kept
  *     positions | all positions of the segments resident in the layer's dynamic slots]; a selected segment that is
  *     not in a dynamic slot counts as a miss (its complement has to be fetched).
  *     Pinned in tests/test_oracle_tokens.py against numpy sorts, a separate numpy softmax and hand-worked cases.
@@ -590,7 +590,6 @@ int wnwo_place_prefill_tokens(Oracle *o, int seq, int layer, const uint16_t *k, 
                               int audio_begin, int audio_end, const uint16_t *q_text, int n_q, const float *retention,
                               int seg, int variant) {
   if (!retention || seg < 1) return WNWO_ERR_ARG;
-  if (o && o->residency == 2 && variant != 0) return WNWO_ERR_ARG; /* tidal bases keep a per-segment quota */
   int rc = place_multi(o, seq, layer, k, v, n_tokens, audio_begin, audio_end, q_text, n_q);
   if (rc) return rc;
   Seq *s = &o->seq[seq];

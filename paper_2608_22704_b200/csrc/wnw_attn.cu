@@ -232,6 +232,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     WorkItem it;
     int item_idx, T_t, v_delta_audio, first, n_my;
     int m_full, m_tail;   // token-granular base: positions of a full / of the last segment that live in the base already
+    const int32_t *seg_kept;   // ... or, where they differ by segment (m_full < 0), the head's per-segment counts
     const CUtensorMap *map_audio;
   };
   // Replayed steps: the recall that refreshed this layer's slots ran outside the captured graph, possibly still
@@ -266,6 +267,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     if (TB && c.it.role == ROLE_TIDAL) {
       const int2 m = cv.tok_m[((long long)c.it.b * G.L + a.layer) * G.Hkv + c.it.h];
       c.m_full = m.x; c.m_tail = m.y;
+      c.seg_kept = cv.seg_kept + ((long long)c.it.b * cv.tid_total + li.tid_prefix + c.it.ridx) * G.C_max;
     }
     c.first = c.it.g0 + warp;
     c.n_my = c.first < c.it.g1 ? (c.it.g1 - c.first + NW - 1) / NW : 0;
@@ -292,7 +294,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
         len = c.it.T_a - cid * G.nc;
         if (len > G.nc) len = G.nc;
         // token base: a fetched segment holds its complement first; the last segment has its own count
-        if (TB) len -= (c.it.T_a - cid * G.nc > G.nc) ? c.m_full : c.m_tail;
+        if (TB) len -= c.m_full < 0 ? c.seg_kept[cid] : (c.it.T_a - cid * G.nc > G.nc) ? c.m_full : c.m_tail;
       }
       len -= off;
     }

@@ -86,7 +86,10 @@ struct CacheView {
   int32_t *sel, *n_sel;              // [B][L][topk], [B][L]
   int32_t *plan, *n_plan;            // [B][L][plan_cap][2] (chunk, slot), [B][L]
   int32_t *fixed_chunks, *fixed_n;   // [B][F_tot][FB], [B][F_tot]
-  int2 *tok_m;                       // [B][L][Hkv] token-granular tidal base: kept positions of a full / the last segment
+  int2 *tok_m;                       // [B][L][Hkv] token-granular tidal base: kept positions of a full / the last segment;
+                                     //   x < 0: they differ by segment (global top-k variant), see seg_kept
+  int32_t *seg_kept;                 // [B][tidal heads over all layers][C_max] kept positions of every segment
+  int32_t tid_total;                 // tidal heads over all layers
   float *pre;                        // [B][L][Hkv][C_max]
   unsigned long long *stats;         // [B][4] hits, misses, evictions, recall_bytes
   bf16 **mirror;                     // [B] pinned host mirrors (device-visible addresses)

@@ -393,6 +393,8 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   CKC(dev_alloc(c, &cv.fixed_chunks, B * std::max(G.F_tot, 1) * std::max(G.FB, 1)));
   CKC(dev_alloc(c, &cv.fixed_n, B * std::max(G.F_tot, 1)));
   CKC(dev_alloc(c, &cv.tok_m, G.token_base ? B * (size_t)L * Hkv : 1));
+  CKC(dev_alloc(c, &cv.seg_kept, G.token_base ? B * (size_t)std::max(t_tot, 1) * std::max(G.C_max, 1) : 1));
+  cv.tid_total = t_tot;
   CKC(dev_alloc(c, &cv.pre, B * L * Hkv * std::max(G.C_max, 1)));
   CKC(dev_alloc(c, &cv.stats, B * 4));
   CKC(dev_alloc(c, &cv.mirror, B));
@@ -927,7 +929,7 @@ extern "C" wnw_status_t wnw_place_prefill_tokens(wnw_cache_t *c, int32_t seq, in
   const LayerInfo &li = c->layers[layer];
   const int T_a = audio_end - audio_begin, n_tidal_base = G.token_base ? li.n_tidal : 0;
   const int n_comp = full ? 0 : li.n_fixed + n_tidal_base;   // compressed heads: the fixed ones, then the tidal bases
-  if (n_tidal_base > 0 && (segment_tokens != G.nc || variant != 0)) return WNW_ERR_UNSUPPORTED;
+  if (n_tidal_base > 0 && segment_tokens != G.nc) return WNW_ERR_UNSUPPORTED;   // the quota's segment is the storage segment
   const int tok_cap = G.FB * G.nc;
   const int C_b = (T_a + G.nc - 1) / G.nc, tail_len = T_a - (C_b - 1) * G.nc;
   std::vector<int> blocks(G.Hkv, -1);
@@ -939,8 +941,9 @@ extern "C" wnw_status_t wnw_place_prefill_tokens(wnw_cache_t *c, int32_t seq, in
     const int n = kept_positions(T_a, segment_tokens, retention[h]);
     if (n > tok_cap) return WNW_ERR_CAPACITY;   // the head's compact store holds FB blocks of chunk_tokens rows
     blocks[h] = (n + G.nc - 1) / G.nc;
-    if (role == ROLE_TIDAL && T_a > 0)
-      m_host[h] = make_int2((int)std::floor((double)retention[h] * (double)G.nc), (int)std::floor((double)retention[h] * (double)tail_len));
+    if (role == ROLE_TIDAL && T_a > 0)   // the global variant keeps a different number per segment: the device table says
+      m_host[h] = variant != 0 ? make_int2(-1, -1)
+                               : make_int2((int)std::floor((double)retention[h] * (double)G.nc), (int)std::floor((double)retention[h] * (double)tail_len));
   }
   wnw_status_t rc = place_multi(c, seq, layer, k_dev, v_dev, n_tokens, audio_begin, audio_end, q_text_dev, n_queries, cuda_stream);
   if (rc != WNW_OK || n_comp == 0 || T_a == 0) return rc;
@@ -1540,6 +1543,11 @@ extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
   CK(cudaMemcpy(slot_chunk.data(), c->cv.slot_chunk, slot_chunk.size() * 4, cudaMemcpyDeviceToHost));
   CK(cudaMemcpy(fixed_n.data(), c->cv.fixed_n, fixed_n.size() * 4, cudaMemcpyDeviceToHost));
   CK(cudaMemcpy(fixed_chunks.data(), c->cv.fixed_chunks, fixed_chunks.size() * 4, cudaMemcpyDeviceToHost));
+  std::vector<int32_t> seg_kept;
+  if (G.token_base) {
+    seg_kept.resize(B * (size_t)std::max(c->tid_total, 1) * std::max(G.C_max, 1));
+    CK(cudaMemcpy(seg_kept.data(), c->cv.seg_kept, seg_kept.size() * 4, cudaMemcpyDeviceToHost));
+  }
   wnw_stats_t r{};
   auto len_of = [&](const SeqHost &sq, int ch) { return std::min(G.nc, sq.T_a - ch * G.nc); };
   for (size_t b = 0; b < B; ++b) {
@@ -1563,11 +1571,12 @@ extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
           if (c->roles[l * G.Hkv + h] != ROLE_TIDAL) continue;
           const size_t fh = b * G.F_tot + G.F_fix + li.tid_prefix + c->role_idx[l * G.Hkv + h];
           const int2 m = sq.tok_m.empty() ? make_int2(0, 0) : sq.tok_m[l * G.Hkv + h];
+          const size_t sk = (b * (size_t)c->tid_total + li.tid_prefix + c->role_idx[l * G.Hkv + h]) * std::max(G.C_max, 1);
           int64_t mine = 0;
           for (int j = 0; j < fixed_n[fh]; ++j) mine += -fixed_chunks[fh * G.FB + j] - 2;
           for (int j = 0; j < sq.S; ++j) {
             const int ch = slot_chunk[(b * G.L + l) * std::max(G.S_max, 1) + j];
-            if (ch >= 0) mine += len_of(sq, ch) - (ch == sq.C - 1 ? m.y : m.x);
+            if (ch >= 0) mine += len_of(sq, ch) - (m.x < 0 ? seg_kept[sk + ch] : ch == sq.C - 1 ? m.y : m.x);
           }
           r.resident_audio_tokens += mine;
           r.host_audio_tokens += sq.T_a - mine;

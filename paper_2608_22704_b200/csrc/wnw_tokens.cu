@@ -156,6 +156,15 @@ __global__ void __launch_bounds__(TOK_THREADS) wnw_token_select_kernel(const __g
   for (int s = threadIdx.x; s < G.FB; s += TOK_THREADS)   // block s of the compact store holds min(nc, n - s*nc) rows
     cv.fixed_chunks[fh * G.FB + s] = s < n_blk ? -(2 + min(G.nc, n - s * G.nc)) : -1;
   if (threadIdx.x == 0) { cv.fixed_n[fh] = n_blk; tok_n[fh] = n; }
+  const LayerInfo &li = cv.layers[layer];
+  if (f >= li.n_fixed) {   // a tidal head's base: how many positions of every segment it holds (what a fetched segment must skip)
+    int32_t *sk = cv.seg_kept + ((long long)b * cv.tid_total + li.tid_prefix + (f - li.n_fixed)) * G.C_max;
+    for (int c = threadIdx.x; c * G.nc < T_a; c += TOK_THREADS) {
+      int k = 0;
+      for (int t = c * G.nc; t < min(T_a, (c + 1) * G.nc); ++t) k += fl[t];
+      sk[c] = k;
+    }
+  }
 }
 
 // grid (FB, fixed heads of the layer); block 128.  Fills block blockIdx.x of the head's compact store.

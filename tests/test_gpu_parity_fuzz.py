@@ -83,7 +83,7 @@ def test_random_configuration_token_compression(seed):
     ret = (rs.rand(w.n_layers, w.n_kv_heads) * r_max).astype(np.float32)
     ret[rs.rand(w.n_layers, w.n_kv_heads) < 0.1] = 0.0
     seg = w.chunk if residency == 2 else int(rs.choice([w.chunk, 25, 7]))
-    variant = 0 if residency == 2 else int(rs.randint(0, 2))
+    variant = int(rs.randint(0, 2))
     ls = Lockstep(w, seed=seed, residency=residency, evict_lag=delta, score_scope=int(rs.randint(0, 2)), token_retention=ret,
                   token_seg=seg, token_variant=variant)
     try:

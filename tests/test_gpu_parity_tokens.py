@@ -150,15 +150,17 @@ def _lag_workload(audio=(640, 300, 77), chunk=25, head_dim=128, n_steps=10):
 RET_LAG = np.array([[1.0, 0.3, 0.45, 0.0], [0.5, 0.2, 0.08, 0.33], [1.0, 0.41, 0.25, 0.5]], np.float32)
 
 
-@pytest.mark.parametrize("scope", [0, 1])
-def test_token_base_tidal_heads_follow_the_oracle(scope):
+@pytest.mark.parametrize("scope,variant", [(0, 0), (1, 0), (0, 1)])
+def test_token_base_tidal_heads_follow_the_oracle(scope, variant):
     """Residency SEGMENT_LAG_TOKEN_BASE: every tidal head keeps its own per-segment best positions for good (retention
     0 to 0.5 per head), tables start empty, selected segments are fetched as complements (host mirror permuted) and
-    released after the lag; per-layer and global score scope; eager and replayed steps; slot bytes checked against the
+    released after the lag; per-layer and global score scope; per-segment quota and the global top-k variant (a base then
+    holds a different number of positions in every segment); eager and replayed steps; slot bytes checked against the
     permuted source rows."""
     from parity_harness import Lockstep
     w = _lag_workload()
-    ls = Lockstep(w, seed=31 + scope, score_scope=scope, residency=2, evict_lag=1, token_retention=RET_LAG, token_seg=25)
+    ls = Lockstep(w, seed=31 + scope, score_scope=scope, residency=2, evict_lag=1, token_retention=RET_LAG, token_seg=25,
+                  token_variant=variant)
     try:
         ls.prefill()
         for b in range(w.batch):
@@ -227,10 +229,9 @@ def test_token_base_placement_rules():
             wnw.wnw_place_prefill(h, 0, 0, k, v, p["audio_begin"], p["audio_end"], q)
         assert e.value.status == wnw.WNW_ERR_STATE
         args = (h, 0, 0, k, v, p["audio_begin"], p["audio_end"], q, RET_LAG[0])
-        for seg, variant in ((50, 0), (25, 1)):      # the quota's segment is the storage segment; no global variant
-            with pytest.raises(wnw.WnwError) as e:
-                wnw.wnw_place_prefill_tokens(*args, seg, variant)
-            assert e.value.status == wnw.WNW_ERR_UNSUPPORTED
+        with pytest.raises(wnw.WnwError) as e:       # the quota's segment is the storage segment
+            wnw.wnw_place_prefill_tokens(*args, 50, 0)
+        assert e.value.status == wnw.WNW_ERR_UNSUPPORTED
         wnw.wnw_place_prefill_tokens(*args, 25, 0)
         wnw.wnw_sync(h)
         assert len(wnw.wnw_get_fixed_tokens(h, 0, 0, 1)) == 25 * 7 + 4       # floor(.3*25)=7, tail floor(.3*15)=4

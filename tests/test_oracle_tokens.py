@@ -189,7 +189,8 @@ def _lag_workload():
     return w
 
 
-def test_token_base_tidal_heads_against_numpy():
+@pytest.mark.parametrize("variant", [0, 1])
+def test_token_base_tidal_heads_against_numpy(variant):
     """Residency 2: no segment is permanent as a whole; a tidal head sees [text | its kept positions | every position of the
     segments in its layer's dynamic slots].  Checked against numpy attention over exactly that key set, with the table
     advanced by the (separately pinned) lag update; retention 0 leaves a head with the fetched segments only, retention 1
@@ -207,9 +208,7 @@ def test_token_base_tidal_heads_against_numpy():
     for l in range(2):
         p = syn.prefill(0, l)
         kb, vb, qt = bf16_bits(p["k"]), bf16_bits(p["v"]), bf16_bits(p["q_text"])
-        with pytest.raises(wo.OracleError):                 # tidal bases keep a per-segment quota: no global variant
-            o.place_prefill_tokens(0, l, kb, vb, p["audio_begin"], p["audio_end"], qt, ret[l], seg, 1)
-        o.place_prefill_tokens(0, l, kb, vb, p["audio_begin"], p["audio_end"], qt, ret[l], seg, 0)
+        o.place_prefill_tokens(0, l, kb, vb, p["audio_begin"], p["audio_end"], qt, ret[l], seg, variant)
         pre[l] = (bf16_bits_to_f64(kb), bf16_bits_to_f64(vb), qt, p["audio_begin"], p["audio_end"])
     T_a, T_t, C, S = o.dims(0)
     assert (C, S, o.base_slots(0)) == (9, 2 * 2 * 2, 0)      # D = 2*topk*(delta+1) dynamic slots, no permanent ones
@@ -227,11 +226,13 @@ def test_token_base_tidal_heads_against_numpy():
                     _, prob = dense_attention(bf16_bits_to_f64(qt[qi, h * 2 + r]), K[:, h], V[:, h], scale)
                     want += prob[ab:ae]
             k32 = want.astype(np.float32).astype(np.float64)
-            exp = []
+            exp, m_tot = [], 0
             for lo in range(0, T_a, seg):
                 n = min(seg, T_a - lo)
-                m = int(math.floor(float(ret[l, h]) * n))
+                m = int(math.floor(float(ret[l, h]) * n)); m_tot += m
                 exp += sorted((lo + np.argsort(-k32[lo:lo + n], kind="stable")[:m]).tolist())
+            if variant == 1:                      # the same budget spent on the best positions of the whole head
+                exp = sorted(np.argsort(-k32, kind="stable")[:m_tot].tolist())
             kept[(l, h)] = o.fixed_tokens(0, l, h)
             assert kept[(l, h)].tolist() == exp
     assert len(kept[(1, 0)]) == 0 and len(kept[(1, 1)]) == T_a
