@@ -687,13 +687,24 @@ __global__ void __maxnreg__(NW == 8 ? 208 : 255) wnw_attn_multi_kernel(const __g
                                                                  const __grid_constant__ TmaMaps maps) {
   int l = 0;
   while (l + 1 < m.n && (int)blockIdx.x >= m.cta_prefix[l + 1]) ++l;
-  attn_body<D, G16, NW, TB>(cv, m.l[l], nullptr, maps, (int)blockIdx.x - m.cta_prefix[l]);
+  attn_body<D, G16, NW, TB>(cv, m.l[l], nullptr, maps, (int)blockIdx.x - m.cta_prefix[l] + m.cta_first[l]);
 }
 
 template <int D, bool G16, int NW, bool TB>
-static cudaError_t launch_multi_tb(const CacheView &cv, const MultiArgs &m, size_t smem, const TmaMaps &maps, cudaStream_t st) {
-  wnw_attn_multi_kernel<D, G16, NW, TB><<<m.cta_prefix[m.n], NW * 32, smem, st>>>(cv, m, maps);
-  return cudaGetLastError();
+static cudaError_t launch_multi_tb(const CacheView &cv, const MultiArgs &m, size_t smem, const TmaMaps &maps, bool pdl,
+                                   cudaStream_t st) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)m.cta_prefix[m.n], 1, 1);
+  cfg.blockDim = dim3(NW * 32, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  if (pdl) {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, wnw_attn_multi_kernel<D, G16, NW, TB>, cv, m, maps);
 }
 
 template <int D, bool G16, int NW, bool TB>
@@ -786,8 +797,8 @@ cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st)
 }
 
 // One launch for the CTAs of n layers (all cut for the one-shot 8-warp variant).
-cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, cudaStream_t st) {
-  if (n <= 0 || n > MULTI_LAYERS_MAX) return cudaErrorInvalidValue;
+cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, const int *n_first, int part, cudaStream_t st) {
+  if (n <= 0 || n > MULTI_LAYERS_MAX || (part >= 0 && !n_first)) return cudaErrorInvalidValue;
   MultiArgs m;
   memset(&m, 0, sizeof(m));
   size_t smem = 0;
@@ -797,24 +808,29 @@ cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, 
     const AttnArgs &a = args[i];
     if (a.n_items <= 0) continue;
     if (a.throughput || !a.maps || a.maps != args[0].maps) return cudaErrorInvalidValue;
+    const int all = a.cta_ranges ? a.n_ctas : a.n_items;
+    const int first = part == 1 ? n_first[i] : 0, count = part == 0 ? n_first[i] : all - first;
+    if (first < 0 || count < 0 || first + count > all) return cudaErrorInvalidValue;
+    if (count == 0) continue;
     m.cta_prefix[n_used] = ctas;
+    m.cta_first[n_used] = first;
     m.l[n_used] = a;
     m.l[n_used].pdl = 0; m.l[n_used].wait_inputs = 0;
     ++n_used;
-    ctas += a.cta_ranges ? a.n_ctas : a.n_items;
+    ctas += count;
     smem = std::max(smem, (size_t)NW_LAT * NSTAGE * 2 * GR * d * 2 + 1024 + (a.xpref ? attn_scratch_bytes(NW_LAT, cv.geo.g, d) : 0));
   }
   if (n_used == 0) return cudaSuccess;
   m.n = n_used; m.cta_prefix[n_used] = ctas;
-  const bool g16 = cv.geo.g > 8, tb = cv.geo.token_base != 0;
+  const bool g16 = cv.geo.g > 8, tb = cv.geo.token_base != 0, pdl = part == 1;
   const TmaMaps &maps = *args[0].maps;
   if (d == 128) {
-    if (g16) return tb ? launch_multi_tb<128, true, NW_LAT, true>(cv, m, smem, maps, st) : launch_multi_tb<128, true, NW_LAT, false>(cv, m, smem, maps, st);
-    return tb ? launch_multi_tb<128, false, NW_LAT, true>(cv, m, smem, maps, st) : launch_multi_tb<128, false, NW_LAT, false>(cv, m, smem, maps, st);
+    if (g16) return tb ? launch_multi_tb<128, true, NW_LAT, true>(cv, m, smem, maps, pdl, st) : launch_multi_tb<128, true, NW_LAT, false>(cv, m, smem, maps, pdl, st);
+    return tb ? launch_multi_tb<128, false, NW_LAT, true>(cv, m, smem, maps, pdl, st) : launch_multi_tb<128, false, NW_LAT, false>(cv, m, smem, maps, pdl, st);
   }
   if (d == 64) {
-    if (g16) return tb ? launch_multi_tb<64, true, NW_LAT, true>(cv, m, smem, maps, st) : launch_multi_tb<64, true, NW_LAT, false>(cv, m, smem, maps, st);
-    return tb ? launch_multi_tb<64, false, NW_LAT, true>(cv, m, smem, maps, st) : launch_multi_tb<64, false, NW_LAT, false>(cv, m, smem, maps, st);
+    if (g16) return tb ? launch_multi_tb<64, true, NW_LAT, true>(cv, m, smem, maps, pdl, st) : launch_multi_tb<64, true, NW_LAT, false>(cv, m, smem, maps, pdl, st);
+    return tb ? launch_multi_tb<64, false, NW_LAT, true>(cv, m, smem, maps, pdl, st) : launch_multi_tb<64, false, NW_LAT, false>(cv, m, smem, maps, pdl, st);
   }
   return cudaErrorInvalidValue;
 }

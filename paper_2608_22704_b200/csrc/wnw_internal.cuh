@@ -173,6 +173,7 @@ constexpr int MULTI_LAYERS_MAX = 48;
 struct MultiArgs {
   int32_t n;
   int32_t cta_prefix[MULTI_LAYERS_MAX + 1];
+  int32_t cta_first[MULTI_LAYERS_MAX];   // the layer's first CTA in this launch (a launch may carry a part of its CTAs)
   AttnArgs l[MULTI_LAYERS_MAX];
 };
 
@@ -234,7 +235,9 @@ cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_c
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
 cudaError_t configure_attn_kernels();
 // the CTAs of several layers' launches (one-shot variant) in one launch
-cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, cudaStream_t st);
+// part < 0: all CTAs of every layer; part 0: the first n_first[l] CTAs of layer l; part 1: the rest, launched
+// programmatically dependent on what precedes it in the stream
+cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, const int *n_first, int part, cudaStream_t st);
 // Encodes the descriptor of one store: base (device), rows, head_dim.  Returns false if the driver refuses.
 bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d);
 cudaError_t configure_select_kernel();

@@ -295,8 +295,11 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
 cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,
                           int skip_copy, RecallSignal sig, cudaStream_t st) {
   if (n_layers <= 0 || n_active <= 0) return cudaSuccess;
-  const int groups = n_layers < RECALL_GROUPS ? n_layers : RECALL_GROUPS;   // few layers: all CTAs on each block
-  wnw_recall_kernel<<<RECALL_CTAS / groups * groups, 256, 0, st>>>(cv, n_active, active, layers_dev, n_layers, groups, skip_copy, sig);
+  int n_groups = RECALL_GROUPS, n_ctas = RECALL_CTAS;
+  if (const char *e = getenv("WNW_RECALL_GROUPS")) n_groups = std::max(1, atoi(e));
+  if (const char *e = getenv("WNW_RECALL_CTAS")) n_ctas = std::max(n_groups, atoi(e));
+  const int groups = n_layers < n_groups ? n_layers : n_groups;   // few layers: all CTAs on each block
+  wnw_recall_kernel<<<n_ctas / groups * groups, 256, 0, st>>>(cv, n_active, active, layers_dev, n_layers, groups, skip_copy, sig);
   return cudaGetLastError();
 }
 

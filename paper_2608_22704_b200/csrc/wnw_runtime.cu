@@ -30,6 +30,7 @@ struct LayerWork {
   bool throughput = false;                         // which kernel variant the items were cut for
   size_t part_off = 0;                             // first partial of this layer in the partial buffers (in items)
   int n_ctas = 0, order_off = 0, ranges_off = 0;   // items per CTA (persistent schedule, or packed short heads): offsets
+  int n_ctas_free = 0;   // BATCHED layers: the first n_ctas_free CTAs hold no tidal head (they need no recall epoch)
   bool packed = false;                             // one-shot CTAs that serve several short heads each
   int head_items_off = 0;                          // offset in the uploaded HeadItems array
 };
@@ -116,8 +117,9 @@ struct wnw_cache {
   void count_launch(int kind, int n, bool capturing) { (capturing ? cap_launches : launches)[kind] += n; }
   int layer_dependency = WNW_LAYERS_INDEPENDENT;
   std::vector<AttnArgs> batch_args;   // BATCHED layers of a captured step: recorded per layer, launched by the last one
-  bool cap_batched = false;
-  int batched_target = 0;             // granules of work per CTA when the step's layers share one launch
+  bool cap_batched = false, batched_two_part = true;
+  int batched_target = 0;             // granules of work per CTA when the step's layers share one launch ...
+  int batched_target_tidal = 0;       // ... and per CTA of its second part, the tidal heads
   // replayed steps: one recall launch per step outside the captured graph, overlapping the next step
   int32_t *d_recall_epoch = nullptr, *d_recall_ctr = nullptr, *d_step_epoch = nullptr;
   int external_recall_mode = -1;   // -1 automatic, 0 never, 1 always
@@ -286,6 +288,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
 #define CKE(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { return fail(_e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA); } } while (0)
   cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
   if (const char *e = getenv("WNW_PDL")) c->pdl_enabled = atoi(e) != 0;
+  if (const char *e = getenv("WNW_BATCH_TWO_PART")) c->batched_two_part = atoi(e) != 0;
   if (const char *e = getenv("WNW_PACK")) { c->pack_granules = atoi(e); c->pack_enabled = c->pack_granules != 0; if (c->pack_granules < 0) c->pack_granules = 0; }
   if (const char *e = getenv("WNW_FOLD_STEP_END")) c->fold_enabled = atoi(e) != 0;
   if (const char *e = getenv("WNW_SELECT_ALL")) c->select_all_enabled = atoi(e) != 0;
@@ -615,7 +618,11 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
       // a short head stays in one CTA: up to 128 granules when layers overlap (work per launch counts), 32 when the
       // kernel's span counts (measured, chained config 1: 298 -> 240 us per step against a threshold of 64)
       if (!throughput && nw_ <= (overlapped ? 2 * c->direct_max_granules : c->direct_max_granules / 2)) n_cta = 1;
-      if (batched) n_cta = nw_ <= gpi * 3 / 2 ? 1 : (nw_ + gpi - 1) / gpi;
+      if (batched) {   // long heads in pieces as fat as a CTA of their part of the launch
+        const int nwp = attn_warps(false);
+        const int tg = role == ROLE_TIDAL ? (c->batched_target_tidal + nwp - 1) / nwp * nwp : gpi;
+        n_cta = nw_ <= tg * 3 / 2 ? 1 : (nw_ + tg - 1) / tg;
+      }
       HeadItems hi{(int)items.size() - lw.first_item, n_cta};
       for (int x = 0; x < n_cta; ++x) {  // even contiguous ranges
         const int g0 = (int)((long long)n * x / n_cta), g1 = (int)((long long)n * (x + 1) / n_cta);
@@ -643,21 +650,28 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
     int pos = 0, in_pack = 0, pack_work = 0, n_packs = 0;
     bool any = false;
     auto close_pack = [&]() { if (in_pack > 0) { ++n_packs; in_pack = 0; pack_work = 0; } };
-    for (size_t hd = (size_t)lw.head_items_off; hd < heads.size(); ++hd) {
-      const HeadItems &hi = heads[hd];
-      if (hi.count > 1) {   // a split head: every piece alone
-        close_pack();
-        for (int x = 0; x < hi.count; ++x) { ranges.push_back(pos); order.push_back(hi.first + x); ++pos; ++n_packs; }
-        continue;
+    // BATCHED layers: the heads that read no slot come first and never share a CTA with a tidal head: the launch goes
+    // out in two parts, the tidal part (cut finer) behind the other
+    for (int pass = 0; pass < (batched ? 2 : 1); ++pass) {
+      const int tgt = batched && pass == 1 ? c->batched_target_tidal : target;
+      for (size_t hd = (size_t)lw.head_items_off; hd < heads.size(); ++hd) {
+        const HeadItems &hi = heads[hd];
+        const WorkItem &wi = items[lw.first_item + hi.first];
+        if (batched && (wi.role == ROLE_TIDAL) != (pass == 1)) continue;
+        if (hi.count > 1) {   // a split head: every piece alone
+          close_pack();
+          for (int x = 0; x < hi.count; ++x) { ranges.push_back(pos); order.push_back(hi.first + x); ++pos; ++n_packs; }
+          continue;
+        }
+        const int work = n_work[(size_t)wi.i * G.Hkv + wi.h];
+        if (in_pack > 0 && pack_work + work > tgt) close_pack();
+        if (in_pack == 0) ranges.push_back(pos);
+        else any = true;
+        order.push_back(hi.first); ++pos; ++in_pack; pack_work += work;
       }
-      const WorkItem &wi = items[lw.first_item + hi.first];
-      const int work = n_work[(size_t)wi.i * G.Hkv + wi.h];
-      if (in_pack > 0 && pack_work + work > target) close_pack();
-      if (in_pack == 0) ranges.push_back(pos);
-      else any = true;
-      order.push_back(hi.first); ++pos; ++in_pack; pack_work += work;
+      close_pack();
+      if (pass == 0) lw.n_ctas_free = batched ? n_packs : 0;
     }
-    close_pack();
     ranges.push_back(pos);
     if (any || batched) { lw.n_ctas = n_packs; lw.packed = true; }
     else { order.resize(lw.order_off); ranges.resize(lw.ranges_off); }
@@ -703,19 +717,43 @@ static wnw_status_t ensure_worklists(wnw_cache *c) {
   c->wl_layers.assign(G.L, LayerWork{});
   c->batched_target = 0;
   if (c->layer_dependency == WNW_LAYERS_BATCHED) {   // the step's whole work over one wave of CTAs
-    long long total = 0;
+    long long total = 0, total_tidal = 0;
     for (int l = 0; l < G.L; ++l)
       for (int b : c->active)
         for (int h = 0; h < G.Hkv; ++h) {
           int n = 0, work = 0;
           head_granules(c, l, mode, c->seqs[b], h, &n, &work);
-          total += work;
+          if (mode == ATTN_DECODE && c->roles[l * G.Hkv + h] == ROLE_TIDAL) total_tidal += work;
+          else total += work;
         }
     // 1.4 x the mean share of an SM: heads are packed whole, so CTAs come out uneven; with this margin the launch stays
     // within one wave (measured, config 1: 57 us per step at 1.2 to 1.7 x the mean, 61 to 65 us at 0.9 and 1.0 x, where
     // a second, nearly empty wave forms, 66 us at 2 x, where too few SMs pull)
+    // Tidal heads form a second part of the launch (its CTAs follow those of the first as SMs come free), each cut the same way.
     c->batched_target = (int)std::max<long long>(32, (total * 14 / 10 + c->n_sm - 1) / c->n_sm);
+    c->batched_target_tidal = (int)std::max<long long>(32, (total_tidal * 14 / 10 + c->n_sm - 1) / c->n_sm);
     if (const char *e = getenv("WNW_BATCH_TARGET")) c->batched_target = std::max(8, atoi(e));
+    if (const char *e = getenv("WNW_BATCH_TARGET_TIDAL")) c->batched_target_tidal = std::max(8, atoi(e));
+    // Where a single layer already fills the machine with CTAs of a decent size its launches stay apart (their steps
+    // keep selection and recall inside the step, so nothing would be issued together anyway): the cut of INDEPENDENT.
+    if ((total + total_tidal) / G.L > 64ll * c->n_sm) c->batched_target = c->batched_target_tidal = 0;
+    if (getenv("WNW_DEBUG_CUT")) fprintf(stderr, "batched cut: work %lld + tidal %lld granules, targets %d / %d\n", total, total_tidal, c->batched_target, c->batched_target_tidal);
+  }
+  if (c->batched_target > 0 && !getenv("WNW_BATCH_TARGET")) {
+    // Whole heads and pieces come out uneven: widen the cut until the first part of the launch (the CTAs that read no slot)
+    // is at most one wave; a few CTAs beyond it would each add a CTA's whole duration to the step (config 2: 152 CTAs of 184
+    // granules 103 us per step, 136 CTAs of 192 granules 75 us).
+    for (int attempt = 0; attempt < 12; ++attempt) {
+      std::vector<WorkItem> it_t; std::vector<HeadItems> hd_t; std::vector<int32_t> or_t, ra_t;
+      int first_part = 0;
+      for (int l = 0; l < G.L; ++l) {
+        LayerWork lw_t;
+        build_layer_items(c, l, mode, c->active, it_t, hd_t, lw_t, or_t, ra_t);
+        first_part += lw_t.packed ? lw_t.n_ctas_free : (lw_t.n_ctas > 0 ? lw_t.n_ctas : lw_t.n_items);
+      }
+      if (first_part <= c->n_sm) break;
+      c->batched_target = c->batched_target * 11 / 10 + 1;
+    }
   }
   size_t part_total = 0;
   for (int l = 0; l < G.L; ++l) {
@@ -1126,6 +1164,12 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     c->cap_batched = c->layer_dependency == WNW_LAYERS_BATCHED && capturing && c->graph_capturing && one_shot &&
                      (!tiered || c->cap_select_all);
     if (c->cap_batched) c->batch_args.assign(G.L, AttnArgs{});
+    if (getenv("WNW_DEBUG_CUT") && capturing) {
+      int mx = 0, tot = 0;
+      for (const LayerWork &w : c->wl_layers) { const int n = w.n_ctas > 0 ? w.n_ctas : w.n_items; mx = std::max(mx, n); tot += n; }
+      fprintf(stderr, "capture: batched %d small %d select_all %d external_recall %d one_shot %d; CTAs per layer max %d, total %d\n",
+              (int)c->cap_batched, (int)small, (int)c->cap_select_all, (int)c->cap_external_recall, (int)one_shot, mx, tot);
+    }
   }
   if (!capturing) {
     if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
@@ -1178,8 +1222,25 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   if (c->cap_batched) {
     c->batch_args[layer] = a;
     if (layer == G.L - 1) {
-      CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, st));
-      c->count_launch(0, 1, capturing);
+      // Two parts when the step has tidal heads: first the CTAs that read no slot, one wave of them; then, programmatically
+      // dependent, those of the tidal heads, which take the SMs as the first part leaves them.  The recall of the previous
+      // step (it runs outside the captured graph, beside this step) has landed by then, so no CTA sits on an SM waiting.
+      std::vector<int> n_free(G.L, 0);
+      bool any_free = false, any_tidal = false;
+      for (int l = 0; l < G.L; ++l) {
+        const LayerWork &w = c->wl_layers[l];
+        n_free[l] = w.packed ? w.n_ctas_free : 0;
+        any_free = any_free || n_free[l] > 0;
+        any_tidal = any_tidal || n_free[l] < (w.n_ctas > 0 ? w.n_ctas : w.n_items);
+      }
+      if (tiered && any_free && any_tidal && c->batched_two_part) {
+        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_free.data(), 0, st));
+        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_free.data(), 1, st));
+        c->count_launch(0, 2, capturing);
+      } else {
+        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, nullptr, -1, st));
+        c->count_launch(0, 1, capturing);
+      }
     }
   } else {
     CK(launch_attn(c->cv, a, st));
