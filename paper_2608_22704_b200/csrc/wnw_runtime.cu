@@ -737,7 +737,6 @@ static wnw_status_t ensure_worklists(wnw_cache *c) {
     // Where a single layer already fills the machine with CTAs of a decent size its launches stay apart (their steps
     // keep selection and recall inside the step, so nothing would be issued together anyway): the cut of INDEPENDENT.
     if ((total + total_tidal) / G.L > 64ll * c->n_sm) c->batched_target = c->batched_target_tidal = 0;
-    if (getenv("WNW_DEBUG_CUT")) fprintf(stderr, "batched cut: work %lld + tidal %lld granules, targets %d / %d\n", total, total_tidal, c->batched_target, c->batched_target_tidal);
   }
   if (c->batched_target > 0 && !getenv("WNW_BATCH_TARGET")) {
     // Whole heads and pieces come out uneven: widen the cut until the first part of the launch (the CTAs that read no slot)
@@ -1164,12 +1163,6 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     c->cap_batched = c->layer_dependency == WNW_LAYERS_BATCHED && capturing && c->graph_capturing && one_shot &&
                      (!tiered || c->cap_select_all);
     if (c->cap_batched) c->batch_args.assign(G.L, AttnArgs{});
-    if (getenv("WNW_DEBUG_CUT") && capturing) {
-      int mx = 0, tot = 0;
-      for (const LayerWork &w : c->wl_layers) { const int n = w.n_ctas > 0 ? w.n_ctas : w.n_items; mx = std::max(mx, n); tot += n; }
-      fprintf(stderr, "capture: batched %d small %d select_all %d external_recall %d one_shot %d; CTAs per layer max %d, total %d\n",
-              (int)c->cap_batched, (int)small, (int)c->cap_select_all, (int)c->cap_external_recall, (int)one_shot, mx, tot);
-    }
   }
   if (!capturing) {
     if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
