@@ -217,6 +217,12 @@ cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st)
 cudaError_t launch_select(const CacheView &cv, const SelectArgs &a, size_t smem_bytes, int groups, cudaStream_t st);
 cudaError_t launch_select_all(const CacheView &cv, const SelectArgs *layer_args_dev, const int4 *map_dev, int n_entries,
                               const SelectArgs &step, size_t smem_bytes, cudaStream_t st);
+// the same with the layers' arguments and the map in the kernel parameters (no global load before the CTA knows its
+// work); n_layers <= SELECT_TABLE_LAYERS and n_entries <= SELECT_TABLE_ENTRIES
+constexpr int SELECT_TABLE_LAYERS = 48, SELECT_TABLE_ENTRIES = 64;
+struct SelectAllTable { int4 map[SELECT_TABLE_ENTRIES]; SelectArgs l[SELECT_TABLE_LAYERS]; };
+cudaError_t launch_select_all_params(const CacheView &cv, const SelectArgs *layer_args_host, int n_layers, const int4 *map_host,
+                                     int n_entries, const SelectArgs &step, size_t smem_bytes, cudaStream_t st);
 cudaError_t launch_step_end(const CacheView &cv, int n_active, const int32_t *active, int appended, int32_t *bump_epoch,
                             cudaStream_t st);
 cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *active, const int32_t *layers_dev, int n_layers,

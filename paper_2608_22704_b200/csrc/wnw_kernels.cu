@@ -10,6 +10,30 @@ namespace wnw {
 // ------------------------------------------------------------------------------------------------
 constexpr int SEL_WARPS = 8;
 // One CTA: sequence i of the active list, group `grp` of `n_grp` over the layer's update list.
+#ifdef WNW_PHASE_STAMPS   // latency studies only (never in the product build): first start and last end of the launch, ns
+__device__ unsigned long long g_sel_time[2] = {~0ull, 0ull};
+extern "C" int wnw_debug_read_select_time(unsigned long long *host, int reset) {
+  int rc = (int)cudaMemcpyFromSymbol(host, g_sel_time, sizeof(g_sel_time));
+  if (reset) { const unsigned long long init[2] = {~0ull, 0ull}; rc |= (int)cudaMemcpyToSymbol(g_sel_time, init, sizeof(init)); }
+  return rc;
+}
+__device__ __forceinline__ unsigned long long sel_gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+__device__ unsigned long long g_sel_phase[8];   // per phase: max over CTAs of the time since the CTA's start, ns
+extern "C" int wnw_debug_read_select_phases(unsigned long long *host, int reset) {
+  int rc = (int)cudaMemcpyFromSymbol(host, g_sel_phase, sizeof(g_sel_phase));
+  if (reset) { const unsigned long long z[8] = {0}; rc |= (int)cudaMemcpyToSymbol(g_sel_phase, z, sizeof(z)); }
+  return rc;
+}
+#define SEL_PHASE(k) do { if (threadIdx.x == 0) atomicMax(&g_sel_phase[k], sel_gtime() - sel_t0); } while (0)
+#define SEL_PHASE_T0() const unsigned long long sel_t0 = sel_gtime()
+#define SEL_STAMP_START() do { if (threadIdx.x == 0) atomicMin(&g_sel_time[0], sel_gtime()); } while (0)
+#define SEL_STAMP_END() do { __syncthreads(); if (threadIdx.x == 0) atomicMax(&g_sel_time[1], sel_gtime()); } while (0)
+#else
+#define SEL_PHASE(k) do { } while (0)
+#define SEL_PHASE_T0() do { } while (0)
+#define SEL_STAMP_START() do { } while (0)
+#define SEL_STAMP_END() do { } while (0)
+#endif
 __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArgs &a, int smem_total, unsigned char *smem,
                                             int i, int grp, int n_grp) {
   const Geometry &G = cv.geo;
@@ -17,8 +41,11 @@ __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArg
   const int b = a.active[i];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const LayerInfo &li = a.li;
+  SEL_PHASE_T0();
   // per-sequence scalars: one batch of independent loads
   const int C_b = cv.C[b], S_b = cv.S[b], T_a = cv.T_a[b];
+  const int epoch_now = a.step_epoch ? *a.step_epoch : 0;   // read here, not on the way out (the step's own bump comes
+                                                            // after every selection CTA has finished)
   const long long step_b = cv.step_snap[(long long)b * G.L + a.layer];   // not cv.steps: an eager step's bookkeeping kernel
                                                                          // follows the attention kernel, not this one
   const int n_aq = a.n_aq;
@@ -89,8 +116,10 @@ __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArg
     upd_of(u_first, lt, src);
     select_stage(cv, b, lt, src, scored && src == a.layer, C_b, S_b, lane, select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b));
   }
+  SEL_PHASE(0);
   cp_async_commit_wait_all();
   __syncthreads();
+  SEL_PHASE(1);
   if (scored) {
     // score_sum[c] = sum over anchor q-heads (head order) of (sum over the chunk's granules of e * 2^(m - M)) / Z
     float *dst = cv.score_sum + ((long long)b * G.L + a.layer) * G.C_max;
@@ -117,6 +146,7 @@ __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArg
       __syncthreads();
     }
   }
+  SEL_PHASE(2);
   if (cv.scope_global && n_upd > 0) {
     // Eq. 2 as printed: one accumulator over all anchor layers of the step, added in layer order
     for (int c = threadIdx.x; c < C_b; c += NT) {
@@ -145,17 +175,20 @@ __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArg
       const int n_copies = G.lag_mode ? select_and_update_lag(cv, b, lt, src, C_b, S_b, cv.S_base[b], T_a, step_b, lane, rank_by, w)
                                       : select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, rank_by, w);
       if (a.epoch_words && n_copies == 0 && lane == 0) {
-        const int prev = atomicAdd(a.empty_ctr + lt, 1);
-        if (prev == a.n_active - 1) {   // nothing to recall for this layer in this step: its slots are current
-          a.empty_ctr[lt] = 0;
+        // one sequence: nobody to count; else the sequence whose plan comes in last publishes
+        const bool last = a.n_active == 1 || atomicAdd(a.empty_ctr + lt, 1) == a.n_active - 1;
+        if (last) {   // nothing to recall for this layer in this step: its slots are current
+          if (a.n_active > 1) a.empty_ctr[lt] = 0;
           __threadfence();
-          const int epoch = *a.step_epoch + 1;   // the step's own bump comes after every selection CTA has finished
-          asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(a.epoch_words + lt), "r"(epoch) : "memory");
+          asm volatile("st.release.gpu.global.s32 [%0], %1;\n" ::"l"(a.epoch_words + lt), "r"(epoch_now + 1) : "memory");
         }
       }
     }
   }
+  __syncthreads();
+  SEL_PHASE(3);
   close_step();
+  SEL_PHASE(4);
 }
 
 __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_kernel(const __grid_constant__ CacheView cv,
@@ -174,6 +207,7 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_all_kernel(const __
                                                                         const __grid_constant__ SelectArgs step, int smem_total) {
   extern __shared__ __align__(16) unsigned char smem[];
   __shared__ SelectArgs a_s;
+  SEL_STAMP_START();
   const int4 m = map[blockIdx.y];
   {
     const int *src = reinterpret_cast<const int *>(layer_args + m.x);
@@ -190,10 +224,51 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_all_kernel(const __
   }
   __syncthreads();
   select_body(cv, a_s, smem_total, smem, blockIdx.x, m.y, m.z);
+  SEL_STAMP_END();
+}
+
+__global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_all_p_kernel(const __grid_constant__ CacheView cv,
+                                                                          const __grid_constant__ SelectAllTable t,
+                                                                          const __grid_constant__ SelectArgs step, int smem_total) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  __shared__ SelectArgs a_s;
+  SEL_STAMP_START();
+  const int4 m = t.map[blockIdx.y];
+  {
+    const int *src = reinterpret_cast<const int *>(&t.l[m.x]);
+    int *dst = reinterpret_cast<int *>(&a_s);
+    for (int x = threadIdx.x; x < (int)(sizeof(SelectArgs) / sizeof(int)); x += blockDim.x) dst[x] = src[x];
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    a_s.n_active = step.n_active; a_s.active = step.active;
+    a_s.do_score = step.do_score; a_s.do_update = step.do_update;
+    a_s.fold_total = step.fold_total; a_s.fold_appended = step.fold_appended;
+    a_s.fold_counter = step.fold_counter; a_s.fold_bump_epoch = step.fold_bump_epoch;
+    a_s.epoch_words = step.epoch_words; a_s.empty_ctr = step.empty_ctr; a_s.step_epoch = step.step_epoch;
+  }
+  __syncthreads();
+  select_body(cv, a_s, smem_total, smem, blockIdx.x, m.y, m.z);
+  SEL_STAMP_END();
+}
+
+cudaError_t launch_select_all_params(const CacheView &cv, const SelectArgs *layer_args_host, int n_layers, const int4 *map_host,
+                                     int n_entries, const SelectArgs &step, size_t smem_bytes, cudaStream_t st) {
+  if (n_entries <= 0 || step.n_active <= 0) return cudaSuccess;
+  if (n_layers > SELECT_TABLE_LAYERS || n_entries > SELECT_TABLE_ENTRIES) return cudaErrorInvalidValue;
+  static_assert(sizeof(SelectAllTable) + sizeof(CacheView) + sizeof(SelectArgs) < 30000, "kernel parameter space");
+  SelectAllTable t;
+  memset(&t, 0, sizeof(t));
+  memcpy(t.map, map_host, sizeof(int4) * n_entries);
+  memcpy(t.l, layer_args_host, sizeof(SelectArgs) * n_layers);
+  wnw_select_all_p_kernel<<<dim3(step.n_active, n_entries), SEL_WARPS * 32, smem_bytes, st>>>(cv, t, step, (int)smem_bytes);
+  return cudaGetLastError();
 }
 
 cudaError_t configure_select_kernel() {
   cudaError_t e = cudaFuncSetAttribute(wnw_select_all_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM_CAP);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(wnw_select_all_p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM_CAP);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(wnw_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM_CAP);
 }

@@ -107,6 +107,8 @@ struct wnw_cache {
   bool select_all_enabled = true, cap_select_all = false, select_single_ok = false;
   SelectArgs *d_sel_args = nullptr;
   int4 *d_sel_map = nullptr;
+  std::vector<SelectArgs> h_sel_args;   // host copies: small stacks pass them in the kernel parameters
+  std::vector<int4> h_sel_map;
   int sel_map_single[2] = {0, 0}, sel_map_score[2] = {0, 0}, sel_map_update[2] = {0, 0};   // offset, entries
   size_t sel_all_smem = 0;
   bool fold_enabled = true, cap_fold = false;   // captured steps: the last selection CTA closes the step
@@ -497,6 +499,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     c->sel_map_score[1] = (int)sel_map.size() - c->sel_map_score[0];
     CKC(dev_upload(c, &c->d_sel_args, sel_args));
     CKC(dev_upload(c, &c->d_sel_map, sel_map));
+    c->h_sel_args = sel_args; c->h_sel_map = sel_map;
   }
   for (int l = 0; l < L; ++l)
     if (!full && (c->layers[l].n_anchor > 0 || c->layers[l].upd_count > 0)) {
@@ -1067,6 +1070,15 @@ extern "C" wnw_status_t wnw_get_fixed_tokens(wnw_cache_t *c, int32_t seq, int32_
   return WNW_OK;
 }
 
+// One selection launch for the map entries [range[0], range[0] + range[1]); small stacks carry the layers' arguments in
+// the kernel parameters.
+static cudaError_t select_all(wnw_cache *c, const int *range, const SelectArgs &stp, cudaStream_t st) {
+  if (c->geo.L <= SELECT_TABLE_LAYERS && range[1] <= SELECT_TABLE_ENTRIES && !c->h_sel_args.empty())
+    return launch_select_all_params(c->cv, c->h_sel_args.data(), c->geo.L, c->h_sel_map.data() + range[0], range[1], stp,
+                                    c->sel_all_smem, st);
+  return launch_select_all(c->cv, c->d_sel_args, c->d_sel_map + range[0], range[1], stp, c->sel_all_smem, st);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Decode step
 // ---------------------------------------------------------------------------------------------
@@ -1320,14 +1332,14 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
     stp.epoch_words = c->d_recall_epoch; stp.empty_ctr = c->d_empty_ctr; stp.step_epoch = c->d_step_epoch;
     if (!c->select_single_ok) {   // first every anchor layer's scores, then every table update
       stp.do_score = 1; stp.do_update = 0;
-      CK(launch_select_all(c->cv, c->d_sel_args, c->d_sel_map + c->sel_map_score[0], c->sel_map_score[1], stp, c->sel_all_smem, st));
+      CK(select_all(c, c->sel_map_score, stp, st));
       if (c->sel_map_score[1] > 0) c->count_launch(1, 1, true);
     }
     const int *range = c->select_single_ok ? c->sel_map_single : c->sel_map_update;
     stp.do_score = c->select_single_ok ? 1 : 0; stp.do_update = 1;
     stp.fold_total = range[1] * stp.n_active; stp.fold_appended = c->appended == 1;
     stp.fold_counter = c->d_fold_ctr; stp.fold_bump_epoch = c->d_step_epoch;
-    CK(launch_select_all(c->cv, c->d_sel_args, c->d_sel_map + range[0], range[1], stp, c->sel_all_smem, st));
+    CK(select_all(c, range, stp, st));
     c->count_launch(1, 1, true);
   }
   if (!(capturing && c->cap_fold)) {
