@@ -127,7 +127,7 @@ struct GranDesc {
 // the row of every granule is static; what may be unknown yet is how many of its 16 rows are visible.
 template <bool TB>
 __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const AttnArgs &a, const LayerInfo &li,
-                                                   const WorkItem &it, int j) {
+                                                   const WorkItem &it, int j, int table_parity) {
   const Geometry &G = cv.geo;
   GranDesc r;
   r.cid = -1; r.off = 0; r.score_idx = -1;
@@ -156,7 +156,7 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
   } else if (it.role == ROLE_TIDAL) {
     const int slot = TB ? ci - it.S : ci;
     r.row = (int)(pool_off(G, li, it.b, slot, it.ridx, 0) / G.d) + off;
-    r.cid = cv.slot_chunk[((long long)it.b * G.L + a.layer) * G.S_max + slot];
+    r.cid = cv.slot_chunk[slot_table_off(G, table_parity, (long long)it.b * G.L + a.layer) + slot];
     // beyond the permanent slots a slot may be empty: its rows are fetched only if it is not
     r.meta = (TB || ci >= it.S) ? -3 : -2;
   } else {
@@ -231,6 +231,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   struct Ctx {
     WorkItem it;
     int item_idx, T_t, v_delta_audio, first, n_my;
+    int table_parity;     // which copy of the slot table this step reads (tidal items)
     int m_full, m_tail;   // token-granular base: positions of a full / of the last segment that live in the base already
     const int32_t *seg_kept;   // ... or, where they differ by segment (m_full < 0), the head's per-segment counts
     const CUtensorMap *map_audio;
@@ -264,6 +265,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     else if (c.it.role == ROLE_TIDAL) { c.v_delta_audio = G.ncp; c.map_audio = &maps.pool; }          // granule's K and
     else { c.v_delta_audio = G.FB * G.ncp; c.map_audio = &maps.fixed; }                            // V rows
     c.m_full = c.m_tail = 0;
+    c.table_parity = (c.it.role == ROLE_TIDAL && cv.steps) ? (int)(cv.steps[c.it.b] & 1) : 0;
     if (TB && c.it.role == ROLE_TIDAL) {
       const int2 m = cv.tok_m[((long long)c.it.b * G.L + a.layer) * G.Hkv + c.it.h];
       c.m_full = m.x; c.m_tail = m.y;
@@ -307,7 +309,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   auto issue_copy = [&](const Ctx &c, int n, uint32_t seq) -> bool {
     if ((n & 31) == 0) {
       const int nn = n + lane;
-      if (nn < c.n_my) blk = decode_granule<TB>(cv, a, li, c.it, c.first + nn * NW);
+      if (nn < c.n_my) blk = decode_granule<TB>(cv, a, li, c.it, c.first + nn * NW, c.table_parity);
       else { blk.meta = 0; blk.cid = -1; blk.score_idx = -1; }
 #ifdef WNW_PHASE_STAMPS
       if (n == 0 && blk.row >= 0) STAMP(12);

@@ -79,7 +79,8 @@ struct CacheView {
   long long *steps;                  // [B]
   long long *step_snap;              // [B][L] the step index as the layer's attention kernel saw it: what the layer's
                                      // selection kernel stamps with (the step-end update may overtake that kernel)
-  int32_t *slot_chunk;               // [B][L][S_max]
+  int32_t *slot_chunk;               // [2][B][L][S_max]: the table a step's attention reads is copy (steps[b] & 1); the step's
+                                     //   selection writes the other copy, which the step's end makes current
   int32_t *chunk_slot;               // [B][L][C_max]
   long long *stamp;                  // [B][L][S_max]
   float *score_sum;                  // [B][L][C_max]
@@ -108,6 +109,10 @@ __host__ __device__ inline long long pool_off(const Geometry &G, const LayerInfo
 }
 __host__ __device__ inline long long fixed_off(const Geometry &G, const LayerInfo &li, int b, int f_idx, int kv) {
   return (long long)b * G.fixed_seq_stride + ((long long)(li.fixed_off + f_idx) * 2 + kv) * G.FB * G.ncp * G.d;
+}
+// slot table of (sequence, layer) in the copy of the given parity (element offset into slot_chunk)
+__host__ __device__ inline long long slot_table_off(const Geometry &G, int parity, long long bl) {
+  return ((long long)parity * G.max_batch * G.L + bl) * G.S_max;
 }
 // compact store of a head by its index among the heads that have one (fixed heads first, then tidal token bases)
 __host__ __device__ inline long long compact_off(const Geometry &G, int b, int head, int kv) {

@@ -48,6 +48,7 @@ __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArg
                                                             // after every selection CTA has finished)
   const long long step_b = cv.step_snap[(long long)b * G.L + a.layer];   // not cv.steps: an eager step's bookkeeping kernel
                                                                          // follows the attention kernel, not this one
+  const int parity = (int)(step_b & 1);   // the copy of the slot tables this step's attention reads; the update writes the other
   const int n_aq = a.n_aq;
   const bool scored = li.n_anchor > 0 && a.score_on && C_b > 0 && a.do_score;
   // shared-memory layout: (M,Z) of the anchor q-heads | this layer's scores | per-warp update workspaces | granule partials
@@ -114,7 +115,7 @@ __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArg
   if (warp < n_par && u_first < n_upd) {
     int lt, src;
     upd_of(u_first, lt, src);
-    select_stage(cv, b, lt, src, scored && src == a.layer, C_b, S_b, lane, select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b));
+    select_stage(cv, b, lt, src, scored && src == a.layer, C_b, S_b, lane, select_ws_at(ws0 + (size_t)warp * ws_bytes, C_b, S_b), parity);
   }
   SEL_PHASE(0);
   cp_async_commit_wait_all();
@@ -167,13 +168,13 @@ __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArg
       const bool local = (scored && src == a.layer) || src == -2;
       if (u != u_first) {  // later rounds stage their own tables
         __syncwarp();
-        select_stage(cv, b, lt, src, local, C_b, S_b, lane, w);
+        select_stage(cv, b, lt, src, local, C_b, S_b, lane, w, parity);
         cp_async_commit_wait_all();
         __syncwarp();
       }
       const float *rank_by = src == -2 ? glob_s : (local ? sc_s : w.sc);
-      const int n_copies = G.lag_mode ? select_and_update_lag(cv, b, lt, src, C_b, S_b, cv.S_base[b], T_a, step_b, lane, rank_by, w)
-                                      : select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, rank_by, w);
+      const int n_copies = G.lag_mode ? select_and_update_lag(cv, b, lt, src, C_b, S_b, cv.S_base[b], T_a, step_b, lane, rank_by, w, parity)
+                                      : select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, rank_by, w, parity);
       if (a.epoch_words && n_copies == 0 && lane == 0) {
         // one sequence: nobody to count; else the sequence whose plan comes in last publishes
         const bool last = a.n_active == 1 || atomicAdd(a.empty_ctr + lt, 1) == a.n_active - 1;
@@ -440,7 +441,9 @@ __global__ void __launch_bounds__(256) wnw_place_scatter_kernel(const __grid_con
         for (int x = 0; x < 4; ++x) cv.stats[(long long)b * 4 + x] = 0ull;
       }
     }
-    for (int s = threadIdx.x; s < G.S_max; s += blockDim.x) { cv.slot_chunk[bl * G.S_max + s] = -1; cv.stamp[bl * G.S_max + s] = 0; }
+    for (int s = threadIdx.x; s < G.S_max; s += blockDim.x) {   // placement resets the step count: copy 0 is current
+      cv.slot_chunk[slot_table_off(G, 0, bl) + s] = -1; cv.slot_chunk[slot_table_off(G, 1, bl) + s] = -1; cv.stamp[bl * G.S_max + s] = 0;
+    }
     for (int c = threadIdx.x; c < G.C_max; c += blockDim.x) { cv.chunk_slot[bl * G.C_max + c] = -1; cv.score_sum[bl * G.C_max + c] = 0.f; }
     const LayerInfo li = cv.layers[layer];
     for (int f = threadIdx.x; f < li.n_fixed; f += blockDim.x) cv.fixed_n[(long long)b * G.F_tot + li.fixed_off + f] = 0;
@@ -548,7 +551,7 @@ __global__ void __launch_bounds__(512) wnw_prefill_select_kernel(const __grid_co
       int rank = 0;
       for (int x = 0; x < C_b; ++x) rank += skey[x] > me;
       if (rank < S_b) {
-        cv.slot_chunk[bl * G.S_max + rank] = c;
+        cv.slot_chunk[slot_table_off(G, 0, bl) + rank] = c;
         cv.chunk_slot[bl * G.C_max + c] = rank;
         cv.stamp[bl * G.S_max + rank] = -1 - (long long)rank;
       }

@@ -389,7 +389,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   CKC(dev_alloc(c, &cv.S_base, B));
   CKC(dev_alloc(c, &cv.steps, B));
   CKC(dev_alloc(c, &cv.step_snap, B * L));
-  CKC(dev_alloc(c, &cv.slot_chunk, B * L * std::max(G.S_max, 1)));
+  CKC(dev_alloc(c, &cv.slot_chunk, 2 * B * L * std::max(G.S_max, 1)));   // two copies, see slot_table_off
   CKC(dev_alloc(c, &cv.chunk_slot, B * L * std::max(G.C_max, 1)));
   CKC(dev_alloc(c, &cv.stamp, B * L * std::max(G.S_max, 1)));
   CKC(dev_alloc(c, &cv.score_sum, B * L * std::max(G.C_max, 1)));
@@ -1553,8 +1553,11 @@ extern "C" wnw_status_t wnw_get_residency(wnw_cache_t *c, int32_t seq, int32_t l
   if ((s = drain(c)) != WNW_OK) return s;
   const int S_b = c->seqs[seq].S;
   const size_t off = ((size_t)seq * c->geo.L + layer) * std::max(c->geo.S_max, 1);
+  long long steps_b = 0;   // the current copy of the table: the one the next step's attention reads
+  CK(cudaMemcpy(&steps_b, c->cv.steps + seq, sizeof(steps_b), cudaMemcpyDeviceToHost));
   if (S_b > 0) {
-    CK(cudaMemcpy(slot_chunk, c->cv.slot_chunk + off, S_b * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(slot_chunk, c->cv.slot_chunk + slot_table_off(c->geo, (int)(steps_b & 1), (long long)seq * c->geo.L + layer),
+                  S_b * sizeof(int32_t), cudaMemcpyDeviceToHost));
     if (stamp) CK(cudaMemcpy(stamp, c->cv.stamp + off, S_b * sizeof(int64_t), cudaMemcpyDeviceToHost));
   }
   *n_slots = S_b;
@@ -1604,9 +1607,13 @@ extern "C" wnw_status_t wnw_get_stats(wnw_cache_t *c, wnw_stats_t *out) {
   std::vector<long long> steps(B);
   CK(cudaMemcpy(st.data(), c->cv.stats, st.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
   CK(cudaMemcpy(steps.data(), c->cv.steps, B * sizeof(long long), cudaMemcpyDeviceToHost));
-  std::vector<int32_t> slot_chunk(B * G.L * std::max(G.S_max, 1)), fixed_n(B * std::max(G.F_tot, 1)),
-      fixed_chunks(B * std::max(G.F_tot, 1) * std::max(G.FB, 1));
-  CK(cudaMemcpy(slot_chunk.data(), c->cv.slot_chunk, slot_chunk.size() * 4, cudaMemcpyDeviceToHost));
+  std::vector<int32_t> slot_both(2 * B * G.L * std::max(G.S_max, 1)), slot_chunk(B * G.L * std::max(G.S_max, 1)),
+      fixed_n(B * std::max(G.F_tot, 1)), fixed_chunks(B * std::max(G.F_tot, 1) * std::max(G.FB, 1));
+  CK(cudaMemcpy(slot_both.data(), c->cv.slot_chunk, slot_both.size() * 4, cudaMemcpyDeviceToHost));
+  for (size_t b = 0; b < B; ++b)   // every sequence's current copy
+    for (int l = 0; l < G.L; ++l)
+      for (int j = 0; j < G.S_max; ++j)
+        slot_chunk[(b * G.L + l) * G.S_max + j] = slot_both[slot_table_off(G, (int)(steps[b] & 1), (long long)(b * G.L + l)) + j];
   CK(cudaMemcpy(fixed_n.data(), c->cv.fixed_n, fixed_n.size() * 4, cudaMemcpyDeviceToHost));
   CK(cudaMemcpy(fixed_chunks.data(), c->cv.fixed_chunks, fixed_chunks.size() * 4, cudaMemcpyDeviceToHost));
   std::vector<int32_t> seg_kept;

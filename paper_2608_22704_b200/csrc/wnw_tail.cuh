@@ -68,11 +68,11 @@ __device__ __forceinline__ SelectWs select_ws_at(unsigned char *p, int C, int S)
 // Stage 1 of a table update (one warp): queue the copies of the layer's table and, if needed, of its source
 // layer's scores.  The caller commits, waits and synchronises.
 __device__ __forceinline__ void select_stage(const CacheView &cv, int b, int lt, int src, bool src_is_local, int C_b, int S_b,
-                                             int lane, const SelectWs &w) {
+                                             int lane, const SelectWs &w, int parity) {
   const Geometry &G = cv.geo;
   const long long bl = (long long)b * G.L + lt;
   for (int s = lane; s < S_b; s += 32) {
-    cp_async_small(w.slot + s, cv.slot_chunk + bl * G.S_max + s, 4);
+    cp_async_small(w.slot + s, cv.slot_chunk + slot_table_off(G, parity, bl) + s, 4);
     cp_async_small(w.stamp + s, cv.stamp + bl * G.S_max + s, 8);
   }
   if (!src_is_local && src >= 0) {
@@ -86,12 +86,12 @@ __device__ __forceinline__ void select_stage(const CacheView &cv, int b, int lt,
 // plan.  Works on the staged table; global memory only receives stores.
 // Returns the number of planned copies (uniform over the warp).
 __device__ __forceinline__ int select_and_update(const CacheView &cv, int b, int lt, int src, int C_b, int S_b, int T_a,
-                                                  long long step, int lane, const float *sc, const SelectWs &w) {
+                                                  long long step, int lane, const float *sc, const SelectWs &w, int parity) {
   const Geometry &G = cv.geo;
   const long long bl = (long long)b * G.L + lt;
   int k = G.topk < S_b ? G.topk : S_b;
   if (src == -1 || C_b <= 0) k = 0;   // -1: nothing to rank by; -2: the global accumulator
-  int *slot_chunk = cv.slot_chunk + bl * G.S_max;
+  int *slot_next = cv.slot_chunk + slot_table_off(G, parity ^ 1, bl);   // the whole updated table goes to the other copy
   int *chunk_slot = cv.chunk_slot + bl * G.C_max;
   long long *stamp = cv.stamp + bl * G.S_max;
   if (k > 0)
@@ -154,13 +154,15 @@ __device__ __forceinline__ int select_and_update(const CacheView &cv, int b, int
       const int old = w.slot[j];
       if (old >= 0) { chunk_slot[old] = -1; ++evictions; }
       w.slot[j] = c; w.stamp[j] = st;
-      slot_chunk[j] = c; chunk_slot[c] = j; stamp[j] = st;
+      chunk_slot[c] = j; stamp[j] = st;
       plan[2 * n_plan] = c;
       plan[2 * n_plan + 1] = j;
     }
     ++n_plan;
     __syncwarp();
   }
+  __syncwarp();
+  for (int s = lane; s < S_b; s += 32) slot_next[s] = w.slot[s];
   if (lane == 0) {
     for (int r = 0; r < k; ++r) cv.sel[bl * G.topk + r] = sel[r];
     cv.n_sel[bl] = k;
@@ -180,13 +182,14 @@ __device__ __forceinline__ int select_and_update(const CacheView &cv, int b, int
 // step - stamp >= delta is released; then the misses take the lowest free dynamic slots in order and are planned.
 // Returns the number of planned copies (uniform over the warp).
 __device__ __forceinline__ int select_and_update_lag(const CacheView &cv, int b, int lt, int src, int C_b, int S_b, int S_base,
-                                                      int T_a, long long step, int lane, const float *sc, const SelectWs &w) {
+                                                      int T_a, long long step, int lane, const float *sc, const SelectWs &w,
+                                                      int parity) {
   const Geometry &G = cv.geo;
   const long long bl = (long long)b * G.L + lt;
   const int n_ch = C_b > 1 ? C_b - 1 : C_b;
   int k = G.topk < n_ch ? G.topk : n_ch;
   if (src == -1 || C_b <= 0) k = 0;
-  int *slot_chunk = cv.slot_chunk + bl * G.S_max;
+  int *slot_next = cv.slot_chunk + slot_table_off(G, parity ^ 1, bl);   // the whole updated table goes to the other copy
   int *chunk_slot = cv.chunk_slot + bl * G.C_max;
   long long *stamp = cv.stamp + bl * G.S_max;
   if (k > 0)
@@ -239,7 +242,7 @@ __device__ __forceinline__ int select_and_update_lag(const CacheView &cv, int b,
     if (s < S_b) {
       const int rc = w.slot[s];
       drop = rc >= 0 && w.stamp[s] != step && step - w.stamp[s] >= (long long)G.delta;
-      if (drop) { w.slot[s] = -1; slot_chunk[s] = -1; chunk_slot[rc] = -1; }
+      if (drop) { w.slot[s] = -1; chunk_slot[rc] = -1; }
     }
     released += __popc(__ballot_sync(0xffffffffu, drop));
   }
@@ -259,13 +262,15 @@ __device__ __forceinline__ int select_and_update_lag(const CacheView &cv, int b,
     }
     if (lane == 0) {
       w.slot[free_j] = segs[i]; w.stamp[free_j] = step;
-      slot_chunk[free_j] = segs[i]; chunk_slot[segs[i]] = free_j; stamp[free_j] = step;
+      chunk_slot[segs[i]] = free_j; stamp[free_j] = step;
       plan[2 * n_plan] = segs[i];
       plan[2 * n_plan + 1] = free_j;
     }
     ++n_plan;
     __syncwarp();
   }
+  __syncwarp();
+  for (int s = lane; s < S_b; s += 32) slot_next[s] = w.slot[s];
   if (lane == 0) {
     for (int r = 0; r < k; ++r) cv.sel[bl * G.topk + r] = sel[r];
     cv.n_sel[bl] = k;
