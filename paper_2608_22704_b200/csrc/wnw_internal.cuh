@@ -205,6 +205,10 @@ struct SelectArgs {
   int32_t *epoch_words;        // [L] or null
   int32_t *empty_ctr;          // [L] sequences with an empty plan (reset by whoever publishes the layer's epoch)
   const int32_t *step_epoch;
+  // Selection that runs beside the step's tidal attention (all layers issued together): the step count is read live (the
+  // snapshot of a layer whose first head is tidal may not be written yet) and, before a layer's plan is rewritten, the
+  // recall of the previous step must be done with it (bounded wait on the layer's epoch word).
+  int32_t overlapped;
 };
 
 // Completion signalling of a recall launch that runs outside the captured step (all null for in-step launches).

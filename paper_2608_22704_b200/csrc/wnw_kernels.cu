@@ -46,7 +46,8 @@ __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArg
   const int C_b = cv.C[b], S_b = cv.S[b], T_a = cv.T_a[b];
   const int epoch_now = a.step_epoch ? *a.step_epoch : 0;   // read here, not on the way out (the step's own bump comes
                                                             // after every selection CTA has finished)
-  const long long step_b = cv.step_snap[(long long)b * G.L + a.layer];   // not cv.steps: an eager step's bookkeeping kernel
+  const long long step_b = a.overlapped ? cv.steps[b]                    // (nothing bumps it before this launch is joined)
+                                        : cv.step_snap[(long long)b * G.L + a.layer];   // not cv.steps: an eager step's bookkeeping kernel
                                                                          // follows the attention kernel, not this one
   const int parity = (int)(step_b & 1);   // the copy of the slot tables this step's attention reads; the update writes the other
   const int n_aq = a.n_aq;
@@ -173,6 +174,20 @@ __device__ __forceinline__ void select_body(const CacheView &cv, const SelectArg
         __syncwarp();
       }
       const float *rank_by = src == -2 ? glob_s : (local ? sc_s : w.sc);
+      if (a.overlapped && a.epoch_words) {
+        // the previous step's recall may still be reading this layer's plan: wait (bounded) until it has published the
+        // layer's epoch; it never waits for anything this kernel does
+        if (lane == 0) {
+          int seen;
+          const long long t0 = clock64();
+          for (;;) {
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];\n" : "=r"(seen) : "l"(a.epoch_words + lt) : "memory");
+            if (seen >= epoch_now) break;
+            if (clock64() - t0 > 2000000000ll) { atomicOr(cv.status, STATUS_TIMEOUT); break; }
+          }
+        }
+        __syncwarp();
+      }
       const int n_copies = G.lag_mode ? select_and_update_lag(cv, b, lt, src, C_b, S_b, cv.S_base[b], T_a, step_b, lane, rank_by, w, parity)
                                       : select_and_update(cv, b, lt, src, C_b, S_b, T_a, step_b, lane, rank_by, w, parity);
       if (a.epoch_words && n_copies == 0 && lane == 0) {
@@ -222,6 +237,7 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_all_kernel(const __
     a_s.fold_total = step.fold_total; a_s.fold_appended = step.fold_appended;
     a_s.fold_counter = step.fold_counter; a_s.fold_bump_epoch = step.fold_bump_epoch;
     a_s.epoch_words = step.epoch_words; a_s.empty_ctr = step.empty_ctr; a_s.step_epoch = step.step_epoch;
+    a_s.overlapped = step.overlapped;
   }
   __syncthreads();
   select_body(cv, a_s, smem_total, smem, blockIdx.x, m.y, m.z);
@@ -247,6 +263,7 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) wnw_select_all_p_kernel(const 
     a_s.fold_total = step.fold_total; a_s.fold_appended = step.fold_appended;
     a_s.fold_counter = step.fold_counter; a_s.fold_bump_epoch = step.fold_bump_epoch;
     a_s.epoch_words = step.epoch_words; a_s.empty_ctr = step.empty_ctr; a_s.step_epoch = step.step_epoch;
+    a_s.overlapped = step.overlapped;
   }
   __syncthreads();
   select_body(cv, a_s, smem_total, smem, blockIdx.x, m.y, m.z);

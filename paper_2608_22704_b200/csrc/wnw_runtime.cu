@@ -120,6 +120,9 @@ struct wnw_cache {
   int layer_dependency = WNW_LAYERS_INDEPENDENT;
   std::vector<AttnArgs> batch_args;   // BATCHED layers of a captured step: recorded per layer, launched by the last one
   bool cap_batched = false, batched_two_part = true;
+  // the step's selection beside its tidal attention (all layers issued together, two parts): forked after the first part
+  bool cap_sel_overlap = false, sel_overlap_enabled = true;
+  cudaEvent_t ev_sel_fork = nullptr, ev_sel_join = nullptr;
   int batched_target = 0;             // granules of work per CTA when the step's layers share one launch ...
   int batched_target_tidal = 0;       // ... and per CTA of its second part, the tidal heads
   // replayed steps: one recall launch per step outside the captured graph, overlapping the next step
@@ -220,6 +223,8 @@ static void destroy_impl(wnw_cache *c) {
   for (auto e : c->ev_side_done) cudaEventDestroy(e);
   for (auto e : c->ev_layer_done_cap) cudaEventDestroy(e);
   for (auto e : c->ev_side_done_cap) cudaEventDestroy(e);
+  if (c->ev_sel_fork) cudaEventDestroy(c->ev_sel_fork);
+  if (c->ev_sel_join) cudaEventDestroy(c->ev_sel_join);
   if (c->ev_place) cudaEventDestroy(c->ev_place);
   if (c->ev_step) cudaEventDestroy(c->ev_step);
   if (c->ev_graph_done) cudaEventDestroy(c->ev_graph_done);
@@ -291,6 +296,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
   if (const char *e = getenv("WNW_PDL")) c->pdl_enabled = atoi(e) != 0;
   if (const char *e = getenv("WNW_BATCH_TWO_PART")) c->batched_two_part = atoi(e) != 0;
+  if (const char *e = getenv("WNW_SELECT_OVERLAP")) c->sel_overlap_enabled = atoi(e) != 0;
   if (const char *e = getenv("WNW_PACK")) { c->pack_granules = atoi(e); c->pack_enabled = c->pack_granules != 0; if (c->pack_granules < 0) c->pack_granules = 0; }
   if (const char *e = getenv("WNW_FOLD_STEP_END")) c->fold_enabled = atoi(e) != 0;
   if (const char *e = getenv("WNW_SELECT_ALL")) c->select_all_enabled = atoi(e) != 0;
@@ -462,6 +468,10 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     CKE(cudaEventCreateWithFlags(&c->ev_side_done[l], cudaEventDisableTiming));
     CKE(cudaEventCreateWithFlags(&c->ev_layer_done_cap[l], cudaEventDisableTiming));
     CKE(cudaEventCreateWithFlags(&c->ev_side_done_cap[l], cudaEventDisableTiming));
+    if (l == 0) {
+      CKE(cudaEventCreateWithFlags(&c->ev_sel_fork, cudaEventDisableTiming));
+      CKE(cudaEventCreateWithFlags(&c->ev_sel_join, cudaEventDisableTiming));
+    }
   }
   CKE(cudaEventCreateWithFlags(&c->ev_place, cudaEventDisableTiming));
   CKE(cudaEventCreateWithFlags(&c->ev_step, cudaEventDisableTiming));
@@ -1079,6 +1089,29 @@ static cudaError_t select_all(wnw_cache *c, const int *range, const SelectArgs &
   return launch_select_all(c->cv, c->d_sel_args, c->d_sel_map + range[0], range[1], stp, c->sel_all_smem, st);
 }
 
+// The selection work of a captured step in one launch (two when a layer ranks by another layer's scores).  overlapped:
+// it runs beside the step's tidal attention and leaves the step's bookkeeping to a step-end kernel.
+static wnw_status_t launch_step_selection(wnw_cache *c, bool overlapped, cudaStream_t st) {
+  SelectArgs stp{};
+  stp.n_active = (int)c->active.size(); stp.active = c->d_active;
+  stp.epoch_words = c->d_recall_epoch; stp.empty_ctr = c->d_empty_ctr; stp.step_epoch = c->d_step_epoch;
+  stp.overlapped = overlapped ? 1 : 0;
+  if (!c->select_single_ok) {   // first every anchor layer's scores, then every table update
+    stp.do_score = 1; stp.do_update = 0;
+    CK(select_all(c, c->sel_map_score, stp, st));
+    if (c->sel_map_score[1] > 0) c->count_launch(1, 1, true);
+  }
+  const int *range = c->select_single_ok ? c->sel_map_single : c->sel_map_update;
+  stp.do_score = c->select_single_ok ? 1 : 0; stp.do_update = 1;
+  if (!overlapped) {
+    stp.fold_total = range[1] * stp.n_active; stp.fold_appended = c->appended == 1;
+    stp.fold_counter = c->d_fold_ctr; stp.fold_bump_epoch = c->d_step_epoch;
+  }
+  CK(select_all(c, range, stp, st));
+  c->count_launch(1, 1, true);
+  return WNW_OK;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Decode step
 // ---------------------------------------------------------------------------------------------
@@ -1175,6 +1208,19 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     c->cap_batched = c->layer_dependency == WNW_LAYERS_BATCHED && capturing && c->graph_capturing && one_shot &&
                      (!tiered || c->cap_select_all);
     if (c->cap_batched) c->batch_args.assign(G.L, AttnArgs{});
+    // Two parts (slot-free CTAs, then the tidal heads'): every anchor head is in the first, so the step's selection can
+    // run beside the second; the step's bookkeeping then waits for both (a step-end kernel instead of the fold).
+    c->cap_sel_overlap = false;
+    if (c->cap_batched && tiered && c->batched_two_part && c->sel_overlap_enabled && c->cap_external_recall && c->cap_select_all) {
+      bool any_free = false, any_tidal = false;
+      for (const LayerWork &w : c->wl_layers) {
+        const int n_free = w.packed ? w.n_ctas_free : 0;
+        any_free = any_free || n_free > 0;
+        any_tidal = any_tidal || n_free < (w.n_ctas > 0 ? w.n_ctas : w.n_items);
+      }
+      c->cap_sel_overlap = any_free && any_tidal;
+      if (c->cap_sel_overlap) c->cap_fold = false;
+    }
   }
   if (!capturing) {
     if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
@@ -1240,6 +1286,14 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
       }
       if (tiered && any_free && any_tidal && c->batched_two_part) {
         CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_free.data(), 0, st));
+        if (c->cap_sel_overlap) {   // the selection depends on the first part only (all anchor heads are in it)
+          c->appended = has_new;
+          CK(cudaEventRecord(c->ev_sel_fork, st));
+          CK(cudaStreamWaitEvent(c->side[0], c->ev_sel_fork, 0));
+          wnw_status_t rs = launch_step_selection(c, true, c->side[0]);
+          if (rs != WNW_OK) return rs;
+          CK(cudaEventRecord(c->ev_sel_join, c->side[0]));
+        }
         CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_free.data(), 1, st));
         c->count_launch(0, 2, capturing);
       } else {
@@ -1327,20 +1381,12 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
       if (ls >= 0) CK(cudaStreamWaitEvent(st, c->ev_side_done_cap[ls], 0));
 
   if (capturing && c->cap_select_all) {
-    SelectArgs stp{};
-    stp.n_active = (int)c->active.size(); stp.active = c->d_active;
-    stp.epoch_words = c->d_recall_epoch; stp.empty_ctr = c->d_empty_ctr; stp.step_epoch = c->d_step_epoch;
-    if (!c->select_single_ok) {   // first every anchor layer's scores, then every table update
-      stp.do_score = 1; stp.do_update = 0;
-      CK(select_all(c, c->sel_map_score, stp, st));
-      if (c->sel_map_score[1] > 0) c->count_launch(1, 1, true);
+    if (c->cap_sel_overlap) {   // forked behind the first part of the attention launch: join it
+      CK(cudaStreamWaitEvent(st, c->ev_sel_join, 0));
+    } else {
+      wnw_status_t rs = launch_step_selection(c, false, st);
+      if (rs != WNW_OK) return rs;
     }
-    const int *range = c->select_single_ok ? c->sel_map_single : c->sel_map_update;
-    stp.do_score = c->select_single_ok ? 1 : 0; stp.do_update = 1;
-    stp.fold_total = range[1] * stp.n_active; stp.fold_appended = c->appended == 1;
-    stp.fold_counter = c->d_fold_ctr; stp.fold_bump_epoch = c->d_step_epoch;
-    CK(select_all(c, range, stp, st));
-    c->count_launch(1, 1, true);
   }
   if (!(capturing && c->cap_fold)) {
     CK(launch_step_end(c->cv, (int)c->active.size(), c->d_active, c->appended == 1,

@@ -129,3 +129,30 @@ def test_undrained_replays_large_launches(dependency, residency):
     b = _run(w, False, 8, dependency=dependency, residency=residency, eager_steps=(2, 5))
     _same(a, b)
     assert b[3][2] > 8      # recall launches per layer, not one per step
+
+
+@pytest.mark.parametrize("budget,chunk,batch,residency", [(0.2, 64, 1, 0), (0.4, 64, 2, 0), (0.2, 25, 2, 1), (0.4, 256, 3, 0)])
+def test_undrained_batched_replays_match_drained(budget, chunk, batch, residency):
+    """All layers issued together (BATCHED): the step's selection runs beside its tidal attention and the recall of the
+    previous step beside both; nothing drained between 16 replays, focus jumping every fourth step (long recalls)."""
+    w = config4(budget=budget, chunk=chunk, batch=batch, n_steps=16)
+    w.n_layers = 8; w.roles = w.roles[:8]
+    a = _run(w, True, 16, dependency=3, residency=residency)
+    b = _run(w, False, 16, dependency=3, residency=residency)
+    _same(a, b)
+    assert a[2]["misses"] > 0 and a[2]["recall_bytes"] > 0
+    attn, sel, rec, end = b[3]
+    assert attn == 2 * 16 and rec == 16 and end == 16     # two attention launches, one recall, one step-end kernel per replay
+    c = _run(w, False, 16, dependency=0, residency=residency)      # and the per-layer launches give the same tables
+    for (t1, s1), (t2, s2) in zip(a[1], c[1]):
+        assert np.array_equal(t1, t2) and np.array_equal(s1, s2)
+    assert a[2] == c[2]
+
+
+def test_undrained_batched_mix_of_eager_steps_and_replays():
+    w = config1(n_steps=14)
+    w.n_layers = 10; w.roles = w.roles[:10]
+    for scope in (0, 1):
+        a = _run(w, True, 14, dependency=3, score_scope=scope, eager_steps=(3, 4, 9))
+        b = _run(w, False, 14, dependency=3, score_scope=scope, eager_steps=(3, 4, 9))
+        _same(a, b)
