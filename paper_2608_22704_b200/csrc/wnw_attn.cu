@@ -256,6 +256,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     epoch_pending = false;
     if (warp == 0) STAMP(13);
   };
+  int parity_b = -1, parity_v = 0;   // slot-table copy of the sequence whose tidal items this CTA is serving
   auto load_ctx = [&](Ctx &c, int qi, bool for_loads) {
     c.item_idx = a.cta_ranges ? a.order[qi] : qi;
     // short item lists travel in the kernel parameters: no global load before the first K/V load is issued
@@ -265,7 +266,11 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     else if (c.it.role == ROLE_TIDAL) { c.v_delta_audio = G.ncp; c.map_audio = &maps.pool; }          // granule's K and
     else { c.v_delta_audio = G.FB * G.ncp; c.map_audio = &maps.fixed; }                            // V rows
     c.m_full = c.m_tail = 0;
-    c.table_parity = (c.it.role == ROLE_TIDAL && cv.steps) ? (int)(cv.steps[c.it.b] & 1) : 0;
+    if (c.it.role == ROLE_TIDAL && cv.steps && c.it.b != parity_b) {   // once per sequence a CTA serves, not per item
+      parity_b = c.it.b;
+      parity_v = (int)(cv.steps[c.it.b] & 1);
+    }
+    c.table_parity = c.it.role == ROLE_TIDAL ? parity_v : 0;
     if (TB && c.it.role == ROLE_TIDAL) {
       const int2 m = cv.tok_m[((long long)c.it.b * G.L + a.layer) * G.Hkv + c.it.h];
       c.m_full = m.x; c.m_tail = m.y;

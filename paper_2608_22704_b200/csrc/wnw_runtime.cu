@@ -1205,8 +1205,8 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     // BATCHED layers: one launch for the whole step where nothing inside the step needs a layer's result earlier
     bool one_shot = G.L <= MULTI_LAYERS_MAX;
     for (const LayerWork &w : c->wl_layers) one_shot = one_shot && !w.throughput;
-    c->cap_batched = c->layer_dependency == WNW_LAYERS_BATCHED && capturing && c->graph_capturing && one_shot &&
-                     (!tiered || c->cap_select_all);
+    c->cap_batched = c->layer_dependency == WNW_LAYERS_BATCHED && c->batched_target > 0 && capturing && c->graph_capturing &&
+                     one_shot && (!tiered || c->cap_select_all);
     if (c->cap_batched) c->batch_args.assign(G.L, AttnArgs{});
     // Two parts (slot-free CTAs, then the tidal heads'): every anchor head is in the first, so the step's selection can
     // run beside the second; the step's bookkeeping then waits for both (a step-end kernel instead of the fold).
