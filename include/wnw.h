@@ -276,9 +276,9 @@ wnw_status_t wnw_get_stats(wnw_cache_t *cache, wnw_stats_t *stats_host);
  *                stream between the layer calls) before the step has ended.  Inside a captured step whose selection
  *                work runs at the end of the step (wnw_graph_begin/end with launches smaller than the machine, recall
  *                not inline; or FULL mode) wnw_decode_layer then only records its arguments and the last layer's call
- *                issues the CTAs of all layers together: one launch, or two when the step has tidal heads (first the
- *                CTAs that read no slot, then, taking the SMs as those leave, the tidal heads', beside which the
- *                step's selection runs); elsewhere the mode behaves as INDEPENDENT.
+ *                issues the CTAs of all layers together: one launch, or up to three when the step has tidal heads
+ *                (the anchor heads, the fixed heads, then, taking the SMs as those leave, the tidal heads'; the step's
+ *                selection runs beside the latter two); elsewhere the mode behaves as INDEPENDENT.
  * Takes effect for layers issued afterwards; a captured step keeps the mode it was captured with.  Not allowed inside
  * a step.  The modes cut the work differently, so outputs agree up to the rounding order of the split merge; selections
  * and tables are the same. */

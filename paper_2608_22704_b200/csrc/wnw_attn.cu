@@ -804,8 +804,9 @@ cudaError_t launch_attn(const CacheView &cv, const AttnArgs &a, cudaStream_t st)
 }
 
 // One launch for the CTAs of n layers (all cut for the one-shot 8-warp variant).
-cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, const int *n_first, int part, cudaStream_t st) {
-  if (n <= 0 || n > MULTI_LAYERS_MAX || (part >= 0 && !n_first)) return cudaErrorInvalidValue;
+cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, const int *first_cta, const int *count_cta,
+                              bool pdl, cudaStream_t st) {
+  if (n <= 0 || n > MULTI_LAYERS_MAX || ((first_cta == nullptr) != (count_cta == nullptr))) return cudaErrorInvalidValue;
   MultiArgs m;
   memset(&m, 0, sizeof(m));
   size_t smem = 0;
@@ -816,7 +817,7 @@ cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, 
     if (a.n_items <= 0) continue;
     if (a.throughput || !a.maps || a.maps != args[0].maps) return cudaErrorInvalidValue;
     const int all = a.cta_ranges ? a.n_ctas : a.n_items;
-    const int first = part == 1 ? n_first[i] : 0, count = part == 0 ? n_first[i] : all - first;
+    const int first = first_cta ? first_cta[i] : 0, count = count_cta ? count_cta[i] : all;
     if (first < 0 || count < 0 || first + count > all) return cudaErrorInvalidValue;
     if (count == 0) continue;
     m.cta_prefix[n_used] = ctas;
@@ -829,7 +830,7 @@ cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, 
   }
   if (n_used == 0) return cudaSuccess;
   m.n = n_used; m.cta_prefix[n_used] = ctas;
-  const bool g16 = cv.geo.g > 8, tb = cv.geo.token_base != 0, pdl = part == 1;
+  const bool g16 = cv.geo.g > 8, tb = cv.geo.token_base != 0;
   const TmaMaps &maps = *args[0].maps;
   if (d == 128) {
     if (g16) return tb ? launch_multi_tb<128, true, NW_LAT, true>(cv, m, smem, maps, pdl, st) : launch_multi_tb<128, true, NW_LAT, false>(cv, m, smem, maps, pdl, st);

@@ -250,9 +250,10 @@ cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_c
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
 cudaError_t configure_attn_kernels();
 // the CTAs of several layers' launches (one-shot variant) in one launch
-// part < 0: all CTAs of every layer; part 0: the first n_first[l] CTAs of layer l; part 1: the rest, launched
-// programmatically dependent on what precedes it in the stream
-cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, const int *n_first, int part, cudaStream_t st);
+// CTAs [first[l], first[l] + count[l]) of every layer l (null: all of them); pdl: launched programmatically dependent on
+// what precedes it in the stream
+cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, const int *first, const int *count, bool pdl,
+                              cudaStream_t st);
 // Encodes the descriptor of one store: base (device), rows, head_dim.  Returns false if the driver refuses.
 bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d);
 cudaError_t configure_select_kernel();

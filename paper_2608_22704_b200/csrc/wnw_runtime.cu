@@ -30,7 +30,8 @@ struct LayerWork {
   bool throughput = false;                         // which kernel variant the items were cut for
   size_t part_off = 0;                             // first partial of this layer in the partial buffers (in items)
   int n_ctas = 0, order_off = 0, ranges_off = 0;   // items per CTA (persistent schedule, or packed short heads): offsets
-  int n_ctas_free = 0;   // BATCHED layers: the first n_ctas_free CTAs hold no tidal head (they need no recall epoch)
+  int n_ctas_free = 0;   // BATCHED layers: the first n_ctas_free CTAs hold no tidal head (they need no recall epoch) ...
+  int n_ctas_anchor = 0; // ... and the first n_ctas_anchor of those hold the anchor heads (what the step's selection waits for)
   bool packed = false;                             // one-shot CTAs that serve several short heads each
   int head_items_off = 0;                          // offset in the uploaded HeadItems array
 };
@@ -665,12 +666,12 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
     auto close_pack = [&]() { if (in_pack > 0) { ++n_packs; in_pack = 0; pack_work = 0; } };
     // BATCHED layers: the heads that read no slot come first and never share a CTA with a tidal head: the launch goes
     // out in two parts, the tidal part (cut finer) behind the other
-    for (int pass = 0; pass < (batched ? 2 : 1); ++pass) {
-      const int tgt = batched && pass == 1 ? c->batched_target_tidal : target;
+    for (int pass = 0; pass < (batched ? 3 : 1); ++pass) {   // anchor heads, then fixed heads, then tidal heads
+      const int tgt = batched && pass == 2 ? c->batched_target_tidal : target;
       for (size_t hd = (size_t)lw.head_items_off; hd < heads.size(); ++hd) {
         const HeadItems &hi = heads[hd];
         const WorkItem &wi = items[lw.first_item + hi.first];
-        if (batched && (wi.role == ROLE_TIDAL) != (pass == 1)) continue;
+        if (batched && (wi.role == ROLE_ANCHOR ? 0 : wi.role == ROLE_TIDAL ? 2 : 1) != pass) continue;
         if (hi.count > 1) {   // a split head: every piece alone
           close_pack();
           for (int x = 0; x < hi.count; ++x) { ranges.push_back(pos); order.push_back(hi.first + x); ++pos; ++n_packs; }
@@ -683,7 +684,8 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
         order.push_back(hi.first); ++pos; ++in_pack; pack_work += work;
       }
       close_pack();
-      if (pass == 0) lw.n_ctas_free = batched ? n_packs : 0;
+      if (pass == 0) lw.n_ctas_anchor = batched ? n_packs : 0;
+      if (pass == 1 || !batched) lw.n_ctas_free = batched ? n_packs : 0;
     }
     ranges.push_back(pos);
     if (any || batched) { lw.n_ctas = n_packs; lw.packed = true; }
@@ -1276,17 +1278,32 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
       // Two parts when the step has tidal heads: first the CTAs that read no slot, one wave of them; then, programmatically
       // dependent, those of the tidal heads, which take the SMs as the first part leaves them.  The recall of the previous
       // step (it runs outside the captured graph, beside this step) has landed by then, so no CTA sits on an SM waiting.
-      std::vector<int> n_free(G.L, 0);
-      bool any_free = false, any_tidal = false;
+      std::vector<int> zero(G.L, 0), n_anchor(G.L, 0), n_fixed(G.L, 0), n_free(G.L, 0), n_tidal(G.L, 0);
+      bool any_free = false, any_tidal = false, any_anchor = false, any_fixed = false;
       for (int l = 0; l < G.L; ++l) {
         const LayerWork &w = c->wl_layers[l];
+        const int all = w.n_ctas > 0 ? w.n_ctas : w.n_items;
         n_free[l] = w.packed ? w.n_ctas_free : 0;
+        n_anchor[l] = w.packed ? w.n_ctas_anchor : 0;
+        n_fixed[l] = n_free[l] - n_anchor[l];
+        n_tidal[l] = all - n_free[l];
         any_free = any_free || n_free[l] > 0;
-        any_tidal = any_tidal || n_free[l] < (w.n_ctas > 0 ? w.n_ctas : w.n_items);
+        any_tidal = any_tidal || n_tidal[l] > 0;
+        any_anchor = any_anchor || n_anchor[l] > 0;
+        any_fixed = any_fixed || n_fixed[l] > 0;
       }
       if (tiered && any_free && any_tidal && c->batched_two_part) {
-        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_free.data(), 0, st));
-        if (c->cap_sel_overlap) {   // the selection depends on the first part only (all anchor heads are in it)
+        // anchor heads first: the step's selection depends on them alone and is forked right behind their launch
+        const bool split_anchor = c->cap_sel_overlap && any_anchor && any_fixed;
+        int n_launch = 0;
+        if (split_anchor) {
+          CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, zero.data(), n_anchor.data(), false, st));
+          ++n_launch;
+        } else {
+          CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, zero.data(), n_free.data(), false, st));
+          ++n_launch;
+        }
+        if (c->cap_sel_overlap) {
           c->appended = has_new;
           CK(cudaEventRecord(c->ev_sel_fork, st));
           CK(cudaStreamWaitEvent(c->side[0], c->ev_sel_fork, 0));
@@ -1294,10 +1311,15 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
           if (rs != WNW_OK) return rs;
           CK(cudaEventRecord(c->ev_sel_join, c->side[0]));
         }
-        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_free.data(), 1, st));
-        c->count_launch(0, 2, capturing);
+        if (split_anchor) {
+          CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_anchor.data(), n_fixed.data(), true, st));
+          ++n_launch;
+        }
+        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_free.data(), n_tidal.data(), true, st));
+        ++n_launch;
+        c->count_launch(0, n_launch, capturing);
       } else {
-        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, nullptr, -1, st));
+        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, nullptr, nullptr, false, st));
         c->count_launch(0, 1, capturing);
       }
     }

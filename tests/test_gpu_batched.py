@@ -1,5 +1,6 @@
 """BATCHED layers: inside a captured step the attention of all layers runs as one launch that carries the CTAs of every
-layer (two with tidal heads: the CTAs that read no slot, cut for one wave, then those of the tidal heads).  Parity against the oracle in the
+layer (three with all head roles: the anchor heads, behind which the step's selection is forked, the fixed heads, the
+tidal heads).  Parity against the oracle in the
 replayed configuration, against the per-layer launches, and the fallbacks.  Needs a B200."""
 import numpy as np
 import pytest
@@ -17,7 +18,7 @@ def _tiny():
                        n_steps=12, roles=[[A, T, T, F], [T, F, T, F], [A, T, F, T]], region=32, jump_every=3)
 
 
-def test_batched_replay_matches_oracle_and_counts_two_attention_launches_per_step():
+def test_batched_replay_matches_oracle_and_counts_three_attention_launches_per_step():
     from parity_harness import Lockstep
     ls = Lockstep(_tiny(), seed=8)
     try:
@@ -26,9 +27,9 @@ def test_batched_replay_matches_oracle_and_counts_two_attention_launches_per_ste
         ls.decode_step(0, check_slots=True)                       # eager: per-layer launches (the mode's fallback)
         c0 = wnw.wnw_get_launch_counts(ls.h)
         for t in range(1, 7):
-            ls.decode_step(t, graph=True, check_slots=True)       # replays: the slot-free CTAs, then the tidal heads'
+            ls.decode_step(t, graph=True, check_slots=True)       # replays: anchor heads, fixed heads, tidal heads
         c1 = wnw.wnw_get_launch_counts(ls.h)
-        assert c1[0] - c0[0] == 2 * 6
+        assert c1[0] - c0[0] == 3 * 6
         ls.decode_step(7, check_slots=True)
         for t in range(8, 12):
             ls.decode_step(t, graph=True, check_slots=True)
@@ -51,7 +52,7 @@ def test_batched_full_size_graph_replay(cfg, steps):
             ls.decode_step(t, graph=True, check_slots=(t == steps - 1))
         ls.check_stats()
         c = wnw.wnw_get_launch_counts(ls.h)
-        assert c[0] == 2 * steps
+        assert c[0] == 3 * steps
         assert ls.max_out_err <= 2e-2
     finally:
         ls.close()

@@ -142,7 +142,7 @@ def test_undrained_batched_replays_match_drained(budget, chunk, batch, residency
     _same(a, b)
     assert a[2]["misses"] > 0 and a[2]["recall_bytes"] > 0
     attn, sel, rec, end = b[3]
-    assert attn == 2 * 16 and rec == 16 and end == 16     # two attention launches, one recall, one step-end kernel per replay
+    assert attn == 3 * 16 and rec == 16 and end == 16     # three attention launches, one recall, one step-end kernel per replay
     c = _run(w, False, 16, dependency=0, residency=residency)      # and the per-layer launches give the same tables
     for (t1, s1), (t2, s2) in zip(a[1], c[1]):
         assert np.array_equal(t1, t2) and np.array_equal(s1, s2)
