@@ -737,7 +737,7 @@ def run_ours(args, rank, world, local_rank):
                                                                                 layers={0: "one launch per layer, overlapping (inputs of every layer resident before the step)",
                                                                                         1: "chained (a layer waits for its predecessor before it reads q)",
                                                                                         2: "serial launches",
-                                                                                        3: "all layers issued together: the CTAs that read no slot in one launch, the tidal heads' in a second (inputs of every layer resident before the step, outputs read after it)"}[args.layer_dependency]),
+                                                                                        3: "all layers issued together: anchor heads, fixed heads and tidal heads in three launches, the selection beside the last two (inputs of every layer resident before the step, outputs read after it)"}[args.layer_dependency]),
         "clocks": clocks, "gpu_launches": int(sum(region_launches)),
         "launches": {"attention": region_launches[0], "selection": region_launches[1], "recall": region_launches[2],
                      "step_end": region_launches[3], "layers_per_attention_launch": w.n_layers / attn_per_step},
@@ -754,8 +754,8 @@ def run_ours(args, rank, world, local_rank):
                      "bytes_per_launch": region_bytes_per_launch, "us_per_launch": region_us_per_launch,
                      "launches": region_launches[0],
                      "duration_kind": "timed region / attention launches (by default the layers of a step are issued together in "
-                                      "two launches, the second filling the SMs as the first leaves them; per-layer launches overlap "
-                                      "inside the replayed step)",
+                                      "three launches that overlap, the last filling the SMs as the others leave them; per-layer "
+                                      "launches overlap inside the replayed step)",
                      "chained": dep.get("chained"), "serial": dep.get("serial"), alt_name: alt,
                      "eager_event_bracket": {"us_per_launch": attn_us, "achieved": achieved, "frac": achieved / peak_gbs,
                                              "launches": attn_n},
