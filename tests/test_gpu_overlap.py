@@ -156,3 +156,13 @@ def test_undrained_batched_mix_of_eager_steps_and_replays():
         a = _run(w, True, 14, dependency=3, score_scope=scope, eager_steps=(3, 4, 9))
         b = _run(w, False, 14, dependency=3, score_scope=scope, eager_steps=(3, 4, 9))
         _same(a, b)
+
+
+def test_undrained_batched_config1_full_stack():
+    """Config 1 at full size (30 layers), 64 replays with nothing drained in between, all layers issued together: the
+    outputs, tables and counters of the drained run."""
+    w = config1(n_steps=64)
+    a = _run(w, True, 64, dependency=3)
+    b = _run(w, False, 64, dependency=3)
+    _same(a, b)
+    assert a[2]["misses"] > 0

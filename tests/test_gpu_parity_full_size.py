@@ -98,15 +98,18 @@ def test_config3_batch32_segment_lag_sampled_sequences():
         ls.close()
 
 
-@pytest.mark.parametrize("residency,seg", [(0, 64), (1, 25)])
-def test_config1_whole_decode_graph_replay(residency, seg):
+@pytest.mark.parametrize("residency,seg,dependency", [(0, 64, 0), (1, 25, 0), (0, 64, 3)])
+def test_config1_whole_decode_graph_replay(residency, seg, dependency):
     """The whole 256-step decode of the 4-minute clip (text 64 -> 320 tokens, one full sweep of the focus through the audio)
-    under graph replay, the oracle following every step: the contract's form and the paper's form."""
+    under graph replay, the oracle following every step: the contract's form and the paper's form with one launch per
+    layer, and the contract's form with all layers issued together (the benchmark's default)."""
+    import paper_2608_22704_b200 as wnw
     from parity_harness import Lockstep
     w = config1(n_steps=256)
     w.chunk = seg
     ls = Lockstep(w, seed=0, gen_device="cuda:0", residency=residency, evict_lag=3)
     try:
+        wnw.wnw_set_layer_dependency(ls.h, dependency)
         ls.prefill(check_slots=False)
         for t in range(256):
             ls.decode_step(t, graph=True, check_slots=(t % 64 == 63))
