@@ -314,25 +314,36 @@ wnw_status_t wnw_measure_host_link(int32_t device, int64_t bytes, int32_t reps, 
  * Some callers cannot call cudaMalloc where they need attention: a serving loop that has given the whole device
  * to its own pool allocator, or a latency-critical decode thread that cannot afford the device-wide
  * synchronisation cudaMalloc and cudaFree imply.  This entry point calls no cudaMalloc, no cudaFree and no
- * allocating library routine; its split-K partials, completion counters and split table live in a fixed array of
- * about 0.8 MB inside the library image, which every GPU that loads the library holds until the process exits.
+ * allocating library routine (no device allocation of any kind; on the host it works from the stack); its
+ * split-K partials, completion counters, split table and status word live in a fixed array of about 0.8 MB inside
+ * the library image, which every GPU that loads the library holds until the process exits.
  *
  *   kv_dev        : DEVICE [n_kv_heads][2][padded_tokens][head_dim] bf16; for each KV head the K rows, then the V
- *                   rows; rows >= n_tokens are never attended to but must be readable
+ *                   rows.  Rows in [n_tokens, padded_tokens) are read (whole 16-row tiles are fetched) but never
+ *                   contribute: they may hold anything, NaN and Inf included
  *   padded_tokens : row capacity per head, a multiple of 16, >= n_tokens
  *   q_dev         : DEVICE [n_q_heads][head_dim] bf16;  out_dev : DEVICE [n_q_heads][head_dim] bf16
  *   softmax_scale : 0 -> 1/sqrt(head_dim)
  * Result: out = softmax(q K^T * scale) V per query head, the same computation wnw_decode_layer_full performs for
  * one sequence.  Limits (beyond them the call returns WNW_ERR_CAPACITY and does nothing): at most 64 KV heads,
  * 128 query heads, group size 16, 1,048,576 padded tokens; head_dim 64 or 128 (else WNW_ERR_UNSUPPORTED).
+ * Each call queues two kernels on cuda_stream: a small one that clears the counters and writes the split table,
+ * then the attention kernel.
  *
  * The first call on a device looks up the array's device address and opts the kernels into their shared-memory
  * size; make that first call before any stream capture on that device.  Every call shares the one array, which
  * keeps the previous call's contents (the call clears what must start at zero): two calls whose GPU work overlaps
- * in time - different streams, or different threads - race on it.  Calls on one stream are safe back to back. */
+ * in time - different streams, or different threads - race on it.  Calls on one stream are safe back to back.
+ *
+ * Every device-side wait of the kernel is bounded.  If one ever runs out (a copy that never lands), the kernel
+ * finishes on what it has, the output is incomplete, and a sticky bit is set in the array's status word;
+ * wnw_attend_static still returned WNW_OK long before.  wnw_attend_static_status waits for the work queued on
+ * cuda_stream, reports whether that happened since it was last asked (timed_out = 1) and clears the bit.  It
+ * allocates nothing either. */
 wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, int32_t padded_tokens, const void *q_dev, void *out_dev,
                                int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, float softmax_scale, int32_t device,
                                void *cuda_stream);
+wnw_status_t wnw_attend_static_status(int32_t device, void *cuda_stream, int32_t *timed_out_host);
 
 const char *wnw_status_string(wnw_status_t status);
 

@@ -79,6 +79,7 @@ _SIGNATURES = {
     "wnw_sync": [_vp],
     "wnw_measure_host_link": [_i32, C.c_int64, _i32, C.POINTER(C.c_double), C.POINTER(C.c_double)],
     "wnw_attend_static": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, C.c_float, _i32, _vp],
+    "wnw_attend_static_status": [_i32, _vp, C.POINTER(_i32)],
 }
 
 
@@ -333,3 +334,11 @@ def wnw_attend_static(kv, n_tokens, q, out, softmax_scale=0.0, stream=None):
     assert two == 2
     _ck(lib().wnw_attend_static(_ptr(kv), n_tokens, padded, _ptr(q), _ptr(out), q.shape[0], n_kv, d, softmax_scale,
                                 kv.device.index or 0, _stream(stream)), "wnw_attend_static")
+
+
+def wnw_attend_static_status(device: int = 0, stream=None) -> bool:
+    """Waits for the stream's queued work; True if a bounded device-side wait of wnw_attend_static ran out since the
+    last query (the output of that call is then incomplete).  Clears the flag."""
+    v = _i32(0)
+    _ck(lib().wnw_attend_static_status(device, _stream(stream), C.byref(v)), "wnw_attend_static_status")
+    return bool(v.value)

@@ -70,7 +70,7 @@ extern "C" int wnw_debug_init_ktime() {
 #endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-// ---- mbarrier + TMA (no cluster multicast anywhere: every CTA fetches its own tiles) ----
+// ---- mbarrier + TMA (every CTA fetches its own tiles) ----
 __device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
 }
@@ -459,6 +459,15 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
         }
         __syncwarp();
       }
+      if (valid < GR) {
+        // rows past the visible ones get probability 0, but 0 x NaN is NaN and a caller-owned buffer (the allocation-free
+        // entry) may hold anything there: clear those V rows (a masked K row only spoils logits that are replaced anyway)
+        for (int r = valid + (lane >> 3); r < GR; r += 4)
+#pragma unroll
+          for (int hf = 0; hf < HALVES; ++hf)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};\n" ::"r"(sV + hf * HALFB + r * 128 + ((lane & 7) << 4)), "r"(0u) : "memory");
+        __syncwarp();
+      }
       float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
       float s2[4] = {0.f, 0.f, 0.f, 0.f}, s3[4] = {0.f, 0.f, 0.f, 0.f};   // odd k-steps: shorter dependent mma chains
       {
@@ -542,7 +551,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     __syncwarp();
     produce();
   }
-  if (timed_out && lane == 0) atomicOr(cv.status, STATUS_TIMEOUT);
+  if (timed_out && lane == 0 && cv.status) atomicOr(cv.status, STATUS_TIMEOUT);
   __syncthreads();
   STAMP(2);
 

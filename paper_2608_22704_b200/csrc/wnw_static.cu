@@ -6,11 +6,11 @@
 // Who this is for: callers that cannot allocate device memory at the point of the call.  A serving loop that has
 // handed the whole device to its own pool allocator, or a latency-critical decode thread for which the implicit
 // device-wide synchronisation of cudaMalloc/cudaFree is not acceptable, can still run an attention step through
-// this entry point: it calls no cudaMalloc, no cudaFree and no allocating library routine.
+// this entry point: it calls no cudaMalloc, no cudaFree and no allocating library routine, and its host side keeps
+// its work list on the stack.
 #include <algorithm>
 #include <cmath>
 #include <cstring>
-#include <vector>
 
 #include "../../include/wnw.h"
 #include "wnw_internal.cuh"
@@ -26,7 +26,9 @@ constexpr long long ST_MAX_TOKENS = 1ll << 20;
 constexpr int ST_MAX_DEVICES = 64;
 
 // layout of the scratch array (byte offsets, all multiples of 256)
-constexpr size_t OFF_ZERO = 0;                                                     // zero words (text length = 0) + head counters
+constexpr size_t OFF_ZERO = 0;                                                     // zero words (text length = 0)
+constexpr size_t OFF_STATUS = 192;                                                 // int32: sticky STATUS_* bits of the kernels' bounded waits;
+                                                                                   //   survives the per-call clearing, reset when it is read
 constexpr size_t OFF_COUNTERS = 256;                                               // int32 [ST_MAX_KV_HEADS]
 constexpr size_t OFF_HEAD_ITEMS = 512;                                             // HeadItems [ST_MAX_KV_HEADS]
 constexpr size_t OFF_HEAD_MZ = 1024;                                               // float2 [ST_MAX_Q_HEADS]
@@ -53,7 +55,39 @@ wnw_status_t scratch_for_current_device(int device, unsigned char **out) {
   return WNW_OK;
 }
 
+// Per call, on the caller's stream ahead of the attention kernel: clears what must start at zero (the zero words, the
+// heads' completion counters) and writes the split table (every head is cut into the same n_cta pieces).  The array
+// keeps the previous call's contents otherwise; the status word is left alone.
+__global__ void static_prepare_kernel(unsigned char *scr, int n_kv_heads, int n_cta) {
+  const int t = threadIdx.x;
+  if (t < (int)(OFF_STATUS / 4)) reinterpret_cast<int32_t *>(scr + OFF_ZERO)[t] = 0;
+  if (t < ST_MAX_KV_HEADS) {
+    reinterpret_cast<int32_t *>(scr + OFF_COUNTERS)[t] = 0;
+    if (t < n_kv_heads) reinterpret_cast<HeadItems *>(scr + OFF_HEAD_ITEMS)[t] = HeadItems{t * n_cta, n_cta};
+  }
+}
+
 }  // namespace
+
+extern "C" wnw_status_t wnw_attend_static_status(int32_t device, void *cuda_stream, int32_t *timed_out) {
+  if (!timed_out) return WNW_ERR_INVALID_ARG;
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) { cudaGetLastError(); return WNW_ERR_CUDA; }
+  if (prev != device && cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return WNW_ERR_CUDA; }
+  struct Restore { int prev, dev; ~Restore() { if (prev != dev) cudaSetDevice(prev); } } restore{prev, device};
+  unsigned char *scr = nullptr;
+  wnw_status_t rc = scratch_for_current_device(device, &scr);
+  if (rc != WNW_OK) return rc;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int32_t word = 0;
+  if (cudaMemcpyAsync(&word, scr + OFF_STATUS, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemsetAsync(scr + OFF_STATUS, 0, sizeof(word), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return WNW_ERR_CUDA;
+  }
+  *timed_out = (word & STATUS_TIMEOUT) ? 1 : 0;
+  return WNW_OK;
+}
 
 extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, int32_t padded_tokens, const void *q_dev,
                                           void *out_dev, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
@@ -84,16 +118,14 @@ extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, 
   int gpi = std::max(nw, (n_gran + per_head_max - 1) / per_head_max);
   gpi = (gpi + nw - 1) / nw * nw;
   const int n_cta = (n_gran + gpi - 1) / gpi;
-  std::vector<WorkItem> items;
-  std::vector<HeadItems> heads;
-  for (int h = 0; h < n_kv_heads; ++h) {
-    heads.push_back(HeadItems{(int)items.size(), n_cta});
+  if (n_cta * n_kv_heads > ST_MAX_ITEMS) return WNW_ERR_CAPACITY;
+  WorkItem items[ST_MAX_ITEMS];   // on the stack: the list travels in the kernel's parameters
+  int n_items = 0;
+  for (int h = 0; h < n_kv_heads; ++h)
     for (int x = 0; x < n_cta; ++x) {
       const int g0 = (int)((long long)n_gran * x / n_cta), g1 = (int)((long long)n_gran * (x + 1) / n_cta);
-      items.push_back(WorkItem{0, h, g0, g1, 0, ROLE_ANCHOR, h, n_tokens, n_gran, 0, 0});
+      items[n_items++] = WorkItem{0, h, g0, g1, 0, ROLE_ANCHOR, h, n_tokens, n_gran, 0, 0};
     }
-  }
-  if ((int)items.size() > ST_MAX_ITEMS) return WNW_ERR_CAPACITY;
 
   CacheView cv;
   memset(&cv, 0, sizeof(cv));
@@ -107,11 +139,11 @@ extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, 
   G.scale_log2 = (float)(scale * 1.4426950408889634);
   cv.text = reinterpret_cast<bf16 *>(scr + OFF_ZERO);
   cv.text_len = reinterpret_cast<int32_t *>(scr + OFF_ZERO);
+  cv.status = reinterpret_cast<int32_t *>(scr + OFF_STATUS);   // where a bounded wait that ran out leaves its mark
 
-  // the array keeps the previous call's contents: clear what must start at zero, then upload the split table
-  if (cudaMemsetAsync(scr + OFF_ZERO, 0, OFF_HEAD_ITEMS, st) != cudaSuccess) { cudaGetLastError(); return WNW_ERR_CUDA; }
-  if (cudaMemcpyAsync(scr + OFF_HEAD_ITEMS, heads.data(), heads.size() * sizeof(HeadItems), cudaMemcpyHostToDevice, st) !=
-      cudaSuccess) { cudaGetLastError(); return WNW_ERR_CUDA; }
+  // the array keeps the previous call's contents: clear what must start at zero and write the split table
+  static_prepare_kernel<<<1, 64, 0, st>>>(scr, n_kv_heads, n_cta);
+  if (cudaGetLastError() != cudaSuccess) return WNW_ERR_CUDA;
 
   // descriptor of the caller's buffer (a host-side encode, no allocation); every role points at it
   TmaMaps maps;
@@ -120,7 +152,7 @@ extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, 
   AttnArgs a{};
   a.maps = &maps;
   a.mode = ATTN_FULL; a.layer = 0; a.n_active = 1; a.has_new = 0; a.score_on = 0;
-  a.items = nullptr; a.items_host = items.data(); a.n_items = (int)items.size(); a.pdl = 0;
+  a.items = nullptr; a.items_host = items; a.n_items = n_items; a.pdl = 0;
   a.head_items = reinterpret_cast<const HeadItems *>(scr + OFF_HEAD_ITEMS);
   a.q = (const bf16 *)q_dev;
   a.anchor_base = (const bf16 *)kv_dev; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
