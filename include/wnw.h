@@ -315,7 +315,7 @@ wnw_status_t wnw_measure_host_link(int32_t device, int64_t bytes, int32_t reps, 
  * to its own pool allocator, or a latency-critical decode thread that cannot afford the device-wide
  * synchronisation cudaMalloc and cudaFree imply.  This entry point calls no cudaMalloc, no cudaFree and no
  * allocating library routine (no device allocation of any kind; on the host it works from the stack); its
- * split-K partials, completion counters, split table and status word live in a fixed array of about 0.8 MB inside
+ * split-K partials, completion counters and status word live in a fixed array of about 0.8 MB inside
  * the library image, which every GPU that loads the library holds until the process exits.
  *
  *   kv_dev        : DEVICE [n_kv_heads][2][padded_tokens][head_dim] bf16; for each KV head the K rows, then the V
@@ -327,8 +327,7 @@ wnw_status_t wnw_measure_host_link(int32_t device, int64_t bytes, int32_t reps, 
  * Result: out = softmax(q K^T * scale) V per query head, the same computation wnw_decode_layer_full performs for
  * one sequence.  Limits (beyond them the call returns WNW_ERR_CAPACITY and does nothing): at most 64 KV heads,
  * 128 query heads, group size 16, 1,048,576 padded tokens; head_dim 64 or 128 (else WNW_ERR_UNSUPPORTED).
- * Each call queues two kernels on cuda_stream: a small one that clears the counters and writes the split table,
- * then the attention kernel.
+ * Each call queues two kernels on cuda_stream: a small one that clears the counters, then the attention kernel.
  *
  * The first call on a device looks up the array's device address and opts the kernels into their shared-memory
  * size; make that first call before any stream capture on that device.  Every call shares the one array, which

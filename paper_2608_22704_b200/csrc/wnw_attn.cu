@@ -20,6 +20,7 @@
 // Chunk scoring, selection and recall are not needed by whatever consumes the attention output next, so they run
 // in wnw_select_kernel / wnw_recall_kernel on a side stream (wnw_kernels.cu), off the critical path.
 #include <cstring>
+#include <type_traits>
 
 #include "wnw_internal.cuh"
 #include "wnw_tail.cuh"
@@ -33,7 +34,7 @@ constexpr int NSTAGE = 3;  // granules in flight per warp
 
 int attn_warps(bool throughput) { return throughput ? NW_THR : NW_LAT; }
 // Merge scratch of a CTA when it sits behind the stages instead of aliasing them: (m, l) and o of every warp.
-static size_t attn_scratch_bytes(int nw, int g, int d) { return (size_t)nw * 128 + (size_t)nw * g * d * 4; }
+static size_t attn_scratch_bytes(int nw, int g, int d) { return (size_t)nw * 128 + (size_t)nw * g * (d + 4) * 4; }
 // One-shot 8-warp CTAs can keep it there while everything fits the 227 KB a CTA may have.
 bool attn_xpref_fits(int g, int d) {
   return (size_t)NW_LAT * NSTAGE * 2 * GR * d * 2 + 1024 + attn_scratch_bytes(NW_LAT, g, d) + 512 <= 227 * 1024;
@@ -42,18 +43,18 @@ bool attn_xpref_fits(int g, int d) {
 
 // Phase stamps for latency studies: compiled in only with -DWNW_PHASE_STAMPS (never in the product build).
 #ifdef WNW_PHASE_STAMPS
-__device__ long long g_stamps[8192 * 16];
-#define STAMP(k) do { if (threadIdx.x == 0 && blockIdx.x < 8192) g_stamps[blockIdx.x * 16 + (k)] = clock64(); } while (0)
+__device__ long long g_stamps[8192 * 32];   // [layer * 64 + CTA of the layer's launch][phase], global-timer nanoseconds
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define STAMP(k) do { if (threadIdx.x == 0 && bid < 64 && a.layer < 128) g_stamps[(a.layer * 64 + bid) * 32 + (k)] = (long long)gtime(); } while (0)
+#define GSTAMP(k) STAMP(k)
 extern "C" int wnw_debug_read_stamps(long long *host, int n_ctas) {
-  return (int)cudaMemcpyFromSymbol(host, g_stamps, sizeof(long long) * 16 * n_ctas);
+  return (int)cudaMemcpyFromSymbol(host, g_stamps, sizeof(long long) * 32 * n_ctas);
 }
 extern "C" int wnw_debug_clear_stamps() {
-  static long long zeros[8192 * 16];
+  static long long zeros[8192 * 32];
   return (int)cudaMemcpyToSymbol(g_stamps, zeros, sizeof(zeros));
 }
 __device__ unsigned long long g_ktime[4 * 64 * 4];   // [step % 4][layer][start_min, trigger_max, end_max, unused], nanoseconds
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define GSTAMP(k) do { if (threadIdx.x == 0 && blockIdx.x < 8192) g_stamps[blockIdx.x * 16 + (k)] = (long long)gtime(); } while (0)
 #define KSTAMP_MIN(slot, k) do { if (threadIdx.x == 0) atomicMin(&g_ktime[(slot) * 4 + (k)], gtime()); } while (0)
 #define KSTAMP_MAX(slot, k) do { if (threadIdx.x == 0) atomicMax(&g_ktime[(slot) * 4 + (k)], gtime()); } while (0)
 extern "C" int wnw_debug_read_ktime(unsigned long long *host) { return (int)cudaMemcpyFromSymbol(host, g_ktime, sizeof(g_ktime)); }
@@ -369,6 +370,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     ++p_n; ++seq_p;
   };
 
+  uint32_t prewaited = 0;   // stages whose bytes have been waited for ahead of the inputs (chained layers)
   for (int qi = q_begin; qi < q_end; ++qi) {
   // without a scratch region of its own the merge below reuses the stages: the previous item's merge must be done
   if (qi > q_begin && !xpref) __syncthreads();
@@ -393,17 +395,58 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   KSTAMP_MIN(kslot, 0);
 #endif
   // the first copies go out before anything else is read; their metadata follows the Q loads
-  bool pro_loaded[NSTAGE - 1];
+  bool pro_loaded[NSTAGE];
   int n_pro = 0;
   if (arm) {
 #pragma unroll
-    for (int n = 0; n < NSTAGE - 1; ++n)
+    for (int n = 0; n < NSTAGE; ++n)
       if (n < n_my) { pro_loaded[n] = issue_copy(prod, n, seq_p + n); n_pro = n + 1; }
   }
   STAMP(1);
+  // Chained layers: while the preceding work still runs, this warp resolves the metadata of the granules it has queued,
+  // waits for their bytes and clears masked V rows; none of it depends on that work.  What is left behind the wait is the
+  // query load, the arithmetic and the merge.
+  const bool early = arm && a.wait_inputs && qi == q_begin;
+  if (early) {
+#pragma unroll
+    for (int n = 0; n < NSTAGE; ++n)
+      if (n < n_pro) issue_meta(prod, n, seq_p + n, pro_loaded[n]);
+    __syncwarp();
+#pragma unroll
+    for (int n = 0; n < NSTAGE; ++n)
+      if (n < n_pro && !timed_out) {
+        const int stage = (int)((seq_p + n) % NSTAGE);
+        const int2 rg = ring[warp][stage];
+        const int valid = rg.x & 255;
+        if (rg.x & 256) {
+          if (!mbar_wait(smem_u32(&bars[warp][stage]), (phase_bits >> stage) & 1u)) timed_out = true;
+          else { phase_bits ^= 1u << stage; prewaited |= 1u << stage; }
+        }
+        if (valid > 0 && valid < GR && !timed_out) {
+          const uint32_t sVz = my_base + stage * 2 * TILEB + TILEB;
+          for (int r = valid + (lane >> 3); r < GR; r += 4)
+#pragma unroll
+            for (int hf = 0; hf < HALVES; ++hf)
+              asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};\n" ::"r"(sVz + hf * HALFB + r * 128 + ((lane & 7) << 4)), "r"(0u) : "memory");
+        }
+      }
+    p_n = n_pro; seq_p += n_pro;
+  }
 
   // Chained layers: the cache loads above never depend on the preceding work, the query and the new token's K/V do.
-  if (a.wait_inputs && qi == q_begin) asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  // Their lines are asked into L2 ahead of the wait (L2 is where the preceding work's stores land, so nothing stale can
+  // be read from it); the loads after the wait go past L1.
+  if (a.wait_inputs && qi == q_begin) {
+    const char *qline = reinterpret_cast<const char *>(a.q + ((long long)it.i * G.Hq + (long long)it.h * g) * D);
+    if (threadIdx.x * 128 < g * D * 2) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(qline + threadIdx.x * 128));
+    if (a.has_new && threadIdx.x < 2) {
+      const bf16 *nb = (threadIdx.x ? a.v_new : a.k_new) + ((long long)it.i * G.Hkv + it.h) * D;
+      asm volatile("prefetch.global.L2 [%0];\n" ::"l"(nb));
+      if (D * 2 > 128) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(reinterpret_cast<const char *>(nb) + 128));
+    }
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
+  }
+  STAMP(6);
   // ---- Q fragments (rows >= g are zero padding); loaded after the first K/V copies are in flight ----
   const int r0 = lane >> 2, cq = (lane & 3) * 2;
   uint32_t qa[KK][NQ];
@@ -411,147 +454,219 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     const bf16 *qb = a.q + ((long long)it.i * G.Hq + (long long)it.h * g) * D;
 #pragma unroll
     for (int kk = 0; kk < KK; ++kk) {
-      qa[kk][0] = r0 < g ? *reinterpret_cast<const uint32_t *>(qb + r0 * D + kk * 16 + cq) : 0u;
-      qa[kk][1] = r0 < g ? *reinterpret_cast<const uint32_t *>(qb + r0 * D + kk * 16 + 8 + cq) : 0u;
+      qa[kk][0] = r0 < g ? __ldcg(reinterpret_cast<const uint32_t *>(qb + r0 * D + kk * 16 + cq)) : 0u;
+      qa[kk][1] = r0 < g ? __ldcg(reinterpret_cast<const uint32_t *>(qb + r0 * D + kk * 16 + 8 + cq)) : 0u;
       if (G16) {
-        qa[kk][2] = r0 + 8 < g ? *reinterpret_cast<const uint32_t *>(qb + (r0 + 8) * D + kk * 16 + cq) : 0u;
-        qa[kk][3] = r0 + 8 < g ? *reinterpret_cast<const uint32_t *>(qb + (r0 + 8) * D + kk * 16 + 8 + cq) : 0u;
+        qa[kk][2] = r0 + 8 < g ? __ldcg(reinterpret_cast<const uint32_t *>(qb + (r0 + 8) * D + kk * 16 + cq)) : 0u;
+        qa[kk][3] = r0 + 8 < g ? __ldcg(reinterpret_cast<const uint32_t *>(qb + (r0 + 8) * D + kk * 16 + 8 + cq)) : 0u;
       }
     }
   }
-  if (arm) {
+  STAMP(16);
+  if (arm && !early) {
 #pragma unroll
-    for (int n = 0; n < NSTAGE - 1; ++n)
+    for (int n = 0; n < NSTAGE; ++n) {
       if (n < n_pro) issue_meta(prod, n, seq_p + n, pro_loaded[n]);
+      if (n == 0) STAMP(23);
+    }
     p_n = n_pro; seq_p += n_pro;
     if (xpref)   // an item shorter than the pipeline: top up from the items that follow
-      for (int n = n_pro; n < NSTAGE - 1; ++n) produce();
+      for (int n = n_pro; n < NSTAGE; ++n) produce();
   }
 
-  float o[D / 8][4];
+  // ---- per-warp state, transposed: tokens on the M side of the tile, query heads on N ----
+  // S^T[token][head] = K q^T and O^T[d][head] = V^T P^T: an m16n8k16 tile then holds 16 tokens x 8 query heads, so a
+  // group of up to 8 heads fills it with no padding rows (16 heads: two n-tiles) and the accumulators are a quarter of
+  // the [head][d] form's.  A lane owns heads hq = nt*8 + cq + {0,1} of every n-tile: for S^T at tokens r0 and r0+8 of
+  // the granule, for O^T at d = 16 t + r0 and 16 t + r0 + 8.
+  constexpr int NTN = G16 ? 2 : 1;
+  float oT[NTN][D / 16][4];
+  float mrun[NTN][2], lrun[NTN][2];   // running max (log2 units, equal in the lanes that share a head) and this lane's share of the denominator
 #pragma unroll
-  for (int t = 0; t < D / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  for (int nt = 0; nt < NTN; ++nt) {
+#pragma unroll
+    for (int t = 0; t < D / 16; ++t) oT[nt][t][0] = oT[nt][t][1] = oT[nt][t][2] = oT[nt][t][3] = 0.f;
+    mrun[nt][0] = mrun[nt][1] = -INFINITY; lrun[nt][0] = lrun[nt][1] = 0.f;
+  }
+  const float sc = G.scale_log2;
 
-  for (int n = 0; n < n_my; ++n, ++seq_c) {
-    __syncwarp();
-    const int stage = (int)(seq_c % NSTAGE);
-    const int2 rg = ring[warp][stage];
-    const int valid = rg.x & 255;
-    if (rg.x & 256) {  // a copy was queued for this stage: wait for its bytes (bounded)
-      if (!mbar_wait(smem_u32(&bars[warp][stage]), (phase_bits >> stage) & 1u)) { timed_out = true; break; }
-      phase_bits ^= 1u << stage;
-    }
-    if (valid > 0 && !timed_out) {
-
-      const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB;
-      // the row of the token being generated: take it from k_new/v_new and store it into the text region
-      const int j = first + n * NW;
-      if (a.has_new && j < G.n_tg && (T_t - 1) / GR == j) {
-        const int nr = (T_t - 1) - j * GR;
-        if (lane < 2 * PPR) {
-          const int kv = lane / PPR, pc = lane - kv * PPR;
-          const long long noff = ((long long)it.i * G.Hkv + it.h) * D + pc * 8;
-          const uint4 val = *reinterpret_cast<const uint4 *>((kv ? a.v_new : a.k_new) + noff);
-          *reinterpret_cast<uint4 *>(cv.text + text_off(G, b, a.layer, it.h, kv) + (long long)(T_t - 1) * D + pc * 8) = val;
-          const uint32_t dst = (kv ? sV : sK) + (pc >> 3) * HALFB + nr * 128 + (((pc & 7) ^ (nr & 7)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(dst), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+  // One step of the online softmax over NU granules (16 or 32 tokens) that sit in the given stages: two granules give the
+  // warp two independent chains of everything (and one max/rescale for both).
+  auto step = [&](auto nu_tag, const uint32_t (&sKs)[2], const uint32_t (&sVs)[2], const int (&valids)[2], const int (&sidxs)[2]) {
+    constexpr int NU = decltype(nu_tag)::value;
+    float sT[NU][NTN][4];
+    {
+      float sO[NU][NTN][4];   // odd k-steps: shorter dependent mma chains
+#pragma unroll
+      for (int u = 0; u < NU; ++u)
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) sT[u][nt][e] = sO[u][nt][e] = 0.f;
+      const int mtx = lane >> 3, row = ((mtx >> 1) << 3) + (lane & 7);
+#pragma unroll
+      for (int kk = 0; kk < KK; ++kk) {
+        const int piece = 2 * kk + (mtx & 1);
+        const uint32_t off = row * 128 + (kk >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4);
+#pragma unroll
+        for (int u = 0; u < NU; ++u) {
+          uint32_t bk[4];   // K rows 0-7 | 8-15 of the granule x d 0-7 | 8-15 of the k-step: the A operand's four quadrants
+          ldsm_x4(bk, sKs[u] + off);
+#pragma unroll
+          for (int nt = 0; nt < NTN; ++nt)
+            mma16816((kk & 1) ? sO[u][nt] : sT[u][nt], bk[0], bk[2], bk[1], bk[3], qa[kk][2 * nt], qa[kk][2 * nt + 1]);
         }
-        __syncwarp();
       }
-      if (valid < GR) {
-        // rows past the visible ones get probability 0, but 0 x NaN is NaN and a caller-owned buffer (the allocation-free
-        // entry) may hold anything there: clear those V rows (a masked K row only spoils logits that are replaced anyway)
-        for (int r = valid + (lane >> 3); r < GR; r += 4)
 #pragma unroll
-          for (int hf = 0; hf < HALVES; ++hf)
-            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};\n" ::"r"(sV + hf * HALFB + r * 128 + ((lane & 7) << 4)), "r"(0u) : "memory");
-        __syncwarp();
+      for (int u = 0; u < NU; ++u)
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) sT[u][nt][e] += sO[u][nt][e];
+    }
+    STAMP(25);
+    // ---- online softmax per query head (a column of S^T), log2 units, fp32 ----
+    uint32_t pb[NU][NTN][2];   // P^T as the B operand of the PV product: tokens 0-7 | 8-15 of the granule x this lane's head
+#pragma unroll
+    for (int nt = 0; nt < NTN; ++nt) {
+      float v[NU][4];
+      float mxA = -INFINITY, mxB = -INFINITY;
+#pragma unroll
+      for (int u = 0; u < NU; ++u) {
+        const bool lo = r0 < valids[u], hi = r0 + 8 < valids[u];
+        v[u][0] = lo ? sT[u][nt][0] * sc : -INFINITY; v[u][1] = lo ? sT[u][nt][1] * sc : -INFINITY;
+        v[u][2] = hi ? sT[u][nt][2] * sc : -INFINITY; v[u][3] = hi ? sT[u][nt][3] * sc : -INFINITY;
+        mxA = fmaxf(mxA, fmaxf(v[u][0], v[u][2])); mxB = fmaxf(mxB, fmaxf(v[u][1], v[u][3]));
       }
-      float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-      float s2[4] = {0.f, 0.f, 0.f, 0.f}, s3[4] = {0.f, 0.f, 0.f, 0.f};   // odd k-steps: shorter dependent mma chains
-      {
-        const int mtx = lane >> 3, row = ((mtx >> 1) << 3) + (lane & 7);
-        const uint32_t rowaddr = sK + row * 128;
 #pragma unroll
-        for (int kk = 0; kk < KK; ++kk) {
-          uint32_t bk[4];
-          const int piece = 2 * kk + (mtx & 1);
-          ldsm_x4(bk, rowaddr + (kk >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4));
-          float (&t0)[4] = (kk & 1) ? s2 : s0;
-          float (&t1)[4] = (kk & 1) ? s3 : s1;
-          if (G16) {
-            mma16816(t0, qa[kk][0], qa[kk][2], qa[kk][1], qa[kk][3], bk[0], bk[1]);
-            mma16816(t1, qa[kk][0], qa[kk][2], qa[kk][1], qa[kk][3], bk[2], bk[3]);
-          } else {
-            mma16816(t0, qa[kk][0], 0u, qa[kk][1], 0u, bk[0], bk[1]);
-            mma16816(t1, qa[kk][0], 0u, qa[kk][1], 0u, bk[2], bk[3]);
+      for (int sh = 4; sh <= 16; sh <<= 1) {
+        mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, sh));
+        mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, sh));
+      }
+      const float mnA = fmaxf(mrun[nt][0], mxA), mnB = fmaxf(mrun[nt][1], mxB);   // finite: the step has a visible token
+      const float alA = exp2f(mrun[nt][0] - mnA), alB = exp2f(mrun[nt][1] - mnB);
+      mrun[nt][0] = mnA; mrun[nt][1] = mnB;
+      float addA = 0.f, addB = 0.f;
+#pragma unroll
+      for (int u = 0; u < NU; ++u) {
+        v[u][0] = exp2f(v[u][0] - mnA); v[u][2] = exp2f(v[u][2] - mnA);
+        v[u][1] = exp2f(v[u][1] - mnB); v[u][3] = exp2f(v[u][3] - mnB);
+        float eA = v[u][0] + v[u][2], eB = v[u][1] + v[u][3];
+        addA += eA; addB += eB;
+        if (sidxs[u] >= 0) {   // softmax-mass partial of this granule (fp32, before any bf16 rounding): anchor-like heads only
+#pragma unroll
+          for (int sh = 4; sh <= 16; sh <<= 1) {
+            eA += __shfl_xor_sync(0xffffffffu, eA, sh);
+            eB += __shfl_xor_sync(0xffffffffu, eB, sh);
+          }
+          if (r0 == 0) {
+            const int hq = nt * 8 + cq;
+            float2 *ge = a.gran_em + ((long long)it.i * a.n_aq + (long long)ridx * g + hq) * a.n_ag_max + sidxs[u];
+            if (hq < g) ge[0] = make_float2(eA, mnA);
+            if (hq + 1 < g) ge[a.n_ag_max] = make_float2(eB, mnB);
           }
         }
+        // P^T tile [token][head] -> [head][token]: what the PV product wants in its B operand
+        uint32_t p01 = pack_bf16(v[u][0], v[u][1]), p23 = pack_bf16(v[u][2], v[u][3]);
+        asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(pb[u][nt][0]) : "r"(p01));
+        asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(pb[u][nt][1]) : "r"(p23));
+      }
+      lrun[nt][0] = lrun[nt][0] * alA + addA; lrun[nt][1] = lrun[nt][1] * alB + addB;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) { s0[e] += s2[e]; s1[e] += s3[e]; }
-      }
-      // ---- online softmax in log2 units, fp32; columns = tokens cq, cq+1, 8+cq, 9+cq ----
-      const float sc = G.scale_log2;
-      const bool k0 = cq < valid, k1 = cq + 1 < valid, k2 = cq + 8 < valid, k3 = cq + 9 < valid;
-      float v0 = k0 ? s0[0] * sc : -INFINITY, v1 = k1 ? s0[1] * sc : -INFINITY;
-      float v2 = k2 ? s1[0] * sc : -INFINITY, v3 = k3 ? s1[1] * sc : -INFINITY;
-      float mx = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      const float mn0 = fmaxf(m0, mx);
-      const float al0 = exp2f(m0 - mn0);
-      v0 = exp2f(v0 - mn0); v1 = exp2f(v1 - mn0); v2 = exp2f(v2 - mn0); v3 = exp2f(v3 - mn0);
-      float rs0 = (v0 + v1) + (v2 + v3);
-      rs0 += __shfl_xor_sync(0xffffffffu, rs0, 1);
-      rs0 += __shfl_xor_sync(0xffffffffu, rs0, 2);
-      l0 = l0 * al0 + rs0;
-      m0 = mn0;
-      uint32_t pa0 = pack_bf16(v0, v1), pa2 = pack_bf16(v2, v3), pa1 = 0u, pa3 = 0u;
-      float al1 = 1.f, rs1 = 0.f;
-      if (G16) {
-        float w0 = k0 ? s0[2] * sc : -INFINITY, w1 = k1 ? s0[3] * sc : -INFINITY;
-        float w2 = k2 ? s1[2] * sc : -INFINITY, w3 = k3 ? s1[3] * sc : -INFINITY;
-        float my = fmaxf(fmaxf(w0, w1), fmaxf(w2, w3));
-        my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 1));
-        my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 2));
-        const float mn1 = fmaxf(m1, my);
-        al1 = exp2f(m1 - mn1);
-        w0 = exp2f(w0 - mn1); w1 = exp2f(w1 - mn1); w2 = exp2f(w2 - mn1); w3 = exp2f(w3 - mn1);
-        rs1 = (w0 + w1) + (w2 + w3);
-        rs1 += __shfl_xor_sync(0xffffffffu, rs1, 1);
-        rs1 += __shfl_xor_sync(0xffffffffu, rs1, 2);
-        l1 = l1 * al1 + rs1;
-        m1 = mn1;
-        pa1 = pack_bf16(w0, w1); pa3 = pack_bf16(w2, w3);
-      }
-      if (rg.y >= 0 && (lane & 3) == 0) {  // softmax-mass partial of this granule (fp32, before any bf16 rounding)
-        float2 *ge = a.gran_em + ((long long)it.i * a.n_aq + (long long)ridx * g) * a.n_ag_max + rg.y;
-        if (r0 < g) ge[(long long)r0 * a.n_ag_max] = make_float2(rs0, m0);
-        if (G16 && r0 + 8 < g) ge[(long long)(r0 + 8) * a.n_ag_max] = make_float2(rs1, m1);
-      }
+      for (int t = 0; t < D / 16; ++t) { oT[nt][t][0] *= alA; oT[nt][t][1] *= alB; oT[nt][t][2] *= alA; oT[nt][t][3] *= alB; }
+    }
+    STAMP(26);
+    {
+      const int mtx = lane >> 3, row = ((mtx & 1) << 3) + (lane & 7);
 #pragma unroll
-      for (int t = 0; t < D / 8; ++t) {
-        o[t][0] *= al0; o[t][1] *= al0;
-        if (G16) { o[t][2] *= al1; o[t][3] *= al1; }
-      }
-      {
-        const int mtx = lane >> 3, row = ((mtx & 1) << 3) + (lane & 7);
-        const uint32_t rowaddr = sV + row * 128;
+      for (int t2 = 0; t2 < KK; ++t2) {
+        const int piece = 2 * t2 + (mtx >> 1);
+        const uint32_t off = row * 128 + (t2 >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4);
 #pragma unroll
-        for (int t2 = 0; t2 < KK; ++t2) {
-          uint32_t bv[4];
-          const int piece = 2 * t2 + (mtx >> 1);
-          ldsm_x4_t(bv, rowaddr + (t2 >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4));
-          mma16816(o[2 * t2], pa0, pa1, pa2, pa3, bv[0], bv[1]);
-          mma16816(o[2 * t2 + 1], pa0, pa1, pa2, pa3, bv[2], bv[3]);
+        for (int u = 0; u < NU; ++u) {
+          uint32_t bv[4];   // V^T: tokens 0-7 | 8-15 x d 0-7 | 8-15 of the 16-wide d tile, transposed on the way out of shared memory
+          ldsm_x4_t(bv, sVs[u] + off);
+#pragma unroll
+          for (int nt = 0; nt < NTN; ++nt) mma16816(oT[nt][t2], bv[0], bv[2], bv[1], bv[3], pb[u][nt][0], pb[u][nt][1]);
+        }
+      }
+    }
+  };
+
+  STAMP(17);
+  for (int n = 0; n < n_my && !timed_out;) {
+    __syncwarp();
+    // up to two granules per step; a granule with nothing visible (an empty slot, text capacity not yet written) is passed over
+    const int cnt = n + 1 < n_my ? 2 : 1;
+    uint32_t sKs[2] = {0u, 0u}, sVs[2] = {0u, 0u};
+    int valids[2] = {0, 0}, sidxs[2] = {-1, -1};
+    int nu = 0, adv = 0;
+    if (n == 0) STAMP(18);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (u < cnt && !timed_out) {
+        const int stage = (int)((seq_c + u) % NSTAGE);
+        const int2 rg = ring[warp][stage];
+        const int valid = rg.x & 255;
+        const bool pre = (prewaited >> stage) & 1u;   // waited for (and masked rows cleared) ahead of the inputs
+        prewaited &= ~(1u << stage);
+        if ((rg.x & 256) && !pre) {  // a copy was queued for this stage: wait for its bytes (bounded)
+          if (!mbar_wait(smem_u32(&bars[warp][stage]), (phase_bits >> stage) & 1u)) timed_out = true;
+          else phase_bits ^= 1u << stage;
+        }
+        if (!timed_out) ++adv;
+        if (n == 0 && u == 0) STAMP(24);
+        if (valid > 0 && !timed_out) {
+          const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB;
+          // the row of the token being generated: take it from k_new/v_new and store it into the text region
+          const int j = first + (n + u) * NW;
+          if (a.has_new && j < G.n_tg && (T_t - 1) / GR == j) {
+            const int nr = (T_t - 1) - j * GR;
+            if (lane < 2 * PPR) {
+              const int kv = lane / PPR, pc = lane - kv * PPR;
+              const long long noff = ((long long)it.i * G.Hkv + it.h) * D + pc * 8;
+              const uint4 val = __ldcg(reinterpret_cast<const uint4 *>((kv ? a.v_new : a.k_new) + noff));
+              *reinterpret_cast<uint4 *>(cv.text + text_off(G, b, a.layer, it.h, kv) + (long long)(T_t - 1) * D + pc * 8) = val;
+              const uint32_t dst = (kv ? sV : sK) + (pc >> 3) * HALFB + nr * 128 + (((pc & 7) ^ (nr & 7)) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(dst), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+            }
+          }
+          if (valid < GR && !pre) {
+            // rows past the visible ones get probability 0, but 0 x NaN is NaN and a caller-owned buffer (the allocation-free
+            // entry) may hold anything there: clear those V rows (a masked K row only spoils logits that are replaced anyway)
+            for (int r = valid + (lane >> 3); r < GR; r += 4)
+#pragma unroll
+              for (int hf = 0; hf < HALVES; ++hf)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};\n" ::"r"(sV + hf * HALFB + r * 128 + ((lane & 7) << 4)), "r"(0u) : "memory");
+          }
+          if (nu == 0) { sKs[0] = sK; sVs[0] = sV; valids[0] = valid; sidxs[0] = rg.y; }
+          else { sKs[1] = sK; sVs[1] = sV; valids[1] = valid; sidxs[1] = rg.y; }
+          ++nu;
         }
       }
     }
     __syncwarp();
-    produce();
+    if (n == 0) STAMP(7);
+    if (timed_out) { seq_c += adv; break; }   // the stages whose bytes never came are drained (bounded) before the CTA ends
+    {
+      if (nu == 2) step(std::integral_constant<int, 2>{}, sKs, sVs, valids, sidxs);
+      else if (nu == 1) step(std::integral_constant<int, 1>{}, sKs, sVs, valids, sidxs);
+    }
+    __syncwarp();
+    if (n == 0) STAMP(8);
+    n += cnt; seq_c += cnt;
+    for (int u = 0; u < cnt; ++u) produce();
   }
+  STAMP(9);
   if (timed_out && lane == 0 && cv.status) atomicOr(cv.status, STATUS_TIMEOUT);
+  // the lanes that share a head add up their shares of its denominator
+#pragma unroll
+  for (int nt = 0; nt < NTN; ++nt)
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      lrun[nt][0] += __shfl_xor_sync(0xffffffffu, lrun[nt][0], sh);
+      lrun[nt][1] += __shfl_xor_sync(0xffffffffu, lrun[nt][1], sh);
+    }
   __syncthreads();
   STAMP(2);
 
@@ -559,23 +674,39 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   // scratch: behind the stages when the pipeline runs across items (copies of the next item are landing in them),
   // otherwise the stages themselves, which are idle by now
   unsigned char *scratch = xpref ? smem + (size_t)NW * NSTAGE * 2 * TILEB : smem;
+  constexpr int RS = D + 4;   // row stride of red_o in floats: the transposed accumulators are stored without bank conflicts
   float2 *red_ml = reinterpret_cast<float2 *>(scratch);                           // [NW][16]
-  float *red_o = reinterpret_cast<float *>(scratch + NW * 16 * sizeof(float2));   // [NW][g][D]
-  if ((lane & 3) == 0) {
-    red_ml[warp * 16 + r0] = make_float2(m0, l0);
-    red_ml[warp * 16 + r0 + 8] = make_float2(G16 ? m1 : -INFINITY, G16 ? l1 : 0.f);
+  float *red_o = reinterpret_cast<float *>(scratch + NW * 16 * sizeof(float2));   // [NW][g][RS]
+  if (r0 == 0) {
+#pragma unroll
+    for (int nt = 0; nt < NTN; ++nt) {
+      red_ml[warp * 16 + nt * 8 + cq] = make_float2(mrun[nt][0], lrun[nt][0]);
+      red_ml[warp * 16 + nt * 8 + cq + 1] = make_float2(mrun[nt][1], lrun[nt][1]);
+    }
+    if (!G16) { red_ml[warp * 16 + 8 + cq] = make_float2(-INFINITY, 0.f); red_ml[warp * 16 + 9 + cq] = make_float2(-INFINITY, 0.f); }
   }
 #pragma unroll
-  for (int t = 0; t < D / 8; ++t) {
-    if (r0 < g) *reinterpret_cast<float2 *>(red_o + ((size_t)warp * g + r0) * D + t * 8 + cq) = make_float2(o[t][0], o[t][1]);
-    if (G16 && r0 + 8 < g)
-      *reinterpret_cast<float2 *>(red_o + ((size_t)warp * g + r0 + 8) * D + t * 8 + cq) = make_float2(o[t][2], o[t][3]);
+  for (int nt = 0; nt < NTN; ++nt) {
+    const int hq = nt * 8 + cq;
+#pragma unroll
+    for (int t = 0; t < D / 16; ++t) {
+      if (hq < g) {
+        red_o[((size_t)warp * g + hq) * RS + t * 16 + r0] = oT[nt][t][0];
+        red_o[((size_t)warp * g + hq) * RS + t * 16 + r0 + 8] = oT[nt][t][2];
+      }
+      if (hq + 1 < g) {
+        red_o[((size_t)warp * g + hq + 1) * RS + t * 16 + r0] = oT[nt][t][1];
+        red_o[((size_t)warp * g + hq + 1) * RS + t * 16 + r0 + 8] = oT[nt][t][3];
+      }
+    }
   }
   __syncthreads();
   // A head served by a single CTA is finished here (bf16 output, final max and denominator); otherwise the CTA
   // leaves one partial in global memory.  The prefill scoring pass always leaves partials.
-  const HeadItems hi = a.head_items[it.i * G.Hkv + it.h];
+  STAMP(20);
+  const HeadItems hi{it.hd_first, it.hd_count};   // travels with the item: no load on the way to the merge
   const bool direct = hi.count == 1 && a.mode != ATTN_PREFILL;
+  if (hi.count > 0) STAMP(21);
   for (int pr = threadIdx.x; pr < g * D / 2; pr += NW * 32) {
     const int idx = pr * 2, row = idx / D;
     float M = -INFINITY;
@@ -587,7 +718,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
       for (int w = 0; w < NW; ++w) {
         const float2 ml = red_ml[w * 16 + row];
         const float f = exp2f(ml.x - M);   // a warp without work has m = -inf -> factor 0
-        const float2 x = *reinterpret_cast<const float2 *>(red_o + ((size_t)w * g + row) * D + (idx - row * D));
+        const float2 x = *reinterpret_cast<const float2 *>(red_o + ((size_t)w * g + row) * RS + (idx - row * D));
         a0 += x.x * f; a1 += x.y * f;
         L += ml.y * f;
       }
@@ -606,10 +737,13 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   if (direct || a.mode == ATTN_PREFILL) continue;
 
   // ---- the CTA that finishes this head last merges its split partials ----
-  __threadfence();
+  // Every thread's partial stores are ordered before the barrier; thread 0's fence after it makes them visible device-wide
+  // before the head's counter moves (cumulative over the barrier).  The CTA that comes last reads the partials past L1,
+  // after it has seen the final count.
   __syncthreads();
   if (threadIdx.x == 0) {
     int *ctr = a.head_done + it.i * G.Hkv + it.h;
+    __threadfence();
     const int prev = atomicAdd(ctr, 1);
     s_flag = prev == hi.count - 1;
     if (s_flag) *ctr = 0;
@@ -617,7 +751,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   __syncthreads();
   STAMP(4);
   if (!s_flag) continue;
-  __threadfence();
+  STAMP(22);
   constexpr int NT = NW * 32;
   {
     // Each thread owns four output columns of one query head.  The partials of up to MB splits are fetched in one
@@ -673,7 +807,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   // after a timeout copies may still be in flight towards this CTA's shared memory: bounded wait before it is released
   for (; seq_c < seq_p; ++seq_c) {
     const int stage = (int)(seq_c % NSTAGE);
-    if (ring[warp][stage].x & 256) {
+    if ((ring[warp][stage].x & 256) && !((prewaited >> stage) & 1u)) {
       mbar_wait(smem_u32(&bars[warp][stage]), (phase_bits >> stage) & 1u);
       phase_bits ^= 1u << stage;
     }

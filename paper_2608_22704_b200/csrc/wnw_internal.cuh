@@ -34,6 +34,7 @@ struct WorkItem {  // one CTA of the attention kernel; everything static about i
   int32_t T_a;     // audio tokens of the sequence
   int32_t C, S;    // chunks of the sequence; its PERMANENT slots (tidal slots from S on may be empty)
   int32_t T_hint;  // text rows known to exist when the list was built (a lower bound: text only grows)
+  int32_t hd_first, hd_count;  // the work items (= split partials) of this item's head: first (relative to the layer's list), number
 };
 constexpr int INLINE_ITEMS_MAX = 96;  // launches with at most this many items carry them in kernel parameters
 struct InlineItems { WorkItem it[INLINE_ITEMS_MAX]; };

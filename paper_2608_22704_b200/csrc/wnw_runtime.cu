@@ -643,7 +643,7 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
         // S: the head's leading permanent units: slots of the table, or blocks of a tidal head's token base
         const int perm = (G.token_base && role == ROLE_TIDAL && !sq.fixed_blocks.empty()) ? std::max(sq.fixed_blocks[layer * G.Hkv + h], 0)
                                                                                          : sq.S_base;
-        items.push_back(WorkItem{(int)i, h, g0, g1, seq_ids[i], role, ridx, sq.T_a, sq.C, perm, sq.T_t});
+        items.push_back(WorkItem{(int)i, h, g0, g1, seq_ids[i], role, ridx, sq.T_a, sq.C, perm, sq.T_t, hi.first, hi.count});
       }
       heads.push_back(hi);
       lw.max_count = std::max(lw.max_count, hi.count);

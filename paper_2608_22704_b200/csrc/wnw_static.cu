@@ -30,7 +30,6 @@ constexpr size_t OFF_ZERO = 0;                                                  
 constexpr size_t OFF_STATUS = 192;                                                 // int32: sticky STATUS_* bits of the kernels' bounded waits;
                                                                                    //   survives the per-call clearing, reset when it is read
 constexpr size_t OFF_COUNTERS = 256;                                               // int32 [ST_MAX_KV_HEADS]
-constexpr size_t OFF_HEAD_ITEMS = 512;                                             // HeadItems [ST_MAX_KV_HEADS]
 constexpr size_t OFF_HEAD_MZ = 1024;                                               // float2 [ST_MAX_Q_HEADS]
 constexpr size_t OFF_PART_ML = 2048;                                               // float2 [ST_MAX_ITEMS][MAX_G]
 constexpr size_t OFF_PART_O = OFF_PART_ML + (size_t)ST_MAX_ITEMS * MAX_G * 8;      // float  [ST_MAX_ITEMS][MAX_G][128]
@@ -56,15 +55,11 @@ wnw_status_t scratch_for_current_device(int device, unsigned char **out) {
 }
 
 // Per call, on the caller's stream ahead of the attention kernel: clears what must start at zero (the zero words, the
-// heads' completion counters) and writes the split table (every head is cut into the same n_cta pieces).  The array
-// keeps the previous call's contents otherwise; the status word is left alone.
-__global__ void static_prepare_kernel(unsigned char *scr, int n_kv_heads, int n_cta) {
+// heads' completion counters).  The array keeps the previous call's contents otherwise; the status word is left alone.
+__global__ void static_prepare_kernel(unsigned char *scr) {
   const int t = threadIdx.x;
   if (t < (int)(OFF_STATUS / 4)) reinterpret_cast<int32_t *>(scr + OFF_ZERO)[t] = 0;
-  if (t < ST_MAX_KV_HEADS) {
-    reinterpret_cast<int32_t *>(scr + OFF_COUNTERS)[t] = 0;
-    if (t < n_kv_heads) reinterpret_cast<HeadItems *>(scr + OFF_HEAD_ITEMS)[t] = HeadItems{t * n_cta, n_cta};
-  }
+  if (t < ST_MAX_KV_HEADS) reinterpret_cast<int32_t *>(scr + OFF_COUNTERS)[t] = 0;
 }
 
 }  // namespace
@@ -124,7 +119,7 @@ extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, 
   for (int h = 0; h < n_kv_heads; ++h)
     for (int x = 0; x < n_cta; ++x) {
       const int g0 = (int)((long long)n_gran * x / n_cta), g1 = (int)((long long)n_gran * (x + 1) / n_cta);
-      items[n_items++] = WorkItem{0, h, g0, g1, 0, ROLE_ANCHOR, h, n_tokens, n_gran, 0, 0};
+      items[n_items++] = WorkItem{0, h, g0, g1, 0, ROLE_ANCHOR, h, n_tokens, n_gran, 0, 0, h * n_cta, n_cta};
     }
 
   CacheView cv;
@@ -141,8 +136,8 @@ extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, 
   cv.text_len = reinterpret_cast<int32_t *>(scr + OFF_ZERO);
   cv.status = reinterpret_cast<int32_t *>(scr + OFF_STATUS);   // where a bounded wait that ran out leaves its mark
 
-  // the array keeps the previous call's contents: clear what must start at zero and write the split table
-  static_prepare_kernel<<<1, 64, 0, st>>>(scr, n_kv_heads, n_cta);
+  // the array keeps the previous call's contents: clear what must start at zero
+  static_prepare_kernel<<<1, 64, 0, st>>>(scr);
   if (cudaGetLastError() != cudaSuccess) return WNW_ERR_CUDA;
 
   // descriptor of the caller's buffer (a host-side encode, no allocation); every role points at it
@@ -153,7 +148,6 @@ extern "C" wnw_status_t wnw_attend_static(const void *kv_dev, int32_t n_tokens, 
   a.maps = &maps;
   a.mode = ATTN_FULL; a.layer = 0; a.n_active = 1; a.has_new = 0; a.score_on = 0;
   a.items = nullptr; a.items_host = items; a.n_items = n_items; a.pdl = 0;
-  a.head_items = reinterpret_cast<const HeadItems *>(scr + OFF_HEAD_ITEMS);
   a.q = (const bf16 *)q_dev;
   a.anchor_base = (const bf16 *)kv_dev; a.anchor_seq_stride = 0; a.anchor_head0 = 0;
   a.part_o = reinterpret_cast<float *>(scr + OFF_PART_O);
