@@ -756,7 +756,10 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   {
     // Each thread owns four output columns of one query head.  The partials of up to MB splits are fetched in one
     // batch of independent loads (one L2 round trip); longer heads continue with an online log-sum-exp merge.
-    constexpr int MB = 16;
+#ifndef WNW_MERGE_BATCH
+#define WNW_MERGE_BATCH 16
+#endif
+    constexpr int MB = WNW_MERGE_BATCH;
     const int nvec = g * D / 4;
     const float4 *po = reinterpret_cast<const float4 *>(a.part_o + (long long)hi.first * g * D);
     const float2 *pml = a.part_ml + (long long)hi.first * g;

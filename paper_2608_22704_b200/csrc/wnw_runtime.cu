@@ -557,7 +557,9 @@ static int granules_per_item(const wnw_cache *c, long long total_granules, int l
     per = std::max<long long>(per, (total_granules + cap - 1) / cap);
     return (int)((per + nw - 1) / nw * nw);
   }
-  long long per = std::max<long long>(2 * min_gpi, (longest_head + 31) / 32);   // two granules per warp: fewer partials to merge
+  int gpw = 2;   // granules per warp of an item
+  if (const char *e = getenv("WNW_GRANULES_PER_WARP")) gpw = std::max(1, atoi(e));
+  long long per = std::max<long long>(gpw * min_gpi, (longest_head + 31) / 32);   // few granules per warp (all in flight at once), few partials to merge
   per = (per + nw - 1) / nw * nw;
   *throughput = (total_granules + per - 1) / per + n_heads > c->n_sm;
   if (const char *e = getenv("WNW_THROUGHPUT")) *throughput = atoi(e) != 0;
