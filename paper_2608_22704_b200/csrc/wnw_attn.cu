@@ -34,7 +34,7 @@ constexpr int NSTAGE = 3;  // granules in flight per warp
 
 int attn_warps(bool throughput) { return throughput ? NW_THR : NW_LAT; }
 // Merge scratch of a CTA when it sits behind the stages instead of aliasing them: (m, l) and o of every warp.
-static size_t attn_scratch_bytes(int nw, int g, int d) { return (size_t)nw * 128 + (size_t)nw * g * (d + 4) * 4; }
+static size_t attn_scratch_bytes(int nw, int g, int d) { return (size_t)nw * 128 + (size_t)nw * g * (d + 2) * 4; }
 // One-shot 8-warp CTAs can keep it there while everything fits the 227 KB a CTA may have.
 bool attn_xpref_fits(int g, int d) {
   return (size_t)NW_LAT * NSTAGE * 2 * GR * d * 2 + 1024 + attn_scratch_bytes(NW_LAT, g, d) + 512 <= 227 * 1024;
@@ -43,15 +43,19 @@ bool attn_xpref_fits(int g, int d) {
 
 // Phase stamps for latency studies: compiled in only with -DWNW_PHASE_STAMPS (never in the product build).
 #ifdef WNW_PHASE_STAMPS
-__device__ long long g_stamps[8192 * 32];   // [layer * 64 + CTA of the layer's launch][phase], global-timer nanoseconds
+#ifndef WNW_STAMP_CTAS
+#define WNW_STAMP_CTAS 64
+#endif
+__device__ long long g_stamps[64 * 512 * 32];   // [layer * WNW_STAMP_CTAS + CTA of the layer's launch][phase], global-timer nanoseconds
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define STAMP(k) do { if (threadIdx.x == 0 && bid < 64 && a.layer < 128) g_stamps[(a.layer * 64 + bid) * 32 + (k)] = (long long)gtime(); } while (0)
+#define STAMP(k) do { if (threadIdx.x == 0 && bid < WNW_STAMP_CTAS && a.layer * WNW_STAMP_CTAS < 64 * 512) g_stamps[(a.layer * WNW_STAMP_CTAS + bid) * 32 + (k)] = (long long)gtime(); } while (0)
 #define GSTAMP(k) STAMP(k)
+#define STAMPV(k, v) do { if (threadIdx.x == 0 && bid < WNW_STAMP_CTAS && a.layer * WNW_STAMP_CTAS < 64 * 512) g_stamps[(a.layer * WNW_STAMP_CTAS + bid) * 32 + (k)] = (long long)(v); } while (0)
 extern "C" int wnw_debug_read_stamps(long long *host, int n_ctas) {
   return (int)cudaMemcpyFromSymbol(host, g_stamps, sizeof(long long) * 32 * n_ctas);
 }
 extern "C" int wnw_debug_clear_stamps() {
-  static long long zeros[8192 * 32];
+  static long long zeros[64 * 512 * 32];
   return (int)cudaMemcpyToSymbol(g_stamps, zeros, sizeof(zeros));
 }
 __device__ unsigned long long g_ktime[4 * 64 * 4];   // [step % 4][layer][start_min, trigger_max, end_max, unused], nanoseconds
@@ -66,6 +70,7 @@ extern "C" int wnw_debug_init_ktime() {
 #else
 #define STAMP(k) do { } while (0)
 #define GSTAMP(k) do { } while (0)
+#define STAMPV(k, v) do { } while (0)
 #define KSTAMP_MIN(slot, k) do { } while (0)
 #define KSTAMP_MAX(slot, k) do { } while (0)
 #endif
@@ -431,6 +436,10 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
         }
       }
     p_n = n_pro; seq_p += n_pro;
+    // the consumer takes two granules at a time and counts on the producer being a full ring ahead: an item shorter than
+    // the pipeline is topped up from the items that follow, here as on the ordinary path
+    if (xpref)
+      for (int n = n_pro; n < NSTAGE; ++n) produce();
   }
 
   // Chained layers: the cache loads above never depend on the preceding work, the query and the new token's K/V do.
@@ -674,7 +683,8 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   // scratch: behind the stages when the pipeline runs across items (copies of the next item are landing in them),
   // otherwise the stages themselves, which are idle by now
   unsigned char *scratch = xpref ? smem + (size_t)NW * NSTAGE * 2 * TILEB : smem;
-  constexpr int RS = D + 4;   // row stride of red_o in floats: the transposed accumulators are stored without bank conflicts
+  constexpr int RS = D + 2;   // row stride of red_o in floats: spreads the transposed accumulators' stores over the banks (two-way
+                              // conflicts left; four more bytes per row and a group of 8 heads no longer fits behind the stages)
   float2 *red_ml = reinterpret_cast<float2 *>(scratch);                           // [NW][16]
   float *red_o = reinterpret_cast<float *>(scratch + NW * 16 * sizeof(float2));   // [NW][g][RS]
   if (r0 == 0) {
@@ -816,6 +826,8 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     }
   }
   GSTAMP(15);
+  STAMPV(27, q_end - q_begin);
+  STAMPV(28, seq_c);
   pdl_finish();
 }
 
@@ -916,7 +928,7 @@ bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long row
 template <int D, bool G16, int NW>
 static cudaError_t configure_t() {
   const size_t want = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024 + attn_scratch_bytes(NW, G16 ? 16 : 8, D);
-  const int bytes = (int)std::min<size_t>(want, 226 * 1024);
+  const int bytes = (int)std::min<size_t>(want, 227 * 1024 - 512);   // what a CTA may have, less this kernel's static shared memory
   cudaError_t e = cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(wnw_attn_multi_kernel<D, G16, NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;

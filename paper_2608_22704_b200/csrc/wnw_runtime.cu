@@ -588,6 +588,88 @@ static void head_granules(const wnw_cache *c, int layer, int mode, const SeqHost
   *work = G.n_tg + audio - (role == ROLE_TIDAL ? (s.S - s.S_base) * G.gpc / 2 : 0);
 }
 
+// Throughput regime (more work than one wave of one-shot CTAs): persistent 4-warp CTAs, two per SM, whose copy pipelines
+// run from one work item into the next.  What an item costs beyond its bytes decides the cut: a head that stays whole is
+// finished inside its CTA, a piece of a split head also pays a fence and a counter round trip under a loaded memory system
+// (measured on 12 layers x 16 sequences x 7500 tokens, chained layers: a CTA with two pieces left 6.5 us after one with a
+// single piece of the same size).  So heads are cut as little as the balance allows: for a piece size T a head becomes
+// round(work / T) even pieces (at least one), the pieces go longest-first to the least loaded CTA, and T is the candidate
+// between 0.3 and three even shares of the launch that gives the shortest longest CTA under that cost model.
+static void build_throughput_items(const wnw_cache *c, int layer, int mode, const std::vector<int> &seq_ids,
+                                   const std::vector<int> &n_gran, const std::vector<int> &n_work, std::vector<WorkItem> &items,
+                                   std::vector<HeadItems> &heads, LayerWork &lw, std::vector<int32_t> &order,
+                                   std::vector<int32_t> &ranges) {
+  const Geometry &G = c->geo;
+  const int nw = attn_warps(true), n_heads = (int)seq_ids.size() * G.Hkv;
+  const double cost_whole = 5.0, cost_piece = 16.0;   // fixed cost of an item in granules' worth: finished in the CTA / left as a partial
+  const double mean_weight = 1.0;   // fixed cost of an item in granules' worth: finished in the CTA / left as a partial
+  const int per_sm = 2;                               // persistent CTAs per SM (4 warps, about 105 KB of shared memory each)
+  double total = 0.0;
+  for (int hd = 0; hd < n_heads; ++hd) total += n_work[hd];
+  const int P = (int)std::min<double>(per_sm * c->n_sm, std::max(1.0, total / (2.0 * nw)));   // at least two granules per warp and CTA
+  const bool may_finish = mode != ATTN_PREFILL;       // the prefill scoring pass leaves partials whatever the cut
+  auto pieces_of = [&](int hd, double T) { return std::max(1, (int)std::lround(n_work[hd] / T)); };
+  auto makespan = [&](double T, std::vector<std::vector<std::pair<int, int>>> *assign) {
+    std::vector<std::pair<double, std::pair<int, int>>> its;   // cost, (head, piece)
+    for (int hd = 0; hd < n_heads; ++hd) {
+      const int np = pieces_of(hd, T);
+      for (int x = 0; x < np; ++x)
+        its.push_back({(double)n_work[hd] / np + ((np > 1 || !may_finish) ? cost_piece : cost_whole), {hd, x}});
+    }
+    std::stable_sort(its.begin(), its.end(), [](const auto &x, const auto &y) { return x.first > y.first; });
+    std::vector<double> load(P, 0.0);
+    if (assign) assign->assign(P, {});
+    for (const auto &e : its) {
+      const int cta = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+      load[cta] += e.first;
+      if (assign) (*assign)[cta].push_back(e.second);
+    }
+    // the longest CTA bounds the launch; the mean load counts too: while some CTAs sit in item overheads the others can
+    // only use the bandwidth they leave if there is work left to overlap, so overhead is never free
+    double sum = 0.0;
+    for (double x : load) sum += x;
+    return *std::max_element(load.begin(), load.end()) + mean_weight * sum / P;
+  };
+  const double share = std::max(total / P, (double)(4 * nw));
+  double best_T = share, best = 1e300;
+  for (int k = 6; k <= 60; ++k) {   // T from 0.3 to three shares in steps of 5 %; ties go to the larger T (fewer items)
+    const double T = share * k / 20.0, ms = makespan(T, nullptr);
+    if (ms <= best) { best = ms; best_T = T; }
+  }
+  std::vector<std::vector<std::pair<int, int>>> assign;
+  makespan(best_T, &assign);
+  // items in head order (a head's pieces are consecutive: the merge reads their partials as one run)
+  std::vector<int> first_item(n_heads, 0);
+  for (int hd = 0; hd < n_heads; ++hd) {
+    const int i = hd / G.Hkv, h = hd % G.Hkv, n = n_gran[hd], np = pieces_of(hd, best_T);
+    const SeqHost &sq = c->seqs[seq_ids[i]];
+    const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
+    const int ridx = mode == ATTN_DECODE ? c->role_idx[layer * G.Hkv + h] : h;
+    const int perm = (G.token_base && role == ROLE_TIDAL && !sq.fixed_blocks.empty()) ? std::max(sq.fixed_blocks[layer * G.Hkv + h], 0)
+                                                                                     : sq.S_base;
+    const HeadItems hi{(int)items.size() - lw.first_item, np};
+    first_item[hd] = hi.first;
+    for (int x = 0; x < np; ++x)
+      items.push_back(WorkItem{i, h, (int)((long long)n * x / np), (int)((long long)n * (x + 1) / np), seq_ids[i], role, ridx, sq.T_a,
+                               sq.C, perm, sq.T_t, hi.first, hi.count});
+    heads.push_back(hi);
+    lw.max_count = std::max(lw.max_count, np);
+  }
+  lw.n_items = (int)items.size() - lw.first_item;
+  lw.order_off = (int)order.size();
+  lw.ranges_off = (int)ranges.size();
+  int pos = 0, n_ctas = 0;
+  for (int cta = 0; cta < P; ++cta) {
+    if (assign[cta].empty()) continue;
+    ranges.push_back(pos);
+    for (const auto &hp : assign[cta]) { order.push_back(first_item[hp.first] + hp.second); ++pos; }
+    ++n_ctas;
+  }
+  ranges.push_back(pos);
+  lw.n_ctas = n_ctas;
+  lw.packed = mode != ATTN_PREFILL;   // the pipeline runs across a CTA's items (its merge scratch sits behind the stages)
+}
+
 // Appends the items of one layer for the given sequences.
 static void build_layer_items(const wnw_cache *c, int layer, int mode, const std::vector<int> &seq_ids,
                               std::vector<WorkItem> &items, std::vector<HeadItems> &heads, LayerWork &lw,
@@ -622,6 +704,10 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   lw.first_item = (int)items.size();
   lw.head_items_off = (int)heads.size();
   lw.max_count = 0;
+  if (throughput) {
+    build_throughput_items(c, layer, mode, seq_ids, n_gran, n_work, items, heads, lw, order, ranges);
+    return;
+  }
   for (size_t i = 0; i < seq_ids.size(); ++i)
     for (int h = 0; h < G.Hkv; ++h) {
       const int n = n_gran[i * G.Hkv + h];
@@ -692,33 +778,6 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
     ranges.push_back(pos);
     if (any || batched) { lw.n_ctas = n_packs; lw.packed = true; }
     else { order.resize(lw.order_off); ranges.resize(lw.ranges_off); }
-  }
-  if (throughput) {
-    // Persistent schedule: one CTA per SM; items go, longest first, to the CTA with the least work so far.  Every
-    // item also costs a prologue and a merge, counted as a few granules' worth.
-    int per_sm = 2;  // persistent CTAs per SM (4 warps, 96 KB of shared memory each)
-    if (const char *e = getenv("WNW_CTAS_PER_SM")) per_sm = std::max(1, atoi(e));
-    const int P = std::min(per_sm * c->n_sm, lw.n_items);
-    std::vector<int> idx(lw.n_items);
-    for (int i = 0; i < lw.n_items; ++i) idx[i] = i;
-    auto weight = [&](int i) { const WorkItem &w = items[lw.first_item + i]; return (w.g1 - w.g0) + 6; };
-    std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return weight(x) > weight(y); });
-    std::vector<long long> load(P, 0);
-    std::vector<std::vector<int>> mine(P);
-    for (int i : idx) {
-      const int cta = (int)(std::min_element(load.begin(), load.end()) - load.begin());
-      mine[cta].push_back(i);
-      load[cta] += weight(i);
-    }
-    lw.order_off = (int)order.size();
-    lw.ranges_off = (int)ranges.size();
-    lw.n_ctas = P;
-    int pos = 0;
-    for (int cta = 0; cta < P; ++cta) {
-      ranges.push_back(pos);
-      for (int i : mine[cta]) { order.push_back(i); ++pos; }
-    }
-    ranges.push_back(pos);
   }
 }
 
