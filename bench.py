@@ -57,11 +57,15 @@ def make_workload(name: str, n_steps: int, seed: int):
         n_l = 4 if name == "prof" else 12
         w = config4(seed=0, budget=0.2, chunk=64, batch=16, n_steps=n_steps)
         w.n_layers = n_l; w.roles = w.roles[:n_l]; w.jump_every = 0; w.sweep_steps = 128; w.name = f"{name}_{n_l}layers_b16_7500"
-    elif name.startswith("b") and "x" in name:   # b<batch>x<audio tokens>: config-1 heads, 12 layers (regime studies)
+    elif name.startswith("b") and "x" in name:   # b<batch>x<audio tokens>[L<layers>]: config-1 heads, 12 layers unless given
         nb, na = name[1:].split("x")
+        n_l = 12
+        if "L" in na:
+            na, n_l = na.split("L")
+        n_l = int(n_l)
         w = config4(seed=0, budget=0.2, chunk=64, batch=int(nb), n_steps=n_steps)
         w.audio_lens = [int(na)] * int(nb)
-        w.n_layers = 12; w.roles = w.roles[:12]; w.jump_every = 0; w.sweep_steps = 256; w.name = f"cfg1heads_12layers_{name}"
+        w.n_layers = n_l; w.roles = w.roles[:n_l]; w.jump_every = 0; w.sweep_steps = 256; w.name = f"cfg1heads_{n_l}layers_{name}"
     else:
         raise SystemExit(f"unknown workload {name}")
     if SWEEP_STEPS_OVERRIDE:
@@ -314,6 +318,48 @@ class Job:
             total += lb
         return total, per_layer
 
+    def set_dependency(self, keys, dep):
+        """Switches how the layers of a step are issued for the given caches (a captured step keeps the form it was
+        captured with, so the captures are dropped)."""
+        for key in keys:
+            self.wnw.wnw_sync(self.caches[key])
+            self.wnw.wnw_set_layer_dependency(self.caches[key], dep)
+            self.captured.discard(key)
+
+    def regen_queries(self, sweep_steps):
+        """New decode queries whose focus crosses the clip in `sweep_steps` steps (k_new, v_new stay)."""
+        self.w.sweep_steps = sweep_steps
+        for b in range(self.B):
+            for l in range(self.w.n_layers):
+                self.q[:, l, b] = self.syn.decode(b, l)["q"]
+
+    def rows_fetched_and_visible(self, key):
+        """(rows the kernels fetch, rows that are visible) per step of a batch-1 cache whose non-anchor heads keep a
+        token-granular base: every store keeps a chunk or segment of n tokens in ceil(n / 16) * 16 rows and the kernels
+        fetch whole 16-row granules of whatever is resident, so short segments move padding."""
+        w, wnw, h = self.w, self.wnw, self.caches[key]
+        pad = lambda n: -(-n // 16) * 16
+        T_a, T_t, C, S = wnw.wnw_get_seq_dims(h, 0)
+        T_t += 1
+        st = wnw.wnw_get_stats(h)
+        visible = st["resident_audio_tokens"] + w.n_layers * w.n_kv_heads * T_t
+        fetched = 0
+        for l in range(w.n_layers):
+            tab = None
+            for hh in range(w.n_kv_heads):
+                role = w.roles[l, hh]
+                fetched += pad(T_t)
+                if role == ROLE_ANCHOR:
+                    fetched += C * pad(w.chunk)
+                    continue
+                kept = len(wnw.wnw_get_fixed_tokens(h, 0, l, hh))
+                fetched += -(-kept // w.chunk) * pad(w.chunk)
+                if role == ROLE_TIDAL:
+                    if tab is None:
+                        tab, _ = wnw.wnw_get_residency(h, 0, l)
+                    fetched += int((tab >= 0).sum()) * pad(w.chunk)
+        return fetched, visible
+
     def destroy(self):
         for h in self.caches.values():
             self.wnw.wnw_destroy(h)
@@ -434,6 +480,95 @@ def run_recall_sweep(args, wnw, dev):
                       "link_memcpy_GBps": link_copy, "link_kernel_GBps": link_kernel, "points": points}), flush=True)
 
 
+def _peak_frac(nbytes, ms, peak_gbs):
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"ms_per_step": ms, "GBps": gbs, "frac": gbs / peak_gbs}
+
+
+def measure_block(wnw, dev, w, peak_gbs, steps=10, warm=3, speech_rate_sweep=0):
+    """One workload, three caches (WnW, WnW with recall copies skipped, own full-cache kernel), each measured in the two
+    ways a step can be issued: `overlapped` (every layer's inputs resident before the step: all layers issued together
+    where they fit one launch, else one overlapping launch per layer) and `chained` (a layer's kernel waits for its
+    predecessor before it reads q: layers that feed one another).  Per form: the replayed step with L2 flushed before
+    it, and K steps back to back in one event bracket (continuous decoding: recall has to pay for what it cannot hide)."""
+    n_total = 2 * (warm + 3 * steps) + (2 * steps + warm if speech_rate_sweep else 0) + 4
+    w.n_steps = n_total
+    job = Job(w, seed=0, device=dev, wnw=wnw)
+    job.create("wnw", wnw.WNW_MODE_TIERED)
+    job.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
+    job.create("full", wnw.WNW_MODE_FULL)
+    job.place_all(["wnw", "skip", "full"])
+    out = {"workload": w.name, "layers": w.n_layers, "batch": w.batch}
+    t = 0
+    for form, dep in (("overlapped", wnw.WNW_LAYERS_BATCHED), ("chained", wnw.WNW_LAYERS_CHAINED)):
+        job.set_dependency(["wnw", "skip", "full"], dep)
+        for tt in range(t, t + warm):
+            for key, full in (("wnw", False), ("skip", False), ("full", True)):
+                job.step(key, tt, full=full)
+        t += warm
+        torch.cuda.synchronize(dev)
+        nb, _ = job.kv_bytes_of_step("wnw")
+        nbf, _ = job.kv_bytes_of_step("full", full=True)
+        s0 = wnw.wnw_get_stats(job.caches["wnw"])
+        ms_w = sum(job.timed_steps("wnw", t, steps)) / steps
+        ms_s = sum(job.timed_steps("skip", t, steps)) / steps
+        ms_f = sum(job.timed_steps("full", t, steps, full=True)) / steps
+        t += steps
+        bb_w = job.timed_region("wnw", t, steps)
+        bb_s = job.timed_region("skip", t, steps)
+        job.timed_region("full", t, steps, full=True)
+        t += steps
+        s1 = wnw.wnw_get_stats(job.caches["wnw"])
+        recall_b = (s1["recall_bytes"] - s0["recall_bytes"]) / (2 * steps)
+        out[form] = {"wnw_copies_skipped": _peak_frac(nb, ms_s, peak_gbs), "full_cache": _peak_frac(nbf, ms_f, peak_gbs),
+                     "wnw": {"ms_per_step": ms_w, "back_to_back_ms_per_step": bb_w, "back_to_back_copies_skipped_ms": bb_s,
+                             "exposed_recall_us_per_step": (bb_w - bb_s) * 1e3, "recall_MB_per_step": recall_b / 1e6,
+                             "tokens_per_s": w.batch / (bb_w * 1e-3)},
+                     "wnw_step_over_full_step": {"flushed": ms_w / ms_f, "copies_skipped": ms_s / ms_f}}
+        out["GB_per_step"], out["full_cache_GB_per_step"] = nb / 1e9, nbf / 1e9
+    if speech_rate_sweep:
+        # the decode focus moving at a speech-like rate (the synthetic sweep crosses the clip 10x faster): same caches
+        job.regen_queries(speech_rate_sweep)
+        for tt in range(t, t + warm):
+            job.step("wnw", tt); job.step("skip", tt)
+        t += warm
+        s0 = wnw.wnw_get_stats(job.caches["wnw"])
+        bb_w = job.timed_region("wnw", t, steps)
+        bb_s = job.timed_region("skip", t, steps)
+        s1 = wnw.wnw_get_stats(job.caches["wnw"])
+        out["speech_rate"] = {"sweep_steps": speech_rate_sweep, "form": "chained", "back_to_back_ms_per_step": bb_w,
+                              "back_to_back_copies_skipped_ms": bb_s, "exposed_recall_us_per_step": (bb_w - bb_s) * 1e3,
+                              "recall_MB_per_step": (s1["recall_bytes"] - s0["recall_bytes"]) / steps / 1e6}
+    job.destroy()
+    del job
+    torch.cuda.empty_cache()
+    return out
+
+
+def chained_batch_sweep(wnw, dev, batches, audio_tokens, steps=8, warm=3):
+    """Chained layers, config-1 shapes at growing batch: the replayed WnW step at 20 % budget against the own full-cache
+    step, L2 flushed before every step: from which batch on the tiered cache is the faster one."""
+    points = []
+    for b in batches:
+        w = make_workload(f"b{b}x{audio_tokens}L30", warm + steps + 2, 0)
+        job = Job(w, seed=0, device=dev, wnw=wnw)
+        job.create("wnw", wnw.WNW_MODE_TIERED, layer_dependency=wnw.WNW_LAYERS_CHAINED)
+        job.create("full", wnw.WNW_MODE_FULL, layer_dependency=wnw.WNW_LAYERS_CHAINED)
+        job.place_all(["wnw", "full"])
+        for tt in range(warm):
+            job.step("wnw", tt); job.step("full", tt, full=True)
+        torch.cuda.synchronize(dev)
+        ms_w = sum(job.timed_steps("wnw", warm, steps)) / steps
+        ms_f = sum(job.timed_steps("full", warm, steps, full=True)) / steps
+        points.append({"batch": b, "wnw_step_us": ms_w * 1e3, "full_cache_step_us": ms_f * 1e3, "wnw_over_full": ms_w / ms_f})
+        job.destroy()
+        del job
+        torch.cuda.empty_cache()
+    below = [p["batch"] for p in points if p["wnw_over_full"] < 1.0]
+    return {"audio_tokens": audio_tokens, "layers": 30, "form": "chained, replayed, L2 flushed, recall on", "points": points,
+            "smallest_batch_with_wnw_below_full_cache": min(below) if below else None}
+
+
 def run_ours(args, rank, world, local_rank):
     import paper_2608_22704_b200 as wnw
     wnw.lib()  # fails loudly if the CUDA library is missing
@@ -446,13 +581,25 @@ def run_ours(args, rank, world, local_rank):
         return
     K, W = args.steps, args.warmup
     R = args.roofline_steps
-    Kc = 0 if (args.quick or args.eager) else min(K, args.chain_steps)
-    Kb = 0 if (args.quick or args.eager) else min(K, args.back_to_back_steps)
-    total = W + R + K + Kb + 2 * Kc   # + the chained and the serial runs
+    DEP = args.layer_dependency
+    dep_names = {0: "one overlapping launch per layer (inputs of every layer resident before the step)",
+                 1: "chained: a layer's kernel waits for its predecessor before it reads q, k_new, v_new (layers that feed one another); its K/V prefetch runs ahead",
+                 2: "serial launches",
+                 3: "all layers issued together (inputs of every layer resident before the step, outputs read after it)"}
+    extras = not (args.quick or args.eager)
+    Kx = min(K, args.alt_steps) if extras else 0        # steps of each alternative issue form
+    Kb = min(K, args.back_to_back_steps) if extras else 0
+    total = W + R + K + Kb + 3 * Kx + 4
     w = make_workload(args.workload, total, 0)
     if args.segment_tokens > 0:
         w.chunk = args.segment_tokens
         w.name += f"_seg{args.segment_tokens}"
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    sampler.start()          # read-only nvidia-smi queries from here to the end of the measured sections
     job = Job(w, seed=rank, device=dev, wnw=wnw, score_scope=args.score_scope, residency=args.residency, evict_lag=args.evict_lag)
     job.create("wnw", wnw.WNW_MODE_FULL if args.quick_full else wnw.WNW_MODE_TIERED, recall_mode=args.recall_mode)
     if args.quick:   # profiler mode: the WnW steps only, nothing else launched
@@ -465,6 +612,7 @@ def run_ours(args, rank, world, local_rank):
         ms, n = wnw.wnw_get_kernel_time(job.caches["wnw"])
         kv_bytes, _ = job.kv_bytes_of_step("wnw", full=args.quick_full)
         ms_step = sum(per_step) / K
+        sampler.stop()
         print(json.dumps({"quick": True, "workload": w.name, "ms_per_step": ms_step, "steps": K,
                           "attn_us_per_launch": ms * 1e3 / max(n, 1), "kv_GB_per_step": kv_bytes / 1e9,
                           "kv_GBps": kv_bytes / (ms_step * 1e-3) / 1e9, "frac_of_peak": kv_bytes / (ms_step * 1e-3) / 1e9 / peak_gbs}),
@@ -473,13 +621,7 @@ def run_ours(args, rank, world, local_rank):
         return
     job.create("full", wnw.WNW_MODE_FULL)
     job.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
-    # the other way to issue layers whose inputs are all resident before the step: one launch for all layers where the
-    # headline uses one per layer (or the reverse); same steps, same state
-    alt_dep = wnw.WNW_LAYERS_INDEPENDENT if Job.layer_dependency == wnw.WNW_LAYERS_BATCHED else wnw.WNW_LAYERS_BATCHED
-    alt_name = "per_layer_launches" if alt_dep == wnw.WNW_LAYERS_INDEPENDENT else "all_layers_one_launch"
-    alt_on = not args.eager and not args.no_alt_form
-    if alt_on:
-        job.create("alt", wnw.WNW_MODE_TIERED, layer_dependency=alt_dep)
+    keys3 = (("wnw", False), ("full", True), ("skip", False))
 
     class Keep:
         store = {}
@@ -487,81 +629,63 @@ def run_ours(args, rank, world, local_rank):
         def __call__(self, b, l):
             return rank == 0 and b == 0 and l < args.oracle_layers
     keep = Keep()
-    job.place_all(["wnw", "full", "skip"] + (["alt"] if alt_on else []), keep_host=keep)
+    job.place_all(["wnw", "full", "skip"], keep_host=keep)
 
     def barrier():
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize(dev)
 
-    # ---- warm-up (all three caches take the same steps so their states stay comparable)
+    # ---- warm-up (all caches take the same steps so their states stay comparable)
     for t in range(W):
-        for key, full in (("wnw", False), ("full", True), ("skip", False)) + ((("alt", False),) if alt_on else ()):
+        for key, full in keys3:
             job.step(key, t, full=full)
     torch.cuda.synchronize(dev)
 
-    # ---- roofline pass: attention-kernel launches bracketed by CUDA events inside the library
+    # ---- eager launches bracketed by CUDA events inside the library (kept for reference: includes host pacing)
     wnw.wnw_set_kernel_timing(job.caches["wnw"], True)
-    wnw.wnw_set_kernel_timing(job.caches["full"], True)
-    algo_bytes = algo_bytes_full = 0
+    algo_bytes = 0
     for t in range(W, W + R):
         b_step, _ = job.kv_bytes_of_step("wnw")
-        bf_step, _ = job.kv_bytes_of_step("full", full=True)
-        algo_bytes += b_step; algo_bytes_full += bf_step
+        algo_bytes += b_step
         job.flush_l2(); job.step("wnw", t)
-        job.flush_l2(); job.step("full", t, full=True)
-        job.step("skip", t)
+        job.step("full", t, full=True); job.step("skip", t)
     attn_ms, attn_n = wnw.wnw_get_kernel_time(job.caches["wnw"])
-    full_ms, full_n = wnw.wnw_get_kernel_time(job.caches["full"])
     wnw.wnw_set_kernel_timing(job.caches["wnw"], False)
-    wnw.wnw_set_kernel_timing(job.caches["full"], False)
 
-    # ---- headline: K steps, device time, L2 flushed between steps, clocks sampled
+    # ---- headline: K replayed steps in the configured issue form, device time, L2 flushed before every step
     stats0 = wnw.wnw_get_stats(job.caches["wnw"])
-    try:
-        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
-    except Exception:
-        gpu_id = str(local_rank)
-    sampler = ClockSampler(gpu_id)
     barrier()
     bytes_before, _ = job.kv_bytes_of_step("wnw")
+    bytes_full, _ = job.kv_bytes_of_step("full", full=True)
     launches0 = wnw.wnw_get_launch_counts(job.caches["wnw"])
-    sampler.start()
     wall0 = time.perf_counter()
     per_step = job.timed_steps("wnw", W + R, K, graph=not args.eager)
     barrier()
     wall = time.perf_counter() - wall0
-    clocks = sampler.stop()
     stats1 = wnw.wnw_get_stats(job.caches["wnw"])
     launches1 = wnw.wnw_get_launch_counts(job.caches["wnw"])
     region_launches = [b - a for a, b in zip(launches0, launches1)]   # attention, selection, recall, step-end kernels
     bytes_after, _ = job.kv_bytes_of_step("wnw")
-    attn_per_step = region_launches[0] / K                             # small layers share a launch
+    attn_per_step = region_launches[0] / K
     region_bytes_per_launch = 0.5 * (bytes_before + bytes_after) / attn_per_step   # the text grows by one token per step
     ms_per_step = dist_max(sum(per_step), dev, world) / K
     value = whole_job_tokens_per_s(world, w.batch, ms_per_step)
 
-    # ---- comparison: own full-cache kernel, and WnW with recall copies skipped (exposed recall time)
-    full_steps = job.timed_steps("full", W + R, K, full=True, graph=not args.eager)
-    skip_steps = job.timed_steps("skip", W + R, K, graph=not args.eager)
-    alt = None
-    if alt_on:
-        for t in range(W, W + R):
-            job.step("alt", t)
-        nb_alt, _ = job.kv_bytes_of_step("alt")
-        ms_alt = dist_max(sum(job.timed_steps("alt", W + R, K)), dev, world) / K
-        alt = {"step_us": ms_alt * 1e3, "achieved": nb_alt / (ms_alt * 1e-3) / 1e9, "frac": nb_alt / (ms_alt * 1e-3) / 1e9 / peak_gbs,
-               "steps": K}
+    # ---- the same steps: own full-cache kernel in the same issue form, and WnW with recall copies skipped
+    ms_full = dist_max(sum(job.timed_steps("full", W + R, K, full=True, graph=not args.eager)), dev, world) / K
+    ms_skip = dist_max(sum(job.timed_steps("skip", W + R, K, graph=not args.eager)), dev, world) / K
+    t_next = W + R + K
     barrier()
-    # ---- continuous decoding: the same steps back to back in one timed region (no flush gaps in which a recall could
-    # finish for free); the difference to the run with copies skipped is the recall time that overlap cannot hide
+    # ---- continuous decoding: steps back to back in one timed region (no flush gaps in which a recall could finish for
+    # free); the difference to the run with copies skipped is the recall time that overlap cannot hide
     bb = None
     if Kb > 0:
-        ms_bb = dist_max(job.timed_region("wnw", W + R + K, Kb), dev, world)
-        ms_bb_skip = dist_max(job.timed_region("skip", W + R + K, Kb), dev, world)
-        if alt is not None:
-            alt["back_to_back_step_us"] = dist_max(job.timed_region("alt", W + R + K, Kb), dev, world) * 1e3
-        bb = {"steps": Kb, "ms_per_step": ms_bb, "ms_per_step_copies_skipped": ms_bb_skip,
+        ms_bb = dist_max(job.timed_region("wnw", t_next, Kb), dev, world)
+        ms_bb_skip = dist_max(job.timed_region("skip", t_next, Kb), dev, world)
+        ms_bb_full = dist_max(job.timed_region("full", t_next, Kb, full=True), dev, world)
+        t_next += Kb
+        bb = {"steps": Kb, "ms_per_step": ms_bb, "ms_per_step_copies_skipped": ms_bb_skip, "full_cache_ms_per_step": ms_bb_full,
               "exposed_recall_us_per_step": (ms_bb - ms_bb_skip) * 1e3, "tokens_per_s": whole_job_tokens_per_s(world, w.batch, ms_bb),
               "note": "K steps in one event bracket, no L2 flush between them (a step reads more than L2 holds only on the "
                       "larger workloads), input staging copies inside the bracket"}
@@ -595,25 +719,30 @@ def run_ours(args, rank, world, local_rank):
     e2e_value = whole_job_tokens_per_s(world, w.batch, dist_max(e2e_ms, dev, world) / n_e2e)
     h2d = job.sslab.numel() * 2
     d2h = job.out.numel() * 2
+    wnw.wnw_destroy(job.caches.pop("e2e"))
 
-    # ---- the same step with layers that feed one another (chained) and with plain serial launches
-    dep = {}
-    if Kc > 0:
-        t_dep = W + R + K + Kb
-        modes = [("chained", wnw.WNW_LAYERS_CHAINED), ("serial", wnw.WNW_LAYERS_SERIAL)]
-        for name, mode in modes:
-            wnw.wnw_sync(job.caches["wnw"])
-            wnw.wnw_set_layer_dependency(job.caches["wnw"], mode)
-            job.captured.discard("wnw")
+    # ---- the other ways to issue the layers of a step, on the same caches (the state simply continues)
+    forms = {}
+    if Kx > 0:
+        others = [(n_, d_) for n_, d_ in (("chained", wnw.WNW_LAYERS_CHAINED), ("upper_bound_all_layers_together", wnw.WNW_LAYERS_BATCHED),
+                                          ("per_layer_overlapped", wnw.WNW_LAYERS_INDEPENDENT), ("serial", wnw.WNW_LAYERS_SERIAL)) if d_ != DEP]
+        for name, mode in others:
+            keys = ["wnw"] if mode == wnw.WNW_LAYERS_SERIAL else ["wnw", "full"]
+            job.set_dependency(keys, mode)
             nb, _ = job.kv_bytes_of_step("wnw")
-            ms = dist_max(sum(job.timed_steps("wnw", t_dep, Kc)), dev, world) / Kc
-            t_dep += Kc
-            us_l = ms * 1e3 / w.n_layers          # one launch per layer in these modes
-            dep[name] = {"step_us": ms * 1e3, "us_per_launch": us_l, "achieved": nb / w.n_layers / (us_l * 1e-6) / 1e9,
-                         "frac": nb / w.n_layers / (us_l * 1e-6) / 1e9 / peak_gbs, "steps": Kc}
-        wnw.wnw_sync(job.caches["wnw"])
-        wnw.wnw_set_layer_dependency(job.caches["wnw"], Job.layer_dependency)
-        job.captured.discard("wnw")
+            l0 = wnw.wnw_get_launch_counts(job.caches["wnw"])[0]
+            ms = dist_max(sum(job.timed_steps("wnw", t_next, Kx)), dev, world) / Kx
+            n_l = (wnw.wnw_get_launch_counts(job.caches["wnw"])[0] - l0) / Kx
+            forms[name] = {"step_us": ms * 1e3, "tokens_per_s": whole_job_tokens_per_s(world, w.batch, ms), "attention_launches_per_step": n_l,
+                           "achieved": nb / (ms * 1e-3) / 1e9, "frac": nb / (ms * 1e-3) / 1e9 / peak_gbs, "steps": Kx}
+            if "full" in keys:
+                ms_f = dist_max(sum(job.timed_steps("full", t_next, Kx, full=True)), dev, world) / Kx
+                forms[name]["full_cache_step_us"] = ms_f * 1e3
+                forms[name]["wnw_step_over_full_step"] = ms / ms_f
+            t_next += Kx
+        job.set_dependency(["wnw", "full"], DEP)
+    clocks = sampler.stop()
+    clocks["window"] = "all measured sections of this run (warm-up to the last issue form); the headline region lies inside it"
 
     if rank != 0:
         job.destroy()
@@ -642,46 +771,26 @@ def run_ours(args, rank, world, local_rank):
                "ms_per_step": ms_oracle,
                "sample": f"sequence 0, first {Ls} of {w.n_layers} layers, {args.oracle_steps} decode steps; time scaled by "
                          f"{w.n_layers}/{Ls} layers and x{w.batch} sequences"}
+    retention = {"r_gpu": stats1["resident_audio_tokens"] / max(stats1["full_audio_tokens"], 1),
+                 "r_gpu_cpu": (stats1["resident_audio_tokens"] + stats1["host_audio_tokens"]) / max(stats1["full_audio_tokens"], 1)}
+    job.destroy()
+    torch.cuda.empty_cache()
 
-    # ---- the HBM-bound regime, in the same run: many long sequences (config-1 heads, 12 layers, 16 x 7500 audio tokens).
-    # Whole-step time of the replayed graph over the algorithmic K,V bytes; recall copies skipped for the WnW figure so
-    # that the host link does not enter (the normal mode is reported beside it).
-    hbm_case = None
-    if not args.no_hbm_case:
-        job.destroy()
-        torch.cuda.empty_cache()
-        wp = make_workload("hbm", 16, 0)
-        jp = Job(wp, seed=0, device=dev, wnw=wnw)
-        jp.create("wnw", wnw.WNW_MODE_TIERED)
-        jp.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
-        jp.create("full", wnw.WNW_MODE_FULL)
-        jp.place_all(["wnw", "skip", "full"])
-        res = {}
-        for key, full in (("wnw", False), ("skip", False), ("full", True)):
-            for tt in range(3):
-                jp.step(key, tt, full=full)
-            torch.cuda.synchronize(dev)
-            nb, _ = jp.kv_bytes_of_step(key, full=full)
-            ms = sum(jp.timed_steps(key, 3, 10, full=full)) / 10
-            res[key] = (nb, ms)
-        hbm_case = {"workload": wp.name, "layers": wp.n_layers, "batch": wp.batch,
-                    "wnw_copies_skipped": {"GB_per_step": res["skip"][0] / 1e9, "ms_per_step": res["skip"][1],
-                                           "GBps": res["skip"][0] / res["skip"][1] / 1e6, "frac": res["skip"][0] / res["skip"][1] / 1e6 / peak_gbs},
-                    "wnw_with_recall": {"ms_per_step": res["wnw"][1], "GBps": res["wnw"][0] / res["wnw"][1] / 1e6},
-                    "full_cache": {"GB_per_step": res["full"][0] / 1e9, "ms_per_step": res["full"][1],
-                                   "GBps": res["full"][0] / res["full"][1] / 1e6, "frac": res["full"][0] / res["full"][1] / 1e6 / peak_gbs},
-                    "note": "whole replayed step over algorithmic K,V bytes; peak = measured copy bandwidth (read+write)"}
-        jp.destroy()
+    # ---- the other configurations of the list, bounded: the 10-minute stack at batch 1, the ragged batch of 32, and the
+    # many-long-sequences case that is HBM-bound at 12 layers; then the chained batch sweep
+    blocks = {}
+    if not args.no_blocks:
+        blocks["hbm_bound_case"] = measure_block(wnw, dev, make_workload("hbm", 64, 0), peak_gbs, steps=10)
+        blocks["cfg2"] = measure_block(wnw, dev, make_workload("cfg2", 64, 0), peak_gbs, steps=10)
+        blocks["cfg3"] = measure_block(wnw, dev, make_workload("cfg3", 96, 0), peak_gbs, steps=8, speech_rate_sweep=1200)
+        blocks["chained_batch_sweep"] = chained_batch_sweep(wnw, dev, (1, 2, 4, 8, 16, 32), 3000)
 
     # ---- the paper's own form of the method on the same model shape: segments of 2 s (25 tokens at 12.5 tokens/s, 50 at
     # 25), chunks of two segments, permanent prefill base with lag-3 release, scores summed over all anchor layers
     paper_form = None
     if not args.no_paper_form:
-        if job.caches:
-            job.destroy()
-        torch.cuda.empty_cache()
-        n_pf, n_bb = 40, 32
-        wq = make_workload(args.workload, W + n_pf + n_bb, 0)
+        n_pf, n_bb = 24, 24
+        wq = make_workload(args.workload, 2 * (W + n_pf) + n_bb + 2, 0)
         wq.chunk = 50 if args.workload == "cfg2" else 25
         jq = Job(wq, seed=0, device=dev, wnw=wnw, score_scope=wnw.WNW_SCOPE_GLOBAL, residency=wnw.WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE,
                  evict_lag=3)
@@ -692,22 +801,33 @@ def run_ours(args, rank, world, local_rank):
         lam_q = 2.0 * wq.budget
         ret_q = wnw.wnw_retention_schedule(np.random.RandomState(0).rand(wq.n_layers * wq.n_kv_heads), lam_q)
         jq.place_all(["wnw", "skip"], token=(ret_q.reshape(wq.n_layers, wq.n_kv_heads), wq.chunk, 0))
-        for tt in range(W):
-            jq.step("wnw", tt); jq.step("skip", tt)
-        torch.cuda.synchronize(dev)
+        res_q = {}
+        tq = 0
+        for form, dep in (("chained", wnw.WNW_LAYERS_CHAINED), ("upper_bound_all_layers_together", wnw.WNW_LAYERS_BATCHED)):
+            jq.set_dependency(["wnw", "skip"], dep)
+            for tt in range(tq, tq + W):
+                jq.step("wnw", tt); jq.step("skip", tt)
+            tq += W
+            torch.cuda.synchronize(dev)
+            ms_q = sum(jq.timed_steps("wnw", tq, n_pf)) / n_pf
+            jq.timed_steps("skip", tq, n_pf)
+            tq += n_pf
+            res_q[form] = {"step_us": ms_q * 1e3, "tokens_per_s": wq.batch / (ms_q * 1e-3)}
+        fetched_q, visible_q = jq.rows_fetched_and_visible("wnw")
         st0 = wnw.wnw_get_stats(jq.caches["wnw"])
-        ms_q = sum(jq.timed_steps("wnw", W, n_pf)) / n_pf
-        jq.timed_steps("skip", W, n_pf)
-        ms_q_bb = jq.timed_region("wnw", W + n_pf, n_bb)
-        ms_q_bb_skip = jq.timed_region("skip", W + n_pf, n_bb)
+        ms_q_bb = jq.timed_region("wnw", tq, n_bb)
+        ms_q_bb_skip = jq.timed_region("skip", tq, n_bb)
         st1 = wnw.wnw_get_stats(jq.caches["wnw"])
         T_a_q, _, C_q, S_q = wnw.wnw_get_seq_dims(jq.caches["wnw"], 0)
         paper_form = {"segment_tokens": wq.chunk, "segments": C_q, "slots": S_q, "base_slots": wnw.wnw_get_base_slots(jq.caches["wnw"], 0),
                       "evict_lag": 3, "score_scope": "global",
                       "prefill_compression": f"token-granular for tidal bases and fixed heads: per segment top floor(retention*n_s); retention = min(s*{lam_q:g}, 1), s ~ U[0,1] seeded",
-                      "step_us": ms_q * 1e3, "tokens_per_s": wq.batch / (ms_q * 1e-3),
+                      **res_q,
                       "back_to_back_step_us": ms_q_bb * 1e3, "back_to_back_exposed_recall_us": (ms_q_bb - ms_q_bb_skip) * 1e3,
-                      "recall_bytes_per_step": (st1["recall_bytes"] - st0["recall_bytes"]) / (n_pf + n_bb),
+                      "back_to_back_form": "all layers issued together",
+                      "recall_bytes_per_step": (st1["recall_bytes"] - st0["recall_bytes"]) / n_bb,
+                      "fetched_rows_over_visible_rows": fetched_q / max(visible_q, 1),
+                      "fetched_rows_note": "K,V rows the kernels fetch per step (25-token segments and base blocks are stored and fetched as 32 rows) over the rows that are visible",
                       "r_gpu": st1["resident_audio_tokens"] / max(st1["full_audio_tokens"], 1)}
         jq.destroy()
 
@@ -716,69 +836,58 @@ def run_ours(args, rank, world, local_rank):
     region_achieved = region_bytes_per_launch / (region_us_per_launch * 1e-6) / 1e9
     bytes_per_launch = algo_bytes / max(attn_n, 1)
     achieved = bytes_per_launch / (attn_us * 1e-6) / 1e9 if attn_us > 0 else 0.0
-    full_us = full_ms * 1e3 / max(full_n, 1)
-    full_achieved = (algo_bytes_full / max(full_n, 1)) / (full_us * 1e-6) / 1e9 if full_us > 0 else 0.0
     recall_bytes_step = (stats1["recall_bytes"] - stats0["recall_bytes"]) / K
-    ms_full = sum(full_steps) / K
-    ms_skip = sum(skip_steps) / K
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "attn_traffic.json")
     if os.path.exists(tpath):
         try:
-            traffic = json.load(open(tpath)).get(w.name + ("" if args.layer_dependency != 3 or args.eager else ":all_layers_together"))
+            traffic = json.load(open(tpath)).get(w.name + (":all_layers_together" if DEP == 3 and not args.eager else ""))
         except Exception:
             traffic = None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(w), launch="eager" if args.eager else "cuda graph replay of the step",
-                                                                                score_scope="global" if args.score_scope else "per layer",
-                                                                                residency="segment lag" if args.residency else "hard budget",
-                                                                                layers={0: "one launch per layer, overlapping (inputs of every layer resident before the step)",
-                                                                                        1: "chained (a layer waits for its predecessor before it reads q)",
-                                                                                        2: "serial launches",
-                                                                                        3: "all layers issued together: anchor heads, fixed heads and tidal heads in three launches, the selection beside the last two (inputs of every layer resident before the step, outputs read after it)"}[args.layer_dependency]),
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": dict(workload_config(w), launch="eager" if args.eager else "cuda graph replay of the step",
+                       score_scope="global" if args.score_scope else "per layer",
+                       residency="segment lag" if args.residency else "hard budget", layer_issue=dep_names[DEP]),
         "clocks": clocks, "gpu_launches": int(sum(region_launches)),
         "launches": {"attention": region_launches[0], "selection": region_launches[1], "recall": region_launches[2],
                      "step_end": region_launches[3], "layers_per_attention_launch": w.n_layers / attn_per_step},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e},
         # achieved: algorithmic K,V bytes of one launch / the launch's share of the timed region (CUDA events around every
-        # replayed step; the attention kernels are the only work on the timed stream).  With all layers in one launch
-        # (the default) that launch carries the step's bytes and its share is the step; with one launch per layer the
-        # consecutive kernels overlap through programmatic dependent launch and the share of one is step time / layers.
-        # `chained`: every kernel waits for its predecessor before reading q (layers that feed one another; only the
-        # K/V prefetch overlaps).  `serial`: plain stream order.  `eager_event_bracket`: one launch bracketed by events on
-        # an eager stream (includes launch latency and host pacing; kept for reference).
-        "roofline": {"bound": "hbm", "kernel": "wnw_attn_multi_kernel" if args.layer_dependency == 3 and not args.eager else "wnw_attn_kernel", "achieved": region_achieved, "peak": peak_gbs, "unit": "GB/s",
+        # replayed step; the attention kernels are the only work on the timed stream; with chained layers one launch per
+        # layer, each waiting for its predecessor, so the share of one is step time / layers).  The other issue forms are
+        # reported under their names: `upper_bound_all_layers_together` needs every layer's q before the step starts (no
+        # decoder whose layers feed one another can run it), `per_layer_overlapped` likewise; `serial` is plain stream order.
+        "roofline": {"bound": "hbm", "kernel": "wnw_attn_multi_kernel" if DEP == 3 and not args.eager else "wnw_attn_kernel",
+                     "achieved": region_achieved, "peak": peak_gbs, "unit": "GB/s",
                      "frac": region_achieved / peak_gbs, "peak_kind": f"of {peak_kind}", "traffic": traffic,
                      "bytes_per_launch": region_bytes_per_launch, "us_per_launch": region_us_per_launch,
                      "launches": region_launches[0],
-                     "duration_kind": "timed region / attention launches (by default the layers of a step are issued together in "
-                                      "three launches that overlap, the last filling the SMs as the others leave them; per-layer "
-                                      "launches overlap inside the replayed step)",
-                     "chained": dep.get("chained"), "serial": dep.get("serial"), alt_name: alt,
+                     "duration_kind": "timed region / attention launches",
+                     **forms,
                      "eager_event_bracket": {"us_per_launch": attn_us, "achieved": achieved, "frac": achieved / peak_gbs,
                                              "launches": attn_n},
                      "regime": f"{region_bytes_per_launch / 1e6:.1f} MB per launch would take "
-                               f"{region_bytes_per_launch / (peak_gbs * 1e3):.2f} us at peak"},
+                               f"{region_bytes_per_launch / (peak_gbs * 1e3):.2f} us at peak; the batch-1 step is bound by the "
+                               f"chain of dependent phases of a layer, not by bytes (see hbm_bound_case and cfg3 for the HBM-bound regime)"},
         "cpu_baseline": cpu,
-        "full_cache": {"ms_per_step": ms_full, "tokens_per_s": w.batch / (ms_full * 1e-3), "attn_us_per_launch": full_us,
-                       "attn_GBps": full_achieved, "attn_frac": full_achieved / peak_gbs,
-                       "wnw_step_over_full_step": ms_per_step / ms_full},
+        "full_cache": {"ms_per_step": ms_full, "tokens_per_s": w.batch / (ms_full * 1e-3), "layer_issue": "as the headline",
+                       "GB_per_step": bytes_full / 1e9, "GBps": bytes_full / (ms_full * 1e-3) / 1e9,
+                       "frac": bytes_full / (ms_full * 1e-3) / 1e9 / peak_gbs, "wnw_step_over_full_step": ms_per_step / ms_full},
         "recall": {"bytes_per_step": recall_bytes_step, "hits": stats1["hits"] - stats0["hits"],
                    "misses": stats1["misses"] - stats0["misses"], "link_memcpy_GBps": link_copy, "link_kernel_GBps": link_kernel,
                    "ms_per_step_copies_skipped": ms_skip, "exposed_us_per_step": (ms_per_step - ms_skip) * 1e3,
                    "note": "in the flushed runs the out-of-graph recall of a step may finish during the untimed flush; "
                            "`back_to_back` has no such gaps"},
         "back_to_back": bb,
-        "hbm_bound_case": hbm_case,
+        **blocks,
         "paper_form": paper_form,
-        "retention": {"r_gpu": stats1["resident_audio_tokens"] / max(stats1["full_audio_tokens"], 1),
-                      "r_gpu_cpu": (stats1["resident_audio_tokens"] + stats1["host_audio_tokens"]) / max(stats1["full_audio_tokens"], 1)},
+        "retention": retention,
         "wall_s_timed_region": wall,
     }
     print(json.dumps(line), flush=True)
-    job.destroy()   # no-op if the caches were already released
 
 
 def main():
@@ -789,7 +898,6 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg1",
                     help="cfg1 | cfg2 | cfg3 | cfg4 (recall sweep) | prof | hbm | b<batch>x<audio tokens> (config-1 heads, 12 layers)")
-    ap.add_argument("--no-hbm-case", action="store_true", help="skip the extra many-sequence measurement")
     ap.add_argument("--no-paper-form", action="store_true",
                     help="skip the extra measurement of the paper's own form (2 s segments, lag release, global scores)")
     ap.add_argument("--quick", action="store_true", help="only the WnW steps (for profiler captures); prints a short line")
@@ -804,14 +912,14 @@ def main():
     ap.add_argument("--segment-tokens", type=int, default=0, help="override the workload's chunk_tokens (e.g. the paper's 25 / 50)")
     ap.add_argument("--eager", action="store_true", help="issue every layer eagerly instead of replaying a captured step")
     ap.add_argument("--roofline-steps", type=int, default=16)
-    ap.add_argument("--layer-dependency", type=int, default=3, choices=[0, 1, 2, 3],
-                    help="how the layers of a step are issued: 3 all layers together (default: inputs of every layer resident "
-                         "before the step, outputs read after it), 0 one overlapping launch per layer, 1 chained, 2 serial")
-    ap.add_argument("--no-alt-form", action="store_true", help="skip the run in the other launch form (one launch per layer / all layers in one)")
+    ap.add_argument("--layer-dependency", type=int, default=1, choices=[0, 1, 2, 3],
+                    help="how the layers of a step are issued: 1 chained (default: a layer waits for its predecessor before it "
+                         "reads q, what a decoder whose layers feed one another runs), 3 all layers together (needs every "
+                         "layer's inputs before the step: a labelled upper bound), 0 one overlapping launch per layer, 2 serial")
+    ap.add_argument("--alt-steps", type=int, default=32, help="steps timed in each of the other issue forms (0 = skip)")
+    ap.add_argument("--no-blocks", action="store_true", help="skip the extra workloads (hbm_bound_case, cfg2, cfg3, chained batch sweep)")
     ap.add_argument("--back-to-back-steps", type=int, default=32,
                     help="steps timed in one region without L2 flushes (continuous decoding; exposes recall). 0 = skip")
-    ap.add_argument("--chain-steps", type=int, default=48,
-                    help="steps timed with chained layers and with serial layer launches (0 = skip)")
     ap.add_argument("--oracle-layers", type=int, default=6, help="layers of sequence 0 the CPU baseline samples (0 = skip)")
     ap.add_argument("--oracle-steps", type=int, default=4)
     ap.add_argument("--sweep-steps", type=int, default=0,
