@@ -60,6 +60,16 @@
  *     positions | all positions of the segments resident in the layer's dynamic slots]; a selected segment that is
  *     not in a dynamic slot counts as a miss (its complement has to be fetched).
  *     Pinned in tests/test_oracle_tokens.py against numpy sorts, a separate numpy softmax and hand-worked cases.
+ *   - streaming audio (wnwo_append_audio; the Limitations section names streaming as the method's setting, the Method
+ *     section does not say how a growing clip enters the tiers, so this is a reading): new audio positions extend the
+ *     clip; the short last chunk fills up first, then new chunks begin.  Anchor heads see every new position at once.
+ *     Tidal heads see a new position only through the residency table: new positions of a chunk that is resident are
+ *     visible with it, a new chunk is on the host until the anchor heads' scores select it; the slot count follows the
+ *     budget, S = max(1, floor(budget * C)) of the grown C, and the added slots start empty.  Fixed heads keep the
+ *     subset chosen at prefill, which is final (Method Overview: static subset, the rest is discarded): they never see
+ *     a position that arrived later, not even inside a chunk they keep.  Hard budget only.
+ *     Pinned in tests/test_oracle_streaming.py: appending in pieces equals placing the whole clip (anchor heads: exactly;
+ *     the full sets of every role against numpy attention over an explicit position mask), slot rule, table carry-over.
  */
 #include <math.h>
 #include <stdint.h>
@@ -78,6 +88,7 @@
 typedef struct {
   int placed_layers;   /* how many layers have been placed */
   int T_a, T_t, T_cap; /* audio tokens, current text tokens, text capacity */
+  int T_a_fixed;       /* audio tokens that had arrived when the sequence was placed: all a fixed head can ever see */
   int C, S;            /* chunks (segments in SEGMENT_LAG), slots of the tidal table */
   int S_base;          /* slots filled at prefill; = S with the hard budget; fixed heads keep S_base chunks */
   long long steps;     /* decode steps this sequence took part in */
@@ -342,6 +353,7 @@ int wnwo_score_source(const Oracle *o, int layer) { return (layer >= 0 && layer 
 static int alloc_seq(Oracle *o, Seq *s, int T_a, int T_t) {
   int L = o->L, Hkv = o->Hkv, d = o->d;
   s->T_a = T_a; s->T_t = T_t; s->T_cap = o->max_text;
+  s->T_a_fixed = T_a;
   s->C = (T_a + o->chunk - 1) / o->chunk;
   int S = (int)floor(o->budget * (double)s->C + 1e-6);
   if (S < 1) S = 1;
@@ -397,6 +409,7 @@ static void attend(const Oracle *o, const Seq *s, int layer, int kvh, const uint
    * its kept positions and every position of the segments resident in its layer's dynamic slots */
   const unsigned char *tok = s->tok_mask ? s->tok_mask[layer * o->Hkv + kvh] : NULL;
   const int tidal_base = o->roles[layer * o->Hkv + kvh] == ROLE_TIDAL;
+  const int fixed_head = o->roles[layer * o->Hkv + kvh] == ROLE_FIXED;   /* sees nothing that arrived after its placement */
   const int d = o->d, T_a = s->T_a;
   const uint16_t *tK = s->txtK[layer] + (size_t)kvh * s->T_cap * d, *tV = s->txtV[layer] + (size_t)kvh * s->T_cap * d;
   const uint16_t *aK = s->audK[layer] + (size_t)kvh * T_a * d, *aV = s->audV[layer] + (size_t)kvh * T_a * d;
@@ -407,7 +420,11 @@ static void attend(const Oracle *o, const Seq *s, int layer, int kvh, const uint
     const uint16_t *krow;
     int vis;
     if (i < T_t) { krow = tK + (size_t)i * d; vis = 1; }
-    else { int tau = i - T_t; krow = aK + (size_t)tau * d; vis = tok ? (tok[tau] != 0 || (tidal_base && allowed[tau / o->chunk] != 0)) : allowed[tau / o->chunk] != 0; }
+    else {
+      int tau = i - T_t; krow = aK + (size_t)tau * d;
+      vis = tok ? (tok[tau] != 0 || (tidal_base && allowed[tau / o->chunk] != 0)) : allowed[tau / o->chunk] != 0;
+      if (fixed_head && tau >= s->T_a_fixed) vis = 0;
+    }
     if (!vis) { logit[i] = -INFINITY; continue; }
     double acc = 0.0;
     for (int x = 0; x < d; ++x) acc += bf16_to_double(q[x]) * bf16_to_double(krow[x]);
@@ -655,6 +672,61 @@ int wnwo_set_fixed_tokens(Oracle *o, int seq, int layer, int kvh, const int *pos
 int wnwo_place_prefill(Oracle *o, int seq, int layer, const uint16_t *k, const uint16_t *v, int n_tokens,
                        int audio_begin, int audio_end, const uint16_t *q_last) {
   return wnwo_place_prefill_multi(o, seq, layer, k, v, n_tokens, audio_begin, audio_end, q_last, 1);
+}
+
+/* ------------------------------------------------------------------ */
+/* Streaming audio: the clip grows between decode steps                 */
+/* ------------------------------------------------------------------ */
+/* k, v: [L][n][Hkv][d] bf16 bits, the n new audio positions of every layer.  See the header for the reading. */
+int wnwo_append_audio(Oracle *o, int seq, const uint16_t *k, const uint16_t *v, int n) {
+  if (!o || seq < 0 || seq >= o->max_batch || n < 0 || (n > 0 && (!k || !v))) return WNWO_ERR_ARG;
+  Seq *s = &o->seq[seq];
+  if (o->in_step || s->placed_layers != o->L || o->residency != 0) return WNWO_ERR_STATE;
+  if (s->T_a + n > o->max_audio) return WNWO_ERR_ARG;
+  if (n == 0) return WNWO_OK;
+  const int L = o->L, Hkv = o->Hkv, d = o->d;
+  Seq old = *s, ns;
+  memset(&ns, 0, sizeof(ns));
+  int rc = alloc_seq(o, &ns, old.T_a + n, old.T_t);   /* the grown clip: C, and S by the slot rule */
+  if (rc) { free_seq(o, &ns); return rc; }
+  ns.placed_layers = L; ns.T_a_fixed = old.T_a_fixed; ns.steps = old.steps;
+  ns.hits = old.hits; ns.misses = old.misses; ns.evictions = old.evictions;
+  for (int l = 0; l < L; ++l) {
+    memcpy(ns.txtK[l], old.txtK[l], (size_t)Hkv * old.T_cap * d * 2);
+    memcpy(ns.txtV[l], old.txtV[l], (size_t)Hkv * old.T_cap * d * 2);
+    for (int h = 0; h < Hkv; ++h) {
+      uint16_t *dk = ns.audK[l] + (size_t)h * ns.T_a * d, *dv = ns.audV[l] + (size_t)h * ns.T_a * d;
+      memcpy(dk, old.audK[l] + (size_t)h * old.T_a * d, (size_t)old.T_a * d * 2);
+      memcpy(dv, old.audV[l] + (size_t)h * old.T_a * d, (size_t)old.T_a * d * 2);
+      for (int i = 0; i < n; ++i) {
+        const size_t src = (((size_t)l * n + i) * Hkv + h) * d;
+        memcpy(dk + (size_t)(old.T_a + i) * d, k + src, (size_t)d * 2);
+        memcpy(dv + (size_t)(old.T_a + i) * d, v + src, (size_t)d * 2);
+      }
+    }
+    /* tables carry over; the slots the grown budget adds start empty (alloc_seq left them at -1, stamp 0) */
+    for (int j = 0; j < old.S; ++j) {
+      ns.slot_chunk[(size_t)l * ns.S + j] = old.slot_chunk[(size_t)l * old.S + j];
+      ns.stamp[(size_t)l * ns.S + j] = old.stamp[(size_t)l * old.S + j];
+    }
+    for (int h = 0; h < Hkv; ++h) {   /* fixed sets are final */
+      const int lh = l * Hkv + h;
+      ns.fixed_n[lh] = old.fixed_n[lh];
+      for (int j = 0; j < old.fixed_n[lh]; ++j) ns.fixed_set[(size_t)lh * ns.S + j] = old.fixed_set[(size_t)lh * old.S + j];
+      for (int c = 0; c < old.C; ++c) ns.pre[(size_t)lh * ns.C + c] = old.pre[(size_t)lh * old.C + c];
+      if (old.tok_mask && old.tok_mask[lh]) {   /* a head placed token by token keeps its positions; later ones are not kept */
+        ns.tok_mask[lh] = (unsigned char *)calloc((size_t)ns.T_a, 1);
+        if (!ns.tok_mask[lh]) { free_seq(o, &ns); return WNWO_ERR_OOM; }
+        memcpy(ns.tok_mask[lh], old.tok_mask[lh], (size_t)old.T_a);
+      }
+    }
+    for (int c = 0; c < old.C; ++c) ns.score_sum[(size_t)l * ns.C + c] = old.score_sum[(size_t)l * old.C + c];
+    for (int r = 0; r < o->topk; ++r) ns.sel[(size_t)l * o->topk + r] = old.sel[(size_t)l * o->topk + r];
+    ns.n_sel[l] = old.n_sel[l];
+  }
+  free_seq(o, &old);
+  *s = ns;
+  return WNWO_OK;
 }
 
 /* ------------------------------------------------------------------ */

@@ -50,6 +50,7 @@ def lib():
                                             C.c_int, C.c_int, C.c_int, C.POINTER(C.c_uint16)]
         _lib.wnwo_place_prefill_multi.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_uint16), C.POINTER(C.c_uint16),
                                                   C.c_int, C.c_int, C.c_int, C.POINTER(C.c_uint16), C.c_int]
+        _lib.wnwo_append_audio.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_uint16), C.POINTER(C.c_uint16), C.c_int]
         _lib.wnwo_step_begin.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.c_int]
         _lib.wnwo_decode_layer.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_uint16), C.POINTER(C.c_uint16),
                                            C.POINTER(C.c_uint16), C.POINTER(C.c_double)]
@@ -236,6 +237,12 @@ class Oracle:
     def set_fixed_tokens(self, seq, layer, kv_head, pos):
         a = np.ascontiguousarray(pos, np.int32)
         _check(lib().wnwo_set_fixed_tokens(self._h, seq, layer, kv_head, _p(a, C.c_int), len(a)), "set_fixed_tokens")
+
+    def append_audio(self, seq, k_bits, v_bits):
+        """The clip of `seq` grows by n audio positions: k_bits, v_bits [n_layers, n, n_kv_heads, head_dim] (every layer)."""
+        k, v = _u16(k_bits), _u16(v_bits)
+        assert k.shape == v.shape and k.shape[0] == self.L and k.shape[2:] == (self.Hkv, self.d), k.shape
+        _check(lib().wnwo_append_audio(self._h, seq, _p(k, C.c_uint16), _p(v, C.c_uint16), k.shape[1]), "append_audio")
 
     def step_begin(self, active: Sequence[int]):
         a = np.ascontiguousarray(active, dtype=np.int32)
