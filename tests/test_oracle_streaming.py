@@ -181,3 +181,29 @@ def test_append_is_refused_inside_a_step_and_beyond_capacity():
     clip.append(o, 32, 64)
     with pytest.raises(OracleError):        # the cache was created for 64 audio tokens
         o.append_audio(0, np.zeros((1, 1, 2, 64), np.uint16), np.zeros((1, 1, 2, 64), np.uint16))
+
+
+def test_a_fixed_head_that_keeps_the_short_last_chunk_does_not_see_it_grow():
+    """Budget 1.0: the fixed head keeps every chunk that existed at placement, the short last one included.  When that
+    chunk fills up and new chunks follow, the fixed head still attends to exactly the positions that had arrived at
+    placement, while the tidal head of the same layer (all of its chunks resident, new slots empty) sees the old chunks
+    grown and the anchor head everything."""
+    w = tiny_custom(n_layers=1, n_q_heads=3, n_kv_heads=3, head_dim=64, n_text=4, audio_lens=(100,), chunk=16, budget=1.0,
+                    n_steps=3, roles=[[A, T, F]])
+    clip = Clip(w, seed=4)
+    o = _oracle(w)
+    T0 = 37                                   # chunks 0, 1 full, chunk 2 holds 5 tokens
+    clip.place(o, T0)
+    assert sorted(o.fixed_set(0, 0, 2).tolist()) == [0, 1, 2]
+    clip.append(o, T0, 100)
+    tab = o.residency(0, 0)[0]
+    assert sorted(tab[tab >= 0].tolist()) == [0, 1, 2] and o.dims(0)[3] == 7
+    outs = clip.step(o, 0)
+    scale = 1 / math.sqrt(w.head_dim)
+    for h, upto in ((0, 100), (1, 48), (2, T0)):       # anchor: all; tidal: chunks 0-2 as they are now; fixed: as they were
+        K = np.concatenate([bf16_bits_to_f64(clip.k[0][:w.n_text, h]), bf16_bits_to_f64(bf16_bits(clip.dec[0]["k_new"][0][h]))[None],
+                            bf16_bits_to_f64(clip.k[0][w.n_text:w.n_text + upto, h])])
+        V = np.concatenate([bf16_bits_to_f64(clip.v[0][:w.n_text, h]), bf16_bits_to_f64(bf16_bits(clip.dec[0]["v_new"][0][h]))[None],
+                            bf16_bits_to_f64(clip.v[0][w.n_text:w.n_text + upto, h])])
+        ref, _ = dense_attention(bf16_bits_to_f64(bf16_bits(clip.dec[0]["q"][0])[h]), K, V, scale)
+        assert np.abs(outs[0][h] - ref).max() < 1e-12, h
