@@ -115,6 +115,9 @@ typedef struct {
   int32_t recall_mode;                     /* WNW_RECALL_* */
   int32_t score_scope;                     /* WNW_SCOPE_* */
   int32_t residency;                       /* WNW_RESIDENCY_* */
+  int32_t streaming_audio;                 /* 1: clips may grow after placement (wnw_append_audio): every sequence's pinned host
+                                            * mirror is sized and laid out for max_audio_tokens.  0: mirrors are sized by the
+                                            * placed clip and wnw_append_audio is refused */
 } wnw_config_t;
 
 typedef struct {
@@ -196,6 +199,25 @@ wnw_status_t wnw_get_token_scores(wnw_cache_t *cache, int32_t seq, int32_t layer
                                   int32_t capacity);
 wnw_status_t wnw_get_fixed_tokens(wnw_cache_t *cache, int32_t seq, int32_t layer, int32_t kv_head, int32_t *positions,
                                   int32_t capacity, int32_t *n);
+
+/* Streaming audio: the clip of a placed sequence grows by n_tokens audio positions between decode steps (the
+ * Limitations section names streaming as the method's setting; how a growing clip enters the tiers is a reading, stated
+ * here).  k_dev, v_dev: [n_tokens][n_kv_heads][head_dim] bf16, the new positions of one layer.  The short last chunk fills
+ * up first, then new chunks begin.
+ *   anchor heads  keep every new position on the GPU and attend to it from the next step on;
+ *   tidal heads   get the new positions in their host mirror; a position that belongs to a chunk resident in the slot
+ *                 pool is written to the slot as well (a resident chunk is seen grown), a new chunk stays on the host
+ *                 until the anchor heads' scores select it.  The slot count follows the budget on the grown clip,
+ *                 S = max(1, floor(budget * C)); the added slots start empty;
+ *   fixed heads   keep the subset chosen at placement, which is final: they never see a position that arrived later,
+ *                 not even inside a chunk they keep.
+ * Layers must be given in order 0..n_layers-1, all with the same n_tokens, outside a step; the grown clip is in force
+ * once the last layer has been appended (wnw_step_begin is refused in between).  The first layer's call waits for all
+ * queued work of the cache.  Work lists are rebuilt by the next step and a captured step must be captured again.
+ * Needs streaming_audio = 1 at creation and the HARD_BUDGET residency (or FULL mode, where every head is stored in
+ * full): WNW_ERR_UNSUPPORTED otherwise; WNW_ERR_CAPACITY beyond max_audio_tokens; WNW_ERR_STATE out of order. */
+wnw_status_t wnw_append_audio(wnw_cache_t *cache, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                              int32_t n_tokens, void *cuda_stream);
 
 /* Open a decode step for the given sequences (HOST array of distinct sequence ids, all fully placed).
  * The order of active_seqs_host is the batch order of q/k_new/v_new/out in wnw_decode_layer. */

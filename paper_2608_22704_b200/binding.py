@@ -30,7 +30,7 @@ class wnw_config_t(C.Structure):
                 ("max_batch", C.c_int32), ("max_audio_tokens", C.c_int32), ("max_text_tokens", C.c_int32),
                 ("chunk_tokens", C.c_int32), ("topk", C.c_int32), ("evict_lag", C.c_int32), ("budget", C.c_float),
                 ("softmax_scale", C.c_float), ("roles", C.POINTER(C.c_uint8)), ("device", C.c_int32), ("mode", C.c_int32),
-                ("recall_mode", C.c_int32), ("score_scope", C.c_int32), ("residency", C.c_int32)]
+                ("recall_mode", C.c_int32), ("score_scope", C.c_int32), ("residency", C.c_int32), ("streaming_audio", C.c_int32)]
 
 
 class wnw_stats_t(C.Structure):
@@ -52,6 +52,7 @@ _SIGNATURES = {
     "wnw_place_prefill": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _vp],
     "wnw_place_prefill_multi": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp],
     "wnw_place_prefill_tokens": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _i32, C.POINTER(C.c_float), _i32, _i32, _vp],
+    "wnw_append_audio": [_vp, _i32, _i32, _vp, _vp, _i32, _vp],
     "wnw_retention_schedule": [C.POINTER(C.c_float), _i32, C.c_float, C.POINTER(C.c_float)],
     "wnw_get_token_scores": [_vp, _i32, _i32, _i32, C.POINTER(C.c_float), _i32],
     "wnw_get_fixed_tokens": [_vp, _i32, _i32, _i32, C.POINTER(_i32), _i32, C.POINTER(_i32)],
@@ -133,11 +134,13 @@ def _stream(stream) -> Optional[int]:
 
 def wnw_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens, chunk_tokens,
                budget, roles, topk=3, evict_lag=3, softmax_scale=0.0, device=0, mode=WNW_MODE_TIERED,
-               recall_mode=WNW_RECALL_SIDE_STREAM, score_scope=WNW_SCOPE_PER_LAYER, residency=WNW_RESIDENCY_HARD_BUDGET) -> int:
+               recall_mode=WNW_RECALL_SIDE_STREAM, score_scope=WNW_SCOPE_PER_LAYER, residency=WNW_RESIDENCY_HARD_BUDGET,
+               streaming_audio=0) -> int:
     roles = np.ascontiguousarray(roles, dtype=np.uint8).reshape(-1)
     cfg = wnw_config_t(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
                        chunk_tokens, topk, evict_lag, budget, softmax_scale,
-                       roles.ctypes.data_as(C.POINTER(C.c_uint8)), device, mode, recall_mode, score_scope, residency)
+                       roles.ctypes.data_as(C.POINTER(C.c_uint8)), device, mode, recall_mode, score_scope, residency,
+                       int(streaming_audio))
     if roles.size != n_layers * n_kv_heads:
         raise WnwError(WNW_ERR_INVALID_ARG, "wnw_create (roles size)")
     h = _vp()
@@ -155,6 +158,11 @@ def wnw_place_prefill(cache, seq, layer, k, v, audio_begin, audio_end, q_last=No
         return wnw_place_prefill_multi(cache, seq, layer, k, v, audio_begin, audio_end, q_last, stream)
     _ck(lib().wnw_place_prefill(cache, seq, layer, _ptr(k), _ptr(v), k.shape[0], audio_begin, audio_end, _ptr(q_last),
                                 _stream(stream)), "wnw_place_prefill")
+
+
+def wnw_append_audio(cache, seq, layer, k, v, stream=None):
+    """k, v: [n_tokens, n_kv_heads, head_dim] bf16 CUDA tensors, the new audio positions of one layer."""
+    _ck(lib().wnw_append_audio(cache, seq, layer, _ptr(k), _ptr(v), k.shape[0], _stream(stream)), "wnw_append_audio")
 
 
 def wnw_place_prefill_multi(cache, seq, layer, k, v, audio_begin, audio_end, q_text, stream=None):

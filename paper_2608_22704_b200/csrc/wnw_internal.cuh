@@ -61,6 +61,7 @@ struct Geometry {
   int32_t token_base;              // SEGMENT_LAG with a token-granular permanent base (no permanent slots)
   int32_t lag_mode, delta, plan_cap;  // SEGMENT_LAG residency; its eviction lag; plan entries per (sequence, layer)
   int32_t max_batch;
+  int32_t mirror_chunks;           // chunks a host mirror is laid out for: 0 = those of the placed clip, else the capacity (streaming audio)
   long long text_seq_stride, anchor_seq_stride, pool_seq_stride, fixed_seq_stride;  // elements
   float scale_log2;                // softmax scale * log2(e)
 };
@@ -119,6 +120,8 @@ __host__ __device__ inline long long slot_table_off(const Geometry &G, int parit
 __host__ __device__ inline long long compact_off(const Geometry &G, int b, int head, int kv) {
   return (long long)b * G.fixed_seq_stride + ((long long)head * 2 + kv) * G.FB * G.ncp * G.d;
 }
+// C_b: the chunks the sequence's mirror is laid out for (mirror_chunks_of)
+__host__ __device__ inline int mirror_chunks_of(const Geometry &G, int C_b) { return G.mirror_chunks ? G.mirror_chunks : C_b; }
 __host__ __device__ inline long long mirror_off(const Geometry &G, const LayerInfo &li, int C_b, int c, int t_idx, int kv) {
   return (((long long)C_b * li.tid_prefix + (long long)c * li.n_tidal + t_idx) * 2 + kv) * G.ncp * G.d;
 }
@@ -248,6 +251,8 @@ cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_c
                                   const bf16 *q_text, int n_q, int T_t, int T_a, int seg, const float *retention_dev,
                                   int variant, float *work, float *p_tok, int32_t *flags, long long p_stride,
                                   int32_t *fixed_tok, int tok_cap, int32_t *tok_n, cudaStream_t st);
+cudaError_t launch_append_audio(const CacheView &cv, int b, int layer, int full_mode, const bf16 *k, const bf16 *v, int n_tokens,
+                                int T_a_old, int S_old, int set_dims, int T_a_new, int C_new, int S_new, cudaStream_t st);
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
 cudaError_t configure_attn_kernels();
 // the CTAs of several layers' launches (one-shot variant) in one launch

@@ -346,7 +346,7 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
           if (threadIdx.x == 0) atomicOr(cv.status, STATUS_BAD_TABLE);
           continue;
         }
-        const uint4 *src = reinterpret_cast<const uint4 *>(cv.mirror[b] + mirror_off(G, li, cv.C[b], c, 0, 0));
+        const uint4 *src = reinterpret_cast<const uint4 *>(cv.mirror[b] + mirror_off(G, li, mirror_chunks_of(G, cv.C[b]), c, 0, 0));
         uint4 *dst = reinterpret_cast<uint4 *>(cv.pool + pool_off(G, li, b, slot, 0, 0));
         for (int v0 = rank * blockDim.x + threadIdx.x; v0 < n; v0 += stride * U) {
           uint4 t[U];
@@ -420,6 +420,46 @@ __global__ void __launch_bounds__(256) wnw_copy_kernel(const uint4 *__restrict__
 }
 cudaError_t launch_copy_plan(const uint4 *src, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st) {
   wnw_copy_kernel<<<n_ctas, 256, 0, st>>>(src, dst, n_vec);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Streaming audio: new positions of one layer go to the tiers their heads keep
+// ------------------------------------------------------------------------------------------------
+// grid (new token, KV head), one thread per 16-byte piece of the K row and of the V row.  Anchor-like heads: the full-audio
+// store.  Tidal heads: the host mirror (mapped pinned memory, written from the device) and, if the position's chunk is
+// resident, its slot.  Fixed heads: nothing (their subset is final).  The tables need no growth: placement left every
+// slot and every chunk entry up to the capacity empty.  The last layer's launch puts the grown dimensions in force.
+__global__ void wnw_append_audio_kernel(const __grid_constant__ CacheView cv, int b, int layer, int full_mode, const bf16 *k,
+                                        const bf16 *v, int T_a_old, int S_old, int set_dims, int T_a_new, int C_new, int S_new) {
+  const Geometry &G = cv.geo;
+  const int ppr = G.d / 8, kv = threadIdx.x / ppr, pc = threadIdx.x - kv * ppr;
+  const int tok = blockIdx.x, h = blockIdx.y, tau = T_a_old + tok, ci = tau / G.nc, off = tau - ci * G.nc;
+  if (set_dims && tok == 0 && h == 0 && threadIdx.x == 0) { cv.T_a[b] = T_a_new; cv.C[b] = C_new; cv.S[b] = S_new; cv.S_base[b] = S_new; }
+  if (kv >= 2) return;
+  const uint4 val = *reinterpret_cast<const uint4 *>((kv ? v : k) + ((long long)tok * G.Hkv + h) * G.d + pc * 8);
+  const int role = full_mode ? ROLE_ANCHOR : cv.roles[layer * G.Hkv + h];
+  const LayerInfo li = cv.layers[layer];
+  if (role == ROLE_ANCHOR) {
+    const int head = full_mode ? layer * G.Hkv + h : li.anchor_off + cv.role_idx[layer * G.Hkv + h];
+    *reinterpret_cast<uint4 *>(cv.anchor + anchor_off(G, G.anchor_seq_stride, b, head, kv) + (long long)(ci * G.ncp + off) * G.d + pc * 8) = val;
+  } else if (role == ROLE_TIDAL) {
+    const int ridx = cv.role_idx[layer * G.Hkv + h];
+    *reinterpret_cast<uint4 *>(cv.mirror[b] + mirror_off(G, li, mirror_chunks_of(G, C_new), ci, ridx, kv) + (long long)off * G.d + pc * 8) = val;
+    const long long bl = (long long)b * G.L + layer;
+    const int32_t *tab = cv.slot_chunk + slot_table_off(G, (int)(cv.steps[b] & 1), bl);   // the table the next step reads
+    for (int j = 0; j < S_old; ++j)
+      if (tab[j] == ci) {
+        *reinterpret_cast<uint4 *>(cv.pool + pool_off(G, li, b, j, ridx, kv) + (long long)off * G.d + pc * 8) = val;
+        break;
+      }
+  }
+}
+cudaError_t launch_append_audio(const CacheView &cv, int b, int layer, int full_mode, const bf16 *k, const bf16 *v, int n_tokens,
+                                int T_a_old, int S_old, int set_dims, int T_a_new, int C_new, int S_new, cudaStream_t st) {
+  const int threads = (2 * cv.geo.d / 8 + 31) / 32 * 32;
+  wnw_append_audio_kernel<<<dim3((unsigned)n_tokens, (unsigned)cv.geo.Hkv), threads, 0, st>>>(cv, b, layer, full_mode, k, v, T_a_old, S_old,
+                                                                                            set_dims, T_a_new, C_new, S_new);
   return cudaGetLastError();
 }
 
@@ -611,7 +651,7 @@ __global__ void __launch_bounds__(128) wnw_place_gather_kernel(const __grid_cons
   } else {
     const int slot = cv.chunk_slot[bl * G.C_max + c];
     for (int kv = 0; kv < 2; ++kv) {
-      dst0[kv] = cv.mirror[b] + mirror_off(G, li, cv.C[b], c, ridx, kv);
+      dst0[kv] = cv.mirror[b] + mirror_off(G, li, mirror_chunks_of(G, cv.C[b]), c, ridx, kv);
       if (slot >= 0) dst1[kv] = cv.pool + pool_off(G, li, b, slot, ridx, kv);
     }
   }

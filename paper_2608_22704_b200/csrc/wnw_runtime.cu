@@ -19,6 +19,8 @@ namespace {
 struct SeqHost {
   int placed_layers = 0;
   int T_a = 0, T_t = 0, C = 0, S = 0, S_base = 0;   // S: all slots of a tidal table; S_base: the permanent ones
+  int T_a_fixed = 0, S_fixed = 0;   // the clip and the slot count at placement: what a fixed head keeps for good (streaming audio)
+  int append_layer = 0, append_n = 0;   // an append of audio in progress: layers done, positions per layer
   bf16 *mirror = nullptr;
   size_t mirror_bytes = 0;
   std::vector<int> fixed_blocks;   // [L][Hkv] blocks of a token-compacted head's store; empty or -1: S_base chunks
@@ -265,7 +267,7 @@ static wnw_status_t validate_config(const wnw_config_t *cfg) {
   if (cfg->score_scope != WNW_SCOPE_PER_LAYER && cfg->score_scope != WNW_SCOPE_GLOBAL) return WNW_ERR_INVALID_ARG;
   if (cfg->residency < WNW_RESIDENCY_HARD_BUDGET || cfg->residency > WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE) return WNW_ERR_INVALID_ARG;
   if (cfg->recall_mode < WNW_RECALL_SIDE_STREAM || cfg->recall_mode > WNW_RECALL_SKIP) return WNW_ERR_INVALID_ARG;
-  if (cfg->device < 0) return WNW_ERR_INVALID_ARG;
+  if (cfg->device < 0 || cfg->streaming_audio < 0 || cfg->streaming_audio > 1) return WNW_ERR_INVALID_ARG;
   bool any_anchor = false, any_tidal = false;
   for (int i = 0; i < cfg->n_layers * cfg->n_kv_heads; ++i) {
     if (cfg->roles[i] > WNW_ROLE_FIXED) return WNW_ERR_INVALID_ARG;
@@ -323,6 +325,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   G.plan_cap = G.lag_mode ? 2 * G.topk : G.topk;
   G.T_a_pad = std::max(G.C_max, 1) * G.ncp;
   G.max_batch = cfg->max_batch;
+  G.mirror_chunks = (!full && cfg->streaming_audio) ? G.C_max : 0;
   const double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / std::sqrt((double)d);
   G.scale_log2 = (float)(scale * 1.4426950408889634);
   // roles -> per-layer tables, score routing, update lists
@@ -578,7 +581,7 @@ static int granules_per_item(const wnw_cache *c, long long total_granules, int l
 static void head_granules(const wnw_cache *c, int layer, int mode, const SeqHost &s, int h, int *n_gran, int *work) {
   const Geometry &G = c->geo;
   const int role = mode == ATTN_DECODE ? c->roles[layer * G.Hkv + h] : ROLE_ANCHOR;
-  int fixed_blocks = s.S_base;   // a token-compacted head: the blocks its kept positions fill
+  int fixed_blocks = s.S_fixed;  // what the head kept at placement; a token-compacted head: the blocks its kept positions fill
   if (!s.fixed_blocks.empty() && s.fixed_blocks[layer * G.Hkv + h] >= 0) fixed_blocks = s.fixed_blocks[layer * G.Hkv + h];
   // a tidal head with a token base: its blocks first, then the table's (all dynamic) slots
   const int tidal_units = s.S + (G.token_base && mode == ATTN_DECODE ? fixed_blocks : 0);
@@ -650,8 +653,8 @@ static void build_throughput_items(const wnw_cache *c, int layer, int mode, cons
     const HeadItems hi{(int)items.size() - lw.first_item, np};
     first_item[hd] = hi.first;
     for (int x = 0; x < np; ++x)
-      items.push_back(WorkItem{i, h, (int)((long long)n * x / np), (int)((long long)n * (x + 1) / np), seq_ids[i], role, ridx, sq.T_a,
-                               sq.C, perm, sq.T_t, hi.first, hi.count});
+      items.push_back(WorkItem{i, h, (int)((long long)n * x / np), (int)((long long)n * (x + 1) / np), seq_ids[i], role, ridx,
+                               role == ROLE_FIXED ? sq.T_a_fixed : sq.T_a, sq.C, perm, sq.T_t, hi.first, hi.count});
     heads.push_back(hi);
     lw.max_count = std::max(lw.max_count, np);
   }
@@ -731,7 +734,8 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
         // S: the head's leading permanent units: slots of the table, or blocks of a tidal head's token base
         const int perm = (G.token_base && role == ROLE_TIDAL && !sq.fixed_blocks.empty()) ? std::max(sq.fixed_blocks[layer * G.Hkv + h], 0)
                                                                                          : sq.S_base;
-        items.push_back(WorkItem{(int)i, h, g0, g1, seq_ids[i], role, ridx, sq.T_a, sq.C, perm, sq.T_t, hi.first, hi.count});
+        items.push_back(WorkItem{(int)i, h, g0, g1, seq_ids[i], role, ridx, role == ROLE_FIXED ? sq.T_a_fixed : sq.T_a, sq.C, perm, sq.T_t,
+                                  hi.first, hi.count});
       }
       heads.push_back(hi);
       lw.max_count = std::max(lw.max_count, hi.count);
@@ -918,7 +922,7 @@ static wnw_status_t place_multi(wnw_cache_t *c, int32_t seq, int32_t layer, cons
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (layer == 0) {
     s.placed_layers = 0;
-    const size_t need = full ? 0 : (size_t)C_b * c->tid_total * 2 * G.ncp * G.d * sizeof(bf16);
+    const size_t need = full ? 0 : (size_t)mirror_chunks_of(G, C_b) * c->tid_total * 2 * G.ncp * G.d * sizeof(bf16);
     if (need != s.mirror_bytes) {
       CK(cudaDeviceSynchronize());
       if (s.mirror) cudaFreeHost(s.mirror);
@@ -929,6 +933,7 @@ static wnw_status_t place_multi(wnw_cache_t *c, int32_t seq, int32_t layer, cons
           cudaGetLastError();
           return WNW_ERR_OOM_HOST;
         }
+        if (G.mirror_chunks) memset(p, 0, need);   // chunks that have not arrived yet must read as padding
         void *dp = nullptr;
         CK(cudaHostGetDevicePointer(&dp, p, 0));
         s.mirror = (bf16 *)p; s.mirror_bytes = need;
@@ -939,6 +944,7 @@ static wnw_status_t place_multi(wnw_cache_t *c, int32_t seq, int32_t layer, cons
       CK(cudaMemcpy(c->cv.mirror + seq, &c->mirror_ptrs[seq], sizeof(bf16 *), cudaMemcpyHostToDevice));
     }
     s.T_a = T_a; s.T_t = T_t; s.C = C_b; s.S = S_b; s.S_base = S_base_b;
+    s.T_a_fixed = T_a; s.S_fixed = S_base_b; s.append_layer = 0; s.append_n = 0;
     s.fixed_blocks.clear(); s.tok_m.clear();
     c->wl_layers.clear();  // dims may have changed
   }
@@ -1012,6 +1018,44 @@ static wnw_status_t place_multi(wnw_cache_t *c, int32_t seq, int32_t layer, cons
 
 static wnw_status_t check_seq_layer(wnw_cache *c, int seq, int layer);
 static wnw_status_t drain(wnw_cache *c);
+
+// Streaming audio: n_tokens new audio positions of one layer (layers in order; the grown clip takes effect with the last).
+extern "C" wnw_status_t wnw_append_audio(wnw_cache_t *c, int32_t seq, int32_t layer, const void *k_dev, const void *v_dev,
+                                         int32_t n_tokens, void *cuda_stream) {
+  if (!c || !k_dev || !v_dev || n_tokens < 1) return WNW_ERR_INVALID_ARG;
+  const Geometry &G = c->geo;
+  if (seq < 0 || seq >= G.max_batch || layer < 0 || layer >= G.L) return WNW_ERR_INVALID_ARG;
+  const bool full = c->cfg.mode == WNW_MODE_FULL;
+  if (!full && (!c->cfg.streaming_audio || c->cfg.residency != WNW_RESIDENCY_HARD_BUDGET)) return WNW_ERR_UNSUPPORTED;
+  if (c->in_step || c->graph_capturing) return WNW_ERR_STATE;
+  SeqHost &s = c->seqs[seq];
+  if (s.placed_layers != G.L || layer != s.append_layer || (layer > 0 && n_tokens != s.append_n)) return WNW_ERR_STATE;
+  if (s.T_a + n_tokens > c->cfg.max_audio_tokens) return WNW_ERR_CAPACITY;
+  if (!s.fixed_blocks.empty()) return WNW_ERR_UNSUPPORTED;   // heads compacted token by token have no chunk geometry to grow
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (layer == 0) {   // selections and recalls of earlier steps read and write the tables and slots this touches
+    wnw_status_t ds = drain(c);
+    if (ds != WNW_OK) return ds;
+    CK(cudaStreamSynchronize(st));
+    s.append_n = n_tokens;
+  }
+  const int T_new = s.T_a + n_tokens, C_new = (T_new + G.nc - 1) / G.nc;
+  const int S_new = full ? 0 : slots_total(c->cfg, C_new);
+  const bool last = layer == G.L - 1;
+  CK(launch_append_audio(c->cv, seq, layer, full ? 1 : 0, (const bf16 *)k_dev, (const bf16 *)v_dev, n_tokens, s.T_a, s.S, last ? 1 : 0,
+                         T_new, C_new, S_new, st));
+  CK(cudaEventRecord(c->ev_place, st));
+  c->place_recorded = true;
+  c->last_stream = st;
+  s.append_layer = last ? 0 : layer + 1;
+  if (last) {
+    s.T_a = T_new; s.C = C_new; s.S = S_new; s.S_base = S_new;
+    c->wl_layers.clear();   // the heads grew: the next step cuts its work anew
+    c->prefill_seq = -1;
+  }
+  return WNW_OK;
+}
 
 // Eq. 1 on the host: retention_i = min(s_tilde_i * lambda, 1).
 extern "C" wnw_status_t wnw_retention_schedule(const float *s_tilde, int32_t n, float lambda, float *retention) {
@@ -1185,7 +1229,7 @@ extern "C" wnw_status_t wnw_step_begin(wnw_cache_t *c, const int32_t *active, in
     if (active[i] < 0 || active[i] >= c->geo.max_batch) return WNW_ERR_INVALID_ARG;
     for (int j = 0; j < i; ++j)
       if (active[j] == active[i]) return WNW_ERR_INVALID_ARG;
-    if (c->seqs[active[i]].placed_layers != c->geo.L) return WNW_ERR_STATE;
+    if (c->seqs[active[i]].placed_layers != c->geo.L || c->seqs[active[i]].append_layer != 0) return WNW_ERR_STATE;
   }
   DeviceGuard guard(c->cfg.device);
   std::vector<int> want(active, active + n_active);

@@ -221,7 +221,7 @@ __global__ void __launch_bounds__(128) wnw_token_mirror_kernel(const __grid_cons
   const int pieces = G.d / 8;
   for (int kv = 0; kv < 2; ++kv) {
     const uint4 *src = reinterpret_cast<const uint4 *>(stage + anchor_off(G, 0, 0, h, kv) + (long long)c * G.ncp * G.d);
-    uint4 *dst = reinterpret_cast<uint4 *>(cv.mirror[b] + mirror_off(G, li, cv.C[b], c, t, kv));
+    uint4 *dst = reinterpret_cast<uint4 *>(cv.mirror[b] + mirror_off(G, li, mirror_chunks_of(G, cv.C[b]), c, t, kv));
     for (int v = threadIdx.x; v < len * pieces; v += blockDim.x) {
       const int r = v / pieces, piece = v - r * pieces;
       dst[(long long)mirror_dst[r] * pieces + piece] = src[v];
