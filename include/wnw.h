@@ -115,6 +115,12 @@ typedef struct {
   int32_t recall_mode;                     /* WNW_RECALL_* */
   int32_t score_scope;                     /* WNW_SCOPE_* */
   int32_t residency;                       /* WNW_RESIDENCY_* */
+  int32_t defer_selection;                 /* 1: head-sharded serving (see wnw_export_scores): a layer's decode call only adds up the
+                                            * chunk scores of the cache's OWN anchor heads; top-k, residency update and recall of every
+                                            * tidal layer run in wnw_step_end, on the scores handed back by wnw_import_scores */
+  const uint8_t *global_anchor_layers;     /* HOST [n_layers] or NULL, copied.  Head-sharded serving: which layers have an anchor head
+                                            * on ANY shard; score routing follows these flags instead of the cache's own roles, and a
+                                            * cache may then hold tidal heads without an anchor head of its own */
   int32_t streaming_audio;                 /* 1: clips may grow after placement (wnw_append_audio): every sequence's pinned host
                                             * mirror is sized and laid out for max_audio_tokens.  0: mirrors are sized by the
                                             * placed clip and wnw_append_audio is refused */
@@ -245,6 +251,24 @@ wnw_status_t wnw_decode_layer(wnw_cache_t *cache, int32_t layer, const void *q_d
  * no scores, no selection.  FULL mode only. */
 wnw_status_t wnw_decode_layer_full(wnw_cache_t *cache, int32_t layer, const void *q_dev, const void *k_new_dev,
                                    const void *v_new_dev, void *out_dev, void *cuda_stream);
+
+/* Head-sharded serving (one process per GPU, each holding a cache over its own KV heads; Eq. 2's chunk-score vector is all
+ * that crosses heads).  With defer_selection = 1, between the last layer's wnw_decode_layer and wnw_step_end:
+ *   wnw_export_scores  copies this cache's partial sums, score_sum[active sequence][layer][chunk] over its own anchor
+ *                      heads (zero rows for layers whose anchor heads sit on other shards), into scores_dev, a DEVICE
+ *                      buffer of [n_active][n_layers][C_max] floats, C_max = ceil(max_audio_tokens / chunk_tokens);
+ *   (the caller adds the buffers of all shards up: one all-reduce(sum) over the ranks, in place, on cuda_stream)
+ *   wnw_import_scores  takes the sums back; wnw_step_end then selects, updates the tables and recalls from them.
+ * Every shard thus makes the same selection for its own tidal heads.  The same exchange runs once per layer at placement
+ * for the tidal tables' initial content, which ranks chunks by the prefill score summed over ALL tidal heads of the layer:
+ *   wnw_export_prefill_tidal  after wnw_place_prefill of (seq, layer): this cache's sum over its own tidal heads, [C_max] floats;
+ *   wnw_import_prefill_tidal  the sum over all shards: the layer's table is ranked anew from it and its slots are filled
+ *                             from the host mirror.
+ * Both calls of a pair work on cuda_stream in order; eager steps only (wnw_graph_begin is refused in this mode). */
+wnw_status_t wnw_export_scores(wnw_cache_t *cache, void *scores_dev, void *cuda_stream);
+wnw_status_t wnw_import_scores(wnw_cache_t *cache, const void *scores_dev, void *cuda_stream);
+wnw_status_t wnw_export_prefill_tidal(wnw_cache_t *cache, int32_t seq, int32_t layer, void *sums_dev, void *cuda_stream);
+wnw_status_t wnw_import_prefill_tidal(wnw_cache_t *cache, int32_t seq, int32_t layer, const void *sums_dev, void *cuda_stream);
 
 /* Close the step: per-sequence step counters and text lengths advance.  All layers must have been called. */
 wnw_status_t wnw_step_end(wnw_cache_t *cache, void *cuda_stream);

@@ -115,6 +115,10 @@ typedef struct {
   int delta;      /* eviction lag of SEGMENT_LAG */
   double budget, scale;
   uint8_t *roles; /* [L][Hkv] */
+  uint8_t *anchor_layer; /* [L] does the layer have an anchor head: over ALL KV heads of the model, which are more than this
+                          * oracle's own when it holds one shard of the heads (wnwo_create_shard) */
+  int sharded;    /* this oracle holds a shard of the KV heads: its chunk scores are partial sums until the shards' sums have
+                   * been added up and handed back (wnwo_set_chunk_scores) */
   int *src;       /* [L] score source layer, -1 if the layer has no tidal heads or no source */
   Seq *seq;
   int *active;
@@ -301,12 +305,25 @@ void wnwo_destroy(Oracle *o) {
   if (!o) return;
   if (o->seq)
     for (int b = 0; b < o->max_batch; ++b) free_seq(o, &o->seq[b]);
-  free(o->seq); free(o->roles); free(o->src); free(o->active);
+  free(o->seq); free(o->roles); free(o->anchor_layer); free(o->src); free(o->active);
   free(o);
 }
 
+/* One shard of the KV heads of a model whose layers' anchor heads may sit in other shards (head-sharded serving: the only
+ * thing that crosses heads is Eq. 2's chunk-score vector).  roles: this shard's heads; global_anchor_layers[l] != 0 iff layer
+ * l has an anchor head in ANY shard (NULL: this oracle holds all heads).  Routing follows the global flags; a layer's
+ * scores are summed over the shard's own anchor heads and are complete only after wnwo_set_chunk_scores. */
+int wnwo_create_shard(int L, int Hq, int Hkv, int d, int max_batch, int max_audio, int max_text, int chunk, int topk,
+                      double budget, double scale, const uint8_t *roles, int scope, int residency, int delta,
+                      const uint8_t *global_anchor_layers, Oracle **out);
 int wnwo_create(int L, int Hq, int Hkv, int d, int max_batch, int max_audio, int max_text, int chunk, int topk,
                 double budget, double scale, const uint8_t *roles, int scope, int residency, int delta, Oracle **out) {
+  return wnwo_create_shard(L, Hq, Hkv, d, max_batch, max_audio, max_text, chunk, topk, budget, scale, roles, scope, residency, delta,
+                           NULL, out);
+}
+int wnwo_create_shard(int L, int Hq, int Hkv, int d, int max_batch, int max_audio, int max_text, int chunk, int topk,
+                      double budget, double scale, const uint8_t *roles, int scope, int residency, int delta,
+                      const uint8_t *global_anchor_layers, Oracle **out) {
   if (!out || !roles || L < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv || d < 1 || max_batch < 1 || chunk < 1 || topk < 1)
     return WNWO_ERR_ARG;
   if (!(budget > 0.0 && budget <= 1.0) || scope < 0 || scope > 1 || residency < 0 || residency > 2 || delta < 0)
@@ -321,16 +338,23 @@ int wnwo_create(int L, int Hq, int Hkv, int d, int max_batch, int max_audio, int
   o->delta = delta;
   o->scale = scale > 0.0 ? scale : 1.0 / sqrt((double)d); /* Eq. 2: q K^T / sqrt(d) */
   o->roles = (uint8_t *)malloc((size_t)L * Hkv);
+  o->anchor_layer = (uint8_t *)calloc((size_t)L, 1);
+  o->sharded = global_anchor_layers != NULL;
   o->src = (int *)malloc(sizeof(int) * L);
   o->seq = (Seq *)calloc((size_t)max_batch, sizeof(Seq));
   o->active = (int *)calloc((size_t)max_batch, sizeof(int));
-  if (!o->roles || !o->src || !o->seq || !o->active) { wnwo_destroy(o); return WNWO_ERR_OOM; }
+  if (!o->roles || !o->anchor_layer || !o->src || !o->seq || !o->active) { wnwo_destroy(o); return WNWO_ERR_OOM; }
   memcpy(o->roles, roles, (size_t)L * Hkv);
   int any_anchor = 0, any_tidal = 0;
   for (int i = 0; i < L * Hkv; ++i) {
     if (roles[i] > ROLE_FIXED) { wnwo_destroy(o); return WNWO_ERR_ARG; }
     any_anchor |= roles[i] == ROLE_ANCHOR;
     any_tidal |= roles[i] == ROLE_TIDAL;
+  }
+  for (int l = 0; l < L; ++l) {
+    o->anchor_layer[l] = global_anchor_layers ? (global_anchor_layers[l] != 0) : (uint8_t)layer_has(o, l, ROLE_ANCHOR);
+    if (global_anchor_layers && layer_has(o, l, ROLE_ANCHOR) && !global_anchor_layers[l]) { wnwo_destroy(o); return WNWO_ERR_ARG; }
+    any_anchor |= o->anchor_layer[l];
   }
   if (any_tidal && !any_anchor) { wnwo_destroy(o); return WNWO_ERR_ARG; }
   /* score routing: own layer if it has an anchor, else the nearest anchor layer, ties to the lower one */
@@ -339,7 +363,7 @@ int wnwo_create(int L, int Hq, int Hkv, int d, int max_batch, int max_audio, int
     if (!layer_has(o, l, ROLE_TIDAL)) continue;
     int best = -1;
     for (int a = 0; a < L; ++a) {
-      if (!layer_has(o, a, ROLE_ANCHOR)) continue;
+      if (!o->anchor_layer[a]) continue;
       if (best < 0 || abs(a - l) < abs(best - l)) best = a; /* ascending a: the lower layer wins a tie */
     }
     o->src[l] = best;
@@ -744,6 +768,11 @@ int wnwo_step_begin(Oracle *o, const int *active, int n_active) {
   }
   memcpy(o->active, active, sizeof(int) * n_active);
   o->n_active = n_active; o->in_step = 1; o->next_layer = 0; o->appended = -1;
+  if (o->sharded) /* a layer whose anchor heads all sit in other shards contributes a zero partial sum */
+    for (int i = 0; i < n_active; ++i) {
+      Seq *s = &o->seq[active[i]];
+      memset(s->score_sum, 0, sizeof(double) * (size_t)o->L * (size_t)(s->C > 0 ? s->C : 1));
+    }
   return WNWO_OK;
 }
 
@@ -809,7 +838,7 @@ int wnwo_step_end(Oracle *o) {
       double *glob = (double *)calloc((size_t)C, sizeof(double));
       if (o->scope == 1) /* Eq. 2: one accumulator over all anchor (layer, q-head) pairs of the step */
         for (int a = 0; a < o->L; ++a)
-          if (layer_has(o, a, ROLE_ANCHOR))
+          if (o->anchor_layer[a])
             for (int c = 0; c < C; ++c) glob[c] += s->score_sum[(size_t)a * C + c];
       int *segs = (int *)malloc(sizeof(int) * 2 * o->topk), *rel = (int *)malloc(sizeof(int) * (size_t)(S > 0 ? S : 1));
       int *pg = (int *)malloc(sizeof(int) * 2 * o->topk), *pj = (int *)malloc(sizeof(int) * 2 * o->topk);
@@ -848,6 +877,16 @@ int wnwo_step_end(Oracle *o) {
 /* ------------------------------------------------------------------ */
 /* Inspection and lock-step helpers                                     */
 /* ------------------------------------------------------------------ */
+
+/* Head-sharded serving: the chunk scores of `layer` summed over all shards replace this shard's partial sum, between
+ * the last layer of a step and wnwo_step_end. */
+int wnwo_set_chunk_scores(Oracle *o, int seq, int layer, const double *scores) {
+  if (!o || !scores || seq < 0 || seq >= o->max_batch || layer < 0 || layer >= o->L) return WNWO_ERR_ARG;
+  if (!o->in_step || o->next_layer != o->L) return WNWO_ERR_STATE;
+  Seq *s = &o->seq[seq];
+  for (int c = 0; c < s->C; ++c) s->score_sum[(size_t)layer * s->C + c] = scores[c];
+  return WNWO_OK;
+}
 
 int wnwo_get_dims(const Oracle *o, int seq, int *T_a, int *T_t, int *C, int *S) {
   if (!o || seq < 0 || seq >= o->max_batch || o->seq[seq].placed_layers == 0) return WNWO_ERR_STATE;

@@ -43,6 +43,9 @@ def lib():
         _lib = C.CDLL(build())
         _lib.wnwo_create.argtypes = [C.c_int] * 9 + [C.c_double, C.c_double, C.POINTER(C.c_uint8), C.c_int, C.c_int, C.c_int,
                                      C.POINTER(C.c_void_p)]
+        _lib.wnwo_create_shard.argtypes = [C.c_int] * 9 + [C.c_double, C.c_double, C.POINTER(C.c_uint8), C.c_int, C.c_int, C.c_int,
+                                           C.POINTER(C.c_uint8), C.POINTER(C.c_void_p)]
+        _lib.wnwo_set_chunk_scores.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_double)]
         _lib.wnwo_destroy.argtypes = [C.c_void_p]
         _lib.wnwo_destroy.restype = None
         _lib.wnwo_score_source.argtypes = [C.c_void_p, C.c_int]
@@ -171,16 +174,20 @@ class Oracle:
     """The stateful decode-step oracle.  Arrays in/out are numpy; bf16 values travel as uint16 bit patterns."""
 
     def __init__(self, n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
-                 chunk_tokens, topk, budget, roles, softmax_scale=0.0, score_scope=0, residency=0, evict_lag=3):
+                 chunk_tokens, topk, budget, roles, softmax_scale=0.0, score_scope=0, residency=0, evict_lag=3,
+                 global_anchor_layers=None):
         self.L, self.Hq, self.Hkv, self.d = n_layers, n_q_heads, n_kv_heads, head_dim
         self.topk_cfg = topk
         roles = np.ascontiguousarray(roles, dtype=np.uint8).reshape(-1)
         assert roles.size == n_layers * n_kv_heads
         h = C.c_void_p()
         # budget is a float32 field in the library's config; mirror that rounding here
-        _check(lib().wnwo_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
-                                 chunk_tokens, topk, float(np.float32(budget)), float(softmax_scale),
-                                 _p(roles, C.c_uint8), score_scope, residency, evict_lag, C.byref(h)), "create")
+        # global_anchor_layers [n_layers]: this oracle holds one shard of the KV heads (see wnwo_create_shard)
+        ga = None if global_anchor_layers is None else np.ascontiguousarray(global_anchor_layers, dtype=np.uint8)
+        _check(lib().wnwo_create_shard(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
+                                       chunk_tokens, topk, float(np.float32(budget)), float(softmax_scale),
+                                       _p(roles, C.c_uint8), score_scope, residency, evict_lag, _p(ga, C.c_uint8), C.byref(h)),
+               "create")
         self.residency_mode, self.evict_lag = residency, evict_lag
         self.score_scope = score_scope
         self._h = h
@@ -271,6 +278,11 @@ class Oracle:
         out = np.zeros(self.dims(seq)[2], np.float64)
         lib().wnwo_get_chunk_scores(self._h, seq, layer, _p(out, C.c_double))
         return out
+
+    def set_chunk_scores(self, seq, layer, scores):
+        sc = np.ascontiguousarray(scores, np.float64)
+        assert len(sc) == self.dims(seq)[2]
+        _check(lib().wnwo_set_chunk_scores(self._h, seq, layer, _p(sc, C.c_double)), "set_chunk_scores")
 
     def prefill_scores(self, seq, layer, kv_head) -> np.ndarray:
         out = np.zeros(self.dims(seq)[2], np.float64)

@@ -30,7 +30,8 @@ class wnw_config_t(C.Structure):
                 ("max_batch", C.c_int32), ("max_audio_tokens", C.c_int32), ("max_text_tokens", C.c_int32),
                 ("chunk_tokens", C.c_int32), ("topk", C.c_int32), ("evict_lag", C.c_int32), ("budget", C.c_float),
                 ("softmax_scale", C.c_float), ("roles", C.POINTER(C.c_uint8)), ("device", C.c_int32), ("mode", C.c_int32),
-                ("recall_mode", C.c_int32), ("score_scope", C.c_int32), ("residency", C.c_int32), ("streaming_audio", C.c_int32)]
+                ("recall_mode", C.c_int32), ("score_scope", C.c_int32), ("residency", C.c_int32), ("defer_selection", C.c_int32),
+                ("global_anchor_layers", C.POINTER(C.c_uint8)), ("streaming_audio", C.c_int32)]
 
 
 class wnw_stats_t(C.Structure):
@@ -52,6 +53,10 @@ _SIGNATURES = {
     "wnw_place_prefill": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _vp],
     "wnw_place_prefill_multi": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp],
     "wnw_place_prefill_tokens": [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _i32, _vp, _i32, C.POINTER(C.c_float), _i32, _i32, _vp],
+    "wnw_export_scores": [_vp, _vp, _vp],
+    "wnw_import_scores": [_vp, _vp, _vp],
+    "wnw_export_prefill_tidal": [_vp, _i32, _i32, _vp, _vp],
+    "wnw_import_prefill_tidal": [_vp, _i32, _i32, _vp, _vp],
     "wnw_append_audio": [_vp, _i32, _i32, _vp, _vp, _i32, _vp],
     "wnw_retention_schedule": [C.POINTER(C.c_float), _i32, C.c_float, C.POINTER(C.c_float)],
     "wnw_get_token_scores": [_vp, _i32, _i32, _i32, C.POINTER(C.c_float), _i32],
@@ -135,12 +140,17 @@ def _stream(stream) -> Optional[int]:
 def wnw_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens, chunk_tokens,
                budget, roles, topk=3, evict_lag=3, softmax_scale=0.0, device=0, mode=WNW_MODE_TIERED,
                recall_mode=WNW_RECALL_SIDE_STREAM, score_scope=WNW_SCOPE_PER_LAYER, residency=WNW_RESIDENCY_HARD_BUDGET,
-               streaming_audio=0) -> int:
+               streaming_audio=0, defer_selection=0, global_anchor_layers=None) -> int:
     roles = np.ascontiguousarray(roles, dtype=np.uint8).reshape(-1)
     cfg = wnw_config_t(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
                        chunk_tokens, topk, evict_lag, budget, softmax_scale,
                        roles.ctypes.data_as(C.POINTER(C.c_uint8)), device, mode, recall_mode, score_scope, residency,
-                       int(streaming_audio))
+                       int(defer_selection), None, int(streaming_audio))
+    if global_anchor_layers is not None:
+        ga = np.ascontiguousarray(global_anchor_layers, dtype=np.uint8).reshape(-1)
+        if ga.size != n_layers:
+            raise WnwError(WNW_ERR_INVALID_ARG, "wnw_create (global_anchor_layers size)")
+        cfg.global_anchor_layers = ga.ctypes.data_as(C.POINTER(C.c_uint8))
     if roles.size != n_layers * n_kv_heads:
         raise WnwError(WNW_ERR_INVALID_ARG, "wnw_create (roles size)")
     h = _vp()
@@ -158,6 +168,24 @@ def wnw_place_prefill(cache, seq, layer, k, v, audio_begin, audio_end, q_last=No
         return wnw_place_prefill_multi(cache, seq, layer, k, v, audio_begin, audio_end, q_last, stream)
     _ck(lib().wnw_place_prefill(cache, seq, layer, _ptr(k), _ptr(v), k.shape[0], audio_begin, audio_end, _ptr(q_last),
                                 _stream(stream)), "wnw_place_prefill")
+
+
+def wnw_export_scores(cache, scores, stream=None):
+    """scores: float32 CUDA tensor [n_active, n_layers, C_max]."""
+    _ck(lib().wnw_export_scores(cache, _ptr(scores), _stream(stream)), "wnw_export_scores")
+
+
+def wnw_import_scores(cache, scores, stream=None):
+    _ck(lib().wnw_import_scores(cache, _ptr(scores), _stream(stream)), "wnw_import_scores")
+
+
+def wnw_export_prefill_tidal(cache, seq, layer, sums, stream=None):
+    """sums: float32 CUDA tensor [C_max]."""
+    _ck(lib().wnw_export_prefill_tidal(cache, seq, layer, _ptr(sums), _stream(stream)), "wnw_export_prefill_tidal")
+
+
+def wnw_import_prefill_tidal(cache, seq, layer, sums, stream=None):
+    _ck(lib().wnw_import_prefill_tidal(cache, seq, layer, _ptr(sums), _stream(stream)), "wnw_import_prefill_tidal")
 
 
 def wnw_append_audio(cache, seq, layer, k, v, stream=None):

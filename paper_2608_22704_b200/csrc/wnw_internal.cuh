@@ -253,6 +253,9 @@ cudaError_t launch_token_compress(const CacheView &cv, int b, int layer, int n_c
                                   int32_t *fixed_tok, int tok_cap, int32_t *tok_n, cudaStream_t st);
 cudaError_t launch_append_audio(const CacheView &cv, int b, int layer, int full_mode, const bf16 *k, const bf16 *v, int n_tokens,
                                 int T_a_old, int S_old, int set_dims, int T_a_new, int C_new, int S_new, cudaStream_t st);
+cudaError_t launch_exchange_scores(const CacheView &cv, int n_active, const int32_t *active, float *buf, int out, cudaStream_t st);
+cudaError_t launch_prefill_tidal_sum(const CacheView &cv, int b, int layer, float *dst, cudaStream_t st);
+cudaError_t launch_prefill_retable(const CacheView &cv, int b, int layer, const float *sums, cudaStream_t st);
 cudaError_t launch_copy_plan(const uint4 *src_host_mapped, uint4 *dst, long long n_vec, int n_ctas, cudaStream_t st);
 cudaError_t configure_attn_kernels();
 // the CTAs of several layers' launches (one-shot variant) in one launch

@@ -619,6 +619,84 @@ __global__ void __launch_bounds__(512) wnw_prefill_select_kernel(const __grid_co
     }
   }
 }
+// Head-sharded placement.  (1) This cache's share of the tidal ranking of (b, layer): the prefill scores of its own tidal
+// heads added in head order, [C_max] floats, zero past the sequence's chunks.
+__global__ void wnw_prefill_tidal_sum_kernel(const __grid_constant__ CacheView cv, int b, int layer, float *dst) {
+  const Geometry &G = cv.geo;
+  const int C_b = cv.C[b];
+  const float *pre = cv.pre + ((long long)b * G.L + layer) * G.Hkv * G.C_max;
+  for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < G.C_max; c += gridDim.x * blockDim.x) {
+    float total = 0.f;
+    if (c < C_b)
+      for (int h = 0; h < G.Hkv; ++h)
+        if (cv.roles[layer * G.Hkv + h] == ROLE_TIDAL) total += pre[(long long)h * G.C_max + c];
+    dst[c] = total;
+  }
+}
+// (2) The table of (b, layer) ranked anew from the sums over all shards (rank r -> slot r, stamp -1-r, as at placement)...
+__global__ void __launch_bounds__(512) wnw_prefill_retable_kernel(const __grid_constant__ CacheView cv, int b, int layer, const float *sums) {
+  extern __shared__ unsigned long long rkey[];
+  const Geometry &G = cv.geo;
+  const int C_b = cv.C[b], S_b = cv.S_base[b], T_a = cv.T_a[b], tid = threadIdx.x;
+  const long long bl = (long long)b * G.L + layer;
+  for (int s = tid; s < G.S_max; s += blockDim.x) {
+    cv.slot_chunk[slot_table_off(G, 0, bl) + s] = -1; cv.slot_chunk[slot_table_off(G, 1, bl) + s] = -1; cv.stamp[bl * G.S_max + s] = 0;
+  }
+  for (int c = tid; c < G.C_max; c += blockDim.x) cv.chunk_slot[bl * G.C_max + c] = -1;
+  for (int c = tid; c < C_b; c += blockDim.x) rkey[c] = rank_key(sums[c], chunk_len(G, T_a, c), c);
+  __syncthreads();
+  const int parity = (int)(cv.steps[b] & 1);
+  for (int c = tid; c < C_b; c += blockDim.x) {
+    const unsigned long long me = rkey[c];
+    int rank = 0;
+    for (int x = 0; x < C_b; ++x) rank += rkey[x] > me;
+    if (rank < S_b) {
+      cv.slot_chunk[slot_table_off(G, parity, bl) + rank] = c;
+      cv.chunk_slot[bl * G.C_max + c] = rank;
+      cv.stamp[bl * G.S_max + rank] = -1 - (long long)rank;
+    }
+  }
+}
+// ... (3) and its slots filled from the host mirror: one CTA per slot copies the chunk's block (all tidal heads, K and V).
+__global__ void wnw_refill_slots_kernel(const __grid_constant__ CacheView cv, int b, int layer) {
+  const Geometry &G = cv.geo;
+  const LayerInfo li = cv.layers[layer];
+  const long long bl = (long long)b * G.L + layer;
+  const int slot = blockIdx.x, c = cv.slot_chunk[slot_table_off(G, (int)(cv.steps[b] & 1), bl) + slot];
+  if (c < 0 || li.n_tidal == 0) return;
+  const long long n_vec = (long long)li.n_tidal * 2 * G.ncp * G.d / 8;
+  const uint4 *src = reinterpret_cast<const uint4 *>(cv.mirror[b] + mirror_off(G, li, mirror_chunks_of(G, cv.C[b]), c, 0, 0));
+  uint4 *dst = reinterpret_cast<uint4 *>(cv.pool + pool_off(G, li, b, slot, 0, 0));
+  for (long long i = threadIdx.x; i < n_vec; i += blockDim.x) dst[i] = src[i];
+}
+// Head-sharded step: grid (active sequence, layer).  Out: the cache's own partial sums of the layer's chunk scores, a zero
+// row where none of the layer's anchor heads is the cache's own (the row may still hold the sums taken back in an earlier
+// step).  In: the sums over all shards.
+__global__ void wnw_exchange_scores_kernel(const __grid_constant__ CacheView cv, const int32_t *active, float *buf, int out) {
+  const Geometry &G = cv.geo;
+  const int i = blockIdx.x, l = blockIdx.y, b = active[i];
+  float *mine = cv.score_sum + ((long long)b * G.L + l) * G.C_max, *theirs = buf + ((long long)i * G.L + l) * G.C_max;
+  const bool own = cv.layers[l].n_anchor > 0;
+  for (int c = threadIdx.x; c < G.C_max; c += blockDim.x) {
+    if (out) theirs[c] = own && c < cv.C[b] ? mine[c] : 0.f;
+    else mine[c] = theirs[c];
+  }
+}
+cudaError_t launch_exchange_scores(const CacheView &cv, int n_active, const int32_t *active, float *buf, int out, cudaStream_t st) {
+  if (cv.geo.C_max < 1) return cudaSuccess;
+  wnw_exchange_scores_kernel<<<dim3((unsigned)n_active, (unsigned)cv.geo.L), 128, 0, st>>>(cv, active, buf, out);
+  return cudaGetLastError();
+}
+cudaError_t launch_prefill_tidal_sum(const CacheView &cv, int b, int layer, float *dst, cudaStream_t st) {
+  wnw_prefill_tidal_sum_kernel<<<4, 256, 0, st>>>(cv, b, layer, dst);
+  return cudaGetLastError();
+}
+cudaError_t launch_prefill_retable(const CacheView &cv, int b, int layer, const float *sums, cudaStream_t st) {
+  wnw_prefill_retable_kernel<<<1, 512, (size_t)std::max(cv.geo.C_max, 1) * 8, st>>>(cv, b, layer, sums);
+  if (cv.geo.S_max > 0) wnw_refill_slots_kernel<<<cv.geo.S_max, 256, 0, st>>>(cv, b, layer);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_prefill_select(const CacheView &cv, int b, int layer, const HeadItems *head_items, const float2 *part_ml,
                                   const float2 *gran_em, int n_ag_max, int first, int last, cudaStream_t st) {
   const size_t smem = (size_t)(2 * cv.geo.Hq + 2) * sizeof(float) + (size_t)cv.geo.C_max * sizeof(unsigned long long);

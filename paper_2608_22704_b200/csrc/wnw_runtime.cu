@@ -58,6 +58,8 @@ struct wnw_cache {
   std::vector<LayerInfo> layers;
   std::vector<int32_t> upd_list, anchor_layers;
   std::vector<int> tail_of;  // layer -> layer whose tail updates its table, -1 if none
+  std::vector<uint8_t> anchor_layer;   // [L] the layer has an anchor head (on any shard, when the cache holds one shard of the heads)
+  bool scores_exported = false, scores_imported = false;   // head-sharded step: where the exchange stands
   int tid_total = 0, n_sm = 148;
   std::vector<SeqHost> seqs;
   std::vector<void *> dev_allocs;
@@ -268,12 +270,20 @@ static wnw_status_t validate_config(const wnw_config_t *cfg) {
   if (cfg->residency < WNW_RESIDENCY_HARD_BUDGET || cfg->residency > WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE) return WNW_ERR_INVALID_ARG;
   if (cfg->recall_mode < WNW_RECALL_SIDE_STREAM || cfg->recall_mode > WNW_RECALL_SKIP) return WNW_ERR_INVALID_ARG;
   if (cfg->device < 0 || cfg->streaming_audio < 0 || cfg->streaming_audio > 1) return WNW_ERR_INVALID_ARG;
+  if (cfg->defer_selection < 0 || cfg->defer_selection > 1) return WNW_ERR_INVALID_ARG;
+  if (cfg->defer_selection && (cfg->score_scope != WNW_SCOPE_PER_LAYER || cfg->residency != WNW_RESIDENCY_HARD_BUDGET ||
+                               cfg->recall_mode == WNW_RECALL_INLINE))
+    return WNW_ERR_UNSUPPORTED;
   bool any_anchor = false, any_tidal = false;
   for (int i = 0; i < cfg->n_layers * cfg->n_kv_heads; ++i) {
     if (cfg->roles[i] > WNW_ROLE_FIXED) return WNW_ERR_INVALID_ARG;
     any_anchor |= cfg->roles[i] == WNW_ROLE_ANCHOR;
     any_tidal |= cfg->roles[i] == WNW_ROLE_TIDAL;
+    // a layer the model-wide flags call anchor-less cannot hold an anchor head here
+    if (cfg->global_anchor_layers && cfg->roles[i] == WNW_ROLE_ANCHOR && !cfg->global_anchor_layers[i / cfg->n_kv_heads]) return WNW_ERR_INVALID_ARG;
   }
+  if (cfg->global_anchor_layers)
+    for (int l = 0; l < cfg->n_layers; ++l) any_anchor |= cfg->global_anchor_layers[l] != 0;
   if (cfg->mode == WNW_MODE_TIERED && any_tidal && !any_anchor) return WNW_ERR_INVALID_ARG;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return WNW_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > MAX_G || cfg->n_q_heads > MAX_AQ || cfg->n_layers > 32767) return WNW_ERR_UNSUPPORTED;
@@ -311,6 +321,13 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   const bool full = cfg->mode == WNW_MODE_FULL;
   c->roles.assign(cfg->roles, cfg->roles + (size_t)L * Hkv);
   c->cfg.roles = nullptr;
+  c->anchor_layer.assign(L, 0);
+  for (int l = 0; l < L; ++l) {
+    bool has = cfg->global_anchor_layers ? cfg->global_anchor_layers[l] != 0 : false;
+    for (int h = 0; h < Hkv && !cfg->global_anchor_layers; ++h) has = has || cfg->roles[l * Hkv + h] == WNW_ROLE_ANCHOR;
+    c->anchor_layer[l] = has;
+  }
+  c->cfg.global_anchor_layers = nullptr;
   Geometry &G = c->geo;
   G.L = L; G.Hq = cfg->n_q_heads; G.Hkv = Hkv; G.d = d; G.g = cfg->n_q_heads / Hkv; G.nc = nc; G.ncp = (nc + GR - 1) / GR * GR; G.gpc = G.ncp / GR;
   G.topk = c->cfg.topk;
@@ -353,7 +370,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     if (full || c->layers[l].n_tidal == 0) continue;
     int best = -1;
     for (int a = 0; a < L; ++a)
-      if (c->layers[a].n_anchor > 0 && (best < 0 || std::abs(a - l) < std::abs(best - l))) best = a;
+      if (c->anchor_layer[a] && (best < 0 || std::abs(a - l) < std::abs(best - l))) best = a;
     const bool global = cfg->score_scope == WNW_SCOPE_GLOBAL;
     c->layers[l].src = (global && best >= 0) ? -2 : best;  // nearest anchor layer, ties to the lower one; -2: the global accumulator
     const int x = global ? L - 1 : std::max(l, best);  // first point at which layer l's attention and its scores are done
@@ -1438,13 +1455,17 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
   }
   // chunk scores, selection, recall: on the side stream, overlapping whatever follows on the caller's stream
   // (captured steps of small launches do all of it in one or two launches at the end of the step instead)
-  const bool side_work = tiered && (li.n_anchor > 0 || li.upd_count > 0) && !c->cap_select_all;
+  const bool defer = tiered && c->cfg.defer_selection;   // head-sharded serving: scores now, everything else at the step's end
+  if (defer && capturing) return WNW_ERR_UNSUPPORTED;
+  if (layer == 0) c->scores_exported = c->scores_imported = false;
+  const bool side_work = tiered && (defer ? li.n_anchor > 0 : (li.n_anchor > 0 || li.upd_count > 0)) && !c->cap_select_all;
   const bool inline_mode = c->cfg.recall_mode == WNW_RECALL_INLINE;
   cudaEvent_t ev_l = capturing ? c->ev_layer_done_cap[layer] : c->ev_layer_done[layer];
   if (side_work && !inline_mode) CK(cudaEventRecord(ev_l, st));
   if (side_work) {
     SelectArgs sa = static_select_args(c, layer);
     sa.n_active = n_active;
+    if (defer) sa.do_update = 0;
     if (c->cap_fold) {
       sa.fold_total = c->n_select_ctas * n_active; sa.fold_appended = has_new; sa.fold_counter = c->d_fold_ctr;
       sa.fold_bump_epoch = c->cap_external_recall ? c->d_step_epoch : nullptr;
@@ -1470,7 +1491,7 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
     }
     CK(launch_select(c->cv, sa, c->sel_smem[layer], select_groups(li), ss));
     c->count_launch(1, 1, capturing);
-    if (li.upd_count > 0 && !c->cap_external_recall) {
+    if (li.upd_count > 0 && !c->cap_external_recall && !defer) {
       CK(launch_recall(c->cv, n_active, c->d_active, c->cv.upd_list + li.upd_first, li.upd_count,
                        c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{nullptr, nullptr, nullptr, 0}, ss));
       c->count_launch(2, 1, capturing);
@@ -1496,6 +1517,64 @@ extern "C" wnw_status_t wnw_decode_layer_full(wnw_cache_t *c, int32_t layer, con
   return decode_layer_impl(c, WNW_MODE_FULL, layer, q, k_new, v_new, out, cuda_stream);
 }
 
+// Head-sharded step: the caller's stream waits for the score kernels of the step's anchor layers (side streams).
+static wnw_status_t wait_for_scores(wnw_cache *c, cudaStream_t st) {
+  for (int l = 0; l < c->geo.L; ++l)
+    if (c->layers[l].n_anchor > 0 && c->side_recorded[l]) CK(cudaStreamWaitEvent(st, c->ev_side_done[l], 0));
+  return WNW_OK;
+}
+
+static wnw_status_t exchange_copy(wnw_cache *c, void *buf, bool out, void *cuda_stream) {
+  if (!c || !buf) return WNW_ERR_INVALID_ARG;
+  if (c->cfg.mode != WNW_MODE_TIERED || !c->cfg.defer_selection) return WNW_ERR_UNSUPPORTED;
+  if (!c->in_step || c->next_layer != c->geo.L || (out ? c->scores_exported : !c->scores_exported || c->scores_imported)) return WNW_ERR_STATE;
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (out) {
+    wnw_status_t ws = wait_for_scores(c, st);
+    if (ws != WNW_OK) return ws;
+  }
+  CK(launch_exchange_scores(c->cv, (int)c->active.size(), c->d_active, (float *)buf, out ? 1 : 0, st));
+  (out ? c->scores_exported : c->scores_imported) = true;
+  c->last_stream = st;
+  return WNW_OK;
+}
+extern "C" wnw_status_t wnw_export_scores(wnw_cache_t *c, void *scores_dev, void *cuda_stream) {
+  return exchange_copy(c, scores_dev, true, cuda_stream);
+}
+extern "C" wnw_status_t wnw_import_scores(wnw_cache_t *c, const void *scores_dev, void *cuda_stream) {
+  return exchange_copy(c, const_cast<void *>(scores_dev), false, cuda_stream);
+}
+
+extern "C" wnw_status_t wnw_export_prefill_tidal(wnw_cache_t *c, int32_t seq, int32_t layer, void *sums_dev, void *cuda_stream) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!sums_dev) return WNW_ERR_INVALID_ARG;
+  if (c->cfg.mode != WNW_MODE_TIERED || !c->cfg.defer_selection) return WNW_ERR_UNSUPPORTED;
+  if (c->in_step) return WNW_ERR_STATE;
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
+  CK(launch_prefill_tidal_sum(c->cv, seq, layer, (float *)sums_dev, st));
+  c->last_stream = st;
+  return WNW_OK;
+}
+extern "C" wnw_status_t wnw_import_prefill_tidal(wnw_cache_t *c, int32_t seq, int32_t layer, const void *sums_dev, void *cuda_stream) {
+  wnw_status_t s = check_seq_layer(c, seq, layer);
+  if (s != WNW_OK) return s;
+  if (!sums_dev) return WNW_ERR_INVALID_ARG;
+  if (c->cfg.mode != WNW_MODE_TIERED || !c->cfg.defer_selection) return WNW_ERR_UNSUPPORTED;
+  if (c->in_step) return WNW_ERR_STATE;
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
+  if (c->layers[layer].n_tidal > 0 && c->seqs[seq].C > 0) CK(launch_prefill_retable(c->cv, seq, layer, (const float *)sums_dev, st));
+  CK(cudaEventRecord(c->ev_place, st));
+  c->place_recorded = true;
+  c->last_stream = st;
+  return WNW_OK;
+}
+
 extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
   if (!c) return WNW_ERR_INVALID_ARG;
   if (!c->in_step || c->next_layer != c->geo.L) return WNW_ERR_STATE;
@@ -1513,6 +1592,21 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
     } else {
       wnw_status_t rs = launch_step_selection(c, false, st);
       if (rs != WNW_OK) return rs;
+    }
+  }
+  if (c->cfg.mode == WNW_MODE_TIERED && c->cfg.defer_selection) {
+    // every tidal layer's selection, table update and recall, from the scores as they stand (the sums over all shards
+    // once wnw_import_scores has run; the cache's own sums if it holds every head)
+    wnw_status_t ws = wait_for_scores(c, st);
+    if (ws != WNW_OK) return ws;
+    if (c->sel_map_update[1] > 0) {
+      SelectArgs stp{};
+      stp.n_active = (int)c->active.size(); stp.active = c->d_active; stp.do_score = 0; stp.do_update = 1;
+      CK(select_all(c, c->sel_map_update, stp, st));
+      c->count_launch(1, 1, false);
+      CK(launch_recall(c->cv, (int)c->active.size(), c->d_active, c->cv.upd_list, (int)c->upd_list.size(),
+                       c->cfg.recall_mode == WNW_RECALL_SKIP, RecallSignal{nullptr, nullptr, nullptr, 0}, st));
+      c->count_launch(2, 1, false);
     }
   }
   if (!(capturing && c->cap_fold)) {
@@ -1539,6 +1633,7 @@ extern "C" wnw_status_t wnw_step_end(wnw_cache_t *c, void *cuda_stream) {
 extern "C" wnw_status_t wnw_graph_begin(wnw_cache_t *c, const int32_t *active, int32_t n_active, void *cuda_stream) {
   if (!c || !active || n_active < 1 || n_active > c->geo.max_batch) return WNW_ERR_INVALID_ARG;
   if (c->in_step || c->graph_capturing) return WNW_ERR_STATE;
+  if (c->cfg.defer_selection) return WNW_ERR_UNSUPPORTED;   // the exchange between the shards is the caller's: eager steps only
   if (!cuda_stream) return WNW_ERR_INVALID_ARG;  // the legacy default stream cannot be captured
   for (int i = 0; i < n_active; ++i) {
     if (active[i] < 0 || active[i] >= c->geo.max_batch) return WNW_ERR_INVALID_ARG;
