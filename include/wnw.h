@@ -106,7 +106,8 @@ typedef struct {
   int32_t max_text_tokens;                 /* per sequence, prompt text + every decode append */
   int32_t chunk_tokens;                    /* n_c >= 1 (e.g. ceil(4 s * 12.5 tok/s) = 50, "Chunk Structure"); stored padded to 16 rows */
   int32_t topk;                            /* k, chunks selected per step; 0 -> 3 (the paper's k) */
-  int32_t evict_lag;                       /* the paper's delta; accepted, reserved (fixed pool evicts least-recent) */
+  int32_t evict_lag;                       /* the paper's delta: steps a fetched segment may stay unselected before it is released
+                                            * (SEGMENT_LAG residencies; HARD_BUDGET evicts the least recently selected chunk instead) */
   float budget;                            /* (0,1]; see S above */
   float softmax_scale;                     /* 0 -> 1/sqrt(head_dim) (Eq. 2) */
   const uint8_t *roles;                    /* HOST [n_layers * n_kv_heads], WNW_ROLE_*, copied */
@@ -331,28 +332,12 @@ wnw_status_t wnw_get_stats(wnw_cache_t *cache, wnw_stats_t *stats_host);
 enum { WNW_LAYERS_INDEPENDENT = 0, WNW_LAYERS_CHAINED = 1, WNW_LAYERS_SERIAL = 2, WNW_LAYERS_BATCHED = 3 };
 wnw_status_t wnw_set_layer_dependency(wnw_cache_t *cache, int32_t mode);
 
-/* Test hook for the bounded waits: adds `delta` to the device's step-epoch word, so that the tidal CTAs of the next
- * replayed step wait for a recall epoch that nothing will publish.  Every such wait gives up after about a second of
- * SM clocks, the kernel finishes on what it has and sets the sticky status that wnw_sync reports as WNW_ERR_TIMEOUT.
- * The cache's results are meaningless afterwards; destroy it.  Not for production use. */
-wnw_status_t wnw_debug_advance_step_epoch(wnw_cache_t *cache, int32_t delta);
-
 /* Kernels this cache has launched on the decode path since creation, replayed captured steps included:
  * counts[0] attention, [1] selection, [2] recall, [3] step-end.  Host counters, no synchronisation. */
 wnw_status_t wnw_get_launch_counts(wnw_cache_t *cache, int64_t counts[4]);
 
-/* Optional per-kernel timing: when enabled the library brackets its attention-kernel launches with CUDA events
- * on the launching stream; wnw_get_kernel_time returns the accumulated milliseconds and launch count since the
- * last call (drains the stream).  Off by default. */
-wnw_status_t wnw_set_kernel_timing(wnw_cache_t *cache, int32_t enable);
-wnw_status_t wnw_get_kernel_time(wnw_cache_t *cache, float *attn_ms, int32_t *attn_launches);
-
 /* Drain the caller's stream and the recall stream; returns the sticky asynchronous status. */
 wnw_status_t wnw_sync(wnw_cache_t *cache);
-
-/* Host-link probe used by the benchmark: copies `bytes` from pinned host memory into device memory `reps` times
- * (a) with cudaMemcpyAsync and (b) with the library's recall kernel on a synthetic plan, and returns GB/s of each. */
-wnw_status_t wnw_measure_host_link(int32_t device, int64_t bytes, int32_t reps, double *memcpy_gbs, double *kernel_gbs);
 
 /* Full attention of ONE query token over a caller-owned K/V buffer, without any allocation.  (The paper has no
  * counterpart: this is a convenience entry for callers that must not allocate.)

@@ -392,9 +392,7 @@ cudaError_t launch_recall(const CacheView &cv, int n_active, const int32_t *acti
   // several times while attention saturates the memory system, so four times the CTAs keep four times the loads in
   // flight (config 1 back to back: 56 -> 53 us per step).  Many tables: the link's rate counts and more CTAs only take
   // SM resources from attention (batch-32 ragged, link-bound: 2.56 -> 2.88 ms per step with the wide launch).
-  int n_groups = RECALL_GROUPS, n_ctas = sig.epoch_words && (long long)n_active * n_layers <= 64 ? 4 * RECALL_CTAS : RECALL_CTAS;
-  if (const char *e = getenv("WNW_RECALL_GROUPS")) n_groups = std::max(1, atoi(e));
-  if (const char *e = getenv("WNW_RECALL_CTAS")) n_ctas = std::max(n_groups, atoi(e));
+  const int n_groups = RECALL_GROUPS, n_ctas = sig.epoch_words && (long long)n_active * n_layers <= 64 ? 4 * RECALL_CTAS : RECALL_CTAS;
   const int groups = n_layers < n_groups ? n_layers : n_groups;   // few layers: all CTAs on each block
   wnw_recall_kernel<<<n_ctas / groups * groups, 256, 0, st>>>(cv, n_active, active, layers_dev, n_layers, groups, skip_copy, sig);
   return cudaGetLastError();

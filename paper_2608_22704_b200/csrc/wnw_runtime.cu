@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "../../include/wnw.h"
+#include "../../include/wnw_debug.h"
 #include "wnw_internal.cuh"
 
 using namespace wnw;
@@ -105,18 +106,16 @@ struct wnw_cache {
   std::vector<size_t> sel_smem;   // dynamic shared memory of each layer's selection launch
   size_t gran_em_layer_stride = 0;
   bool step_capturing = false;
-  bool pdl_enabled = true, pack_enabled = true;
-  int pack_granules = 0;   // work per packed CTA (0: automatic)
   // Captured steps of small launches: the selection work of all layers in one launch at the end of the step (two when a
   // layer ranks by another layer's scores: first all scores, then all updates).
-  bool select_all_enabled = true, cap_select_all = false, select_single_ok = false;
+  bool cap_select_all = false, select_single_ok = false;
   SelectArgs *d_sel_args = nullptr;
   int4 *d_sel_map = nullptr;
   std::vector<SelectArgs> h_sel_args;   // host copies: small stacks pass them in the kernel parameters
   std::vector<int4> h_sel_map;
   int sel_map_single[2] = {0, 0}, sel_map_score[2] = {0, 0}, sel_map_update[2] = {0, 0};   // offset, entries
   size_t sel_all_smem = 0;
-  bool fold_enabled = true, cap_fold = false;   // captured steps: the last selection CTA closes the step
+  bool cap_fold = false;   // captured steps: the last selection CTA closes the step
   int n_side_layers = 0, n_select_ctas = 0;   // layers with a selection kernel; its CTAs per sequence over all layers
   int32_t *d_fold_ctr = nullptr, *d_empty_ctr = nullptr;
   int32_t host_epoch = 0;   // replayed steps with out-of-graph recall so far = the value of the device's step epoch after them
@@ -124,19 +123,18 @@ struct wnw_cache {
   void count_launch(int kind, int n, bool capturing) { (capturing ? cap_launches : launches)[kind] += n; }
   int layer_dependency = WNW_LAYERS_INDEPENDENT;
   std::vector<AttnArgs> batch_args;   // BATCHED layers of a captured step: recorded per layer, launched by the last one
-  bool cap_batched = false, batched_two_part = true;
+  bool cap_batched = false;
   // the step's selection beside its tidal attention (all layers issued together, two parts): forked after the first part
-  bool cap_sel_overlap = false, sel_overlap_enabled = true;
+  bool cap_sel_overlap = false;
   cudaEvent_t ev_sel_fork = nullptr, ev_sel_join = nullptr;
   int batched_target = 0;             // granules of work per CTA when the step's layers share one launch ...
   int batched_target_tidal = 0;       // ... and per CTA of its second part, the tidal heads
   // replayed steps: one recall launch per step outside the captured graph, overlapping the next step
   int32_t *d_recall_epoch = nullptr, *d_recall_ctr = nullptr, *d_step_epoch = nullptr;
-  int external_recall_mode = -1;   // -1 automatic, 0 never, 1 always
   bool cap_external_recall = false, graph_external_recall = false, recall_all_pending = false;
   cudaEvent_t ev_graph_done = nullptr, ev_recall_all = nullptr;
-  int direct_max_granules = 64;   // scale of the one-CTA rule: a head of up to 2x (overlapping layers) or x/2 (chained layers)
-                                  // this many granules (text capacity included) is not split
+  static constexpr int direct_max_granules = 64;   // scale of the one-CTA rule: a head of up to 2x (overlapping layers) or x/2
+                                                   // (chained layers) this many granules (text capacity included) is not split
   // captured step
   bool graph_capturing = false;
   cudaGraph_t graph = nullptr;
@@ -307,14 +305,6 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
 #define CKC(call) do { wnw_status_t _s = (call); if (_s != WNW_OK) return fail(_s); } while (0)
 #define CKE(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { return fail(_e == cudaErrorMemoryAllocation ? WNW_ERR_OOM_DEVICE : WNW_ERR_CUDA); } } while (0)
   cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, cfg->device);
-  if (const char *e = getenv("WNW_PDL")) c->pdl_enabled = atoi(e) != 0;
-  if (const char *e = getenv("WNW_BATCH_TWO_PART")) c->batched_two_part = atoi(e) != 0;
-  if (const char *e = getenv("WNW_SELECT_OVERLAP")) c->sel_overlap_enabled = atoi(e) != 0;
-  if (const char *e = getenv("WNW_PACK")) { c->pack_granules = atoi(e); c->pack_enabled = c->pack_granules != 0; if (c->pack_granules < 0) c->pack_granules = 0; }
-  if (const char *e = getenv("WNW_FOLD_STEP_END")) c->fold_enabled = atoi(e) != 0;
-  if (const char *e = getenv("WNW_SELECT_ALL")) c->select_all_enabled = atoi(e) != 0;
-  if (const char *e = getenv("WNW_EXTERNAL_RECALL")) c->external_recall_mode = atoi(e);
-  if (const char *e = getenv("WNW_DIRECT_MAX_GRANULES")) c->direct_max_granules = atoi(e);
   CKE(configure_attn_kernels());
   CKE(configure_select_kernel());
   const int L = cfg->n_layers, Hkv = cfg->n_kv_heads, d = cfg->head_dim, nc = cfg->chunk_tokens;
@@ -567,9 +557,7 @@ extern "C" wnw_status_t wnw_destroy(wnw_cache_t *c) {
 // SM, over items sized for about one item per CTA and placed longest-first by the host.
 static int granules_per_item(const wnw_cache *c, long long total_granules, int longest_head, int n_heads, bool overlapped,
                              bool *throughput) {
-  int nw = attn_warps(false);
-  int min_gpi = nw;
-  if (const char *e = getenv("WNW_MIN_GRANULES_PER_ITEM")) min_gpi = std::max(nw, atoi(e) / nw * nw);
+  const int nw = attn_warps(false), min_gpi = nw;
   if (overlapped) {
     *throughput = false;
     const int cap = c->n_sm / 3;
@@ -577,21 +565,12 @@ static int granules_per_item(const wnw_cache *c, long long total_granules, int l
     per = std::max<long long>(per, (total_granules + cap - 1) / cap);
     return (int)((per + nw - 1) / nw * nw);
   }
-  int gpw = 2;   // granules per warp of an item
-  if (const char *e = getenv("WNW_GRANULES_PER_WARP")) gpw = std::max(1, atoi(e));
-  long long per = std::max<long long>(gpw * min_gpi, (longest_head + 31) / 32);   // few granules per warp (all in flight at once), few partials to merge
+  // two granules per warp: all of an item's bytes are in flight at once and few partials are left to merge (measured on
+  // config 1, chained: 212 us per step; one granule per warp 259 us, three 237 us)
+  long long per = std::max<long long>(2 * min_gpi, (longest_head + 31) / 32);
   per = (per + nw - 1) / nw * nw;
-  *throughput = (total_granules + per - 1) / per + n_heads > c->n_sm;
-  if (const char *e = getenv("WNW_THROUGHPUT")) *throughput = atoi(e) != 0;
-  if (!*throughput) return (int)per;
-  nw = attn_warps(true);
-  int waves = 1;
-  if (const char *e = getenv("WNW_WAVES")) waves = std::max(1, atoi(e));
-  const long long target = 2ll * c->n_sm * waves;
-  per = (total_granules + target - 1) / target;
-  per = std::max<long long>(per, (longest_head + 31) / 32);
-  per = std::max<long long>(per, 2 * nw);          // at least two granules per warp: the per-CTA overhead must amortise
-  return (int)((per + nw - 1) / nw * nw);
+  *throughput = (total_granules + per - 1) / per + n_heads > c->n_sm;   // more than one wave: build_throughput_items cuts the work
+  return (int)per;
 }
 
 // Granules of one head: n_gran its whole virtual key space, work those expected to hold data.
@@ -718,7 +697,7 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   // BATCHED layers share one launch: the work of the whole step is cut for one wave of CTAs, long heads into pieces as
   // fat as a pack of short ones, short heads packed whole
   const bool batched = overlapped && !throughput && c->layer_dependency == WNW_LAYERS_BATCHED && c->batched_target > 0 &&
-                       c->pack_enabled && attn_xpref_fits(G.g, G.d);
+                       attn_xpref_fits(G.g, G.d);
   if (batched) gpi = (c->batched_target + attn_warps(false) - 1) / attn_warps(false) * attn_warps(false);
   lw.throughput = throughput;
   lw.first_item = (int)items.size();
@@ -760,14 +739,14 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   lw.n_items = (int)items.size() - lw.first_item;
   lw.n_ctas = 0;
   lw.packed = false;
-  if (!throughput && overlapped && c->pack_enabled && attn_xpref_fits(G.g, G.d) &&
-      (c->pack_granules > 0 || lw.n_items > c->n_sm || batched)) {
+  if (!throughput && overlapped && attn_xpref_fits(G.g, G.d) &&
+      (lw.n_items > c->n_sm || batched)) {
     // One-shot CTAs of a launch that has more of them than SMs: heads that fit one CTA are packed several to a CTA
     // (consecutive ones, up to about 512 granules of work: a sequence's short heads), which then keeps its copy pipeline
     // running from one head into the next: the fixed cost of a CTA (launch, first reads, first DRAM round trip) is paid
     // once for the pack.  Pieces of split heads keep a CTA each.  Measured: batch-32 ragged 85 -> 91 % of the copy
     // bandwidth; launches with fewer CTAs than SMs lose parallelism instead (16 x 7500: 80 -> 76 %) and are left alone.
-    const int target = batched ? gpi : c->pack_granules > 0 ? c->pack_granules : 512;
+    const int target = batched ? gpi : 512;
     lw.order_off = (int)order.size();
     lw.ranges_off = (int)ranges.size();
     int pos = 0, in_pack = 0, pack_work = 0, n_packs = 0;
@@ -829,13 +808,11 @@ static wnw_status_t ensure_worklists(wnw_cache *c) {
     // Tidal heads form a second part of the launch (its CTAs follow those of the first as SMs come free), each cut the same way.
     c->batched_target = (int)std::max<long long>(32, (total * 14 / 10 + c->n_sm - 1) / c->n_sm);
     c->batched_target_tidal = (int)std::max<long long>(32, (total_tidal * 14 / 10 + c->n_sm - 1) / c->n_sm);
-    if (const char *e = getenv("WNW_BATCH_TARGET")) c->batched_target = std::max(8, atoi(e));
-    if (const char *e = getenv("WNW_BATCH_TARGET_TIDAL")) c->batched_target_tidal = std::max(8, atoi(e));
     // Where a single layer already fills the machine with CTAs of a decent size its launches stay apart (their steps
     // keep selection and recall inside the step, so nothing would be issued together anyway): the cut of INDEPENDENT.
     if ((total + total_tidal) / G.L > 64ll * c->n_sm) c->batched_target = c->batched_target_tidal = 0;
   }
-  if (c->batched_target > 0 && !getenv("WNW_BATCH_TARGET")) {
+  if (c->batched_target > 0) {
     // Whole heads and pieces come out uneven: widen the cut until the first part of the launch (the CTAs that read no slot)
     // is at most one wave; a few CTAs beyond it would each add a CTA's whole duration to the step (config 2: 152 CTAs of 184
     // granules 103 us per step, 136 CTAs of 192 granules 75 us).
@@ -1287,174 +1264,127 @@ static SelectArgs static_select_args(const wnw_cache *c, int layer) {
   return sa;
 }
 
-static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer, const void *q, const void *k_new,
-                                      const void *v_new, void *out, void *cuda_stream) {
-  if (!c || !q || !out || ((k_new == nullptr) != (v_new == nullptr))) return WNW_ERR_INVALID_ARG;
-  if (c->cfg.mode != want_mode) return WNW_ERR_STATE;
-  if (!c->in_step || layer != c->next_layer) return WNW_ERR_STATE;
-  const int has_new = k_new != nullptr;
-  if (c->appended >= 0 && c->appended != has_new) return WNW_ERR_STATE;
-  if (has_new)
-    for (int b : c->active)
-      if (c->seqs[b].T_t + 1 > c->cfg.max_text_tokens) return WNW_ERR_CAPACITY;
+// Decided once per step, at its first layer: how a captured step issues its selection, recall and attention launches.
+static void plan_step(wnw_cache *c, bool capturing, bool tiered) {
   const Geometry &G = c->geo;
-  DeviceGuard guard(c->cfg.device);
-  cudaStream_t st = (cudaStream_t)cuda_stream;
-  const int n_active = (int)c->active.size();
-  const bool tiered = want_mode == WNW_MODE_TIERED;
-  // Inside a stream capture the step is one graph: cross-step ordering comes from the join in wnw_step_end, and
-  // events recorded outside the capture must not be waited on.
-  const bool capturing = stream_is_capturing(st);
-  if (layer == 0) c->step_capturing = capturing;
-  else if (capturing != c->step_capturing) return WNW_ERR_STATE;
-  if (layer == 0) {
-    // Replayed steps of small launches take their recall out of the captured graph, so that it can overlap the next
-    // replay.  Where a launch could fill the machine, its attention CTAs would sit on their SMs while they wait for
-    // it, so recall stays inside the step there.
-    bool small = true;   // no launch can fill the machine with CTAs that wait
-    for (const LayerWork &w : c->wl_layers) small = small && !w.throughput && (w.n_ctas > 0 ? w.n_ctas : w.n_items) <= c->n_sm / 2;
-    // the selection kernel of the last layer starts after every attention kernel of the step has completed, so the
-    // selection CTA that finishes last in the step may update what those kernels read
-    const LayerInfo &last = c->layers[G.L - 1];
-    c->cap_fold = c->fold_enabled && capturing && c->graph_capturing && tiered && c->cfg.recall_mode != WNW_RECALL_INLINE &&
-                  (last.n_anchor > 0 || last.upd_count > 0);
-    c->cap_select_all = false;
-    c->cap_external_recall = capturing && c->graph_capturing && tiered && c->cfg.recall_mode != WNW_RECALL_INLINE &&
-                             (c->external_recall_mode == 1 || (c->external_recall_mode < 0 && small));
-    // With the recall outside the graph nothing inside it needs a layer's selection before the step ends: all of it
-    // goes into one launch (or two) behind the last attention kernel.
-    c->cap_select_all = c->select_all_enabled && c->cap_external_recall && c->fold_enabled && small &&
-                        (c->select_single_ok ? c->sel_map_single[1] : c->sel_map_update[1]) > 0;
-    if (c->cap_select_all) c->cap_fold = true;
-    // BATCHED layers: one launch for the whole step where nothing inside the step needs a layer's result earlier
-    bool one_shot = G.L <= MULTI_LAYERS_MAX;
-    for (const LayerWork &w : c->wl_layers) one_shot = one_shot && !w.throughput;
-    c->cap_batched = c->layer_dependency == WNW_LAYERS_BATCHED && c->batched_target > 0 && capturing && c->graph_capturing &&
-                     one_shot && (!tiered || c->cap_select_all);
-    if (c->cap_batched) c->batch_args.assign(G.L, AttnArgs{});
-    // Two parts (slot-free CTAs, then the tidal heads'): every anchor head is in the first, so the step's selection can
-    // run beside the second; the step's bookkeeping then waits for both (a step-end kernel instead of the fold).
-    c->cap_sel_overlap = false;
-    if (c->cap_batched && tiered && c->batched_two_part && c->sel_overlap_enabled && c->cap_external_recall && c->cap_select_all) {
-      bool any_free = false, any_tidal = false;
-      for (const LayerWork &w : c->wl_layers) {
-        const int n_free = w.packed ? w.n_ctas_free : 0;
-        any_free = any_free || n_free > 0;
-        any_tidal = any_tidal || n_free < (w.n_ctas > 0 ? w.n_ctas : w.n_items);
-      }
-      c->cap_sel_overlap = any_free && any_tidal;
-      if (c->cap_sel_overlap) c->cap_fold = false;
+  // Replayed steps of small launches take their recall out of the captured graph, so that it can overlap the next
+  // replay.  Where a launch could fill the machine, its attention CTAs would sit on their SMs while they wait for
+  // it, so recall stays inside the step there.
+  bool small = true;   // no launch can fill the machine with CTAs that wait
+  for (const LayerWork &w : c->wl_layers) small = small && !w.throughput && (w.n_ctas > 0 ? w.n_ctas : w.n_items) <= c->n_sm / 2;
+  // the selection kernel of the last layer starts after every attention kernel of the step has completed, so the
+  // selection CTA that finishes last in the step may update what those kernels read
+  const LayerInfo &last = c->layers[G.L - 1];
+  c->cap_fold = capturing && c->graph_capturing && tiered && c->cfg.recall_mode != WNW_RECALL_INLINE &&
+                (last.n_anchor > 0 || last.upd_count > 0);
+  c->cap_select_all = false;
+  c->cap_external_recall = capturing && c->graph_capturing && tiered && c->cfg.recall_mode != WNW_RECALL_INLINE &&
+                           small;
+  // With the recall outside the graph nothing inside it needs a layer's selection before the step ends: all of it
+  // goes into one launch (or two) behind the last attention kernel.
+  c->cap_select_all = c->cap_external_recall && small &&
+                      (c->select_single_ok ? c->sel_map_single[1] : c->sel_map_update[1]) > 0;
+  if (c->cap_select_all) c->cap_fold = true;
+  // BATCHED layers: one launch for the whole step where nothing inside the step needs a layer's result earlier
+  bool one_shot = G.L <= MULTI_LAYERS_MAX;
+  for (const LayerWork &w : c->wl_layers) one_shot = one_shot && !w.throughput;
+  c->cap_batched = c->layer_dependency == WNW_LAYERS_BATCHED && c->batched_target > 0 && capturing && c->graph_capturing &&
+                   one_shot && (!tiered || c->cap_select_all);
+  if (c->cap_batched) c->batch_args.assign(G.L, AttnArgs{});
+  // Two parts (slot-free CTAs, then the tidal heads'): every anchor head is in the first, so the step's selection can
+  // run beside the second; the step's bookkeeping then waits for both (a step-end kernel instead of the fold).
+  c->cap_sel_overlap = false;
+  if (c->cap_batched && tiered && c->cap_external_recall && c->cap_select_all) {
+    bool any_free = false, any_tidal = false;
+    for (const LayerWork &w : c->wl_layers) {
+      const int n_free = w.packed ? w.n_ctas_free : 0;
+      any_free = any_free || n_free > 0;
+      any_tidal = any_tidal || n_free < (w.n_ctas > 0 ? w.n_ctas : w.n_items);
     }
+    c->cap_sel_overlap = any_free && any_tidal;
+    if (c->cap_sel_overlap) c->cap_fold = false;
   }
-  if (!capturing) {
-    if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
-    if (layer == 0 && c->recall_all_pending) {  // the recall launch that followed the last replayed step
-      CK(cudaStreamWaitEvent(st, c->ev_recall_all, 0));
-      c->recall_all_pending = false;
-    }
-    // side-stream work of the previous step that this layer depends on must have landed: the selection kernel that
-    // read this layer's partial buffers, and the recall that refreshed this layer's slots
-    if (tiered && c->cfg.recall_mode != WNW_RECALL_INLINE) {
-      if (c->side_recorded[layer]) CK(cudaStreamWaitEvent(st, c->ev_side_done[layer], 0));
-      const int x = c->tail_of[layer];
-      if (x >= 0 && x != layer && c->side_recorded[x]) CK(cudaStreamWaitEvent(st, c->ev_side_done[x], 0));
-    }
+}
+
+// An eager layer waits for what earlier work on other streams has to have finished: placements, the recall launch that
+// followed the last replayed step, and the previous step's side-stream work on this layer's partials, table and slots.
+static wnw_status_t wait_for_earlier_steps(wnw_cache *c, int layer, bool tiered, cudaStream_t st) {
+  if (layer == 0 && c->place_recorded) CK(cudaStreamWaitEvent(st, c->ev_place, 0));
+  if (layer == 0 && c->recall_all_pending) {  // the recall launch that followed the last replayed step
+    CK(cudaStreamWaitEvent(st, c->ev_recall_all, 0));
+    c->recall_all_pending = false;
   }
-  const LayerWork &lw = c->wl_layers[layer];
-  const LayerInfo &li = c->layers[layer];
-  float2 *gran_em_l = c->gran_em + (size_t)layer * c->gran_em_layer_stride;
-  float2 *head_mz_l = c->head_mz + (size_t)layer * G.max_batch * G.Hq;
-  AttnArgs a{};
-  a.mode = tiered ? ATTN_DECODE : ATTN_FULL; a.layer = layer; a.li = li; a.n_active = n_active; a.has_new = has_new;
-  a.score_on = tiered && li.n_anchor > 0;
-  a.active = c->d_active; a.items = c->d_items + lw.first_item; a.items_host = c->h_items.data() + lw.first_item;
-  a.n_items = lw.n_items; a.maps = &c->maps_decode; a.throughput = lw.throughput;
-  if (lw.n_ctas > 0) {
-    a.order = c->d_sched + lw.order_off; a.cta_ranges = c->d_sched + c->sched_ranges_base + lw.ranges_off; a.n_ctas = lw.n_ctas;
-    a.xpref = lw.packed;
+  // side-stream work of the previous step that this layer depends on must have landed: the selection kernel that
+  // read this layer's partial buffers, and the recall that refreshed this layer's slots
+  if (tiered && c->cfg.recall_mode != WNW_RECALL_INLINE) {
+    if (c->side_recorded[layer]) CK(cudaStreamWaitEvent(st, c->ev_side_done[layer], 0));
+    const int x = c->tail_of[layer];
+    if (x >= 0 && x != layer && c->side_recorded[x]) CK(cudaStreamWaitEvent(st, c->ev_side_done[x], 0));
   }
-  a.head_items = c->d_head_items + lw.head_items_off;
-  a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
-  a.head_done = c->head_done + (size_t)layer * G.max_batch * G.Hkv; a.head_mz = head_mz_l; a.out = (bf16 *)out;
-  a.anchor_base = c->cv.anchor; a.anchor_seq_stride = G.anchor_seq_stride;
-  a.anchor_head0 = tiered ? li.anchor_off : layer * G.Hkv;
-  a.part_o = c->part_o + lw.part_off * G.g * G.d; a.part_ml = c->part_ml + lw.part_off * G.g;
-  a.gran_em = gran_em_l;
-  if (c->cap_external_recall && li.n_tidal > 0) { a.wait_epoch = c->d_recall_epoch + layer; a.expect_epoch = c->d_step_epoch; }
-  // overlap with the previous layer's kernel when that is what precedes this launch in the stream
-  a.pdl = layer > 0 && c->pdl_enabled && c->layer_dependency != WNW_LAYERS_SERIAL;
-  a.wait_inputs = a.pdl && c->layer_dependency == WNW_LAYERS_CHAINED;
-  a.n_aq = std::max(li.n_anchor * G.g, 1); a.n_ag_max = c->n_ag_max;
-  cudaEvent_t t0 = nullptr, t1 = nullptr;
-  const bool timing = c->timing && !capturing;
-  if (timing) {
-    for (cudaEvent_t *e : {&t0, &t1}) {
-      if (!c->t_free.empty()) { *e = c->t_free.back(); c->t_free.pop_back(); }
-      else CK(cudaEventCreate(e));
-    }
-    CK(cudaEventRecord(t0, st));
+  return WNW_OK;
+}
+
+// All layers of a captured step issued together (BATCHED), at the step's last layer: one launch, or the anchor heads, the
+// fixed heads and the tidal heads in turn with the step's selection forked behind the anchor heads.
+static wnw_status_t issue_batched_step(wnw_cache *c, bool tiered, bool capturing, int has_new, cudaStream_t st) {
+  const Geometry &G = c->geo;
+  // Two parts when the step has tidal heads: first the CTAs that read no slot, one wave of them; then, programmatically
+  // dependent, those of the tidal heads, which take the SMs as the first part leaves them.  The recall of the previous
+  // step (it runs outside the captured graph, beside this step) has landed by then, so no CTA sits on an SM waiting.
+  std::vector<int> zero(G.L, 0), n_anchor(G.L, 0), n_fixed(G.L, 0), n_free(G.L, 0), n_tidal(G.L, 0);
+  bool any_free = false, any_tidal = false, any_anchor = false, any_fixed = false;
+  for (int l = 0; l < G.L; ++l) {
+    const LayerWork &w = c->wl_layers[l];
+    const int all = w.n_ctas > 0 ? w.n_ctas : w.n_items;
+    n_free[l] = w.packed ? w.n_ctas_free : 0;
+    n_anchor[l] = w.packed ? w.n_ctas_anchor : 0;
+    n_fixed[l] = n_free[l] - n_anchor[l];
+    n_tidal[l] = all - n_free[l];
+    any_free = any_free || n_free[l] > 0;
+    any_tidal = any_tidal || n_tidal[l] > 0;
+    any_anchor = any_anchor || n_anchor[l] > 0;
+    any_fixed = any_fixed || n_fixed[l] > 0;
   }
-  if (c->cap_batched) {
-    c->batch_args[layer] = a;
-    if (layer == G.L - 1) {
-      // Two parts when the step has tidal heads: first the CTAs that read no slot, one wave of them; then, programmatically
-      // dependent, those of the tidal heads, which take the SMs as the first part leaves them.  The recall of the previous
-      // step (it runs outside the captured graph, beside this step) has landed by then, so no CTA sits on an SM waiting.
-      std::vector<int> zero(G.L, 0), n_anchor(G.L, 0), n_fixed(G.L, 0), n_free(G.L, 0), n_tidal(G.L, 0);
-      bool any_free = false, any_tidal = false, any_anchor = false, any_fixed = false;
-      for (int l = 0; l < G.L; ++l) {
-        const LayerWork &w = c->wl_layers[l];
-        const int all = w.n_ctas > 0 ? w.n_ctas : w.n_items;
-        n_free[l] = w.packed ? w.n_ctas_free : 0;
-        n_anchor[l] = w.packed ? w.n_ctas_anchor : 0;
-        n_fixed[l] = n_free[l] - n_anchor[l];
-        n_tidal[l] = all - n_free[l];
-        any_free = any_free || n_free[l] > 0;
-        any_tidal = any_tidal || n_tidal[l] > 0;
-        any_anchor = any_anchor || n_anchor[l] > 0;
-        any_fixed = any_fixed || n_fixed[l] > 0;
-      }
-      if (tiered && any_free && any_tidal && c->batched_two_part) {
-        // anchor heads first: the step's selection depends on them alone and is forked right behind their launch
-        const bool split_anchor = c->cap_sel_overlap && any_anchor && any_fixed;
-        int n_launch = 0;
-        if (split_anchor) {
-          CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, zero.data(), n_anchor.data(), false, st));
-          ++n_launch;
-        } else {
-          CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, zero.data(), n_free.data(), false, st));
-          ++n_launch;
-        }
-        if (c->cap_sel_overlap) {
-          c->appended = has_new;
-          CK(cudaEventRecord(c->ev_sel_fork, st));
-          CK(cudaStreamWaitEvent(c->side[0], c->ev_sel_fork, 0));
-          wnw_status_t rs = launch_step_selection(c, true, c->side[0]);
-          if (rs != WNW_OK) return rs;
-          CK(cudaEventRecord(c->ev_sel_join, c->side[0]));
-        }
-        if (split_anchor) {
-          CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_anchor.data(), n_fixed.data(), true, st));
-          ++n_launch;
-        }
-        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_free.data(), n_tidal.data(), true, st));
-        ++n_launch;
-        c->count_launch(0, n_launch, capturing);
-      } else {
-        CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, nullptr, nullptr, false, st));
-        c->count_launch(0, 1, capturing);
-      }
+  if (tiered && any_free && any_tidal) {
+    // anchor heads first: the step's selection depends on them alone and is forked right behind their launch
+    const bool split_anchor = c->cap_sel_overlap && any_anchor && any_fixed;
+    int n_launch = 0;
+    if (split_anchor) {
+      CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, zero.data(), n_anchor.data(), false, st));
+      ++n_launch;
+    } else {
+      CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, zero.data(), n_free.data(), false, st));
+      ++n_launch;
     }
+    if (c->cap_sel_overlap) {
+      c->appended = has_new;
+      CK(cudaEventRecord(c->ev_sel_fork, st));
+      CK(cudaStreamWaitEvent(c->side[0], c->ev_sel_fork, 0));
+      wnw_status_t rs = launch_step_selection(c, true, c->side[0]);
+      if (rs != WNW_OK) return rs;
+      CK(cudaEventRecord(c->ev_sel_join, c->side[0]));
+    }
+    if (split_anchor) {
+      CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_anchor.data(), n_fixed.data(), true, st));
+      ++n_launch;
+    }
+    CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, n_free.data(), n_tidal.data(), true, st));
+    ++n_launch;
+    c->count_launch(0, n_launch, capturing);
   } else {
-    CK(launch_attn(c->cv, a, st));
+    CK(launch_attn_multi(c->cv, c->batch_args.data(), G.L, nullptr, nullptr, false, st));
     c->count_launch(0, 1, capturing);
   }
-  if (timing) {
-    CK(cudaEventRecord(t1, st));
-    c->t_used.emplace_back(t0, t1);
-  }
-  // chunk scores, selection, recall: on the side stream, overlapping whatever follows on the caller's stream
-  // (captured steps of small launches do all of it in one or two launches at the end of the step instead)
+  return WNW_OK;
+}
+
+// Chunk scores, selection and recall of a layer: on a side stream, overlapping whatever follows on the caller's stream
+// (captured steps of small launches do all of it in one or two launches at the end of the step instead; head-sharded
+// caches only add up their own scores here).
+static wnw_status_t issue_side_work(wnw_cache *c, int layer, bool tiered, bool capturing, int has_new, int n_active, cudaStream_t st) {
+  const Geometry &G = c->geo;
+  (void)G;
+  const LayerInfo &li = c->layers[layer];
   const bool defer = tiered && c->cfg.defer_selection;   // head-sharded serving: scores now, everything else at the step's end
   if (defer && capturing) return WNW_ERR_UNSUPPORTED;
   if (layer == 0) c->scores_exported = c->scores_imported = false;
@@ -1501,6 +1431,86 @@ static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer
       if (!capturing) c->side_recorded[layer] = 1;
       c->last_side_layer[si] = layer;
     }
+  }
+  return WNW_OK;
+}
+
+static wnw_status_t decode_layer_impl(wnw_cache *c, int want_mode, int32_t layer, const void *q, const void *k_new,
+                                      const void *v_new, void *out, void *cuda_stream) {
+  if (!c || !q || !out || ((k_new == nullptr) != (v_new == nullptr))) return WNW_ERR_INVALID_ARG;
+  if (c->cfg.mode != want_mode) return WNW_ERR_STATE;
+  if (!c->in_step || layer != c->next_layer) return WNW_ERR_STATE;
+  const int has_new = k_new != nullptr;
+  if (c->appended >= 0 && c->appended != has_new) return WNW_ERR_STATE;
+  if (has_new)
+    for (int b : c->active)
+      if (c->seqs[b].T_t + 1 > c->cfg.max_text_tokens) return WNW_ERR_CAPACITY;
+  const Geometry &G = c->geo;
+  DeviceGuard guard(c->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const int n_active = (int)c->active.size();
+  const bool tiered = want_mode == WNW_MODE_TIERED;
+  // Inside a stream capture the step is one graph: cross-step ordering comes from the join in wnw_step_end, and
+  // events recorded outside the capture must not be waited on.
+  const bool capturing = stream_is_capturing(st);
+  if (layer == 0) c->step_capturing = capturing;
+  else if (capturing != c->step_capturing) return WNW_ERR_STATE;
+  if (layer == 0) plan_step(c, capturing, tiered);
+  if (!capturing) {
+    wnw_status_t ws = wait_for_earlier_steps(c, layer, tiered, st);
+    if (ws != WNW_OK) return ws;
+  }
+  const LayerWork &lw = c->wl_layers[layer];
+  const LayerInfo &li = c->layers[layer];
+  float2 *gran_em_l = c->gran_em + (size_t)layer * c->gran_em_layer_stride;
+  float2 *head_mz_l = c->head_mz + (size_t)layer * G.max_batch * G.Hq;
+  AttnArgs a{};
+  a.mode = tiered ? ATTN_DECODE : ATTN_FULL; a.layer = layer; a.li = li; a.n_active = n_active; a.has_new = has_new;
+  a.score_on = tiered && li.n_anchor > 0;
+  a.active = c->d_active; a.items = c->d_items + lw.first_item; a.items_host = c->h_items.data() + lw.first_item;
+  a.n_items = lw.n_items; a.maps = &c->maps_decode; a.throughput = lw.throughput;
+  if (lw.n_ctas > 0) {
+    a.order = c->d_sched + lw.order_off; a.cta_ranges = c->d_sched + c->sched_ranges_base + lw.ranges_off; a.n_ctas = lw.n_ctas;
+    a.xpref = lw.packed;
+  }
+  a.head_items = c->d_head_items + lw.head_items_off;
+  a.q = (const bf16 *)q; a.k_new = (const bf16 *)k_new; a.v_new = (const bf16 *)v_new;
+  a.head_done = c->head_done + (size_t)layer * G.max_batch * G.Hkv; a.head_mz = head_mz_l; a.out = (bf16 *)out;
+  a.anchor_base = c->cv.anchor; a.anchor_seq_stride = G.anchor_seq_stride;
+  a.anchor_head0 = tiered ? li.anchor_off : layer * G.Hkv;
+  a.part_o = c->part_o + lw.part_off * G.g * G.d; a.part_ml = c->part_ml + lw.part_off * G.g;
+  a.gran_em = gran_em_l;
+  if (c->cap_external_recall && li.n_tidal > 0) { a.wait_epoch = c->d_recall_epoch + layer; a.expect_epoch = c->d_step_epoch; }
+  // overlap with the previous layer's kernel when that is what precedes this launch in the stream
+  a.pdl = layer > 0 && c->layer_dependency != WNW_LAYERS_SERIAL;
+  a.wait_inputs = a.pdl && c->layer_dependency == WNW_LAYERS_CHAINED;
+  a.n_aq = std::max(li.n_anchor * G.g, 1); a.n_ag_max = c->n_ag_max;
+  cudaEvent_t t0 = nullptr, t1 = nullptr;
+  const bool timing = c->timing && !capturing;
+  if (timing) {
+    for (cudaEvent_t *e : {&t0, &t1}) {
+      if (!c->t_free.empty()) { *e = c->t_free.back(); c->t_free.pop_back(); }
+      else CK(cudaEventCreate(e));
+    }
+    CK(cudaEventRecord(t0, st));
+  }
+  if (c->cap_batched) {
+    c->batch_args[layer] = a;
+    if (layer == G.L - 1) {
+      wnw_status_t bs = issue_batched_step(c, tiered, capturing, has_new, st);
+      if (bs != WNW_OK) return bs;
+    }
+  } else {
+    CK(launch_attn(c->cv, a, st));
+    c->count_launch(0, 1, capturing);
+  }
+  if (timing) {
+    CK(cudaEventRecord(t1, st));
+    c->t_used.emplace_back(t0, t1);
+  }
+  {
+    wnw_status_t ss = issue_side_work(c, layer, tiered, capturing, has_new, n_active, st);
+    if (ss != WNW_OK) return ss;
   }
   c->appended = has_new;
   c->next_layer = layer + 1;

@@ -1,9 +1,9 @@
-// Device-side pieces of the decode tail: ranking key, top-k, residency update and recall plan, chunk-score
-// finalize.  Included by the fused attention kernel and by the prefill selection kernel.
+// Device-side pieces of the selection: ranking key, top-k, residency update (hard budget; segment lag) and recall plan.
+// Included by the selection kernel and the placement kernels (wnw_kernels.cu).
 //
-// The tail runs in the one CTA that finishes a sequence last, so its cost is pure latency.  Everything it reads
-// from global memory is therefore staged into shared memory by cp.async in ONE batch (one round trip), and all
-// arithmetic then runs out of shared memory in a fixed order (deterministic scores and selections).
+// The selection kernel runs one CTA per sequence on a side stream, off the attention's critical path; its cost is pure
+// latency.  Everything it reads from global memory is therefore staged into shared memory by cp.async in ONE batch (one
+// round trip), and all arithmetic then runs out of shared memory in a fixed order (deterministic scores and selections).
 #pragma once
 #include "wnw_internal.cuh"
 

@@ -13,9 +13,13 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared():
-    text = open(os.path.join(ROOT, "include", "wnw.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(wnw_[a-z_]+)\s*\(", text)))
+    """Every function declared in include/*.h (the decode path's interface and the test / measurement hooks)."""
+    import glob
+    names = set()
+    for path in glob.glob(os.path.join(ROOT, "include", "*.h")):
+        text = re.sub(r"/\*.*?\*/", "", open(path).read(), flags=re.S)
+        names |= set(re.findall(r"\b(wnw_[a-z_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_builds_and_exports_every_declared_symbol():

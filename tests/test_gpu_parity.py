@@ -151,18 +151,18 @@ def test_prefill_scores_summed_over_text_queries_config1_shape():
     _run(w, check_slots=False)
 
 
-@pytest.mark.parametrize("pack", ["48", "400"])
-def test_short_heads_packed_into_shared_ctas(monkeypatch, pack):
-    """Several short heads served by one CTA whose copy pipeline runs from one head into the next (the library does this
-    by itself only for launches with more CTAs than SMs; the environment knob forces it on small shapes)."""
-    monkeypatch.setenv("WNW_PACK", pack)
+@pytest.mark.parametrize("residency", [0, 1])
+def test_short_heads_packed_into_shared_ctas(residency):
+    """Several short heads served by one CTA whose copy pipeline runs from one head into the next: the cut of a captured
+    step whose layers are issued together, at a small shape, under the hard budget and under the lag residency."""
+    import paper_2608_22704_b200 as wnw
     roles = [[A, T, T, F, T, F, T, T], [T, F, T, F, A, T, T, F], [A, T, F, T, T, T, F, F]]
     w = tiny_custom(n_layers=3, n_q_heads=16, n_kv_heads=8, head_dim=128, n_text=9, audio_lens=(640, 300, 75), chunk=32,
                     budget=0.2, n_steps=8, roles=roles, region=32, jump_every=3)
-    _run(w, seed=8)
     from parity_harness import Lockstep
-    ls = Lockstep(w, seed=8, residency=1, evict_lag=2)
+    ls = Lockstep(w, seed=8, residency=residency, evict_lag=2)
     try:
+        wnw.wnw_set_layer_dependency(ls.h, wnw.WNW_LAYERS_BATCHED)
         ls.prefill()
         for t in range(8):
             ls.decode_step(t, graph=t >= 2, check_slots=True)
