@@ -699,6 +699,12 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   const bool batched = overlapped && !throughput && c->layer_dependency == WNW_LAYERS_BATCHED && c->batched_target > 0 &&
                        attn_xpref_fits(G.g, G.d);
   if (batched) gpi = (c->batched_target + attn_warps(false) - 1) / attn_warps(false) * attn_warps(false);
+  // Overlapping layers of a tiered cache whose launch is large but would still come out as one unpacked wave (one one-shot
+  // CTA per short head, each alone on its SM: nothing covers its start-up and its merge): two persistent 4-warp CTAs per SM
+  // cover one another's instead.  Measured on 12 layers x 16 sequences x 7500 tokens with copies skipped: 0.365 -> 0.340 ms
+  // per step.  Launches with more heads than SMs keep the packed one-shot CTAs (batch-32 ragged: 1.06 against 1.12 ms), and
+  // so does the full-cache kernel (0.878 against 0.895 ms).
+  const bool big_single_wave = overlapped && !batched && mode == ATTN_DECODE && total >= 64ll * c->n_sm;   // decided once the cut is known
   lw.throughput = throughput;
   lw.first_item = (int)items.size();
   lw.head_items_off = (int)heads.size();
@@ -739,6 +745,13 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   lw.n_items = (int)items.size() - lw.first_item;
   lw.n_ctas = 0;
   lw.packed = false;
+  if (big_single_wave && lw.n_items <= c->n_sm) {   // see above: the persistent two-per-SM cut instead
+    items.resize(lw.first_item);
+    heads.resize(lw.head_items_off);
+    lw.throughput = true;
+    build_throughput_items(c, layer, mode, seq_ids, n_gran, n_work, items, heads, lw, order, ranges);
+    return;
+  }
   if (!throughput && overlapped && attn_xpref_fits(G.g, G.d) &&
       (lw.n_items > c->n_sm || batched)) {
     // One-shot CTAs of a launch that has more of them than SMs: heads that fit one CTA are packed several to a CTA
