@@ -458,21 +458,37 @@ def run_recall_sweep(args, wnw, dev):
             job = Job(w, seed=0, device=dev, wnw=wnw)
             job.create("wnw", wnw.WNW_MODE_TIERED)
             job.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
-            job.place_all(["wnw", "skip"])
+            job.create("count", wnw.WNW_MODE_TIERED)
+            job.place_all(["wnw", "skip", "count"])
             for t in range(W):
-                job.step("wnw", t); job.step("skip", t)
+                job.step("wnw", t); job.step("skip", t); job.step("count", t)
             torch.cuda.synchronize(dev)
+            # bytes recalled by every single step (a drained run of the same steps on a cache of its own: the selections are
+            # deterministic): the jumps make the demand bursty, and a selection made at step s is used at step s+1, so the copies
+            # of a step can hide behind one step of attention at most
+            per_step, last = [], wnw.wnw_get_stats(job.caches["count"])["recall_bytes"]
+            for t in range(W, W + K):
+                job.step("count", t)
+                wnw.wnw_sync(job.caches["count"])
+                now = wnw.wnw_get_stats(job.caches["count"])["recall_bytes"]
+                per_step.append(now - last)
+                last = now
             s0 = wnw.wnw_get_stats(job.caches["wnw"])
             ms = job.timed_region("wnw", W, K)          # a step reads 1.6-3.6 GB: far more than L2 holds
             s1 = wnw.wnw_get_stats(job.caches["wnw"])
             ms_skip = job.timed_region("skip", W, K)
             rb = (s1["recall_bytes"] - s0["recall_bytes"]) / K
             T_a, _, C, S = wnw.wnw_get_seq_dims(job.caches["wnw"], 0)
+            floor_ms = sum(max(ms_skip, b / (link_kernel * 1e9) * 1e3) for b in per_step) / K
             points.append({"budget": budget, "chunk": chunk, "chunks": C, "slots": S, "step_us": ms * 1e3,
                            "step_us_copies_skipped": ms_skip * 1e3, "exposed_recall_us": (ms - ms_skip) * 1e3,
                            "recall_MB_per_step": rb / 1e6, "misses_per_step": (s1["misses"] - s0["misses"]) / K,
                            "sustained_recall_GBps": rb / (ms * 1e-3) / 1e9,
-                           "sustained_over_link": rb / (ms * 1e-3) / 1e9 / link_kernel})
+                           "sustained_over_link": rb / (ms * 1e-3) / 1e9 / link_kernel,
+                           "largest_step_recall_MB": max(per_step) / 1e6,
+                           "floor_us": floor_ms * 1e3, "step_over_floor": ms / floor_ms,
+                           "floor_note": "mean over the steps of max(step with copies skipped, that step's recalled bytes / "
+                                         "link_kernel_GBps): a step's copies are needed by the next step"})
             job.destroy()
             del job
             torch.cuda.empty_cache()

@@ -601,7 +601,7 @@ static void build_throughput_items(const wnw_cache *c, int layer, int mode, cons
   const Geometry &G = c->geo;
   const int nw = attn_warps(true), n_heads = (int)seq_ids.size() * G.Hkv;
   const double cost_whole = 5.0, cost_piece = 16.0;   // fixed cost of an item in granules' worth: finished in the CTA / left as a partial
-  const double mean_weight = 1.0;   // fixed cost of an item in granules' worth: finished in the CTA / left as a partial
+  const double mean_weight = 1.0;                     // weight of the mean CTA load beside the longest one in the objective
   const int per_sm = 2;                               // persistent CTAs per SM (4 warps, about 105 KB of shared memory each)
   double total = 0.0;
   for (int hd = 0; hd < n_heads; ++hd) total += n_work[hd];
