@@ -147,6 +147,7 @@ class Job:
     """Caches, resident inputs and launch helpers of one rank."""
 
     layer_dependency = 3   # WNW_LAYERS_*: how the layers of a step are issued (set from --layer-dependency)
+    kv_fp8 = False         # tiered caches keep their tidal tier as e4m3 (set from --tidal-kv fp8)
 
     def __init__(self, w, seed, device, wnw, score_scope=0, residency=0, evict_lag=3):
         self.score_scope = score_scope
@@ -155,6 +156,7 @@ class Job:
         self.syn = Synth(w, seed=seed, device=str(device))
         self.B = w.batch
         self.caches = {}
+        self.fp8_keys = set()
         L, n = w.n_layers, w.n_steps
         # decode inputs resident in HBM; one step is one contiguous slab [q of all layers | k_new | v_new]
         nq, nk = L * self.B * w.n_q_heads * w.head_dim, L * self.B * w.n_kv_heads * w.head_dim
@@ -177,12 +179,17 @@ class Job:
         self.stream = torch.cuda.Stream(device=device)
         self.captured = set()
 
-    def create(self, key, mode, recall_mode=0, layer_dependency=None):
+    def create(self, key, mode, recall_mode=0, layer_dependency=None, kv_fp8=None):
+        """kv_fp8: the tidal tier (host mirror, slot pool) as e4m3 with a scale per chunk; default: the job's setting."""
         w, wnw = self.w, self.wnw
+        kv_fp8 = Job.kv_fp8 if kv_fp8 is None else kv_fp8
         h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, self.B, max(w.audio_lens), w.text_capacity,
                            w.chunk, w.budget, w.roles, topk=w.topk, device=self.dev.index or 0, mode=mode,
                            recall_mode=recall_mode, score_scope=self.score_scope, residency=self.residency,
-                           evict_lag=self.evict_lag)
+                           evict_lag=self.evict_lag,
+                           tidal_kv_format=wnw.WNW_TIDAL_KV_FP8_E4M3 if kv_fp8 and mode == wnw.WNW_MODE_TIERED else wnw.WNW_TIDAL_KV_BF16)
+        if kv_fp8 and mode == wnw.WNW_MODE_TIERED:
+            self.fp8_keys.add(key)
         wnw.wnw_set_layer_dependency(h, Job.layer_dependency if layer_dependency is None else layer_dependency)
         self.caches[key] = h
         return h
@@ -296,6 +303,7 @@ class Job:
         w, wnw, h = self.w, self.wnw, self.caches[key]
         total = 0
         per_layer = []
+        half_tok = 0
         for l in range(w.n_layers):
             lb = 0
             for b in range(self.B):
@@ -310,10 +318,16 @@ class Job:
                     n_tid = int((roles == ROLE_TIDAL).sum())
                     if n_tid:
                         tab, _ = wnw.wnw_get_residency(h, b, l)
-                        tok += n_tid * (T_t + sum(clen(c) for c in tab.tolist() if c >= 0))
+                        res = sum(clen(c) for c in tab.tolist() if c >= 0)
+                        if key in self.fp8_keys:      # an e4m3 slot row is d bytes for K and d for V: half a bf16 row
+                            tok += n_tid * T_t
+                            half_tok += n_tid * res
+                        else:
+                            tok += n_tid * (T_t + res)
                     for hh in np.nonzero(roles == ROLE_FIXED)[0]:
                         tok += T_t + sum(clen(c) for c in wnw.wnw_get_fixed_set(h, b, l, int(hh)).tolist())
-                lb += tok * 4 * w.head_dim
+                lb += tok * 4 * w.head_dim + half_tok * 2 * w.head_dim
+                half_tok = 0
             per_layer.append(lb)
             total += lb
         return total, per_layer
@@ -493,6 +507,7 @@ def run_recall_sweep(args, wnw, dev):
             del job
             torch.cuda.empty_cache()
     print(json.dumps({"workload": "cfg4_recall_stress_sweep", "batch": 8, "audio_tokens": 7500, "steps": K, "warmup": W,
+                      "tidal_kv": "fp8_e4m3" if Job.kv_fp8 else "bf16",
                       "link_memcpy_GBps": link_copy, "link_kernel_GBps": link_kernel, "points": points}), flush=True)
 
 
@@ -513,13 +528,17 @@ def measure_block(wnw, dev, w, peak_gbs, steps=10, warm=3, speech_rate_sweep=0):
     job.create("wnw", wnw.WNW_MODE_TIERED)
     job.create("skip", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP)
     job.create("full", wnw.WNW_MODE_FULL)
-    job.place_all(["wnw", "skip", "full"])
+    fp8 = w.head_dim == 128
+    if fp8:   # the same workload with the tidal tier stored as e4m3 (half the recalled bytes, half the bytes tidal heads read)
+        job.create("wnw8", wnw.WNW_MODE_TIERED, kv_fp8=True)
+        job.create("skip8", wnw.WNW_MODE_TIERED, recall_mode=wnw.WNW_RECALL_SKIP, kv_fp8=True)
+    job.place_all(["wnw", "skip", "full"] + (["wnw8", "skip8"] if fp8 else []))
     out = {"workload": w.name, "layers": w.n_layers, "batch": w.batch}
     t = 0
     for form, dep in (("overlapped", wnw.WNW_LAYERS_BATCHED), ("chained", wnw.WNW_LAYERS_CHAINED)):
-        job.set_dependency(["wnw", "skip", "full"], dep)
+        job.set_dependency(["wnw", "skip", "full"] + (["wnw8", "skip8"] if fp8 else []), dep)
         for tt in range(t, t + warm):
-            for key, full in (("wnw", False), ("skip", False), ("full", True)):
+            for key, full in (("wnw", False), ("skip", False), ("full", True)) + ((("wnw8", False), ("skip8", False)) if fp8 else ()):
                 job.step(key, tt, full=full)
         t += warm
         torch.cuda.synchronize(dev)
@@ -530,9 +549,18 @@ def measure_block(wnw, dev, w, peak_gbs, steps=10, warm=3, speech_rate_sweep=0):
         ms_s = sum(job.timed_steps("skip", t, steps)) / steps
         ms_f = sum(job.timed_steps("full", t, steps, full=True)) / steps
         t += steps
+        if fp8:
+            nb8, _ = job.kv_bytes_of_step("wnw8")
+            z0 = wnw.wnw_get_stats(job.caches["wnw8"])
+            ms_w8 = sum(job.timed_steps("wnw8", t - steps, steps)) / steps
+            ms_s8 = sum(job.timed_steps("skip8", t - steps, steps)) / steps
         bb_w = job.timed_region("wnw", t, steps)
         bb_s = job.timed_region("skip", t, steps)
         job.timed_region("full", t, steps, full=True)
+        if fp8:
+            bb_w8 = job.timed_region("wnw8", t, steps)
+            bb_s8 = job.timed_region("skip8", t, steps)
+            z1 = wnw.wnw_get_stats(job.caches["wnw8"])
         t += steps
         s1 = wnw.wnw_get_stats(job.caches["wnw"])
         recall_b = (s1["recall_bytes"] - s0["recall_bytes"]) / (2 * steps)
@@ -541,6 +569,12 @@ def measure_block(wnw, dev, w, peak_gbs, steps=10, warm=3, speech_rate_sweep=0):
                              "exposed_recall_us_per_step": (bb_w - bb_s) * 1e3, "recall_MB_per_step": recall_b / 1e6,
                              "tokens_per_s": w.batch / (bb_w * 1e-3)},
                      "wnw_step_over_full_step": {"flushed": ms_w / ms_f, "copies_skipped": ms_s / ms_f}}
+        if fp8:
+            out[form]["wnw_fp8_tidal_tier"] = {
+                "copies_skipped": _peak_frac(nb8, ms_s8, peak_gbs), "ms_per_step": ms_w8, "back_to_back_ms_per_step": bb_w8,
+                "back_to_back_copies_skipped_ms": bb_s8, "exposed_recall_us_per_step": (bb_w8 - bb_s8) * 1e3,
+                "recall_MB_per_step": (z1["recall_bytes"] - z0["recall_bytes"]) / (2 * steps) / 1e6,
+                "tokens_per_s": w.batch / (bb_w8 * 1e-3), "back_to_back_over_bf16_tier": bb_w8 / bb_w}
         out["GB_per_step"], out["full_cache_GB_per_step"] = nb / 1e9, nbf / 1e9
     if speech_rate_sweep:
         # the decode focus moving at a speech-like rate (the synthetic sweep crosses the clip 10x faster): same caches
@@ -866,7 +900,8 @@ def run_ours(args, rank, world, local_rank):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": dict(workload_config(w), launch="eager" if args.eager else "cuda graph replay of the step",
                        score_scope="global" if args.score_scope else "per layer",
-                       residency="segment lag" if args.residency else "hard budget", layer_issue=dep_names[DEP]),
+                       residency="segment lag" if args.residency else "hard budget", layer_issue=dep_names[DEP],
+                       tidal_kv="fp8_e4m3" if Job.kv_fp8 else "bf16"),
         "clocks": clocks, "gpu_launches": int(sum(region_launches)),
         "launches": {"attention": region_launches[0], "selection": region_launches[1], "recall": region_launches[2],
                      "step_end": region_launches[3], "layers_per_attention_launch": w.n_layers / attn_per_step},
@@ -920,6 +955,9 @@ def main():
     ap.add_argument("--no-flush", action="store_true", help="with --quick: do not flush L2 between steps")
     ap.add_argument("--recall-mode", type=int, default=0, help="with --quick: 0 side stream, 1 inline, 2 copies skipped")
     ap.add_argument("--quick-full", action="store_true", help="with --quick: time the full-cache comparison path instead")
+    ap.add_argument("--tidal-kv", default="bf16", choices=["bf16", "fp8"],
+                    help="storage of the tidal tier in every tiered cache of the run (the default line stays bf16 and reports "
+                         "the e4m3 tier beside it in its workload blocks)")
     ap.add_argument("--score-scope", type=int, default=0, choices=[0, 1],
                     help="0: every layer ranks by its own (or the nearest) anchor heads; 1: Eq. 2's sum over all anchor layers")
     ap.add_argument("--residency", type=int, default=0, choices=[0, 1],
@@ -945,6 +983,7 @@ def main():
     global SWEEP_STEPS_OVERRIDE
     SWEEP_STEPS_OVERRIDE = args.sweep_steps
     Job.layer_dependency = args.layer_dependency
+    Job.kv_fp8 = args.tidal_kv == "fp8"
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     rank = int(os.environ.get("RANK", "0"))

@@ -98,6 +98,20 @@ enum { WNW_RESIDENCY_HARD_BUDGET = 0, WNW_RESIDENCY_SEGMENT_LAG = 1, WNW_RESIDEN
  *   2  skipped: tables update, no bytes move (timing experiments only; outputs become wrong) */
 enum { WNW_RECALL_SIDE_STREAM = 0, WNW_RECALL_INLINE = 1, WNW_RECALL_SKIP = 2 };
 
+/* Storage format of the tidal tier: the audio K,V of tidal heads in the pinned host mirror and in the GPU slot pool
+ * (KV quantisation is orthogonal to the method: Baselines paragraph, footnote on KV quantisation).
+ *   BF16      as given (default)
+ *   FP8_E4M3  one byte per element: e4m3 (4 exponent bits, bias 7, 3 mantissa bits, subnormals, largest finite 448) with
+ *             one power-of-two scale 2^e per (chunk, tidal head, K|V), e the integer with max|x| / 2^e in (224, 448]
+ *             (0 for an all-zero block); elements are x / 2^e rounded to nearest, ties to even.  Host-link bytes per
+ *             recalled chunk and the HBM bytes tidal heads read both halve.  The stored value of an element, e4m3 * 2^e,
+ *             is an exact bf16 number, and EVERYTHING the library computes for a tidal head (prefill scores included)
+ *             uses stored values, so results equal those of a BF16 cache given the stored values as input.  Text rows,
+ *             anchor heads and fixed heads stay bf16.  Needs head_dim 128, a residency other than SEGMENT_LAG_TOKEN_BASE
+ *             and streaming_audio = 0 (a growing chunk would have to be re-scaled): WNW_ERR_UNSUPPORTED otherwise.
+ *             wnw_get_slot_kv returns the stored values as bf16. */
+enum { WNW_TIDAL_KV_BF16 = 0, WNW_TIDAL_KV_FP8_E4M3 = 1 };
+
 typedef struct {
   int32_t n_layers, n_q_heads, n_kv_heads; /* n_q_heads % n_kv_heads == 0, group <= 16 */
   int32_t head_dim;                        /* 64 or 128 */
@@ -125,6 +139,7 @@ typedef struct {
   int32_t streaming_audio;                 /* 1: clips may grow after placement (wnw_append_audio): every sequence's pinned host
                                             * mirror is sized and laid out for max_audio_tokens.  0: mirrors are sized by the
                                             * placed clip and wnw_append_audio is refused */
+  int32_t tidal_kv_format;                 /* WNW_TIDAL_KV_* */
 } wnw_config_t;
 
 typedef struct {

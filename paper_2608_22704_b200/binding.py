@@ -23,6 +23,7 @@ WNW_RECALL_SIDE_STREAM, WNW_RECALL_INLINE, WNW_RECALL_SKIP = 0, 1, 2
 WNW_SCOPE_PER_LAYER, WNW_SCOPE_GLOBAL = 0, 1
 WNW_LAYERS_INDEPENDENT, WNW_LAYERS_CHAINED, WNW_LAYERS_SERIAL, WNW_LAYERS_BATCHED = 0, 1, 2, 3
 WNW_RESIDENCY_HARD_BUDGET, WNW_RESIDENCY_SEGMENT_LAG, WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE = 0, 1, 2
+WNW_TIDAL_KV_BF16, WNW_TIDAL_KV_FP8_E4M3 = 0, 1
 
 
 class wnw_config_t(C.Structure):
@@ -31,7 +32,7 @@ class wnw_config_t(C.Structure):
                 ("chunk_tokens", C.c_int32), ("topk", C.c_int32), ("evict_lag", C.c_int32), ("budget", C.c_float),
                 ("softmax_scale", C.c_float), ("roles", C.POINTER(C.c_uint8)), ("device", C.c_int32), ("mode", C.c_int32),
                 ("recall_mode", C.c_int32), ("score_scope", C.c_int32), ("residency", C.c_int32), ("defer_selection", C.c_int32),
-                ("global_anchor_layers", C.POINTER(C.c_uint8)), ("streaming_audio", C.c_int32)]
+                ("global_anchor_layers", C.POINTER(C.c_uint8)), ("streaming_audio", C.c_int32), ("tidal_kv_format", C.c_int32)]
 
 
 class wnw_stats_t(C.Structure):
@@ -140,12 +141,12 @@ def _stream(stream) -> Optional[int]:
 def wnw_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens, chunk_tokens,
                budget, roles, topk=3, evict_lag=3, softmax_scale=0.0, device=0, mode=WNW_MODE_TIERED,
                recall_mode=WNW_RECALL_SIDE_STREAM, score_scope=WNW_SCOPE_PER_LAYER, residency=WNW_RESIDENCY_HARD_BUDGET,
-               streaming_audio=0, defer_selection=0, global_anchor_layers=None) -> int:
+               streaming_audio=0, defer_selection=0, global_anchor_layers=None, tidal_kv_format=WNW_TIDAL_KV_BF16) -> int:
     roles = np.ascontiguousarray(roles, dtype=np.uint8).reshape(-1)
     cfg = wnw_config_t(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_audio_tokens, max_text_tokens,
                        chunk_tokens, topk, evict_lag, budget, softmax_scale,
                        roles.ctypes.data_as(C.POINTER(C.c_uint8)), device, mode, recall_mode, score_scope, residency,
-                       int(defer_selection), None, int(streaming_audio))
+                       int(defer_selection), None, int(streaming_audio), int(tidal_kv_format))
     if global_anchor_layers is not None:
         ga = np.ascontiguousarray(global_anchor_layers, dtype=np.uint8).reshape(-1)
         if ga.size != n_layers:

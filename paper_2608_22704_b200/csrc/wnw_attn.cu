@@ -22,6 +22,8 @@
 #include <cstring>
 #include <type_traits>
 
+#include <cuda_fp16.h>
+
 #include "wnw_internal.cuh"
 #include "wnw_tail.cuh"
 
@@ -120,6 +122,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t *>(&v);
 }
 
+// Two e4m3 bytes (low 16 bits of x) as two bf16 numbers: exact, every e4m3 value is a bf16 value.
+__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t x) {
+  uint32_t h;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;\n" : "=r"(h) : "h"((unsigned short)x));
+  const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h));
+  return pack_bf16(f.x, f.y);
+}
+
 struct GranDesc {
   int row;         // first K row of the granule in its store's 2-D view [rows][d] (V row = row + v_delta)
   int meta;        // >= 0: visible tokens, known statically; -1: text granule, needs the text length; -2: needs `cid`;
@@ -127,6 +137,7 @@ struct GranDesc {
   int cid;         // chunk id held by the slot / compact position (filled by a load that is not waited on here)
   int off;         // token offset of the granule inside its chunk
   int score_idx;   // audio granule index for score partials, -1 = none
+  int ex;          // e4m3 tidal tier: K scale exponent | V scale exponent << 8 | 1 << 16 for a slot granule (filled with the metadata)
 };
 
 // Maps granule j of a head's virtual key space [text capacity | audio] to memory WITHOUT waiting on any global load:
@@ -136,7 +147,7 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
                                                    const WorkItem &it, int j, int table_parity) {
   const Geometry &G = cv.geo;
   GranDesc r;
-  r.cid = -1; r.off = 0; r.score_idx = -1;
+  r.cid = -1; r.off = 0; r.score_idx = -1; r.ex = 0;
   if (j < G.n_tg) {
     const int tok0 = j * GR;
     r.row = (int)(text_off(G, it.b, a.layer, it.h, 0) / G.d) + tok0;
@@ -174,10 +185,13 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
   return r;
 }
 
-// TB: tidal heads keep a token-granular permanent base (their key space is [text | base blocks | dynamic slots])
+// VAR 1 (TB): tidal heads keep a token-granular permanent base (their key space is [text | base blocks | dynamic slots]);
+// VAR 2 (F8): the slot pool holds e4m3 bytes (one 16 x 128-byte box per K or V granule) with a power-of-two scale per
+//   (chunk, head, K|V): the bytes become bf16 fragments on their way from ldmatrix to mma.sync, the scales are folded into
+//   the logits and into P; the default path (VAR 0) carries none of either variant's branches.
 // bid: the CTA's index within its layer's launch (a launch may carry the CTAs of several layers back to back);
 // inl: the layer's work items when they travel in the kernel parameters, else null (read from a.items).
-template <int D, bool G16, int NW, bool TB>
+template <int D, bool G16, int NW, int VAR>
 __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a, const InlineItems *inl, const TmaMaps &maps,
                                           const int bid) {
   extern __shared__ unsigned char smem_raw[];
@@ -190,6 +204,8 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   constexpr int PPR = D / 8;              // 16-byte pieces per row
   constexpr int KK = D / 16;              // k16 steps of QK^T; also pairs of n8 tiles of PV
   constexpr int NQ = G16 ? 4 : 2;
+  constexpr bool TB = VAR == 1, F8 = VAR == 2;
+  static_assert(!F8 || D == 128, "an e4m3 row must fill one 128-byte swizzle atom");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   STAMP(0);
@@ -293,7 +309,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   int p_n = 0;
   uint32_t seq_p = 0, seq_c = 0;
   GranDesc blk;  // descriptor this lane decoded for the producer's current block of 32 granules
-  blk.row = 0; blk.meta = 0; blk.cid = -1; blk.off = 0; blk.score_idx = -1;
+  blk.row = 0; blk.meta = 0; blk.cid = -1; blk.off = 0; blk.score_idx = -1; blk.ex = 0;
 
   // Visible rows of a granule once its metadata has arrived.
   auto visible = [&](const Ctx &c, int meta, int cid, int off, int j) -> int {
@@ -321,7 +337,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     if ((n & 31) == 0) {
       const int nn = n + lane;
       if (nn < c.n_my) blk = decode_granule<TB>(cv, a, li, c.it, c.first + nn * NW, c.table_parity);
-      else { blk.meta = 0; blk.cid = -1; blk.score_idx = -1; }
+      else { blk.meta = 0; blk.cid = -1; blk.score_idx = -1; blk.ex = 0; }
 #ifdef WNW_PHASE_STAMPS
       if (n == 0 && blk.row >= 0) STAMP(12);
 #endif
@@ -343,11 +359,17 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
       const CUtensorMap *map = is_text ? &maps.text : (base_blk ? &maps.fixed : c.map_audio);
       const int vrow = row + (is_text ? v_delta_text : (base_blk ? G.FB * G.ncp : c.v_delta_audio));
       fence_proxy_async();  // the stage was last read through the generic proxy (ldmatrix)
-      mbar_expect_tx(bar, 2 * TILEB);
+      if (F8 && !is_text && c.it.role == ROLE_TIDAL) {   // an e4m3 granule: one box of 16 rows x 128 bytes each for K and V
+        mbar_expect_tx(bar, 2 * HALFB);
+        tma_load_2d(sK, map, 0, row, bar);
+        tma_load_2d(sV, map, 0, vrow, bar);
+      } else {
+        mbar_expect_tx(bar, 2 * TILEB);
 #pragma unroll
-      for (int hf = 0; hf < HALVES; ++hf) {
-        tma_load_2d(sK + hf * HALFB, map, hf * 64, row, bar);
-        tma_load_2d(sV + hf * HALFB, map, hf * 64, vrow, bar);
+        for (int hf = 0; hf < HALVES; ++hf) {
+          tma_load_2d(sK + hf * HALFB, map, hf * 64, row, bar);
+          tma_load_2d(sV + hf * HALFB, map, hf * 64, vrow, bar);
+        }
       }
     }
     return load;
@@ -358,7 +380,19 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     const int src_lane = n & 31;
     const int valid = __shfl_sync(0xffffffffu, visible(c, blk.meta, blk.cid, blk.off, c.first + (n - src_lane + lane) * NW), src_lane);
     const int sidx = __shfl_sync(0xffffffffu, blk.score_idx, src_lane);
-    if (lane == 0) ring[warp][seq % NSTAGE] = make_int2(valid | (loaded ? 256 : 0), sidx);
+    int ex = 0;
+    if (F8) {
+      // the scales of the chunks this block of 32 granules touches: one load per lane and block, once the chunk ids are there
+      if (src_lane == 0) {
+        blk.ex = 0;
+        if (n + lane < c.n_my && c.first + (n + lane) * NW >= G.n_tg && c.it.role == ROLE_TIDAL && blk.cid >= 0)
+          blk.ex = 0x10000 | *reinterpret_cast<const unsigned short *>(
+                                 cv.kv_exp + kv_exp_off(G, cv.tid_total, c.it.b, li.tid_prefix + c.it.ridx, blk.cid));
+      }
+      ex = __shfl_sync(0xffffffffu, blk.ex, src_lane);
+    }
+    // x: visible rows | copy queued << 8 | e4m3 granule << 9 | K exponent << 16 | V exponent << 24
+    if (lane == 0) ring[warp][seq % NSTAGE] = make_int2(valid | (loaded ? 256 : 0) | ((ex >> 16) << 9) | (int)(((unsigned)ex & 0xffffu) << 16), sidx);
   };
   // Fetches the producer's next granule, moving on to the CTA's next work item when this warp has none left in the
   // current one (only when the pipeline runs across items).
@@ -501,9 +535,20 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
 
   // One step of the online softmax over NU granules (16 or 32 tokens) that sit in the given stages: two granules give the
   // warp two independent chains of everything (and one max/rescale for both).
-  auto step = [&](auto nu_tag, const uint32_t (&sKs)[2], const uint32_t (&sVs)[2], const int (&valids)[2], const int (&sidxs)[2]) {
+  // fmt (e4m3 tier only): per granule 0 = bf16 tile, else 1 | K exponent << 16 | V exponent << 24 (as in the ring entry >> 9)
+  auto step = [&](auto nu_tag, const uint32_t (&sKs)[2], const uint32_t (&sVs)[2], const int (&valids)[2], const int (&sidxs)[2],
+                  const int (&fmt)[2]) {
     constexpr int NU = decltype(nu_tag)::value;
     float sT[NU][NTN][4];
+    float scu[NU], pscale[NU];   // softmax scale times the K scale of the granule; the V scale, folded into P
+#pragma unroll
+    for (int u = 0; u < NU; ++u) {
+      scu[u] = sc; pscale[u] = 1.f;
+      if (F8 && (fmt[u] & 1)) {
+        scu[u] = sc * exp2f((float)(int8_t)((fmt[u] >> 7) & 0xff));
+        pscale[u] = exp2f((float)(int8_t)((fmt[u] >> 15) & 0xff));
+      }
+    }
     {
       float sO[NU][NTN][4];   // odd k-steps: shorter dependent mma chains
 #pragma unroll
@@ -513,17 +558,44 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
 #pragma unroll
           for (int e = 0; e < 4; ++e) sT[u][nt][e] = sO[u][nt][e] = 0.f;
       const int mtx = lane >> 3, row = ((mtx >> 1) << 3) + (lane & 7);
-#pragma unroll
-      for (int kk = 0; kk < KK; ++kk) {
+      auto qk_bf16 = [&](int kk, int u) {
         const int piece = 2 * kk + (mtx & 1);
         const uint32_t off = row * 128 + (kk >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4);
+        uint32_t bk[4];   // K rows 0-7 | 8-15 of the granule x d 0-7 | 8-15 of the k-step: the A operand's four quadrants
+        ldsm_x4(bk, sKs[u] + off);
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt)
+          mma16816((kk & 1) ? sO[u][nt] : sT[u][nt], bk[0], bk[2], bk[1], bk[3], qa[kk][2 * nt], qa[kk][2 * nt + 1]);
+      };
+      if constexpr (!F8) {
+#pragma unroll
+        for (int kk = 0; kk < KK; ++kk)
+#pragma unroll
+          for (int u = 0; u < NU; ++u) qk_bf16(kk, u);
+      } else {
 #pragma unroll
         for (int u = 0; u < NU; ++u) {
-          uint32_t bk[4];   // K rows 0-7 | 8-15 of the granule x d 0-7 | 8-15 of the k-step: the A operand's four quadrants
-          ldsm_x4(bk, sKs[u] + off);
+          if (fmt[u] & 1) {
+            // e4m3 tile: rows of 128 bytes; one ldmatrix.x4 brings rows 0-7 | 8-15 x the 16-byte groups 2p | 2p+1, i.e. two
+            // k-steps; a lane's four bytes are the elements 2t, 2t+1, 2t+8, 2t+9 of the group (e4m3_store_pos)
+            const int row8 = ((mtx & 1) << 3) + (lane & 7);
 #pragma unroll
-          for (int nt = 0; nt < NTN; ++nt)
-            mma16816((kk & 1) ? sO[u][nt] : sT[u][nt], bk[0], bk[2], bk[1], bk[3], qa[kk][2 * nt], qa[kk][2 * nt + 1]);
+            for (int p = 0; p < KK / 2; ++p) {
+              uint32_t bk[4];
+              ldsm_x4(bk, sKs[u] + row8 * 128 + ((((2 * p + (mtx >> 1)) & 7) ^ (row8 & 7)) << 4));
+#pragma unroll
+              for (int hk = 0; hk < 2; ++hk) {
+                const uint32_t a0 = e4m3x2_to_bf16x2(bk[2 * hk]), a1 = e4m3x2_to_bf16x2(bk[2 * hk + 1]);
+                const uint32_t a2 = e4m3x2_to_bf16x2(bk[2 * hk] >> 16), a3 = e4m3x2_to_bf16x2(bk[2 * hk + 1] >> 16);
+#pragma unroll
+                for (int nt = 0; nt < NTN; ++nt)
+                  mma16816(hk ? sO[u][nt] : sT[u][nt], a0, a1, a2, a3, qa[2 * p + hk][2 * nt], qa[2 * p + hk][2 * nt + 1]);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < KK; ++kk) qk_bf16(kk, u);
+          }
         }
       }
 #pragma unroll
@@ -543,8 +615,8 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
 #pragma unroll
       for (int u = 0; u < NU; ++u) {
         const bool lo = r0 < valids[u], hi = r0 + 8 < valids[u];
-        v[u][0] = lo ? sT[u][nt][0] * sc : -INFINITY; v[u][1] = lo ? sT[u][nt][1] * sc : -INFINITY;
-        v[u][2] = hi ? sT[u][nt][2] * sc : -INFINITY; v[u][3] = hi ? sT[u][nt][3] * sc : -INFINITY;
+        v[u][0] = lo ? sT[u][nt][0] * scu[u] : -INFINITY; v[u][1] = lo ? sT[u][nt][1] * scu[u] : -INFINITY;
+        v[u][2] = hi ? sT[u][nt][2] * scu[u] : -INFINITY; v[u][3] = hi ? sT[u][nt][3] * scu[u] : -INFINITY;
         mxA = fmaxf(mxA, fmaxf(v[u][0], v[u][2])); mxB = fmaxf(mxB, fmaxf(v[u][1], v[u][3]));
       }
 #pragma unroll
@@ -576,7 +648,12 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
           }
         }
         // P^T tile [token][head] -> [head][token]: what the PV product wants in its B operand
-        uint32_t p01 = pack_bf16(v[u][0], v[u][1]), p23 = pack_bf16(v[u][2], v[u][3]);
+        uint32_t p01, p23;
+        if constexpr (F8) {   // the V scale of an e4m3 granule rides on P: a power of two, so rounding P to bf16 commutes with it
+          p01 = pack_bf16(v[u][0] * pscale[u], v[u][1] * pscale[u]); p23 = pack_bf16(v[u][2] * pscale[u], v[u][3] * pscale[u]);
+        } else {
+          p01 = pack_bf16(v[u][0], v[u][1]); p23 = pack_bf16(v[u][2], v[u][3]);
+        }
         asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(pb[u][nt][0]) : "r"(p01));
         asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(pb[u][nt][1]) : "r"(p23));
       }
@@ -587,16 +664,42 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     STAMP(26);
     {
       const int mtx = lane >> 3, row = ((mtx & 1) << 3) + (lane & 7);
-#pragma unroll
-      for (int t2 = 0; t2 < KK; ++t2) {
+      auto pv_bf16 = [&](int t2, int u) {
         const int piece = 2 * t2 + (mtx >> 1);
         const uint32_t off = row * 128 + (t2 >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4);
+        uint32_t bv[4];   // V^T: tokens 0-7 | 8-15 x d 0-7 | 8-15 of the 16-wide d tile, transposed on the way out of shared memory
+        ldsm_x4_t(bv, sVs[u] + off);
+#pragma unroll
+        for (int nt = 0; nt < NTN; ++nt) mma16816(oT[nt][t2], bv[0], bv[2], bv[1], bv[3], pb[u][nt][0], pb[u][nt][1]);
+      };
+      if constexpr (!F8) {
+#pragma unroll
+        for (int t2 = 0; t2 < KK; ++t2)
+#pragma unroll
+          for (int u = 0; u < NU; ++u) pv_bf16(t2, u);
+      } else {
 #pragma unroll
         for (int u = 0; u < NU; ++u) {
-          uint32_t bv[4];   // V^T: tokens 0-7 | 8-15 x d 0-7 | 8-15 of the 16-wide d tile, transposed on the way out of shared memory
-          ldsm_x4_t(bv, sVs[u] + off);
+          if (fmt[u] & 1) {
+            // e4m3 tile, transposed in 16-bit units: a lane gets tokens 2t, 2t+1 of the unit (bytes 2r, 2r+1 of the group) that
+            // holds the elements r and r+8 of the d-tile: one byte permute sorts them into the two accumulator rows
 #pragma unroll
-          for (int nt = 0; nt < NTN; ++nt) mma16816(oT[nt][t2], bv[0], bv[2], bv[1], bv[3], pb[u][nt][0], pb[u][nt][1]);
+            for (int p = 0; p < KK / 2; ++p) {
+              uint32_t bv[4];   // tokens 0-7 | 8-15 x the 16-byte groups 2p | 2p+1 (two d-tiles)
+              ldsm_x4_t(bv, sVs[u] + row * 128 + ((((2 * p + (mtx >> 1)) & 7) ^ (row & 7)) << 4));
+#pragma unroll
+              for (int hk = 0; hk < 2; ++hk) {
+                const uint32_t x0 = __byte_perm(bv[2 * hk], 0, 0x3120), x1 = __byte_perm(bv[2 * hk + 1], 0, 0x3120);
+                const uint32_t a0 = e4m3x2_to_bf16x2(x0), a1 = e4m3x2_to_bf16x2(x0 >> 16);
+                const uint32_t a2 = e4m3x2_to_bf16x2(x1), a3 = e4m3x2_to_bf16x2(x1 >> 16);
+#pragma unroll
+                for (int nt = 0; nt < NTN; ++nt) mma16816(oT[nt][2 * p + hk], a0, a1, a2, a3, pb[u][nt][0], pb[u][nt][1]);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int t2 = 0; t2 < KK; ++t2) pv_bf16(t2, u);
+          }
         }
       }
     }
@@ -608,7 +711,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     // up to two granules per step; a granule with nothing visible (an empty slot, text capacity not yet written) is passed over
     const int cnt = n + 1 < n_my ? 2 : 1;
     uint32_t sKs[2] = {0u, 0u}, sVs[2] = {0u, 0u};
-    int valids[2] = {0, 0}, sidxs[2] = {-1, -1};
+    int valids[2] = {0, 0}, sidxs[2] = {-1, -1}, fmt[2] = {0, 0};
     int nu = 0, adv = 0;
     if (n == 0) STAMP(18);
 #pragma unroll
@@ -648,8 +751,8 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
               for (int hf = 0; hf < HALVES; ++hf)
                 asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};\n" ::"r"(sV + hf * HALFB + r * 128 + ((lane & 7) << 4)), "r"(0u) : "memory");
           }
-          if (nu == 0) { sKs[0] = sK; sVs[0] = sV; valids[0] = valid; sidxs[0] = rg.y; }
-          else { sKs[1] = sK; sVs[1] = sV; valids[1] = valid; sidxs[1] = rg.y; }
+          if (nu == 0) { sKs[0] = sK; sVs[0] = sV; valids[0] = valid; sidxs[0] = rg.y; fmt[0] = rg.x >> 9; }
+          else { sKs[1] = sK; sVs[1] = sV; valids[1] = valid; sidxs[1] = rg.y; fmt[1] = rg.x >> 9; }
           ++nu;
         }
       }
@@ -658,8 +761,8 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     if (n == 0) STAMP(7);
     if (timed_out) { seq_c += adv; break; }   // the stages whose bytes never came are drained (bounded) before the CTA ends
     {
-      if (nu == 2) step(std::integral_constant<int, 2>{}, sKs, sVs, valids, sidxs);
-      else if (nu == 1) step(std::integral_constant<int, 1>{}, sKs, sVs, valids, sidxs);
+      if (nu == 2) step(std::integral_constant<int, 2>{}, sKs, sVs, valids, sidxs, fmt);
+      else if (nu == 1) step(std::integral_constant<int, 1>{}, sKs, sVs, valids, sidxs, fmt);
     }
     __syncwarp();
     if (n == 0) STAMP(8);
@@ -831,12 +934,12 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   pdl_finish();
 }
 
-template <int D, bool G16, int NW, bool TB>
+template <int D, bool G16, int NW, int VAR>
 __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant__ CacheView cv,
                                                            const __grid_constant__ AttnArgs a,
                                                            const __grid_constant__ InlineItems inl,
                                                            const __grid_constant__ TmaMaps maps) {
-  attn_body<D, G16, NW, TB>(cv, a, &inl, maps, (int)blockIdx.x);
+  attn_body<D, G16, NW, VAR>(cv, a, &inl, maps, (int)blockIdx.x);
 }
 
 // The CTAs of several layers in one launch (layers whose inputs are all ready and whose outputs are read after the
@@ -846,16 +949,16 @@ __global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant
 // the recall of the previous step runs while this launch fills the machine.  (The layer's arguments are read through a
 // run-time index into the parameters, which costs registers: uncapped this kernel takes about 240, and the recall then
 // waits for attention CTAs to retire: config 1 back to back 84 us per step.)
-template <int D, bool G16, int NW, bool TB>
+template <int D, bool G16, int NW, int VAR>
 __global__ void __maxnreg__(NW == 8 ? 208 : 255) wnw_attn_multi_kernel(const __grid_constant__ CacheView cv,
                                                                  const __grid_constant__ MultiArgs m,
                                                                  const __grid_constant__ TmaMaps maps) {
   int l = 0;
   while (l + 1 < m.n && (int)blockIdx.x >= m.cta_prefix[l + 1]) ++l;
-  attn_body<D, G16, NW, TB>(cv, m.l[l], nullptr, maps, (int)blockIdx.x - m.cta_prefix[l] + m.cta_first[l]);
+  attn_body<D, G16, NW, VAR>(cv, m.l[l], nullptr, maps, (int)blockIdx.x - m.cta_prefix[l] + m.cta_first[l]);
 }
 
-template <int D, bool G16, int NW, bool TB>
+template <int D, bool G16, int NW, int VAR>
 static cudaError_t launch_multi_tb(const CacheView &cv, const MultiArgs &m, size_t smem, const TmaMaps &maps, bool pdl,
                                    cudaStream_t st) {
   cudaLaunchConfig_t cfg{};
@@ -869,10 +972,10 @@ static cudaError_t launch_multi_tb(const CacheView &cv, const MultiArgs &m, size
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
   }
-  return cudaLaunchKernelEx(&cfg, wnw_attn_multi_kernel<D, G16, NW, TB>, cv, m, maps);
+  return cudaLaunchKernelEx(&cfg, wnw_attn_multi_kernel<D, G16, NW, VAR>, cv, m, maps);
 }
 
-template <int D, bool G16, int NW, bool TB>
+template <int D, bool G16, int NW, int VAR>
 static cudaError_t launch_tb(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
   // stages + slack to align them to the swizzle atom + the merge scratch when it does not alias the stages
   const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024 + (a.xpref ? attn_scratch_bytes(NW, cv.geo.g, D) : 0);
@@ -891,11 +994,14 @@ static cudaError_t launch_tb(const CacheView &cv, const AttnArgs &a, cudaStream_
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
   }
-  return cudaLaunchKernelEx(&cfg, wnw_attn_kernel<D, G16, NW, TB>, cv, a, inl, *a.maps);
+  return cudaLaunchKernelEx(&cfg, wnw_attn_kernel<D, G16, NW, VAR>, cv, a, inl, *a.maps);
 }
 template <int D, bool G16, int NW>
 static cudaError_t launch_t(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
-  return cv.geo.token_base ? launch_tb<D, G16, NW, true>(cv, a, st) : launch_tb<D, G16, NW, false>(cv, a, st);
+  if constexpr (D == 128)
+    if (cv.geo.kv8) return launch_tb<D, G16, NW, 2>(cv, a, st);
+  if (cv.geo.kv8) return cudaErrorInvalidValue;
+  return cv.geo.token_base ? launch_tb<D, G16, NW, 1>(cv, a, st) : launch_tb<D, G16, NW, 0>(cv, a, st);
 }
 
 // ---- TMA descriptors ----
@@ -903,7 +1009,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d) {
+static EncodeTiledFn tiled_encoder() {
   static EncodeTiledFn fn = nullptr;
   if (!fn) {  // the driver entry point is looked up at run time: the library does not link against libcuda
     void *p = nullptr;
@@ -911,10 +1017,16 @@ bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long row
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess || !p ||
         qres != cudaDriverEntryPointSuccess) {
       cudaGetLastError();
-      return false;
+      return nullptr;
     }
     fn = (EncodeTiledFn)p;
   }
+  return fn;
+}
+
+bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d) {
+  const EncodeTiledFn fn = tiled_encoder();
+  if (!fn) return false;
   if (rows < 1) rows = 1;
   const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)d * 2};          // bytes between rows
@@ -925,15 +1037,33 @@ bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long row
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The slot pool of an e4m3 tidal tier: rows of 128 one-byte elements (head_dim 128), boxes of 16 rows, 128-byte swizzle.
+bool encode_store_map_e4m3(CUtensorMap *map, const void *base, unsigned long long rows) {
+  const EncodeTiledFn fn = tiled_encoder();
+  if (!fn) return false;
+  if (rows < 1) rows = 1;
+  const cuuint64_t dims[2] = {128, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {128, (cuuint32_t)GR};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int D, bool G16, int NW>
 static cudaError_t configure_t() {
   const size_t want = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024 + attn_scratch_bytes(NW, G16 ? 16 : 8, D);
   const int bytes = (int)std::min<size_t>(want, 227 * 1024 - 512);   // what a CTA may have, less this kernel's static shared memory
-  cudaError_t e = cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  cudaError_t e = cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(wnw_attn_multi_kernel<D, G16, NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(wnw_attn_multi_kernel<D, G16, NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;
-  return cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if ((e = cudaFuncSetAttribute(wnw_attn_multi_kernel<D, G16, NW, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(wnw_attn_multi_kernel<D, G16, NW, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;
+  if constexpr (D == 128) {   // the e4m3 tidal tier
+    if ((e = cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(wnw_attn_multi_kernel<D, G16, NW, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;
+  }
+  return cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 // Opt-in shared-memory sizes, set once per device at cache creation (never during a stream capture).
 cudaError_t configure_attn_kernels() {
@@ -990,13 +1120,15 @@ cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, 
   m.n = n_used; m.cta_prefix[n_used] = ctas;
   const bool g16 = cv.geo.g > 8, tb = cv.geo.token_base != 0;
   const TmaMaps &maps = *args[0].maps;
+  if (d == 128 && cv.geo.kv8)
+    return g16 ? launch_multi_tb<128, true, NW_LAT, 2>(cv, m, smem, maps, pdl, st) : launch_multi_tb<128, false, NW_LAT, 2>(cv, m, smem, maps, pdl, st);
   if (d == 128) {
-    if (g16) return tb ? launch_multi_tb<128, true, NW_LAT, true>(cv, m, smem, maps, pdl, st) : launch_multi_tb<128, true, NW_LAT, false>(cv, m, smem, maps, pdl, st);
-    return tb ? launch_multi_tb<128, false, NW_LAT, true>(cv, m, smem, maps, pdl, st) : launch_multi_tb<128, false, NW_LAT, false>(cv, m, smem, maps, pdl, st);
+    if (g16) return tb ? launch_multi_tb<128, true, NW_LAT, 1>(cv, m, smem, maps, pdl, st) : launch_multi_tb<128, true, NW_LAT, 0>(cv, m, smem, maps, pdl, st);
+    return tb ? launch_multi_tb<128, false, NW_LAT, 1>(cv, m, smem, maps, pdl, st) : launch_multi_tb<128, false, NW_LAT, 0>(cv, m, smem, maps, pdl, st);
   }
-  if (d == 64) {
-    if (g16) return tb ? launch_multi_tb<64, true, NW_LAT, true>(cv, m, smem, maps, pdl, st) : launch_multi_tb<64, true, NW_LAT, false>(cv, m, smem, maps, pdl, st);
-    return tb ? launch_multi_tb<64, false, NW_LAT, true>(cv, m, smem, maps, pdl, st) : launch_multi_tb<64, false, NW_LAT, false>(cv, m, smem, maps, pdl, st);
+  if (d == 64 && !cv.geo.kv8) {
+    if (g16) return tb ? launch_multi_tb<64, true, NW_LAT, 1>(cv, m, smem, maps, pdl, st) : launch_multi_tb<64, true, NW_LAT, 0>(cv, m, smem, maps, pdl, st);
+    return tb ? launch_multi_tb<64, false, NW_LAT, 1>(cv, m, smem, maps, pdl, st) : launch_multi_tb<64, false, NW_LAT, 0>(cv, m, smem, maps, pdl, st);
   }
   return cudaErrorInvalidValue;
 }

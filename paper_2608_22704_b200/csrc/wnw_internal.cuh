@@ -62,6 +62,7 @@ struct Geometry {
   int32_t lag_mode, delta, plan_cap;  // SEGMENT_LAG residency; its eviction lag; plan entries per (sequence, layer)
   int32_t max_batch;
   int32_t mirror_chunks;           // chunks a host mirror is laid out for: 0 = those of the placed clip, else the capacity (streaming audio)
+  int32_t kv8;                     // the tidal tier (host mirror, slot pool) holds e4m3 bytes with a power-of-two scale per (chunk, head, K|V)
   long long text_seq_stride, anchor_seq_stride, pool_seq_stride, fixed_seq_stride;  // elements
   float scale_log2;                // softmax scale * log2(e)
 };
@@ -96,6 +97,7 @@ struct CacheView {
   float *pre;                        // [B][L][Hkv][C_max]
   unsigned long long *stats;         // [B][4] hits, misses, evictions, recall_bytes
   bf16 **mirror;                     // [B] pinned host mirrors (device-visible addresses)
+  int8_t *kv_exp;                    // [B][tidal heads over all layers][C_max][K|V] e4m3 tidal tier: the chunk's scale exponent
   int32_t *status;
 };
 
@@ -124,6 +126,24 @@ __host__ __device__ inline long long compact_off(const Geometry &G, int b, int h
 __host__ __device__ inline int mirror_chunks_of(const Geometry &G, int C_b) { return G.mirror_chunks ? G.mirror_chunks : C_b; }
 __host__ __device__ inline long long mirror_off(const Geometry &G, const LayerInfo &li, int C_b, int c, int t_idx, int kv) {
   return (((long long)C_b * li.tid_prefix + (long long)c * li.n_tidal + t_idx) * 2 + kv) * G.ncp * G.d;
+}
+
+// ---- e4m3 tidal tier ----
+// Offsets into the pool and the mirrors count ELEMENTS; an element is one byte there (two as bf16).
+__host__ __device__ inline int tidal_elem_bytes(const Geometry &G) { return G.kv8 ? 1 : 2; }
+__host__ __device__ inline long long kv_exp_off(const Geometry &G, int tid_total, int b, int tidal_head, int chunk) {
+  return (((long long)b * tid_total + tidal_head) * G.C_max + chunk) * 2;
+}
+// Where element e (0..15) of a 16-element group of a row sits among the group's 16 bytes.  The order is chosen so that
+// ldmatrix on the byte tile hands every lane exactly the elements its mma fragment wants:
+//   K rows (A operand of S^T = K q^T, not transposed): lane t of a quad gets bytes 4t..4t+3 and needs elements
+//     2t, 2t+1 (k-columns of its first register) and 2t+8, 2t+9 (of its third);
+//   V rows (A operand of O^T = V^T P^T, transposed on the way out of shared memory in 16-bit units): the unit a lane
+//     gets holds the elements j and j+8 of the d-tile (its accumulator rows).
+__host__ __device__ inline int e4m3_store_pos(int kv, int e) {
+  if (kv) return (e & 7) * 2 + (e >> 3);
+  const int t = (e & 7) >> 1;
+  return 4 * t + (e & 1) + ((e >> 3) << 1);
 }
 
 // shared-memory workspace of one table update in the selection kernel: keys[C] u64, stamp[S] i64, slot[S] i32, scores[C] f32
@@ -265,6 +285,11 @@ cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, 
                               cudaStream_t st);
 // Encodes the descriptor of one store: base (device), rows, head_dim.  Returns false if the driver refuses.
 bool encode_store_map(CUtensorMap *map, const void *base, unsigned long long rows, int d);
+// the slot pool as e4m3: rows of 128 bytes, boxes of 16 rows, 128-byte swizzle
+bool encode_store_map_e4m3(CUtensorMap *map, const void *base, unsigned long long rows);
+// e4m3 tidal tier, at placement: per (chunk, tidal head, K|V) the scale exponent from the staged rows, which are then
+// replaced by the values their bytes decode to
+cudaError_t launch_quantise_stage(const CacheView &cv, int b, int layer, bf16 *stage, int C_b, cudaStream_t st);
 cudaError_t configure_select_kernel();
 constexpr int SELECT_SMEM_CAP = 200 * 1024;  // dynamic shared memory the selection kernel may be launched with
 bool attn_xpref_fits(int g, int d);  // a one-shot CTA can hold its merge scratch behind the copy stages

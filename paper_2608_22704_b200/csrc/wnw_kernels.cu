@@ -1,8 +1,15 @@
 // Recall, step bookkeeping and prefill placement kernels (sm_100a).
+#include <cuda_fp8.h>
+
 #include "wnw_internal.cuh"
 #include "wnw_tail.cuh"
 
 namespace wnw {
+
+// Address of element `off` of a tidal-tier store (slot pool, host mirror): bf16 elements, or single bytes as e4m3.
+__device__ __forceinline__ char *tier_ptr(const Geometry &G, bf16 *base, long long off) {
+  return reinterpret_cast<char *>(base) + off * tidal_elem_bytes(G);
+}
 
 // ------------------------------------------------------------------------------------------------
 // Selection (side stream): grid (n_active), one CTA per sequence.  "Decode-Step Score Aggregation" summed per
@@ -331,7 +338,7 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
       if (seen >= sig.publish_epoch) continue;
     }
     const LayerInfo &li = cv.layers[l];
-    const int n = li.n_tidal * 2 * G.ncp * G.d / 8;  // 16-byte vectors per chunk block (far below 2^31)
+    const int n = li.n_tidal * 2 * G.ncp * G.d * tidal_elem_bytes(G) / 16;  // 16-byte vectors per chunk block (far below 2^31)
     bool copies = false;                             // uniform over the whole grid: the plans do not change under this kernel
     for (int i = 0; i < n_active; ++i) {
       const int b = active[i];
@@ -346,8 +353,8 @@ __global__ void __launch_bounds__(256, 6) wnw_recall_kernel(const __grid_constan
           if (threadIdx.x == 0) atomicOr(cv.status, STATUS_BAD_TABLE);
           continue;
         }
-        const uint4 *src = reinterpret_cast<const uint4 *>(cv.mirror[b] + mirror_off(G, li, mirror_chunks_of(G, cv.C[b]), c, 0, 0));
-        uint4 *dst = reinterpret_cast<uint4 *>(cv.pool + pool_off(G, li, b, slot, 0, 0));
+        const uint4 *src = reinterpret_cast<const uint4 *>(tier_ptr(G, cv.mirror[b], mirror_off(G, li, mirror_chunks_of(G, cv.C[b]), c, 0, 0)));
+        uint4 *dst = reinterpret_cast<uint4 *>(tier_ptr(G, cv.pool, pool_off(G, li, b, slot, 0, 0)));
         for (int v0 = rank * blockDim.x + threadIdx.x; v0 < n; v0 += stride * U) {
           uint4 t[U];
 #pragma unroll
@@ -662,9 +669,9 @@ __global__ void wnw_refill_slots_kernel(const __grid_constant__ CacheView cv, in
   const long long bl = (long long)b * G.L + layer;
   const int slot = blockIdx.x, c = cv.slot_chunk[slot_table_off(G, (int)(cv.steps[b] & 1), bl) + slot];
   if (c < 0 || li.n_tidal == 0) return;
-  const long long n_vec = (long long)li.n_tidal * 2 * G.ncp * G.d / 8;
-  const uint4 *src = reinterpret_cast<const uint4 *>(cv.mirror[b] + mirror_off(G, li, mirror_chunks_of(G, cv.C[b]), c, 0, 0));
-  uint4 *dst = reinterpret_cast<uint4 *>(cv.pool + pool_off(G, li, b, slot, 0, 0));
+  const long long n_vec = (long long)li.n_tidal * 2 * G.ncp * G.d * tidal_elem_bytes(G) / 16;
+  const uint4 *src = reinterpret_cast<const uint4 *>(tier_ptr(G, cv.mirror[b], mirror_off(G, li, mirror_chunks_of(G, cv.C[b]), c, 0, 0)));
+  uint4 *dst = reinterpret_cast<uint4 *>(tier_ptr(G, cv.pool, pool_off(G, li, b, slot, 0, 0)));
   for (long long i = threadIdx.x; i < n_vec; i += blockDim.x) dst[i] = src[i];
 }
 // Head-sharded step: grid (active sequence, layer).  Out: the cache's own partial sums of the layer's chunk scores, a zero
@@ -724,6 +731,27 @@ __global__ void __launch_bounds__(128) wnw_place_gather_kernel(const __grid_cons
       if (cv.fixed_chunks[fh * G.FB + s] == c) pos = s;
     if (pos < 0) return;
     for (int kv = 0; kv < 2; ++kv) dst0[kv] = cv.fixed + fixed_off(G, li, b, ridx, kv) + (long long)pos * G.ncp * G.d;
+  } else if (G.kv8) {
+    // e4m3 tidal tier: the staged rows already hold values on the e4m3 grid of the chunk's scale (wnw_quantise_stage_kernel),
+    // so the conversion is exact; bytes go out in the order the decode kernel's ldmatrix wants (e4m3_store_pos)
+    const int slot = cv.chunk_slot[bl * G.C_max + c];
+    const int groups = G.ncp * G.d / 16;
+    for (int kv = 0; kv < 2; ++kv) {
+      const float inv = exp2f(-(float)cv.kv_exp[kv_exp_off(G, cv.tid_total, b, li.tid_prefix + ridx, c) + kv]);
+      const bf16 *src = stage + anchor_off(G, 0, 0, h, kv) + (long long)c * G.ncp * G.d;
+      uint4 *m = reinterpret_cast<uint4 *>(tier_ptr(G, cv.mirror[b], mirror_off(G, li, mirror_chunks_of(G, cv.C[b]), c, ridx, kv)));
+      uint4 *p = slot >= 0 ? reinterpret_cast<uint4 *>(tier_ptr(G, cv.pool, pool_off(G, li, b, slot, ridx, kv))) : nullptr;
+      for (int gidx = threadIdx.x; gidx < groups; gidx += blockDim.x) {
+        union { uint4 v; uint8_t b[16]; } out;
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+          out.b[e4m3_store_pos(kv, e)] =
+              (uint8_t)__nv_cvt_float_to_fp8(__bfloat162float(src[(long long)gidx * 16 + e]) * inv, __NV_SATFINITE, __NV_E4M3);
+        m[gidx] = out.v;
+        if (p) p[gidx] = out.v;
+      }
+    }
+    return;
   } else {
     const int slot = cv.chunk_slot[bl * G.C_max + c];
     for (int kv = 0; kv < 2; ++kv) {
@@ -741,6 +769,45 @@ __global__ void __launch_bounds__(128) wnw_place_gather_kernel(const __grid_cons
     }
   }
 }
+// e4m3 tidal tier, grid (C_b, Hkv), CTAs of tidal heads only.  Per K and V of one chunk of one head: the largest magnitude of
+// the staged rows gives the scale exponent e (the integer with max / 2^e in (224, 448], e4m3's top binade; 0 for an all-zero
+// block), and every staged element is replaced by e4m3(x / 2^e) * 2^e, rounded to nearest even: the value its byte will
+// decode to, an exact bf16 number.
+__global__ void __launch_bounds__(128) wnw_quantise_stage_kernel(const __grid_constant__ CacheView cv, int b, int layer, bf16 *stage) {
+  const Geometry &G = cv.geo;
+  const int c = blockIdx.x, h = blockIdx.y;
+  if (cv.roles[layer * G.Hkv + h] != ROLE_TIDAL) return;
+  const LayerInfo li = cv.layers[layer];
+  const int ridx = cv.role_idx[layer * G.Hkv + h], n = G.ncp * G.d;
+  __shared__ unsigned int s_max[4];
+  for (int kv = 0; kv < 2; ++kv) {
+    bf16 *rows = stage + anchor_off(G, 0, 0, h, kv) + (long long)c * G.ncp * G.d;
+    unsigned int mx = 0;   // magnitudes of finite bf16 numbers order like their bit patterns
+    for (int i = threadIdx.x; i < n; i += blockDim.x) mx = max(mx, (unsigned int)(__bfloat16_as_ushort(rows[i]) & 0x7fffu));
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = max(max(s_max[0], s_max[1]), max(s_max[2], s_max[3]));
+    __syncthreads();
+    int e = 0;
+    if (mx) {   // max = 1.m * 2^x; 448 = 1.75 * 2^8
+      e = (int)(mx >> 7) - 127 - 8 + ((mx & 0x7fu) > 96u ? 1 : 0);
+      e = e < -127 ? -127 : (e > 127 ? 127 : e);
+    }
+    if (threadIdx.x == 0) cv.kv_exp[kv_exp_off(G, cv.tid_total, b, li.tid_prefix + ridx, c) + kv] = (int8_t)e;
+    const float inv = exp2f(-(float)e), sc = exp2f((float)e);
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      const __nv_fp8_storage_t q = __nv_cvt_float_to_fp8(__bfloat162float(rows[i]) * inv, __NV_SATFINITE, __NV_E4M3);
+      rows[i] = __float2bfloat16_rn(__half2float(__half(__nv_cvt_fp8_to_halfraw(q, __NV_E4M3))) * sc);
+    }
+  }
+}
+cudaError_t launch_quantise_stage(const CacheView &cv, int b, int layer, bf16 *stage, int C_b, cudaStream_t st) {
+  if (C_b <= 0 || cv.layers == nullptr) return cudaSuccess;
+  wnw_quantise_stage_kernel<<<dim3(C_b, cv.geo.Hkv), 128, 0, st>>>(cv, b, layer, stage);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_place_gather(const CacheView &cv, int b, int layer, int full_mode, const bf16 *stage, int C_b,
                                   cudaStream_t st) {
   if (C_b <= 0) return cudaSuccess;

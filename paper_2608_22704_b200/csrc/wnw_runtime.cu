@@ -284,6 +284,11 @@ static wnw_status_t validate_config(const wnw_config_t *cfg) {
     for (int l = 0; l < cfg->n_layers; ++l) any_anchor |= cfg->global_anchor_layers[l] != 0;
   if (cfg->mode == WNW_MODE_TIERED && any_tidal && !any_anchor) return WNW_ERR_INVALID_ARG;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return WNW_ERR_UNSUPPORTED;
+  if (cfg->tidal_kv_format != WNW_TIDAL_KV_BF16 && cfg->tidal_kv_format != WNW_TIDAL_KV_FP8_E4M3) return WNW_ERR_INVALID_ARG;
+  // e4m3 tidal tier: one swizzle atom per row (head_dim 128); a chunk's scale is fixed when the chunk is placed
+  if (cfg->mode == WNW_MODE_TIERED && cfg->tidal_kv_format == WNW_TIDAL_KV_FP8_E4M3 &&
+      (cfg->head_dim != 128 || cfg->residency == WNW_RESIDENCY_SEGMENT_LAG_TOKEN_BASE || cfg->streaming_audio))
+    return WNW_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > MAX_G || cfg->n_q_heads > MAX_AQ || cfg->n_layers > 32767) return WNW_ERR_UNSUPPORTED;
   return WNW_OK;
 }
@@ -333,6 +338,7 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   G.T_a_pad = std::max(G.C_max, 1) * G.ncp;
   G.max_batch = cfg->max_batch;
   G.mirror_chunks = (!full && cfg->streaming_audio) ? G.C_max : 0;
+  G.kv8 = !full && cfg->tidal_kv_format == WNW_TIDAL_KV_FP8_E4M3;
   const double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / std::sqrt((double)d);
   G.scale_log2 = (float)(scale * 1.4426950408889634);
   // roles -> per-layer tables, score routing, update lists
@@ -399,7 +405,8 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
   }
   CKC(dev_alloc(c, &cv.text, B * (size_t)G.text_seq_stride));
   CKC(dev_alloc(c, &cv.anchor, B * (size_t)G.anchor_seq_stride));
-  CKC(dev_alloc(c, &cv.pool, B * (size_t)G.pool_seq_stride));
+  CKC(dev_alloc(c, &cv.pool, G.kv8 ? (B * (size_t)G.pool_seq_stride + 1) / 2 : B * (size_t)G.pool_seq_stride));   // one byte per element as e4m3
+  CKC(dev_alloc(c, &cv.kv_exp, G.kv8 ? B * (size_t)std::max(t_tot, 1) * std::max(G.C_max, 1) * 2 : 1));
   CKC(dev_alloc(c, &cv.fixed, B * (size_t)G.fixed_seq_stride));
   CKC(dev_alloc(c, &c->stage, (size_t)Hkv * 2 * G.T_a_pad * d));
   CKC(dev_alloc(c, &cv.text_len, B)); CKC(dev_alloc(c, &cv.T_a, B)); CKC(dev_alloc(c, &cv.C, B)); CKC(dev_alloc(c, &cv.S, B));
@@ -462,7 +469,8 @@ extern "C" wnw_status_t wnw_create(const wnw_config_t *cfg, wnw_cache_t **out) {
     if (std::max({r_text, r_anchor, r_pool, r_fixed}) >= (1ull << 31)) return fail(WNW_ERR_UNSUPPORTED);  // rows are 32-bit TMA coordinates
     bool ok = encode_store_map(&c->maps_decode.text, cv.text, r_text, d);
     ok = ok && encode_store_map(&c->maps_decode.anchor, cv.anchor, r_anchor, d);
-    ok = ok && encode_store_map(&c->maps_decode.pool, r_pool ? (void *)cv.pool : (void *)cv.text, r_pool ? r_pool : r_text, d);
+    if (G.kv8 && r_pool) ok = ok && encode_store_map_e4m3(&c->maps_decode.pool, cv.pool, r_pool);
+    else ok = ok && encode_store_map(&c->maps_decode.pool, r_pool ? (void *)cv.pool : (void *)cv.text, r_pool ? r_pool : r_text, d);
     ok = ok && encode_store_map(&c->maps_decode.fixed, r_fixed ? (void *)cv.fixed : (void *)cv.text, r_fixed ? r_fixed : r_text, d);
     c->maps_prefill = c->maps_decode;
     ok = ok && encode_store_map(&c->maps_prefill.anchor, c->stage, r_stage, d);
@@ -929,7 +937,7 @@ static wnw_status_t place_multi(wnw_cache_t *c, int32_t seq, int32_t layer, cons
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (layer == 0) {
     s.placed_layers = 0;
-    const size_t need = full ? 0 : (size_t)mirror_chunks_of(G, C_b) * c->tid_total * 2 * G.ncp * G.d * sizeof(bf16);
+    const size_t need = full ? 0 : (size_t)mirror_chunks_of(G, C_b) * c->tid_total * 2 * G.ncp * G.d * tidal_elem_bytes(G);
     if (need != s.mirror_bytes) {
       CK(cudaDeviceSynchronize());
       if (s.mirror) cudaFreeHost(s.mirror);
@@ -963,6 +971,9 @@ static wnw_status_t place_multi(wnw_cache_t *c, int32_t seq, int32_t layer, cons
   CK(cudaMemsetAsync(c->stage, 0, (size_t)G.Hkv * 2 * G.T_a_pad * G.d * sizeof(bf16), st));
   CK(launch_place_scatter(c->cv, seq, layer, (const bf16 *)k_dev, (const bf16 *)v_dev, n_tokens, audio_begin, audio_end, T_t,
                           C_b, S_b, S_base_b, c->stage, st));
+  // e4m3 tidal tier: scales per chunk, and the staged rows of the tidal heads become the values their bytes will decode
+  // to, so that the prefill scores below already see what decoding will see
+  if (G.kv8 && C_b > 0) CK(launch_quantise_stage(c->cv, seq, layer, c->stage, C_b, st));
   if (!full && C_b > 0) {
     if (c->prefill_seq != seq || c->prefill_T_a != T_a) {
       std::vector<WorkItem> items;
@@ -1882,8 +1893,36 @@ extern "C" wnw_status_t wnw_get_slot_kv(wnw_cache_t *c, int32_t seq, int32_t lay
   if (slot < 0 || slot >= c->seqs[seq].S) return WNW_ERR_INVALID_ARG;
   DeviceGuard guard(c->cfg.device);
   if ((s = drain(c)) != WNW_OK) return s;
-  const long long off = pool_off(c->geo, c->layers[layer], seq, slot, c->role_idx[layer * c->geo.Hkv + kv_head], which);
-  CK(cudaMemcpy(rows, c->cv.pool + off, (size_t)c->geo.nc * c->geo.d * sizeof(bf16), cudaMemcpyDeviceToHost));
+  const int ridx = c->role_idx[layer * c->geo.Hkv + kv_head];
+  const long long off = pool_off(c->geo, c->layers[layer], seq, slot, ridx, which);
+  if (!c->geo.kv8) {
+    CK(cudaMemcpy(rows, c->cv.pool + off, (size_t)c->geo.nc * c->geo.d * sizeof(bf16), cudaMemcpyDeviceToHost));
+    return WNW_OK;
+  }
+  // e4m3 slots: the bytes, the chunk the table names and its scale; decoded here to the bf16 values they stand for
+  const Geometry &G = c->geo;
+  std::vector<uint8_t> raw((size_t)G.nc * G.d);
+  CK(cudaMemcpy(raw.data(), reinterpret_cast<const uint8_t *>(c->cv.pool) + off, raw.size(), cudaMemcpyDeviceToHost));
+  int32_t chunk = -1;
+  long long steps = 0;
+  CK(cudaMemcpy(&steps, c->cv.steps + seq, sizeof(steps), cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(&chunk, c->cv.slot_chunk + slot_table_off(G, (int)(steps & 1), (long long)seq * G.L + layer) + slot, sizeof(chunk),
+                cudaMemcpyDeviceToHost));
+  int8_t ex = 0;
+  if (chunk >= 0)
+    CK(cudaMemcpy(&ex, c->cv.kv_exp + kv_exp_off(G, c->cv.tid_total, seq, c->layers[layer].tid_prefix + ridx, chunk) + which, 1,
+                  cudaMemcpyDeviceToHost));
+  uint16_t *out = static_cast<uint16_t *>(rows);
+  for (int r = 0; r < G.nc; ++r)
+    for (int e = 0; e < G.d; ++e) {
+      const uint8_t byte = raw[(size_t)r * G.d + (e & ~15) + e4m3_store_pos(which, e & 15)];
+      const int E = (byte >> 3) & 15, M = byte & 7;
+      const float mag = E == 0 ? std::ldexp((float)M, -9) : std::ldexp(1.f + M / 8.f, E - 7);
+      const float val = std::ldexp((byte & 0x80) ? -mag : mag, ex);
+      uint32_t u;
+      memcpy(&u, &val, 4);
+      out[(size_t)r * G.d + e] = (uint16_t)(u >> 16);   // exact: three mantissa bits
+    }
   return WNW_OK;
 }
 

@@ -15,7 +15,7 @@ import numpy as np
 import torch
 
 import paper_2608_22704_b200 as wnw
-from helpers import bf16_bits_to_f64, make_oracle
+from helpers import bf16_bits_to_f64, dequantised_tidal_bits, make_oracle
 from oracle import wnw_oracle as wo
 from workloads import ROLE_ANCHOR, ROLE_FIXED, ROLE_TIDAL, Synth, Workload
 from workloads.synth import bf16_bits
@@ -49,8 +49,11 @@ def near_tie(scores64, lens, sel_a, sel_b):
 
 class Lockstep:
     def __init__(self, w: Workload, seed=0, device="cuda:0", recall_mode=0, gen_device=None, oracle_seqs=None,
-                 score_scope=0, residency=0, evict_lag=3, token_retention=None, token_seg=25, token_variant=0):
+                 score_scope=0, residency=0, evict_lag=3, token_retention=None, token_seg=25, token_variant=0, kv_fp8=False):
         self.w = w
+        # e4m3 storage of the tidal tier: the library gets the plain bf16 prefix and the format flag; the oracle, which knows
+        # nothing of storage formats, gets the values the stored bytes decode to (helpers.dequantised_tidal_bits)
+        self.kv_fp8 = kv_fp8
         # token-granular compression of fixed heads: retention [n_layers][n_kv_heads], segment size, variant
         self.tok_ret = None if token_retention is None else np.asarray(token_retention, np.float32)
         self.tok_seg, self.tok_variant = token_seg, token_variant
@@ -62,7 +65,8 @@ class Lockstep:
         self.o = make_oracle(w, score_scope=score_scope, residency=residency, evict_lag=evict_lag)
         self.h = wnw.wnw_create(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max(max(w.audio_lens), 0),
                                 w.text_capacity, w.chunk, w.budget, w.roles, topk=w.topk, device=self.dev.index or 0,
-                                recall_mode=recall_mode, score_scope=score_scope, residency=residency, evict_lag=evict_lag)
+                                recall_mode=recall_mode, score_scope=score_scope, residency=residency, evict_lag=evict_lag,
+                                tidal_kv_format=wnw.WNW_TIDAL_KV_FP8_E4M3 if kv_fp8 else wnw.WNW_TIDAL_KV_BF16)
         self.kept = {}
         self.tok_kept = {}
         self.near_ties = 0
@@ -96,6 +100,8 @@ class Lockstep:
                     torch.cuda.synchronize(self.dev)   # the generator's buffers are released right after
                 if b in self.oracle_seqs:
                     kb, vb = bf16_bits(p["k"]), bf16_bits(p["v"])
+                    if self.kv_fp8:
+                        kb, vb = dequantised_tidal_bits(kb, vb, w.roles[l], p["audio_begin"], p["audio_end"], w.chunk)
                     if self.tok_ret is not None:
                         self.o.place_prefill_tokens(b, l, kb, vb, p["audio_begin"], p["audio_end"], bf16_bits(p[qname]),
                                                     self.tok_ret[l], self.tok_seg, self.tok_variant)
@@ -312,7 +318,7 @@ class Lockstep:
                     assert g_sel.tolist() == want_sel.tolist(), f"selection (ii) step {t} b{b} l{l}"
                     plan, _ = wo.table_update(tab, stamp, want_sel, steps_before[b], w.topk)
                 n_tid = int((w.roles[l] == ROLE_TIDAL).sum())
-                self.expected_recall_bytes += len(plan) * n_tid * 2 * (-(-w.chunk // 16) * 16) * w.head_dim * 2   # blocks are stored padded to 16 rows
+                self.expected_recall_bytes += len(plan) * n_tid * 2 * (-(-w.chunk // 16) * 16) * w.head_dim * (1 if self.kv_fp8 else 2)   # blocks are stored padded to 16 rows
                 assert g_tab.tolist() == tab.tolist(), f"table (ii) step {t} b{b} l{l}"
                 assert g_stamp.tolist() == stamp.tolist(), f"stamps (ii) step {t} b{b} l{l}"
                 # (iii) oracle on its own scores
