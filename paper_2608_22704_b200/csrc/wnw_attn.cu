@@ -122,12 +122,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t *>(&v);
 }
 
-// Two e4m3 bytes (low 16 bits of x) as two bf16 numbers: exact, every e4m3 value is a bf16 value.
-__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t x) {
+// Two e4m3 bytes (low 16 bits of x) as two fp16 numbers: one instruction, exact (every e4m3 value is an fp16 value).
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
   uint32_t h;
   asm("cvt.rn.f16x2.e4m3x2 %0, %1;\n" : "=r"(h) : "h"((unsigned short)x));
-  const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h));
-  return pack_bf16(f.x, f.y);
+  return h;
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+// bf16 pair -> fp16 pair: exact for magnitudes inside fp16's normal range
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t x) { return pack_f16(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u)); }
+__device__ __forceinline__ void mma16816_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 struct GranDesc {
@@ -187,8 +197,11 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
 
 // VAR 1 (TB): tidal heads keep a token-granular permanent base (their key space is [text | base blocks | dynamic slots]);
 // VAR 2 (F8): the slot pool holds e4m3 bytes (one 16 x 128-byte box per K or V granule) with a power-of-two scale per
-//   (chunk, head, K|V): the bytes become bf16 fragments on their way from ldmatrix to mma.sync, the scales are folded into
-//   the logits and into P; the default path (VAR 0) carries none of either variant's branches.
+//   (chunk, head, K|V).  The bytes become fp16 fragments on their way from ldmatrix to mma.sync (one conversion per two
+//   elements, exact), and the products with such a granule run on the fp16 form of mma.sync with q and P taken as fp16 (q
+//   exactly while its elements lie in fp16's normal range; P in [0,1] with three more mantissa bits than bf16 gives it).  The
+//   K scale multiplies the logits; the V scale enters the exponent of the granule's weights (see the softmax step).  The
+//   default path (VAR 0) carries none of either variant's branches.
 // bid: the CTA's index within its layer's launch (a launch may carry the CTAs of several layers back to back);
 // inl: the layer's work items when they travel in the kernel parameters, else null (read from a.items).
 template <int D, bool G16, int NW, int VAR>
@@ -505,6 +518,15 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
       }
     }
   }
+  uint32_t qh[F8 ? KK : 1][NQ];   // the query as fp16, for the products with e4m3 granules
+  if constexpr (F8) {
+    if (it.role == ROLE_TIDAL) {
+#pragma unroll
+      for (int kk = 0; kk < KK; ++kk)
+#pragma unroll
+        for (int x = 0; x < NQ; ++x) qh[kk][x] = bf16x2_to_f16x2(qa[kk][x]);
+    }
+  }
   STAMP(16);
   if (arm && !early) {
 #pragma unroll
@@ -540,13 +562,18 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
                   const int (&fmt)[2]) {
     constexpr int NU = decltype(nu_tag)::value;
     float sT[NU][NTN][4];
-    float scu[NU], pscale[NU];   // softmax scale times the K scale of the granule; the V scale, folded into P
+    // e4m3 granules: the K scale 2^eK multiplies the logits.  The V scale 2^eV is carried in the exponent: the granule's
+    // logits are shifted by eV for the running maximum and the weights, so that P = 2^(s + eV - m) <= 1 multiplies the raw
+    // e4m3 values of V, and the denominator takes each weight times 2^-eV.  The triple (m, l, o) stays consistent for every
+    // merge: both l and o are relative to the same m, whatever m is.
+    float scu[NU], vshift[NU], vinv[NU];
 #pragma unroll
     for (int u = 0; u < NU; ++u) {
-      scu[u] = sc; pscale[u] = 1.f;
+      scu[u] = sc; vshift[u] = 0.f; vinv[u] = 1.f;
       if (F8 && (fmt[u] & 1)) {
         scu[u] = sc * exp2f((float)(int8_t)((fmt[u] >> 7) & 0xff));
-        pscale[u] = exp2f((float)(int8_t)((fmt[u] >> 15) & 0xff));
+        vshift[u] = (float)(int8_t)((fmt[u] >> 15) & 0xff);
+        vinv[u] = exp2f(-vshift[u]);
       }
     }
     {
@@ -585,11 +612,11 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
               ldsm_x4(bk, sKs[u] + row8 * 128 + ((((2 * p + (mtx >> 1)) & 7) ^ (row8 & 7)) << 4));
 #pragma unroll
               for (int hk = 0; hk < 2; ++hk) {
-                const uint32_t a0 = e4m3x2_to_bf16x2(bk[2 * hk]), a1 = e4m3x2_to_bf16x2(bk[2 * hk + 1]);
-                const uint32_t a2 = e4m3x2_to_bf16x2(bk[2 * hk] >> 16), a3 = e4m3x2_to_bf16x2(bk[2 * hk + 1] >> 16);
+                const uint32_t a0 = e4m3x2_to_f16x2(bk[2 * hk]), a1 = e4m3x2_to_f16x2(bk[2 * hk + 1]);
+                const uint32_t a2 = e4m3x2_to_f16x2(bk[2 * hk] >> 16), a3 = e4m3x2_to_f16x2(bk[2 * hk + 1] >> 16);
 #pragma unroll
                 for (int nt = 0; nt < NTN; ++nt)
-                  mma16816(hk ? sO[u][nt] : sT[u][nt], a0, a1, a2, a3, qa[2 * p + hk][2 * nt], qa[2 * p + hk][2 * nt + 1]);
+                  mma16816_f16(hk ? sO[u][nt] : sT[u][nt], a0, a1, a2, a3, qh[2 * p + hk][2 * nt], qh[2 * p + hk][2 * nt + 1]);
               }
             }
           } else {
@@ -615,8 +642,8 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
 #pragma unroll
       for (int u = 0; u < NU; ++u) {
         const bool lo = r0 < valids[u], hi = r0 + 8 < valids[u];
-        v[u][0] = lo ? sT[u][nt][0] * scu[u] : -INFINITY; v[u][1] = lo ? sT[u][nt][1] * scu[u] : -INFINITY;
-        v[u][2] = hi ? sT[u][nt][2] * scu[u] : -INFINITY; v[u][3] = hi ? sT[u][nt][3] * scu[u] : -INFINITY;
+        v[u][0] = lo ? fmaf(sT[u][nt][0], scu[u], vshift[u]) : -INFINITY; v[u][1] = lo ? fmaf(sT[u][nt][1], scu[u], vshift[u]) : -INFINITY;
+        v[u][2] = hi ? fmaf(sT[u][nt][2], scu[u], vshift[u]) : -INFINITY; v[u][3] = hi ? fmaf(sT[u][nt][3], scu[u], vshift[u]) : -INFINITY;
         mxA = fmaxf(mxA, fmaxf(v[u][0], v[u][2])); mxB = fmaxf(mxB, fmaxf(v[u][1], v[u][3]));
       }
 #pragma unroll
@@ -633,7 +660,8 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
         v[u][0] = exp2f(v[u][0] - mnA); v[u][2] = exp2f(v[u][2] - mnA);
         v[u][1] = exp2f(v[u][1] - mnB); v[u][3] = exp2f(v[u][3] - mnB);
         float eA = v[u][0] + v[u][2], eB = v[u][1] + v[u][3];
-        addA += eA; addB += eB;
+        if constexpr (F8) { addA += eA * vinv[u]; addB += eB * vinv[u]; }
+        else { addA += eA; addB += eB; }
         if (sidxs[u] >= 0) {   // softmax-mass partial of this granule (fp32, before any bf16 rounding): anchor-like heads only
 #pragma unroll
           for (int sh = 4; sh <= 16; sh <<= 1) {
@@ -649,8 +677,8 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
         }
         // P^T tile [token][head] -> [head][token]: what the PV product wants in its B operand
         uint32_t p01, p23;
-        if constexpr (F8) {   // the V scale of an e4m3 granule rides on P: a power of two, so rounding P to bf16 commutes with it
-          p01 = pack_bf16(v[u][0] * pscale[u], v[u][1] * pscale[u]); p23 = pack_bf16(v[u][2] * pscale[u], v[u][3] * pscale[u]);
+        if (F8 && (fmt[u] & 1)) {   // fp16 weights for the fp16 product with an e4m3 granule
+          p01 = pack_f16(v[u][0], v[u][1]); p23 = pack_f16(v[u][2], v[u][3]);
         } else {
           p01 = pack_bf16(v[u][0], v[u][1]); p23 = pack_bf16(v[u][2], v[u][3]);
         }
@@ -690,10 +718,10 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
 #pragma unroll
               for (int hk = 0; hk < 2; ++hk) {
                 const uint32_t x0 = __byte_perm(bv[2 * hk], 0, 0x3120), x1 = __byte_perm(bv[2 * hk + 1], 0, 0x3120);
-                const uint32_t a0 = e4m3x2_to_bf16x2(x0), a1 = e4m3x2_to_bf16x2(x0 >> 16);
-                const uint32_t a2 = e4m3x2_to_bf16x2(x1), a3 = e4m3x2_to_bf16x2(x1 >> 16);
+                const uint32_t a0 = e4m3x2_to_f16x2(x0), a1 = e4m3x2_to_f16x2(x0 >> 16);
+                const uint32_t a2 = e4m3x2_to_f16x2(x1), a3 = e4m3x2_to_f16x2(x1 >> 16);
 #pragma unroll
-                for (int nt = 0; nt < NTN; ++nt) mma16816(oT[nt][2 * p + hk], a0, a1, a2, a3, pb[u][nt][0], pb[u][nt][1]);
+                for (int nt = 0; nt < NTN; ++nt) mma16816_f16(oT[nt][2 * p + hk], a0, a1, a2, a3, pb[u][nt][0], pb[u][nt][1]);
               }
             }
           } else {
