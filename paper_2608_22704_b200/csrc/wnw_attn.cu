@@ -30,16 +30,34 @@
 namespace wnw {
 
 constexpr int NW_LAT = 8;  // warps of a one-shot CTA (one work item each): 1 CTA per SM
-constexpr int NW_THR = 4;  // warps of a persistent CTA (large launches of chained layers): two per SM, whose phases drift apart,
-                           // so one CTA's prologue and merge overlap the other's streaming
-constexpr int NSTAGE = 3;  // granules in flight per warp
+constexpr int NW_THR = 4;  // warps of a persistent CTA (launches of more than one wave): several per SM, whose phases drift apart,
+                           // so one CTA's prologue and merge overlap the others' streaming
+// Granules in flight per warp, and persistent CTAs per SM.  Three stages and two 4-warp CTAs per SM are what was kept after
+// measuring the alternative that shared memory allows, two-stage rings (exactly the pair a softmax step consumes) with
+// three CTAs, i.e. twelve warps, per SM: 16 x 7500 tokens chained 0.417 -> 0.402 ms and overlapped 0.344 -> 0.360 ms,
+// batch-32 ragged chained 1.31 -> 1.41 ms; two stages with two CTAs: 0.445, 0.355, 1.28 ms.  The macros are the sweep's.
+#ifndef WNW_THR_CTAS_PER_SM
+#define WNW_THR_CTAS_PER_SM 2
+#endif
+#ifndef WNW_NSTAGE_THR
+#define WNW_NSTAGE_THR 3
+#endif
+constexpr int nstage_of(int nw) { return nw == NW_THR ? WNW_NSTAGE_THR : 3; }
 
 int attn_warps(bool throughput) { return throughput ? NW_THR : NW_LAT; }
 // Merge scratch of a CTA when it sits behind the stages instead of aliasing them: (m, l) and o of every warp.
 static size_t attn_scratch_bytes(int nw, int g, int d) { return (size_t)nw * 128 + (size_t)nw * g * (d + 2) * 4; }
+// Persistent CTAs an SM holds: what the shared memory allows (stages, alignment slack, merge scratch behind the stages,
+// 1 KB the system keeps per CTA) up to what the kernel's register bound was compiled for.
+int attn_persistent_ctas_per_sm(int g, int d) {
+  const size_t per_cta = (size_t)NW_THR * nstage_of(NW_THR) * 2 * GR * d * 2 + 1024 + attn_scratch_bytes(NW_THR, g, d) + 512 + 1024;
+  const int fit = (int)((228 * 1024) / per_cta);
+  const int cap = g > 8 ? 2 : WNW_THR_CTAS_PER_SM;   // registers: the two-tile variant is compiled for two CTAs per SM
+  return fit < 1 ? 1 : (fit > cap ? cap : fit);
+}
 // One-shot 8-warp CTAs can keep it there while everything fits the 227 KB a CTA may have.
 bool attn_xpref_fits(int g, int d) {
-  return (size_t)NW_LAT * NSTAGE * 2 * GR * d * 2 + 1024 + attn_scratch_bytes(NW_LAT, g, d) + 512 <= 227 * 1024;
+  return (size_t)NW_LAT * nstage_of(NW_LAT) * 2 * GR * d * 2 + 1024 + attn_scratch_bytes(NW_LAT, g, d) + 512 <= 227 * 1024;
 }
 
 
@@ -218,6 +236,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   constexpr int KK = D / 16;              // k16 steps of QK^T; also pairs of n8 tiles of PV
   constexpr int NQ = G16 ? 4 : 2;
   constexpr bool TB = VAR == 1, F8 = VAR == 2;
+  constexpr int NSTAGE = nstage_of(NW);
   static_assert(!F8 || D == 128, "an e4m3 row must fill one 128-byte swizzle atom");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -319,6 +338,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
 
   // ---- producer side of the per-warp pipeline: (prod, p_n) is the next granule to fetch, seq_p its stage sequence ----
   Ctx prod;
+  prod.n_my = 0;   // loaded by the first work item before anything is produced
   int p_n = 0;
   uint32_t seq_p = 0, seq_c = 0;
   GranDesc blk;  // descriptor this lane decoded for the producer's current block of 32 granules
@@ -963,7 +983,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
 }
 
 template <int D, bool G16, int NW, int VAR>
-__global__ void __launch_bounds__(NW * 32) wnw_attn_kernel(const __grid_constant__ CacheView cv,
+__global__ void __launch_bounds__(NW * 32, NW == NW_THR ? (G16 ? 2 : WNW_THR_CTAS_PER_SM) : 1) wnw_attn_kernel(const __grid_constant__ CacheView cv,
                                                            const __grid_constant__ AttnArgs a,
                                                            const __grid_constant__ InlineItems inl,
                                                            const __grid_constant__ TmaMaps maps) {
@@ -1006,7 +1026,7 @@ static cudaError_t launch_multi_tb(const CacheView &cv, const MultiArgs &m, size
 template <int D, bool G16, int NW, int VAR>
 static cudaError_t launch_tb(const CacheView &cv, const AttnArgs &a, cudaStream_t st) {
   // stages + slack to align them to the swizzle atom + the merge scratch when it does not alias the stages
-  const size_t smem = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024 + (a.xpref ? attn_scratch_bytes(NW, cv.geo.g, D) : 0);
+  const size_t smem = (size_t)NW * nstage_of(NW) * 2 * GR * D * 2 + 1024 + (a.xpref ? attn_scratch_bytes(NW, cv.geo.g, D) : 0);
   if (!a.maps) return cudaErrorInvalidValue;
   InlineItems inl;
   if (a.n_items <= INLINE_ITEMS_MAX && a.items_host) memcpy(inl.it, a.items_host, sizeof(WorkItem) * a.n_items);
@@ -1081,7 +1101,7 @@ bool encode_store_map_e4m3(CUtensorMap *map, const void *base, unsigned long lon
 
 template <int D, bool G16, int NW>
 static cudaError_t configure_t() {
-  const size_t want = (size_t)NW * NSTAGE * 2 * GR * D * 2 + 1024 + attn_scratch_bytes(NW, G16 ? 16 : 8, D);
+  const size_t want = (size_t)NW * nstage_of(NW) * 2 * GR * D * 2 + 1024 + attn_scratch_bytes(NW, G16 ? 16 : 8, D);
   const int bytes = (int)std::min<size_t>(want, 227 * 1024 - 512);   // what a CTA may have, less this kernel's static shared memory
   cudaError_t e = cudaFuncSetAttribute(wnw_attn_kernel<D, G16, NW, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
   if (e != cudaSuccess) return e;
@@ -1142,7 +1162,7 @@ cudaError_t launch_attn_multi(const CacheView &cv, const AttnArgs *args, int n, 
     m.l[n_used].pdl = 0; m.l[n_used].wait_inputs = 0;
     ++n_used;
     ctas += count;
-    smem = std::max(smem, (size_t)NW_LAT * NSTAGE * 2 * GR * d * 2 + 1024 + (a.xpref ? attn_scratch_bytes(NW_LAT, cv.geo.g, d) : 0));
+    smem = std::max(smem, (size_t)NW_LAT * nstage_of(NW_LAT) * 2 * GR * d * 2 + 1024 + (a.xpref ? attn_scratch_bytes(NW_LAT, cv.geo.g, d) : 0));
   }
   if (n_used == 0) return cudaSuccess;
   m.n = n_used; m.cta_prefix[n_used] = ctas;

@@ -294,5 +294,6 @@ cudaError_t configure_select_kernel();
 constexpr int SELECT_SMEM_CAP = 200 * 1024;  // dynamic shared memory the selection kernel may be launched with
 bool attn_xpref_fits(int g, int d);  // a one-shot CTA can hold its merge scratch behind the copy stages
 int attn_warps(bool throughput);  // warps per attention CTA in the latency / throughput variant
+int attn_persistent_ctas_per_sm(int g, int d);  // persistent (throughput-variant) CTAs that fit one SM
 
 }  // namespace wnw

@@ -610,7 +610,7 @@ static void build_throughput_items(const wnw_cache *c, int layer, int mode, cons
   const int nw = attn_warps(true), n_heads = (int)seq_ids.size() * G.Hkv;
   const double cost_whole = 5.0, cost_piece = 16.0;   // fixed cost of an item in granules' worth: finished in the CTA / left as a partial
   const double mean_weight = 1.0;                     // weight of the mean CTA load beside the longest one in the objective
-  const int per_sm = 2;                               // persistent CTAs per SM (4 warps, about 105 KB of shared memory each)
+  const int per_sm = attn_persistent_ctas_per_sm(G.g, G.d);   // persistent 4-warp CTAs an SM holds
   double total = 0.0;
   for (int hd = 0; hd < n_heads; ++hd) total += n_work[hd];
   const int P = (int)std::min<double>(per_sm * c->n_sm, std::max(1.0, total / (2.0 * nw)));   // at least two granules per warp and CTA
