@@ -7,7 +7,7 @@ import pytest
 import torch
 
 import paper_2608_22704_b200 as wnw
-from helpers import bf16_bits_to_f64, make_oracle
+from helpers import bf16_bits_to_f64, dequantised_tidal_bits, make_oracle
 from oracle import wnw_oracle as wo
 from paper_2608_22704_b200.sharded import create_shard_cache, shard_plan, sharded_step
 from parity_harness import OUT_TOL, assert_scores_close, chunk_lens
@@ -18,22 +18,27 @@ pytestmark = pytest.mark.gpu
 A, T, F = ROLE_ANCHOR, ROLE_TIDAL, ROLE_FIXED
 
 
-def _run(roles, world, n_steps=6, seed=13):
-    w = tiny_custom(n_layers=len(roles), n_q_heads=8, n_kv_heads=4, head_dim=64, n_text=6, audio_lens=(200, 90), chunk=16, budget=0.3,
-                    n_steps=n_steps, roles=roles, region=16)
+def _run(roles, world, n_steps=6, seed=13, kv_fp8=False):
+    """kv_fp8: the shards keep their tidal tier as e4m3 (head_dim 128); the oracle gets the values the bytes decode to."""
+    w = tiny_custom(n_layers=len(roles), n_q_heads=8, n_kv_heads=4, head_dim=128 if kv_fp8 else 64, n_text=6, audio_lens=(200, 90),
+                    chunk=16, budget=0.3, n_steps=n_steps, roles=roles, region=16)
     dev = torch.device("cuda:0")
     syn = Synth(w, seed=seed)
     o = make_oracle(w)
     plan = shard_plan(w.roles, w.n_q_heads, world)
     caches = [create_shard_cache(sh, w.n_q_heads, w.n_kv_heads, w.head_dim, w.batch, max(w.audio_lens), w.text_capacity, w.chunk,
-                                 w.budget, topk=w.topk) for sh in plan]
+                                 w.budget, topk=w.topk,
+                                 tidal_kv_format=wnw.WNW_TIDAL_KV_FP8_E4M3 if kv_fp8 else wnw.WNW_TIDAL_KV_BF16) for sh in plan]
     C_max = -(-max(w.audio_lens) // w.chunk)
     try:
         # ---- placement, with the exchange of the tidal heads' prefill sums per (sequence, layer)
         for b in range(w.batch):
             for l in range(w.n_layers):
                 p = syn.prefill(b, l)
-                o.place_prefill(b, l, bf16_bits(p["k"]), bf16_bits(p["v"]), p["audio_begin"], p["audio_end"], bf16_bits(p["q_last"]))
+                kb, vb = bf16_bits(p["k"]), bf16_bits(p["v"])
+                if kv_fp8:
+                    kb, vb = dequantised_tidal_bits(kb, vb, w.roles[l], p["audio_begin"], p["audio_end"], w.chunk)
+                o.place_prefill(b, l, kb, vb, p["audio_begin"], p["audio_end"], bf16_bits(p["q_last"]))
                 sums = []
                 for sh, h in zip(plan, caches):
                     wnw.wnw_place_prefill(h, b, l, p["k"][:, sh.kv_heads].contiguous().to(dev), p["v"][:, sh.kv_heads].contiguous().to(dev),
@@ -109,6 +114,11 @@ def test_head_shards_match_one_oracle(world):
     """Anchor heads of a layer on one shard (the others contribute zero rows), layers without any anchor routed by the
     model-wide flags, tidal heads of one layer spread over the shards (one table, ranked by the sum over all of them)."""
     assert _run([[A, T, T, F], [T, F, T, T], [F, T, A, T]], world) > 0
+
+
+def test_head_shards_with_an_e4m3_tidal_tier():
+    """The shards' slots are refilled from e4m3 mirrors after the exchange of the prefill sums."""
+    assert _run([[A, T, T, F], [T, F, T, T], [F, T, A, T]], 2, kv_fp8=True) > 0
 
 
 def test_head_shards_with_a_layers_anchor_heads_split_over_shards():
