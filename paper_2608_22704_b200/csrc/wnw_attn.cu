@@ -166,6 +166,7 @@ struct GranDesc {
   int off;         // token offset of the granule inside its chunk
   int score_idx;   // audio granule index for score partials, -1 = none
   int ex;          // e4m3 tidal tier: K scale exponent | V scale exponent << 8 | 1 << 16 for a slot granule (filled with the metadata)
+  int vis;         // visible rows, resolved with the first metadata of the descriptor's block of 32 granules
 };
 
 // Maps granule j of a head's virtual key space [text capacity | audio] to memory WITHOUT waiting on any global load:
@@ -175,7 +176,7 @@ __device__ __forceinline__ GranDesc decode_granule(const CacheView &cv, const At
                                                    const WorkItem &it, int j, int table_parity) {
   const Geometry &G = cv.geo;
   GranDesc r;
-  r.cid = -1; r.off = 0; r.score_idx = -1; r.ex = 0;
+  r.cid = -1; r.off = 0; r.score_idx = -1; r.ex = 0; r.vis = 0;
   if (j < G.n_tg) {
     const int tok0 = j * GR;
     r.row = (int)(text_off(G, it.b, a.layer, it.h, 0) / G.d) + tok0;
@@ -342,7 +343,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   int p_n = 0;
   uint32_t seq_p = 0, seq_c = 0;
   GranDesc blk;  // descriptor this lane decoded for the producer's current block of 32 granules
-  blk.row = 0; blk.meta = 0; blk.cid = -1; blk.off = 0; blk.score_idx = -1; blk.ex = 0;
+  blk.row = 0; blk.meta = 0; blk.cid = -1; blk.off = 0; blk.score_idx = -1; blk.ex = 0; blk.vis = 0;
 
   // Visible rows of a granule once its metadata has arrived.
   auto visible = [&](const Ctx &c, int meta, int cid, int off, int j) -> int {
@@ -386,24 +387,18 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     bool load = meta != 0;
     if (meta == -1) load = visible(c, -1, 0, 0, j) > 0;  // waits for the text length
     if (meta == -3) load = __shfl_sync(0xffffffffu, blk.cid, src_lane) >= 0;  // waits for the table entry
-    if (load && lane == 0) {
+    // The boxes of a granule (K and V, HALVES each) are issued by as many lanes at once, one box per lane: lane = 2 * half + (V).
+    // The stage's barrier cannot complete before lane 0 has arrived with the byte count, whichever copy lands first.
+    const bool f8g = F8 && !is_text && c.it.role == ROLE_TIDAL;   // an e4m3 granule: one box of 16 rows x 128 bytes each for K and V
+    if (load && lane < (f8g ? 2 : 2 * HALVES)) {
       const int stage = (int)(seq % NSTAGE);
-      const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB, bar = smem_u32(&bars[warp][stage]);
+      const uint32_t bar = smem_u32(&bars[warp][stage]);
       const CUtensorMap *map = is_text ? &maps.text : (base_blk ? &maps.fixed : c.map_audio);
-      const int vrow = row + (is_text ? v_delta_text : (base_blk ? G.FB * G.ncp : c.v_delta_audio));
+      const int v_delta = is_text ? v_delta_text : (base_blk ? G.FB * G.ncp : c.v_delta_audio);
+      const int hf = lane >> 1, isv = lane & 1;
       fence_proxy_async();  // the stage was last read through the generic proxy (ldmatrix)
-      if (F8 && !is_text && c.it.role == ROLE_TIDAL) {   // an e4m3 granule: one box of 16 rows x 128 bytes each for K and V
-        mbar_expect_tx(bar, 2 * HALFB);
-        tma_load_2d(sK, map, 0, row, bar);
-        tma_load_2d(sV, map, 0, vrow, bar);
-      } else {
-        mbar_expect_tx(bar, 2 * TILEB);
-#pragma unroll
-        for (int hf = 0; hf < HALVES; ++hf) {
-          tma_load_2d(sK + hf * HALFB, map, hf * 64, row, bar);
-          tma_load_2d(sV + hf * HALFB, map, hf * 64, vrow, bar);
-        }
-      }
+      if (lane == 0) mbar_expect_tx(bar, f8g ? 2 * HALFB : 2 * TILEB);
+      tma_load_2d(my_base + stage * 2 * TILEB + isv * TILEB + hf * HALFB, map, hf * 64, row + isv * v_delta, bar);
     }
     return load;
   };
@@ -411,7 +406,9 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   // metadata loads.
   auto issue_meta = [&](const Ctx &c, int n, uint32_t seq, bool loaded) {
     const int src_lane = n & 31;
-    const int valid = __shfl_sync(0xffffffffu, visible(c, blk.meta, blk.cid, blk.off, c.first + (n - src_lane + lane) * NW), src_lane);
+    // every lane resolves its own granule of the block once (this is where the table entries and the text length are waited for)
+    if (src_lane == 0) blk.vis = visible(c, blk.meta, blk.cid, blk.off, c.first + (n + lane) * NW);
+    const int valid = __shfl_sync(0xffffffffu, blk.vis, src_lane);
     const int sidx = __shfl_sync(0xffffffffu, blk.score_idx, src_lane);
     int ex = 0;
     if (F8) {
@@ -604,12 +601,14 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
         for (int nt = 0; nt < NTN; ++nt)
 #pragma unroll
           for (int e = 0; e < 4; ++e) sT[u][nt][e] = sO[u][nt][e] = 0.f;
-      const int mtx = lane >> 3, row = ((mtx >> 1) << 3) + (lane & 7);
+      const int mtx = lane >> 3;
+      // A lane's ldmatrix row address inside a 16 x 128-byte box with the 128-byte swizzle: row * 128 + ((piece ^ row % 8) << 4),
+      // piece = 2 * kk + (0 or 1 by lane).  The lane's part, row * 128 + (((0 or 1) ^ row % 8) << 4), is a constant of the
+      // lane; a k-step then costs one XOR with an immediate (stages start on 1024-byte boundaries, so the base adds in freely).
+      const uint32_t lane_k = (uint32_t)((((mtx >> 1) << 3) + (lane & 7)) * 128 + (((mtx & 1) ^ (lane & 7)) << 4));
       auto qk_bf16 = [&](int kk, int u) {
-        const int piece = 2 * kk + (mtx & 1);
-        const uint32_t off = row * 128 + (kk >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4);
         uint32_t bk[4];   // K rows 0-7 | 8-15 of the granule x d 0-7 | 8-15 of the k-step: the A operand's four quadrants
-        ldsm_x4(bk, sKs[u] + off);
+        ldsm_x4(bk, ((sKs[u] + lane_k) ^ (uint32_t)(((2 * kk) & 7) << 4)) + (kk >> 2) * HALFB);
 #pragma unroll
         for (int nt = 0; nt < NTN; ++nt)
           mma16816((kk & 1) ? sO[u][nt] : sT[u][nt], bk[0], bk[2], bk[1], bk[3], qa[kk][2 * nt], qa[kk][2 * nt + 1]);
@@ -625,11 +624,11 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
           if (fmt[u] & 1) {
             // e4m3 tile: rows of 128 bytes; one ldmatrix.x4 brings rows 0-7 | 8-15 x the 16-byte groups 2p | 2p+1, i.e. two
             // k-steps; a lane's four bytes are the elements 2t, 2t+1, 2t+8, 2t+9 of the group (e4m3_store_pos)
-            const int row8 = ((mtx & 1) << 3) + (lane & 7);
+            const uint32_t lane_k8 = (uint32_t)((((mtx & 1) << 3) + (lane & 7)) * 128 + (((mtx >> 1) ^ (lane & 7)) << 4));
 #pragma unroll
             for (int p = 0; p < KK / 2; ++p) {
               uint32_t bk[4];
-              ldsm_x4(bk, sKs[u] + row8 * 128 + ((((2 * p + (mtx >> 1)) & 7) ^ (row8 & 7)) << 4));
+              ldsm_x4(bk, (sKs[u] + lane_k8) ^ (uint32_t)((2 * p) << 4));
 #pragma unroll
               for (int hk = 0; hk < 2; ++hk) {
                 const uint32_t a0 = e4m3x2_to_f16x2(bk[2 * hk]), a1 = e4m3x2_to_f16x2(bk[2 * hk + 1]);
@@ -711,12 +710,11 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     }
     STAMP(26);
     {
-      const int mtx = lane >> 3, row = ((mtx & 1) << 3) + (lane & 7);
+      const int mtx = lane >> 3;
+      const uint32_t lane_v = (uint32_t)((((mtx & 1) << 3) + (lane & 7)) * 128 + (((mtx >> 1) ^ (lane & 7)) << 4));   // as lane_k above
       auto pv_bf16 = [&](int t2, int u) {
-        const int piece = 2 * t2 + (mtx >> 1);
-        const uint32_t off = row * 128 + (t2 >> 2) * HALFB + (((piece & 7) ^ (row & 7)) << 4);
         uint32_t bv[4];   // V^T: tokens 0-7 | 8-15 x d 0-7 | 8-15 of the 16-wide d tile, transposed on the way out of shared memory
-        ldsm_x4_t(bv, sVs[u] + off);
+        ldsm_x4_t(bv, ((sVs[u] + lane_v) ^ (uint32_t)(((2 * t2) & 7) << 4)) + (t2 >> 2) * HALFB);
 #pragma unroll
         for (int nt = 0; nt < NTN; ++nt) mma16816(oT[nt][t2], bv[0], bv[2], bv[1], bv[3], pb[u][nt][0], pb[u][nt][1]);
       };
@@ -734,7 +732,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
 #pragma unroll
             for (int p = 0; p < KK / 2; ++p) {
               uint32_t bv[4];   // tokens 0-7 | 8-15 x the 16-byte groups 2p | 2p+1 (two d-tiles)
-              ldsm_x4_t(bv, sVs[u] + row * 128 + ((((2 * p + (mtx >> 1)) & 7) ^ (row & 7)) << 4));
+              ldsm_x4_t(bv, (sVs[u] + lane_v) ^ (uint32_t)((2 * p) << 4));
 #pragma unroll
               for (int hk = 0; hk < 2; ++hk) {
                 const uint32_t x0 = __byte_perm(bv[2 * hk], 0, 0x3120), x1 = __byte_perm(bv[2 * hk + 1], 0, 0x3120);
@@ -754,6 +752,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
   };
 
   STAMP(17);
+  const int new_j = a.has_new ? (T_t - 1) / GR : -1;   // the text granule that takes the row of the token being generated
   for (int n = 0; n < n_my && !timed_out;) {
     __syncwarp();
     // up to two granules per step; a granule with nothing visible (an empty slot, text capacity not yet written) is passed over
@@ -780,7 +779,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
           const uint32_t sK = my_base + stage * 2 * TILEB, sV = sK + TILEB;
           // the row of the token being generated: take it from k_new/v_new and store it into the text region
           const int j = first + (n + u) * NW;
-          if (a.has_new && j < G.n_tg && (T_t - 1) / GR == j) {
+          if (j == new_j) {
             const int nr = (T_t - 1) - j * GR;
             if (lane < 2 * PPR) {
               const int kv = lane / PPR, pc = lane - kv * PPR;
