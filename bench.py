@@ -413,7 +413,7 @@ def run_reference(args, rank, world):
     if rank != 0:
         return
     total = args.steps + args.warmup
-    w = make_workload(args.workload, max(total, 1), 0)
+    w = make_workload(args.workload, max(total, 3), 0)   # the probe below runs three steps
     syn = Synth(w, seed=0, device="cpu")
     threads = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
     # bound the run: sample the first Ls layers of sequence 0 so that (K+W) steps stay within about two minutes
@@ -444,10 +444,22 @@ def run_reference(args, rank, world):
               f"{w.n_layers}/{Ls} layers and x{w.batch} sequences")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic", "config": workload_config(w),
+            "dtype": "f64", "data": "synthetic",
+            # the oracle runs the layers of a step one after the other with the default settings of the method
+            "config": method_config(w), "issue": {"launch": "host loops over layers, OpenMP over query heads"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
+
+
+ISSUE_NAMES = {0: "independent", 1: "chained", 2: "serial", 3: "all_layers_together"}
+
+
+def method_config(w, layer_dependency=1, score_scope=0, residency=0, kv_fp8=False):
+    """The `config` of a benchmark line: the workload and the method's settings, the same keys in both arms (how an arm
+    launches its steps is reported outside it)."""
+    return dict(workload_config(w), layer_issue=ISSUE_NAMES[layer_dependency], score_scope="global" if score_scope else "per layer",
+                residency="segment lag" if residency else "hard budget", tidal_kv="fp8_e4m3" if kv_fp8 else "bf16")
 
 
 def workload_config(w):
@@ -898,10 +910,8 @@ def run_ours(args, rank, world, local_rank):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": dict(workload_config(w), launch="eager" if args.eager else "cuda graph replay of the step",
-                       score_scope="global" if args.score_scope else "per layer",
-                       residency="segment lag" if args.residency else "hard budget", layer_issue=dep_names[DEP],
-                       tidal_kv="fp8_e4m3" if Job.kv_fp8 else "bf16"),
+        "config": method_config(w, DEP, args.score_scope, args.residency, Job.kv_fp8),
+        "issue": {"launch": "eager" if args.eager else "cuda graph replay of the step", "layers": dep_names[DEP]},
         "clocks": clocks, "gpu_launches": int(sum(region_launches)),
         "launches": {"attention": region_launches[0], "selection": region_launches[1], "recall": region_launches[2],
                      "step_end": region_launches[3], "layers_per_attention_launch": w.n_layers / attn_per_step},
