@@ -2,15 +2,16 @@
 //
 // One launch per layer serves every KV head of every active sequence:
 //   anchor heads : text + all audio (contiguous store); per 16-token granule the kernel also emits
-//                  sum_tau 2^(s_tau - m) and the running max m, from which the tail kernel rebuilds the
+//                  sum_tau 2^(s_tau - m) and the running max m, from which the selection kernel rebuilds the
 //                  per-chunk softmax mass of Eq. 2 (Method section, "Decode-Step Score Aggregation");
 //   tidal heads  : text + the chunks resident in the slot pool (gather by slot table);
 //   fixed heads  : text + the compacted prefill subset.
-// A CTA takes one work item = a granule range of one (sequence, KV head).  Each of its warps streams its
-// own granules (16 tokens x d, K and V) through a private TMA pipeline (cp.async.bulk.tensor, 128-byte
-// swizzle, one mbarrier per stage, issued by one elected lane) and keeps a private online-softmax state; QK^T and PV run on mma.sync m16n8k16 with the g query
-// heads of the group padded to the 16 rows of the tile (bf16 in, fp32 accumulate).  Warps merge through
-// shared memory and the CTA writes one (m, l, o[g][d]) partial.
+// A CTA takes one work item = a granule range of one (sequence, KV head), or walks a host-assigned list of them.  Each
+// of its warps streams its own granules (16 tokens x d, K and V) through a private TMA pipeline (cp.async.bulk.tensor,
+// 128-byte swizzle, one mbarrier per stage, issued by elected lanes) and keeps a private online-softmax state.  QK^T and PV
+// run on mma.sync m16n8k16 (bf16 in, fp32 accumulate) in transposed form, tokens on the M side of the tile and the group's
+// query heads on N: S^T = K q^T, O^T = V^T P^T, so a group of up to 8 heads fills one n-tile without padding rows.  Warps
+// merge through shared memory and the CTA writes the head's output, or one (m, l, o[g][d]) partial of a split head.
 //
 // The same launch also does the rest of the layer's step, with no further kernel and no host round trip:
 //   - the warp that owns the text granule of the token being generated reads that row from k_new/v_new and
@@ -520,7 +521,7 @@ __device__ __forceinline__ void attn_body(const CacheView &cv, const AttnArgs &a
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
   }
   STAMP(6);
-  // ---- Q fragments (rows >= g are zero padding); loaded after the first K/V copies are in flight ----
+  // ---- Q fragments (the B operand of S^T = K q^T; heads >= g are zero columns); loaded after the first K/V copies are in flight ----
   const int r0 = lane >> 2, cq = (lane & 3) * 2;
   uint32_t qa[KK][NQ];
   {
