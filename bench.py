@@ -908,7 +908,9 @@ def run_ours(args, rank, world, local_rank):
             traffic = None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "ms_per_step": ms_per_step, "step_us": ms_per_step * 1e3,
+        "step_us_median": float(np.median(per_step)) * 1e3, "step_us_p95": float(np.percentile(per_step, 95)) * 1e3,   # this rank's K steps
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": method_config(w, DEP, args.score_scope, args.residency, Job.kv_fp8),
         "issue": {"launch": "eager" if args.eager else "cuda graph replay of the step", "layers": dep_names[DEP]},
