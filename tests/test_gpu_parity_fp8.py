@@ -128,3 +128,31 @@ def test_refused_combinations():
     assert e.value.status == wnw.WNW_ERR_INVALID_ARG
     h = create()
     wnw.wnw_destroy(h)
+
+
+def test_prefill_scores_over_several_text_queries():
+    """The sum over text queries (one scoring pass per query) reads the staged rows every time: they must hold the stored
+    values from the first pass on."""
+    roles = [[A, T, T, F], [T, F, T, T]]
+    w = tiny_custom(n_layers=2, n_q_heads=8, n_kv_heads=4, head_dim=128, n_text=8, audio_lens=(400, 130), chunk=32, budget=0.25,
+                    n_steps=5, roles=roles)
+    w.n_prefill_queries = 4
+    _run(w, seed=8)
+
+
+def test_token_compressed_fixed_heads_beside_an_e4m3_tidal_tier():
+    """wnw_place_prefill_tokens on a cache whose tidal tier is e4m3: fixed heads keep their best positions (bf16, from the
+    plain prefix), tidal heads stay chunk-granular and quantised."""
+    from parity_harness import Lockstep
+    roles = [[A, T, F, F], [T, F, A, T]]
+    w = tiny_custom(n_layers=2, n_q_heads=8, n_kv_heads=4, head_dim=128, n_text=6, audio_lens=(500, 210), chunk=50, budget=0.3,
+                    n_steps=6, roles=roles)
+    ret = np.array([[1.0, 1.0, 0.25, 0.1], [1.0, 0.2, 1.0, 1.0]], np.float32)   # a head's store holds floor(0.3 * C) blocks of 50
+    ls = Lockstep(w, seed=12, kv_fp8=True, token_retention=ret, token_seg=25)
+    try:
+        ls.prefill()
+        for t in range(6):
+            ls.decode_step(t, graph=(t % 2 == 1), check_slots=True)
+        ls.check_stats()
+    finally:
+        ls.close()
