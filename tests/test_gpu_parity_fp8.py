@@ -156,3 +156,13 @@ def test_token_compressed_fixed_heads_beside_an_e4m3_tidal_tier():
         ls.check_stats()
     finally:
         ls.close()
+
+
+def test_degenerate_sequences():
+    """A sequence without audio beside one with a single short chunk, budget 1.0 (every chunk resident, nothing recalled),
+    fewer chunks than k."""
+    roles = [[A, T], [T, F]]
+    w = tiny_custom(n_layers=2, n_q_heads=4, n_kv_heads=2, head_dim=128, n_text=12, audio_lens=(0, 9, 40), chunk=16, budget=1.0,
+                    n_steps=4, roles=roles)
+    ls = _run(w, seed=6)
+    assert ls.near_ties == 0
