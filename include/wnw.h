@@ -106,8 +106,10 @@ enum { WNW_RECALL_SIDE_STREAM = 0, WNW_RECALL_INLINE = 1, WNW_RECALL_SKIP = 2 };
  *             (0 for an all-zero block); elements are x / 2^e rounded to nearest, ties to even.  Host-link bytes per
  *             recalled chunk and the HBM bytes tidal heads read both halve.  The stored value of an element, e4m3 * 2^e,
  *             is an exact bf16 number, and EVERYTHING the library computes for a tidal head (prefill scores included)
- *             uses stored values, so results equal those of a BF16 cache given the stored values as input.  Text rows,
- *             anchor heads and fixed heads stay bf16.  Needs head_dim 128, a residency other than SEGMENT_LAG_TOKEN_BASE
+ *             uses stored values, so results agree, within the tolerances stated for outputs and scores, with those of a
+ *             BF16 cache given the stored values as input (the two products with an e4m3 block take the query and the
+ *             softmax weights as fp16: exact for query elements inside fp16's normal range; |q| > 65504 is not supported
+ *             with this format).  Text rows, anchor heads and fixed heads stay bf16.  Needs head_dim 128, a residency other than SEGMENT_LAG_TOKEN_BASE
  *             and streaming_audio = 0 (a growing chunk would have to be re-scaled): WNW_ERR_UNSUPPORTED otherwise.
  *             wnw_get_slot_kv returns the stored values as bf16. */
 enum { WNW_TIDAL_KV_BF16 = 0, WNW_TIDAL_KV_FP8_E4M3 = 1 };
