@@ -712,7 +712,10 @@ static void build_layer_items(const wnw_cache *c, int layer, int mode, const std
   // cover one another's instead.  Measured on 12 layers x 16 sequences x 7500 tokens with copies skipped: 0.365 -> 0.340 ms
   // per step.  Launches with more heads than SMs keep the packed one-shot CTAs (batch-32 ragged: 1.06 against 1.12 ms), and
   // so does the full-cache kernel (0.878 against 0.895 ms).
-  const bool big_single_wave = overlapped && !batched && mode == ATTN_DECODE && total >= 64ll * c->n_sm;   // decided once the cut is known
+  // (What marks such a launch is about as many heads as SMs, not its size: with 64 heads of 7500 tokens the one-shot CTAs
+  // win, 0.70 against 0.58 of the copy bandwidth; with 128 heads of 3000 tokens the persistent ones, 0.62 against 0.55.)
+  const bool big_single_wave = overlapped && !batched && mode == ATTN_DECODE && total >= 32ll * c->n_sm &&
+                               4 * (long long)seq_ids.size() * G.Hkv >= 3ll * c->n_sm;   // decided once the cut is known
   lw.throughput = throughput;
   lw.first_item = (int)items.size();
   lw.head_items_off = (int)heads.size();
