@@ -74,3 +74,38 @@ def test_dequantised_rows_touch_only_tidal_audio_and_stay_close():
     # idempotent: stored values are on the grid of their own scale
     kq2, vq2 = dequantised_tidal_bits(kq, vq, roles, ab, ae, chunk)
     assert np.array_equal(kq2, kq) and np.array_equal(vq2, vq)
+
+
+def test_what_the_format_costs_on_the_small_configuration():
+    """Two oracles on config 0, one fed the plain prefix and one the values an e4m3 tidal tier stores: decode selections
+    are the same (they come from anchor heads, which stay bf16) and outputs move by what three mantissa bits of V allow
+    (values of O(1): well under 0.3).  A record of the format's cost, not a parity bar."""
+    from helpers import make_oracle
+    from workloads import Synth, config0
+    from workloads.synth import bf16_bits
+    w = config0()
+    syn = Synth(w, seed=0)
+    plain, stored = make_oracle(w), make_oracle(w)
+    try:
+        for l in range(w.n_layers):
+            p = syn.prefill(0, l)
+            kb, vb, qb = bf16_bits(p["k"]), bf16_bits(p["v"]), bf16_bits(p["q_last"])
+            plain.place_prefill(0, l, kb, vb, p["audio_begin"], p["audio_end"], qb)
+            kq, vq = dequantised_tidal_bits(kb, vb, w.roles[l], p["audio_begin"], p["audio_end"], w.chunk)
+            stored.place_prefill(0, l, kq, vq, p["audio_begin"], p["audio_end"], qb)
+        dec = {l: syn.decode(0, l) for l in range(w.n_layers)}
+        worst = 0.0
+        for t in range(w.n_steps):
+            outs = []
+            for o in (plain, stored):
+                o.step_begin([0])
+                outs.append([o.decode_layer(l, bf16_bits(dec[l]["q"][t])[None], bf16_bits(dec[l]["k_new"][t])[None],
+                                            bf16_bits(dec[l]["v_new"][t])[None]) for l in range(w.n_layers)])
+                o.step_end()
+            for l in range(w.n_layers):
+                worst = max(worst, float(np.abs(outs[0][l] - outs[1][l]).max()))
+                if (w.roles[l] == ROLE_TIDAL).any():
+                    assert plain.selected(0, l).tolist() == stored.selected(0, l).tolist()
+        assert 0.0 < worst < 0.3
+    finally:
+        plain.close(); stored.close()
